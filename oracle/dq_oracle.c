@@ -83,12 +83,10 @@ uint32_t dqo_u16(uint64_t seed, uint32_t round, uint32_t worker, uint32_t stream
     return (i & 1) ? (w >> 16) : (w & 0xFFFFu);
 }
 
-/* 15 uniform bits for coordinate i: bits [0,15) of the word for even i,
- * bits [17,32) for odd i. */
+/* 15 uniform bits for coordinate i: the top 15 of its 16-bit draw. */
 uint32_t dqo_u15(uint64_t seed, uint32_t round, uint32_t worker, uint32_t stream, uint64_t i)
 {
-    uint32_t w = word_of(seed, round, worker, stream, i);
-    return (i & 1) ? (w >> 17) : (w & 0x7FFFu);
+    return dqo_u16(seed, round, worker, stream, i) >> 1;
 }
 
 /* ------------------------------------------------------------------------ */
