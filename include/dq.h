@@ -1,0 +1,192 @@
+/*
+ * dq.h -- C ABI of libdq: one round of double quantization on one NVIDIA B200 (sm_100a).
+ *
+ * Method: "Double Quantization for Communication-Efficient Distributed Optimization"
+ * (AsyLPG = Algorithm 1, Sparse-AsyLPG = Algorithm 2, Acc-AsyLPG = Algorithm 3).  The problem is
+ * eq. (1): min_{x in Omega} f(x) + h(x), f = (1/n) sum_i f_i.  Here f_i is the logistic loss
+ * log(1 + exp(-y_i <a_i, x>)) with labels y_i = +-1, h = lambda1 |x|_1 + (lambda2/2) |x|^2, and Omega is
+ * the box [box_lo, box_hi]^d.  M workers are simulated as independent lanes of one GPU; a "round" is one
+ * inner iteration (Algorithm 1 steps 6-13) in which all M workers answer the same broadcast model and the
+ * master averages their messages before one prox step.
+ *
+ * General rules
+ *   - Every function returns a DQ_* status and never throws, exits or allocates behind the caller's back
+ *     except dq_create (which allocates the context's scratch) and dq_destroy (which frees it).
+ *   - Unless a parameter is marked HOST, pointers are DEVICE pointers owned by the caller; they must stay
+ *     valid until the stream work that uses them has finished.  Vectors are contiguous fp32.
+ *   - Work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t cast to void*; NULL is the
+ *     default stream).  No call synchronises the device unless it says so.
+ *   - Errors found on the host (bad argument, bad bit width, misaligned buffer) are returned immediately.
+ *     Errors found by a kernel (non-finite norm, sparse message over capacity) set a sticky status word that
+ *     dq_poll_status reads.
+ *   - Bit widths b, b_x must be 2, 4 or 8 (b = 1 would give 2^(b-1)-1 = 0 levels).
+ *   - All random draws come from Philox4x32-10 with key = seed and counter
+ *     (coordinate >> 3, round, worker, stream); the master's worker id is 0xFFFFFFFF; streams are
+ *     0 model rounding, 1 gradient rounding, 2 sparsification mask, 3 minibatch sampling.  Equal
+ *     (seed, round, inputs) give equal bytes.
+ *
+ * Packed code layout (message of Section 3.1: 32 bits for delta plus b bits per coordinate): codes are b-bit
+ * two's complement; coordinate j of a message sits in byte j / (8/b) at bit offset (j mod (8/b)) * b.  The
+ * bytes of one message are padded with zeros to dq_packed_bytes(d, b), a multiple of 16.  delta is kept in a
+ * separate fp32 array.
+ */
+#ifndef DQ_H_
+#define DQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    DQ_OK = 0,
+    DQ_ERR_ARG = 1,        /* NULL pointer, non-positive size, misaligned buffer                     */
+    DQ_ERR_SHAPE = 2,      /* sizes inconsistent with the context (d, M, stride, capacity)            */
+    DQ_ERR_BITS = 3,       /* bit width not in {2, 4, 8}                                              */
+    DQ_ERR_NONFINITE = 4,  /* a vector to be quantised holds NaN or Inf                               */
+    DQ_ERR_CAPACITY = 5,   /* a sparse message had more survivors than the buffers can hold           */
+    DQ_ERR_CUDA = 6,       /* a CUDA runtime call failed                                              */
+    DQ_ERR_TIMEOUT = 7     /* reserved                                                                */
+};
+
+enum { DQ_DENSE_F32 = 0, DQ_CSR_F32 = 1, DQ_DENSE_BF16 = 2 };   /* dq_data.format */
+enum { DQ_MSG_DENSE = 0, DQ_MSG_SPARSE = 1 };                   /* dq_config.msg_format */
+
+/* The training set {a_i, y_i} of eq. (1).  values: DENSE_F32 [n][d] float; DENSE_BF16 [n][d] bfloat16;
+ * CSR_F32 [nnz] float with col_idx [nnz] (ascending inside a row, < d) and row_ptr [n+1].  labels [n] = +-1.
+ * All device pointers, read-only, 16-byte aligned. */
+typedef struct {
+    int32_t format; int32_t reserved;
+    int64_t n, d;
+    const void* values;
+    const int32_t* col_idx;
+    const int64_t* row_ptr;
+    const float* labels;
+} dq_data;
+
+/* Inputs of Algorithms 1-3 that stay fixed during a run. */
+typedef struct {
+    int64_t d;                 /* model size                                                            */
+    int32_t M, B;              /* simulated workers; minibatch rows per worker and round                */
+    int32_t bx, b;             /* bits for the model (step 8) and for the gradient (step 12)            */
+    float lambda1, lambda2;    /* h = lambda1 |x|_1 + (lambda2/2) |x|^2                                  */
+    float box_lo, box_hi;      /* Omega = [box_lo, box_hi]^d; -INFINITY/+INFINITY for no constraint      */
+    int32_t sparsify;          /* 1: Algorithm 2 (eq. (4) before quantising)                            */
+    float phi;                 /* sparsity budget sum p_i; <= 0 or too large: |alpha|_1/|alpha|_inf (Lemma 2) */
+    int32_t msg_format;        /* DQ_MSG_SPARSE needs sparsify = 1                                      */
+    int32_t accelerated;       /* 1: Algorithm 3                                                        */
+    int32_t snapshot_flag;     /* 1: send one flag bit instead of the model when x equals the snapshot  */
+    int32_t reserved;
+    uint64_t seed;
+    int64_t sparse_cap;        /* entries per worker in the context's own sparse message buffers; 0: d   */
+} dq_config;
+
+/* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3
+ * only (may be NULL otherwise).  norm_x is one device float holding ||x||_inf, maintained by the library.
+ * z_snap [n] caches the margins <a_i, x_snap> (written at epoch begin). */
+typedef struct {
+    float* x; float* x_snap; float* g_full; float* y; float* x_sum;
+    float* norm_x; float* z_snap;
+} dq_state;
+
+/* M worker messages.  Dense: codes [M][stride] bytes (stride >= dq_packed_bytes(d, b), multiple of 16) and
+ * scale [M] (= delta).  Sparse (Section 4.2's encoding: position then value per nonzero of beta): nnz [M],
+ * idx [M][cap] ascending coordinate indices, and the value codes packed b bits each in list order in
+ * codes [M][stride] (stride >= dq_packed_bytes(cap, b)). */
+typedef struct {
+    uint8_t* codes; int64_t stride; float* scale;
+    uint32_t* idx; int64_t cap; uint32_t* nnz;
+} dq_msgs;
+
+typedef struct dq_ctx dq_ctx;
+
+/* Bytes of one packed message of `count` codes of b bits, padded to a multiple of 16. */
+int64_t dq_packed_bytes(int64_t count, int b);
+
+/* Create a context for `cfg` on the current device.  `data` may be NULL when only the codec entry points
+ * (dq_quantize_model, dq_quantize_sparsify_pack, dq_master_unpack_aggregate_prox, dq_codec_round,
+ * dq_unpack) will be used.  Allocates the context's scratch (norms, message buffers for dq_round,
+ * survivor staging); the structs are copied, the arrays they point to are not. */
+int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data);
+int dq_destroy(dq_ctx* ctx);
+
+/* Epoch boundary (Algorithm 1 steps 3-5 and 14; Algorithm 3 steps 3-5 and 15).
+ * Algorithms 1/2: x_snap <- x.  Algorithm 3: if rounds have run since the last call, x_snap <- x_sum / m
+ * (m = number of those rounds) and x_sum <- 0; y is carried over; x <- x_snap + theta (y - x_snap).
+ * Then g_full <- grad f(x_snap) in full precision over all n rows, z_snap <- margins, norm_x <- ||x||_inf. */
+int dq_epoch_begin(dq_ctx* ctx, dq_state* st, float theta, void* stream);
+
+/* Master step 8: delta_x = ||x||_inf / (2^(bx-1)-1); codes_x <- packed Q_(delta_x,bx)(x) (Section 3.1).
+ * norm_x: device float holding ||x||_inf, or NULL to have it computed.  codes_x must hold
+ * dq_packed_bytes(d, bx) bytes; delta_x is one device float. */
+int dq_quantize_model(dq_ctx* ctx, const float* x, const float* norm_x, uint32_t round,
+                      uint8_t* codes_x, float* delta_x, void* stream);
+
+/* Worker step 11 for all M workers: alpha_w = (1/B) sum_{a in batch_w} [grad f_a(xhat) - grad f_a(x_snap)],
+ * xhat = dequantised broadcast model (code * delta_x), or x_snap itself when is_snapshot != 0 (flag bit of
+ * the "Model Parameter Quantization" paragraph; codes_x/delta_x are then ignored).  batch_idx: [M][B] row
+ * indices (int32) or NULL to draw them from the batch stream (worker w samples its own contiguous
+ * partition of the rows, with replacement).  Outputs alpha [M][d], norm_inf [M] = ||alpha_w||_inf. */
+int dq_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot,
+                   const dq_state* st, uint32_t round, const int32_t* batch_idx,
+                   float* alpha, float* norm_inf, void* stream);
+
+/* Worker steps 12(-13) for all M workers: optional sparsification by eq. (4) with Lemma 2's probabilities,
+ * then delta = ||.||_inf / (2^(b-1)-1), Q_(delta,b), and bit packing into `out`.
+ * v [M][d]; norm_inf [M] = ||v_w||_inf as produced by dq_worker_grad, or NULL to have it computed. */
+int dq_quantize_sparsify_pack(dq_ctx* ctx, const float* v, const float* norm_inf, uint32_t round,
+                              dq_msgs* out, void* stream);
+
+/* Master step 9: g = (1/M) sum_w dequantised message w; u = g + g_full;
+ * Algorithms 1/2: x <- prox_{eta h}(x - eta u).
+ * Algorithm 3:    y <- prox_{eta h}(y - eta u); x <- x_snap + theta (y - x_snap); x_sum <- x_sum + x.
+ * Also writes ||x||_inf of the new model to st->norm_x. */
+int dq_master_unpack_aggregate_prox(dq_ctx* ctx, const dq_msgs* msgs, dq_state* st, float eta, float theta,
+                                    void* stream);
+
+/* One whole round on the context's own message buffers: model quantisation, M worker gradients,
+ * (sparsify,) quantise, pack, master step, bit accounting.  bits_down / bits_up (device uint64, may be
+ * NULL) receive the transmitted bits of this round by the paper's message sizes: down = M (32 + bx d), or M
+ * flag bits on a snapshot round; up = sum_w (32 + b d) dense, sum_w (32 + nnz_w (ceil(log2 d) + b)) sparse.
+ * The round is a snapshot round when snapshot_flag is set and it is the first round after dq_epoch_begin
+ * (Algorithm 3: of the first epoch only). */
+int dq_round(dq_ctx* ctx, dq_state* st, uint32_t round, float eta, float theta,
+             uint64_t* bits_down, uint64_t* bits_up, void* stream);
+
+/* The round without its gradient stage, for callers that bring their own M gradient vectors v [M][d]:
+ * quantise(+sparsify)+pack into the context's buffers, master step on `st`, then model quantisation of the
+ * new x into codes_x / delta_x. */
+int dq_codec_round(dq_ctx* ctx, const float* v, dq_state* st, uint32_t round, float eta, float theta,
+                   uint8_t* codes_x, float* delta_x, void* stream);
+
+/* Same as dq_codec_round with HOST buffers: copies v [M][d] to the device, runs the round on the context's
+ * device-resident state (set by dq_codec_host_setup), copies codes_x (dq_packed_bytes(d, bx) bytes) and
+ * delta_x back, and synchronises the stream.  Host buffers should be pinned for full copy speed. */
+int dq_codec_host_setup(dq_ctx* ctx, const float* x_host, const float* g_full_host);
+int dq_codec_round_host(dq_ctx* ctx, const float* v_host, uint32_t round, float eta,
+                        uint8_t* codes_x_host, float* delta_x_host, void* stream);
+
+/* Test utility: dequantise message w of `msgs` into out [d] (zeros where a sparse message has no entry). */
+int dq_unpack(dq_ctx* ctx, const dq_msgs* msgs, int w, float* out, void* stream);
+
+/* Diagnostic: P(x) = f(x) + h(x) of eq. (1) over all n rows into one device double. */
+int dq_objective(dq_ctx* ctx, const float* x, double* P, void* stream);
+
+/* The context's own message buffers and last-round intermediates (device pointers, valid until
+ * dq_destroy), for inspection after dq_round: alpha [M][d], norm_inf [M], batch rows [M][B]. */
+int dq_round_buffers(dq_ctx* ctx, dq_msgs* msgs, const float** alpha, const float** norm_inf,
+                     const int32_t** batch_idx, const uint8_t** codes_x, const float** delta_x);
+
+/* Synchronises `stream`, returns the sticky device status through *status (HOST) and clears it. */
+int dq_poll_status(dq_ctx* ctx, int* status, void* stream);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t dq_launch_count(const dq_ctx* ctx);
+
+const char* dq_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DQ_H_ */

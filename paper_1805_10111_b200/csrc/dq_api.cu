@@ -1,0 +1,320 @@
+// C ABI of libdq (see include/dq.h): argument checks, scratch ownership and the order of kernel launches.
+#include <math.h>
+#include <new>
+
+#include "dq_kernels.cuh"
+
+using namespace dq;
+
+namespace {
+
+bool bits_ok(int b) { return b == 2 || b == 4 || b == 8; }
+bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
+
+template <class T>
+int dev_alloc(T** p, size_t count)
+{
+    *p = nullptr;
+    if (count == 0) count = 1;
+    return cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T)) == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+}
+
+int last_error() { return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA; }
+
+bool sparse_messages(const dq_ctx* ctx) { return ctx->cfg.sparsify && ctx->cfg.msg_format == DQ_MSG_SPARSE; }
+
+int check_msgs(const dq_ctx* ctx, const dq_msgs* m)
+{
+    if (!m || !m->codes || !m->scale) return DQ_ERR_ARG;
+    if (!aligned(m->codes, 16) || (m->stride & 15)) return DQ_ERR_ARG;
+    if (sparse_messages(ctx)) {
+        if (!m->idx || !m->nnz || m->cap < 1) return DQ_ERR_ARG;
+        if (m->stride < dq_packed_bytes(m->cap, ctx->cfg.b)) return DQ_ERR_SHAPE;
+    } else if (m->stride < dq_packed_bytes(ctx->cfg.d, ctx->cfg.b)) {
+        return DQ_ERR_SHAPE;
+    }
+    return DQ_OK;
+}
+
+int check_state(const dq_ctx* ctx, const dq_state* s)
+{
+    if (!s || !s->x || !s->g_full || !s->norm_x) return DQ_ERR_ARG;
+    if (!aligned(s->x, 16) || !aligned(s->g_full, 16)) return DQ_ERR_ARG;
+    if (ctx->cfg.accelerated) {
+        if (!s->y || !s->x_sum || !s->x_snap) return DQ_ERR_ARG;
+        if (!aligned(s->y, 16) || !aligned(s->x_sum, 16) || !aligned(s->x_snap, 16)) return DQ_ERR_ARG;
+    }
+    return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int64_t dq_packed_bytes(int64_t count, int b)
+{
+    const int64_t bytes = (count * b + 7) / 8;
+    return (bytes + 15) / 16 * 16;
+}
+
+const char* dq_strerror(int status)
+{
+    switch (status) {
+        case DQ_OK: return "ok";
+        case DQ_ERR_ARG: return "bad argument (null, non-positive or misaligned)";
+        case DQ_ERR_SHAPE: return "sizes inconsistent with the context";
+        case DQ_ERR_BITS: return "bit width must be 2, 4 or 8";
+        case DQ_ERR_NONFINITE: return "vector to quantise holds NaN or Inf";
+        case DQ_ERR_CAPACITY: return "sparse message exceeds its capacity";
+        case DQ_ERR_CUDA: return "CUDA runtime error";
+        case DQ_ERR_TIMEOUT: return "timeout";
+        default: return "unknown status";
+    }
+}
+
+int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
+{
+    if (!out || !cfg) return DQ_ERR_ARG;
+    *out = nullptr;
+    if (cfg->d < 1 || cfg->d > ((int64_t)1 << 32) || cfg->M < 1 || cfg->M > 4096 || cfg->B < 1) return DQ_ERR_ARG;
+    if (!bits_ok(cfg->b) || !bits_ok(cfg->bx)) return DQ_ERR_BITS;
+    if (cfg->msg_format == DQ_MSG_SPARSE && !cfg->sparsify) return DQ_ERR_ARG;
+    if (cfg->msg_format != DQ_MSG_SPARSE && cfg->msg_format != DQ_MSG_DENSE) return DQ_ERR_ARG;
+    if (!(cfg->box_lo <= cfg->box_hi) || cfg->lambda1 < 0 || cfg->lambda2 < 0) return DQ_ERR_ARG;
+    if (cfg->sparse_cap < 0 || cfg->sparse_cap > cfg->d) return DQ_ERR_ARG;
+    if (data) {
+        if (data->n < 1 || data->d != cfg->d || !data->values || !data->labels) return DQ_ERR_SHAPE;
+        if (data->format == DQ_CSR_F32 && (!data->col_idx || !data->row_ptr)) return DQ_ERR_ARG;
+        if (data->format < DQ_DENSE_F32 || data->format > DQ_DENSE_BF16) return DQ_ERR_ARG;
+        if (!aligned(data->values, 16)) return DQ_ERR_ARG;
+        if (data->n < cfg->M) return DQ_ERR_SHAPE;
+    }
+    dq_ctx* c = new (std::nothrow) dq_ctx();
+    if (!c) return DQ_ERR_CUDA;
+    c->cfg = *cfg;
+    c->has_data = data != nullptr;
+    if (data) c->data = *data;
+    c->keys = expand_keys(cfg->seed);
+    int dev = 0; cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { delete c; return DQ_ERR_CUDA; }
+    c->sm_count = prop.multiProcessorCount;
+    const int64_t d = cfg->d; const int M = cfg->M;
+    c->nchunks = (d + kChunk - 1) / kChunk;
+    const bool sparse = cfg->sparsify && cfg->msg_format == DQ_MSG_SPARSE;
+    int rc = DQ_OK;
+    rc |= dev_alloc(&c->norm_bits, M);
+    rc |= dev_alloc(&c->beta_norm_bits, M);
+    rc |= dev_alloc(&c->l1_sum, M);
+    rc |= dev_alloc(&c->chunk_off, cfg->sparsify ? (size_t)M * (c->nchunks + 1) : 1);
+    rc |= dev_alloc(&c->tile_ptr, sparse ? (size_t)M * (c->nchunks + 1) : 1);
+    rc |= dev_alloc(&c->xnorm_bits, 1);
+    rc |= dev_alloc(&c->status, 1);
+    rc |= dev_alloc(&c->bits, 2);
+    // message buffers of dq_round / dq_codec_round
+    c->msgs.cap = sparse ? (cfg->sparse_cap > 0 ? cfg->sparse_cap : d) : 0;
+    c->msgs.stride = sparse ? dq_packed_bytes(c->msgs.cap, cfg->b) : dq_packed_bytes(d, cfg->b);
+    rc |= dev_alloc(&c->msgs.codes, (size_t)c->msgs.stride * M);
+    rc |= dev_alloc(&c->msgs.scale, M);
+    rc |= dev_alloc(&c->msgs.idx, sparse ? (size_t)c->msgs.cap * M : 1);
+    rc |= dev_alloc(&c->msgs.nnz, M);
+    rc |= dev_alloc(&c->codes_x, (size_t)dq_packed_bytes(d, cfg->bx));
+    rc |= dev_alloc(&c->delta_x, 1);
+    rc |= dev_alloc(&c->ninf, M);
+    if (data) {
+        rc |= dev_alloc(&c->alpha, (size_t)M * d);
+        rc |= dev_alloc(&c->rows, (size_t)M * cfg->B);
+        rc |= dev_alloc(&c->xhat_diff, (size_t)d);
+        rc |= dev_alloc(&c->g64, (size_t)d);
+    }
+    if (rc == DQ_OK && cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess) rc = DQ_ERR_CUDA;
+    if (rc != DQ_OK) { dq_destroy(c); cudaGetLastError(); return DQ_ERR_CUDA; }
+    c->epoch = -1;
+    *out = c;
+    return DQ_OK;
+}
+
+int dq_destroy(dq_ctx* c)
+{
+    if (!c) return DQ_ERR_ARG;
+    void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->xnorm_bits, c->status, c->bits,
+                    c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
+                    c->rows, c->xhat_diff, c->g64, c->hx, c->hg, c->hv, c->hnorm};
+    for (void* p : ptrs) if (p) cudaFree(p);
+    delete c;
+    return DQ_OK;
+}
+
+int dq_quantize_model(dq_ctx* ctx, const float* x, const float* norm_x, uint32_t round, uint8_t* codes_x, float* delta_x,
+                      void* stream)
+{
+    if (!ctx || !x || !codes_x || !delta_x) return DQ_ERR_ARG;
+    if (!aligned(codes_x, 16) || !aligned(x, 4)) return DQ_ERR_ARG;
+    cudaStream_t st = as_stream(stream);
+    const uint32_t* nb = reinterpret_cast<const uint32_t*>(norm_x);
+    if (!nb) { launch_norm_inf(ctx, x, ctx->cfg.d, 1, ctx->xnorm_bits, st); nb = ctx->xnorm_bits; }
+    launch_quantize_pack(ctx, x, ctx->cfg.d, 1, ctx->cfg.bx, nb, codes_x, dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx), delta_x,
+                         round, kMaster, kStreamModel, st);
+    return last_error();
+}
+
+int dq_quantize_sparsify_pack(dq_ctx* ctx, const float* v, const float* norm_inf, uint32_t round, dq_msgs* out, void* stream)
+{
+    if (!ctx || !v) return DQ_ERR_ARG;
+    if (!aligned(v, 4)) return DQ_ERR_ARG;
+    int rc = check_msgs(ctx, out);
+    if (rc != DQ_OK) return rc;
+    cudaStream_t st = as_stream(stream);
+    const dq_config& c = ctx->cfg;
+    const uint32_t* nb = reinterpret_cast<const uint32_t*>(norm_inf);
+    if (!nb) { launch_norm_inf(ctx, v, c.d, c.M, ctx->norm_bits, st); nb = ctx->norm_bits; }
+    if (!c.sparsify)
+        launch_quantize_pack(ctx, v, c.d, c.M, c.b, nb, out->codes, out->stride, out->scale, round, 0u, kStreamGrad, st);
+    else
+        launch_sparsify_pack(ctx, v, c.d, c.M, c.b, nb, round, out, sparse_messages(ctx), st);
+    return last_error();
+}
+
+int dq_master_unpack_aggregate_prox(dq_ctx* ctx, const dq_msgs* msgs, dq_state* s, float eta, float theta, void* stream)
+{
+    if (!ctx) return DQ_ERR_ARG;
+    int rc = check_msgs(ctx, msgs);
+    if (rc == DQ_OK) rc = check_state(ctx, s);
+    if (rc != DQ_OK) return rc;
+    if (!(eta > 0.0f) || !isfinite(eta)) return DQ_ERR_ARG;
+    launch_master(ctx, msgs, sparse_messages(ctx), s, eta, theta, as_stream(stream));
+    return last_error();
+}
+
+int dq_unpack(dq_ctx* ctx, const dq_msgs* msgs, int w, float* out, void* stream)
+{
+    if (!ctx || !out) return DQ_ERR_ARG;
+    int rc = check_msgs(ctx, msgs);
+    if (rc != DQ_OK) return rc;
+    if (w < 0 || w >= ctx->cfg.M) return DQ_ERR_SHAPE;
+    launch_unpack(ctx, msgs, sparse_messages(ctx), w, out, as_stream(stream));
+    return last_error();
+}
+
+int dq_codec_round(dq_ctx* ctx, const float* v, dq_state* s, uint32_t round, float eta, float theta, uint8_t* codes_x,
+                   float* delta_x, void* stream)
+{
+    if (!ctx || !v || !codes_x || !delta_x) return DQ_ERR_ARG;
+    int rc = check_state(ctx, s);
+    if (rc != DQ_OK) return rc;
+    rc = dq_quantize_sparsify_pack(ctx, v, nullptr, round, &ctx->msgs, stream);
+    if (rc == DQ_OK) rc = dq_master_unpack_aggregate_prox(ctx, &ctx->msgs, s, eta, theta, stream);
+    if (rc == DQ_OK) rc = dq_quantize_model(ctx, s->x, s->norm_x, round, codes_x, delta_x, stream);
+    return rc;
+}
+
+int dq_codec_host_setup(dq_ctx* ctx, const float* x_host, const float* g_full_host)
+{
+    if (!ctx || !x_host || !g_full_host || ctx->cfg.accelerated) return DQ_ERR_ARG;
+    const size_t d = (size_t)ctx->cfg.d;
+    int rc = DQ_OK;
+    if (!ctx->hx) {
+        rc |= dev_alloc(&ctx->hx, d); rc |= dev_alloc(&ctx->hg, d); rc |= dev_alloc(&ctx->hnorm, 1);
+        rc |= dev_alloc(&ctx->hv, d * ctx->cfg.M);
+    }
+    if (rc != DQ_OK) return DQ_ERR_CUDA;
+    if (cudaMemcpy(ctx->hx, x_host, d * 4, cudaMemcpyHostToDevice) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpy(ctx->hg, g_full_host, d * 4, cudaMemcpyHostToDevice) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int dq_codec_round_host(dq_ctx* ctx, const float* v_host, uint32_t round, float eta, uint8_t* codes_x_host, float* delta_x_host,
+                        void* stream)
+{
+    if (!ctx || !ctx->hx || !v_host || !codes_x_host || !delta_x_host) return DQ_ERR_ARG;
+    cudaStream_t st = as_stream(stream);
+    const size_t d = (size_t)ctx->cfg.d;
+    if (cudaMemcpyAsync(ctx->hv, v_host, d * ctx->cfg.M * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return DQ_ERR_CUDA;
+    dq_state s = {ctx->hx, nullptr, ctx->hg, nullptr, nullptr, ctx->hnorm, nullptr};
+    int rc = dq_codec_round(ctx, ctx->hv, &s, round, eta, 0.0f, ctx->codes_x, ctx->delta_x, stream);
+    if (rc != DQ_OK) return rc;
+    if (cudaMemcpyAsync(codes_x_host, ctx->codes_x, (size_t)dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaMemcpyAsync(delta_x_host, ctx->delta_x, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+}
+
+int dq_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, void* stream)
+{
+    if (!ctx || !ctx->has_data) return DQ_ERR_ARG;
+    int rc = check_state(ctx, s);
+    if (rc != DQ_OK) return rc;
+    if (!s->x_snap || !s->z_snap || !aligned(s->x_snap, 16)) return DQ_ERR_ARG;
+    launch_epoch_begin(ctx, s, theta, as_stream(stream));
+    ctx->rounds_in_epoch = 0;
+    ctx->epoch += 1;
+    return last_error();
+}
+
+int dq_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot, const dq_state* s,
+                   uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, void* stream)
+{
+    if (!ctx || !ctx->has_data || !s || !s->x_snap || !s->z_snap || !alpha || !norm_inf) return DQ_ERR_ARG;
+    if (!is_snapshot && (!codes_x || !delta_x)) return DQ_ERR_ARG;
+    if (!aligned(alpha, 16) || (codes_x && !aligned(codes_x, 16))) return DQ_ERR_ARG;
+    launch_worker_grad(ctx, codes_x, delta_x, is_snapshot, s, round, batch_idx, alpha, norm_inf, as_stream(stream));
+    return last_error();
+}
+
+int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, uint64_t* bits_down, uint64_t* bits_up,
+             void* stream)
+{
+    if (!ctx || !ctx->has_data) return DQ_ERR_ARG;
+    int rc = check_state(ctx, s);
+    if (rc != DQ_OK) return rc;
+    if (!s->x_snap || !s->z_snap) return DQ_ERR_ARG;
+    if (ctx->epoch < 0) return DQ_ERR_ARG;                     // dq_epoch_begin has not run
+    const dq_config& c = ctx->cfg;
+    const int flag = c.snapshot_flag && ctx->rounds_in_epoch == 0 && (!c.accelerated || ctx->epoch == 0);
+    if (!flag) {
+        rc = dq_quantize_model(ctx, s->x, s->norm_x, round, ctx->codes_x, ctx->delta_x, stream);
+        if (rc != DQ_OK) return rc;
+    }
+    rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, stream);
+    if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, stream);
+    if (rc == DQ_OK) rc = dq_master_unpack_aggregate_prox(ctx, &ctx->msgs, s, eta, theta, stream);
+    if (rc != DQ_OK) return rc;
+    if (bits_down || bits_up)
+        launch_bits(ctx, flag, sparse_messages(ctx), ctx->msgs.nnz, bits_down ? bits_down : ctx->bits,
+                    bits_up ? bits_up : ctx->bits + 1, as_stream(stream));
+    ctx->rounds_in_epoch += 1;
+    return last_error();
+}
+
+int dq_objective(dq_ctx* ctx, const float* x, double* P, void* stream)
+{
+    if (!ctx || !ctx->has_data || !x || !P) return DQ_ERR_ARG;
+    launch_objective(ctx, x, P, as_stream(stream));
+    return last_error();
+}
+
+int dq_round_buffers(dq_ctx* ctx, dq_msgs* msgs, const float** alpha, const float** norm_inf, const int32_t** batch_idx,
+                     const uint8_t** codes_x, const float** delta_x)
+{
+    if (!ctx) return DQ_ERR_ARG;
+    if (msgs) *msgs = ctx->msgs;
+    if (alpha) *alpha = ctx->alpha;
+    if (norm_inf) *norm_inf = ctx->ninf;
+    if (batch_idx) *batch_idx = ctx->rows;
+    if (codes_x) *codes_x = ctx->codes_x;
+    if (delta_x) *delta_x = ctx->delta_x;
+    return DQ_OK;
+}
+
+int dq_poll_status(dq_ctx* ctx, int* status, void* stream)
+{
+    if (!ctx || !status) return DQ_ERR_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(status, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return DQ_ERR_CUDA;
+    if (*status != 0 && cudaMemsetAsync(ctx->status, 0, sizeof(int), st) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int64_t dq_launch_count(const dq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,598 @@
+// Streaming codec kernels: infinity norm, Q_(delta,b) + bit packing (Section 3.1; Algorithm 1 steps 8
+// and 12), sparsification (eq. (4), Lemma 2; Algorithm 2 steps 12-13), and the master's unpack +
+// aggregate + prox step (Algorithm 1 step 9, Algorithm 3 step 9).  All are bandwidth kernels: 256-bit
+// coalesced loads, one Philox call per eight coordinates, codes packed in registers.
+#include "dq_common.cuh"
+#include "dq_kernels.cuh"
+
+namespace dq {
+
+// ---------------------------------------------------------------------------------------------------
+// ||v_w||_inf as the maximum of the absolute-value bit patterns (exact, order-free).  NaN/Inf patterns
+// compare above every finite value, so a non-finite input surfaces as a non-finite norm.
+// grid (blocks, M); norm_bits must be zero on entry.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) norm_inf_kernel(const float* __restrict__ v, int64_t d, int vec_ok,
+                                                            uint32_t* __restrict__ norm_bits)
+{
+    const float* row = v + (int64_t)blockIdx.y * d;
+    uint32_t m = 0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (int64_t)gridDim.x * blockDim.x;
+    if (vec_ok) {
+        const int64_t ng = d >> 3;
+        for (int64_t g = tid; g < ng; g += nth) {
+            float a[8]; load8(row + (g << 3), a);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) m = max(m, __float_as_uint(a[j]) & 0x7FFFFFFFu);
+        }
+        for (int64_t i = (ng << 3) + tid; i < d; i += nth) m = max(m, __float_as_uint(__ldg(row + i)) & 0x7FFFFFFFu);
+    } else {
+        for (int64_t i = tid; i < d; i += nth) m = max(m, __float_as_uint(__ldg(row + i)) & 0x7FFFFFFFu);
+    }
+    block_atomic_max(m, norm_bits + blockIdx.y);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Dense Q_(delta,b) + pack.  grid (blocks, M).  Each thread turns groups of eight coordinates into BITS
+// bytes.  ngroups covers the zero padding of the packed message (coordinates >= d quantise to code 0).
+// ---------------------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(kThreads)
+quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
+                     uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
+                     const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker_base, uint32_t stream,
+                     int64_t ngroups, int* __restrict__ status)
+{
+    const int w = blockIdx.y;
+    const uint32_t nb = norm_bits[w];
+    const float nrm = __uint_as_float(nb);
+    const bool finite = nb < 0x7F800000u;
+    // delta = nrm / L; inv = 1/delta rounded toward zero so that |v| <= nrm stays inside the hull.
+    const float inv = (finite && nb != 0u) ? __fdiv_rd((float)levels(BITS), nrm) : 0.0f;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        scale[w] = (finite && nb != 0u) ? __fdiv_rn(nrm, (float)levels(BITS)) : 0.0f;
+        if (!finite) set_status(status, DQ_ERR_NONFINITE);
+    }
+    const float* row = v + (int64_t)w * d;
+    uint8_t* out = codes + (int64_t)w * stride;
+    const uint32_t worker = worker_base + (uint32_t)w;
+    const int64_t nth = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += nth) {
+        float a[8];
+        const int64_t i0 = g << 3;
+        if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+        uint32_t r[4], s[8];
+        philox4x32_10((uint32_t)g, round, worker, stream, K, r);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+        store_group<BITS>(out + g * BITS, pack8<BITS>(s));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// ||alpha_w||_1 on an integer grid (order-free): with ||alpha||_inf in [2^(e-1), 2^e) each |alpha_i| is
+// scaled by 2^(35-e), truncated, and the integers are added.  l1_sum must be zero on entry.
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned long long l1_term(float a, double scale)
+{
+    return __double2ull_rz((double)fabsf(a) * scale);
+}
+
+__global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restrict__ v, int64_t d, int vec_ok,
+                                                           const uint32_t* __restrict__ norm_bits,
+                                                           unsigned long long* __restrict__ l1_sum)
+{
+    const int w = blockIdx.y;
+    const uint32_t nb = norm_bits[w];
+    if (nb == 0u || nb >= 0x7F800000u) return;
+    int e; (void)frexpf(__uint_as_float(nb), &e);
+    const double scale = ldexp(1.0, 35 - e);
+    const float* row = v + (int64_t)w * d;
+    unsigned long long acc = 0;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (int64_t)gridDim.x * blockDim.x;
+    const int64_t ng = vec_ok ? (d >> 3) : 0;
+    for (int64_t g = tid; g < ng; g += nth) {
+        float a[8]; load8(row + (g << 3), a);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], scale);
+    }
+    for (int64_t i = (ng << 3) + tid; i < d; i += nth) acc += l1_term(__ldg(row + i), scale);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    __shared__ unsigned long long s_acc[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) s_acc[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long t = 0;
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += s_acc[i];
+        if (t) atomicAdd(l1_sum + w, t);
+    }
+}
+
+// Per-worker constants of eq. (4) with Lemma 2's probabilities, from the two norms.
+struct SparsifyScale { float s; bool empty; };
+
+__device__ __forceinline__ SparsifyScale sparsify_scale(uint32_t nb, unsigned long long l1, float phi)
+{
+    SparsifyScale r; r.s = 0.0f; r.empty = true;
+    if (nb == 0u || nb >= 0x7F800000u) return r;
+    const float ninf = __uint_as_float(nb);
+    int e; (void)frexpf(ninf, &e);
+    const float n1 = (float)ldexp((double)l1, e - 35);
+    if (n1 == 0.0f) return r;
+    const float cap = __fdiv_rn(n1, ninf);                       // Lemma 2: phi <= |alpha|_1 / |alpha|_inf
+    const float phi_eff = (phi > 0.0f) ? fminf(phi, cap) : cap;
+    r.s = __fdiv_rn(phi_eff, n1); r.empty = false;
+    return r;
+}
+
+// m_i = p_i * 2^16 rounded up, p_i = min(1, |alpha_i| s).
+__device__ __forceinline__ uint32_t mask_threshold(float a, float s)
+{
+    const float scaled = ceilf(__fmul_rn(__fmul_rn(fabsf(a), s), 65536.0f));
+    return (scaled >= 65536.0f) ? 65536u : (uint32_t)scaled;
+}
+
+// Survivor mask of one group of eight coordinates and the survivors' beta_i = alpha_i / p_i.
+__device__ __forceinline__ uint32_t sparsify8(const float (&a)[8], float s, const uint32_t (&r)[4], float (&beta)[8])
+{
+    uint32_t mask = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t m = mask_threshold(a[j], s);
+        const bool z = half16(r, j) < m;
+        beta[j] = z ? __fdiv_rn(__fmul_rn(a[j], 65536.0f), (float)m) : 0.0f;
+        mask |= (uint32_t)z << j;
+    }
+    return mask;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Sparsifier pass 1: draw the mask, record ||beta_w||_inf over survivors and, for sparse messages, the
+// number of survivors of every chunk of kChunk coordinates (one warp per chunk, no block-level sync).
+// grid (blocks, M), blockDim = kThreads.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
+                      const unsigned long long* __restrict__ l1_sum, float phi,
+                      const __grid_constant__ PhiloxKeys K, uint32_t round,
+                      uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
+                      int64_t nchunks)
+{
+    const int w = blockIdx.y, lane = threadIdx.x & 31;
+    const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
+    const float* row = v + (int64_t)w * d;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    uint32_t bmax = 0;
+    for (int64_t c = warp; c < nchunks; c += nwarps) {
+        uint32_t cnt = 0;
+        if (!sc.empty) {
+#pragma unroll 2
+            for (int it = 0; it < kChunk / 256; ++it) {
+                const int64_t g = c * (kChunk / 8) + it * 32 + lane, i0 = g << 3;
+                if (i0 >= d) break;
+                float a[8], beta[8];
+                if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+                uint32_t r[4];
+                philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamMask, K, r);
+                const uint32_t mask = sparsify8(a, sc.s, r, beta);
+                if (mask) {
+                    cnt += __popc(mask);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) bmax = max(bmax, __float_as_uint(beta[j]) & 0x7FFFFFFFu);
+                }
+            }
+        }
+        if (chunk_cnt) {
+            cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+            if (lane == 0) chunk_cnt[(int64_t)w * (nchunks + 1) + c] = cnt;
+        }
+    }
+    block_atomic_max(bmax, beta_norm_bits + w);
+}
+
+// Exclusive prefix of the chunk counts of each worker (one block per worker); writes nnz and flags
+// messages that exceed the capacity (their tail is dropped).
+__global__ void __launch_bounds__(kThreads)
+chunk_scan_kernel(uint32_t* __restrict__ chunk_off, int64_t nchunks, int64_t cap, uint32_t* __restrict__ nnz,
+                  int* __restrict__ status)
+{
+    uint32_t* off = chunk_off + (int64_t)blockIdx.x * (nchunks + 1);
+    __shared__ uint32_t s_warp[kThreads / 32];
+    __shared__ uint32_t s_carry;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < nchunks; base += blockDim.x) {
+        const int64_t i = base + threadIdx.x;
+        const uint32_t c = (i < nchunks) ? off[i] : 0u;
+        uint32_t incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if ((threadIdx.x & 31) >= o) incl += t; }
+        if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
+        __syncthreads();
+        uint32_t before = s_carry;
+        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) before += s_warp[k];
+        if (i < nchunks) off[i] = before + incl - c;
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) s_carry = before + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        uint32_t total = s_carry;
+        off[nchunks] = total;
+        if ((int64_t)total > cap) { set_status(status, DQ_ERR_CAPACITY); total = (uint32_t)cap; }
+        nnz[blockIdx.x] = total;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Sparsifier pass 2: redraw the mask, quantise the survivors with delta = ||beta||_inf / L (rounding draw
+// keyed by the coordinate) and emit either the dense packed message (SPARSE_OUT = false) or the
+// (position, code) list at the chunk's offset (SPARSE_OUT = true; codes OR-ed into a zeroed buffer).
+// ---------------------------------------------------------------------------------------------------
+template <int BITS, bool SPARSE_OUT>
+__global__ void __launch_bounds__(kThreads)
+sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
+                     const unsigned long long* __restrict__ l1_sum, float phi,
+                     const __grid_constant__ PhiloxKeys K, uint32_t round,
+                     const uint32_t* __restrict__ beta_norm_bits, const uint32_t* __restrict__ chunk_off,
+                     int64_t nchunks, int64_t ngroups,
+                     uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
+                     uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status)
+{
+    const int w = blockIdx.y, lane = threadIdx.x & 31;
+    const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
+    const uint32_t bb = beta_norm_bits[w];
+    const bool finite = bb < 0x7F800000u && norm_bits[w] < 0x7F800000u;
+    const float bnrm = __uint_as_float(bb);
+    const float inv = (finite && bb != 0u) ? __fdiv_rd((float)levels(BITS), bnrm) : 0.0f;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        scale[w] = (finite && bb != 0u) ? __fdiv_rn(bnrm, (float)levels(BITS)) : 0.0f;
+        if (!finite) set_status(status, DQ_ERR_NONFINITE);
+    }
+    const float* row = v + (int64_t)w * d;
+    uint8_t* out = codes + (int64_t)w * stride;
+    uint32_t* oidx = SPARSE_OUT ? idx + (int64_t)w * cap : nullptr;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t c = warp; c < nchunks; c += nwarps) {
+        uint32_t pos = SPARSE_OUT ? chunk_off[(int64_t)w * (nchunks + 1) + c] : 0u;
+        for (int it = 0; it < kChunk / 256; ++it) {
+            const int64_t g = c * (kChunk / 8) + it * 32 + lane, i0 = g << 3;
+            uint32_t mask = 0;
+            uint32_t s8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s8[j] = 128u << 16;                        // code 0
+            if (!sc.empty && i0 < d) {
+                float a[8], beta[8];
+                if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+                uint32_t r[4];
+                philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamMask, K, r);
+                mask = sparsify8(a, sc.s, r, beta);
+                if (mask) {
+                    philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamGrad, K, r);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) if ((mask >> j) & 1u) s8[j] = round_fixed<BITS>(beta[j], inv, half16(r, j));
+                }
+            }
+            if (!SPARSE_OUT) {
+                if (g < ngroups) store_group<BITS>(out + g * BITS, pack8<BITS>(s8));
+            } else {
+                // ordered positions inside the warp: survivors of lower lanes come first
+                const uint32_t cnt = __popc(mask);
+                uint32_t incl = cnt;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+                uint32_t p = pos + incl - cnt;
+                pos += __shfl_sync(0xFFFFFFFFu, incl, 31);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if ((mask >> j) & 1u) {
+                        if ((int64_t)p < cap) {
+                            oidx[p] = (uint32_t)(i0 + j);
+                            const uint32_t field = ((s8[j] >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
+                            const int64_t bit = (int64_t)p * BITS;
+                            atomicOr(reinterpret_cast<uint32_t*>(out) + (bit >> 5), field << (bit & 31));
+                        }
+                        ++p;
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// First list entry of every coordinate tile of kChunk coordinates in each worker's ascending index
+// list (binary search; one thread per (tile boundary, worker)).
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+tile_ptr_kernel(const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* __restrict__ nnz, int64_t ntiles,
+                uint32_t* __restrict__ tile_ptr)
+{
+    const int w = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t > ntiles) return;
+    const uint32_t* list = idx + (int64_t)w * cap;
+    const uint64_t bound = (uint64_t)t * kChunk;
+    uint32_t lo = 0, hi = nnz[w];
+    while (lo < hi) { uint32_t mid = (lo + hi) >> 1; if ((uint64_t)list[mid] < bound) lo = mid + 1; else hi = mid; }
+    tile_ptr[(int64_t)w * (ntiles + 1) + t] = lo;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Master step: g = (1/M) sum_w code_w delta_w (fused multiply-adds in worker order), u = g + g_full,
+// prox step on x (Algorithms 1/2) or on y with the momentum combination (Algorithm 3), ||x||_inf.
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float prox_h(float v, float thr, float den, float lo, float hi)
+{
+    const float a = __fsub_rn(fabsf(v), thr);
+    float r = (a > 0.0f) ? copysignf(a, v) : 0.0f;
+    if (den != 1.0f) r = __fdiv_rn(r, den);
+    return fminf(fmaxf(r, lo), hi);
+}
+
+template <bool ACC>
+__device__ __forceinline__ float master_update(float acc, float inv_m, float eta, float theta, float thr, float den,
+                                               const ProxParams& pp, float g_full, float x_or_y, float xsnap,
+                                               float& y_out, float& xsum_io)
+{
+    const float u = __fadd_rn(__fmul_rn(acc, inv_m), g_full);
+    const float p = prox_h(__fmaf_rn(-eta, u, x_or_y), thr, den, pp.lo, pp.hi);
+    if (!ACC) return p;
+    y_out = p;
+    const float x = __fmaf_rn(theta, __fsub_rn(p, xsnap), xsnap);
+    xsum_io = __fadd_rn(xsum_io, x);
+    return x;
+}
+
+// Dense messages.  Each thread owns the 32/BITS coordinates of one 32-bit code word per worker.
+template <int BITS, bool ACC>
+__global__ void __launch_bounds__(kThreads)
+master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
+                    const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
+                    const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
+                    uint32_t* __restrict__ normx_bits)
+{
+    constexpr int C = 32 / BITS;
+    extern __shared__ float s_scale[];
+    for (int i = threadIdx.x; i < M; i += blockDim.x) s_scale[i] = scale[i];
+    __syncthreads();
+    const float inv_m = __fdiv_rn(1.0f, (float)M);
+    const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
+    const int64_t nwords = (d + C - 1) / C;
+    const int64_t wstride = stride >> 2;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(codes);
+    uint32_t nmax = 0;
+    const int64_t nth = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nwords; t += nth) {
+        float acc[C];
+#pragma unroll
+        for (int j = 0; j < C; ++j) acc[j] = 0.0f;
+#pragma unroll 4
+        for (int w = 0; w < M; ++w) {
+            const uint32_t word = __ldg(words + (int64_t)w * wstride + t);
+            const float dl = s_scale[w];
+#pragma unroll
+            for (int j = 0; j < C; ++j) acc[j] = __fmaf_rn((float)code_of<BITS>(word, j), dl, acc[j]);
+        }
+        const int64_t i0 = t * C;
+        float* target = ACC ? y : x;
+        if (i0 + C <= d) {
+#pragma unroll
+            for (int q = 0; q < C / 4; ++q) {
+                const int64_t i = i0 + q * 4;
+                const float4 gf = *reinterpret_cast<const float4*>(g_full + i);
+                const float4 cur = *reinterpret_cast<const float4*>(target + i);
+                float4 xs = make_float4(0, 0, 0, 0), sm = make_float4(0, 0, 0, 0), yo, xo;
+                if (ACC) { xs = *reinterpret_cast<const float4*>(xsnap + i); sm = *reinterpret_cast<const float4*>(xsum + i); }
+                xo.x = master_update<ACC>(acc[q * 4 + 0], inv_m, eta, theta, thr, den, pp, gf.x, cur.x, xs.x, yo.x, sm.x);
+                xo.y = master_update<ACC>(acc[q * 4 + 1], inv_m, eta, theta, thr, den, pp, gf.y, cur.y, xs.y, yo.y, sm.y);
+                xo.z = master_update<ACC>(acc[q * 4 + 2], inv_m, eta, theta, thr, den, pp, gf.z, cur.z, xs.z, yo.z, sm.z);
+                xo.w = master_update<ACC>(acc[q * 4 + 3], inv_m, eta, theta, thr, den, pp, gf.w, cur.w, xs.w, yo.w, sm.w);
+                *reinterpret_cast<float4*>(x + i) = xo;
+                if (ACC) { *reinterpret_cast<float4*>(y + i) = yo; *reinterpret_cast<float4*>(xsum + i) = sm; }
+                nmax = max(nmax, max(max(__float_as_uint(xo.x) & 0x7FFFFFFFu, __float_as_uint(xo.y) & 0x7FFFFFFFu),
+                                     max(__float_as_uint(xo.z) & 0x7FFFFFFFu, __float_as_uint(xo.w) & 0x7FFFFFFFu)));
+            }
+        } else {
+            for (int j = 0; j < C && i0 + j < d; ++j) {
+                const int64_t i = i0 + j;
+                float yo = 0.0f, sm = ACC ? xsum[i] : 0.0f;
+                const float xo = master_update<ACC>(acc[j], inv_m, eta, theta, thr, den, pp, g_full[i], target[i],
+                                                    ACC ? xsnap[i] : 0.0f, yo, sm);
+                x[i] = xo;
+                if (ACC) { y[i] = yo; xsum[i] = sm; }
+                nmax = max(nmax, __float_as_uint(xo) & 0x7FFFFFFFu);
+            }
+        }
+    }
+    block_atomic_max(nmax, normx_bits);
+}
+
+// Sparse messages.  One block per tile of kChunk coordinates: the tile's sum is built in shared memory
+// worker by worker (indices inside one message are distinct, so no two threads meet), then the prox.
+template <int BITS, bool ACC>
+__global__ void __launch_bounds__(kThreads)
+master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale,
+                     const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* __restrict__ tile_ptr, int64_t ntiles,
+                     int M, int64_t d, const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
+                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
+                     uint32_t* __restrict__ normx_bits)
+{
+    __shared__ float s_acc[kChunk];
+    const float inv_m = __fdiv_rn(1.0f, (float)M);
+    const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
+    uint32_t nmax = 0;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t lo = tile * kChunk;
+        for (int i = threadIdx.x; i < kChunk; i += blockDim.x) s_acc[i] = 0.0f;
+        __syncthreads();
+        for (int w = 0; w < M; ++w) {
+            const uint32_t* tp = tile_ptr + (int64_t)w * (ntiles + 1) + tile;
+            const uint32_t e0 = tp[0], e1 = tp[1];
+            const uint32_t* list = idx + (int64_t)w * cap;
+            const uint32_t* words = reinterpret_cast<const uint32_t*>(codes + (int64_t)w * stride);
+            const float dl = scale[w];
+            for (uint32_t e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
+                const int64_t bit = (int64_t)e * BITS;
+                const int k = code_of<BITS>(__ldg(words + (bit >> 5)), (int)((bit & 31) / BITS));
+                const int li = (int)((int64_t)list[e] - lo);
+                s_acc[li] = __fmaf_rn((float)k, dl, s_acc[li]);
+            }
+            __syncthreads();
+        }
+        float* target = ACC ? y : x;
+        for (int li = threadIdx.x; li < kChunk && lo + li < d; li += blockDim.x) {
+            const int64_t i = lo + li;
+            float yo = 0.0f, sm = ACC ? xsum[i] : 0.0f;
+            const float xo = master_update<ACC>(s_acc[li], inv_m, eta, theta, thr, den, pp, g_full[i], target[i],
+                                                ACC ? xsnap[i] : 0.0f, yo, sm);
+            x[i] = xo;
+            if (ACC) { y[i] = yo; xsum[i] = sm; }
+            nmax = max(nmax, __float_as_uint(xo) & 0x7FFFFFFFu);
+        }
+        __syncthreads();
+    }
+    block_atomic_max(nmax, normx_bits);
+}
+
+// Test utility: dequantise one message into a dense fp32 vector.
+template <int BITS>
+__global__ void unpack_dense_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scale, int64_t d,
+                                    float* __restrict__ out)
+{
+    const float dl = scale[0];
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t bit = i * BITS;
+        out[i] = __fmul_rn((float)code_of<BITS>(reinterpret_cast<const uint32_t*>(codes)[bit >> 5], (int)((bit & 31) / BITS)), dl);
+    }
+}
+
+template <int BITS>
+__global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scale,
+                                     const uint32_t* __restrict__ idx, const uint32_t* __restrict__ nnz,
+                                     float* __restrict__ out)
+{
+    const float dl = scale[0];
+    const uint32_t n = nnz[0];
+    for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
+        const int64_t bit = (int64_t)e * BITS;
+        out[idx[e]] = __fmul_rn((float)code_of<BITS>(reinterpret_cast<const uint32_t*>(codes)[bit >> 5], (int)((bit & 31) / BITS)), dl);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Host launchers
+// ---------------------------------------------------------------------------------------------------
+static inline int grid_for(int64_t items_per_thread_units, int sm_count, int per_sm = 8)
+{
+    int64_t need = (items_per_thread_units + kThreads - 1) / kThreads;
+    int64_t cap = (int64_t)sm_count * per_sm;
+    if (need < 1) need = 1;
+    return (int)(need < cap ? need : cap);
+}
+
+static inline int vec_ok_for(const float* v, int64_t d) { return ((reinterpret_cast<uintptr_t>(v) & 31) == 0 && (d & 7) == 0) ? 1 : 0; }
+
+void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* norm_bits, cudaStream_t st)
+{
+    cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * M, st);
+    dim3 grid(grid_for((d + 7) / 8, ctx->sm_count), M);
+    norm_inf_kernel<<<grid, kThreads, 0, st>>>(v, d, vec_ok_for(v, d), norm_bits);
+    ctx->launches += 1;
+}
+
+void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
+                          uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
+                          uint32_t stream_id, cudaStream_t st)
+{
+    const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
+    dim3 grid(grid_for(ngroups, ctx->sm_count), M);
+    DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_><<<grid, kThreads, 0, st>>>(
+        v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status)));
+    ctx->launches += 1;
+}
+
+void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
+                          uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st)
+{
+    const int vec_ok = vec_ok_for(v, d);
+    const int64_t nchunks = (d + kChunk - 1) / kChunk;
+    cudaMemsetAsync(ctx->l1_sum, 0, sizeof(unsigned long long) * M, st);
+    cudaMemsetAsync(ctx->beta_norm_bits, 0, sizeof(uint32_t) * M, st);
+    dim3 grid_l1(grid_for((d + 7) / 8, ctx->sm_count), M);
+    norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
+    dim3 grid_c(grid_for(nchunks * 32, ctx->sm_count), M);
+    sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
+                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks);
+    ctx->launches += 2;
+    if (sparse_out) {
+        chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
+        cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
+        DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
+            v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
+            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status)));
+        ctx->launches += 2;
+    } else {
+        const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
+        DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
+            v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
+            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status)));
+        ctx->launches += 1;
+    }
+}
+
+void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg;
+    const int64_t d = c.d;
+    ProxParams pp{c.lambda1, c.lambda2, c.box_lo, c.box_hi};
+    uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
+    cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
+    if (!sparse_msgs) {
+        const int64_t nwords = (d + (32 / c.b) - 1) / (32 / c.b);
+        const int grid = grid_for(nwords, ctx->sm_count);
+        const size_t smem = sizeof(float) * c.M;
+        if (c.accelerated) {
+            DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+        } else {
+            DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+        }
+        ctx->launches += 1;
+    } else {
+        const int64_t ntiles = (d + kChunk - 1) / kChunk;
+        dim3 grid_t((unsigned)((ntiles + 1 + kThreads - 1) / kThreads), c.M);
+        tile_ptr_kernel<<<grid_t, kThreads, 0, st>>>(msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
+        const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
+        if (c.accelerated) {
+            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
+                msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+        } else {
+            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, false><<<grid, kThreads, 0, st>>>(
+                msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+        }
+        ctx->launches += 2;
+    }
+}
+
+void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, float* out, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg;
+    const uint8_t* codes = msgs->codes + (int64_t)w * msgs->stride;
+    if (!sparse_msgs) {
+        DQ_DISPATCH_BITS(c.b, (unpack_dense_kernel<BITS_><<<grid_for(c.d, ctx->sm_count), kThreads, 0, st>>>(codes, msgs->scale + w, c.d, out)));
+    } else {
+        cudaMemsetAsync(out, 0, sizeof(float) * c.d, st);
+        DQ_DISPATCH_BITS(c.b, (unpack_sparse_kernel<BITS_><<<grid_for(msgs->cap, ctx->sm_count), kThreads, 0, st>>>(
+            codes, msgs->scale + w, msgs->idx + (int64_t)w * msgs->cap, msgs->nnz + w, out)));
+    }
+    ctx->launches += 1;
+}
+
+}  // namespace dq

@@ -1,0 +1,176 @@
+// Shared device helpers for the double-quantization kernels (sm_100a).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dq.h"
+
+namespace dq {
+
+constexpr uint32_t kMaster = 0xFFFFFFFFu;
+enum : uint32_t { kStreamModel = 0, kStreamGrad = 1, kStreamMask = 2, kStreamBatch = 3 };
+constexpr int kThreads = 256;
+constexpr int kChunk = 2048;   // coordinates one warp owns per step of the sparsifier (32 lanes x 8 x 8)
+
+// The ten round keys of Philox4x32-10 depend on the seed only; the host expands them once so that the
+// kernels read them from the constant bank.
+struct PhiloxKeys { uint32_t k0[10]; uint32_t k1[10]; };
+
+inline PhiloxKeys expand_keys(uint64_t seed)
+{
+    PhiloxKeys K;
+    uint32_t a = (uint32_t)seed, b = (uint32_t)(seed >> 32);
+    for (int r = 0; r < 10; ++r) { K.k0[r] = a; K.k1[r] = b; a += 0x9E3779B9u; b += 0xBB67AE85u; }
+    return K;
+}
+
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and a word shuffle.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              const PhiloxKeys& K, uint32_t (&out)[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+        uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ K.k0[r];
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ K.k1[r];
+        c1 = (uint32_t)p1; c3 = (uint32_t)p0; c0 = n0; c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// 16-bit draw of coordinate lane j (0..7) of a Philox call: low / high half of word j >> 1.
+__device__ __forceinline__ uint32_t half16(const uint32_t (&w)[4], int j)
+{
+    return (j & 1) ? (w[j >> 1] >> 16) : (w[j >> 1] & 0xFFFFu);
+}
+
+constexpr __host__ __device__ int levels(int bits) { return (1 << (bits - 1)) - 1; }
+
+// Fixed-point stochastic rounding of one coordinate.  r = fl(v*inv + 384) lies in [256,512) where the
+// fp32 spacing is 2^-15, so bits(r) is (v*inv + 128) * 2^15 plus a constant.  Doubling it and adding the
+// raw 16-bit draw h = 2u + c puts floor(((v*inv + 128) * 2^15 + u) / 2^15) into byte 2 of the result;
+// the constant only touches bits above byte 2.  Returns that word; byte 2 is the code plus 128.
+template <int BITS>
+__device__ __forceinline__ uint32_t round_fixed(float v, float inv, uint32_t h16)
+{
+    float r = __fmaf_rn(v, inv, 384.0f);
+    r = fminf(fmaxf(r, 384.0f - (float)(1 << (BITS - 1))), 384.0f + (float)levels(BITS));
+    return (__float_as_uint(r) << 1) + h16;
+}
+
+// Packs the codes held in byte 2 of s[0..7] into BITS-bit two's complement, coordinate 0 lowest.
+// (code + 128) mod 2^BITS equals the two's complement field for BITS < 8; for BITS = 8 flip bit 7.
+template <int BITS>
+__device__ __forceinline__ uint64_t pack8(const uint32_t (&s)[8])
+{
+    uint32_t a = __byte_perm(__byte_perm(s[0], s[1], 0x0062), __byte_perm(s[2], s[3], 0x0062), 0x5410);
+    uint32_t b = __byte_perm(__byte_perm(s[4], s[5], 0x0062), __byte_perm(s[6], s[7], 0x0062), 0x5410);
+    if (BITS == 8) return ((uint64_t)(b ^ 0x80808080u) << 32) | (uint64_t)(a ^ 0x80808080u);
+    if (BITS == 4) {
+        a &= 0x0F0F0F0Fu; b &= 0x0F0F0F0Fu;
+        a |= a >> 4; b |= b >> 4;                       // bytes 0 and 2 now hold two codes each
+        return (uint64_t)__byte_perm(a, b, 0x6420);
+    }
+    a &= 0x03030303u; b &= 0x03030303u;                 // BITS == 2
+    a |= a >> 6; b |= b >> 6;                           // bytes 0 and 2 hold two codes in bits 0..3
+    a = (a & 0xFu) | ((a >> 12) & 0xF0u);
+    b = (b & 0xFu) | ((b >> 12) & 0xF0u);
+    return (uint64_t)(a | (b << 8));
+}
+
+template <int BITS>
+__device__ __forceinline__ void store_group(uint8_t* dst, uint64_t word)
+{
+    if (BITS == 8) *reinterpret_cast<uint2*>(dst) = make_uint2((uint32_t)word, (uint32_t)(word >> 32));
+    else if (BITS == 4) *reinterpret_cast<uint32_t*>(dst) = (uint32_t)word;
+    else *reinterpret_cast<uint16_t*>(dst) = (uint16_t)word;
+}
+
+// Sign-extended code j of a 32-bit word of packed BITS-bit codes.
+template <int BITS>
+__device__ __forceinline__ int code_of(uint32_t word, int j)
+{
+    return ((int)(word << (32 - BITS * (j + 1)))) >> (32 - BITS);
+}
+
+// Eight consecutive floats with one 256-bit read-only load (pointer 32-byte aligned).
+__device__ __forceinline__ void load8(const float* p, float (&v)[8])
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p));
+}
+
+// Eight floats starting at coordinate i0 of a row of length d, zero beyond the end; any alignment.
+__device__ __forceinline__ void load8_guarded(const float* row, int64_t i0, int64_t d, float (&v)[8])
+{
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = (i0 + j < d) ? __ldg(row + i0 + j) : 0.0f;
+}
+
+__device__ __forceinline__ void set_status(int* status, int code)
+{
+    if (*reinterpret_cast<volatile int*>(status) == 0) atomicCAS(status, 0, code);
+}
+
+__device__ __forceinline__ uint32_t warp_max_u32(uint32_t v) { return __reduce_max_sync(0xFFFFFFFFu, v); }
+
+// Block-wide maximum of unsigned values folded into *dst with one atomic per block.
+__device__ __forceinline__ void block_atomic_max(uint32_t v, uint32_t* dst)
+{
+    __shared__ uint32_t s_max[kThreads / 32];
+    v = warp_max_u32(v);
+    if ((threadIdx.x & 31) == 0) s_max[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        uint32_t t = (threadIdx.x < (blockDim.x >> 5)) ? s_max[threadIdx.x] : 0u;
+        t = warp_max_u32(t);
+        if (threadIdx.x == 0 && t != 0u) atomicMax(dst, t);
+    }
+}
+
+struct ProxParams { float lambda1, lambda2, lo, hi; };
+
+#define DQ_DISPATCH_BITS(bits, CALL)                 \
+    switch (bits) {                                  \
+        case 2: { constexpr int BITS_ = 2; CALL; } break; \
+        case 4: { constexpr int BITS_ = 4; CALL; } break; \
+        default: { constexpr int BITS_ = 8; CALL; } break; \
+    }
+
+}  // namespace dq
+
+// Host-side context behind the opaque dq_ctx.
+struct dq_ctx {
+    dq_config cfg;
+    dq_data data;
+    bool has_data;
+    dq::PhiloxKeys keys;
+    int sm_count;
+    // scratch owned by the context
+    uint32_t* norm_bits;        // [M]   ||v_w||_inf bit patterns when the caller supplies none
+    uint32_t* beta_norm_bits;   // [M]   ||beta_w||_inf over survivors
+    unsigned long long* l1_sum; // [M]   fixed-point ||alpha_w||_1
+    uint32_t* chunk_off;        // [M][nchunks + 1] survivors per chunk, then their exclusive prefix
+    uint32_t* tile_ptr;         // [M][nchunks + 1] first list entry of each coordinate tile (sparse master)
+    uint32_t* xnorm_bits;       // [1]   ||x||_inf when the caller supplies none
+    int* status;                // sticky device status word
+    int64_t nchunks;
+    // buffers of dq_round / dq_codec_round
+    float* alpha;               // [M][d]
+    float* ninf;                // [M]
+    int32_t* rows;              // [M][B]
+    uint8_t* codes_x;           // packed model
+    float* delta_x;
+    float* xhat_diff;           // [d] dequantised model minus snapshot
+    double* g64;                // [d] full-gradient accumulator
+    dq_msgs msgs;
+    uint64_t* bits;             // [2] device counters
+    // device-resident state for the host-buffer entry point
+    float *hx, *hg, *hv, *hnorm;
+    // bookkeeping
+    int64_t launches;
+    int64_t rounds_in_epoch;
+    int64_t epoch;
+};

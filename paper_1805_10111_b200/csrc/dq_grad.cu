@@ -1,0 +1,351 @@
+// Gradient kernels: the worker's variance-reduced minibatch gradient (Algorithm 1 step 11), the epoch's
+// full gradient (step 5), the epoch-boundary state update (steps 3/14, Algorithm 3 steps 3/15), the
+// objective of eq. (1) and the transmitted-bit counters.  f_a(x) = log(1 + exp(-y_a <a_a, x>)).
+#include <cuda_bf16.h>
+
+#include "dq_common.cuh"
+#include "dq_kernels.cuh"
+
+namespace dq {
+
+constexpr int kRowsPerBlock = 16;   // rows of one worker handled by one block of the dense kernels
+
+__device__ __forceinline__ float sigmoidf_(float t) { return __fdiv_rn(1.0f, 1.0f + expf(-t)); }
+
+// slope(z) = d/dz log(1+exp(-y z)) = -y sigma(-y z).  The worker needs slope(zs + dz) - slope(zs); written
+// as y * sigma(-y (zs+dz)) * sigma(y zs) * expm1(y dz) it has no cancellation when dz is small.
+__device__ __forceinline__ float slope_difference(float y, float zs, float dz)
+{
+    return y * sigmoidf_(-y * (zs + dz)) * sigmoidf_(y * zs) * expm1f(y * dz);
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+// <a_row, vec> for one dense row, computed by one warp (fp32 partial sums per lane, double across lanes).
+template <class T>
+__device__ __forceinline__ double warp_dot_dense(const T* __restrict__ row, const float* __restrict__ vec, int64_t d, int lane)
+{
+    float s0 = 0.0f, s1 = 0.0f;
+    int64_t i = lane;
+    for (; i + 32 < d; i += 64) { s0 = fmaf(to_float(row[i]), vec[i], s0); s1 = fmaf(to_float(row[i + 32]), vec[i + 32], s1); }
+    if (i < d) s0 = fmaf(to_float(row[i]), vec[i], s0);
+    return warp_sum((double)s0 + (double)s1);
+}
+
+__device__ __forceinline__ double warp_dot_csr(const float* __restrict__ val, const int32_t* __restrict__ col, int64_t k0, int64_t k1,
+                                                const float* __restrict__ vec, int lane)
+{
+    double s = 0.0;
+    for (int64_t k = k0 + lane; k < k1; k += 32) s += (double)__ldg(val + k) * (double)__ldg(vec + __ldg(col + k));
+    return warp_sum(s);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Minibatch rows: worker w draws slot j from its partition [floor(w n/M), floor((w+1) n/M)) with word
+// (j & 3) of Philox counter (j >> 2, round, w, batch stream).
+// ---------------------------------------------------------------------------------------------------
+__global__ void sample_rows_kernel(const __grid_constant__ PhiloxKeys K, uint32_t round, int M, int B, int64_t n,
+                                   int32_t* __restrict__ rows)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= M * B) return;
+    const int w = t / B, j = t % B;
+    const int64_t lo = ((int64_t)w * n) / M, hi = ((int64_t)(w + 1) * n) / M;
+    uint32_t r[4];
+    philox4x32_10((uint32_t)(j >> 2), round, (uint32_t)w, kStreamBatch, K, r);
+    const uint32_t word = (j & 3) == 0 ? r[0] : (j & 3) == 1 ? r[1] : (j & 3) == 2 ? r[2] : r[3];
+    rows[t] = (int32_t)(lo + (int64_t)(((uint64_t)word * (uint64_t)(hi - lo)) >> 32));
+}
+
+// xhat - xsnap with xhat_i = code_i * delta_x (the transmitted low-precision model).
+template <int BITS>
+__global__ void dequant_diff_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ delta_x,
+                                    const float* __restrict__ xsnap, int64_t d, float* __restrict__ diff)
+{
+    const float dl = *delta_x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t bit = i * BITS;
+        const int k = code_of<BITS>(reinterpret_cast<const uint32_t*>(codes)[bit >> 5], (int)((bit & 31) / BITS));
+        diff[i] = __fsub_rn(__fmul_rn((float)k, dl), xsnap[i]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// CSR worker gradient: one warp per sampled row.  dz = <a, xhat - xsnap>, slope difference, then the
+// row is scattered into alpha_w with fp32 atomics (alpha must be zero on entry).
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict__ col, const int64_t* __restrict__ row_ptr,
+                       const float* __restrict__ labels, const float* __restrict__ diff, const float* __restrict__ z_snap,
+                       const int32_t* __restrict__ rows, int M, int B, int64_t d, float* __restrict__ alpha)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (slot >= (int64_t)M * B) return;
+    const int w = (int)(slot / B);
+    const int64_t a = rows[slot];
+    const int64_t k0 = row_ptr[a], k1 = row_ptr[a + 1];
+    const float dz = (float)warp_dot_csr(val, col, k0, k1, diff, lane);
+    const float r = slope_difference(labels[a], z_snap[a], dz) / (float)B;
+    float* out = alpha + (int64_t)w * d;
+    for (int64_t k = k0 + lane; k < k1; k += 32) atomicAdd(out + __ldg(col + k), r * __ldg(val + k));
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Dense worker gradient (fp32 or bf16 features).  grid (ceil(B / kRowsPerBlock), M).  Phase A: one warp
+// per row computes the slope difference; phase B: threads own columns and add the block's rows.
+// alpha must be zero on entry when more than one block serves a worker.
+// ---------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void __launch_bounds__(kThreads)
+worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
+                         const float* __restrict__ z_snap, const int32_t* __restrict__ rows, int B, int64_t d,
+                         float* __restrict__ alpha)
+{
+    __shared__ float s_r[kRowsPerBlock];
+    __shared__ int64_t s_row[kRowsPerBlock];
+    const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int j0 = blockIdx.x * kRowsPerBlock;
+    const int nrows = min(kRowsPerBlock, B - j0);
+    for (int j = warp; j < nrows; j += kThreads / 32) {
+        const int64_t a = rows[(int64_t)w * B + j0 + j];
+        const float dz = (float)warp_dot_dense(X + a * d, diff, d, lane);
+        if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_row[j] = a; }
+    }
+    __syncthreads();
+    float* out = alpha + (int64_t)w * d;
+    for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
+        float s = 0.0f;
+        for (int j = 0; j < nrows; ++j) s = fmaf(s_r[j], to_float(X[s_row[j] * d + i]), s);
+        if (gridDim.x == 1) out[i] = s; else atomicAdd(out + i, s);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Full gradient over all n rows at xsnap, accumulated in double; also stores the margins z_snap.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+full_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict__ col, const int64_t* __restrict__ row_ptr,
+                     const float* __restrict__ labels, const float* __restrict__ x, int64_t n, float* __restrict__ z_out,
+                     double* __restrict__ g64)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    for (int64_t a = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; a < n; a += nwarps) {
+        const int64_t k0 = row_ptr[a], k1 = row_ptr[a + 1];
+        const double z = warp_dot_csr(val, col, k0, k1, x, lane);
+        const double y = (double)labels[a];
+        const double c = -y / (1.0 + exp(y * z));
+        if (lane == 0 && z_out) z_out[a] = (float)z;
+        for (int64_t k = k0 + lane; k < k1; k += 32) atomicAdd(g64 + __ldg(col + k), c * (double)__ldg(val + k));
+    }
+}
+
+template <class T>
+__global__ void __launch_bounds__(kThreads)
+full_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ x, int64_t n,
+                       int64_t d, float* __restrict__ z_out, double* __restrict__ g64)
+{
+    __shared__ float s_c[kRowsPerBlock];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int64_t a0 = (int64_t)blockIdx.x * kRowsPerBlock; a0 < n; a0 += (int64_t)gridDim.x * kRowsPerBlock) {
+        const int nrows = (int)min((int64_t)kRowsPerBlock, n - a0);
+        for (int j = warp; j < nrows; j += kThreads / 32) {
+            const double z = warp_dot_dense(X + (a0 + j) * d, x, d, lane);
+            const double y = (double)labels[a0 + j];
+            if (lane == 0) { s_c[j] = (float)(-y / (1.0 + exp(y * z))); if (z_out) z_out[a0 + j] = (float)z; }
+        }
+        __syncthreads();
+        for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
+            double s = 0.0;
+            for (int j = 0; j < nrows; ++j) s += (double)s_c[j] * (double)to_float(X[(a0 + j) * d + i]);
+            atomicAdd(g64 + i, s);
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void finish_full_grad_kernel(const double* __restrict__ g64, int64_t d, double inv_n, float* __restrict__ g)
+{
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x)
+        g[i] = (float)(g64[i] * inv_n);
+}
+
+// Epoch boundary on the iterates.  Algorithms 1/2: xsnap <- x.  Algorithm 3: xsnap <- xsum / m (if m > 0),
+// xsum <- 0, x <- xsnap + theta (y - xsnap).  Also ||x||_inf.
+__global__ void __launch_bounds__(kThreads)
+epoch_state_kernel(float* __restrict__ x, float* __restrict__ xsnap, const float* __restrict__ y, float* __restrict__ xsum,
+                   int64_t d, int accelerated, int64_t m_prev, float theta, uint32_t* __restrict__ normx_bits)
+{
+    uint32_t nmax = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        float xi;
+        if (!accelerated) {
+            xi = x[i]; xsnap[i] = xi;
+        } else {
+            float xs = xsnap[i];
+            if (m_prev > 0) { xs = __fdiv_rn(xsum[i], (float)m_prev); xsnap[i] = xs; }
+            xsum[i] = 0.0f;
+            xi = __fmaf_rn(theta, __fsub_rn(y[i], xs), xs);
+            x[i] = xi;
+        }
+        nmax = max(nmax, __float_as_uint(xi) & 0x7FFFFFFFu);
+    }
+    block_atomic_max(nmax, normx_bits);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Objective P(x) = (1/n) sum log(1+exp(-y z)) + lambda1 |x|_1 + (lambda2/2) |x|^2 into one double.
+// ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ double softplus(double m) { return m > 0.0 ? m + log1p(exp(-m)) : log1p(exp(m)); }
+
+__device__ __forceinline__ void block_add_double(double v, double* dst)
+{
+    __shared__ double s_part[kThreads / 32];
+    v = warp_sum(v);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x == 0) { double t = 0.0; for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += s_part[i]; atomicAdd(dst, t); }
+    __syncthreads();
+}
+
+template <int FMT>
+__global__ void __launch_bounds__(kThreads)
+objective_loss_kernel(dq_data D, const float* __restrict__ x, double* __restrict__ P)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    double acc = 0.0;
+    for (int64_t a = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; a < D.n; a += nwarps) {
+        double z;
+        if (FMT == DQ_CSR_F32) z = warp_dot_csr((const float*)D.values, D.col_idx, D.row_ptr[a], D.row_ptr[a + 1], x, lane);
+        else if (FMT == DQ_DENSE_F32) z = warp_dot_dense((const float*)D.values + a * D.d, x, D.d, lane);
+        else z = warp_dot_dense((const __nv_bfloat16*)D.values + a * D.d, x, D.d, lane);
+        if (lane == 0) acc += softplus(-(double)D.labels[a] * z) / (double)D.n;
+    }
+    block_add_double(acc, P);
+}
+
+__global__ void __launch_bounds__(kThreads)
+objective_reg_kernel(const float* __restrict__ x, int64_t d, float l1, float l2, double* __restrict__ P)
+{
+    double acc = 0.0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        const double v = (double)x[i];
+        acc += (double)l1 * fabs(v) + 0.5 * (double)l2 * v * v;
+    }
+    block_add_double(acc, P);
+}
+
+// Transmitted bits of one round by the paper's message sizes (Section 3.1; remark after Theorem 3).
+__global__ void bits_kernel(int M, int64_t d, int bx, int b, int flag_round, int sparse_msgs, const uint32_t* __restrict__ nnz,
+                            uint64_t* __restrict__ bits_down, uint64_t* __restrict__ bits_up)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    *bits_down = flag_round ? (uint64_t)M : (uint64_t)M * (32ull + (uint64_t)bx * (uint64_t)d);
+    uint64_t up = 0;
+    int logd = 0; while (((int64_t)1 << logd) < d) ++logd;
+    for (int w = 0; w < M; ++w) up += sparse_msgs ? 32ull + (uint64_t)nnz[w] * (uint64_t)(logd + b) : 32ull + (uint64_t)b * (uint64_t)d;
+    *bits_up = up;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Host launchers
+// ---------------------------------------------------------------------------------------------------
+static inline int blocks_for(int64_t threads_needed, int sm_count, int per_sm = 8)
+{
+    int64_t need = (threads_needed + kThreads - 1) / kThreads, cap = (int64_t)sm_count * per_sm;
+    if (need < 1) need = 1;
+    return (int)(need < cap ? need : cap);
+}
+
+void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
+    cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
+    epoch_state_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(s->x, s->x_snap, s->y, s->x_sum, c.d, c.accelerated,
+                                                                            ctx->rounds_in_epoch, theta, nx);
+    cudaMemsetAsync(ctx->g64, 0, sizeof(double) * c.d, st);
+    if (D.format == DQ_CSR_F32) {
+        full_grad_csr_kernel<<<blocks_for(D.n * 32, ctx->sm_count), kThreads, 0, st>>>(
+            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, s->x_snap, D.n, s->z_snap, ctx->g64);
+    } else {
+        const int64_t nblk = (D.n + kRowsPerBlock - 1) / kRowsPerBlock;
+        const int grid = (int)(nblk < (int64_t)ctx->sm_count * 8 ? nblk : (int64_t)ctx->sm_count * 8);
+        if (D.format == DQ_DENSE_F32)
+            full_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+        else
+            full_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+    }
+    finish_full_grad_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(ctx->g64, c.d, 1.0 / (double)D.n, s->g_full);
+    ctx->launches += 3;
+}
+
+void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot, const dq_state* s,
+                        uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    if (is_snapshot) {                     // xhat = xsnap: every slope difference is exactly zero
+        cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        cudaMemsetAsync(norm_inf, 0, sizeof(float) * c.M, st);
+        return;
+    }
+    if (!batch_idx) {
+        sample_rows_kernel<<<(c.M * c.B + kThreads - 1) / kThreads, kThreads, 0, st>>>(ctx->keys, round, c.M, c.B, D.n, ctx->rows);
+        batch_idx = ctx->rows;
+        ctx->launches += 1;
+    }
+    DQ_DISPATCH_BITS(c.bx, (dequant_diff_kernel<BITS_><<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(
+        codes_x, delta_x, s->x_snap, c.d, ctx->xhat_diff)));
+    if (D.format == DQ_CSR_F32) {
+        cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        worker_grad_csr_kernel<<<(int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st>>>(
+            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.M, c.B, c.d, alpha);
+    } else {
+        dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
+        if (grid.x > 1) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        if (D.format == DQ_DENSE_F32)
+            worker_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+        else
+            worker_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+    }
+    ctx->launches += 2;
+    launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
+}
+
+void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    cudaMemsetAsync(P, 0, sizeof(double), st);
+    const int grid = blocks_for(D.n * 32, ctx->sm_count);
+    if (D.format == DQ_CSR_F32) objective_loss_kernel<DQ_CSR_F32><<<grid, kThreads, 0, st>>>(D, x, P);
+    else if (D.format == DQ_DENSE_F32) objective_loss_kernel<DQ_DENSE_F32><<<grid, kThreads, 0, st>>>(D, x, P);
+    else objective_loss_kernel<DQ_DENSE_BF16><<<grid, kThreads, 0, st>>>(D, x, P);
+    objective_reg_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(x, c.d, c.lambda1, c.lambda2, P);
+    ctx->launches += 2;
+}
+
+void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* nnz, uint64_t* bits_down, uint64_t* bits_up,
+                 cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg;
+    bits_kernel<<<1, 32, 0, st>>>(c.M, c.d, c.bx, c.b, flag_round, sparse_msgs ? 1 : 0, nnz, bits_down, bits_up);
+    ctx->launches += 1;
+}
+
+}  // namespace dq

@@ -1,0 +1,25 @@
+// Host-side launchers shared between the translation units of libdq.
+#pragma once
+#include "dq_common.cuh"
+
+namespace dq {
+
+// codec (dq_codec.cu)
+void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* norm_bits, cudaStream_t st);
+void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
+                          uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
+                          uint32_t stream_id, cudaStream_t st);
+void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
+                          uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
+void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st);
+void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, float* out, cudaStream_t st);
+
+// gradients (dq_grad.cu)
+void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st);
+void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot, const dq_state* s,
+                        uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st);
+void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st);
+void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* nnz, uint64_t* bits_down,
+                 uint64_t* bits_up, cudaStream_t st);
+
+}  // namespace dq
