@@ -1,0 +1,358 @@
+"""GPU parity of the gradient stages and of whole rounds against the CPU oracle, through the C ABI.
+
+Float stages (worker gradient, full gradient, objective) are compared within
+    |gpu - ora| <= 1e-5 * max(|ora|, S_i, 1e-3 * ||ora||_inf)
+where S_i is the oracle's sum of absolute contributions to coordinate i (a cancelling sum has no
+meaningful relative error).  Integer stages are bit-exact given the same fp32 inputs.  In lockstep runs the
+GPU starts every round from the oracle's state; its codes are checked bit-exactly against the oracle's
+quantiser applied to the GPU's own gradient, and disagreements with the oracle's own codes ("flips", which
+need the rounding position to sit within a few 2^-15 steps of the decision threshold) are counted."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1805_10111_b200 import synth
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+
+
+@pytest.fixture(scope="module")
+def dq():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_1805_10111_b200 as dq
+    dq.lib()
+    return dq
+
+
+def _dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _odata(h):
+    return oracle.Dataset(h.format, h.n, h.d, h.values, h.labels, h.col_idx, h.row_ptr)
+
+
+def _close(gpu, ora, S=None, rel=1e-5):
+    """Number of coordinates outside the tolerance and the worst error in units of the tolerance scale."""
+    ora = ora.astype(np.float64); gpu = gpu.astype(np.float64)
+    scale = np.maximum(np.abs(ora), 1e-3 * np.abs(ora).max())
+    if S is not None:
+        scale = np.maximum(scale, S.astype(np.float64))
+    bad = np.abs(gpu - ora) > rel * scale + 1e-37
+    return int(bad.sum()), float((np.abs(gpu - ora) / (scale + 1e-300)).max())
+
+
+_PROBLEMS = {}
+
+
+def _problem(name):
+    if name not in _PROBLEMS:
+        if name == "dense":
+            _PROBLEMS[name] = synth.dense_logistic(500, 203, 60)             # d not a multiple of 4
+        elif name == "csr":
+            _PROBLEMS[name] = synth.sparse_logistic(3000, 5003, 30.0, 1.1, 61)
+        elif name == "bf16":
+            _PROBLEMS[name] = synth.dense_bf16_logistic(700, 520, 62)
+        elif name == "c1":
+            _PROBLEMS[name] = synth.config1()
+        elif name == "c2":
+            _PROBLEMS[name] = synth.config2()
+        elif name == "c3":
+            _PROBLEMS[name] = synth.config3(n=60000)                          # full width d = 2^20, fewer rows
+        elif name == "c4":
+            _PROBLEMS[name] = synth.config4(n=16384)                          # full width d = 4096, fewer rows
+    return _PROBLEMS[name]
+
+
+def _abs_grad_scale(h, x):
+    """(1/n) sum_a |slope_a| |a_ai|: the magnitude that bounds the rounding error of the full gradient."""
+    od = _odata(h)
+    _, z = oracle.full_grad(od, x)
+    y = h.labels.astype(np.float64)
+    c = np.abs(-y / (1.0 + np.exp(y * z.astype(np.float64))))
+    if h.format == synth.CSR_F32:
+        rows = np.repeat(np.arange(h.n), np.diff(h.row_ptr))
+        S = np.bincount(h.col_idx, weights=c[rows] * np.abs(h.values.astype(np.float64)), minlength=h.d)
+    else:
+        X = h.values if h.format == synth.DENSE_F32 else synth.bf16_bits_to_f32(h.values)
+        S = c @ np.abs(X.astype(np.float64))
+    return (S / h.n).astype(F32)
+
+
+@pytest.mark.parametrize("name", ["dense", "csr", "bf16"])
+def test_epoch_begin_full_gradient(dq, name):
+    import torch
+    h = _problem(name)
+    x0 = synth.normal_vector(h.d, 70, 0.3)
+    cfg = dq.make_config(h.d, 3, B=4, seed=1)
+    rc, ctx = dq.dq_create(cfg, dq.Data(h)); assert rc == 0
+    st = dq.State(x0, n=h.n)
+    st.x_snap.zero_()
+    assert dq.dq_epoch_begin(ctx, st) == 0
+    g, z = oracle.full_grad(_odata(h), x0)
+    assert np.array_equal(st.x_snap.cpu().numpy(), x0)                        # step 3: snapshot <- x
+    assert st.norm_x.item() == np.abs(x0).max()
+    assert np.allclose(st.z_snap.cpu().numpy(), z, rtol=2e-6, atol=1e-6)
+    nbad, worst = _close(st.g_full.cpu().numpy(), g, _abs_grad_scale(h, x0), rel=1e-6)
+    assert nbad == 0, (nbad, worst)
+    P = torch.zeros(1, dtype=torch.float64, device="cuda")
+    assert dq.dq_objective(ctx, st.x, P) == 0
+    cfg2 = dq.make_config(h.d, 3, B=4, seed=1, lambda1=0.01, lambda2=0.1)
+    rc, ctx2 = dq.dq_create(cfg2, dq.Data(h)); assert rc == 0
+    P2 = torch.zeros(1, dtype=torch.float64, device="cuda")
+    assert dq.dq_objective(ctx2, st.x, P2) == 0
+    assert abs(P.item() - oracle.objective(_odata(h), x0, 0, 0)) < 1e-7
+    assert abs(P2.item() - oracle.objective(_odata(h), x0, 0.01, 0.1)) < 1e-7 * max(1.0, P2.item())
+    dq.dq_destroy(ctx); dq.dq_destroy(ctx2)
+
+
+@pytest.mark.parametrize("name", ["dense", "csr", "bf16"])
+@pytest.mark.parametrize("bx", [4, 8])
+def test_worker_gradient(dq, name, bx):
+    import torch
+    h = _problem(name)
+    M, B, seed, rnd = 3, 37, 21, 5
+    xs = synth.normal_vector(h.d, 71, 0.3)
+    x = (xs + synth.normal_vector(h.d, 72, 0.02)).astype(F32)
+    cfg = dq.make_config(h.d, M, B=B, bx=bx, seed=seed)
+    rc, ctx = dq.dq_create(cfg, dq.Data(h)); assert rc == 0
+    st = dq.State(xs, n=h.n)
+    assert dq.dq_epoch_begin(ctx, st) == 0
+    cx, dx, _ = oracle.quantize(x, bx, seed, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+    xhat = cx.astype(F32) * dx
+    codes_x = _dev(oracle.pack(cx, bx)); delta_x = _dev(np.array([dx], F32))
+    alpha = torch.full((M, h.d), 3.0, device="cuda"); ninf = torch.zeros(M, device="cuda")
+    assert dq.dq_worker_grad(ctx, codes_x, delta_x, 0, st, rnd, None, alpha, ninf) == 0
+    rows_gpu = dq.device_view(dq.dq_round_buffers(ctx)[1]["batch_idx"], M * B, torch.int32).cpu().numpy().reshape(M, B)
+    a_gpu = alpha.cpu().numpy()
+    for w in range(M):
+        rows = oracle.sample_batch(seed, rnd, w, M, h.n, B)
+        assert np.array_equal(rows_gpu[w], rows)
+        a, S = oracle.worker_grad(_odata(h), xhat, xs, rows)
+        nbad, worst = _close(a_gpu[w], a, S)
+        assert nbad == 0, (w, nbad, worst)
+        assert ninf[w].item() == np.abs(a_gpu[w]).max()
+    # explicit batch indices, and the flag round (xhat = xsnap gives exactly zero)
+    mine = np.stack([np.arange(B) * 3 % h.n for _ in range(M)]).astype(np.int32)
+    assert dq.dq_worker_grad(ctx, codes_x, delta_x, 0, st, rnd, _dev(mine), alpha, ninf) == 0
+    a, S = oracle.worker_grad(_odata(h), xhat, xs, mine[1].astype(np.int64))
+    assert _close(alpha[1].cpu().numpy(), a, S)[0] == 0
+    assert dq.dq_worker_grad(ctx, None, None, 1, st, rnd, None, alpha, ninf) == 0
+    assert not alpha.any().item() and not ninf.any().item()
+    dq.dq_destroy(ctx)
+
+
+class Lockstep:
+    """Runs the GPU library and the oracle side by side, restarting the GPU from the oracle's state every round."""
+
+    def __init__(self, dq, h, x0, **kw):
+        self.dq, self.h = dq, h
+        okw = dict(l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0), box_lo=kw.get("box_lo", -np.inf),
+                   box_hi=kw.get("box_hi", np.inf), sparsify=kw.get("sparsify", 0), phi=kw.get("phi", 0.0),
+                   msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"])
+        self.cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
+        self.ocfg = oracle.make_config(h.d, kw["M"], kw["B"], kw["bx"], kw["b"], **okw)
+        self.data = dq.Data(h)
+        rc, self.ctx = dq.dq_create(self.cfg, self.data); assert rc == 0
+        self.st = dq.State(x0, n=h.n, accelerated=bool(self.cfg.accelerated))
+        self.run = oracle.Run(self.ocfg, _odata(h), x0)
+        self.flips = 0; self.far_flips = 0; self.coords = 0; self.worst_alpha = 0.0
+        import torch
+        self.bits = torch.zeros(2, dtype=torch.int64, device="cuda")
+
+    def sync_state(self):
+        st, run = self.st, self.run
+        st.x.copy_(_dev(run.x)); st.x_snap.copy_(_dev(run.xsnap)); st.g_full.copy_(_dev(run.gfull))
+        if self.cfg.accelerated:
+            st.y.copy_(_dev(run.y)); st.x_sum.copy_(_dev(run.xsum))
+        st.norm_x.copy_(_dev(np.array([np.abs(run.x).max()], F32)))
+
+    def epoch(self, theta=0.0):
+        dq = self.dq
+        self.sync_state()
+        assert dq.dq_epoch_begin(self.ctx, self.st, theta) == 0
+        self.run.epoch_begin(theta)
+        assert np.array_equal(self.st.x_snap.cpu().numpy(), self.run.xsnap)
+        assert np.array_equal(self.st.x.cpu().numpy(), self.run.x)
+        nbad, worst = _close(self.st.g_full.cpu().numpy(), self.run.gfull, _abs_grad_scale(self.h, self.run.xsnap), rel=1e-6)
+        assert nbad == 0, ("g_full", nbad, worst)
+        self.st.z_snap.copy_(_dev(self.run.z_snap))
+
+    def round(self, rnd, eta, theta=0.0):
+        import torch
+        dq, cfg, st, run = self.dq, self.cfg, self.st, self.run
+        M, d, b = cfg.M, cfg.d, cfg.b
+        self.sync_state()
+        x_before = run.x.copy(); y_before = run.y.copy(); xsum_before = run.xsum.copy()
+        assert dq.dq_round(self.ctx, st, rnd, eta, theta, self.bits[0:1], self.bits[1:2]) == 0
+        tr = run.round(rnd, eta, theta, trace=True)
+        assert tr["status"] == 0 and dq.dq_poll_status(self.ctx) == (0, 0)
+        _, buf = dq.dq_round_buffers(self.ctx)
+        m = buf["msgs"]
+        # model codes: same x, so bit-exact
+        if not tr["flag_round"]:
+            nbx = dq.dq_packed_bytes(d, cfg.bx)
+            assert np.array_equal(dq.device_view(buf["codes_x"], nbx, torch.uint8).cpu().numpy(), oracle.pack(tr["codes_x"], cfg.bx, nbx))
+            assert dq.device_view(buf["delta_x"], 1, torch.float32).item() == tr["delta_x"][0]
+        a_gpu = dq.device_view(buf["alpha"], M * d, torch.float32).cpu().numpy().reshape(M, d)
+        scale = dq.device_view(m.scale, M, torch.float32).cpu().numpy()
+        codes_b = dq.device_view(m.codes, M * m.stride, torch.uint8).cpu().numpy().reshape(M, m.stride)
+        sparse = bool(cfg.sparsify) and cfg.msg_format == dq.DQ_MSG_SPARSE
+        raw_gpu = np.zeros((M, d), np.int32)
+        round_flips = 0
+        for w in range(M):
+            nbad, worst = _close(a_gpu[w], tr["alpha"][w], tr["S"][w])
+            self.worst_alpha = max(self.worst_alpha, worst)
+            assert nbad == 0, ("alpha", rnd, w, nbad, worst)
+            # the GPU's codes are exactly the oracle's quantiser applied to the GPU's gradient
+            if cfg.sparsify:
+                r = oracle.sparsify(a_gpu[w], cfg.phi, cfg.seed, rnd, w)
+                cw, dw, _ = oracle.quantize_survivors(r["beta"], r["Z"], b, cfg.seed, rnd, w)
+            else:
+                cw, dw, _ = oracle.quantize(a_gpu[w], b, cfg.seed, rnd, w, oracle.STREAM_GRAD)
+            assert scale[w] == dw, ("delta", rnd, w)
+            if sparse:
+                pos = np.nonzero(r["Z"])[0]
+                nnz = dq.device_view(m.nnz, M, torch.int32).cpu().numpy()
+                idx = dq.device_view(m.idx, M * m.cap, torch.int32).cpu().numpy().reshape(M, m.cap)
+                assert nnz[w] == pos.size and np.array_equal(idx[w, :pos.size], pos)
+                assert np.array_equal(codes_b[w], oracle.pack(cw[pos], b, m.stride))
+            else:
+                assert np.array_equal(codes_b[w], oracle.pack(cw, b, m.stride)), ("codes", rnd, w)
+            raw_gpu[w] = cw
+            # disagreements with the oracle's own codes
+            diff = np.nonzero(cw != tr["codes"][w])[0]
+            round_flips += diff.size; self.coords += d
+            if diff.size and not cfg.sparsify:
+                inv = oracle.scale_inv(np.abs(tr["alpha"][w]).max(), b)
+                for i in diff:
+                    t = float(tr["alpha"][w][i]) * float(inv)
+                    F = int(round((t + 128.0) * 32768.0))
+                    pos15 = (F + oracle.u15(cfg.seed, rnd, w, oracle.STREAM_GRAD, int(i))) & 0x7FFF
+                    steps = min(pos15, 32768 - pos15)
+                    if steps > 2 + 1e-6 * max(1.0, abs(t)) * 32768 or abs(int(cw[i]) - int(tr["codes"][w][i])) > 1:
+                        self.far_flips += 1
+        self.flips += round_flips
+        # master: bit-exact on the GPU's own codes
+        x = x_before.copy(); y = y_before.copy(); xs = xsum_before.copy()
+        nx = oracle.master_step(raw_gpu, scale, run.gfull, x, eta, theta, bool(cfg.accelerated), y, run.xsnap, xs,
+                                cfg.lambda1, cfg.lambda2, cfg.box_lo, cfg.box_hi)
+        assert np.array_equal(st.x.cpu().numpy(), x), ("x", rnd)
+        assert st.norm_x.item() == nx
+        if cfg.accelerated:
+            assert np.array_equal(st.y.cpu().numpy(), y) and np.array_equal(st.x_sum.cpu().numpy(), xs)
+        # and equal to the oracle's iterate wherever no code flipped
+        if np.array_equal(scale, tr["delta"]):
+            same = np.all(raw_gpu == tr["codes"], axis=0)
+            assert np.array_equal(x[same], run.x[same])
+        # transmitted bits
+        bits = self.bits.cpu().numpy()
+        assert int(bits[0]) == tr["bits_down"]
+        if not sparse or round_flips == 0:
+            assert int(bits[1]) == tr["bits_up"]
+        return tr
+
+    def close(self):
+        self.dq.dq_destroy(self.ctx)
+
+
+@pytest.mark.parametrize("name,kw,eta", [
+    ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=5), 0.5),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=6), 0.5),
+    ("bf16", dict(M=4, B=16, bx=8, b=8, box_lo=-1.0, box_hi=1.0, seed=7), 0.01),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, seed=8), 0.5),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=50.0, msg_format=1, seed=9), 0.5),
+])
+def test_lockstep_small(dq, name, kw, eta):
+    h = _problem(name)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 73, 0.05), **kw)
+    rnd = 0
+    for epoch in range(3):
+        ls.epoch()
+        for t in range(12):
+            tr = ls.round(rnd, eta)
+            assert tr["flag_round"] == (t == 0)
+            rnd += 1
+    assert ls.far_flips == 0 and ls.flips <= 1e-3 * ls.coords
+    ls.close()
+
+
+def test_lockstep_accelerated_small(dq):
+    h = _problem("bf16")
+    kw = dict(M=4, B=16, bx=8, b=8, box_lo=-0.5, box_hi=0.5, accelerated=1, seed=10)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 74, 0.05), **kw)
+    rnd = 0
+    for s in range(1, 4):
+        theta = F32(2.0 / (s + 2)); eta = F32(0.004) / theta                # Section 5.1 schedule
+        ls.epoch(theta)
+        for t in range(10):
+            tr = ls.round(rnd, eta, theta)
+            assert tr["flag_round"] == (s == 1 and t == 0)
+            rnd += 1
+    assert ls.far_flips == 0
+    ls.close()
+
+
+def _full_config(name):
+    if name == "c1":
+        return dict(M=4, B=16, bx=8, b=8, lambda1=1e-4, seed=101), 1.0, 200
+    if name == "c2":
+        return dict(M=8, B=64, bx=8, b=4, lambda2=1e-5, seed=102), 1.0, 50
+    if name == "c3":
+        return dict(M=16, B=128, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1, seed=103), 1.0, 5
+    if name == "c4":
+        return dict(M=32, B=256, bx=8, b=8, box_lo=-10.0, box_hi=10.0, accelerated=1, seed=104), 1e-4, 10
+
+
+@pytest.mark.parametrize("name,rounds", [("c1", 100), ("c2", 100), ("c3", 4), ("c4", 20)])
+def test_lockstep_full_configs(dq, name, rounds):
+    """The benchmark configurations at their full model width (c3, c4 with fewer rows so that the oracle
+    finishes in seconds); c4 reads "momentum 0.9" as theta = 0.1, eta = lr / theta."""
+    h = _problem(name)
+    kw, lr, m = _full_config(name)
+    ls = Lockstep(dq, h, np.zeros(h.d, F32) if name != "c4" else synth.normal_vector(h.d, 75, 0.01), **kw)
+    theta = F32(0.1) if name == "c4" else F32(0.0)
+    eta = F32(lr) / theta if name == "c4" else F32(lr)
+    for rnd in range(rounds):
+        if rnd % m == 0:
+            ls.epoch(theta)
+        ls.round(rnd, eta, theta)
+    print("\n[%s] flips %d of %d coordinate codes, %d beyond the threshold band, worst alpha error %.2e of tolerance scale"
+          % (name, ls.flips, ls.coords, ls.far_flips, ls.worst_alpha))
+    assert ls.far_flips == 0
+    ls.close()
+
+
+@pytest.mark.parametrize("name", ["c1", "c2"])
+def test_free_running_loss_trajectory(dq, name):
+    """Both sides run on their own for 100+ rounds; the objective must agree within 1e-4 relative throughout."""
+    import torch
+    h = _problem(name)
+    kw, lr, m = _full_config(name)
+    cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
+    rc, ctx = dq.dq_create(cfg, dq.Data(h)); assert rc == 0
+    x0 = np.zeros(h.d, F32)
+    st = dq.State(x0, n=h.n)
+    ocfg = oracle.make_config(h.d, kw["M"], kw["B"], kw["bx"], kw["b"], l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0), seed=kw["seed"])
+    run = oracle.Run(ocfg, _odata(h), x0)
+    P = torch.zeros(1, dtype=torch.float64, device="cuda")
+    first = last = None
+    rounds = 250 if name == "c1" else 120
+    for rnd in range(rounds):
+        if rnd % m == 0:
+            assert dq.dq_epoch_begin(ctx, st) == 0; run.epoch_begin()
+        assert dq.dq_round(ctx, st, rnd, lr) == 0; run.round(rnd, lr)
+        if rnd % 10 == 9:
+            assert dq.dq_objective(ctx, st.x, P) == 0
+            Po = oracle.objective(_odata(h), run.x, cfg.lambda1, cfg.lambda2)
+            assert abs(P.item() - Po) <= 1e-4 * max(abs(Po), 1e-3), (rnd, P.item(), Po)
+            first = first if first is not None else Po; last = Po
+    assert last < first                                                    # and it is optimising
+    assert dq.dq_poll_status(ctx) == (0, 0)
+    nbad, worst = _close(st.x.cpu().numpy(), run.x, rel=1e-3)
+    print("\n[%s] free-running: final objective %.6f, iterate mismatches beyond 1e-3: %d (worst %.2e)" % (name, last, nbad, worst))
+    dq.dq_destroy(ctx)
