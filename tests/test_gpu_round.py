@@ -89,7 +89,8 @@ def test_epoch_begin_full_gradient(dq, name):
     h = _problem(name)
     x0 = synth.normal_vector(h.d, 70, 0.3)
     cfg = dq.make_config(h.d, 3, B=4, seed=1)
-    rc, ctx = dq.dq_create(cfg, dq.Data(h)); assert rc == 0
+    data = dq.Data(h)                                     # must outlive the context
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
     st = dq.State(x0, n=h.n)
     st.x_snap.zero_()
     assert dq.dq_epoch_begin(ctx, st) == 0
@@ -102,7 +103,7 @@ def test_epoch_begin_full_gradient(dq, name):
     P = torch.zeros(1, dtype=torch.float64, device="cuda")
     assert dq.dq_objective(ctx, st.x, P) == 0
     cfg2 = dq.make_config(h.d, 3, B=4, seed=1, lambda1=0.01, lambda2=0.1)
-    rc, ctx2 = dq.dq_create(cfg2, dq.Data(h)); assert rc == 0
+    rc, ctx2 = dq.dq_create(cfg2, data); assert rc == 0
     P2 = torch.zeros(1, dtype=torch.float64, device="cuda")
     assert dq.dq_objective(ctx2, st.x, P2) == 0
     assert abs(P.item() - oracle.objective(_odata(h), x0, 0, 0)) < 1e-7
@@ -119,7 +120,8 @@ def test_worker_gradient(dq, name, bx):
     xs = synth.normal_vector(h.d, 71, 0.3)
     x = (xs + synth.normal_vector(h.d, 72, 0.02)).astype(F32)
     cfg = dq.make_config(h.d, M, B=B, bx=bx, seed=seed)
-    rc, ctx = dq.dq_create(cfg, dq.Data(h)); assert rc == 0
+    data = dq.Data(h)                                     # must outlive the context
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
     st = dq.State(xs, n=h.n)
     assert dq.dq_epoch_begin(ctx, st) == 0
     cx, dx, _ = oracle.quantize(x, bx, seed, rnd, oracle.MASTER, oracle.STREAM_MODEL)
@@ -334,7 +336,8 @@ def test_free_running_loss_trajectory(dq, name):
     h = _problem(name)
     kw, lr, m = _full_config(name)
     cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
-    rc, ctx = dq.dq_create(cfg, dq.Data(h)); assert rc == 0
+    data = dq.Data(h)                                     # must outlive the context
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
     x0 = np.zeros(h.d, F32)
     st = dq.State(x0, n=h.n)
     ocfg = oracle.make_config(h.d, kw["M"], kw["B"], kw["bx"], kw["b"], l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0), seed=kw["seed"])
