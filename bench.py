@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the double-quantization round on B200.
+
+Default workload ("c5"): the quantiser/packer bandwidth configuration -- M = 8 worker gradient vectors of
+d = 2^27 fp32 coordinates (N(0,1) with 0.1 % outliers x100), quantised to b = 4 bits and packed, aggregated
+and prox-updated by the master, and the new model requantised to b_x = 8 bits.  One "step" is one such
+round: ||v||_inf pass, quantise+pack, master unpack+aggregate+prox, model norm is fused, model quantise.
+Prints ONE JSON line (see README / DESIGN for the keys).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--log2d 27] [--bits 4]
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the workload (the
+path is single-GPU by definition; there is no exchange step) and the value is the sum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import re
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "simulated-worker rounds/sec"
+UNIT = "rounds/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--log2d", type=int, default=27)
+    ap.add_argument("--bits", type=int, default=4)
+    ap.add_argument("--workers", type=int, default=8)
+    ap.add_argument("--sparsify", type=int, default=0)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def workload_config(a):
+    d = 1 << a.log2d
+    return {"workload": "c5 quantiser/packer sweep point: d=2^%d, M=%d, b=%d, b_x=8, sparsify=%s, lambda1=1e-6, eta=0.1"
+                        % (a.log2d, a.workers, a.bits, "on(phi=0.01d)" if a.sparsify else "off"),
+            "d": d, "M": a.workers, "b": a.bits, "bx": 8, "sparsify": a.sparsify,
+            "l2_policy": "inputs larger than L2 (%.0f MiB per round)" % (a.workers * d * 4 / 2 ** 20)}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline of the main line, and the whole of --impl reference)
+# ---------------------------------------------------------------------------------------------------------------
+def oracle_rounds_per_sec(a, steps, warmup, log2_sample=22):
+    """Times the oracle's codec round on a d = 2^log2_sample slice of the workload; work is linear in d, so
+    the rate is scaled by 2^log2_sample / d.  Returns (scaled rounds/s, seconds per sampled round, description)."""
+    import numpy as np
+    import oracle
+    from paper_1805_10111_b200 import synth
+    ds = 1 << min(log2_sample, a.log2d)
+    M, b = a.workers, a.bits
+    v, x, g = synth.config5(ds, M)
+    x = x.copy()
+    times = []
+    for rnd in range(warmup + steps):
+        t0 = time.perf_counter()
+        raw = np.zeros((M, ds), np.int32); delta = np.zeros(M, np.float32)
+        for w in range(M):
+            if a.sparsify:
+                r = oracle.sparsify(v[w], 0.01 * ds, 1805, rnd, w)
+                raw[w], delta[w], _ = oracle.quantize_survivors(r["beta"], r["Z"], b, 1805, rnd, w)
+            else:
+                raw[w], delta[w], _ = oracle.quantize(v[w], b, 1805, rnd, w, oracle.STREAM_GRAD)
+        oracle.master_step(raw, delta, g, x, 0.1, l1=1e-6)
+        oracle.quantize(x, 8, 1805, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+        if rnd >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = sum(times) / len(times)
+    scaled = (1.0 / sec) * ds / (1 << a.log2d)
+    return scaled, sec, "oracle codec round on a d=2^%d slice (%d rounds, single thread), rate scaled by d" % (min(log2_sample, a.log2d), steps)
+
+
+def run_reference(a):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(a.steps, 8)); warm = max(0, min(a.warmup, 1))
+    val, sec, what = oracle_rounds_per_sec(a, steps, warm)
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": a.gpus, "steps": a.steps,
+            "warmup": a.warmup, "ms_per_step": 1000.0 / val, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(a),
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# helpers
+# ---------------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill(); out, _ = self.proc.communicate()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.strip().splitlines():
+            p = [t.strip() for t in ln.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0])); smax.append(float(p[1])); power.append(float(p[2]))
+            except ValueError:
+                continue
+            for nm, flag in zip(names, p[3:7]):
+                if flag.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(smax), "power_w_max": max(power), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def kernel_source_hash():
+    h = hashlib.sha256()
+    for f in ("dq_codec.cu", "dq_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_1805_10111_b200", "csrc", f), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(bits):
+    """DRAM bytes per coordinate of quantize_pack_kernel from the committed ncu summary, or None if the kernel
+    source has changed since that capture."""
+    p = os.path.join(ROOT, "profiles", "quantize_pack_kernel_c5.md")
+    if not os.path.exists(p):
+        return None
+    t = open(p).read()
+    m = re.search(r"source_sha256_16:\s*([0-9a-f]{16})", t)
+    k = re.search(r"dram_bytes_per_coordinate_b%d:\s*([0-9.]+)" % bits, t)
+    if not m or not k or m.group(1) != kernel_source_hash():
+        return None
+    return float(k.group(1))
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# GPU leg
+# ---------------------------------------------------------------------------------------------------------------
+def run_ours(a):
+    import numpy as np
+    import torch
+    import paper_1805_10111_b200 as dq
+    from paper_1805_10111_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0")); world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dq.lib()
+
+    d, M, b, bx, eta, seed = 1 << a.log2d, a.workers, a.bits, 8, 0.1, 1805
+    cfg = dq.make_config(d, M, b=b, bx=bx, seed=seed, lambda1=1e-6, sparsify=a.sparsify, phi=0.01 * d if a.sparsify else 0.0)
+    rc, ctx = dq.dq_create(cfg); dq.ok(rc, "dq_create")
+
+    # seeded synthetic inputs, generated on the host straight into pinned memory (also the e2e source)
+    hv = torch.empty((M, d), dtype=torch.float32).pin_memory()
+    g = synth.rng(5 + 100 * rank)
+    hv_np = hv.numpy()
+    for w in range(M):
+        row = hv_np[w]
+        g.standard_normal(d, dtype=np.float32, out=row)
+        row[g.integers(0, d, max(1, d // 1000))] *= np.float32(100.0)
+    x0 = synth.normal_vector(d, 6); gf = synth.normal_vector(d, 7)
+    v = hv.cuda(non_blocking=False)
+    st = dq.State(x0); st.g_full.copy_(torch.from_numpy(gf).cuda())
+    msgs = dq.Msgs(cfg)
+    ninf = torch.zeros(M, device="cuda")
+    nbx = dq.dq_packed_bytes(d, bx)
+    codes_x = torch.zeros(nbx, dtype=torch.uint8, device="cuda"); delta_x = torch.zeros(1, device="cuda")
+
+    def step(rnd, ev=None):
+        if ev: ev[0].record()
+        dq.ok(dq.dq_norm_inf(ctx, v, M, ninf))
+        if ev: ev[1].record()
+        dq.ok(dq.dq_quantize_sparsify_pack(ctx, v, ninf, rnd, msgs))
+        if ev: ev[2].record()
+        dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta))
+        if ev: ev[3].record()
+        dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, rnd, codes_x, delta_x))
+        if ev: ev[4].record()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for rnd in range(max(3, a.warmup)):
+        step(rnd)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(a.steps)]
+    barrier()
+    sampler = ClockSampler(local)
+    launches0 = dq.dq_launch_count(ctx)
+    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for k in range(a.steps):
+        step(1000 + k, events[k])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop()
+    launches = dq.dq_launch_count(ctx) - launches0
+    total_ms = t_begin.elapsed_time(t_end)
+    rc, status = dq.dq_poll_status(ctx)
+    assert rc == 0 and status == 0, "device status %d" % status
+    stage_ms = [sum(events[k][i].elapsed_time(events[k][i + 1]) for k in range(a.steps)) / a.steps for i in range(4)]
+    if dist is not None:
+        t = torch.tensor([total_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); total_ms = t.item()
+    ms_per_step = total_ms / a.steps
+    value = world * a.steps / (total_ms / 1000.0)
+
+    # end to end through the host-buffer entry point: H2D of the M gradient vectors, the round, D2H of the model codes
+    e2e = None
+    if a.e2e_steps > 0:
+        dq.ok(dq.dq_codec_host_setup(ctx, x0, gf))
+        hcodes = torch.zeros(nbx, dtype=torch.uint8).pin_memory(); hdelta = torch.zeros(1).pin_memory()
+        dq.ok(dq.dq_codec_round_host(ctx, hv, 0, eta, hcodes, hdelta))
+        barrier()
+        t0 = time.perf_counter()
+        for k in range(a.e2e_steps):
+            dq.ok(dq.dq_codec_round_host(ctx, hv, 2000 + k, eta, hcodes, hdelta))
+        torch.cuda.synchronize()
+        e2e_s = time.perf_counter() - t0
+        if dist is not None:
+            t = torch.tensor([e2e_s], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_s = t.item()
+        e2e = {"value": world * a.e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": M * d * 4,
+               "d2h_bytes_per_step": nbx + 4, "steps": a.e2e_steps}
+
+    if rank != 0:
+        dq.dq_destroy(ctx)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peak, peak_src = measured_peak()
+    # algorithmic bytes per launch ("bytes per unit"): norm 4 B, quantise+pack 4 + b/8 B per message
+    # coordinate; master M*b/8 + 12 B, model quantise 4 + b_x/8 B per model coordinate.
+    alg = [M * d * 4.0, M * d * (4.0 + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
+    names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
+    stages = {n: {"ms": round(ms, 4), "alg_GBps": round(by / ms / 1e6, 1), "frac_of_peak": round(by / ms / 1e6 / peak, 4)}
+              for n, ms, by in zip(names, stage_ms, alg)}
+    qp = stages["quantize_pack"]
+    tr = recorded_traffic(b) if not a.sparsify else None
+    roofline = {"kernel": "quantize_pack_kernel<%d>" % b if not a.sparsify else "sparsify (l1 + count + emit)",
+                "bound": "hbm", "achieved": qp["alg_GBps"], "peak": peak, "unit": "GB/s",
+                "frac": round(qp["alg_GBps"] / peak, 4), "peak_source": peak_src,
+                "traffic": None if tr is None else tr * M * d,
+                "alg_bytes_per_launch": alg[1]}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(3, a.warmup),
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": workload_config(a), "roofline": roofline,
+            "stages": stages, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "bits_per_round": {"down": M * (32 + bx * d), "up_dense": M * (32 + b * d), "full_precision": 2 * M * 32 * d}}
+    if world == 1 and not a.no_cpu_baseline:
+        val, sec, what = oracle_rounds_per_sec(a, steps=6, warmup=1)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
+    dq.dq_destroy(ctx)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)
+
+
+if __name__ == "__main__":
+    main()

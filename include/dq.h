@@ -132,6 +132,10 @@ int dq_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, in
                    const dq_state* st, uint32_t round, const int32_t* batch_idx,
                    float* alpha, float* norm_inf, void* stream);
 
+/* ||v_w||_inf for the M rows of v [M][d] into norm_inf [M] (device floats): the numerator of the scale
+ * delta of Algorithm 1 steps 8 and 12, for callers whose gradient producer does not supply it. */
+int dq_norm_inf(dq_ctx* ctx, const float* v, int M, float* norm_inf, void* stream);
+
 /* Worker steps 12(-13) for all M workers: optional sparsification by eq. (4) with Lemma 2's probabilities,
  * then delta = ||.||_inf / (2^(b-1)-1), Q_(delta,b), and bit packing into `out`.
  * v [M][d]; norm_inf [M] = ||v_w||_inf as produced by dq_worker_grad, or NULL to have it computed. */

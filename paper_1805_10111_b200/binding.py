@@ -17,7 +17,7 @@ DQ_DENSE_F32, DQ_CSR_F32, DQ_DENSE_BF16 = 0, 1, 2
 DQ_MSG_DENSE, DQ_MSG_SPARSE = 0, 1
 
 EXPORTS = ["dq_packed_bytes", "dq_create", "dq_destroy", "dq_epoch_begin", "dq_quantize_model", "dq_worker_grad",
-           "dq_quantize_sparsify_pack", "dq_master_unpack_aggregate_prox", "dq_round", "dq_codec_round",
+           "dq_norm_inf", "dq_quantize_sparsify_pack", "dq_master_unpack_aggregate_prox", "dq_round", "dq_codec_round",
            "dq_codec_host_setup", "dq_codec_round_host", "dq_unpack", "dq_objective", "dq_round_buffers",
            "dq_poll_status", "dq_launch_count", "dq_strerror"]
 
@@ -68,6 +68,7 @@ def lib():
             "dq_epoch_begin": (i32, [vp, C.POINTER(dq_state), f32, vp]),
             "dq_quantize_model": (i32, [vp, vp, vp, u32, vp, vp, vp]),
             "dq_worker_grad": (i32, [vp, vp, vp, i32, C.POINTER(dq_state), u32, vp, vp, vp, vp]),
+            "dq_norm_inf": (i32, [vp, vp, i32, vp, vp]),
             "dq_quantize_sparsify_pack": (i32, [vp, vp, vp, u32, C.POINTER(dq_msgs), vp]),
             "dq_master_unpack_aggregate_prox": (i32, [vp, C.POINTER(dq_msgs), C.POINTER(dq_state), f32, f32, vp]),
             "dq_round": (i32, [vp, C.POINTER(dq_state), u32, f32, f32, vp, vp, vp]),
@@ -191,6 +192,10 @@ def dq_quantize_model(ctx, x, norm_x, round_, codes_x, delta_x, stream=None):
 def dq_worker_grad(ctx, codes_x, delta_x, is_snapshot, st: State, round_, batch_idx, alpha, norm_inf, stream=None):
     return lib().dq_worker_grad(ctx, _ptr(codes_x), _ptr(delta_x), int(is_snapshot), C.byref(st.c), int(round_),
                                 _ptr(batch_idx), _ptr(alpha), _ptr(norm_inf), _stream(stream))
+
+
+def dq_norm_inf(ctx, v, M, norm_inf, stream=None):
+    return lib().dq_norm_inf(ctx, _ptr(v), int(M), _ptr(norm_inf), _stream(stream))
 
 
 def dq_quantize_sparsify_pack(ctx, v, norm_inf, round_, out: Msgs, stream=None):

@@ -158,6 +158,13 @@ int dq_quantize_model(dq_ctx* ctx, const float* x, const float* norm_x, uint32_t
     return last_error();
 }
 
+int dq_norm_inf(dq_ctx* ctx, const float* v, int M, float* norm_inf, void* stream)
+{
+    if (!ctx || !v || !norm_inf || M < 1 || !aligned(v, 4)) return DQ_ERR_ARG;
+    launch_norm_inf(ctx, v, ctx->cfg.d, M, reinterpret_cast<uint32_t*>(norm_inf), as_stream(stream));
+    return last_error();
+}
+
 int dq_quantize_sparsify_pack(dq_ctx* ctx, const float* v, const float* norm_inf, uint32_t round, dq_msgs* out, void* stream)
 {
     if (!ctx || !v) return DQ_ERR_ARG;
