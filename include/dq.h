@@ -171,6 +171,26 @@ int dq_codec_host_setup(dq_ctx* ctx, const float* x_host, const float* g_full_ho
 int dq_codec_round_host(dq_ctx* ctx, const float* v_host, uint32_t round, float eta,
                         uint8_t* codes_x_host, float* delta_x_host, void* stream);
 
+/* Dense quantise + pack WITHOUT a context and without any allocation.  The paper has no counterpart: this
+ * entry point exists for callers that must not allocate device memory at the time of the call -- code running
+ * inside another framework's memory pool or allocator callback, a process whose device memory is fully
+ * budgeted up front, or a plug-in that is handed buffers and a stream and nothing else.  dq_create would call
+ * cudaMalloc for its scratch; here the only scratch the dense path needs (one norm word per message) lives in
+ * a fixed device array inside the library, which every GPU that loads the library holds until exit (about
+ * 4 KiB).  It computes exactly what dq_quantize_sparsify_pack computes for sparsify = 0 with the same
+ * (seed, round): v [M][d] -> codes [M][stride] packed b-bit codes and scale [M] = delta.
+ *   - M may not exceed DQ_STATIC_MAX_MESSAGES; larger M returns DQ_ERR_SHAPE.  b must be 2, 4 or 8
+ *     (DQ_ERR_BITS); stride >= dq_packed_bytes(d, b) and a multiple of 16; codes 16-byte aligned.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
+ *     device current; make that first call outside any stream capture.  No call allocates or frees.
+ *   - All calls on a device share the one array, which still holds the previous call's norms; each call
+ *     clears what it needs on `stream` first.  Two calls whose GPU work overlaps (different streams, or
+ *     different threads) race on it: serialise them.
+ *   - A non-finite vector gets scale 0 and all-zero codes; there is no status word to poll. */
+#define DQ_STATIC_MAX_MESSAGES 1024
+int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, uint64_t seed, uint32_t round,
+                            uint8_t* codes, int64_t stride, float* scale, void* stream);
+
 /* Test utility: dequantise message w of `msgs` into out [d] (zeros where a sparse message has no entry). */
 int dq_unpack(dq_ctx* ctx, const dq_msgs* msgs, int w, float* out, void* stream);
 

@@ -19,7 +19,7 @@ DQ_MSG_DENSE, DQ_MSG_SPARSE = 0, 1
 EXPORTS = ["dq_packed_bytes", "dq_create", "dq_destroy", "dq_epoch_begin", "dq_quantize_model", "dq_worker_grad",
            "dq_norm_inf", "dq_quantize_sparsify_pack", "dq_master_unpack_aggregate_prox", "dq_round", "dq_codec_round",
            "dq_codec_host_setup", "dq_codec_round_host", "dq_unpack", "dq_objective", "dq_round_buffers",
-           "dq_poll_status", "dq_launch_count", "dq_strerror"]
+           "dq_poll_status", "dq_launch_count", "dq_strerror", "dq_quantize_pack_static"]
 
 
 class dq_data(C.Structure):
@@ -81,6 +81,7 @@ def lib():
             "dq_poll_status": (i32, [vp, C.POINTER(C.c_int), vp]),
             "dq_launch_count": (i64, [vp]),
             "dq_strerror": (C.c_char_p, [i32]),
+            "dq_quantize_pack_static": (i32, [vp, i64, i32, i32, C.c_uint64, u32, vp, i64, vp, vp]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
@@ -251,6 +252,12 @@ def dq_poll_status(ctx, stream=None):
 
 def dq_launch_count(ctx):
     return int(lib().dq_launch_count(ctx))
+
+
+def dq_quantize_pack_static(v, d, M, b, seed, round_, codes, stride, scale, stream=None):
+    """Context-free dense quantise + pack that allocates nothing (scratch is a fixed array inside the library)."""
+    return lib().dq_quantize_pack_static(_ptr(v), int(d), int(M), int(b), int(seed), int(round_), _ptr(codes), int(stride),
+                                         _ptr(scale), _stream(stream))
 
 
 def ok(rc, where=""):

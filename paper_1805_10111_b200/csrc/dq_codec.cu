@@ -596,3 +596,67 @@ void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, fl
 }
 
 }  // namespace dq
+
+// ---------------------------------------------------------------------------------------------------
+// dq_quantize_pack_static: dense quantise + pack for callers that cannot allocate device memory.
+// The per-message norm words that the other entry points keep in a context's scratch live here in a
+// file-scope device array instead.  Host code must not hand the array's name to a kernel (on the
+// host that name is only a handle); the device address is looked up once per device below.
+// ---------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxMessages = DQ_STATIC_MAX_MESSAGES;
+constexpr int kStaticMaxDevices = 64;
+
+// [0, kStaticMaxMessages): ||v_w||_inf bit patterns; [kStaticMaxMessages]: non-finite flag of the last call.
+static __device__ __align__(256) uint32_t g_static_scratch[kStaticMaxMessages + 64];
+
+struct StaticSlot { uint32_t* ptr; int sm_count; bool ready; };
+StaticSlot g_static_slot[kStaticMaxDevices];
+
+// Looks up the device address of the scratch array for the current device (first call on that device).
+int static_scratch_for_current_device(uint32_t** ptr, int* sm_count)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return DQ_ERR_CUDA;
+    StaticSlot& s = g_static_slot[dev];
+    if (!s.ready) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) { cudaGetLastError(); return DQ_ERR_CUDA; }
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return DQ_ERR_CUDA;
+        s.ptr = static_cast<uint32_t*>(p); s.sm_count = sms; s.ready = true;
+    }
+    *ptr = s.ptr; *sm_count = s.sm_count;
+    return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, uint64_t seed, uint32_t round,
+                                       uint8_t* codes, int64_t stride, float* scale, void* stream)
+{
+    using namespace dq;
+    if (!v || !codes || !scale || d < 1 || M < 1) return DQ_ERR_ARG;
+    if (b != 2 && b != 4 && b != 8) return DQ_ERR_BITS;
+    if (M > kStaticMaxMessages) return DQ_ERR_SHAPE;                       // beyond the fixed scratch
+    if (d > ((int64_t)1 << 32)) return DQ_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(codes) & 15) || (stride & 15) || (reinterpret_cast<uintptr_t>(v) & 3)) return DQ_ERR_ARG;
+    if (stride < dq_packed_bytes(d, b)) return DQ_ERR_SHAPE;
+    uint32_t* scratch = nullptr; int sms = 0;
+    int rc = static_scratch_for_current_device(&scratch, &sms);
+    if (rc != DQ_OK) return rc;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    // the array keeps the previous call's norms: the maxima must start from zero again
+    if (cudaMemsetAsync(scratch, 0, sizeof(uint32_t) * (kStaticMaxMessages + 1), st) != cudaSuccess) return DQ_ERR_CUDA;
+    const int vec_ok = vec_ok_for(v, d);
+    dim3 grid_n(grid_for((d + 7) / 8, sms), M);
+    norm_inf_kernel<<<grid_n, kThreads, 0, st>>>(v, d, vec_ok, scratch);
+    const int64_t ngroups = dq_packed_bytes(d, b) / b;
+    dim3 grid_q(grid_for(ngroups, sms), M);
+    const PhiloxKeys keys = expand_keys(seed);
+    int* flag = reinterpret_cast<int*>(scratch + kStaticMaxMessages);
+    DQ_DISPATCH_BITS(b, (quantize_pack_kernel<BITS_><<<grid_q, kThreads, 0, st>>>(
+        v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag)));
+    return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+}
