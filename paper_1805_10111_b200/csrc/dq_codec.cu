@@ -347,13 +347,42 @@ __device__ __forceinline__ float master_update(float acc, float inv_m, float eta
     return x;
 }
 
+// acc[j] = fma(code_j, delta, acc[j]) for the 32/BITS codes of one packed word.  The integer-to-float
+// conversion avoids the conversion pipe: the code, biased by 2^(BITS-1), is placed in the mantissa of 2^23
+// (one byte permute) and the bias is subtracted exactly.
+template <int BITS>
+__device__ __forceinline__ void accumulate_word(uint32_t word, float dl, float (&acc)[32 / BITS])
+{
+    constexpr float kBias = 8388608.0f + (float)(1 << (BITS - 1));
+    if (BITS == 8) {
+        const uint32_t wb = word ^ 0x80808080u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            acc[j] = __fmaf_rn(__fsub_rn(__uint_as_float(__byte_perm(wb, 0x4B000000u, 0x7540u | j)), kBias), dl, acc[j]);
+    } else if (BITS == 4) {
+        const uint32_t wb = word ^ 0x88888888u;
+        const uint32_t ev = wb & 0x0F0F0F0Fu, od = (wb >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            acc[j] = __fmaf_rn(__fsub_rn(__uint_as_float(__byte_perm((j & 1) ? od : ev, 0x4B000000u, 0x7540u | (j >> 1))), kBias), dl, acc[j]);
+    } else {
+        const uint32_t wb = word ^ 0xAAAAAAAAu;
+        uint32_t p[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) p[k] = (wb >> (2 * k)) & 0x03030303u;
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+            acc[j] = __fmaf_rn(__fsub_rn(__uint_as_float(__byte_perm(p[j & 3], 0x4B000000u, 0x7540u | (j >> 2))), kBias), dl, acc[j]);
+    }
+}
+
 // Dense messages.  Each thread owns the 32/BITS coordinates of one 32-bit code word per worker.
 template <int BITS, bool ACC>
 __global__ void __launch_bounds__(kThreads)
 master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
                     const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
-                    uint32_t* __restrict__ normx_bits)
+                    int vec8_ok, uint32_t* __restrict__ normx_bits)
 {
     constexpr int C = 32 / BITS;
     extern __shared__ float s_scale[];
@@ -370,16 +399,41 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
         float acc[C];
 #pragma unroll
         for (int j = 0; j < C; ++j) acc[j] = 0.0f;
-#pragma unroll 4
-        for (int w = 0; w < M; ++w) {
-            const uint32_t word = __ldg(words + (int64_t)w * wstride + t);
-            const float dl = s_scale[w];
-#pragma unroll
-            for (int j = 0; j < C; ++j) acc[j] = __fmaf_rn((float)code_of<BITS>(word, j), dl, acc[j]);
-        }
         const int64_t i0 = t * C;
+        const bool fast = C >= 8 && vec8_ok && i0 + C <= d;
+        float gfp[C >= 8 ? C : 8], curp[C >= 8 ? C : 8];     // issued before the code words so that all loads overlap
+        if (fast) {
+#pragma unroll
+            for (int q = 0; q < C / 8; ++q) {
+                load8(g_full + i0 + q * 8, *reinterpret_cast<float(*)[8]>(gfp + q * 8));
+                load8_rw((ACC ? y : x) + i0 + q * 8, *reinterpret_cast<float(*)[8]>(curp + q * 8));
+            }
+        }
+        for (int w0 = 0; w0 < M; w0 += 8) {                 // eight code words in flight per thread
+            uint32_t wd[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) wd[k] = (w0 + k < M) ? __ldg(words + (int64_t)(w0 + k) * wstride + t) : 0u;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (w0 + k < M) accumulate_word<BITS>(wd[k], s_scale[w0 + k], acc);
+        }
         float* target = ACC ? y : x;
-        if (i0 + C <= d) {
+        if (fast) {                                          // 256-bit accesses: every 32-byte sector is used whole
+#pragma unroll
+            for (int q = 0; q < C / 8; ++q) {
+                const int64_t i = i0 + q * 8;
+                float xs[8], sm[8], yo[8], xo[8];
+                const float* gf = gfp + q * 8; const float* cur = curp + q * 8;
+                if (ACC) { load8(xsnap + i, xs); load8_rw(xsum + i, sm); }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (!ACC) { xs[j] = 0.0f; sm[j] = 0.0f; }
+                    xo[j] = master_update<ACC>(acc[q * 8 + j], inv_m, eta, theta, thr, den, pp, gf[j], cur[j], xs[j], yo[j], sm[j]);
+                    nmax = max(nmax, __float_as_uint(xo[j]) & 0x7FFFFFFFu);
+                }
+                store8(x + i, xo);
+                if (ACC) { store8(y + i, yo); store8(xsum + i, sm); }
+            }
+        } else if (i0 + C <= d) {
 #pragma unroll
             for (int q = 0; q < C / 4; ++q) {
                 const int64_t i = i0 + q * 4;
@@ -555,12 +609,14 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         const int64_t nwords = (d + (32 / c.b) - 1) / (32 / c.b);
         const int grid = grid_for(nwords, ctx->sm_count);
         const size_t smem = sizeof(float) * c.M;
+        auto al32 = [](const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 31) == 0; };
+        const int vec8_ok = al32(s->x) && al32(s->g_full) && al32(s->y) && al32(s->x_snap) && al32(s->x_sum);
         if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx)));
         } else {
             DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx)));
         }
         ctx->launches += 1;
     } else {

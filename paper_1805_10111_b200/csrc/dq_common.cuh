@@ -102,6 +102,19 @@ __device__ __forceinline__ void load8(const float* p, float (&v)[8])
                  : "l"(p));
 }
 
+// Eight consecutive floats of a buffer that the same kernel also writes (no read-only path), and the store.
+__device__ __forceinline__ void load8_rw(const float* p, float (&v)[8])
+{
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p) : "memory");
+}
+__device__ __forceinline__ void store8(float* p, const float (&v)[8])
+{
+    asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 :: "l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+
 // Eight floats starting at coordinate i0 of a row of length d, zero beyond the end; any alignment.
 __device__ __forceinline__ void load8_guarded(const float* row, int64_t i0, int64_t d, float (&v)[8])
 {
