@@ -378,13 +378,15 @@ __device__ __forceinline__ void accumulate_word(uint32_t word, float dl, float (
 
 // Dense messages.  Each thread owns the 32/BITS coordinates of one 32-bit code word per worker.
 template <int BITS, bool ACC>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, BITS == 2 ? 3 : 4)
 master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
                     const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
                     int vec8_ok, uint32_t* __restrict__ normx_bits)
 {
-    constexpr int C = 32 / BITS;
+    constexpr int W = (BITS == 8) ? 2 : 1;                  // code words per worker and thread
+    constexpr int CW = 32 / BITS;                           // coordinates per code word
+    constexpr int C = W * CW;                               // coordinates per thread: 8, 8, 16 for 8, 4, 2 bits
     extern __shared__ float s_scale[];
     for (int i = threadIdx.x; i < M; i += blockDim.x) s_scale[i] = scale[i];
     __syncthreads();
@@ -396,9 +398,9 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
     uint32_t nmax = 0;
     const int64_t nth = (int64_t)gridDim.x * blockDim.x;
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nwords; t += nth) {
-        float acc[C];
+        float acc[W][CW];
 #pragma unroll
-        for (int j = 0; j < C; ++j) acc[j] = 0.0f;
+        for (int j = 0; j < C; ++j) acc[j / CW][j % CW] = 0.0f;
         const int64_t i0 = t * C;
         const bool fast = C >= 8 && vec8_ok && i0 + C <= d;
         float gfp[C >= 8 ? C : 8], curp[C >= 8 ? C : 8];     // issued before the code words so that all loads overlap
@@ -410,11 +412,21 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
             }
         }
         for (int w0 = 0; w0 < M; w0 += 8) {                 // eight code words in flight per thread
-            uint32_t wd[8];
+            uint32_t wd[8][W];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) wd[k] = (w0 + k < M) ? __ldg(words + (int64_t)(w0 + k) * wstride + t) : 0u;
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t* wp = words + (int64_t)min(w0 + k, M - 1) * wstride;    // clamped: always a valid row
+                if (W == 2) { const uint2 u = __ldg(reinterpret_cast<const uint2*>(wp) + t); wd[k][0] = u.x; wd[k][W - 1] = u.y; }
+                else wd[k][0] = __ldg(wp + t);
+            }
 #pragma unroll
-            for (int k = 0; k < 8; ++k) if (w0 + k < M) accumulate_word<BITS>(wd[k], s_scale[w0 + k], acc);
+            for (int k = 0; k < 8; ++k) {
+                if (w0 + k < M) {
+#pragma unroll
+                    for (int q = 0; q < W; ++q)
+                        accumulate_word<BITS>(wd[k][q], s_scale[w0 + k], acc[q]);
+                }
+            }
         }
         float* target = ACC ? y : x;
         if (fast) {                                          // 256-bit accesses: every 32-byte sector is used whole
@@ -427,7 +439,7 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     if (!ACC) { xs[j] = 0.0f; sm[j] = 0.0f; }
-                    xo[j] = master_update<ACC>(acc[q * 8 + j], inv_m, eta, theta, thr, den, pp, gf[j], cur[j], xs[j], yo[j], sm[j]);
+                    xo[j] = master_update<ACC>(acc[(q * 8 + j) / CW][(q * 8 + j) % CW], inv_m, eta, theta, thr, den, pp, gf[j], cur[j], xs[j], yo[j], sm[j]);
                     nmax = max(nmax, __float_as_uint(xo[j]) & 0x7FFFFFFFu);
                 }
                 store8(x + i, xo);
@@ -441,20 +453,22 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
                 const float4 cur = *reinterpret_cast<const float4*>(target + i);
                 float4 xs = make_float4(0, 0, 0, 0), sm = make_float4(0, 0, 0, 0), yo, xo;
                 if (ACC) { xs = *reinterpret_cast<const float4*>(xsnap + i); sm = *reinterpret_cast<const float4*>(xsum + i); }
-                xo.x = master_update<ACC>(acc[q * 4 + 0], inv_m, eta, theta, thr, den, pp, gf.x, cur.x, xs.x, yo.x, sm.x);
-                xo.y = master_update<ACC>(acc[q * 4 + 1], inv_m, eta, theta, thr, den, pp, gf.y, cur.y, xs.y, yo.y, sm.y);
-                xo.z = master_update<ACC>(acc[q * 4 + 2], inv_m, eta, theta, thr, den, pp, gf.z, cur.z, xs.z, yo.z, sm.z);
-                xo.w = master_update<ACC>(acc[q * 4 + 3], inv_m, eta, theta, thr, den, pp, gf.w, cur.w, xs.w, yo.w, sm.w);
+                xo.x = master_update<ACC>(acc[(q * 4 + 0) / CW][(q * 4 + 0) % CW], inv_m, eta, theta, thr, den, pp, gf.x, cur.x, xs.x, yo.x, sm.x);
+                xo.y = master_update<ACC>(acc[(q * 4 + 1) / CW][(q * 4 + 1) % CW], inv_m, eta, theta, thr, den, pp, gf.y, cur.y, xs.y, yo.y, sm.y);
+                xo.z = master_update<ACC>(acc[(q * 4 + 2) / CW][(q * 4 + 2) % CW], inv_m, eta, theta, thr, den, pp, gf.z, cur.z, xs.z, yo.z, sm.z);
+                xo.w = master_update<ACC>(acc[(q * 4 + 3) / CW][(q * 4 + 3) % CW], inv_m, eta, theta, thr, den, pp, gf.w, cur.w, xs.w, yo.w, sm.w);
                 *reinterpret_cast<float4*>(x + i) = xo;
                 if (ACC) { *reinterpret_cast<float4*>(y + i) = yo; *reinterpret_cast<float4*>(xsum + i) = sm; }
                 nmax = max(nmax, max(max(__float_as_uint(xo.x) & 0x7FFFFFFFu, __float_as_uint(xo.y) & 0x7FFFFFFFu),
                                      max(__float_as_uint(xo.z) & 0x7FFFFFFFu, __float_as_uint(xo.w) & 0x7FFFFFFFu)));
             }
         } else {
-            for (int j = 0; j < C && i0 + j < d; ++j) {
+#pragma unroll
+            for (int j = 0; j < C; ++j) {
                 const int64_t i = i0 + j;
+                if (i >= d) break;
                 float yo = 0.0f, sm = ACC ? xsum[i] : 0.0f;
-                const float xo = master_update<ACC>(acc[j], inv_m, eta, theta, thr, den, pp, g_full[i], target[i],
+                const float xo = master_update<ACC>(acc[j / CW][j % CW], inv_m, eta, theta, thr, den, pp, g_full[i], target[i],
                                                     ACC ? xsnap[i] : 0.0f, yo, sm);
                 x[i] = xo;
                 if (ACC) { y[i] = yo; xsum[i] = sm; }
@@ -606,7 +620,8 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
     uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
     cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
     if (!sparse_msgs) {
-        const int64_t nwords = (d + (32 / c.b) - 1) / (32 / c.b);
+        const int64_t cpt = c.b == 2 ? 16 : 8;               // coordinates per thread of master_dense_kernel
+        const int64_t nwords = (d + cpt - 1) / cpt;
         const int grid = grid_for(nwords, ctx->sm_count);
         const size_t smem = sizeof(float) * c.M;
         auto al32 = [](const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 31) == 0; };
