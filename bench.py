@@ -42,6 +42,7 @@ def parse_args():
     ap.add_argument("--sparsify", type=int, default=0)
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--configs", default="c1,c2,c3,c4", help="training configurations to time with dq_round ('' for none)")
     return ap.parse_args()
 
 
@@ -177,6 +178,53 @@ def recorded_traffic(bits):
 
 
 # ---------------------------------------------------------------------------------------------------------------
+# whole training rounds (dq_round) on the four training configurations
+# ---------------------------------------------------------------------------------------------------------------
+TRAIN_CONFIGS = {
+    "c1": dict(gen="config1", kw=dict(M=4, B=16, bx=8, b=8, lambda1=1e-4), lr=1.0, theta=0.0, m=200),
+    "c2": dict(gen="config2", kw=dict(M=8, B=64, bx=8, b=4, lambda2=1e-5), lr=1.0, theta=0.0, m=200),
+    "c3": dict(gen="config3", kw=dict(M=16, B=128, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1),
+               lr=1.0, theta=0.0, m=200),
+    "c4": dict(gen="config4", kw=dict(M=32, B=256, bx=8, b=8, box_lo=-10.0, box_hi=10.0, accelerated=1), lr=1e-4,
+               theta=0.1, m=200),
+}
+
+
+def time_training_config(name, rounds=200, warmup=20):
+    """rounds/s of dq_round on one of the training configurations (full size, synthetic data), plus the bits
+    the paper's accounting charges per round."""
+    import numpy as np
+    import torch
+    import paper_1805_10111_b200 as dq
+    from paper_1805_10111_b200 import synth
+    spec = TRAIN_CONFIGS[name]
+    h = getattr(synth, spec["gen"])()
+    cfg = dq.make_config(h.d, spec["kw"]["M"], seed=1805, **{k: v for k, v in spec["kw"].items() if k != "M"})
+    data = dq.Data(h)
+    rc, ctx = dq.dq_create(cfg, data); dq.ok(rc, "dq_create " + name)
+    st = dq.State(np.zeros(h.d, np.float32), n=h.n, accelerated=bool(cfg.accelerated))
+    theta = spec["theta"]; eta = spec["lr"] / theta if theta else spec["lr"]
+    bits = torch.zeros(2, dtype=torch.int64, device="cuda")
+    dq.ok(dq.dq_epoch_begin(ctx, st, theta))
+    for r in range(warmup):
+        dq.ok(dq.dq_round(ctx, st, r, eta, theta))
+    torch.cuda.synchronize()
+    l0 = dq.dq_launch_count(ctx)
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for r in range(rounds):
+        dq.ok(dq.dq_round(ctx, st, warmup + r, eta, theta, bits[0:1], bits[1:2]))
+    e1.record(); torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / rounds
+    rc, status = dq.dq_poll_status(ctx)
+    out = {"rounds_per_s": round(1000.0 / ms, 1), "ms_per_round": round(ms, 4), "n": h.n, "d": h.d, "M": cfg.M, "B": cfg.B,
+           "launches_per_round": (dq.dq_launch_count(ctx) - l0) / rounds, "bits_down": int(bits[0].item()),
+           "bits_up": int(bits[1].item()), "bits_full_precision": 2 * cfg.M * 32 * h.d, "device_status": status}
+    dq.dq_destroy(ctx)
+    return out
+
+
+# ---------------------------------------------------------------------------------------------------------------
 # GPU leg
 # ---------------------------------------------------------------------------------------------------------------
 def run_ours(a):
@@ -300,6 +348,10 @@ def run_ours(a):
         val, sec, what = oracle_rounds_per_sec(a, steps=6, warmup=1)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
     dq.dq_destroy(ctx)
+    del v, hv, st, msgs
+    torch.cuda.empty_cache()
+    if world == 1 and a.configs:
+        line["training_configs"] = {c: time_training_config(c) for c in a.configs.split(",") if c in TRAIN_CONFIGS}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -77,7 +77,7 @@ typedef struct {
     int32_t msg_format;        /* DQ_MSG_SPARSE needs sparsify = 1                                      */
     int32_t accelerated;       /* 1: Algorithm 3                                                        */
     int32_t snapshot_flag;     /* 1: send one flag bit instead of the model when x equals the snapshot  */
-    int32_t reserved;
+    int32_t no_graph;          /* 1: dq_round launches its kernels one by one instead of replaying a CUDA graph */
     uint64_t seed;
     int64_t sparse_cap;        /* entries per worker in the context's own sparse message buffers; 0: d   */
 } dq_config;
@@ -154,7 +154,10 @@ int dq_master_unpack_aggregate_prox(dq_ctx* ctx, const dq_msgs* msgs, dq_state* 
  * NULL) receive the transmitted bits of this round by the paper's message sizes: down = M (32 + bx d), or M
  * flag bits on a snapshot round; up = sum_w (32 + b d) dense, sum_w (32 + nnz_w (ceil(log2 d) + b)) sparse.
  * The round is a snapshot round when snapshot_flag is set and it is the first round after dq_epoch_begin
- * (Algorithm 3: of the first epoch only). */
+ * (Algorithm 3: of the first epoch only).
+ * Unless no_graph is set, the first non-snapshot round on a given set of state/counter pointers records its
+ * kernel sequence as a CUDA graph (this allocates); later rounds copy (round, eta, theta) to the device and
+ * replay it.  Calling with other pointers records again. */
 int dq_round(dq_ctx* ctx, dq_state* st, uint32_t round, float eta, float theta,
              uint64_t* bits_down, uint64_t* bits_up, void* stream);
 

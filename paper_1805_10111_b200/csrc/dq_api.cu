@@ -111,6 +111,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     rc |= dev_alloc(&c->xnorm_bits, 1);
     rc |= dev_alloc(&c->status, 1);
     rc |= dev_alloc(&c->bits, 2);
+    rc |= dev_alloc(&c->rp_dev, 1);
     // message buffers of dq_round / dq_codec_round
     c->msgs.cap = sparse ? (cfg->sparse_cap > 0 ? cfg->sparse_cap : d) : 0;
     c->msgs.stride = sparse ? dq_packed_bytes(c->msgs.cap, cfg->b) : dq_packed_bytes(d, cfg->b);
@@ -139,7 +140,9 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->rp_dev, c->hx, c->hg, c->hv, c->hnorm};
+    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);
     delete c;
     return DQ_OK;
@@ -267,6 +270,44 @@ int dq_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, in
     return last_error();
 }
 
+// The stages of one round, enqueued on `st` (directly, or into a stream capture).
+static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, float eta, float theta, uint64_t* bits_down,
+                         uint64_t* bits_up, void* st)
+{
+    int rc = DQ_OK;
+    if (!flag) rc = dq_quantize_model(ctx, s->x, s->norm_x, round, ctx->codes_x, ctx->delta_x, st);
+    if (rc == DQ_OK) rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
+    if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, st);
+    if (rc == DQ_OK) rc = dq_master_unpack_aggregate_prox(ctx, &ctx->msgs, s, eta, theta, st);
+    if (rc != DQ_OK) return rc;
+    if (bits_down || bits_up)
+        launch_bits(ctx, flag, sparse_messages(ctx), ctx->msgs.nnz, bits_down ? bits_down : ctx->bits,
+                    bits_up ? bits_up : ctx->bits + 1, as_stream(st));
+    return DQ_OK;
+}
+
+// Captures the kernel sequence of a non-flag round into a graph whose kernels read (round, eta, theta) from
+// device memory, so that the same executable graph serves every later round on the same buffers.
+static int capture_round(dq_ctx* ctx, dq_state* s, uint64_t* bits_down, uint64_t* bits_up)
+{
+    if (ctx->graph_exec) { cudaGraphExecDestroy(ctx->graph_exec); ctx->graph_exec = nullptr; }
+    if (!ctx->cap_stream && cudaStreamCreateWithFlags(&ctx->cap_stream, cudaStreamNonBlocking) != cudaSuccess) return DQ_ERR_CUDA;
+    if (cudaStreamBeginCapture(ctx->cap_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return DQ_ERR_CUDA;
+    const int64_t before = ctx->launches;
+    ctx->rp_active = ctx->rp_dev;
+    int rc = enqueue_round(ctx, s, 0u, 0, 1.0f, 0.0f, bits_down, bits_up, ctx->cap_stream);
+    ctx->rp_active = nullptr;
+    ctx->graph_launches = ctx->launches - before;
+    ctx->launches = before;
+    cudaGraph_t graph = nullptr;
+    if (cudaStreamEndCapture(ctx->cap_stream, &graph) != cudaSuccess || !graph) rc = DQ_ERR_CUDA;
+    if (rc == DQ_OK && cudaGraphInstantiate(&ctx->graph_exec, graph, 0) != cudaSuccess) rc = DQ_ERR_CUDA;
+    if (graph) cudaGraphDestroy(graph);
+    if (rc != DQ_OK) { cudaGetLastError(); ctx->graph_exec = nullptr; return rc; }
+    ctx->graph_state = *s; ctx->graph_bits[0] = bits_down; ctx->graph_bits[1] = bits_up;
+    return DQ_OK;
+}
+
 int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, uint64_t* bits_down, uint64_t* bits_up,
              void* stream)
 {
@@ -274,20 +315,29 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
     int rc = check_state(ctx, s);
     if (rc != DQ_OK) return rc;
     if (!s->x_snap || !s->z_snap) return DQ_ERR_ARG;
+    if (!(eta > 0.0f) || !isfinite(eta)) return DQ_ERR_ARG;
     if (ctx->epoch < 0) return DQ_ERR_ARG;                     // dq_epoch_begin has not run
     const dq_config& c = ctx->cfg;
     const int flag = c.snapshot_flag && ctx->rounds_in_epoch == 0 && (!c.accelerated || ctx->epoch == 0);
-    if (!flag) {
-        rc = dq_quantize_model(ctx, s->x, s->norm_x, round, ctx->codes_x, ctx->delta_x, stream);
+    bool replayed = false;
+    if (!flag && !ctx->graph_off && !c.no_graph) {
+        const dq_state& g = ctx->graph_state;
+        const bool same = ctx->graph_exec && g.x == s->x && g.x_snap == s->x_snap && g.g_full == s->g_full && g.y == s->y &&
+                          g.x_sum == s->x_sum && g.norm_x == s->norm_x && g.z_snap == s->z_snap &&
+                          ctx->graph_bits[0] == bits_down && ctx->graph_bits[1] == bits_up;
+        if (!same && capture_round(ctx, s, bits_down, bits_up) != DQ_OK) ctx->graph_off = true;   // fall back to direct launches
+        if (!ctx->graph_off) {
+            cudaStream_t st = as_stream(stream);
+            launch_set_round_params(ctx, round, eta, theta, st);    // scalars travel as kernel arguments: no host buffer to keep alive
+            if (cudaGraphLaunch(ctx->graph_exec, st) != cudaSuccess) return DQ_ERR_CUDA;
+            ctx->launches += ctx->graph_launches;
+            replayed = true;
+        }
+    }
+    if (!replayed) {
+        rc = enqueue_round(ctx, s, round, flag, eta, theta, bits_down, bits_up, stream);
         if (rc != DQ_OK) return rc;
     }
-    rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, stream);
-    if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, stream);
-    if (rc == DQ_OK) rc = dq_master_unpack_aggregate_prox(ctx, &ctx->msgs, s, eta, theta, stream);
-    if (rc != DQ_OK) return rc;
-    if (bits_down || bits_up)
-        launch_bits(ctx, flag, sparse_messages(ctx), ctx->msgs.nnz, bits_down ? bits_down : ctx->bits,
-                    bits_up ? bits_up : ctx->bits + 1, as_stream(stream));
     ctx->rounds_in_epoch += 1;
     return last_error();
 }

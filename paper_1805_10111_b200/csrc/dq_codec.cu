@@ -41,8 +41,9 @@ __global__ void __launch_bounds__(kThreads)
 quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
                      const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker_base, uint32_t stream,
-                     int64_t ngroups, int* __restrict__ status)
+                     int64_t ngroups, int* __restrict__ status, const RoundParams* __restrict__ rp)
 {
+    if (rp) round = rp->round;
     const int w = blockIdx.y;
     const uint32_t nb = norm_bits[w];
     const float nrm = __uint_as_float(nb);
@@ -157,8 +158,9 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
                       const unsigned long long* __restrict__ l1_sum, float phi,
                       const __grid_constant__ PhiloxKeys K, uint32_t round,
                       uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
-                      int64_t nchunks)
+                      int64_t nchunks, const RoundParams* __restrict__ rp)
 {
+    if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
     const float* row = v + (int64_t)w * d;
@@ -239,8 +241,9 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      const uint32_t* __restrict__ beta_norm_bits, const uint32_t* __restrict__ chunk_off,
                      int64_t nchunks, int64_t ngroups,
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
-                     uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status)
+                     uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status, const RoundParams* __restrict__ rp)
 {
+    if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
     const uint32_t bb = beta_norm_bits[w];
@@ -382,8 +385,9 @@ __global__ void __launch_bounds__(kThreads, BITS == 2 ? 3 : 4)
 master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
                     const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
-                    int vec8_ok, uint32_t* __restrict__ normx_bits)
+                    int vec8_ok, uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp)
 {
+    if (rp) { eta = rp->eta; theta = rp->theta; }
     constexpr int W = (BITS == 8) ? 2 : 1;                  // code words per worker and thread
     constexpr int CW = 32 / BITS;                           // coordinates per code word
     constexpr int C = W * CW;                               // coordinates per thread: 8, 8, 16 for 8, 4, 2 bits
@@ -487,8 +491,9 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
                      const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* __restrict__ tile_ptr, int64_t ntiles,
                      int M, int64_t d, const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                      const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
-                     uint32_t* __restrict__ normx_bits)
+                     uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp)
 {
+    if (rp) { eta = rp->eta; theta = rp->theta; }
     __shared__ float s_acc[kChunk];
     const float inv_m = __fdiv_rn(1.0f, (float)M);
     const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
@@ -579,7 +584,7 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
     DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_><<<grid, kThreads, 0, st>>>(
-        v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status)));
+        v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active)));
     ctx->launches += 1;
 }
 
@@ -594,20 +599,20 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
     dim3 grid_c(grid_for(nchunks * 32, ctx->sm_count), M);
     sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
-                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks);
+                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks, ctx->rp_active);
     ctx->launches += 2;
     if (sparse_out) {
         chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
         cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
-            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status)));
+            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active)));
         ctx->launches += 2;
     } else {
         const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
-            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status)));
+            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active)));
         ctx->launches += 1;
     }
 }
@@ -628,10 +633,10 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         const int vec8_ok = al32(s->x) && al32(s->g_full) && al32(s->y) && al32(s->x_snap) && al32(s->x_sum);
         if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx)));
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active)));
         } else {
             DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx)));
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active)));
         }
         ctx->launches += 1;
     } else {
@@ -642,11 +647,11 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
                 msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
-                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active)));
         } else {
             DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, false><<<grid, kThreads, 0, st>>>(
                 msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
-                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx)));
+                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active)));
         }
         ctx->launches += 2;
     }
@@ -728,6 +733,6 @@ extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, 
     const PhiloxKeys keys = expand_keys(seed);
     int* flag = reinterpret_cast<int*>(scratch + kStaticMaxMessages);
     DQ_DISPATCH_BITS(b, (quantize_pack_kernel<BITS_><<<grid_q, kThreads, 0, st>>>(
-        v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag)));
+        v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr)));
     return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }

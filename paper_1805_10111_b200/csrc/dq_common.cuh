@@ -145,6 +145,9 @@ __device__ __forceinline__ void block_atomic_max(uint32_t v, uint32_t* dst)
 
 struct ProxParams { float lambda1, lambda2, lo, hi; };
 
+// Per-round scalars kept in device memory so that a captured graph of a round can be replayed unchanged.
+struct RoundParams { uint32_t round; float eta; float theta; uint32_t pad; };
+
 #define DQ_DISPATCH_BITS(bits, CALL)                 \
     switch (bits) {                                  \
         case 2: { constexpr int BITS_ = 2; CALL; } break; \
@@ -182,6 +185,15 @@ struct dq_ctx {
     uint64_t* bits;             // [2] device counters
     // device-resident state for the host-buffer entry point
     float *hx, *hg, *hv, *hnorm;
+    // replay of whole rounds: per-round scalars on the device and the captured graph of a non-flag round
+    dq::RoundParams* rp_dev;
+    const dq::RoundParams* rp_active;   // non-null while a round is being captured
+    cudaStream_t cap_stream;
+    cudaGraphExec_t graph_exec;
+    dq_state graph_state;
+    uint64_t* graph_bits[2];
+    int64_t graph_launches;
+    bool graph_off;
     // bookkeeping
     int64_t launches;
     int64_t rounds_in_epoch;

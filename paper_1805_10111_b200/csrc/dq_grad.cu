@@ -59,8 +59,9 @@ __device__ __forceinline__ double warp_dot_csr(const float* __restrict__ val, co
 // (j & 3) of Philox counter (j >> 2, round, w, batch stream).
 // ---------------------------------------------------------------------------------------------------
 __global__ void sample_rows_kernel(const __grid_constant__ PhiloxKeys K, uint32_t round, int M, int B, int64_t n,
-                                   int32_t* __restrict__ rows)
+                                   int32_t* __restrict__ rows, const RoundParams* __restrict__ rp)
 {
+    if (rp) round = rp->round;
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= M * B) return;
     const int w = t / B, j = t % B;
@@ -136,6 +137,93 @@ worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labe
 }
 
 // ---------------------------------------------------------------------------------------------------
+// 16-byte vector access to a row of features: 4 floats or 8 bfloat16 per load.
+// ---------------------------------------------------------------------------------------------------
+template <class T> struct RowVec;
+template <> struct RowVec<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ void unpack(const uint4& u, float (&f)[4])
+    { f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w); }
+};
+template <> struct RowVec<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ void unpack(const uint4& u, float (&f)[8])
+    {   // a bfloat16 is the upper half of an fp32
+        f[0] = __uint_as_float(u.x << 16); f[1] = __uint_as_float(u.x & 0xFFFF0000u);
+        f[2] = __uint_as_float(u.y << 16); f[3] = __uint_as_float(u.y & 0xFFFF0000u);
+        f[4] = __uint_as_float(u.z << 16); f[5] = __uint_as_float(u.z & 0xFFFF0000u);
+        f[6] = __uint_as_float(u.w << 16); f[7] = __uint_as_float(u.w & 0xFFFF0000u);
+    }
+};
+
+// <a_row, vec> by one warp with 16-byte loads (d a multiple of the vector width, row 16-byte aligned).
+template <class T>
+__device__ __forceinline__ double warp_dot_dense_vec(const T* __restrict__ row, const float* __restrict__ vec, int64_t d, int lane)
+{
+    constexpr int N = RowVec<T>::N;
+    const uint4* rv = reinterpret_cast<const uint4*>(row);
+    const float4* vv = reinterpret_cast<const float4*>(vec);
+    const int nv = (int)(d / N);
+    float s[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll 4
+    for (int v = lane; v < nv; v += 32) {
+        float f[N];
+        RowVec<T>::unpack(__ldg(rv + v), f);
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q) {
+            const float4 x4 = __ldg(vv + v * (N / 4) + q);
+            s[0] = fmaf(f[q * 4 + 0], x4.x, s[0]); s[1] = fmaf(f[q * 4 + 1], x4.y, s[1]);
+            s[2] = fmaf(f[q * 4 + 2], x4.z, s[2]); s[3] = fmaf(f[q * 4 + 3], x4.w, s[3]);
+        }
+    }
+    return warp_sum(((double)s[0] + (double)s[1]) + ((double)s[2] + (double)s[3]));
+}
+
+// Vectorised dense worker gradient: same plan as worker_grad_dense_kernel with 16-byte loads and
+// 16-byte atomics (d a multiple of the vector width).  The rows read in phase A are read again in phase
+// B while they are still in L2.
+template <class T>
+__global__ void __launch_bounds__(kThreads)
+worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
+                             const float* __restrict__ z_snap, const int32_t* __restrict__ rows, int B, int64_t d,
+                             float* __restrict__ alpha)
+{
+    constexpr int N = RowVec<T>::N;
+    __shared__ float s_r[kRowsPerBlock];
+    __shared__ const uint4* s_rowp[kRowsPerBlock];
+    const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int j0 = blockIdx.x * kRowsPerBlock;
+    const int nrows = min(kRowsPerBlock, B - j0);
+    for (int j = warp; j < nrows; j += kThreads / 32) {
+        const int64_t a = rows[(int64_t)w * B + j0 + j];
+        const float dz = (float)warp_dot_dense_vec(X + a * d, diff, d, lane);
+        if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_rowp[j] = reinterpret_cast<const uint4*>(X + a * d); }
+    }
+    __syncthreads();
+    const int nv = (int)(d / N);
+    float* out = alpha + (int64_t)w * d;
+    for (int v = threadIdx.x; v < nv; v += blockDim.x) {
+        float acc[N];
+#pragma unroll
+        for (int q = 0; q < N; ++q) acc[q] = 0.0f;
+#pragma unroll 4
+        for (int j = 0; j < nrows; ++j) {
+            float f[N];
+            RowVec<T>::unpack(__ldg(s_rowp[j] + v), f);
+            const float r = s_r[j];
+#pragma unroll
+            for (int q = 0; q < N; ++q) acc[q] = fmaf(r, f[q], acc[q]);
+        }
+        float4* o4 = reinterpret_cast<float4*>(out + (int64_t)v * N);
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q) {
+            const float4 val = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
+            if (gridDim.x == 1) o4[q] = val; else atomicAdd(o4 + q, val);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Full gradient over all n rows at xsnap, accumulated in double; also stores the margins z_snap.
 // ---------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
@@ -174,6 +262,42 @@ full_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labels
             double s = 0.0;
             for (int j = 0; j < nrows; ++j) s += (double)s_c[j] * (double)to_float(X[(a0 + j) * d + i]);
             atomicAdd(g64 + i, s);
+        }
+        __syncthreads();
+    }
+}
+
+// Vectorised variant of full_grad_dense_kernel (d a multiple of the 16-byte vector width).
+template <class T>
+__global__ void __launch_bounds__(kThreads)
+full_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ x, int64_t n,
+                           int64_t d, float* __restrict__ z_out, double* __restrict__ g64)
+{
+    constexpr int N = RowVec<T>::N;
+    __shared__ float s_c[kRowsPerBlock];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nv = (int)(d / N);
+    for (int64_t a0 = (int64_t)blockIdx.x * kRowsPerBlock; a0 < n; a0 += (int64_t)gridDim.x * kRowsPerBlock) {
+        const int nrows = (int)min((int64_t)kRowsPerBlock, n - a0);
+        for (int j = warp; j < nrows; j += kThreads / 32) {
+            const double z = warp_dot_dense_vec(X + (a0 + j) * d, x, d, lane);
+            const double y = (double)labels[a0 + j];
+            if (lane == 0) { s_c[j] = (float)(-y / (1.0 + exp(y * z))); if (z_out) z_out[a0 + j] = (float)z; }
+        }
+        __syncthreads();
+        for (int v = threadIdx.x; v < nv; v += blockDim.x) {
+            double acc[N];
+#pragma unroll
+            for (int q = 0; q < N; ++q) acc[q] = 0.0;
+            for (int j = 0; j < nrows; ++j) {
+                float f[N];
+                RowVec<T>::unpack(__ldg(reinterpret_cast<const uint4*>(X + (a0 + j) * d) + v), f);
+                const double c = (double)s_c[j];
+#pragma unroll
+                for (int q = 0; q < N; ++q) acc[q] += c * (double)f[q];
+            }
+#pragma unroll
+            for (int q = 0; q < N; ++q) atomicAdd(g64 + (int64_t)v * N + q, acc[q]);
         }
         __syncthreads();
     }
@@ -287,8 +411,14 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
     } else {
         const int64_t nblk = (D.n + kRowsPerBlock - 1) / kRowsPerBlock;
         const int grid = (int)(nblk < (int64_t)ctx->sm_count * 8 ? nblk : (int64_t)ctx->sm_count * 8);
-        if (D.format == DQ_DENSE_F32)
+        const bool f32 = D.format == DQ_DENSE_F32;
+        const bool vec = (D.d % (f32 ? 4 : 8)) == 0;
+        if (f32 && vec)
+            full_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+        else if (f32)
             full_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+        else if (vec)
+            full_grad_dense_vec_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
         else
             full_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
     }
@@ -306,7 +436,7 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         return;
     }
     if (!batch_idx) {
-        sample_rows_kernel<<<(c.M * c.B + kThreads - 1) / kThreads, kThreads, 0, st>>>(ctx->keys, round, c.M, c.B, D.n, ctx->rows);
+        sample_rows_kernel<<<(c.M * c.B + kThreads - 1) / kThreads, kThreads, 0, st>>>(ctx->keys, round, c.M, c.B, D.n, ctx->rows, ctx->rp_active);
         batch_idx = ctx->rows;
         ctx->launches += 1;
     }
@@ -319,8 +449,14 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
     } else {
         dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
         if (grid.x > 1) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
-        if (D.format == DQ_DENSE_F32)
+        const bool f32 = D.format == DQ_DENSE_F32;
+        const bool vec = (c.d % (f32 ? 4 : 8)) == 0 && (reinterpret_cast<uintptr_t>(alpha) & 15) == 0;   // data is 16-byte aligned by contract
+        if (f32 && vec)
+            worker_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+        else if (f32)
             worker_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+        else if (vec)
+            worker_grad_dense_vec_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
         else
             worker_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
     }
@@ -338,6 +474,17 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
     else objective_loss_kernel<DQ_DENSE_BF16><<<grid, kThreads, 0, st>>>(D, x, P);
     objective_reg_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(x, c.d, c.lambda1, c.lambda2, P);
     ctx->launches += 2;
+}
+
+__global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float eta, float theta)
+{
+    rp->round = round; rp->eta = eta; rp->theta = theta; rp->pad = 0u;
+}
+
+void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st)
+{
+    set_round_params_kernel<<<1, 1, 0, st>>>(ctx->rp_dev, round, eta, theta);
+    ctx->launches += 1;
 }
 
 void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* nnz, uint64_t* bits_down, uint64_t* bits_up,

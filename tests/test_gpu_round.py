@@ -57,6 +57,10 @@ def _problem(name):
             _PROBLEMS[name] = synth.sparse_logistic(3000, 5003, 30.0, 1.1, 61)
         elif name == "bf16":
             _PROBLEMS[name] = synth.dense_bf16_logistic(700, 520, 62)
+        elif name == "bf16odd":
+            _PROBLEMS[name] = synth.dense_bf16_logistic(300, 301, 63)         # rows off the 16-byte grid: scalar path
+        elif name == "dense8":
+            _PROBLEMS[name] = synth.dense_logistic(400, 256, 64)              # vector path for fp32 features
         elif name == "c1":
             _PROBLEMS[name] = synth.config1()
         elif name == "c2":
@@ -83,7 +87,7 @@ def _abs_grad_scale(h, x):
     return (S / h.n).astype(F32)
 
 
-@pytest.mark.parametrize("name", ["dense", "csr", "bf16"])
+@pytest.mark.parametrize("name", ["dense", "csr", "bf16", "bf16odd", "dense8"])
 def test_epoch_begin_full_gradient(dq, name):
     import torch
     h = _problem(name)
@@ -111,7 +115,7 @@ def test_epoch_begin_full_gradient(dq, name):
     dq.dq_destroy(ctx); dq.dq_destroy(ctx2)
 
 
-@pytest.mark.parametrize("name", ["dense", "csr", "bf16"])
+@pytest.mark.parametrize("name", ["dense", "csr", "bf16", "bf16odd", "dense8"])
 @pytest.mark.parametrize("bx", [4, 8])
 def test_worker_gradient(dq, name, bx):
     import torch
