@@ -275,15 +275,20 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
                          uint64_t* bits_up, void* st)
 {
     int rc = DQ_OK;
-    if (!flag) rc = dq_quantize_model(ctx, s->x, s->norm_x, round, ctx->codes_x, ctx->delta_x, st);
-    if (rc == DQ_OK) rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
+    if (!flag) {     // model quantisation that also emits xhat - xsnap for the workers
+        launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, reinterpret_cast<const uint32_t*>(s->norm_x), ctx->codes_x,
+                             dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx), ctx->delta_x, round, kMaster, kStreamModel, as_stream(st),
+                             s->x_snap, ctx->xhat_diff);
+        ctx->diff_ready = true;
+    }
+    rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
+    ctx->diff_ready = false;
     if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, st);
-    if (rc == DQ_OK) rc = dq_master_unpack_aggregate_prox(ctx, &ctx->msgs, s, eta, theta, st);
     if (rc != DQ_OK) return rc;
-    if (bits_down || bits_up)
-        launch_bits(ctx, flag, sparse_messages(ctx), ctx->msgs.nnz, bits_down ? bits_down : ctx->bits,
-                    bits_up ? bits_up : ctx->bits + 1, as_stream(st));
-    return DQ_OK;
+    const BitsArgs ba = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag,
+                         sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b};
+    launch_master(ctx, &ctx->msgs, sparse_messages(ctx), s, eta, theta, as_stream(st), (bits_down || bits_up) ? &ba : nullptr);
+    return last_error();
 }
 
 // Captures the kernel sequence of a non-flag round into a graph whose kernels read (round, eta, theta) from

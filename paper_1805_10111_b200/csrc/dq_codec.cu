@@ -36,12 +36,15 @@ __global__ void __launch_bounds__(kThreads) norm_inf_kernel(const float* __restr
 // Dense Q_(delta,b) + pack.  grid (blocks, M).  Each thread turns groups of eight coordinates into BITS
 // bytes.  ngroups covers the zero padding of the packed message (coordinates >= d quantise to code 0).
 // ---------------------------------------------------------------------------------------------------
-template <int BITS>
+// With DIFF the kernel also writes code*delta - ref (the dequantised vector minus a reference), which is what the
+// worker-gradient stage needs from the broadcast model.
+template <int BITS, bool DIFF = false>
 __global__ void __launch_bounds__(kThreads)
 quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
                      const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker_base, uint32_t stream,
-                     int64_t ngroups, int* __restrict__ status, const RoundParams* __restrict__ rp)
+                     int64_t ngroups, int* __restrict__ status, const RoundParams* __restrict__ rp,
+                     const float* __restrict__ ref = nullptr, float* __restrict__ diff = nullptr)
 {
     if (rp) round = rp->round;
     const int w = blockIdx.y;
@@ -50,8 +53,9 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
     const bool finite = nb < 0x7F800000u;
     // delta = nrm / L; inv = 1/delta rounded toward zero so that |v| <= nrm stays inside the hull.
     const float inv = (finite && nb != 0u) ? __fdiv_rd((float)levels(BITS), nrm) : 0.0f;
+    const float delta = (finite && nb != 0u) ? __fdiv_rn(nrm, (float)levels(BITS)) : 0.0f;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        scale[w] = (finite && nb != 0u) ? __fdiv_rn(nrm, (float)levels(BITS)) : 0.0f;
+        scale[w] = delta;
         if (!finite) set_status(status, DQ_ERR_NONFINITE);
     }
     const float* row = v + (int64_t)w * d;
@@ -67,6 +71,15 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
 #pragma unroll
         for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
         store_group<BITS>(out + g * BITS, pack8<BITS>(s));
+        if (DIFF) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (i0 + j < d) {
+                    const float k = (float)((int)((s[j] >> 16) & 0xFFu) - 128);
+                    diff[i0 + j] = __fsub_rn(__fmul_rn(k, delta), ref[i0 + j]);
+                }
+            }
+        }
     }
 }
 
@@ -385,9 +398,10 @@ __global__ void __launch_bounds__(kThreads, BITS == 2 ? 3 : 4)
 master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
                     const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
-                    int vec8_ok, uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp)
+                    int vec8_ok, uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
 {
     if (rp) { eta = rp->eta; theta = rp->theta; }
+    if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     constexpr int W = (BITS == 8) ? 2 : 1;                  // code words per worker and thread
     constexpr int CW = 32 / BITS;                           // coordinates per code word
     constexpr int C = W * CW;                               // coordinates per thread: 8, 8, 16 for 8, 4, 2 bits
@@ -491,9 +505,10 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
                      const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* __restrict__ tile_ptr, int64_t ntiles,
                      int M, int64_t d, const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                      const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
-                     uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp)
+                     uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
 {
     if (rp) { eta = rp->eta; theta = rp->theta; }
+    if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     __shared__ float s_acc[kChunk];
     const float inv_m = __fdiv_rn(1.0f, (float)M);
     const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
@@ -579,10 +594,17 @@ void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* no
 
 void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
-                          uint32_t stream_id, cudaStream_t st)
+                          uint32_t stream_id, cudaStream_t st, const float* ref, float* diff)
 {
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
+    if (diff) {
+        DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
+            v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
+            ctx->rp_active, ref, diff)));
+        ctx->launches += 1;
+        return;
+    }
     DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_><<<grid, kThreads, 0, st>>>(
         v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active)));
     ctx->launches += 1;
@@ -617,8 +639,11 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     }
 }
 
-void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st)
+void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,
+                   const BitsArgs* bits)
 {
+    BitsArgs ba = {nullptr, nullptr, nullptr, 0, 0, 0, 0};
+    if (bits) ba = *bits;
     const dq_config& c = ctx->cfg;
     const int64_t d = c.d;
     ProxParams pp{c.lambda1, c.lambda2, c.box_lo, c.box_hi};
@@ -633,10 +658,10 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         const int vec8_ok = al32(s->x) && al32(s->g_full) && al32(s->y) && al32(s->x_snap) && al32(s->x_sum);
         if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active)));
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
         } else {
             DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active)));
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
         }
         ctx->launches += 1;
     } else {
@@ -647,11 +672,11 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
                 msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
-                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active)));
+                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         } else {
             DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, false><<<grid, kThreads, 0, st>>>(
                 msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
-                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active)));
+                s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         }
         ctx->launches += 2;
     }
@@ -732,7 +757,7 @@ extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, 
     dim3 grid_q(grid_for(ngroups, sms), M);
     const PhiloxKeys keys = expand_keys(seed);
     int* flag = reinterpret_cast<int*>(scratch + kStaticMaxMessages);
-    DQ_DISPATCH_BITS(b, (quantize_pack_kernel<BITS_><<<grid_q, kThreads, 0, st>>>(
+    DQ_DISPATCH_BITS(b, (quantize_pack_kernel<BITS_, false><<<grid_q, kThreads, 0, st>>>(
         v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr)));
     return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }

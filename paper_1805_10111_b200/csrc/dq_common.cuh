@@ -145,6 +145,19 @@ __device__ __forceinline__ void block_atomic_max(uint32_t v, uint32_t* dst)
 
 struct ProxParams { float lambda1, lambda2, lo, hi; };
 
+// Transmitted-bit counters of a round, written by the master kernel when `down` is set (Section 3.1 message sizes).
+struct BitsArgs { uint64_t* down; uint64_t* up; const uint32_t* nnz; int flag_round, sparse_msgs, bx, b; };
+
+__device__ __forceinline__ void write_round_bits(const BitsArgs& ba, int M, int64_t d)
+{
+    *ba.down = ba.flag_round ? (uint64_t)M : (uint64_t)M * (32ull + (uint64_t)ba.bx * (uint64_t)d);
+    int logd = 0; while (((int64_t)1 << logd) < d) ++logd;
+    uint64_t up = 0;
+    for (int w = 0; w < M; ++w)
+        up += ba.sparse_msgs ? 32ull + (uint64_t)ba.nnz[w] * (uint64_t)(logd + ba.b) : 32ull + (uint64_t)ba.b * (uint64_t)d;
+    *ba.up = up;
+}
+
 // Per-round scalars kept in device memory so that a captured graph of a round can be replayed unchanged.
 struct RoundParams { uint32_t round; float eta; float theta; uint32_t pad; };
 
@@ -194,6 +207,7 @@ struct dq_ctx {
     uint64_t* graph_bits[2];
     int64_t graph_launches;
     bool graph_off;
+    bool diff_ready;            // the model-quantise kernel of this round already wrote xhat - xsnap
     // bookkeeping
     int64_t launches;
     int64_t rounds_in_epoch;

@@ -58,18 +58,27 @@ __device__ __forceinline__ double warp_dot_csr(const float* __restrict__ val, co
 // Minibatch rows: worker w draws slot j from its partition [floor(w n/M), floor((w+1) n/M)) with word
 // (j & 3) of Philox counter (j >> 2, round, w, batch stream).
 // ---------------------------------------------------------------------------------------------------
-__global__ void sample_rows_kernel(const __grid_constant__ PhiloxKeys K, uint32_t round, int M, int B, int64_t n,
-                                   int32_t* __restrict__ rows, const RoundParams* __restrict__ rp)
+__device__ __forceinline__ int64_t sample_row(const PhiloxKeys& K, uint32_t round, int w, int j, int M, int64_t n)
 {
-    if (rp) round = rp->round;
-    const int t = blockIdx.x * blockDim.x + threadIdx.x;
-    if (t >= M * B) return;
-    const int w = t / B, j = t % B;
     const int64_t lo = ((int64_t)w * n) / M, hi = ((int64_t)(w + 1) * n) / M;
     uint32_t r[4];
     philox4x32_10((uint32_t)(j >> 2), round, (uint32_t)w, kStreamBatch, K, r);
     const uint32_t word = (j & 3) == 0 ? r[0] : (j & 3) == 1 ? r[1] : (j & 3) == 2 ? r[2] : r[3];
-    rows[t] = (int32_t)(lo + (int64_t)(((uint64_t)word * (uint64_t)(hi - lo)) >> 32));
+    return lo + (int64_t)(((uint64_t)word * (uint64_t)(hi - lo)) >> 32);
+}
+
+// Where a worker's minibatch comes from: explicit indices, or the batch stream (then also recorded in rows_out).
+struct BatchSource {
+    const int32_t* rows_in; int32_t* rows_out; uint32_t round; const RoundParams* rp; int M; int64_t n;
+};
+
+__device__ __forceinline__ int64_t batch_row(const BatchSource& bs, const PhiloxKeys& K, int w, int j, int B, bool writer)
+{
+    const int64_t slot = (int64_t)w * B + j;
+    if (bs.rows_in) return bs.rows_in[slot];
+    const int64_t a = sample_row(K, bs.rp ? bs.rp->round : bs.round, w, j, bs.M, bs.n);
+    if (writer && bs.rows_out) bs.rows_out[slot] = (int32_t)a;
+    return a;
 }
 
 // xhat - xsnap with xhat_i = code_i * delta_x (the transmitted low-precision model).
@@ -92,13 +101,13 @@ __global__ void dequant_diff_kernel(const uint8_t* __restrict__ codes, const flo
 __global__ void __launch_bounds__(kThreads)
 worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict__ col, const int64_t* __restrict__ row_ptr,
                        const float* __restrict__ labels, const float* __restrict__ diff, const float* __restrict__ z_snap,
-                       const int32_t* __restrict__ rows, int M, int B, int64_t d, float* __restrict__ alpha)
+                       const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, float* __restrict__ alpha)
 {
     const int lane = threadIdx.x & 31;
     const int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (slot >= (int64_t)M * B) return;
     const int w = (int)(slot / B);
-    const int64_t a = rows[slot];
+    const int64_t a = batch_row(bs, K, w, (int)(slot % B), B, lane == 0);
     const int64_t k0 = row_ptr[a], k1 = row_ptr[a + 1];
     const float dz = (float)warp_dot_csr(val, col, k0, k1, diff, lane);
     const float r = slope_difference(labels[a], z_snap[a], dz) / (float)B;
@@ -114,7 +123,7 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
 template <class T>
 __global__ void __launch_bounds__(kThreads)
 worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
-                         const float* __restrict__ z_snap, const int32_t* __restrict__ rows, int B, int64_t d,
+                         const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int64_t d,
                          float* __restrict__ alpha)
 {
     __shared__ float s_r[kRowsPerBlock];
@@ -123,7 +132,7 @@ worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labe
     const int j0 = blockIdx.x * kRowsPerBlock;
     const int nrows = min(kRowsPerBlock, B - j0);
     for (int j = warp; j < nrows; j += kThreads / 32) {
-        const int64_t a = rows[(int64_t)w * B + j0 + j];
+        const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
         const float dz = (float)warp_dot_dense(X + a * d, diff, d, lane);
         if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_row[j] = a; }
     }
@@ -185,7 +194,7 @@ __device__ __forceinline__ double warp_dot_dense_vec(const T* __restrict__ row, 
 template <class T>
 __global__ void __launch_bounds__(kThreads)
 worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
-                             const float* __restrict__ z_snap, const int32_t* __restrict__ rows, int B, int64_t d,
+                             const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int64_t d,
                              float* __restrict__ alpha)
 {
     constexpr int N = RowVec<T>::N;
@@ -195,7 +204,7 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
     const int j0 = blockIdx.x * kRowsPerBlock;
     const int nrows = min(kRowsPerBlock, B - j0);
     for (int j = warp; j < nrows; j += kThreads / 32) {
-        const int64_t a = rows[(int64_t)w * B + j0 + j];
+        const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
         const float dz = (float)warp_dot_dense_vec(X + a * d, diff, d, lane);
         if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_rowp[j] = reinterpret_cast<const uint4*>(X + a * d); }
     }
@@ -435,32 +444,31 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         cudaMemsetAsync(norm_inf, 0, sizeof(float) * c.M, st);
         return;
     }
-    if (!batch_idx) {
-        sample_rows_kernel<<<(c.M * c.B + kThreads - 1) / kThreads, kThreads, 0, st>>>(ctx->keys, round, c.M, c.B, D.n, ctx->rows, ctx->rp_active);
-        batch_idx = ctx->rows;
+    const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n};
+    if (!ctx->diff_ready) {
+        DQ_DISPATCH_BITS(c.bx, (dequant_diff_kernel<BITS_><<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(
+            codes_x, delta_x, s->x_snap, c.d, ctx->xhat_diff)));
         ctx->launches += 1;
     }
-    DQ_DISPATCH_BITS(c.bx, (dequant_diff_kernel<BITS_><<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(
-        codes_x, delta_x, s->x_snap, c.d, ctx->xhat_diff)));
     if (D.format == DQ_CSR_F32) {
         cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         worker_grad_csr_kernel<<<(int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.M, c.B, c.d, alpha);
+            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha);
     } else {
         dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
         if (grid.x > 1) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         const bool f32 = D.format == DQ_DENSE_F32;
         const bool vec = (c.d % (f32 ? 4 : 8)) == 0 && (reinterpret_cast<uintptr_t>(alpha) & 15) == 0;   // data is 16-byte aligned by contract
         if (f32 && vec)
-            worker_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+            worker_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else if (f32)
-            worker_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+            worker_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else if (vec)
-            worker_grad_dense_vec_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+            worker_grad_dense_vec_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else
-            worker_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, batch_idx, c.B, c.d, alpha);
+            worker_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
     }
-    ctx->launches += 2;
+    ctx->launches += 1;
     launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
 }
 

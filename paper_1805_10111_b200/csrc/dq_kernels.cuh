@@ -8,10 +8,11 @@ namespace dq {
 void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* norm_bits, cudaStream_t st);
 void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
-                          uint32_t stream_id, cudaStream_t st);
+                          uint32_t stream_id, cudaStream_t st, const float* ref = nullptr, float* diff = nullptr);
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
-void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st);
+void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,
+                   const BitsArgs* bits = nullptr);
 void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, float* out, cudaStream_t st);
 
 // gradients (dq_grad.cu)
