@@ -278,16 +278,18 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     if (!flag) {     // model quantisation that also emits xhat - xsnap for the workers
         launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, reinterpret_cast<const uint32_t*>(s->norm_x), ctx->codes_x,
                              dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx), ctx->delta_x, round, kMaster, kStreamModel, as_stream(st),
-                             s->x_snap, ctx->xhat_diff);
-        ctx->diff_ready = true;
+                             s->x_snap, ctx->xhat_diff, ctx->alpha, (int64_t)ctx->cfg.M * ctx->cfg.d,
+                             reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
+        ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = ctx->normx_zeroed = true;
     }
     rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
-    ctx->diff_ready = false;
+    ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = false;
     if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, st);
-    if (rc != DQ_OK) return rc;
+    if (rc != DQ_OK) { ctx->normx_zeroed = false; return rc; }
     const BitsArgs ba = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag,
                          sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b};
     launch_master(ctx, &ctx->msgs, sparse_messages(ctx), s, eta, theta, as_stream(st), (bits_down || bits_up) ? &ba : nullptr);
+    ctx->normx_zeroed = false;
     return last_error();
 }
 

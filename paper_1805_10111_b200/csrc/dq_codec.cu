@@ -44,9 +44,16 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
                      const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker_base, uint32_t stream,
                      int64_t ngroups, int* __restrict__ status, const RoundParams* __restrict__ rp,
-                     const float* __restrict__ ref = nullptr, float* __restrict__ diff = nullptr)
+                     const float* __restrict__ ref = nullptr, float* __restrict__ diff = nullptr,
+                     float* __restrict__ zero_f = nullptr, int64_t zero_n = 0, uint32_t* __restrict__ zero_u = nullptr, int zero_un = 0)
 {
     if (rp) round = rp->round;
+    if (DIFF) {   // also clears the buffers that the next stages of the round accumulate into
+        const int64_t nth0 = (int64_t)gridDim.x * gridDim.y * blockDim.x;
+        const int64_t tid0 = ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
+        for (int64_t i = tid0; i < zero_n; i += nth0) zero_f[i] = 0.0f;
+        if (tid0 < zero_un) zero_u[tid0] = 0u;
+    }
     const int w = blockIdx.y;
     const uint32_t nb = norm_bits[w];
     const float nrm = __uint_as_float(nb);
@@ -586,7 +593,7 @@ static inline int vec_ok_for(const float* v, int64_t d) { return ((reinterpret_c
 
 void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* norm_bits, cudaStream_t st)
 {
-    cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * M, st);
+    if (!ctx->ninf_zeroed) cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * M, st);
     dim3 grid(grid_for((d + 7) / 8, ctx->sm_count), M);
     norm_inf_kernel<<<grid, kThreads, 0, st>>>(v, d, vec_ok_for(v, d), norm_bits);
     ctx->launches += 1;
@@ -594,14 +601,15 @@ void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* no
 
 void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
-                          uint32_t stream_id, cudaStream_t st, const float* ref, float* diff)
+                          uint32_t stream_id, cudaStream_t st, const float* ref, float* diff, float* zero_f, int64_t zero_n,
+                          uint32_t* zero_u, int zero_un)
 {
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
     if (diff) {
         DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
             v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
-            ctx->rp_active, ref, diff)));
+            ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un)));
         ctx->launches += 1;
         return;
     }
@@ -648,7 +656,7 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
     const int64_t d = c.d;
     ProxParams pp{c.lambda1, c.lambda2, c.box_lo, c.box_hi};
     uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
-    cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
+    if (!ctx->normx_zeroed) cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
     if (!sparse_msgs) {
         const int64_t cpt = c.b == 2 ? 16 : 8;               // coordinates per thread of master_dense_kernel
         const int64_t nwords = (d + cpt - 1) / cpt;

@@ -207,6 +207,7 @@ struct dq_ctx {
     uint64_t* graph_bits[2];
     int64_t graph_launches;
     bool graph_off;
+    bool alpha_zeroed, ninf_zeroed, normx_zeroed;   // an earlier kernel of this round already cleared these
     bool diff_ready;            // the model-quantise kernel of this round already wrote xhat - xsnap
     // bookkeeping
     int64_t launches;

@@ -70,7 +70,13 @@ __device__ __forceinline__ int64_t sample_row(const PhiloxKeys& K, uint32_t roun
 // Where a worker's minibatch comes from: explicit indices, or the batch stream (then also recorded in rows_out).
 struct BatchSource {
     const int32_t* rows_in; int32_t* rows_out; uint32_t round; const RoundParams* rp; int M; int64_t n;
+    uint32_t* zero_word;   // cleared by the first thread of the grid (the next stage's maximum), may be NULL
 };
+
+__device__ __forceinline__ void clear_word(const BatchSource& bs)
+{
+    if (bs.zero_word && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *bs.zero_word = 0u;
+}
 
 __device__ __forceinline__ int64_t batch_row(const BatchSource& bs, const PhiloxKeys& K, int w, int j, int B, bool writer)
 {
@@ -103,6 +109,7 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
                        const float* __restrict__ labels, const float* __restrict__ diff, const float* __restrict__ z_snap,
                        const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, float* __restrict__ alpha)
 {
+    clear_word(bs);
     const int lane = threadIdx.x & 31;
     const int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (slot >= (int64_t)M * B) return;
@@ -128,6 +135,7 @@ worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labe
 {
     __shared__ float s_r[kRowsPerBlock];
     __shared__ int64_t s_row[kRowsPerBlock];
+    clear_word(bs);
     const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int j0 = blockIdx.x * kRowsPerBlock;
     const int nrows = min(kRowsPerBlock, B - j0);
@@ -200,6 +208,7 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
     constexpr int N = RowVec<T>::N;
     __shared__ float s_r[kRowsPerBlock];
     __shared__ const uint4* s_rowp[kRowsPerBlock];
+    clear_word(bs);
     const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int j0 = blockIdx.x * kRowsPerBlock;
     const int nrows = min(kRowsPerBlock, B - j0);
@@ -444,19 +453,20 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         cudaMemsetAsync(norm_inf, 0, sizeof(float) * c.M, st);
         return;
     }
-    const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n};
+    const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n,
+                            ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr};
     if (!ctx->diff_ready) {
         DQ_DISPATCH_BITS(c.bx, (dequant_diff_kernel<BITS_><<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(
             codes_x, delta_x, s->x_snap, c.d, ctx->xhat_diff)));
         ctx->launches += 1;
     }
     if (D.format == DQ_CSR_F32) {
-        cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        if (!ctx->alpha_zeroed) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         worker_grad_csr_kernel<<<(int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st>>>(
             (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha);
     } else {
         dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
-        if (grid.x > 1) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        if (grid.x > 1 && !ctx->alpha_zeroed) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         const bool f32 = D.format == DQ_DENSE_F32;
         const bool vec = (c.d % (f32 ? 4 : 8)) == 0 && (reinterpret_cast<uintptr_t>(alpha) & 15) == 0;   // data is 16-byte aligned by contract
         if (f32 && vec)

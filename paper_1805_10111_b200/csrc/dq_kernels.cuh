@@ -8,7 +8,8 @@ namespace dq {
 void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* norm_bits, cudaStream_t st);
 void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
-                          uint32_t stream_id, cudaStream_t st, const float* ref = nullptr, float* diff = nullptr);
+                          uint32_t stream_id, cudaStream_t st, const float* ref = nullptr, float* diff = nullptr,
+                          float* zero_f = nullptr, int64_t zero_n = 0, uint32_t* zero_u = nullptr, int zero_un = 0);
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
 void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,
