@@ -130,6 +130,38 @@ __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restri
     }
 }
 
+// The same sum over an ascending list of groups (all other coordinates are zero).
+__global__ void __launch_bounds__(kThreads) norm_l1_list_kernel(const float* __restrict__ v, int64_t d, int vec_ok, GroupList gl,
+                                                                const uint32_t* __restrict__ norm_bits,
+                                                                unsigned long long* __restrict__ l1_sum)
+{
+    const int w = blockIdx.y;
+    const uint32_t nb = norm_bits[w];
+    if (nb == 0u || nb >= 0x7F800000u) return;
+    int e; (void)frexpf(__uint_as_float(nb), &e);
+    const double scale = ldexp(1.0, 35 - e);
+    const float* row = v + (int64_t)w * d;
+    unsigned long long acc = 0;
+    const int64_t n = gl.count[w];
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i0 = (int64_t)gl.groups[(int64_t)w * gl.cap + p] << 3;
+        float a[8];
+        if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], scale);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+    __shared__ unsigned long long s_acc[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) s_acc[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long t = 0;
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) t += s_acc[i];
+        if (t) atomicAdd(l1_sum + w, t);
+    }
+}
+
 // Per-worker constants of eq. (4) with Lemma 2's probabilities, from the two norms.
 struct SparsifyScale { float s; bool empty; };
 
@@ -178,7 +210,7 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
                       const unsigned long long* __restrict__ l1_sum, float phi,
                       const __grid_constant__ PhiloxKeys K, uint32_t round,
                       uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
-                      int64_t nchunks, const RoundParams* __restrict__ rp)
+                      int64_t nchunks, const RoundParams* __restrict__ rp, GroupList gl)
 {
     if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
@@ -187,13 +219,14 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     uint32_t bmax = 0;
+    const int64_t nch_eff = gl.groups ? ((int64_t)gl.count[w] + kChunk / 8 - 1) / (kChunk / 8) : nchunks;   // chunks that hold groups
     for (int64_t c = warp; c < nchunks; c += nwarps) {
         uint32_t cnt = 0;
-        if (!sc.empty) {
+        if (!sc.empty && c < nch_eff) {
 #pragma unroll 2
             for (int it = 0; it < kChunk / 256; ++it) {
-                const int64_t g = c * (kChunk / 8) + it * 32 + lane, i0 = g << 3;
-                if (i0 >= d) break;
+                const int64_t g = group_at(gl, w, c * (kChunk / 8) + it * 32 + lane, d), i0 = g << 3;
+                if (g < 0) break;
                 float a[8], beta[8];
                 if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
                 uint32_t r[4];
@@ -261,7 +294,8 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      const uint32_t* __restrict__ beta_norm_bits, const uint32_t* __restrict__ chunk_off,
                      int64_t nchunks, int64_t ngroups,
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
-                     uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status, const RoundParams* __restrict__ rp)
+                     uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status, const RoundParams* __restrict__ rp,
+                     GroupList gl)
 {
     if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
@@ -279,15 +313,17 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
     uint32_t* oidx = SPARSE_OUT ? idx + (int64_t)w * cap : nullptr;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    for (int64_t c = warp; c < nchunks; c += nwarps) {
+    const int64_t nch_eff = (SPARSE_OUT && gl.groups) ? ((int64_t)gl.count[w] + kChunk / 8 - 1) / (kChunk / 8) : nchunks;
+    for (int64_t c = warp; c < nch_eff; c += nwarps) {
         uint32_t pos = SPARSE_OUT ? chunk_off[(int64_t)w * (nchunks + 1) + c] : 0u;
         for (int it = 0; it < kChunk / 256; ++it) {
-            const int64_t g = c * (kChunk / 8) + it * 32 + lane, i0 = g << 3;
+            const int64_t pos_g = c * (kChunk / 8) + it * 32 + lane;
+            const int64_t g = SPARSE_OUT ? group_at(gl, w, pos_g, d) : pos_g, i0 = g << 3;
             uint32_t mask = 0;
             uint32_t s8[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) s8[j] = 128u << 16;                        // code 0
-            if (!sc.empty && i0 < d) {
+            if (!sc.empty && g >= 0 && i0 < d) {
                 float a[8], beta[8];
                 if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
                 uint32_t r[4];
@@ -579,6 +615,69 @@ __global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const fl
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Sparse gradients.  The worker kernel marks every group of eight coordinates it adds to in a bitmap.
+// build_group_list turns each worker's bitmap into the ascending list of those groups, clears the bitmap
+// and folds ||alpha_w||_inf over the listed groups (all other coordinates are zero).  One block per worker.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const float* __restrict__ alpha, int64_t d, int vec_ok,
+                        uint32_t* __restrict__ glist, int64_t cap, uint32_t* __restrict__ gcount, uint32_t* __restrict__ norm_bits)
+{
+    const int w = blockIdx.x;
+    uint32_t* bm = touched + (int64_t)w * bm_words;
+    uint32_t* list = glist + (int64_t)w * cap;
+    const float* row = alpha + (int64_t)w * d;
+    __shared__ uint32_t s_warp[kThreads / 32];
+    __shared__ uint32_t s_carry;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    uint32_t nmax = 0;
+    for (int64_t base = 0; base < bm_words; base += blockDim.x) {
+        const int64_t i = base + threadIdx.x;
+        uint32_t word = 0;
+        if (i < bm_words) { word = bm[i]; if (word) bm[i] = 0u; }
+        const uint32_t c = __popc(word);
+        uint32_t incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if ((threadIdx.x & 31) >= o) incl += t; }
+        if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
+        __syncthreads();
+        uint32_t pos = s_carry + incl - c;
+        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) pos += s_warp[k];
+        const uint32_t last = pos + c;
+        while (word) {
+            const int bit = __ffs(word) - 1; word &= word - 1;
+            const int64_t g = (i << 5) + bit, i0 = g << 3;
+            list[pos++] = (uint32_t)g;
+            float a[8];
+            if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) nmax = max(nmax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
+        }
+        __syncthreads();
+        if (threadIdx.x == blockDim.x - 1) s_carry = last;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) gcount[w] = s_carry;
+    block_atomic_max(nmax, norm_bits + w);
+}
+
+// Puts back zeros in the groups listed by the previous round, so that alpha is all-zero again.  grid (blocks, M).
+__global__ void __launch_bounds__(kThreads)
+clear_listed_groups_kernel(float* __restrict__ alpha, int64_t d, const uint32_t* __restrict__ glist, int64_t cap,
+                           const uint32_t* __restrict__ gcount)
+{
+    const int w = blockIdx.y;
+    float* row = alpha + (int64_t)w * d;
+    const int64_t n = gcount[w];
+    for (int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; p < n; p += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i0 = (int64_t)glist[(int64_t)w * cap + p] << 3;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) if (i0 + j < d) row[i0 + j] = 0.0f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Host launchers
 // ---------------------------------------------------------------------------------------------------
 static inline int grid_for(int64_t items_per_thread_units, int sm_count, int per_sm = 8)
@@ -618,31 +717,54 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     ctx->launches += 1;
 }
 
+void launch_clear_listed(dq_ctx* ctx, cudaStream_t st)
+{
+    dim3 grid(16, ctx->cfg.M);
+    clear_listed_groups_kernel<<<grid, kThreads, 0, st>>>(ctx->alpha, ctx->cfg.d, ctx->glist, ctx->glist_cap, ctx->gcount);
+    ctx->launches += 1;
+}
+
+void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg;
+    if (!ctx->ninf_zeroed) cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * c.M, st);
+    build_group_list_kernel<<<c.M, kThreads, 0, st>>>(ctx->touched, ctx->bm_words, ctx->alpha, c.d, vec_ok_for(ctx->alpha, c.d),
+                                                        ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
+    ctx->launches += 1;
+}
+
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st)
 {
     const int vec_ok = vec_ok_for(v, d);
     const int64_t nchunks = (d + kChunk - 1) / kChunk;
+    const bool list = ctx->list_ready && sparse_out && v == ctx->alpha;     // only the listed groups can be nonzero
+    const GroupList gl = list ? GroupList{ctx->glist, ctx->gcount, ctx->glist_cap} : GroupList{nullptr, nullptr, 0};
     cudaMemsetAsync(ctx->l1_sum, 0, sizeof(unsigned long long) * M, st);
     cudaMemsetAsync(ctx->beta_norm_bits, 0, sizeof(uint32_t) * M, st);
-    dim3 grid_l1(grid_for((d + 7) / 8, ctx->sm_count), M);
-    norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
-    dim3 grid_c(grid_for(nchunks * 32, ctx->sm_count), M);
+    if (list) {
+        norm_l1_list_kernel<<<dim3(16, M), kThreads, 0, st>>>(v, d, vec_ok, gl, norm_bits, ctx->l1_sum);
+    } else {
+        dim3 grid_l1(grid_for((d + 7) / 8, ctx->sm_count), M);
+        norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
+    }
+    dim3 grid_c(list ? 16 : grid_for(nchunks * 32, ctx->sm_count), M);
     sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
-                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks, ctx->rp_active);
+                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks,
+                                                       ctx->rp_active, gl);
     ctx->launches += 2;
     if (sparse_out) {
         chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
         cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
-            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active)));
+            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl)));
         ctx->launches += 2;
     } else {
         const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
-            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active)));
+            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl)));
         ctx->launches += 1;
     }
 }

@@ -145,6 +145,17 @@ __device__ __forceinline__ void block_atomic_max(uint32_t v, uint32_t* dst)
 
 struct ProxParams { float lambda1, lambda2, lo, hi; };
 
+// Where the sparsifier finds its groups of eight coordinates: every group of the vector (groups == NULL), or
+// an ascending list of the groups that can hold a nonzero (groups [M][cap], count [M]).
+struct GroupList { const uint32_t* groups; const uint32_t* count; int64_t cap; };
+
+// Group at position p of worker w, or -1 past the end.
+__device__ __forceinline__ int64_t group_at(const GroupList& gl, int w, int64_t p, int64_t d)
+{
+    if (!gl.groups) return ((p << 3) < d) ? p : -1;
+    return (p < (int64_t)gl.count[w]) ? (int64_t)gl.groups[(int64_t)w * gl.cap + p] : -1;
+}
+
 // Transmitted-bit counters of a round, written by the master kernel when `down` is set (Section 3.1 message sizes).
 struct BitsArgs { uint64_t* down; uint64_t* up; const uint32_t* nnz; int flag_round, sparse_msgs, bx, b; };
 
@@ -207,6 +218,10 @@ struct dq_ctx {
     uint64_t* graph_bits[2];
     int64_t graph_launches;
     bool graph_off;
+    // sparse gradients (CSR data, sparse messages): bitmap of touched groups, their ascending list, its length
+    uint32_t* touched; uint32_t* glist; uint32_t* gcount; int64_t bm_words; int64_t glist_cap;
+    bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only
+    bool list_ready;            // the list of this round has been built (consumed by the sparsifier launch)
     bool alpha_zeroed, ninf_zeroed, normx_zeroed;   // an earlier kernel of this round already cleared these
     bool diff_ready;            // the model-quantise kernel of this round already wrote xhat - xsnap
     // bookkeeping

@@ -107,7 +107,8 @@ __global__ void dequant_diff_kernel(const uint8_t* __restrict__ codes, const flo
 __global__ void __launch_bounds__(kThreads)
 worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict__ col, const int64_t* __restrict__ row_ptr,
                        const float* __restrict__ labels, const float* __restrict__ diff, const float* __restrict__ z_snap,
-                       const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, float* __restrict__ alpha)
+                       const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, float* __restrict__ alpha,
+                       uint32_t* __restrict__ touched /* bitmap of groups of eight coordinates, may be NULL */, int64_t bm_words)
 {
     clear_word(bs);
     const int lane = threadIdx.x & 31;
@@ -119,7 +120,16 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
     const float dz = (float)warp_dot_csr(val, col, k0, k1, diff, lane);
     const float r = slope_difference(labels[a], z_snap[a], dz) / (float)B;
     float* out = alpha + (int64_t)w * d;
-    for (int64_t k = k0 + lane; k < k1; k += 32) atomicAdd(out + __ldg(col + k), r * __ldg(val + k));
+    uint32_t* bm = touched ? touched + (int64_t)w * bm_words : nullptr;
+    for (int64_t k = k0 + lane; k < k1; k += 32) {
+        const int32_t c = __ldg(col + k);
+        atomicAdd(out + c, r * __ldg(val + k));
+        if (bm) {
+            const uint32_t bit = 1u << ((c >> 3) & 31);
+            uint32_t* word = bm + (c >> 8);
+            if (!(*reinterpret_cast<volatile uint32_t*>(word) & bit)) atomicOr(word, bit);
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -448,11 +458,14 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
                         uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st)
 {
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    const bool list = ctx->list_mode && alpha == ctx->alpha;   // sparse gradients tracked as a list of touched groups
     if (is_snapshot) {                     // xhat = xsnap: every slope difference is exactly zero
         cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         cudaMemsetAsync(norm_inf, 0, sizeof(float) * c.M, st);
+        if (list) cudaMemsetAsync(ctx->gcount, 0, sizeof(uint32_t) * c.M, st);
         return;
     }
+    if (list) launch_clear_listed(ctx, st);                      // alpha is all-zero again before this round adds to it
     const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n,
                             ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr};
     if (!ctx->diff_ready) {
@@ -461,9 +474,10 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         ctx->launches += 1;
     }
     if (D.format == DQ_CSR_F32) {
-        if (!ctx->alpha_zeroed) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        if (!ctx->alpha_zeroed && !list) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         worker_grad_csr_kernel<<<(int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha);
+            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha,
+            list ? ctx->touched : nullptr, ctx->bm_words);
     } else {
         dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
         if (grid.x > 1 && !ctx->alpha_zeroed) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
@@ -479,7 +493,8 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
             worker_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
     }
     ctx->launches += 1;
-    launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
+    if (list) { launch_build_group_list(ctx, reinterpret_cast<uint32_t*>(norm_inf), st); ctx->list_ready = true; }
+    else launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
 }
 
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)

@@ -12,6 +12,8 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
                           float* zero_f = nullptr, int64_t zero_n = 0, uint32_t* zero_u = nullptr, int zero_un = 0);
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
+void launch_clear_listed(dq_ctx* ctx, cudaStream_t st);
+void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st);
 void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,
                    const BitsArgs* bits = nullptr);
 void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, float* out, cudaStream_t st);
