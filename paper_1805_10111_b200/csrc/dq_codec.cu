@@ -94,9 +94,16 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
 // ||alpha_w||_1 on an integer grid (order-free): with ||alpha||_inf in [2^(e-1), 2^e) each |alpha_i| is
 // scaled by 2^(35-e), truncated, and the integers are added.  l1_sum must be zero on entry.
 // ---------------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned long long l1_term(float a, double scale)
+// trunc(|a| * 2^(35-e)) in integer arithmetic: the 24-bit significand shifted by the exponent distance.
+// (|a| < 2^e, so the result is below 2^35; bits that fall off the right end are the truncation.)
+__device__ __forceinline__ unsigned long long l1_term(float a, int e)
 {
-    return __double2ull_rz((double)fabsf(a) * scale);
+    const uint32_t bits = __float_as_uint(a) & 0x7FFFFFFFu;
+    uint32_t ex = bits >> 23, mant = bits & 0x007FFFFFu;
+    if (ex != 0u) mant |= 0x00800000u; else ex = 1u;                 // subnormals have no hidden bit
+    const int sh = (int)ex - 115 - e;                                // value = mant * 2^(ex-150); times 2^(35-e)
+    if (sh >= 0) return (unsigned long long)mant << sh;              // sh <= 11
+    return (sh > -24) ? (unsigned long long)(mant >> (-sh)) : 0ull;
 }
 
 __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restrict__ v, int64_t d, int vec_ok,
@@ -107,7 +114,6 @@ __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restri
     const uint32_t nb = norm_bits[w];
     if (nb == 0u || nb >= 0x7F800000u) return;
     int e; (void)frexpf(__uint_as_float(nb), &e);
-    const double scale = ldexp(1.0, 35 - e);
     const float* row = v + (int64_t)w * d;
     unsigned long long acc = 0;
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (int64_t)gridDim.x * blockDim.x;
@@ -115,9 +121,9 @@ __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restri
     for (int64_t g = tid; g < ng; g += nth) {
         float a[8]; load8(row + (g << 3), a);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], scale);
+        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], e);
     }
-    for (int64_t i = (ng << 3) + tid; i < d; i += nth) acc += l1_term(__ldg(row + i), scale);
+    for (int64_t i = (ng << 3) + tid; i < d; i += nth) acc += l1_term(__ldg(row + i), e);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
     __shared__ unsigned long long s_acc[kThreads / 32];
@@ -139,7 +145,6 @@ __global__ void __launch_bounds__(kThreads) norm_l1_list_kernel(const float* __r
     const uint32_t nb = norm_bits[w];
     if (nb == 0u || nb >= 0x7F800000u) return;
     int e; (void)frexpf(__uint_as_float(nb), &e);
-    const double scale = ldexp(1.0, 35 - e);
     const float* row = v + (int64_t)w * d;
     unsigned long long acc = 0;
     const int64_t n = gl.count[w];
@@ -148,7 +153,7 @@ __global__ void __launch_bounds__(kThreads) norm_l1_list_kernel(const float* __r
         float a[8];
         if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], scale);
+        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], e);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
@@ -179,23 +184,29 @@ __device__ __forceinline__ SparsifyScale sparsify_scale(uint32_t nb, unsigned lo
     return r;
 }
 
-// m_i = p_i * 2^16 rounded up, p_i = min(1, |alpha_i| s).
-__device__ __forceinline__ uint32_t mask_threshold(float a, float s)
-{
-    const float scaled = ceilf(__fmul_rn(__fmul_rn(fabsf(a), s), 65536.0f));
-    return (scaled >= 65536.0f) ? 65536u : (uint32_t)scaled;
-}
-
-// Survivor mask of one group of eight coordinates and the survivors' beta_i = alpha_i / p_i.
+// Survivor mask of one group of eight coordinates and the survivors' beta_i = alpha_i / p_i, with
+// p_i = m_i / 2^16, m_i = min(2^16, ceil(|alpha_i| s 2^16)).  For an integer draw u, u < ceil(y) is the same
+// as u < y, so the test needs neither the rounding nor an integer conversion; the draw becomes a float by
+// placing it in the significand of 2^23.  m_i is only formed for the rare survivors.
 __device__ __forceinline__ uint32_t sparsify8(const float (&a)[8], float s, const uint32_t (&r)[4], float (&beta)[8])
 {
     uint32_t mask = 0;
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const uint32_t m = mask_threshold(a[j], s);
-        const bool z = half16(r, j) < m;
-        beta[j] = z ? __fdiv_rn(__fmul_rn(a[j], 65536.0f), (float)m) : 0.0f;
-        mask |= (uint32_t)z << j;
+        const float y = __fmul_rn(__fmul_rn(fabsf(a[j]), s), 65536.0f);
+        const float uf = __fsub_rn(__uint_as_float(0x4B000000u | half16(r, j)), 8388608.0f);
+        mask |= (uint32_t)(uf < y) << j;
+        beta[j] = 0.0f;
+    }
+    if (mask) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if ((mask >> j) & 1u) {
+                const float y = __fmul_rn(__fmul_rn(fabsf(a[j]), s), 65536.0f);
+                const float m = fminf(ceilf(y), 65536.0f);
+                beta[j] = __fdiv_rn(__fmul_rn(a[j], 65536.0f), m);
+            }
+        }
     }
     return mask;
 }
