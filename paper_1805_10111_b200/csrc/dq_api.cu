@@ -127,6 +127,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
         rc |= dev_alloc(&c->rows, (size_t)M * cfg->B);
         rc |= dev_alloc(&c->xhat_diff, (size_t)d);
         rc |= dev_alloc(&c->g64, (size_t)d);
+        rc |= dev_alloc(&c->rbuf, (size_t)M * cfg->B);
         c->list_mode = sparse && data->format == DQ_CSR_F32;
         if (c->list_mode) {
             c->glist_cap = (d + 7) / 8;
@@ -151,7 +152,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->rp_dev, c->touched, c->glist, c->gcount, c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -289,8 +290,8 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     if (!flag) {     // model quantisation that also emits xhat - xsnap for the workers
         launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, reinterpret_cast<const uint32_t*>(s->norm_x), ctx->codes_x,
                              dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx), ctx->delta_x, round, kMaster, kStreamModel, as_stream(st),
-                             s->x_snap, ctx->xhat_diff, ctx->list_mode ? nullptr : ctx->alpha,
-                             ctx->list_mode ? 0 : (int64_t)ctx->cfg.M * ctx->cfg.d,
+                             s->x_snap, ctx->xhat_diff, worker_accumulates(ctx) ? ctx->alpha : nullptr,
+                             worker_accumulates(ctx) ? (int64_t)ctx->cfg.M * ctx->cfg.d : 0,
                              reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
         ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = ctx->normx_zeroed = true;
     }

@@ -717,6 +717,7 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
     if (diff) {
+        grid.x = max(grid.x, (unsigned)grid_for(zero_n / 4, ctx->sm_count));   // enough blocks for the clearing loop too
         DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
             v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
             ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un)));

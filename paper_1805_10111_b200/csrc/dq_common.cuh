@@ -205,6 +205,7 @@ struct dq_ctx {
     float* delta_x;
     float* xhat_diff;           // [d] dequantised model minus snapshot
     double* g64;                // [d] full-gradient accumulator
+    float* rbuf;                // [M][B] slope differences of the sampled rows
     dq_msgs msgs;
     uint64_t* bits;             // [2] device counters
     // device-resident state for the host-buffer entry point

@@ -252,6 +252,75 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Dense worker gradient for large minibatches, in two kernels and without atomics:
+//   worker_margins_kernel   one warp per sampled row: slope difference r_{w,j} / B
+//   worker_colsum_kernel    block (column slab, worker): alpha_w[slab] = sum_j r_{w,j} a_j[slab], rows split over
+//                           the warps and combined in a fixed order, so alpha is reproducible bit for bit;
+//                           also folds ||alpha_w||_inf.  The rows were just read by the first kernel and are
+//                           served from L2.
+// ---------------------------------------------------------------------------------------------------
+template <class T>
+__global__ void __launch_bounds__(kThreads)
+worker_margins_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
+                      const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d,
+                      float* __restrict__ rbuf)
+{
+    clear_word(bs);
+    const int lane = threadIdx.x & 31;
+    const int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (slot >= (int64_t)M * B) return;
+    const int w = (int)(slot / B), j = (int)(slot % B);
+    const int64_t a = batch_row(bs, K, w, j, B, lane == 0);
+    const float dz = (float)warp_dot_dense_vec(X + a * d, diff, d, lane);
+    if (lane == 0) rbuf[slot] = slope_difference(labels[a], z_snap[a], dz) / (float)B;
+}
+
+template <class T>
+__global__ void __launch_bounds__(kThreads)
+worker_colsum_kernel(const T* __restrict__ X, const int32_t* __restrict__ rows, const float* __restrict__ rbuf, int B, int64_t d,
+                     float* __restrict__ alpha, uint32_t* __restrict__ norm_bits)
+{
+    constexpr int N = RowVec<T>::N;
+    constexpr int kWarps = kThreads / 32;
+    __shared__ float s_part[kWarps][32 * N];
+    extern __shared__ float s_r[];                 // [B] slope differences, then [B] row indices as int32
+    int32_t* s_row = reinterpret_cast<int32_t*>(s_r + B);
+    const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int j = threadIdx.x; j < B; j += blockDim.x) { s_r[j] = rbuf[(int64_t)w * B + j]; s_row[j] = rows[(int64_t)w * B + j]; }
+    __syncthreads();
+    const int nv = (int)(d / N);
+    const int v = blockIdx.x * 32 + lane;          // this lane's 16-byte column group
+    float acc[N];
+#pragma unroll
+    for (int q = 0; q < N; ++q) acc[q] = 0.0f;
+    if (v < nv) {
+#pragma unroll 8
+        for (int j = warp; j < B; j += kWarps) {
+            float f[N];
+            RowVec<T>::unpack(__ldg(reinterpret_cast<const uint4*>(X + (int64_t)s_row[j] * d) + v), f);
+            const float r = s_r[j];
+#pragma unroll
+            for (int q = 0; q < N; ++q) acc[q] = fmaf(r, f[q], acc[q]);
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < N; ++q) s_part[warp][lane * N + q] = acc[q];
+    __syncthreads();
+    uint32_t nmax = 0;
+    for (int c = threadIdx.x; c < 32 * N; c += blockDim.x) {
+        const int64_t i = (int64_t)blockIdx.x * 32 * N + c;
+        if (i < d) {
+            float sum = 0.0f;
+#pragma unroll
+            for (int k = 0; k < kWarps; ++k) sum += s_part[k][c];
+            alpha[(int64_t)w * d + i] = sum;
+            nmax = max(nmax, __float_as_uint(sum) & 0x7FFFFFFFu);
+        }
+    }
+    block_atomic_max(nmax, norm_bits + w);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Full gradient over all n rows at xsnap, accumulated in double; also stores the margins z_snap.
 // ---------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
@@ -454,6 +523,16 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
     ctx->launches += 3;
 }
 
+// Whether the worker stage accumulates into alpha with atomics (and so needs it cleared first).
+bool worker_accumulates(const dq_ctx* ctx)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    if (D.format == DQ_CSR_F32) return !ctx->list_mode;
+    const bool vec = (c.d % (D.format == DQ_DENSE_F32 ? 4 : 8)) == 0;
+    if (vec && c.B >= 64) return false;                        // column sums are stored, not added
+    return (c.B + kRowsPerBlock - 1) / kRowsPerBlock > 1;
+}
+
 void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot, const dq_state* s,
                         uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st)
 {
@@ -480,10 +559,30 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
             list ? ctx->touched : nullptr, ctx->bm_words);
     } else {
         dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
-        if (grid.x > 1 && !ctx->alpha_zeroed) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         const bool f32 = D.format == DQ_DENSE_F32;
         const bool vec = (c.d % (f32 ? 4 : 8)) == 0 && (reinterpret_cast<uintptr_t>(alpha) & 15) == 0;   // data is 16-byte aligned by contract
-        if (f32 && vec)
+        if (grid.x > 1 && !ctx->alpha_zeroed && !(vec && c.B >= 64)) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
+        if (vec && c.B >= 64) {        // large minibatch: margins, then atomics-free column sums with the norm folded in
+            const int32_t* rows_eff = batch_idx ? batch_idx : ctx->rows;
+            uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
+            if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
+            const int gm = (int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads);
+            const size_t smem = sizeof(float) * 2 * c.B;
+            if (f32) {
+                worker_margins_kernel<float><<<gm, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap,
+                                                                       ctx->keys, bs, c.M, c.B, c.d, ctx->rbuf);
+                dim3 gc((unsigned)((c.d / 4 + 31) / 32), c.M);
+                worker_colsum_kernel<float><<<gc, kThreads, smem, st>>>((const float*)D.values, rows_eff, ctx->rbuf, c.B, c.d, alpha, nb);
+            } else {
+                worker_margins_kernel<__nv_bfloat16><<<gm, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff,
+                                                                               s->z_snap, ctx->keys, bs, c.M, c.B, c.d, ctx->rbuf);
+                dim3 gc((unsigned)((c.d / 8 + 31) / 32), c.M);
+                worker_colsum_kernel<__nv_bfloat16><<<gc, kThreads, smem, st>>>((const __nv_bfloat16*)D.values, rows_eff, ctx->rbuf, c.B,
+                                                                                 c.d, alpha, nb);
+            }
+            ctx->launches += 2;
+            return;
+        } else if (f32 && vec)
             worker_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else if (f32)
             worker_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);

@@ -152,6 +152,41 @@ def test_worker_gradient(dq, name, bx):
     dq.dq_destroy(ctx)
 
 
+@pytest.mark.parametrize("name", ["bf16", "dense8"])
+def test_worker_gradient_large_minibatch(dq, name):
+    """B >= 64 takes the two-kernel dense path (margins, then column sums without atomics): reproducible bit for bit."""
+    import torch
+    h = _problem(name)
+    M, B, seed, rnd, bx = 2, 70, 31, 8, 8
+    xs = synth.normal_vector(h.d, 76, 0.3)
+    x = (xs + synth.normal_vector(h.d, 77, 0.02)).astype(F32)
+    cfg = dq.make_config(h.d, M, B=B, bx=bx, seed=seed)
+    data = dq.Data(h)
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+    st = dq.State(xs, n=h.n)
+    assert dq.dq_epoch_begin(ctx, st) == 0
+    cx, dx, _ = oracle.quantize(x, bx, seed, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+    xhat = cx.astype(F32) * dx
+    codes_x = _dev(oracle.pack(cx, bx)); delta_x = _dev(np.array([dx], F32))
+    alpha = torch.full((M, h.d), 3.0, device="cuda"); ninf = torch.zeros(M, device="cuda")
+    assert dq.dq_worker_grad(ctx, codes_x, delta_x, 0, st, rnd, None, alpha, ninf) == 0
+    first = alpha.clone()
+    for w in range(M):
+        rows = oracle.sample_batch(seed, rnd, w, M, h.n, B)
+        a, S = oracle.worker_grad(_odata(h), xhat, xs, rows)
+        nbad, worst = _close(alpha[w].cpu().numpy(), a, S)
+        assert nbad == 0, (w, nbad, worst)
+        assert ninf[w].item() == np.abs(alpha[w].cpu().numpy()).max()
+    alpha.fill_(7.0)
+    assert dq.dq_worker_grad(ctx, codes_x, delta_x, 0, st, rnd, None, alpha, ninf) == 0
+    assert torch.equal(alpha, first)
+    mine = np.stack([(np.arange(B) * 7 + w) % h.n for w in range(M)]).astype(np.int32)
+    assert dq.dq_worker_grad(ctx, codes_x, delta_x, 0, st, rnd, _dev(mine), alpha, ninf) == 0
+    a, S = oracle.worker_grad(_odata(h), xhat, xs, mine[1].astype(np.int64))
+    assert _close(alpha[1].cpu().numpy(), a, S)[0] == 0
+    dq.dq_destroy(ctx)
+
+
 class Lockstep:
     """Runs the GPU library and the oracle side by side, restarting the GPU from the oracle's state every round."""
 
