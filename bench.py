@@ -146,6 +146,21 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value, dist=None, device="cpu"):
+    """The slowest rank's time: every rank must have finished before the job has."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world, steps, slowest_ms):
+    """Replicas are independent: the job processed world * steps rounds in the slowest rank's time."""
+    return world * steps / (slowest_ms / 1000.0)
+
+
 def measured_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -298,10 +313,9 @@ def run_ours(a):
     rc, status = dq.dq_poll_status(ctx)
     assert rc == 0 and status == 0, "device status %d" % status
     stage_ms = [sum(events[k][i].elapsed_time(events[k][i + 1]) for k in range(a.steps)) / a.steps for i in range(4)]
-    if dist is not None:
-        t = torch.tensor([total_ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); total_ms = t.item()
+    total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / a.steps
-    value = world * a.steps / (total_ms / 1000.0)
+    value = whole_job_rate(world, a.steps, total_ms)
 
     # end to end through the host-buffer entry point: H2D of the M gradient vectors, the round, D2H of the model codes
     e2e = None
@@ -315,8 +329,7 @@ def run_ours(a):
             dq.ok(dq.dq_codec_round_host(ctx, hv, 2000 + k, eta, hcodes, hdelta))
         torch.cuda.synchronize()
         e2e_s = time.perf_counter() - t0
-        if dist is not None:
-            t = torch.tensor([e2e_s], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); e2e_s = t.item()
+        e2e_s = max_over_ranks(e2e_s, dist, "cuda")
         e2e = {"value": world * a.e2e_steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": M * d * 4,
                "d2h_bytes_per_step": nbx + 4, "steps": a.e2e_steps}
 
