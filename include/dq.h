@@ -138,7 +138,8 @@ int dq_norm_inf(dq_ctx* ctx, const float* v, int M, float* norm_inf, void* strea
 
 /* Worker steps 12(-13) for all M workers: optional sparsification by eq. (4) with Lemma 2's probabilities,
  * then delta = ||.||_inf / (2^(b-1)-1), Q_(delta,b), and bit packing into `out`.
- * v [M][d]; norm_inf [M] = ||v_w||_inf as produced by dq_worker_grad, or NULL to have it computed. */
+ * v [M][d]; norm_inf [M] = ||v_w||_inf exactly as produced by dq_worker_grad or dq_norm_inf, or NULL to have it
+ * computed.  A value below the true maximum gives unspecified codes for the coordinates that exceed it. */
 int dq_quantize_sparsify_pack(dq_ctx* ctx, const float* v, const float* norm_inf, uint32_t round,
                               dq_msgs* out, void* stream);
 

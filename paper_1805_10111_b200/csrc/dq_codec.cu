@@ -483,20 +483,47 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
                 load8_rw((ACC ? y : x) + i0 + q * 8, *reinterpret_cast<float(*)[8]>(curp + q * 8));
             }
         }
-        for (int w0 = 0; w0 < M; w0 += 8) {                 // eight code words in flight per thread
-            uint32_t wd[8][W];
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t* wp = words + (int64_t)min(w0 + k, M - 1) * wstride;    // clamped: always a valid row
-                if (W == 2) { const uint2 u = __ldg(reinterpret_cast<const uint2*>(wp) + t); wd[k][0] = u.x; wd[k][W - 1] = u.y; }
-                else wd[k][0] = __ldg(wp + t);
+        if (BITS == 4) {      // the two loop shapes compute the same thing; each bit width uses the one that the
+                              // compiler schedules better (measured: registers and load placement differ)
+            const uint32_t* wp = words + t * W;
+            int w0 = 0;
+            for (; w0 + 8 <= M; w0 += 8) {                       // full batches: eight code words in flight, no predicates
+                uint32_t wd[8][W];
+    #pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (W == 2) { const uint2 u = __ldg(reinterpret_cast<const uint2*>(wp)); wd[k][0] = u.x; wd[k][W - 1] = u.y; }
+                    else wd[k][0] = __ldg(wp);
+                    wp += wstride;
+                }
+    #pragma unroll
+                for (int k = 0; k < 8; ++k) {
+    #pragma unroll
+                    for (int q = 0; q < W; ++q) accumulate_word<BITS>(wd[k][q], s_scale[w0 + k], acc[q]);
+                }
             }
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                if (w0 + k < M) {
-#pragma unroll
-                    for (int q = 0; q < W; ++q)
-                        accumulate_word<BITS>(wd[k][q], s_scale[w0 + k], acc[q]);
+            for (; w0 < M; ++w0) {                               // remaining workers
+                uint32_t wd[W];
+                if (W == 2) { const uint2 u = __ldg(reinterpret_cast<const uint2*>(wp)); wd[0] = u.x; wd[W - 1] = u.y; }
+                else wd[0] = __ldg(wp);
+                wp += wstride;
+    #pragma unroll
+                for (int q = 0; q < W; ++q) accumulate_word<BITS>(wd[q], s_scale[w0], acc[q]);
+            }
+        } else {
+            for (int w0 = 0; w0 < M; w0 += 8) {             // batches of eight code words in flight; rows clamped, tail predicated
+                uint32_t wd[8][W];
+    #pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint32_t* wq = words + (int64_t)min(w0 + k, M - 1) * wstride;
+                    if (W == 2) { const uint2 u = __ldg(reinterpret_cast<const uint2*>(wq) + t); wd[k][0] = u.x; wd[k][W - 1] = u.y; }
+                    else wd[k][0] = __ldg(wq + t);
+                }
+    #pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (w0 + k < M) {
+    #pragma unroll
+                        for (int q = 0; q < W; ++q) accumulate_word<BITS>(wd[k][q], s_scale[w0 + k], acc[q]);
+                    }
                 }
             }
         }

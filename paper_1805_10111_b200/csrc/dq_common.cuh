@@ -51,12 +51,14 @@ constexpr __host__ __device__ int levels(int bits) { return (1 << (bits - 1)) - 
 // fp32 spacing is 2^-15, so bits(r) is (v*inv + 128) * 2^15 plus a constant.  Doubling it and adding the
 // raw 16-bit draw h = 2u + c puts floor(((v*inv + 128) * 2^15 + u) / 2^15) into byte 2 of the result;
 // the constant only touches bits above byte 2.  Returns that word; byte 2 is the code plus 128.
+// No clamp is needed: inv is 1/delta rounded toward zero and |v| <= ||v||_inf, so |v*inv| <= 2^(b-1)-1 and
+// Section 3.1's rule (ii) (values outside the hull) cannot fire.  A caller-supplied norm below the true
+// maximum breaks that premise and gives unspecified (but in-range, memory-safe) codes for the offending
+// coordinates.
 template <int BITS>
 __device__ __forceinline__ uint32_t round_fixed(float v, float inv, uint32_t h16)
 {
-    float r = __fmaf_rn(v, inv, 384.0f);
-    r = fminf(fmaxf(r, 384.0f - (float)(1 << (BITS - 1))), 384.0f + (float)levels(BITS));
-    return (__float_as_uint(r) << 1) + h16;
+    return (__float_as_uint(__fmaf_rn(v, inv, 384.0f)) << 1) + h16;
 }
 
 // Packs the codes held in byte 2 of s[0..7] into BITS-bit two's complement, coordinate 0 lowest.
