@@ -177,6 +177,21 @@ def test_master_dense_bit_exact(dq, b, reg):
         dq.dq_destroy(ctx)
 
 
+@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("M", [1, 8, 19, 33])
+def test_master_dense_worker_counts(dq, b, M):
+    """Worker counts around the batches of eight that the master kernel keeps in flight (none, exact, remainder)."""
+    d, seed = 4104, 17
+    v = _vectors(M, d, 100 + M, outliers=False)
+    cfg = dq.make_config(d, M, b=b, seed=seed, lambda1=1e-3, lambda2=0.01)
+    rc, ctx = dq.dq_create(cfg); assert rc == 0
+    msgs = dq.Msgs(cfg)
+    assert dq.dq_quantize_sparsify_pack(ctx, _dev(v), None, 2, msgs) == 0
+    _, delta, raw = _oracle_dense_msgs(v, b, seed, 2, msgs.stride)
+    _run_master(dq, cfg, raw, delta, synth.normal_vector(d, 50), synth.normal_vector(d, 51), 0.21, msgs=msgs, ctx=ctx)
+    dq.dq_destroy(ctx)
+
+
 def _oracle_sparse(v, b, phi, seed, rnd):
     M, d = v.shape
     out = []

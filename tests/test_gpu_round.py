@@ -338,6 +338,21 @@ def test_lockstep_accelerated_small(dq):
     ls.close()
 
 
+def test_lockstep_accelerated_sparse(dq):
+    """Momentum acceleration composed with sparsification (the paper notes Algorithm 3 applies to Algorithm 2 as well)."""
+    h = _problem("csr")
+    kw = dict(M=4, B=16, bx=8, b=4, box_lo=-2.0, box_hi=2.0, accelerated=1, sparsify=1, phi=0.0, msg_format=1, seed=12)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 78, 0.05), **kw)
+    rnd = 0
+    for s in range(1, 3):
+        theta = F32(2.0 / (s + 2)); eta = F32(0.3) / theta
+        ls.epoch(theta)
+        for t in range(8):
+            ls.round(rnd, eta, theta)
+            rnd += 1
+    ls.close()
+
+
 def _full_config(name):
     if name == "c1":
         return dict(M=4, B=16, bx=8, b=8, lambda1=1e-4, seed=101), 1.0, 200
