@@ -106,7 +106,9 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     rc |= dev_alloc(&c->norm_bits, M);
     rc |= dev_alloc(&c->beta_norm_bits, M);
     rc |= dev_alloc(&c->l1_sum, M);
-    rc |= dev_alloc(&c->chunk_off, cfg->sparsify ? (size_t)M * (c->nchunks + 1) : 1);
+    // offset table of the sparsifier: one entry per chunk; list mode uses chunks of 32 groups (256 coordinates)
+    const int64_t chunk_slots = (d + 255) / 256 + 1;
+    rc |= dev_alloc(&c->chunk_off, cfg->sparsify ? (size_t)M * chunk_slots : 1);
     rc |= dev_alloc(&c->tile_ptr, sparse ? (size_t)M * (c->nchunks + 1) : 1);
     rc |= dev_alloc(&c->xnorm_bits, 1);
     rc |= dev_alloc(&c->status, 1);

@@ -221,7 +221,7 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
                       const unsigned long long* __restrict__ l1_sum, float phi,
                       const __grid_constant__ PhiloxKeys K, uint32_t round,
                       uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
-                      int64_t nchunks, const RoundParams* __restrict__ rp, GroupList gl)
+                      int64_t nchunks, const RoundParams* __restrict__ rp, GroupList gl, int iters /* warp steps per chunk */)
 {
     if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
@@ -230,13 +230,14 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     uint32_t bmax = 0;
-    const int64_t nch_eff = gl.groups ? ((int64_t)gl.count[w] + kChunk / 8 - 1) / (kChunk / 8) : nchunks;   // chunks that hold groups
+    const int64_t gpc = 32 * (int64_t)iters;                                       // groups per chunk
+    const int64_t nch_eff = gl.groups ? ((int64_t)gl.count[w] + gpc - 1) / gpc : nchunks;   // chunks that hold groups
     for (int64_t c = warp; c < nchunks; c += nwarps) {
         uint32_t cnt = 0;
         if (!sc.empty && c < nch_eff) {
 #pragma unroll 2
-            for (int it = 0; it < kChunk / 256; ++it) {
-                const int64_t g = group_at(gl, w, c * (kChunk / 8) + it * 32 + lane, d), i0 = g << 3;
+            for (int it = 0; it < iters; ++it) {
+                const int64_t g = group_at(gl, w, c * gpc + it * 32 + lane, d), i0 = g << 3;
                 if (g < 0) break;
                 float a[8], beta[8];
                 if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
@@ -306,9 +307,10 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      int64_t nchunks, int64_t ngroups,
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
                      uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status, const RoundParams* __restrict__ rp,
-                     GroupList gl)
+                     GroupList gl, int iters)
 {
     if (rp) round = rp->round;
+    const int64_t gpc = 32 * (int64_t)iters;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
     const uint32_t bb = beta_norm_bits[w];
@@ -324,11 +326,11 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
     uint32_t* oidx = SPARSE_OUT ? idx + (int64_t)w * cap : nullptr;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int64_t nch_eff = (SPARSE_OUT && gl.groups) ? ((int64_t)gl.count[w] + kChunk / 8 - 1) / (kChunk / 8) : nchunks;
+    const int64_t nch_eff = (SPARSE_OUT && gl.groups) ? ((int64_t)gl.count[w] + gpc - 1) / gpc : nchunks;
     for (int64_t c = warp; c < nch_eff; c += nwarps) {
         uint32_t pos = SPARSE_OUT ? chunk_off[(int64_t)w * (nchunks + 1) + c] : 0u;
-        for (int it = 0; it < kChunk / 256; ++it) {
-            const int64_t pos_g = c * (kChunk / 8) + it * 32 + lane;
+        for (int it = 0; it < iters; ++it) {
+            const int64_t pos_g = c * gpc + it * 32 + lane;
             const int64_t g = SPARSE_OUT ? group_at(gl, w, pos_g, d) : pos_g, i0 = g << 3;
             uint32_t mask = 0;
             uint32_t s8[8];
@@ -591,16 +593,21 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
     if (rp) { eta = rp->eta; theta = rp->theta; }
     if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     __shared__ float s_acc[kChunk];
+    extern __shared__ uint32_t s_seg[];                          // [M][2] list segment of each worker in the tile
     const float inv_m = __fdiv_rn(1.0f, (float)M);
     const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
     uint32_t nmax = 0;
     for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
         const int64_t lo = tile * kChunk;
         for (int i = threadIdx.x; i < kChunk; i += blockDim.x) s_acc[i] = 0.0f;
-        __syncthreads();
-        for (int w = 0; w < M; ++w) {
+        for (int w = threadIdx.x; w < M; w += blockDim.x) {      // every worker's segment of this tile, fetched at once
             const uint32_t* tp = tile_ptr + (int64_t)w * (ntiles + 1) + tile;
-            const uint32_t e0 = tp[0], e1 = tp[1];
+            s_seg[2 * w] = tp[0]; s_seg[2 * w + 1] = tp[1];
+        }
+        __syncthreads();
+        for (int w = 0; w < M; ++w) {                            // worker order is the oracle's order of the fused adds
+            const uint32_t e0 = s_seg[2 * w], e1 = s_seg[2 * w + 1];
+            if (e0 == e1) continue;                              // nothing from this worker here (uniform for the block)
             const uint32_t* list = idx + (int64_t)w * cap;
             const uint32_t* words = reinterpret_cast<const uint32_t*>(codes + (int64_t)w * stride);
             const float dl = scale[w];
@@ -776,9 +783,12 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st)
 {
     const int vec_ok = vec_ok_for(v, d);
-    const int64_t nchunks = (d + kChunk - 1) / kChunk;
     const bool list = ctx->list_ready && sparse_out && v == ctx->alpha;     // only the listed groups can be nonzero
     const GroupList gl = list ? GroupList{ctx->glist, ctx->gcount, ctx->glist_cap} : GroupList{nullptr, nullptr, 0};
+    // a chunk is what one warp compacts on its own: 8 steps of 32 groups when streaming the whole vector, a single
+    // step in list mode, where the work is small and parallelism matters more than the size of the offset table
+    const int iters = list ? 1 : kChunk / 256;
+    const int64_t nchunks = list ? (ctx->glist_cap + 31) / 32 : (d + kChunk - 1) / kChunk;
     cudaMemsetAsync(ctx->l1_sum, 0, sizeof(unsigned long long) * M, st);
     cudaMemsetAsync(ctx->beta_norm_bits, 0, sizeof(uint32_t) * M, st);
     if (list) {
@@ -787,23 +797,23 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
         dim3 grid_l1(grid_for((d + 7) / 8, ctx->sm_count), M);
         norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
     }
-    dim3 grid_c(list ? 16 : grid_for(nchunks * 32, ctx->sm_count), M);
+    dim3 grid_c(list ? 64 : grid_for(nchunks * 32, ctx->sm_count), M);
     sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
                                                        ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks,
-                                                       ctx->rp_active, gl);
+                                                       ctx->rp_active, gl, iters);
     ctx->launches += 2;
     if (sparse_out) {
         chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
         cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
-            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl)));
+            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters)));
         ctx->launches += 2;
     } else {
         const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
-            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl)));
+            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl, iters)));
         ctx->launches += 1;
     }
 }
@@ -839,11 +849,11 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         tile_ptr_kernel<<<grid_t, kThreads, 0, st>>>(msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
         const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
         if (c.accelerated) {
-            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
+            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
                 msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                 s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         } else {
-            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, false><<<grid, kThreads, 0, st>>>(
+            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, false><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
                 msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                 s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         }
