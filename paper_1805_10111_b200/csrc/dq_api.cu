@@ -137,6 +137,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
             rc |= dev_alloc(&c->touched, (size_t)M * c->bm_words);
             rc |= dev_alloc(&c->glist, (size_t)M * c->glist_cap);
             rc |= dev_alloc(&c->gcount, M);
+            rc |= dev_alloc(&c->seg_count, (size_t)M * ((c->bm_words + kThreads - 1) / kThreads));
             if (rc == DQ_OK && (cudaMemset(c->touched, 0, sizeof(uint32_t) * M * c->bm_words) != cudaSuccess ||
                                 cudaMemset(c->gcount, 0, sizeof(uint32_t) * M) != cudaSuccess ||
                                 cudaMemset(c->alpha, 0, sizeof(float) * M * d) != cudaSuccess)) rc = DQ_ERR_CUDA;
@@ -154,7 +155,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);

@@ -267,26 +267,21 @@ chunk_scan_kernel(uint32_t* __restrict__ chunk_off, int64_t nchunks, int64_t cap
 {
     uint32_t* off = chunk_off + (int64_t)blockIdx.x * (nchunks + 1);
     __shared__ uint32_t s_warp[kThreads / 32];
-    __shared__ uint32_t s_carry;
-    if (threadIdx.x == 0) s_carry = 0;
-    __syncthreads();
-    for (int64_t base = 0; base < nchunks; base += blockDim.x) {
-        const int64_t i = base + threadIdx.x;
-        const uint32_t c = (i < nchunks) ? off[i] : 0u;
-        uint32_t incl = c;
+    // each thread owns a contiguous run of entries: local sum, one block-wide scan of the sums, local prefix
+    const int64_t per = (nchunks + blockDim.x - 1) / blockDim.x;
+    const int64_t i0 = (int64_t)threadIdx.x * per, i1 = min(i0 + per, nchunks);
+    uint32_t sum = 0;
+    for (int64_t i = i0; i < i1; ++i) sum += off[i];
+    uint32_t incl = sum;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if ((threadIdx.x & 31) >= o) incl += t; }
-        if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
-        __syncthreads();
-        uint32_t before = s_carry;
-        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) before += s_warp[k];
-        if (i < nchunks) off[i] = before + incl - c;
-        __syncthreads();
-        if (threadIdx.x == blockDim.x - 1) s_carry = before + incl;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        uint32_t total = s_carry;
+    for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if ((threadIdx.x & 31) >= o) incl += t; }
+    if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
+    __syncthreads();
+    uint32_t run = incl - sum;
+    for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) run += s_warp[k];
+    for (int64_t i = i0; i < i1; ++i) { const uint32_t c = off[i]; off[i] = run; run += c; }
+    if (threadIdx.x == blockDim.x - 1) {
+        uint32_t total = run;
         off[nchunks] = total;
         if ((int64_t)total > cap) { set_status(status, DQ_ERR_CAPACITY); total = (uint32_t)cap; }
         nnz[blockIdx.x] = total;
@@ -665,45 +660,62 @@ __global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const fl
 // and folds ||alpha_w||_inf over the listed groups (all other coordinates are zero).  One block per worker.
 // ---------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
-build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const float* __restrict__ alpha, int64_t d, int vec_ok,
+count_touched_kernel(const uint32_t* __restrict__ touched, int64_t bm_words, uint32_t* __restrict__ seg_count, int nseg)
+{
+    // grid (nseg, M): set bits of one segment of kThreads bitmap words
+    const int w = blockIdx.y;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t c = (i < bm_words) ? __popc(touched[(int64_t)w * bm_words + i]) : 0u;
+    c = __reduce_add_sync(0xFFFFFFFFu, c);
+    __shared__ uint32_t s_c[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) s_c[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (int k = 0; k < (int)(blockDim.x >> 5); ++k) t += s_c[k];
+        seg_count[(int64_t)w * nseg + blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(kThreads)
+build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const uint32_t* __restrict__ seg_count, int nseg,
+                        const float* __restrict__ alpha, int64_t d, int vec_ok,
                         uint32_t* __restrict__ glist, int64_t cap, uint32_t* __restrict__ gcount, uint32_t* __restrict__ norm_bits)
 {
-    const int w = blockIdx.x;
+    // grid (nseg, M): this segment's groups go to the list after those of the segments before it
+    const int w = blockIdx.y;
     uint32_t* bm = touched + (int64_t)w * bm_words;
     uint32_t* list = glist + (int64_t)w * cap;
     const float* row = alpha + (int64_t)w * d;
     __shared__ uint32_t s_warp[kThreads / 32];
-    __shared__ uint32_t s_carry;
-    if (threadIdx.x == 0) s_carry = 0;
+    __shared__ uint32_t s_base[kThreads / 32];
+    // base = sum of the earlier segments' counts (all threads help)
+    uint32_t part = 0;
+    for (int k = threadIdx.x; k < (int)blockIdx.x; k += blockDim.x) part += seg_count[(int64_t)w * nseg + k];
+    part = __reduce_add_sync(0xFFFFFFFFu, part);
+    if ((threadIdx.x & 31) == 0) s_base[threadIdx.x >> 5] = part;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t word = 0;
+    if (i < bm_words) { word = bm[i]; if (word) bm[i] = 0u; }
+    const uint32_t c = __popc(word);
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if ((threadIdx.x & 31) >= o) incl += t; }
+    if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
     __syncthreads();
+    uint32_t pos = incl - c;
+    for (int k = 0; k < (int)(blockDim.x >> 5); ++k) { pos += s_base[k]; if (k < (int)(threadIdx.x >> 5)) pos += s_warp[k]; }
+    if (blockIdx.x == gridDim.x - 1 && threadIdx.x == blockDim.x - 1) gcount[w] = pos + c;     // the last word closes the list
     uint32_t nmax = 0;
-    for (int64_t base = 0; base < bm_words; base += blockDim.x) {
-        const int64_t i = base + threadIdx.x;
-        uint32_t word = 0;
-        if (i < bm_words) { word = bm[i]; if (word) bm[i] = 0u; }
-        const uint32_t c = __popc(word);
-        uint32_t incl = c;
+    while (word) {
+        const int bit = __ffs(word) - 1; word &= word - 1;
+        const int64_t g = (i << 5) + bit, i0 = g << 3;
+        list[pos++] = (uint32_t)g;
+        float a[8];
+        if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if ((threadIdx.x & 31) >= o) incl += t; }
-        if ((threadIdx.x & 31) == 31) s_warp[threadIdx.x >> 5] = incl;
-        __syncthreads();
-        uint32_t pos = s_carry + incl - c;
-        for (int k = 0; k < (int)(threadIdx.x >> 5); ++k) pos += s_warp[k];
-        const uint32_t last = pos + c;
-        while (word) {
-            const int bit = __ffs(word) - 1; word &= word - 1;
-            const int64_t g = (i << 5) + bit, i0 = g << 3;
-            list[pos++] = (uint32_t)g;
-            float a[8];
-            if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) nmax = max(nmax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
-        }
-        __syncthreads();
-        if (threadIdx.x == blockDim.x - 1) s_carry = last;
-        __syncthreads();
+        for (int j = 0; j < 8; ++j) nmax = max(nmax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
     }
-    if (threadIdx.x == 0) gcount[w] = s_carry;
     block_atomic_max(nmax, norm_bits + w);
 }
 
@@ -774,8 +786,12 @@ void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st)
 {
     const dq_config& c = ctx->cfg;
     if (!ctx->ninf_zeroed) cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * c.M, st);
-    build_group_list_kernel<<<c.M, kThreads, 0, st>>>(ctx->touched, ctx->bm_words, ctx->alpha, c.d, vec_ok_for(ctx->alpha, c.d),
-                                                        ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
+    const int nseg = (int)((ctx->bm_words + kThreads - 1) / kThreads);
+    dim3 grid(nseg, c.M);
+    count_touched_kernel<<<grid, kThreads, 0, st>>>(ctx->touched, ctx->bm_words, ctx->seg_count, nseg);
+    build_group_list_kernel<<<grid, kThreads, 0, st>>>(ctx->touched, ctx->bm_words, ctx->seg_count, nseg, ctx->alpha, c.d,
+                                                        vec_ok_for(ctx->alpha, c.d), ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
+    ctx->launches += 2;
     ctx->launches += 1;
 }
 

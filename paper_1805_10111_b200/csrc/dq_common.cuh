@@ -222,7 +222,7 @@ struct dq_ctx {
     int64_t graph_launches;
     bool graph_off;
     // sparse gradients (CSR data, sparse messages): bitmap of touched groups, their ascending list, its length
-    uint32_t* touched; uint32_t* glist; uint32_t* gcount; int64_t bm_words; int64_t glist_cap;
+    uint32_t* touched; uint32_t* glist; uint32_t* gcount; uint32_t* seg_count; int64_t bm_words; int64_t glist_cap;
     bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only
     bool list_ready;            // the list of this round has been built (consumed by the sparsifier launch)
     bool alpha_zeroed, ninf_zeroed, normx_zeroed;   // an earlier kernel of this round already cleared these
