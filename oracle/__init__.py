@@ -57,7 +57,7 @@ class Config(C.Structure):
                 ("l1", C.c_float), ("l2", C.c_float), ("box_lo", C.c_float), ("box_hi", C.c_float),
                 ("sparsify", C.c_int32), ("phi", C.c_float),
                 ("msg_format", C.c_int32), ("accelerated", C.c_int32), ("snapshot_flag", C.c_int32), ("pad_", C.c_int32),
-                ("seed", C.c_uint64)]
+                ("seed", C.c_uint64), ("mu", C.c_float), ("pad2_", C.c_float)]
 
 
 class State(C.Structure):
@@ -69,7 +69,8 @@ class Trace(C.Structure):
                 ("alpha", C.c_void_p), ("S", C.c_void_p), ("beta", C.c_void_p), ("Z", C.c_void_p),
                 ("codes", C.c_void_p), ("delta", C.c_void_p), ("ninf", C.c_void_p), ("n1", C.c_void_p),
                 ("phi_eff", C.c_void_p), ("nnz", C.c_void_p),
-                ("bits_down", C.c_uint64), ("bits_up", C.c_uint64), ("normx", C.c_float), ("flag_round", C.c_int32)]
+                ("bits_down", C.c_uint64), ("bits_up", C.c_uint64), ("normx", C.c_float), ("flag_round", C.c_int32),
+                ("bx_used", C.c_int32), ("pad_", C.c_int32)]
 
 
 def _declare(L):
@@ -97,6 +98,9 @@ def _declare(L):
         "dqo_prox": (f32, [f32, f32, f32, f32, f32, f32]),
         "dqo_master_step": (None, [vp, vp, i32, i64, vp, vp, vp, vp, vp, f32, f32, i32, f32, f32, f32, f32, vp]),
         "dqo_epoch_begin": (None, [vp, vp, vp, f32, i64, vp]),
+        "dqo_expected_sq_error": (f64, [vp, i64, i32]),
+        "dqo_sq_distance": (f64, [vp, vp, i64]),
+        "dqo_select_bx": (i32, [vp, vp, i64, f32, vp, vp]),
         "dqo_round": (i32, [vp, vp, vp, u32, i32, f32, f32, vp]),
     }
     for name, (res, args) in sig.items():
@@ -271,11 +275,25 @@ def master_step(codes, delta, gfull, x, eta, theta=0.0, accelerated=False, y=Non
     return nx[0]
 
 
+# ---- model precision (condition (3)) ----------------------------------------------------------------
+def expected_sq_error(x, b):
+    x = _f32(x)
+    return float(lib().dqo_expected_sq_error(_p(x), x.size, b))
+
+
+def select_bx(x, xsnap, mu):
+    """Returns (chosen width, expected errors at 2/4/8 bits, ||x - xsnap||^2)."""
+    x, xsnap = _f32(x), _f32(xsnap)
+    err = np.zeros(3, np.float64); dist = np.zeros(1, np.float64)
+    b = lib().dqo_select_bx(_p(x), _p(xsnap), x.size, float(mu), _p(err), _p(dist))
+    return int(b), err, float(dist[0])
+
+
 # ---- drivers ------------------------------------------------------------------------
 def make_config(d, M, B, bx, b, l1=0.0, l2=0.0, box_lo=-np.inf, box_hi=np.inf, sparsify=0, phi=0.0,
-                msg_format=MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0):
+                msg_format=MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, mu=0.0):
     return Config(d, M, B, bx, b, l1, l2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                  int(snapshot_flag), 0, seed)
+                  int(snapshot_flag), 0, seed, mu, 0.0)
 
 
 class Run:
@@ -321,5 +339,5 @@ class Run:
                              float(eta), float(theta), C.addressof(T))
         self.rounds_in_epoch += 1
         keep.update(bits_down=int(T.bits_down), bits_up=int(T.bits_up), normx=np.float32(T.normx),
-                    flag_round=bool(T.flag_round), status=rc)
+                    flag_round=bool(T.flag_round), bx_used=int(T.bx_used), status=rc)
         return keep

@@ -429,6 +429,50 @@ void dqo_master_step(const int32_t* codes /*[M][d]*/, const float* delta /*[M]*/
 }
 
 /* ------------------------------------------------------------------------ */
+/* Model precision: the master quantises x "subject to" condition (3),        */
+/*   E_Q ||Q(x) - x||^2 <= mu ||x - xsnap||^2                                 */
+/* (condition (6) of Algorithm 3 has theta_s mu), and Section 5.2 searches    */
+/* b_x so that it holds.  Under rule (i) a coordinate between the grid points */
+/* z and z + delta has expected squared error (x - z)(z + delta - x)          */
+/* (proof of the appendix's first lemma), so the left side is a closed form.  */
+/* This build packs 2, 4 or 8 bits; the search is over those widths.          */
+/* ------------------------------------------------------------------------ */
+double dqo_expected_sq_error(const float* x, int64_t d, int b)
+{
+    float nrm = dqo_norm_inf(x, d);
+    if (nrm == 0.0f) return 0.0;
+    double delta = (double)dqo_scale_delta(nrm, b), e = 0.0;
+    for (int64_t i = 0; i < d; ++i) {
+        double t = (double)x[i] / delta, frac = t - floor(t);
+        e += frac * (1.0 - frac);                                  /* (x - z)(z + delta - x) / delta^2 */
+    }
+    return e * delta * delta;
+}
+
+double dqo_sq_distance(const float* x, const float* y, int64_t d)
+{
+    double s = 0.0;
+    for (int64_t i = 0; i < d; ++i) { double t = (double)x[i] - (double)y[i]; s += t * t; }
+    return s;
+}
+
+/* Smallest width in {2, 4, 8} that satisfies the condition; 8 when none does.
+ * err[0..2] receive the expected errors at 2, 4, 8 bits, *dist2 the squared distance. */
+int dqo_select_bx(const float* x, const float* xsnap, int64_t d, float mu, double* err, double* dist2)
+{
+    static const int widths[3] = { 2, 4, 8 };
+    double D = dqo_sq_distance(x, xsnap, d);
+    int chosen = 8;
+    for (int k = 2; k >= 0; --k) {
+        double e = dqo_expected_sq_error(x, d, widths[k]);
+        if (err) err[k] = e;
+        if (e <= (double)mu * D) chosen = widths[k];
+    }
+    if (dist2) *dist2 = D;
+    return chosen;
+}
+
+/* ------------------------------------------------------------------------ */
 /* Round and epoch drivers.                                                  */
 /* ------------------------------------------------------------------------ */
 typedef struct {
@@ -437,6 +481,7 @@ typedef struct {
     int32_t sparsify; float phi;
     int32_t msg_format, accelerated, snapshot_flag, pad_;
     uint64_t seed;
+    float mu; float pad2_;          /* mu > 0: choose b_x per round by condition (3)/(6); 0: fixed b_x */
 } dqo_config;
 
 typedef struct { float *x, *xsnap, *gfull, *y, *xsum; } dqo_state;
@@ -452,6 +497,7 @@ typedef struct {
     int64_t* nnz;      /* [M] */
     uint64_t bits_down, bits_up;
     float normx; int32_t flag_round;
+    int32_t bx_used; int32_t pad_;
 } dqo_trace;
 
 static int ceil_log2(int64_t d) { int k = 0; while (((int64_t)1 << k) < d) ++k; return k; }
@@ -493,6 +539,7 @@ int dqo_round(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t rou
     int64_t* rows = (int64_t*)malloc((size_t)B * 8);
     uint64_t bits_down, bits_up = 0;
     float delta_x = 0.0f;
+    int bx = C->bx;
 
     /* master (i): model quantisation, step 8 */
     if (flag_round) {
@@ -500,15 +547,18 @@ int dqo_round(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t rou
         for (int64_t i = 0; i < d; ++i) codes_x[i] = 0;
         bits_down = (uint64_t)M;
     } else {
-        rc = dqo_quantize(S->x, d, C->bx, C->seed, round, DQO_MASTER, DQO_STREAM_MODEL, codes_x, &delta_x);
+        if (C->mu > 0.0f)      /* condition (3); Algorithm 3 uses theta_s mu (condition (6)) */
+            bx = dqo_select_bx(S->x, S->xsnap, d, C->accelerated ? theta * C->mu : C->mu, NULL, NULL);
+        rc = dqo_quantize(S->x, d, bx, C->seed, round, DQO_MASTER, DQO_STREAM_MODEL, codes_x, &delta_x);
         for (int64_t i = 0; i < d; ++i) xhat[i] = (float)codes_x[i] * delta_x;
-        bits_down = (uint64_t)M * (32u + (uint64_t)C->bx * (uint64_t)d);
+        bits_down = (uint64_t)M * (32u + (uint64_t)bx * (uint64_t)d);
     }
     if (T) {
         if (T->codes_x) memcpy(T->codes_x, codes_x, (size_t)d * 4);
         if (T->delta_x) *T->delta_x = delta_x;
         if (T->xhat) memcpy(T->xhat, xhat, (size_t)d * 4);
         T->flag_round = flag_round;
+        T->bx_used = flag_round ? 0 : bx;
     }
 
     /* workers, steps 11-13 */

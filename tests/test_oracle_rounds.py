@@ -170,3 +170,61 @@ def test_accelerated_identities_and_snapshot_mean():
             assert np.allclose(run.x - x0, theta * (run.y - y0), rtol=1e-4, atol=2e-7)
             xs_hist.append(run.x.copy()); rnd += 1
         assert np.allclose(run.xsum, np.sum(xs_hist, axis=0), rtol=1e-6, atol=1e-7)
+
+
+def test_expected_error_closed_form_and_bit_width_search():
+    """Condition (3): E_Q||Q(x) - x||^2 <= mu ||x - xsnap||^2.  The closed form sum (x - z)(z + delta - x) is pinned
+    by brute force over the grid and by the empirical mean of the oracle's own quantiser; the search returns the
+    smallest admissible width, is monotone in mu, and the expected error falls about 4x per extra bit pair."""
+    g = np.random.default_rng(31)
+    d = 400
+    x = g.standard_normal(d).astype(F32)
+    for b in (2, 4, 8):
+        L = 2 ** (b - 1) - 1
+        delta = float(np.abs(x).max() / F32(L))
+        grid = np.arange(-L - 1, L + 2) * delta
+        want = 0.0
+        for xi in x.astype(np.float64):
+            z = grid[np.searchsorted(grid, xi, side="right") - 1]           # the grid point at or below x_i
+            want += (xi - z) * (z + delta - xi)
+        got = oracle.expected_sq_error(x, b)
+        assert abs(got - want) <= 1e-9 * want
+        assert got <= d * delta ** 2 / 4                                     # the variance bound of the appendix's first lemma
+        acc = 0.0; N = 3000
+        for rnd in range(N):
+            codes, dl, _ = oracle.quantize(x, b, 77, rnd, 0, oracle.STREAM_MODEL)
+            acc += float(((codes.astype(np.float64) * float(dl) - x) ** 2).sum())
+        assert abs(acc / N - got) < 0.02 * got                               # Monte-Carlo over the oracle's quantiser
+    xs = (x + F32(0.05) * g.standard_normal(d).astype(F32)).astype(F32)
+    dist = float(((x.astype(np.float64) - xs) ** 2).sum())
+    errs = [oracle.expected_sq_error(x, b) for b in (2, 4, 8)]
+    assert errs[0] > errs[1] > errs[2]
+    for mu, want_b in ((errs[2] / dist * 0.5, 8), (errs[2] / dist * 1.01, 8), (errs[1] / dist * 1.01, 4), (errs[0] / dist * 1.01, 2),
+                       (errs[0] / dist * 100, 2)):
+        b, e3, D = oracle.select_bx(x, xs, mu)
+        assert b == want_b and np.allclose(e3, errs) and abs(D - dist) < 1e-12 * dist
+    assert oracle.select_bx(x, x, 1e9)[0] == 8                               # x = xsnap: nothing admissible (the flag bit handles it)
+
+
+def test_round_with_searched_model_bits():
+    """With mu > 0 every non-flag round quantises the model with the searched width and pays for that width."""
+    h, data = _problem()
+    M, B = 2, 8
+    seen = set()
+    for mu in (1e-3, 50.0, 1e6):
+        cfg = oracle.make_config(h.d, M, B, 8, 8, l1=1e-4, seed=3, mu=mu)
+        run = oracle.Run(cfg, data, synth.normal_vector(h.d, 34, 0.2))
+        run.epoch_begin()
+        for rnd in range(6):
+            x_before = run.x.copy()
+            tr = run.round(rnd, 0.5, trace=True)
+            if tr["flag_round"]:
+                assert tr["bx_used"] == 0 and tr["bits_down"] == M
+                continue
+            want_b = oracle.select_bx(x_before, run.xsnap, mu)[0]
+            assert tr["bx_used"] == want_b
+            cx, dx, _ = oracle.quantize(x_before, want_b, 3, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+            assert np.array_equal(tr["codes_x"], cx) and tr["delta_x"][0] == dx
+            assert tr["bits_down"] == M * (32 + want_b * h.d)
+            seen.add(want_b)
+    assert seen == {2, 4, 8} or seen >= {2, 8}
