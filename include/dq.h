@@ -80,6 +80,8 @@ typedef struct {
     int32_t no_graph;          /* 1: dq_round launches its kernels one by one instead of replaying a CUDA graph */
     uint64_t seed;
     int64_t sparse_cap;        /* entries per worker in the context's own sparse message buffers; 0: d   */
+    float mu;                  /* > 0: dq_round picks b_x in {2,4,8} each round by condition (3)/(6); 0: fixed bx */
+    int32_t reserved;
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3
@@ -122,6 +124,16 @@ int dq_epoch_begin(dq_ctx* ctx, dq_state* st, float theta, void* stream);
  * dq_packed_bytes(d, bx) bytes; delta_x is one device float. */
 int dq_quantize_model(dq_ctx* ctx, const float* x, const float* norm_x, uint32_t round,
                       uint8_t* codes_x, float* delta_x, void* stream);
+
+/* Model precision (condition (3); condition (6) for Algorithm 3 passes theta_s * mu): writes to *bits (device int)
+ * the smallest width b in {2, 4, 8} with  E_Q ||Q_(delta,b)(x) - x||^2 <= mu ||x - x_snap||^2, 8 if none, where the
+ * left side is the closed form sum_i (x_i - z_i)(z_i + delta - x_i) of rule (i).  stats (device double[4], may be
+ * NULL) receives the expected errors at 2, 4, 8 bits and ||x - x_snap||^2.  norm_x: device ||x||_inf or NULL. */
+int dq_select_model_bits(dq_ctx* ctx, const float* x, const float* x_snap, const float* norm_x, float mu,
+                         int32_t* bits, double* stats, void* stream);
+
+/* Width chosen by the last dq_round of a context with mu > 0 (synchronises `stream`); 0 after a snapshot round. */
+int dq_last_model_bits(dq_ctx* ctx, int32_t* bits_host, void* stream);
 
 /* Worker step 11 for all M workers: alpha_w = (1/B) sum_{a in batch_w} [grad f_a(xhat) - grad f_a(x_snap)],
  * xhat = dequantised broadcast model (code * delta_x), or x_snap itself when is_snapshot != 0 (flag bit of

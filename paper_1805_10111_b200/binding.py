@@ -19,7 +19,8 @@ DQ_MSG_DENSE, DQ_MSG_SPARSE = 0, 1
 EXPORTS = ["dq_packed_bytes", "dq_create", "dq_destroy", "dq_epoch_begin", "dq_quantize_model", "dq_worker_grad",
            "dq_norm_inf", "dq_quantize_sparsify_pack", "dq_master_unpack_aggregate_prox", "dq_round", "dq_codec_round",
            "dq_codec_host_setup", "dq_codec_round_host", "dq_unpack", "dq_objective", "dq_round_buffers",
-           "dq_poll_status", "dq_launch_count", "dq_strerror", "dq_quantize_pack_static"]
+           "dq_poll_status", "dq_launch_count", "dq_strerror", "dq_quantize_pack_static", "dq_select_model_bits",
+           "dq_last_model_bits"]
 
 
 class dq_data(C.Structure):
@@ -31,7 +32,7 @@ class dq_config(C.Structure):
     _fields_ = [("d", C.c_int64), ("M", C.c_int32), ("B", C.c_int32), ("bx", C.c_int32), ("b", C.c_int32),
                 ("lambda1", C.c_float), ("lambda2", C.c_float), ("box_lo", C.c_float), ("box_hi", C.c_float),
                 ("sparsify", C.c_int32), ("phi", C.c_float), ("msg_format", C.c_int32), ("accelerated", C.c_int32),
-                ("snapshot_flag", C.c_int32), ("no_graph", C.c_int32), ("seed", C.c_uint64), ("sparse_cap", C.c_int64)]
+                ("snapshot_flag", C.c_int32), ("no_graph", C.c_int32), ("seed", C.c_uint64), ("sparse_cap", C.c_int64), ("mu", C.c_float), ("reserved", C.c_int32)]
 
 
 class dq_state(C.Structure):
@@ -81,6 +82,8 @@ def lib():
             "dq_poll_status": (i32, [vp, C.POINTER(C.c_int), vp]),
             "dq_launch_count": (i64, [vp]),
             "dq_strerror": (C.c_char_p, [i32]),
+            "dq_select_model_bits": (i32, [vp, vp, vp, vp, f32, vp, vp, vp]),
+            "dq_last_model_bits": (i32, [vp, C.POINTER(C.c_int32), vp]),
             "dq_quantize_pack_static": (i32, [vp, i64, i32, i32, C.c_uint64, u32, vp, i64, vp, vp]),
         }
         for name, (res, args) in sig.items():
@@ -157,9 +160,9 @@ class Msgs:
 
 
 def make_config(d, M, B=1, bx=8, b=8, lambda1=0.0, lambda2=0.0, box_lo=float("-inf"), box_hi=float("inf"), sparsify=0,
-                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0) -> dq_config:
+                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0) -> dq_config:
     return dq_config(d, M, B, bx, b, lambda1, lambda2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                     int(snapshot_flag), int(no_graph), seed, sparse_cap)
+                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, 0)
 
 
 # ---- entry points (same names and order of arguments as include/dq.h) ---------------------------------------------
@@ -252,6 +255,17 @@ def dq_poll_status(ctx, stream=None):
 
 def dq_launch_count(ctx):
     return int(lib().dq_launch_count(ctx))
+
+
+def dq_select_model_bits(ctx, x, x_snap, norm_x, mu, bits, stats, stream=None):
+    return lib().dq_select_model_bits(ctx, _ptr(x), _ptr(x_snap), _ptr(norm_x), float(mu), _ptr(bits), _ptr(stats), _stream(stream))
+
+
+def dq_last_model_bits(ctx, stream=None):
+    """Returns (status, width chosen by the last dq_round)."""
+    v = C.c_int32(0)
+    rc = lib().dq_last_model_bits(ctx, C.byref(v), _stream(stream))
+    return rc, v.value
 
 
 def dq_quantize_pack_static(v, d, M, b, seed, round_, codes, stride, scale, stream=None):

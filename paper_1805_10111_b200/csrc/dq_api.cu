@@ -83,6 +83,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (cfg->msg_format != DQ_MSG_SPARSE && cfg->msg_format != DQ_MSG_DENSE) return DQ_ERR_ARG;
     if (!(cfg->box_lo <= cfg->box_hi) || cfg->lambda1 < 0 || cfg->lambda2 < 0) return DQ_ERR_ARG;
     if (cfg->sparse_cap < 0 || cfg->sparse_cap > cfg->d) return DQ_ERR_ARG;
+    if (!(cfg->mu >= 0.0f)) return DQ_ERR_ARG;
     if (data) {
         if (data->n < 1 || data->d != cfg->d || !data->values || !data->labels) return DQ_ERR_SHAPE;
         if (data->format == DQ_CSR_F32 && (!data->col_idx || !data->row_ptr)) return DQ_ERR_ARG;
@@ -121,7 +122,9 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     rc |= dev_alloc(&c->msgs.scale, M);
     rc |= dev_alloc(&c->msgs.idx, sparse ? (size_t)c->msgs.cap * M : 1);
     rc |= dev_alloc(&c->msgs.nnz, M);
-    rc |= dev_alloc(&c->codes_x, (size_t)dq_packed_bytes(d, cfg->bx));
+    rc |= dev_alloc(&c->codes_x, (size_t)dq_packed_bytes(d, cfg->mu > 0.0f ? 8 : cfg->bx));
+    rc |= dev_alloc(&c->bx_dev, 1);
+    rc |= dev_alloc(&c->prec_stats, 4);
     rc |= dev_alloc(&c->delta_x, 1);
     rc |= dev_alloc(&c->ninf, M);
     if (data) {
@@ -144,6 +147,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
         }
     }
     if (rc == DQ_OK && cudaMemset(c->status, 0, sizeof(int)) != cudaSuccess) rc = DQ_ERR_CUDA;
+    if (rc == DQ_OK && cudaMemset(c->bx_dev, 0, sizeof(int32_t)) != cudaSuccess) rc = DQ_ERR_CUDA;
     if (rc != DQ_OK) { dq_destroy(c); cudaGetLastError(); return DQ_ERR_CUDA; }
     c->epoch = -1;
     *out = c;
@@ -155,7 +159,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -290,13 +294,25 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
                          uint64_t* bits_up, void* st)
 {
     int rc = DQ_OK;
+    const bool adaptive = ctx->cfg.mu > 0.0f;
     if (!flag) {     // model quantisation that also emits xhat - xsnap for the workers
-        launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, reinterpret_cast<const uint32_t*>(s->norm_x), ctx->codes_x,
-                             dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx), ctx->delta_x, round, kMaster, kStreamModel, as_stream(st),
-                             s->x_snap, ctx->xhat_diff, worker_accumulates(ctx) ? ctx->alpha : nullptr,
-                             worker_accumulates(ctx) ? (int64_t)ctx->cfg.M * ctx->cfg.d : 0,
-                             reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
+        const uint32_t* nx = reinterpret_cast<const uint32_t*>(s->norm_x);
+        float* zf = worker_accumulates(ctx) ? ctx->alpha : nullptr;
+        const int64_t zn = worker_accumulates(ctx) ? (int64_t)ctx->cfg.M * ctx->cfg.d : 0;
+        if (!adaptive) {
+            launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx),
+                                 ctx->delta_x, round, kMaster, kStreamModel, as_stream(st), s->x_snap, ctx->xhat_diff, zf, zn,
+                                 reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
+        } else {     // condition (3): pick the width on the device, then launch all three widths; two return at once
+            launch_select_bits(ctx, s->x, s->x_snap, nx, ctx->cfg.mu, theta, ctx->bx_dev, ctx->prec_stats, as_stream(st));
+            for (int bits = 2; bits <= 8; bits *= 2)
+                launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, bits, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, bits), ctx->delta_x,
+                                     round, kMaster, kStreamModel, as_stream(st), s->x_snap, ctx->xhat_diff, zf, zn,
+                                     reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M, ctx->bx_dev);
+        }
         ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = ctx->normx_zeroed = true;
+    } else if (adaptive) {
+        cudaMemsetAsync(ctx->bx_dev, 0, sizeof(int32_t), as_stream(st));
     }
     rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
     ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = false;
@@ -304,7 +320,7 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     ctx->list_ready = false;
     if (rc != DQ_OK) { ctx->normx_zeroed = false; return rc; }
     const BitsArgs ba = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag,
-                         sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b};
+                         sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b, (adaptive && !flag) ? ctx->bx_dev : nullptr};
     launch_master(ctx, &ctx->msgs, sparse_messages(ctx), s, eta, theta, as_stream(st), (bits_down || bits_up) ? &ba : nullptr);
     ctx->normx_zeroed = false;
     return last_error();
@@ -364,6 +380,28 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
     }
     ctx->rounds_in_epoch += 1;
     return last_error();
+}
+
+int dq_select_model_bits(dq_ctx* ctx, const float* x, const float* x_snap, const float* norm_x, float mu, int32_t* bits,
+                         double* stats, void* stream)
+{
+    if (!ctx || !x || !x_snap || !bits || !(mu >= 0.0f)) return DQ_ERR_ARG;
+    cudaStream_t st = as_stream(stream);
+    const uint32_t* nb = reinterpret_cast<const uint32_t*>(norm_x);
+    if (!nb) { launch_norm_inf(ctx, x, ctx->cfg.d, 1, ctx->xnorm_bits, st); nb = ctx->xnorm_bits; }
+    // theta is folded into mu by the caller here, so the kernel is told "not accelerated"
+    const int acc = ctx->cfg.accelerated; ctx->cfg.accelerated = 0;
+    launch_select_bits(ctx, x, x_snap, nb, mu, 0.0f, bits, stats ? stats : ctx->prec_stats, st);
+    ctx->cfg.accelerated = acc;
+    return last_error();
+}
+
+int dq_last_model_bits(dq_ctx* ctx, int32_t* bits_host, void* stream)
+{
+    if (!ctx || !bits_host) return DQ_ERR_ARG;
+    cudaStream_t st = as_stream(stream);
+    if (cudaMemcpyAsync(bits_host, ctx->bx_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st) != cudaSuccess) return DQ_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }
 
 int dq_objective(dq_ctx* ctx, const float* x, double* P, void* stream)

@@ -45,8 +45,10 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker_base, uint32_t stream,
                      int64_t ngroups, int* __restrict__ status, const RoundParams* __restrict__ rp,
                      const float* __restrict__ ref = nullptr, float* __restrict__ diff = nullptr,
-                     float* __restrict__ zero_f = nullptr, int64_t zero_n = 0, uint32_t* __restrict__ zero_u = nullptr, int zero_un = 0)
+                     float* __restrict__ zero_f = nullptr, int64_t zero_n = 0, uint32_t* __restrict__ zero_u = nullptr, int zero_un = 0,
+                     const int32_t* __restrict__ bits_gate = nullptr /* run only if *bits_gate == BITS */)
 {
+    if (bits_gate && *bits_gate != BITS) return;
     if (rp) round = rp->round;
     if (DIFF) {   // also clears the buffers that the next stages of the round accumulate into
         const int64_t nth0 = (int64_t)gridDim.x * gridDim.y * blockDim.x;
@@ -735,6 +737,61 @@ clear_listed_groups_kernel(float* __restrict__ alpha, int64_t d, const uint32_t*
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Model precision, condition (3): sums of frac (1 - frac) of x / delta_b for b = 2, 4, 8 (the expected squared
+// error of rule (i) in units of delta_b^2) and ||x - xsnap||^2, in double.  stats must be zero on entry.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+model_precision_kernel(const float* __restrict__ x, const float* __restrict__ xsnap, int64_t d, const uint32_t* __restrict__ norm_bits,
+                       double* __restrict__ stats)
+{
+    const float nrm = __uint_as_float(norm_bits[0]);
+    double inv[3];
+    inv[0] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 1.0f) : 0.0;
+    inv[1] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 7.0f) : 0.0;
+    inv[2] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 127.0f) : 0.0;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        const double xi = (double)x[i], df = xi - (double)xsnap[i];
+#pragma unroll
+        for (int k = 0; k < 3; ++k) { const double t = xi * inv[k], fr = t - floor(t); acc[k] += fr * (1.0 - fr); }
+        acc[3] += df * df;
+    }
+    __shared__ double s_part[kThreads / 32][4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        double v = acc[k];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+        if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5][k] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < 4) {
+        double t = 0.0;
+        for (int k = 0; k < (int)(blockDim.x >> 5); ++k) t += s_part[k][threadIdx.x];
+        atomicAdd(stats + threadIdx.x, t);
+    }
+}
+
+// Smallest width whose expected error is within mu ||x - xsnap||^2 (Algorithm 3: theta mu), 8 if none.
+__global__ void select_bits_kernel(double* __restrict__ stats, const uint32_t* __restrict__ norm_bits, float mu, int accelerated,
+                                   float theta, const RoundParams* __restrict__ rp, int32_t* __restrict__ bits)
+{
+    if (rp) theta = rp->theta;
+    const float nrm = __uint_as_float(norm_bits[0]);
+    const double mu_eff = accelerated ? (double)__fmul_rn(theta, mu) : (double)mu;
+    const float L[3] = {1.0f, 7.0f, 127.0f};
+    const int widths[3] = {2, 4, 8};
+    int chosen = 8;
+    for (int k = 2; k >= 0; --k) {
+        const double delta = nrm > 0.0f ? (double)__fdiv_rn(nrm, L[k]) : 0.0;
+        const double e = stats[k] * delta * delta;
+        stats[k] = e;
+        if (e <= mu_eff * stats[3]) chosen = widths[k];
+    }
+    *bits = chosen;
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Host launchers
 // ---------------------------------------------------------------------------------------------------
 static inline int grid_for(int64_t items_per_thread_units, int sm_count, int per_sm = 8)
@@ -758,7 +815,7 @@ void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* no
 void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
                           uint32_t stream_id, cudaStream_t st, const float* ref, float* diff, float* zero_f, int64_t zero_n,
-                          uint32_t* zero_u, int zero_un)
+                          uint32_t* zero_u, int zero_un, const int32_t* bits_gate)
 {
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
@@ -766,13 +823,22 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
         grid.x = max(grid.x, (unsigned)grid_for(zero_n / 4, ctx->sm_count));   // enough blocks for the clearing loop too
         DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
             v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
-            ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un)));
+            ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits_gate)));
         ctx->launches += 1;
         return;
     }
     DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_><<<grid, kThreads, 0, st>>>(
         v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active)));
     ctx->launches += 1;
+}
+
+void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, float theta,
+                        int32_t* bits, double* stats, cudaStream_t st)
+{
+    cudaMemsetAsync(stats, 0, sizeof(double) * 4, st);
+    model_precision_kernel<<<grid_for(ctx->cfg.d / 4 + 1, ctx->sm_count), kThreads, 0, st>>>(x, xsnap, ctx->cfg.d, norm_bits, stats);
+    select_bits_kernel<<<1, 1, 0, st>>>(stats, norm_bits, mu, ctx->cfg.accelerated, theta, ctx->rp_active, bits);
+    ctx->launches += 2;
 }
 
 void launch_clear_listed(dq_ctx* ctx, cudaStream_t st)

@@ -159,11 +159,13 @@ __device__ __forceinline__ int64_t group_at(const GroupList& gl, int w, int64_t 
 }
 
 // Transmitted-bit counters of a round, written by the master kernel when `down` is set (Section 3.1 message sizes).
-struct BitsArgs { uint64_t* down; uint64_t* up; const uint32_t* nnz; int flag_round, sparse_msgs, bx, b; };
+struct BitsArgs { uint64_t* down; uint64_t* up; const uint32_t* nnz; int flag_round, sparse_msgs, bx, b;
+                  const int32_t* bx_dev; /* width chosen on the device this round, overrides bx when set */ };
 
 __device__ __forceinline__ void write_round_bits(const BitsArgs& ba, int M, int64_t d)
 {
-    *ba.down = ba.flag_round ? (uint64_t)M : (uint64_t)M * (32ull + (uint64_t)ba.bx * (uint64_t)d);
+    const int bx = ba.bx_dev ? *ba.bx_dev : ba.bx;
+    *ba.down = ba.flag_round ? (uint64_t)M : (uint64_t)M * (32ull + (uint64_t)bx * (uint64_t)d);
     int logd = 0; while (((int64_t)1 << logd) < d) ++logd;
     uint64_t up = 0;
     for (int w = 0; w < M; ++w)
@@ -208,6 +210,8 @@ struct dq_ctx {
     float* xhat_diff;           // [d] dequantised model minus snapshot
     double* g64;                // [d] full-gradient accumulator
     float* rbuf;                // [M][B] slope differences of the sampled rows
+    int32_t* bx_dev;            // model width chosen by condition (3) this round
+    double* prec_stats;         // [4] expected errors at 2/4/8 bits and ||x - xsnap||^2
     dq_msgs msgs;
     uint64_t* bits;             // [2] device counters
     // device-resident state for the host-buffer entry point

@@ -9,7 +9,10 @@ void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* no
 void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint8_t* codes, int64_t stride, float* scale, uint32_t round, uint32_t worker_base,
                           uint32_t stream_id, cudaStream_t st, const float* ref = nullptr, float* diff = nullptr,
-                          float* zero_f = nullptr, int64_t zero_n = 0, uint32_t* zero_u = nullptr, int zero_un = 0);
+                          float* zero_f = nullptr, int64_t zero_n = 0, uint32_t* zero_u = nullptr, int zero_un = 0,
+                          const int32_t* bits_gate = nullptr);
+void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, float theta,
+                        int32_t* bits, double* stats, cudaStream_t st);
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
 void launch_clear_listed(dq_ctx* ctx, cudaStream_t st);

@@ -194,7 +194,8 @@ class Lockstep:
         self.dq, self.h = dq, h
         okw = dict(l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0), box_lo=kw.get("box_lo", -np.inf),
                    box_hi=kw.get("box_hi", np.inf), sparsify=kw.get("sparsify", 0), phi=kw.get("phi", 0.0),
-                   msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"])
+                   msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"],
+                   mu=kw.get("mu", 0.0))
         self.cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
         self.ocfg = oracle.make_config(h.d, kw["M"], kw["B"], kw["bx"], kw["b"], **okw)
         self.data = dq.Data(h)
@@ -235,9 +236,12 @@ class Lockstep:
         _, buf = dq.dq_round_buffers(self.ctx)
         m = buf["msgs"]
         # model codes: same x, so bit-exact
+        if cfg.mu > 0:
+            assert dq.dq_last_model_bits(self.ctx) == (0, tr["bx_used"])       # width searched by condition (3)/(6)
         if not tr["flag_round"]:
-            nbx = dq.dq_packed_bytes(d, cfg.bx)
-            assert np.array_equal(dq.device_view(buf["codes_x"], nbx, torch.uint8).cpu().numpy(), oracle.pack(tr["codes_x"], cfg.bx, nbx))
+            bx = tr["bx_used"]
+            nbx = dq.dq_packed_bytes(d, bx)
+            assert np.array_equal(dq.device_view(buf["codes_x"], nbx, torch.uint8).cpu().numpy(), oracle.pack(tr["codes_x"], bx, nbx))
             assert dq.device_view(buf["delta_x"], 1, torch.float32).item() == tr["delta_x"][0]
         a_gpu = dq.device_view(buf["alpha"], M * d, torch.float32).cpu().numpy().reshape(M, d)
         scale = dq.device_view(m.scale, M, torch.float32).cpu().numpy()
@@ -351,6 +355,44 @@ def test_lockstep_accelerated_sparse(dq):
             ls.round(rnd, eta, theta)
             rnd += 1
     ls.close()
+
+
+@pytest.mark.parametrize("mu,acc", [(1e-3, 0), (30.0, 0), (1e5, 0), (30.0, 1)])
+def test_lockstep_searched_model_bits(dq, mu, acc):
+    """mu > 0: each round's model width comes from condition (3) (theta mu for Algorithm 3); codes, bits and iterates
+    follow the oracle round by round."""
+    h = _problem("dense8")
+    kw = dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=14, mu=mu, accelerated=acc)
+    if acc:
+        kw.update(box_lo=-1.0, box_hi=1.0)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 79, 0.2), **kw)
+    widths = set()
+    rnd = 0
+    for s_ in range(1, 3):
+        theta = F32(2.0 / (s_ + 2)) if acc else F32(0.0)
+        ls.epoch(theta)
+        for t in range(8):
+            tr = ls.round(rnd, 0.5, theta)
+            widths.add(tr["bx_used"]); rnd += 1
+    assert widths - {0} <= {2, 4, 8} and len(widths - {0}) >= 1
+    ls.close()
+
+
+def test_select_model_bits_standalone(dq):
+    import torch
+    d = 100003
+    x = synth.normal_vector(d, 80); xs = (x + synth.normal_vector(d, 81, 0.02)).astype(F32)
+    cfg = dq.make_config(d, 2)
+    rc, ctx = dq.dq_create(cfg); assert rc == 0
+    bits = torch.zeros(1, dtype=torch.int32, device="cuda"); stats = torch.zeros(4, dtype=torch.float64, device="cuda")
+    _, errs, dist = oracle.select_bx(x, xs, 1.0)
+    for mu in (errs[2] / dist * 0.5, errs[2] / dist * 1.5, errs[1] / dist * 1.5, errs[0] / dist * 1.5):
+        assert dq.dq_select_model_bits(ctx, _dev(x), _dev(xs), None, mu, bits, stats) == 0
+        want, _, _ = oracle.select_bx(x, xs, mu)
+        assert bits.item() == want
+        got = stats.cpu().numpy()
+        assert np.allclose(got[:3], errs, rtol=1e-9) and abs(got[3] - dist) <= 1e-11 * dist
+    dq.dq_destroy(ctx)
 
 
 def _full_config(name):
