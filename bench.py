@@ -317,6 +317,19 @@ def run_ours(a):
     ms_per_step = total_ms / a.steps
     value = whole_job_rate(world, a.steps, total_ms)
 
+    # the optional width search of condition (3) on the same model (not part of the default round, mu = 0)
+    sel_bits = torch.zeros(1, dtype=torch.int32, device="cuda"); sel_stats = torch.zeros(4, dtype=torch.float64, device="cuda")
+    xs_dev = torch.from_numpy(x0).cuda()
+    for _ in range(3):
+        dq.ok(dq.dq_select_model_bits(ctx, st.x, xs_dev, st.norm_x, 1.0, sel_bits, sel_stats))
+    s0 = torch.cuda.Event(enable_timing=True); s1 = torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for _ in range(20):
+        dq.ok(dq.dq_select_model_bits(ctx, st.x, xs_dev, st.norm_x, 1.0, sel_bits, sel_stats))
+    s1.record(); torch.cuda.synchronize()
+    select_ms = s0.elapsed_time(s1) / 20
+    del xs_dev
+
     # end to end through the host-buffer entry point: H2D of the M gradient vectors, the round, D2H of the model codes
     e2e = None
     if a.e2e_steps > 0:
@@ -345,6 +358,8 @@ def run_ours(a):
     names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
     stages = {n: {"ms": round(ms, 4), "alg_GBps": round(by / ms / 1e6, 1), "frac_of_peak": round(by / ms / 1e6 / peak, 4)}
               for n, ms, by in zip(names, stage_ms, alg)}
+    stages["select_model_bits(optional)"] = {"ms": round(select_ms, 4), "alg_GBps": round(d * 8.0 / select_ms / 1e6, 1),
+                                              "frac_of_peak": round(d * 8.0 / select_ms / 1e6 / peak, 4)}
     qp = stages["quantize_pack"]
     tr = recorded_traffic(b) if not a.sparsify else None
     roofline = {"kernel": "quantize_pack_kernel<%d>" % b if not a.sparsify else "sparsify (l1 + count + emit)",
