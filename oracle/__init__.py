@@ -57,7 +57,7 @@ class Config(C.Structure):
                 ("l1", C.c_float), ("l2", C.c_float), ("box_lo", C.c_float), ("box_hi", C.c_float),
                 ("sparsify", C.c_int32), ("phi", C.c_float),
                 ("msg_format", C.c_int32), ("accelerated", C.c_int32), ("snapshot_flag", C.c_int32), ("pad_", C.c_int32),
-                ("seed", C.c_uint64), ("mu", C.c_float), ("pad2_", C.c_float)]
+                ("seed", C.c_uint64), ("mu", C.c_float), ("sequential", C.c_int32)]
 
 
 class State(C.Structure):
@@ -98,6 +98,7 @@ def _declare(L):
         "dqo_prox": (f32, [f32, f32, f32, f32, f32, f32]),
         "dqo_master_step": (None, [vp, vp, i32, i64, vp, vp, vp, vp, vp, f32, f32, i32, f32, f32, f32, f32, vp]),
         "dqo_epoch_begin": (None, [vp, vp, vp, f32, i64, vp]),
+        "dqo_master_step_sequential": (None, [vp, vp, i32, i64, vp, vp, vp, vp, vp, f32, f32, i32, f32, f32, f32, f32, vp]),
         "dqo_expected_sq_error": (f64, [vp, i64, i32]),
         "dqo_sq_distance": (f64, [vp, vp, i64]),
         "dqo_select_bx": (i32, [vp, vp, i64, f32, vp, vp]),
@@ -262,15 +263,16 @@ def prox(v, eta, l1, l2, lo, hi):
 
 
 def master_step(codes, delta, gfull, x, eta, theta=0.0, accelerated=False, y=None, xsnap=None, xsum=None,
-                l1=0.0, l2=0.0, lo=-np.inf, hi=np.inf):
-    """Updates x (and y, xsum) in place; returns ||x||_inf."""
+                l1=0.0, l2=0.0, lo=-np.inf, hi=np.inf, sequential=False):
+    """Updates x (and y, xsum) in place; returns ||x||_inf.  sequential: one prox step per message."""
     codes = np.ascontiguousarray(codes, dtype=np.int32); M, d = codes.shape
     delta = _f32(delta); gfull = _f32(gfull)
     for a in (x, y, xsum):
         assert a is None or (a.dtype == np.float32 and a.flags.c_contiguous)
     xsnap_ = None if xsnap is None else _f32(xsnap)
     nx = np.zeros(1, np.float32)
-    lib().dqo_master_step(_p(codes), _p(delta), M, d, _p(gfull), _p(x), _p(y), _p(xsnap_), _p(xsum),
+    fn = lib().dqo_master_step_sequential if sequential else lib().dqo_master_step
+    fn(_p(codes), _p(delta), M, d, _p(gfull), _p(x), _p(y), _p(xsnap_), _p(xsum),
                           float(eta), float(theta), int(accelerated), float(l1), float(l2), float(lo), float(hi), _p(nx))
     return nx[0]
 
@@ -291,9 +293,9 @@ def select_bx(x, xsnap, mu):
 
 # ---- drivers ------------------------------------------------------------------------
 def make_config(d, M, B, bx, b, l1=0.0, l2=0.0, box_lo=-np.inf, box_hi=np.inf, sparsify=0, phi=0.0,
-                msg_format=MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, mu=0.0):
+                msg_format=MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, mu=0.0, sequential=0):
     return Config(d, M, B, bx, b, l1, l2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                  int(snapshot_flag), 0, seed, mu, 0.0)
+                  int(snapshot_flag), 0, seed, mu, int(sequential))
 
 
 class Run:
@@ -307,12 +309,14 @@ class Run:
         self.z_snap = np.zeros(data.n, np.float32)
         self.state = State(_p(self.x), _p(self.xsnap), _p(self.gfull), _p(self.y), _p(self.xsum))
         self.rounds_in_epoch = 0
+        self.ticks_in_epoch = 0
         self.epoch = -1
 
     def epoch_begin(self, theta=0.0):
         lib().dqo_epoch_begin(C.addressof(self.cfg), self.data.ref, C.addressof(self.state), float(theta),
-                              self.rounds_in_epoch, _p(self.z_snap))
+                              self.ticks_in_epoch, _p(self.z_snap))       # Algorithm 3 averages over master ticks
         self.rounds_in_epoch = 0
+        self.ticks_in_epoch = 0
         self.epoch += 1
 
     def is_flag_round(self):
@@ -338,6 +342,7 @@ class Run:
         rc = lib().dqo_round(C.addressof(cfg), self.data.ref, C.addressof(self.state), round_, int(flag),
                              float(eta), float(theta), C.addressof(T))
         self.rounds_in_epoch += 1
+        self.ticks_in_epoch += cfg.M if cfg.sequential else 1
         keep.update(bits_down=int(T.bits_down), bits_up=int(T.bits_up), normx=np.float32(T.normx),
                     flag_round=bool(T.flag_round), bx_used=int(T.bx_used), status=rc)
         return keep

@@ -428,6 +428,35 @@ void dqo_master_step(const int32_t* codes /*[M][d]*/, const float* delta /*[M]*/
     if (normx) *normx = nx;
 }
 
+/* Master step 9 as Algorithm 1 states it, one message per master tick: the M
+ * workers of a round all pulled the model broadcast at the round's start, and
+ * the master applies their messages one after the other in worker order, each
+ * with its own semi-stochastic gradient u = Q(alpha_w) + grad f(xsnap) and its
+ * own prox step.  Message w therefore meets a model that is w ticks newer than
+ * the one it was computed on: the delay t - D(t) = w <= tau = M - 1 of
+ * Assumption 3.  Algorithm 3 updates y, x and the running sum at every tick. */
+void dqo_master_step_sequential(const int32_t* codes, const float* delta, int M, int64_t d,
+                                const float* gfull, float* x, float* y, const float* xsnap, float* xsum,
+                                float eta, float theta, int accelerated,
+                                float l1, float l2, float lo, float hi, float* normx)
+{
+    float nx = 0.0f;
+    for (int64_t i = 0; i < d; ++i) {
+        for (int w = 0; w < M; ++w) {
+            float u = (float)codes[(int64_t)w * d + i] * delta[w] + gfull[i];
+            if (!accelerated) {
+                x[i] = dqo_prox(fmaf(-eta, u, x[i]), eta, l1, l2, lo, hi);
+            } else {
+                y[i] = dqo_prox(fmaf(-eta, u, y[i]), eta, l1, l2, lo, hi);
+                x[i] = fmaf(theta, y[i] - xsnap[i], xsnap[i]);
+                xsum[i] = xsum[i] + x[i];
+            }
+        }
+        float a = fabsf(x[i]); if (a > nx) nx = a;
+    }
+    if (normx) *normx = nx;
+}
+
 /* ------------------------------------------------------------------------ */
 /* Model precision: the master quantises x "subject to" condition (3),        */
 /*   E_Q ||Q(x) - x||^2 <= mu ||x - xsnap||^2                                 */
@@ -481,7 +510,8 @@ typedef struct {
     int32_t sparsify; float phi;
     int32_t msg_format, accelerated, snapshot_flag, pad_;
     uint64_t seed;
-    float mu; float pad2_;          /* mu > 0: choose b_x per round by condition (3)/(6); 0: fixed b_x */
+    float mu;                       /* mu > 0: choose b_x per round by condition (3)/(6); 0: fixed b_x */
+    int32_t sequential;             /* 1: one prox step per message (dqo_master_step_sequential) */
 } dqo_config;
 
 typedef struct { float *x, *xsnap, *gfull, *y, *xsum; } dqo_state;
@@ -598,8 +628,9 @@ int dqo_round(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t rou
     /* master (ii), step 9 */
     float normx = 0.0f;
     if (rc == DQO_OK)
-        dqo_master_step(codes, delta, M, d, S->gfull, S->x, S->y, S->xsnap, S->xsum, eta, theta, C->accelerated,
-                        C->l1, C->l2, C->box_lo, C->box_hi, &normx);
+        (C->sequential ? dqo_master_step_sequential : dqo_master_step)(
+            codes, delta, M, d, S->gfull, S->x, S->y, S->xsnap, S->xsum, eta, theta, C->accelerated,
+            C->l1, C->l2, C->box_lo, C->box_hi, &normx);
     if (T) {
         if (T->codes) memcpy(T->codes, codes, (size_t)M * d * 4);
         if (T->delta) memcpy(T->delta, delta, (size_t)M * 4);

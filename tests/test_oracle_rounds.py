@@ -228,3 +228,52 @@ def test_round_with_searched_model_bits():
             assert tr["bits_down"] == M * (32 + want_b * h.d)
             seen.add(want_b)
     assert seen == {2, 4, 8} or seen >= {2, 8}
+
+
+def test_sequential_master_is_one_prox_svrg_step_per_message():
+    """Algorithm 1 as written applies one message per master tick.  The sequential master must equal M successive
+    textbook steps x <- prox(x - eta (Q(alpha_w) + grad f(xsnap))) in independent float64 numpy, reduce to the
+    synchronous master for M = 1, and for Algorithm 3 keep x = xsnap + theta (y - xsnap) with the running sum taking
+    every tick's x."""
+    g = np.random.default_rng(41)
+    d, M, eta, l1, l2 = 60, 5, 0.3, 0.02, 0.1
+    codes = g.integers(-7, 8, (M, d)).astype(np.int32); delta = (g.random(M) * 0.1).astype(F32)
+    gfull = g.standard_normal(d).astype(F32); x0 = g.standard_normal(d).astype(F32)
+    x = x0.copy()
+    nx = oracle.master_step(codes, delta, gfull, x, eta, l1=l1, l2=l2, sequential=True)
+    ref = x0.astype(np.float64)
+    for w in range(M):
+        u = codes[w].astype(np.float64) * float(delta[w]) + gfull
+        ref = _np_soft(ref - eta * u, eta * l1) / (1 + eta * l2)
+    assert np.allclose(x, ref, rtol=5e-6, atol=1e-6) and nx == np.abs(x).max()
+    # differs from the averaged step, but coincides with it for one worker
+    xa = x0.copy(); oracle.master_step(codes, delta, gfull, xa, eta, l1=l1, l2=l2)
+    assert np.abs(xa - x).max() > 1e-3
+    x1 = x0.copy(); x2 = x0.copy()
+    oracle.master_step(codes[:1], delta[:1], gfull, x1, eta, l1=l1, l2=l2, sequential=True)
+    oracle.master_step(codes[:1], delta[:1], gfull, x2, eta, l1=l1, l2=l2)
+    assert np.array_equal(x1, x2)
+    # Algorithm 3
+    theta = F32(0.4); xs = g.standard_normal(d).astype(F32); y0 = g.standard_normal(d).astype(F32)
+    y = y0.copy(); xx = x0.copy(); xsum = np.zeros(d, F32)
+    oracle.master_step(codes, delta, gfull, xx, eta, theta, True, y, xs, xsum, lo=-1.0, hi=1.0, sequential=True)
+    yr = y0.astype(np.float64); acc = np.zeros(d)
+    for w in range(M):
+        yr = np.clip(yr - eta * (codes[w] * float(delta[w]) + gfull), -1.0, 1.0)
+        acc += xs + float(theta) * (yr - xs)
+    assert np.allclose(y, yr, rtol=5e-6, atol=1e-6)
+    assert np.allclose(xx, xs + theta * (y - xs), rtol=1e-6, atol=1e-6) and np.allclose(xsum, acc, rtol=1e-5, atol=1e-5)
+
+
+def test_sequential_rounds_average_over_ticks():
+    h, data = _problem(n=200, d=25, seed=25)
+    M, m = 3, 4
+    cfg = oracle.make_config(h.d, M, 8, 8, 8, box_lo=-0.5, box_hi=0.5, accelerated=1, seed=15, sequential=1)
+    run = oracle.Run(cfg, data, synth.normal_vector(h.d, 35, 0.1))
+    theta = F32(0.5)
+    run.epoch_begin(theta)
+    for rnd in range(m):
+        run.round(rnd, 0.2, theta)
+    xsum = run.xsum.copy()
+    run.epoch_begin(theta)
+    assert np.allclose(run.xsnap, xsum / F32(m * M), rtol=1e-6, atol=1e-8)     # mean over the m*M master ticks
