@@ -81,7 +81,8 @@ typedef struct {
     uint64_t seed;
     int64_t sparse_cap;        /* entries per worker in the context's own sparse message buffers; 0: d   */
     float mu;                  /* > 0: dq_round picks b_x in {2,4,8} each round by condition (3)/(6); 0: fixed bx */
-    int32_t reserved;
+    int32_t sequential;        /* 1: master applies the M messages one by one, one prox step each (Algorithm 1 step 9 as
+                                  written; message w is w steps stale, delay <= M-1); 0: one step on their average */
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3

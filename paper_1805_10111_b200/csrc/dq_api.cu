@@ -275,6 +275,7 @@ int dq_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, void* stream)
     if (!s->x_snap || !s->z_snap || !aligned(s->x_snap, 16)) return DQ_ERR_ARG;
     launch_epoch_begin(ctx, s, theta, as_stream(stream));
     ctx->rounds_in_epoch = 0;
+    ctx->ticks_in_epoch = 0;
     ctx->epoch += 1;
     return last_error();
 }
@@ -379,6 +380,7 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
         if (rc != DQ_OK) return rc;
     }
     ctx->rounds_in_epoch += 1;
+    ctx->ticks_in_epoch += ctx->cfg.sequential ? ctx->cfg.M : 1;
     return last_error();
 }
 

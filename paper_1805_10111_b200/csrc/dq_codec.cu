@@ -631,6 +631,131 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
     block_atomic_max(nmax, normx_bits);
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Sequential master (Algorithm 1 step 9 as written): one prox step per message, in worker order; message w
+// meets a model that is w steps newer than the one it was computed on.  Same traffic as the averaged step,
+// M times the update arithmetic.  Each thread owns the 32/BITS coordinates of one code word.
+// ---------------------------------------------------------------------------------------------------
+template <int BITS, bool ACC>
+__global__ void __launch_bounds__(kThreads)
+master_dense_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
+                        const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
+                        const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
+                        uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
+{
+    if (rp) { eta = rp->eta; theta = rp->theta; }
+    if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
+    constexpr int C = 32 / BITS;
+    extern __shared__ float s_scale[];
+    for (int i = threadIdx.x; i < M; i += blockDim.x) s_scale[i] = scale[i];
+    __syncthreads();
+    const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
+    const int64_t nwords = (d + C - 1) / C, wstride = stride >> 2;
+    const uint32_t* words = reinterpret_cast<const uint32_t*>(codes);
+    float* target = ACC ? y : x;
+    uint32_t nmax = 0;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nwords; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i0 = t * C;
+        float cur[C], g[C], xs[C], sm[C], xo[C];
+#pragma unroll
+        for (int j = 0; j < C; ++j) {
+            const bool in = i0 + j < d;
+            cur[j] = in ? target[i0 + j] : 0.0f; g[j] = in ? g_full[i0 + j] : 0.0f;
+            xs[j] = (ACC && in) ? xsnap[i0 + j] : 0.0f; sm[j] = (ACC && in) ? xsum[i0 + j] : 0.0f;
+            xo[j] = cur[j];
+        }
+#pragma unroll 4
+        for (int w = 0; w < M; ++w) {
+            const uint32_t word = __ldg(words + (int64_t)w * wstride + t);
+            const float dl = s_scale[w];
+#pragma unroll
+            for (int j = 0; j < C; ++j) {
+                float yo = 0.0f;
+                xo[j] = master_update<ACC>((float)code_of<BITS>(word, j), dl, eta, theta, thr, den, pp, g[j], cur[j], xs[j], yo, sm[j]);
+                cur[j] = ACC ? yo : xo[j];
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < C; ++j) {
+            if (i0 + j < d) {
+                x[i0 + j] = xo[j];
+                if (ACC) { y[i0 + j] = cur[j]; xsum[i0 + j] = sm[j]; }
+                nmax = max(nmax, __float_as_uint(xo[j]) & 0x7FFFFFFFu);
+            }
+        }
+    }
+    block_atomic_max(nmax, normx_bits);
+}
+
+// Sparse messages, sequential: per tile, every worker's (possibly empty) message is expanded into shared memory and
+// followed by a prox sweep over the tile; each thread keeps its eight coordinates of the tile in registers.
+template <int BITS, bool ACC>
+__global__ void __launch_bounds__(kThreads)
+master_sparse_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale,
+                         const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* __restrict__ tile_ptr, int64_t ntiles,
+                         int M, int64_t d, const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
+                         const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
+                         uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
+{
+    if (rp) { eta = rp->eta; theta = rp->theta; }
+    if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
+    constexpr int R = kChunk / kThreads;                       // coordinates of the tile per thread
+    __shared__ float s_q[kChunk];
+    extern __shared__ uint32_t s_seg[];
+    const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
+    float* target = ACC ? y : x;
+    uint32_t nmax = 0;
+    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const int64_t lo = tile * kChunk;
+        for (int w = threadIdx.x; w < M; w += blockDim.x) {
+            const uint32_t* tp = tile_ptr + (int64_t)w * (ntiles + 1) + tile;
+            s_seg[2 * w] = tp[0]; s_seg[2 * w + 1] = tp[1];
+        }
+        float cur[R], g[R], xs[R], sm[R], xo[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int64_t i = lo + threadIdx.x + r * kThreads;
+            const bool in = i < d;
+            cur[r] = in ? target[i] : 0.0f; g[r] = in ? g_full[i] : 0.0f;
+            xs[r] = (ACC && in) ? xsnap[i] : 0.0f; sm[r] = (ACC && in) ? xsum[i] : 0.0f;
+            xo[r] = cur[r];
+        }
+        __syncthreads();
+        for (int w = 0; w < M; ++w) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) s_q[threadIdx.x + r * kThreads] = 0.0f;
+            __syncthreads();
+            const uint32_t e0 = s_seg[2 * w], e1 = s_seg[2 * w + 1];
+            const uint32_t* list = idx + (int64_t)w * cap;
+            const uint32_t* words = reinterpret_cast<const uint32_t*>(codes + (int64_t)w * stride);
+            for (uint32_t e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
+                const int64_t bit = (int64_t)e * BITS;
+                s_q[(int)((int64_t)list[e] - lo)] = (float)code_of<BITS>(__ldg(words + (bit >> 5)), (int)((bit & 31) / BITS));
+            }
+            __syncthreads();
+            const float dl = scale[w];
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                float yo = 0.0f;
+                xo[r] = master_update<ACC>(s_q[threadIdx.x + r * kThreads], dl, eta, theta, thr, den, pp, g[r], cur[r], xs[r], yo, sm[r]);
+                cur[r] = ACC ? yo : xo[r];
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+            const int64_t i = lo + threadIdx.x + r * kThreads;
+            if (i < d) {
+                x[i] = xo[r];
+                if (ACC) { y[i] = cur[r]; xsum[i] = sm[r]; }
+                nmax = max(nmax, __float_as_uint(xo[r]) & 0x7FFFFFFFu);
+            }
+        }
+        __syncthreads();
+    }
+    block_atomic_max(nmax, normx_bits);
+}
+
 // Test utility: dequantise one message into a dense fp32 vector.
 template <int BITS>
 __global__ void unpack_dense_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scale, int64_t d,
@@ -910,6 +1035,20 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
     ProxParams pp{c.lambda1, c.lambda2, c.box_lo, c.box_hi};
     uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
     if (!ctx->normx_zeroed) cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
+    if (c.sequential && !sparse_msgs) {
+        const int64_t nw = (d + (32 / c.b) - 1) / (32 / c.b);
+        const int grid = grid_for(nw, ctx->sm_count);
+        const size_t smem = sizeof(float) * c.M;
+        if (c.accelerated) {
+            DQ_DISPATCH_BITS(c.b, (master_dense_seq_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
+        } else {
+            DQ_DISPATCH_BITS(c.b, (master_dense_seq_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
+                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
+        }
+        ctx->launches += 1;
+        return;
+    }
     if (!sparse_msgs) {
         const int64_t cpt = c.b == 2 ? 16 : 8;               // coordinates per thread of master_dense_kernel
         const int64_t nwords = (d + cpt - 1) / cpt;
@@ -929,6 +1068,20 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         const int64_t ntiles = (d + kChunk - 1) / kChunk;
         dim3 grid_t((unsigned)((ntiles + 1 + kThreads - 1) / kThreads), c.M);
         tile_ptr_kernel<<<grid_t, kThreads, 0, st>>>(msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
+        if (c.sequential) {
+            const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
+            if (c.accelerated) {
+                DQ_DISPATCH_BITS(c.b, (master_sparse_seq_kernel<BITS_, true><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
+                    msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+                    s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
+            } else {
+                DQ_DISPATCH_BITS(c.b, (master_sparse_seq_kernel<BITS_, false><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
+                    msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+                    s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
+            }
+            ctx->launches += 2;
+            return;
+        }
         const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
         if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(

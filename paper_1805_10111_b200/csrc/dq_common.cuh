@@ -234,5 +234,6 @@ struct dq_ctx {
     // bookkeeping
     int64_t launches;
     int64_t rounds_in_epoch;
+    int64_t ticks_in_epoch;     // master steps since the epoch began (M per round in sequential mode)
     int64_t epoch;
 };

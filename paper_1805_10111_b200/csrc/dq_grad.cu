@@ -500,7 +500,7 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
     uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
     cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
     epoch_state_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(s->x, s->x_snap, s->y, s->x_sum, c.d, c.accelerated,
-                                                                            ctx->rounds_in_epoch, theta, nx);
+                                                                            ctx->ticks_in_epoch, theta, nx);
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * c.d, st);
     if (D.format == DQ_CSR_F32) {
         full_grad_csr_kernel<<<blocks_for(D.n * 32, ctx->sm_count), kThreads, 0, st>>>(

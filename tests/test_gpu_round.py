@@ -195,7 +195,7 @@ class Lockstep:
         okw = dict(l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0), box_lo=kw.get("box_lo", -np.inf),
                    box_hi=kw.get("box_hi", np.inf), sparsify=kw.get("sparsify", 0), phi=kw.get("phi", 0.0),
                    msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"],
-                   mu=kw.get("mu", 0.0))
+                   mu=kw.get("mu", 0.0), sequential=kw.get("sequential", 0))
         self.cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
         self.ocfg = oracle.make_config(h.d, kw["M"], kw["B"], kw["bx"], kw["b"], **okw)
         self.data = dq.Data(h)
@@ -285,7 +285,7 @@ class Lockstep:
         # master: bit-exact on the GPU's own codes
         x = x_before.copy(); y = y_before.copy(); xs = xsum_before.copy()
         nx = oracle.master_step(raw_gpu, scale, run.gfull, x, eta, theta, bool(cfg.accelerated), y, run.xsnap, xs,
-                                cfg.lambda1, cfg.lambda2, cfg.box_lo, cfg.box_hi)
+                                cfg.lambda1, cfg.lambda2, cfg.box_lo, cfg.box_hi, sequential=bool(cfg.sequential))
         assert np.array_equal(st.x.cpu().numpy(), x), ("x", rnd)
         assert st.norm_x.item() == nx
         if cfg.accelerated:
@@ -375,6 +375,29 @@ def test_lockstep_searched_model_bits(dq, mu, acc):
             tr = ls.round(rnd, 0.5, theta)
             widths.add(tr["bx_used"]); rnd += 1
     assert widths - {0} <= {2, 4, 8} and len(widths - {0}) >= 1
+    ls.close()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("dense8", dict(M=5, B=8, bx=8, b=8, lambda1=1e-3, lambda2=0.05, seed=16)),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, seed=17)),
+    ("csr", dict(M=4, B=16, bx=8, b=2, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=18)),
+    ("bf16", dict(M=3, B=16, bx=8, b=8, box_lo=-0.5, box_hi=0.5, accelerated=1, seed=19)),
+    ("csr", dict(M=3, B=16, bx=8, b=4, box_lo=-1.0, box_hi=1.0, accelerated=1, sparsify=1, phi=0.0, msg_format=1, seed=20)),
+])
+def test_lockstep_sequential_master(dq, name, kw):
+    """One prox step per message (delay up to M-1 master steps): bit-exact iterates, and Algorithm 3's snapshot is the
+    mean over master ticks."""
+    h = _problem(name)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 82, 0.05), sequential=1, **kw)
+    acc = kw.get("accelerated", 0)
+    rnd = 0
+    for s_ in range(1, 4):
+        theta = F32(2.0 / (s_ + 2)) if acc else F32(0.0)
+        ls.epoch(theta)
+        for t in range(6):
+            ls.round(rnd, 0.05 if acc else 0.3, theta)
+            rnd += 1
     ls.close()
 
 
