@@ -40,6 +40,7 @@ def parse_args():
     ap.add_argument("--bits", type=int, default=4)
     ap.add_argument("--workers", type=int, default=8)
     ap.add_argument("--sparsify", type=int, default=0)
+    ap.add_argument("--sequential", type=int, default=0, help="1: master applies one prox step per message")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--configs", default="c1,c2,c3,c4", help="training configurations to time with dq_round ('' for none)")
@@ -50,7 +51,7 @@ def workload_config(a):
     d = 1 << a.log2d
     return {"workload": "c5 quantiser/packer sweep point: d=2^%d, M=%d, b=%d, b_x=8, sparsify=%s, lambda1=1e-6, eta=0.1"
                         % (a.log2d, a.workers, a.bits, "on(phi=0.01d)" if a.sparsify else "off"),
-            "d": d, "M": a.workers, "b": a.bits, "bx": 8, "sparsify": a.sparsify,
+            "d": d, "M": a.workers, "b": a.bits, "bx": 8, "sparsify": a.sparsify, "sequential_master": a.sequential,
             "l2_policy": "inputs larger than L2 (%.0f MiB per round)" % (a.workers * d * 4 / 2 ** 20)}
 
 
@@ -260,7 +261,8 @@ def run_ours(a):
     dq.lib()
 
     d, M, b, bx, eta, seed = 1 << a.log2d, a.workers, a.bits, 8, 0.1, 1805
-    cfg = dq.make_config(d, M, b=b, bx=bx, seed=seed, lambda1=1e-6, sparsify=a.sparsify, phi=0.01 * d if a.sparsify else 0.0)
+    cfg = dq.make_config(d, M, b=b, bx=bx, seed=seed, lambda1=1e-6, sparsify=a.sparsify, phi=0.01 * d if a.sparsify else 0.0,
+                         sequential=a.sequential)
     rc, ctx = dq.dq_create(cfg); dq.ok(rc, "dq_create")
 
     # seeded synthetic inputs, generated on the host straight into pinned memory (also the e2e source)

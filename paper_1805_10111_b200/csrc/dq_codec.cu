@@ -631,6 +631,30 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
     block_atomic_max(nmax, normx_bits);
 }
 
+// The 32/BITS codes of one packed word as floats (same conversion-free trick as accumulate_word).
+template <int BITS>
+__device__ __forceinline__ void codes_as_float(uint32_t word, float (&kf)[32 / BITS])
+{
+    constexpr float kBias = 8388608.0f + (float)(1 << (BITS - 1));
+    if (BITS == 8) {
+        const uint32_t wb = word ^ 0x80808080u;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) kf[j] = __fsub_rn(__uint_as_float(__byte_perm(wb, 0x4B000000u, 0x7540u | j)), kBias);
+    } else if (BITS == 4) {
+        const uint32_t wb = word ^ 0x88888888u;
+        const uint32_t ev = wb & 0x0F0F0F0Fu, od = (wb >> 4) & 0x0F0F0F0Fu;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) kf[j] = __fsub_rn(__uint_as_float(__byte_perm((j & 1) ? od : ev, 0x4B000000u, 0x7540u | (j >> 1))), kBias);
+    } else {
+        const uint32_t wb = word ^ 0xAAAAAAAAu;
+        uint32_t p[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) p[k] = (wb >> (2 * k)) & 0x03030303u;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) kf[j] = __fsub_rn(__uint_as_float(__byte_perm(p[j & 3], 0x4B000000u, 0x7540u | (j >> 2))), kBias);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Sequential master (Algorithm 1 step 9 as written): one prox step per message, in worker order; message w
 // meets a model that is w steps newer than the one it was computed on.  Same traffic as the averaged step,
@@ -657,29 +681,56 @@ master_dense_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, const
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < nwords; t += (int64_t)gridDim.x * blockDim.x) {
         const int64_t i0 = t * C;
         float cur[C], g[C], xs[C], sm[C], xo[C];
+        const bool full = i0 + C <= d;                       // whole group inside the vector: 16-byte accesses
+        if (full) {
+#pragma unroll
+            for (int q = 0; q < C / 4; ++q) {
+                const float4 c4 = *reinterpret_cast<const float4*>(target + i0 + 4 * q), g4 = *reinterpret_cast<const float4*>(g_full + i0 + 4 * q);
+                cur[4 * q] = c4.x; cur[4 * q + 1] = c4.y; cur[4 * q + 2] = c4.z; cur[4 * q + 3] = c4.w;
+                g[4 * q] = g4.x; g[4 * q + 1] = g4.y; g[4 * q + 2] = g4.z; g[4 * q + 3] = g4.w;
+                if (ACC) {
+                    const float4 s4 = *reinterpret_cast<const float4*>(xsnap + i0 + 4 * q), m4 = *reinterpret_cast<const float4*>(xsum + i0 + 4 * q);
+                    xs[4 * q] = s4.x; xs[4 * q + 1] = s4.y; xs[4 * q + 2] = s4.z; xs[4 * q + 3] = s4.w;
+                    sm[4 * q] = m4.x; sm[4 * q + 1] = m4.y; sm[4 * q + 2] = m4.z; sm[4 * q + 3] = m4.w;
+                }
+            }
+        }
 #pragma unroll
         for (int j = 0; j < C; ++j) {
-            const bool in = i0 + j < d;
-            cur[j] = in ? target[i0 + j] : 0.0f; g[j] = in ? g_full[i0 + j] : 0.0f;
-            xs[j] = (ACC && in) ? xsnap[i0 + j] : 0.0f; sm[j] = (ACC && in) ? xsum[i0 + j] : 0.0f;
+            if (!full) {
+                const bool in = i0 + j < d;
+                cur[j] = in ? target[i0 + j] : 0.0f; g[j] = in ? g_full[i0 + j] : 0.0f;
+                xs[j] = (ACC && in) ? xsnap[i0 + j] : 0.0f; sm[j] = (ACC && in) ? xsum[i0 + j] : 0.0f;
+            } else if (!ACC) { xs[j] = 0.0f; sm[j] = 0.0f; }
             xo[j] = cur[j];
         }
 #pragma unroll 4
         for (int w = 0; w < M; ++w) {
             const uint32_t word = __ldg(words + (int64_t)w * wstride + t);
             const float dl = s_scale[w];
+            float kf[C];
+            codes_as_float<BITS>(word, kf);
 #pragma unroll
             for (int j = 0; j < C; ++j) {
                 float yo = 0.0f;
-                xo[j] = master_update<ACC>((float)code_of<BITS>(word, j), dl, eta, theta, thr, den, pp, g[j], cur[j], xs[j], yo, sm[j]);
+                xo[j] = master_update<ACC>(kf[j], dl, eta, theta, thr, den, pp, g[j], cur[j], xs[j], yo, sm[j]);
                 cur[j] = ACC ? yo : xo[j];
+            }
+        }
+        if (full) {
+#pragma unroll
+            for (int q = 0; q < C / 4; ++q) {
+                *reinterpret_cast<float4*>(x + i0 + 4 * q) = make_float4(xo[4 * q], xo[4 * q + 1], xo[4 * q + 2], xo[4 * q + 3]);
+                if (ACC) {
+                    *reinterpret_cast<float4*>(y + i0 + 4 * q) = make_float4(cur[4 * q], cur[4 * q + 1], cur[4 * q + 2], cur[4 * q + 3]);
+                    *reinterpret_cast<float4*>(xsum + i0 + 4 * q) = make_float4(sm[4 * q], sm[4 * q + 1], sm[4 * q + 2], sm[4 * q + 3]);
+                }
             }
         }
 #pragma unroll
         for (int j = 0; j < C; ++j) {
             if (i0 + j < d) {
-                x[i0 + j] = xo[j];
-                if (ACC) { y[i0 + j] = cur[j]; xsum[i0 + j] = sm[j]; }
+                if (!full) { x[i0 + j] = xo[j]; if (ACC) { y[i0 + j] = cur[j]; xsum[i0 + j] = sm[j]; } }
                 nmax = max(nmax, __float_as_uint(xo[j]) & 0x7FFFFFFFu);
             }
         }
