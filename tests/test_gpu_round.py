@@ -401,6 +401,44 @@ def test_lockstep_sequential_master(dq, name, kw):
     ls.close()
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=21)),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=22)),
+    ("bf16", dict(M=3, B=70, bx=8, b=8, box_lo=-1.0, box_hi=1.0, accelerated=1, seed=23)),
+])
+def test_graph_replay_equals_direct_launches(dq, name, kw):
+    """dq_round replays a captured CUDA graph by default; with no_graph = 1 it launches the same kernels one by one.
+    Both must leave identical bytes everywhere (CSR gradients use float atomics, so those are compared within the
+    float tolerance and the dense bf16 path bit for bit), also after switching to a second state (re-capture)."""
+    import torch
+    h = _problem(name)
+    data = dq.Data(h)
+    x0 = synth.normal_vector(h.d, 83, 0.05)
+    acc = bool(kw.get("accelerated", 0))
+    outs = []
+    for no_graph in (0, 1):
+        cfg = dq.make_config(h.d, kw["M"], no_graph=no_graph, **{k: v for k, v in kw.items() if k != "M"})
+        rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+        states = [dq.State(x0, n=h.n, accelerated=acc), dq.State(x0 * F32(0.5), n=h.n, accelerated=acc)]
+        bits = torch.zeros(2, dtype=torch.int64, device="cuda")
+        rnd = 0
+        for st in states:                                   # the second state forces a new capture
+            for epoch in range(2):
+                assert dq.dq_epoch_begin(ctx, st, 0.5 if acc else 0.0) == 0
+                for t in range(5):
+                    assert dq.dq_round(ctx, st, rnd, 0.05 if acc else 0.3, 0.5 if acc else 0.0, bits[0:1], bits[1:2]) == 0
+                    rnd += 1
+        assert dq.dq_poll_status(ctx) == (0, 0)
+        outs.append([st.x.cpu().numpy().copy() for st in states] + [bits.cpu().numpy().copy()])
+        dq.dq_destroy(ctx)
+    for a, b in zip(outs[0][:2], outs[1][:2]):
+        if name == "bf16":
+            assert np.array_equal(a, b)
+        else:
+            assert np.allclose(a, b, rtol=1e-4, atol=1e-6)
+    assert np.array_equal(outs[0][2], outs[1][2]) or name != "bf16"
+
+
 def test_select_model_bits_standalone(dq):
     import torch
     d = 100003
