@@ -57,7 +57,8 @@ class Config(C.Structure):
                 ("l1", C.c_float), ("l2", C.c_float), ("box_lo", C.c_float), ("box_hi", C.c_float),
                 ("sparsify", C.c_int32), ("phi", C.c_float),
                 ("msg_format", C.c_int32), ("accelerated", C.c_int32), ("snapshot_flag", C.c_int32), ("pad_", C.c_int32),
-                ("seed", C.c_uint64), ("mu", C.c_float), ("sequential", C.c_int32)]
+                ("seed", C.c_uint64), ("mu", C.c_float), ("sequential", C.c_int32),
+                ("model", C.c_int32), ("hidden", C.c_int32), ("classes", C.c_int32), ("pad3_", C.c_int32)]
 
 
 class State(C.Structure):
@@ -98,6 +99,11 @@ def _declare(L):
         "dqo_prox": (f32, [f32, f32, f32, f32, f32, f32]),
         "dqo_master_step": (None, [vp, vp, i32, i64, vp, vp, vp, vp, vp, f32, f32, i32, f32, f32, f32, f32, vp]),
         "dqo_epoch_begin": (None, [vp, vp, vp, f32, i64, vp]),
+        "dqo_mlp_params": (i64, [i64, i32, i32]),
+        "dqo_mlp_loss": (f64, [vp, i32, i32, vp, vp, i64]),
+        "dqo_mlp_grad": (None, [vp, i32, i32, vp, vp, i64, vp]),
+        "dqo_mlp_worker_grad": (None, [vp, i32, i32, vp, vp, vp, i32, vp, vp]),
+        "dqo_mlp_objective": (f64, [vp, i32, i32, vp, f32, f32]),
         "dqo_master_step_sequential": (None, [vp, vp, i32, i64, vp, vp, vp, vp, vp, f32, f32, i32, f32, f32, f32, f32, vp]),
         "dqo_expected_sq_error": (f64, [vp, i64, i32]),
         "dqo_sq_distance": (f64, [vp, vp, i64]),
@@ -257,6 +263,42 @@ def sample_batch(seed, round_, w, M, n, B):
     return rows
 
 
+# ---- the 3-layer network --------------------------------------------------------------------------------
+MODEL_LOGISTIC, MODEL_MLP = 0, 1
+
+
+def mlp_params(n_in, hidden, classes):
+    return int(lib().dqo_mlp_params(n_in, hidden, classes))
+
+
+def mlp_loss(data, hidden, classes, x, rows=None):
+    x = _f32(x)
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    return float(lib().dqo_mlp_loss(data.ref, hidden, classes, _p(x), _p(r), data.n if r is None else r.size))
+
+
+def mlp_grad(data, hidden, classes, x, rows=None):
+    x = _f32(x)
+    r = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    g = np.zeros(mlp_params(data.d, hidden, classes), np.float32)
+    lib().dqo_mlp_grad(data.ref, hidden, classes, _p(x), _p(r), data.n if r is None else r.size, _p(g))
+    return g
+
+
+def mlp_worker_grad(data, hidden, classes, xhat, xsnap, rows):
+    xhat, xsnap = _f32(xhat), _f32(xsnap)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    P = mlp_params(data.d, hidden, classes)
+    alpha = np.zeros(P, np.float32); S = np.zeros(P, np.float32)
+    lib().dqo_mlp_worker_grad(data.ref, hidden, classes, _p(xhat), _p(xsnap), _p(rows), rows.size, _p(alpha), _p(S))
+    return alpha, S
+
+
+def mlp_objective(data, hidden, classes, x, l1, l2):
+    x = _f32(x)
+    return float(lib().dqo_mlp_objective(data.ref, hidden, classes, _p(x), float(l1), float(l2)))
+
+
 # ---- master -----------------------------------------------------------------------
 def prox(v, eta, l1, l2, lo, hi):
     return np.float32(lib().dqo_prox(float(v), float(eta), float(l1), float(l2), float(lo), float(hi)))
@@ -293,9 +335,9 @@ def select_bx(x, xsnap, mu):
 
 # ---- drivers ------------------------------------------------------------------------
 def make_config(d, M, B, bx, b, l1=0.0, l2=0.0, box_lo=-np.inf, box_hi=np.inf, sparsify=0, phi=0.0,
-                msg_format=MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, mu=0.0, sequential=0):
+                msg_format=MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, mu=0.0, sequential=0, model=0, hidden=0, classes=0):
     return Config(d, M, B, bx, b, l1, l2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                  int(snapshot_flag), 0, seed, mu, int(sequential))
+                  int(snapshot_flag), 0, seed, mu, int(sequential), int(model), int(hidden), int(classes), 0)
 
 
 class Run:

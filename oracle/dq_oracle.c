@@ -368,6 +368,115 @@ double dqo_objective(const dqo_data* D, const float* x, float l1, float l2)
     return dqo_smooth_loss(D, x) + (double)l1 * a + 0.5 * (double)l2 * q;
 }
 
+/* ------------------------------------------------------------------------ */
+/* Second smooth part (Section 5.2): a 3-layer fully connected network,      */
+/* input -> hidden (ReLU) -> classes, softmax cross-entropy.  The parameter   */
+/* vector is x = [W1 (hidden x in, row-major), b1 (hidden), W2 (classes x     */
+/* hidden), b2 (classes)]; labels hold the class index.  The L2 regulariser   */
+/* of Section 5.2 lives in h like the others.                                 */
+/* ------------------------------------------------------------------------ */
+int64_t dqo_mlp_params(int64_t in, int hidden, int classes) { return (int64_t)hidden * (in + 1) + (int64_t)classes * (hidden + 1); }
+
+/* Loss of one sample; if grad != NULL adds w * d loss / d x to grad and, if mag != NULL, the absolute values of the
+ * same terms to mag (for tolerances). */
+static double mlp_sample(const float* a, int label, int64_t in, int hidden, int classes, const float* x,
+                         double w, double* grad, double* mag)
+{
+    const float* W1 = x; const float* b1 = W1 + (int64_t)hidden * in;
+    const float* W2 = b1 + hidden; const float* b2 = W2 + (int64_t)classes * hidden;
+    double* h = (double*)malloc(sizeof(double) * (size_t)(hidden + 2 * classes));
+    double* z = h + hidden; double* p = z + classes;
+    for (int j = 0; j < hidden; ++j) {
+        double s = (double)b1[j];
+        for (int64_t i = 0; i < in; ++i) s += (double)W1[(int64_t)j * in + i] * (double)a[i];
+        h[j] = s > 0.0 ? s : 0.0;
+    }
+    double zmax = -INFINITY;
+    for (int c = 0; c < classes; ++c) {
+        double s = (double)b2[c];
+        for (int j = 0; j < hidden; ++j) s += (double)W2[(int64_t)c * hidden + j] * h[j];
+        z[c] = s; if (s > zmax) zmax = s;
+    }
+    double sum = 0.0;
+    for (int c = 0; c < classes; ++c) { p[c] = exp(z[c] - zmax); sum += p[c]; }
+    for (int c = 0; c < classes; ++c) p[c] /= sum;
+    double loss = -(z[label] - zmax - log(sum));
+    if (grad) {
+        double* gW1 = grad; double* gb1 = gW1 + (int64_t)hidden * in; double* gW2 = gb1 + hidden; double* gb2 = gW2 + (int64_t)classes * hidden;
+        double* mW1 = mag; double* mb1 = mag ? mW1 + (int64_t)hidden * in : NULL; double* mW2 = mag ? mb1 + hidden : NULL;
+        double* mb2 = mag ? mW2 + (int64_t)classes * hidden : NULL;
+        double* dh = (double*)calloc((size_t)hidden, sizeof(double));
+        for (int c = 0; c < classes; ++c) {
+            double dz = w * (p[c] - (c == label ? 1.0 : 0.0));
+            gb2[c] += dz; if (mag) mb2[c] += fabs(dz);
+            for (int j = 0; j < hidden; ++j) {
+                gW2[(int64_t)c * hidden + j] += dz * h[j]; if (mag) mW2[(int64_t)c * hidden + j] += fabs(dz * h[j]);
+                dh[j] += dz * (double)W2[(int64_t)c * hidden + j];
+            }
+        }
+        for (int j = 0; j < hidden; ++j) {
+            if (h[j] <= 0.0) continue;                                   /* ReLU gate */
+            gb1[j] += dh[j]; if (mag) mb1[j] += fabs(dh[j]);
+            for (int64_t i = 0; i < in; ++i) {
+                gW1[(int64_t)j * in + i] += dh[j] * (double)a[i]; if (mag) mW1[(int64_t)j * in + i] += fabs(dh[j] * (double)a[i]);
+            }
+        }
+        free(dh);
+    }
+    free(h);
+    return loss;
+}
+
+/* f(x) = (1/n) sum_i loss_i(x) over the rows listed (rows == NULL: all n rows). */
+double dqo_mlp_loss(const dqo_data* D, int hidden, int classes, const float* x, const int64_t* rows, int64_t count)
+{
+    double s = 0.0;
+    for (int64_t k = 0; k < count; ++k) {
+        int64_t a = rows ? rows[k] : k;
+        s += mlp_sample((const float*)D->values + a * D->d, (int)D->labels[a], D->d, hidden, classes, x, 0.0, NULL, NULL);
+    }
+    return s / (double)count;
+}
+
+/* g = (1/count) sum grad loss_i(x) over the listed rows, rounded to fp32 once. */
+void dqo_mlp_grad(const dqo_data* D, int hidden, int classes, const float* x, const int64_t* rows, int64_t count, float* g)
+{
+    int64_t P = dqo_mlp_params(D->d, hidden, classes);
+    double* acc = (double*)calloc((size_t)P, sizeof(double));
+    for (int64_t k = 0; k < count; ++k) {
+        int64_t a = rows ? rows[k] : k;
+        mlp_sample((const float*)D->values + a * D->d, (int)D->labels[a], D->d, hidden, classes, x, 1.0 / (double)count, acc, NULL);
+    }
+    for (int64_t i = 0; i < P; ++i) g[i] = (float)acc[i];
+    free(acc);
+}
+
+/* Worker step 11 for the network: alpha = minibatch grad at xhat minus minibatch grad at xsnap; S = sum of the
+ * absolute per-sample terms of both gradients (tolerance scale). */
+void dqo_mlp_worker_grad(const dqo_data* D, int hidden, int classes, const float* xhat, const float* xsnap,
+                         const int64_t* rows, int B, float* alpha, float* S)
+{
+    int64_t P = dqo_mlp_params(D->d, hidden, classes);
+    double* acc = (double*)calloc((size_t)P, sizeof(double));
+    double* mag = (double*)calloc((size_t)P, sizeof(double));
+    for (int k = 0; k < B; ++k) {
+        const float* a = (const float*)D->values + rows[k] * D->d; int label = (int)D->labels[rows[k]];
+        mlp_sample(a, label, D->d, hidden, classes, xhat, 1.0 / (double)B, acc, mag);
+        mlp_sample(a, label, D->d, hidden, classes, xsnap, -1.0 / (double)B, acc, mag);
+    }
+    for (int64_t i = 0; i < P; ++i) { alpha[i] = (float)acc[i]; if (S) S[i] = (float)mag[i]; }
+    free(acc); free(mag);
+}
+
+/* P(x) = f(x) + h(x) for the network. */
+double dqo_mlp_objective(const dqo_data* D, int hidden, int classes, const float* x, float l1, float l2)
+{
+    int64_t P = dqo_mlp_params(D->d, hidden, classes);
+    double a = 0.0, q = 0.0;
+    for (int64_t i = 0; i < P; ++i) { a += fabs((double)x[i]); q += (double)x[i] * (double)x[i]; }
+    return dqo_mlp_loss(D, hidden, classes, x, NULL, D->n) + (double)l1 * a + 0.5 * (double)l2 * q;
+}
+
 /* Worker w keeps the contiguous partition [floor(w n/M), floor((w+1) n/M))
  * (Section 3.2: "keeps a disjoint partition") and draws its minibatch from it
  * with replacement: slot j takes word (j & 3) of Philox counter
@@ -512,6 +621,7 @@ typedef struct {
     uint64_t seed;
     float mu;                       /* mu > 0: choose b_x per round by condition (3)/(6); 0: fixed b_x */
     int32_t sequential;             /* 1: one prox step per message (dqo_master_step_sequential) */
+    int32_t model, hidden, classes, pad3_;   /* model 0: logistic regression; 1: the 3-layer network */
 } dqo_config;
 
 typedef struct { float *x, *xsnap, *gfull, *y, *xsum; } dqo_state;
@@ -546,7 +656,8 @@ void dqo_epoch_begin(const dqo_config* C, const dqo_data* D, dqo_state* S, float
         if (m_prev > 0) for (int64_t i = 0; i < d; ++i) S->xsnap[i] = S->xsum[i] / (float)m_prev;
         for (int64_t i = 0; i < d; ++i) { S->xsum[i] = 0.0f; S->x[i] = fmaf(theta, S->y[i] - S->xsnap[i], S->xsnap[i]); }
     }
-    dqo_full_grad(D, S->xsnap, S->gfull, z_snap);
+    if (C->model == 1) dqo_mlp_grad(D, C->hidden, C->classes, S->xsnap, NULL, D->n, S->gfull);
+    else dqo_full_grad(D, S->xsnap, S->gfull, z_snap);
 }
 
 /* One inner iteration (Algorithm 1 steps 6-13, with Algorithm 2's step 12-13
@@ -597,7 +708,8 @@ int dqo_round(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t rou
         int64_t nnz = d;
         float ninf = 0.0f, n1 = 0.0f, phi_eff = 0.0f;
         dqo_sample_batch(C->seed, round, w, M, D->n, B, rows);
-        dqo_worker_grad(D, xhat, S->xsnap, rows, B, alpha, Sabs);
+        if (C->model == 1) dqo_mlp_worker_grad(D, C->hidden, C->classes, xhat, S->xsnap, rows, B, alpha, Sabs);
+        else dqo_worker_grad(D, xhat, S->xsnap, rows, B, alpha, Sabs);
         if (C->sparsify) {
             rc = dqo_sparsify(alpha, d, C->phi, C->seed, round, (uint32_t)w, beta, Z, NULL, &ninf, &n1, &phi_eff);
             if (rc == DQO_OK) rc = dqo_quantize_survivors(beta, Z, d, C->b, C->seed, round, (uint32_t)w, cw, &delta[w]);

@@ -118,6 +118,26 @@ def normal_vector(d: int, seed_k: int, scale: float = 1.0) -> np.ndarray:
     return (rng(seed_k).standard_normal(d, dtype=np.float32) * np.float32(scale)).astype(np.float32)
 
 
+def image_classification(n: int, n_in: int, classes: int, seed_k: int) -> HostData:
+    """Inputs shaped like small grey-scale images (values in [0,1], about 80 % exactly zero, the rest a smooth
+    random blob per class plus noise) with the class index as label: stands in for the MNIST subset of Section 5.2."""
+    g = rng(seed_k)
+    proto = g.random((classes, n_in), dtype=np.float32) ** 4                  # class prototypes, mostly dark
+    y = g.integers(0, classes, n)
+    X = proto[y] + np.float32(0.15) * g.standard_normal((n, n_in), dtype=np.float32)
+    X = np.clip(X, 0.0, 1.0).astype(np.float32)
+    X[X < 0.35] = 0.0
+    return HostData(DENSE_F32, n, n_in, np.ascontiguousarray(X), y.astype(np.float32))
+
+
+def mlp_init(n_in: int, hidden: int, classes: int, seed_k: int) -> np.ndarray:
+    """Small random weights, zero biases, in the flat layout [W1, b1, W2, b2]."""
+    g = rng(seed_k)
+    w1 = g.standard_normal((hidden, n_in), dtype=np.float32) * np.float32(1.0 / np.sqrt(n_in))
+    w2 = g.standard_normal((classes, hidden), dtype=np.float32) * np.float32(1.0 / np.sqrt(hidden))
+    return np.concatenate([w1.ravel(), np.zeros(hidden, np.float32), w2.ravel(), np.zeros(classes, np.float32)]).astype(np.float32)
+
+
 # ---- the five configurations ---------------------------------------------------------------------------
 def config1() -> HostData:
     """Tiny dense L1 logistic regression: n=2,000, d=1,000."""
@@ -137,6 +157,11 @@ def config3(n: int = 200000, d: int = 1 << 20) -> HostData:
 def config4(n: int = 65536, d: int = 4096) -> HostData:
     """Dense bf16 features for the tensor-core path."""
     return dense_bf16_logistic(n, d, 4)
+
+
+def config_nn(n: int = 10000):
+    """MNIST-shaped classification data for the 3-layer network (784-100-10)."""
+    return image_classification(n, 784, 10, 8)
 
 
 def config5(d: int, M: int = 8):
