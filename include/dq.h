@@ -52,6 +52,7 @@ enum {
 
 enum { DQ_DENSE_F32 = 0, DQ_CSR_F32 = 1, DQ_DENSE_BF16 = 2 };   /* dq_data.format */
 enum { DQ_MSG_DENSE = 0, DQ_MSG_SPARSE = 1 };                   /* dq_config.msg_format */
+enum { DQ_MODEL_LOGISTIC = 0, DQ_MODEL_MLP = 1 };               /* dq_config.model */
 
 /* The training set {a_i, y_i} of eq. (1).  values: DENSE_F32 [n][d] float; DENSE_BF16 [n][d] bfloat16;
  * CSR_F32 [nnz] float with col_idx [nnz] (ascending inside a row, < d) and row_ptr [n+1].  labels [n] = +-1.
@@ -83,6 +84,12 @@ typedef struct {
     float mu;                  /* > 0: dq_round picks b_x in {2,4,8} each round by condition (3)/(6); 0: fixed bx */
     int32_t sequential;        /* 1: master applies the M messages one by one, one prox step each (Algorithm 1 step 9 as
                                   written; message w is w steps stale, delay <= M-1); 0: one step on their average */
+    int32_t model;             /* DQ_MODEL_LOGISTIC (default) or DQ_MODEL_MLP: the 3-layer fully connected network of
+                                  Section 5.2, in -> hidden (ReLU) -> classes with softmax cross-entropy.  For the network
+                                  the data must be DQ_DENSE_F32 with labels = class index, data.d = number of inputs, and
+                                  d = hidden*(in+1) + classes*(hidden+1) with x = [W1 (hidden x in), b1, W2 (classes x hidden), b2] */
+    int32_t hidden, classes;
+    int32_t reserved2;
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3

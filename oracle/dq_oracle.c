@@ -384,12 +384,13 @@ static double mlp_sample(const float* a, int label, int64_t in, int hidden, int 
 {
     const float* W1 = x; const float* b1 = W1 + (int64_t)hidden * in;
     const float* W2 = b1 + hidden; const float* b2 = W2 + (int64_t)classes * hidden;
-    double* h = (double*)malloc(sizeof(double) * (size_t)(hidden + 2 * classes));
-    double* z = h + hidden; double* p = z + classes;
+    double* h = (double*)malloc(sizeof(double) * (size_t)(2 * hidden + 2 * classes));
+    double* z = h + hidden; double* p = z + classes; double* habs = p + classes;
     for (int j = 0; j < hidden; ++j) {
-        double s = (double)b1[j];
-        for (int64_t i = 0; i < in; ++i) s += (double)W1[(int64_t)j * in + i] * (double)a[i];
+        double s = (double)b1[j], sa = fabs((double)b1[j]);
+        for (int64_t i = 0; i < in; ++i) { double t = (double)W1[(int64_t)j * in + i] * (double)a[i]; s += t; sa += fabs(t); }
         h[j] = s > 0.0 ? s : 0.0;
+        habs[j] = sa;             /* magnitude of the terms behind h_j: a hidden unit near its kink is a cancelling sum */
     }
     double zmax = -INFINITY;
     for (int c = 0; c < classes; ++c) {
@@ -410,7 +411,7 @@ static double mlp_sample(const float* a, int label, int64_t in, int hidden, int 
             double dz = w * (p[c] - (c == label ? 1.0 : 0.0));
             gb2[c] += dz; if (mag) mb2[c] += fabs(dz);
             for (int j = 0; j < hidden; ++j) {
-                gW2[(int64_t)c * hidden + j] += dz * h[j]; if (mag) mW2[(int64_t)c * hidden + j] += fabs(dz * h[j]);
+                gW2[(int64_t)c * hidden + j] += dz * h[j]; if (mag) mW2[(int64_t)c * hidden + j] += fabs(dz) * habs[j];
                 dh[j] += dz * (double)W2[(int64_t)c * hidden + j];
             }
         }

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_PKG, "libdq.so")
 DQ_OK, DQ_ERR_ARG, DQ_ERR_SHAPE, DQ_ERR_BITS, DQ_ERR_NONFINITE, DQ_ERR_CAPACITY, DQ_ERR_CUDA, DQ_ERR_TIMEOUT = range(8)
 DQ_DENSE_F32, DQ_CSR_F32, DQ_DENSE_BF16 = 0, 1, 2
 DQ_MSG_DENSE, DQ_MSG_SPARSE = 0, 1
+DQ_MODEL_LOGISTIC, DQ_MODEL_MLP = 0, 1
 
 EXPORTS = ["dq_packed_bytes", "dq_create", "dq_destroy", "dq_epoch_begin", "dq_quantize_model", "dq_worker_grad",
            "dq_norm_inf", "dq_quantize_sparsify_pack", "dq_master_unpack_aggregate_prox", "dq_round", "dq_codec_round",
@@ -32,7 +33,8 @@ class dq_config(C.Structure):
     _fields_ = [("d", C.c_int64), ("M", C.c_int32), ("B", C.c_int32), ("bx", C.c_int32), ("b", C.c_int32),
                 ("lambda1", C.c_float), ("lambda2", C.c_float), ("box_lo", C.c_float), ("box_hi", C.c_float),
                 ("sparsify", C.c_int32), ("phi", C.c_float), ("msg_format", C.c_int32), ("accelerated", C.c_int32),
-                ("snapshot_flag", C.c_int32), ("no_graph", C.c_int32), ("seed", C.c_uint64), ("sparse_cap", C.c_int64), ("mu", C.c_float), ("sequential", C.c_int32)]
+                ("snapshot_flag", C.c_int32), ("no_graph", C.c_int32), ("seed", C.c_uint64), ("sparse_cap", C.c_int64), ("mu", C.c_float), ("sequential", C.c_int32),
+                ("model", C.c_int32), ("hidden", C.c_int32), ("classes", C.c_int32), ("reserved2", C.c_int32)]
 
 
 class dq_state(C.Structure):
@@ -160,9 +162,9 @@ class Msgs:
 
 
 def make_config(d, M, B=1, bx=8, b=8, lambda1=0.0, lambda2=0.0, box_lo=float("-inf"), box_hi=float("inf"), sparsify=0,
-                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0, sequential=0) -> dq_config:
+                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0, sequential=0, model=0, hidden=0, classes=0) -> dq_config:
     return dq_config(d, M, B, bx, b, lambda1, lambda2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, int(sequential))
+                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, int(sequential), int(model), int(hidden), int(classes), 0)
 
 
 # ---- entry points (same names and order of arguments as include/dq.h) ---------------------------------------------

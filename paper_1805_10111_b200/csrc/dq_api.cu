@@ -85,7 +85,13 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (cfg->sparse_cap < 0 || cfg->sparse_cap > cfg->d) return DQ_ERR_ARG;
     if (!(cfg->mu >= 0.0f)) return DQ_ERR_ARG;
     if (data) {
-        if (data->n < 1 || data->d != cfg->d || !data->values || !data->labels) return DQ_ERR_SHAPE;
+        if (data->n < 1 || !data->values || !data->labels) return DQ_ERR_SHAPE;
+        if (cfg->model == DQ_MODEL_MLP) {
+            if (data->format != DQ_DENSE_F32 || cfg->hidden < 1 || cfg->classes < 2 || data->d < 1) return DQ_ERR_ARG;
+            if (cfg->d != (int64_t)cfg->hidden * (data->d + 1) + (int64_t)cfg->classes * (cfg->hidden + 1)) return DQ_ERR_SHAPE;
+        } else if (cfg->model != DQ_MODEL_LOGISTIC || data->d != cfg->d) {
+            return DQ_ERR_SHAPE;
+        }
         if (data->format == DQ_CSR_F32 && (!data->col_idx || !data->row_ptr)) return DQ_ERR_ARG;
         if (data->format < DQ_DENSE_F32 || data->format > DQ_DENSE_BF16) return DQ_ERR_ARG;
         if (!aligned(data->values, 16)) return DQ_ERR_ARG;
@@ -133,6 +139,15 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
         rc |= dev_alloc(&c->xhat_diff, (size_t)d);
         rc |= dev_alloc(&c->g64, (size_t)d);
         rc |= dev_alloc(&c->rbuf, (size_t)M * cfg->B);
+        if (cfg->model == DQ_MODEL_MLP) {
+            const size_t rmax = (size_t)((int64_t)M * cfg->B > data->n ? (int64_t)M * cfg->B : data->n);
+            rc |= dev_alloc(&c->mlp_rows, rmax);
+            for (int k = 0; k < 2; ++k) {
+                rc |= dev_alloc(&c->mlp_act[k], rmax * cfg->hidden);
+                rc |= dev_alloc(&c->mlp_dh[k], rmax * cfg->hidden);
+                rc |= dev_alloc(&c->mlp_dz[k], rmax * cfg->classes);
+            }
+        }
         c->list_mode = sparse && data->format == DQ_CSR_F32;
         if (c->list_mode) {
             c->glist_cap = (d + 7) / 8;
@@ -159,7 +174,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -300,15 +315,16 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
         const uint32_t* nx = reinterpret_cast<const uint32_t*>(s->norm_x);
         float* zf = worker_accumulates(ctx) ? ctx->alpha : nullptr;
         const int64_t zn = worker_accumulates(ctx) ? (int64_t)ctx->cfg.M * ctx->cfg.d : 0;
+        const float* ref = ctx->cfg.model == DQ_MODEL_MLP ? nullptr : s->x_snap;    // the network wants xhat itself
         if (!adaptive) {
             launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx),
-                                 ctx->delta_x, round, kMaster, kStreamModel, as_stream(st), s->x_snap, ctx->xhat_diff, zf, zn,
+                                 ctx->delta_x, round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
                                  reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
         } else {     // condition (3): pick the width on the device, then launch all three widths; two return at once
             launch_select_bits(ctx, s->x, s->x_snap, nx, ctx->cfg.mu, theta, ctx->bx_dev, ctx->prec_stats, as_stream(st));
             for (int bits = 2; bits <= 8; bits *= 2)
                 launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, bits, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, bits), ctx->delta_x,
-                                     round, kMaster, kStreamModel, as_stream(st), s->x_snap, ctx->xhat_diff, zf, zn,
+                                     round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
                                      reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M, ctx->bx_dev);
         }
         ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = ctx->normx_zeroed = true;

@@ -85,7 +85,7 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
             for (int j = 0; j < 8; ++j) {
                 if (i0 + j < d) {
                     const float k = (float)((int)((s[j] >> 16) & 0xFFu) - 128);
-                    diff[i0 + j] = __fsub_rn(__fmul_rn(k, delta), ref[i0 + j]);
+                    diff[i0 + j] = __fsub_rn(__fmul_rn(k, delta), ref ? ref[i0 + j] : 0.0f);
                 }
             }
         }

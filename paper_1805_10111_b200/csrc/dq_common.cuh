@@ -211,6 +211,8 @@ struct dq_ctx {
     double* g64;                // [d] full-gradient accumulator
     float* rbuf;                // [M][B] slope differences of the sampled rows
     int32_t* bx_dev;            // model width chosen by condition (3) this round
+    // network workload: sampled-row indices and per-row activations / derivatives of the two parameter vectors
+    int32_t* mlp_rows; float* mlp_act[2]; float* mlp_dz[2]; float* mlp_dh[2];
     double* prec_stats;         // [4] expected errors at 2/4/8 bits and ||x - xsnap||^2
     dq_msgs msgs;
     uint64_t* bits;             // [2] device counters

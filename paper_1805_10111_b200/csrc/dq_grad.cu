@@ -2,6 +2,7 @@
 // full gradient (step 5), the epoch-boundary state update (steps 3/14, Algorithm 3 steps 3/15), the
 // objective of eq. (1) and the transmitted-bit counters.  f_a(x) = log(1 + exp(-y_a <a_a, x>)).
 #include <cuda_bf16.h>
+#include <type_traits>
 
 #include "dq_common.cuh"
 #include "dq_kernels.cuh"
@@ -96,7 +97,7 @@ __global__ void dequant_diff_kernel(const uint8_t* __restrict__ codes, const flo
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t bit = i * BITS;
         const int k = code_of<BITS>(reinterpret_cast<const uint32_t*>(codes)[bit >> 5], (int)((bit & 31) / BITS));
-        diff[i] = __fsub_rn(__fmul_rn((float)k, dl), xsnap[i]);
+        diff[i] = __fsub_rn(__fmul_rn((float)k, dl), xsnap ? xsnap[i] : 0.0f);
     }
 }
 
@@ -485,6 +486,160 @@ __global__ void bits_kernel(int M, int64_t d, int bx, int b, int flag_round, int
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Second smooth part (Section 5.2): 3-layer fully connected network, in -> hidden (ReLU) -> classes, softmax
+// cross-entropy.  Parameters x = [W1 (hidden x in, row-major), b1, W2 (classes x hidden), b2]; labels hold class
+// indices.  The worker needs grad f_B(xhat) - grad f_B(xsnap): three small kernels evaluate both parameter
+// vectors side by side (either may be absent: NULL), rows listed explicitly or drawn from the batch stream.
+//   mlp_hidden_kernel   block per sampled row: hidden activations (one warp per hidden unit, coalesced along in)
+//   mlp_output_kernel   block per sampled row: logits, softmax, d loss / d logits, d loss / d hidden (ReLU-gated)
+//   mlp_param_kernel    block per (hidden unit or the tail, worker): sums over the worker's rows, no atomics
+// ---------------------------------------------------------------------------------------------------
+struct MlpShape { int64_t in; int hidden, classes; };
+
+__device__ __forceinline__ int64_t mlp_off_b1(const MlpShape& s) { return (int64_t)s.hidden * s.in; }
+__device__ __forceinline__ int64_t mlp_off_w2(const MlpShape& s) { return mlp_off_b1(s) + s.hidden; }
+__device__ __forceinline__ int64_t mlp_off_b2(const MlpShape& s) { return mlp_off_w2(s) + (int64_t)s.classes * s.hidden; }
+
+__global__ void __launch_bounds__(kThreads)
+mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restrict__ xa, const float* __restrict__ xb,
+                  const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
+                  float* __restrict__ act_a, float* __restrict__ act_b)
+{
+    extern __shared__ float s_in[];                      // the row's features
+    __shared__ int64_t s_row;
+    clear_word(bs);
+    const int64_t slot = blockIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        const int64_t a = B > 0 ? batch_row(bs, K, (int)(slot / B), (int)(slot % B), B, true) : slot;   // B = 0: row = slot
+        s_row = a; if (row_of_slot) row_of_slot[slot] = (int32_t)a;
+    }
+    __syncthreads();
+    const float* row = X + s_row * sh.in;
+    for (int64_t i = threadIdx.x; i < sh.in; i += blockDim.x) s_in[i] = row[i];
+    __syncthreads();
+    for (int j = warp; j < sh.hidden; j += kThreads / 32) {
+        float sa = 0.0f, sb = 0.0f;
+        for (int64_t i = lane; i < sh.in; i += 32) {
+            const float f = s_in[i];
+            if (xa) sa = fmaf(xa[(int64_t)j * sh.in + i], f, sa);
+            if (xb) sb = fmaf(xb[(int64_t)j * sh.in + i], f, sb);
+        }
+        sa = warp_sum(sa); sb = warp_sum(sb);
+        if (lane == 0) {
+            if (xa) act_a[slot * sh.hidden + j] = fmaxf(sa + xa[mlp_off_b1(sh) + j], 0.0f);
+            if (xb) act_b[slot * sh.hidden + j] = fmaxf(sb + xb[mlp_off_b1(sh) + j], 0.0f);
+        }
+    }
+}
+
+// One model of one row: logits -> softmax -> dz = (p - onehot) * wgt, dh_j = relu'(h_j) sum_c dz_c W2[c][j]; returns loss.
+__device__ __forceinline__ void mlp_output_one(const MlpShape& sh, const float* __restrict__ x, const float* __restrict__ act,
+                                               int label, float wgt, float* __restrict__ dz, float* __restrict__ dh,
+                                               float* s_z, double* loss_out)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int c = warp; c < sh.classes; c += kThreads / 32) {
+        float s = 0.0f;
+        for (int j = lane; j < sh.hidden; j += 32) s = fmaf(x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], act[j], s);
+        s = warp_sum(s);
+        if (lane == 0) s_z[c] = s + x[mlp_off_b2(sh) + c];
+    }
+    __syncthreads();
+    float zmax = -INFINITY, sum = 0.0f, others = 0.0f;      // others: the sum without the label's term, so that
+    for (int c = 0; c < sh.classes; ++c) zmax = fmaxf(zmax, s_z[c]);     // p_label - 1 = -others/sum has no cancellation
+    for (int c = 0; c < sh.classes; ++c) { const float e = expf(s_z[c] - zmax); sum += e; if (c != label) others += e; }
+    if (threadIdx.x == 0 && loss_out) *loss_out = (double)(zmax + logf(sum)) - (double)s_z[label];
+    __syncthreads();
+    for (int c = threadIdx.x; c < sh.classes; c += blockDim.x) {
+        const float v = (c == label ? -others / sum : expf(s_z[c] - zmax) / sum) * wgt;
+        s_z[sh.classes + c] = v;
+        if (dz) dz[c] = v;
+    }
+    __syncthreads();
+    if (dh) {
+        for (int j = threadIdx.x; j < sh.hidden; j += blockDim.x) {
+            float s = 0.0f;
+            for (int c = 0; c < sh.classes; ++c) s = fmaf(s_z[sh.classes + c], x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], s);
+            dh[j] = act[j] > 0.0f ? s : 0.0f;
+        }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads)
+mlp_output_kernel(MlpShape sh, const float* __restrict__ labels, const int32_t* __restrict__ row_of_slot,
+                  const float* __restrict__ xa, const float* __restrict__ xb, const float* __restrict__ act_a,
+                  const float* __restrict__ act_b, float wgt, float* __restrict__ dz_a, float* __restrict__ dz_b,
+                  float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b)
+{
+    extern __shared__ float s_z[];                       // [2 * classes]
+    const int64_t slot = blockIdx.x;
+    const int label = (int)labels[row_of_slot[slot]];
+    if (xa) mlp_output_one(sh, xa, act_a + slot * sh.hidden, label, wgt, dz_a + slot * sh.classes, dh_a + slot * sh.hidden, s_z, nullptr);
+    if (xb) {
+        double loss = 0.0;
+        mlp_output_one(sh, xb, act_b + slot * sh.hidden, label, wgt, dz_b ? dz_b + slot * sh.classes : nullptr,
+                       dh_b ? dh_b + slot * sh.hidden : nullptr, s_z, loss_b ? &loss : nullptr);
+        if (loss_b && threadIdx.x == 0) atomicAdd(loss_b, loss * (double)wgt);
+    }
+}
+
+// grid (hidden + 1, groups): block (j, w) sums over the rows [w*B, (w+1)*B) of its group.  j < hidden: row j of W1 and
+// b1[j]; j == hidden: W2 and b2.  Output = model a minus model b (either may be absent).  FULL: double sums added to
+// g64 with atomics (epoch gradient over many groups); otherwise stored to out [groups][P] with the norm folded in.
+template <bool FULL>
+__global__ void __launch_bounds__(kThreads)
+mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __restrict__ row_of_slot, int B, int64_t total_rows,
+                 const float* __restrict__ act_a, const float* __restrict__ act_b, const float* __restrict__ dz_a,
+                 const float* __restrict__ dz_b, const float* __restrict__ dh_a, const float* __restrict__ dh_b,
+                 float* __restrict__ out, int64_t P, uint32_t* __restrict__ norm_bits, double* __restrict__ g64)
+{
+    typedef typename std::conditional<FULL, double, float>::type acc_t;
+    extern __shared__ float s_w[];                       // per row of the group: dh_a[j] - handled below
+    const int j = blockIdx.x, w = blockIdx.y;
+    const int64_t r0 = (int64_t)w * B;
+    const int nrows = (int)min((int64_t)B, total_rows - r0);
+    uint32_t nmax = 0;
+    float* o = FULL ? nullptr : out + (int64_t)w * P;
+    if (j < sh.hidden) {
+        // s_w[r] = dh_a[r][j], s_w[B + r] = dh_b[r][j]
+        for (int r = threadIdx.x; r < nrows; r += blockDim.x) {
+            s_w[r] = dh_a ? dh_a[(r0 + r) * sh.hidden + j] : 0.0f;
+            s_w[B + r] = dh_b ? dh_b[(r0 + r) * sh.hidden + j] : 0.0f;
+        }
+        __syncthreads();
+        for (int64_t i = threadIdx.x; i <= sh.in; i += blockDim.x) {       // i == in: the bias b1[j]
+            acc_t s = 0;
+            for (int r = 0; r < nrows; ++r) {
+                const float f = (i < sh.in) ? X[(int64_t)row_of_slot[r0 + r] * sh.in + i] : 1.0f;
+                s += (acc_t)((s_w[r] - s_w[B + r]) * f);
+            }
+            const int64_t pidx = (i < sh.in) ? (int64_t)j * sh.in + i : mlp_off_b1(sh) + j;
+            if (FULL) atomicAdd(g64 + pidx, (double)s);
+            else { o[pidx] = (float)s; nmax = max(nmax, __float_as_uint((float)s) & 0x7FFFFFFFu); }
+        }
+    } else {
+        const int nout = sh.classes * (sh.hidden + 1);                       // W2 entries then b2
+        for (int t = threadIdx.x; t < nout; t += blockDim.x) {
+            const bool bias = t >= sh.classes * sh.hidden;
+            const int c = bias ? t - sh.classes * sh.hidden : t / sh.hidden, jj = bias ? 0 : t % sh.hidden;
+            acc_t s = 0;
+            for (int r = 0; r < nrows; ++r) {
+                const int64_t q = r0 + r;
+                const float ta = dz_a ? dz_a[q * sh.classes + c] * (bias ? 1.0f : act_a[q * sh.hidden + jj]) : 0.0f;
+                const float tb = dz_b ? dz_b[q * sh.classes + c] * (bias ? 1.0f : act_b[q * sh.hidden + jj]) : 0.0f;
+                s += (acc_t)(ta - tb);
+            }
+            const int64_t pidx = bias ? mlp_off_b2(sh) + c : mlp_off_w2(sh) + (int64_t)c * sh.hidden + jj;
+            if (FULL) atomicAdd(g64 + pidx, (double)s);
+            else { o[pidx] = (float)s; nmax = max(nmax, __float_as_uint((float)s) & 0x7FFFFFFFu); }
+        }
+    }
+    if (!FULL) block_atomic_max(nmax, norm_bits + w);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Host launchers
 // ---------------------------------------------------------------------------------------------------
 static inline int blocks_for(int64_t threads_needed, int sm_count, int per_sm = 8)
@@ -494,6 +649,46 @@ static inline int blocks_for(int64_t threads_needed, int sm_count, int per_sm = 
     return (int)(need < cap ? need : cap);
 }
 
+// ---- network launchers ------------------------------------------------------------------------------------
+static MlpShape mlp_shape(const dq_ctx* ctx) { return MlpShape{ctx->data.d, ctx->cfg.hidden, ctx->cfg.classes}; }
+constexpr int kMlpGroup = 256;      // rows per block of the epoch-gradient sums
+
+// g <- (1/n) sum_i grad loss_i(x) over all rows (double sums), via the "a" slots of the activation buffers.
+static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStream_t st)
+{
+    const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
+    const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
+    const int64_t P = ctx->cfg.d;
+    mlp_hidden_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * sh.in, st>>>((const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
+                                                                             ctx->mlp_rows, ctx->mlp_act[0], nullptr);
+    mlp_output_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st>>>(sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
+        nullptr, (float)(1.0 / (double)D.n), ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr);
+    cudaMemsetAsync(ctx->g64, 0, sizeof(double) * P, st);
+    dim3 grid(sh.hidden + 1, (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
+    mlp_param_kernel<true><<<grid, kThreads, sizeof(float) * 2 * kMlpGroup, st>>>((const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
+        ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
+    finish_full_grad_kernel<<<blocks_for(P, ctx->sm_count), kThreads, 0, st>>>(ctx->g64, P, 1.0, g);
+    ctx->launches += 4;
+}
+
+// alpha_w = minibatch grad at xhat minus minibatch grad at xsnap, and ||alpha_w||_inf.
+static void launch_mlp_worker_grad(dq_ctx* ctx, const float* xhat, const dq_state* s, const BatchSource& bs, float* alpha,
+                                   float* norm_inf, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
+    const unsigned R = (unsigned)(c.M * c.B);
+    uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
+    mlp_hidden_kernel<<<R, kThreads, sizeof(float) * sh.in, st>>>((const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
+                                                                   ctx->mlp_act[0], ctx->mlp_act[1]);
+    mlp_output_kernel<<<R, kThreads, sizeof(float) * 2 * sh.classes, st>>>(sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
+        ctx->mlp_act[1], 1.0f / (float)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr);
+    if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
+    dim3 grid(sh.hidden + 1, c.M);
+    mlp_param_kernel<false><<<grid, kThreads, sizeof(float) * 2 * c.B, st>>>((const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
+        ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
+    ctx->launches += 3;
+}
+
 void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
 {
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
@@ -501,6 +696,7 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
     cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
     epoch_state_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(s->x, s->x_snap, s->y, s->x_sum, c.d, c.accelerated,
                                                                             ctx->ticks_in_epoch, theta, nx);
+    if (c.model == DQ_MODEL_MLP) { launch_mlp_full_grad(ctx, s->x_snap, s->g_full, st); ctx->launches += 1; return; }
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * c.d, st);
     if (D.format == DQ_CSR_F32) {
         full_grad_csr_kernel<<<blocks_for(D.n * 32, ctx->sm_count), kThreads, 0, st>>>(
@@ -527,6 +723,7 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
 bool worker_accumulates(const dq_ctx* ctx)
 {
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    if (c.model == DQ_MODEL_MLP) return false;
     if (D.format == DQ_CSR_F32) return !ctx->list_mode;
     const bool vec = (c.d % (D.format == DQ_DENSE_F32 ? 4 : 8)) == 0;
     if (vec && c.B >= 64) return false;                        // column sums are stored, not added
@@ -549,8 +746,12 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
                             ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr};
     if (!ctx->diff_ready) {
         DQ_DISPATCH_BITS(c.bx, (dequant_diff_kernel<BITS_><<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(
-            codes_x, delta_x, s->x_snap, c.d, ctx->xhat_diff)));
+            codes_x, delta_x, c.model == DQ_MODEL_MLP ? nullptr : s->x_snap, c.d, ctx->xhat_diff)));
         ctx->launches += 1;
+    }
+    if (c.model == DQ_MODEL_MLP) {        // xhat_diff holds xhat itself for the network (no reference subtracted)
+        launch_mlp_worker_grad(ctx, ctx->xhat_diff, s, bs, alpha, norm_inf, st);
+        return;
     }
     if (D.format == DQ_CSR_F32) {
         if (!ctx->alpha_zeroed && !list) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
@@ -600,6 +801,17 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
 {
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
     cudaMemsetAsync(P, 0, sizeof(double), st);
+    if (c.model == DQ_MODEL_MLP) {
+        const MlpShape sh = mlp_shape(ctx);
+        const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
+        mlp_hidden_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * sh.in, st>>>((const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
+                                                                                 ctx->mlp_rows, nullptr, ctx->mlp_act[1]);
+        mlp_output_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st>>>(sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
+            ctx->mlp_act[1], (float)(1.0 / (double)D.n), nullptr, nullptr, nullptr, nullptr, P);
+        objective_reg_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(x, c.d, c.lambda1, c.lambda2, P);
+        ctx->launches += 3;
+        return;
+    }
     const int grid = blocks_for(D.n * 32, ctx->sm_count);
     if (D.format == DQ_CSR_F32) objective_loss_kernel<DQ_CSR_F32><<<grid, kThreads, 0, st>>>(D, x, P);
     else if (D.format == DQ_DENSE_F32) objective_loss_kernel<DQ_DENSE_F32><<<grid, kThreads, 0, st>>>(D, x, P);

@@ -1,0 +1,86 @@
+"""GPU parity of the 3-layer network workload (Section 5.2) against the CPU oracle: epoch gradient, objective, the
+worker's gradient difference, and whole rounds in lockstep (codes bit-exact given the GPU's own gradient)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_1805_10111_b200 import synth
+from test_gpu_round import Lockstep, _close, _dev, dq  # noqa: F401  (fixture and helpers)
+
+pytestmark = pytest.mark.gpu
+F32 = np.float32
+
+
+def _net(n, n_in, hidden, classes, seed):
+    h = synth.image_classification(n, n_in, classes, 300 + seed)
+    x = synth.mlp_init(n_in, hidden, classes, 310 + seed)
+    x = (x + F32(0.05) * np.random.default_rng(seed).standard_normal(x.size).astype(F32)).astype(F32)
+    return h, x
+
+
+@pytest.mark.parametrize("n,n_in,hidden,classes", [(300, 37, 9, 4), (700, 784, 100, 10)])
+def test_network_epoch_gradient_objective_and_worker_gradient(dq, n, n_in, hidden, classes):
+    import torch
+    h, x = _net(n, n_in, hidden, classes, 1)
+    od = oracle.Dataset(h.format, h.n, h.d, h.values, h.labels)
+    P = x.size
+    M, B, bx, seed, rnd = 3, 20, 8, 33, 4
+    cfg = dq.make_config(P, M, B=B, bx=bx, seed=seed, lambda2=1e-4, model=dq.DQ_MODEL_MLP, hidden=hidden, classes=classes)
+    data = dq.Data(h)
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+    st = dq.State(x, n=h.n)
+    assert dq.dq_epoch_begin(ctx, st) == 0
+    g = oracle.mlp_grad(od, hidden, classes, x)
+    nbad, worst = _close(st.g_full.cpu().numpy(), g, rel=2e-5)
+    assert nbad == 0, (nbad, worst)
+    Pobj = torch.zeros(1, dtype=torch.float64, device="cuda")
+    assert dq.dq_objective(ctx, st.x, Pobj) == 0
+    want = oracle.mlp_objective(od, hidden, classes, x, 0.0, 1e-4)
+    assert abs(Pobj.item() - want) < 2e-6 * max(1.0, want)
+    # worker gradient difference at a quantised model
+    xq = (x + F32(0.01) * np.random.default_rng(2).standard_normal(P).astype(F32)).astype(F32)
+    cx, dx, _ = oracle.quantize(xq, bx, seed, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+    xhat = cx.astype(F32) * dx
+    alpha = torch.full((M, P), 3.0, device="cuda"); ninf = torch.zeros(M, device="cuda")
+    assert dq.dq_worker_grad(ctx, _dev(oracle.pack(cx, bx)), _dev(np.array([dx], F32)), 0, st, rnd, None, alpha, ninf) == 0
+    for w in range(M):
+        rows = oracle.sample_batch(seed, rnd, w, M, h.n, B)
+        a, S = oracle.mlp_worker_grad(od, hidden, classes, xhat, x, rows)
+        nbad, worst = _close(alpha[w].cpu().numpy(), a, S)
+        assert nbad == 0, (w, nbad, worst)
+        assert ninf[w].item() == np.abs(alpha[w].cpu().numpy()).max()
+    first = alpha.clone()
+    assert dq.dq_worker_grad(ctx, _dev(oracle.pack(cx, bx)), _dev(np.array([dx], F32)), 0, st, rnd, None, alpha, ninf) == 0
+    assert torch.equal(alpha, first)                                        # no atomics: reproducible
+    dq.dq_destroy(ctx)
+
+
+@pytest.mark.parametrize("extra", [dict(), dict(sparsify=1, phi=0.0, msg_format=1), dict(accelerated=1, box_lo=-2.0, box_hi=2.0)])
+def test_network_lockstep_rounds(dq, extra):
+    h, x = _net(400, 48, 12, 5, 2)
+    kw = dict(M=4, B=20, bx=8, b=4, lambda2=1e-4, seed=40, model=1, hidden=12, classes=5)
+    kw.update(extra)
+    ls = Lockstep(dq, h, x, **kw)
+    acc = bool(extra.get("accelerated", 0))
+    rnd = 0
+    for s_ in range(1, 3):
+        theta = F32(2.0 / (s_ + 2)) if acc else F32(0.0)
+        ls.epoch(theta)
+        for t in range(8):
+            ls.round(rnd, 0.05 if acc else 0.2, theta)
+            rnd += 1
+    assert ls.far_flips == 0
+    ls.close()
+
+
+def test_network_full_size_rounds(dq):
+    """784-100-10 on 2,000 image-shaped rows, M = 8 workers, B = 20, b_x = 8, b = 4 (the paper's setting for this model)."""
+    h, x = _net(2000, 784, 100, 10, 3)
+    kw = dict(M=8, B=20, bx=8, b=4, lambda2=1e-4, seed=41, model=1, hidden=100, classes=10)
+    ls = Lockstep(dq, h, x, **kw)
+    ls.epoch()
+    for rnd in range(6):
+        ls.round(rnd, 0.1)
+    print("\n[nn] flips %d of %d, beyond band %d, worst alpha error %.2e" % (ls.flips, ls.coords, ls.far_flips, ls.worst_alpha))
+    assert ls.far_flips == 0
+    ls.close()
