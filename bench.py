@@ -43,7 +43,7 @@ def parse_args():
     ap.add_argument("--sequential", type=int, default=0, help="1: master applies one prox step per message")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--configs", default="c1,c2,c3,c4", help="training configurations to time with dq_round ('' for none)")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_round ('' for none)")
     return ap.parse_args()
 
 
@@ -201,6 +201,7 @@ TRAIN_CONFIGS = {
     "c2": dict(gen="config2", kw=dict(M=8, B=64, bx=8, b=4, lambda2=1e-5), lr=1.0, theta=0.0, m=200),
     "c3": dict(gen="config3", kw=dict(M=16, B=128, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1),
                lr=1.0, theta=0.0, m=200),
+    "nn": dict(gen="config_nn", kw=dict(M=8, B=20, bx=8, b=4, lambda2=1e-4, model=1, hidden=100, classes=10), lr=0.1, theta=0.0, m=500),
     "c4": dict(gen="config4", kw=dict(M=32, B=256, bx=8, b=8, box_lo=-10.0, box_hi=10.0, accelerated=1), lr=1e-4,
                theta=0.1, m=200),
 }
@@ -215,10 +216,12 @@ def time_training_config(name, rounds=200, warmup=20):
     from paper_1805_10111_b200 import synth
     spec = TRAIN_CONFIGS[name]
     h = getattr(synth, spec["gen"])()
-    cfg = dq.make_config(h.d, spec["kw"]["M"], seed=1805, **{k: v for k, v in spec["kw"].items() if k != "M"})
+    is_nn = spec["kw"].get("model", 0) == 1
+    x0 = synth.mlp_init(h.d, spec["kw"]["hidden"], spec["kw"]["classes"], 9) if is_nn else np.zeros(h.d, np.float32)
+    cfg = dq.make_config(x0.size, spec["kw"]["M"], seed=1805, **{k: v for k, v in spec["kw"].items() if k != "M"})
     data = dq.Data(h)
     rc, ctx = dq.dq_create(cfg, data); dq.ok(rc, "dq_create " + name)
-    st = dq.State(np.zeros(h.d, np.float32), n=h.n, accelerated=bool(cfg.accelerated))
+    st = dq.State(x0, n=h.n, accelerated=bool(cfg.accelerated))
     theta = spec["theta"]; eta = spec["lr"] / theta if theta else spec["lr"]
     bits = torch.zeros(2, dtype=torch.int64, device="cuda")
     dq.ok(dq.dq_epoch_begin(ctx, st, theta))
@@ -233,9 +236,9 @@ def time_training_config(name, rounds=200, warmup=20):
     e1.record(); torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / rounds
     rc, status = dq.dq_poll_status(ctx)
-    out = {"rounds_per_s": round(1000.0 / ms, 1), "ms_per_round": round(ms, 4), "n": h.n, "d": h.d, "M": cfg.M, "B": cfg.B,
+    out = {"rounds_per_s": round(1000.0 / ms, 1), "ms_per_round": round(ms, 4), "n": h.n, "d": int(cfg.d), "M": cfg.M, "B": cfg.B,
            "launches_per_round": (dq.dq_launch_count(ctx) - l0) / rounds, "bits_down": int(bits[0].item()),
-           "bits_up": int(bits[1].item()), "bits_full_precision": 2 * cfg.M * 32 * h.d, "device_status": status}
+           "bits_up": int(bits[1].item()), "bits_full_precision": 2 * cfg.M * 32 * int(cfg.d), "device_status": status}
     dq.dq_destroy(ctx)
     return out
 
