@@ -5,7 +5,8 @@ Default workload ("c5"): the quantiser/packer bandwidth configuration -- M = 8 w
 d = 2^27 fp32 coordinates (N(0,1) with 0.1 % outliers x100), quantised to b = 4 bits and packed, aggregated
 and prox-updated by the master, and the new model requantised to b_x = 8 bits.  One "step" is one such
 round: ||v||_inf pass, quantise+pack, master unpack+aggregate+prox, model norm is fused, model quantise.
-Prints ONE JSON line (see README / DESIGN for the keys).
+Prints ONE JSON line: metric, value (whole-job rounds/s), per-stage times, roofline of the dominant kernel, clocks,
+end-to-end rate through host buffers, the CPU oracle's rate, and rounds/s of the training configurations.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--log2d 27] [--bits 4]
 
@@ -357,7 +358,7 @@ def run_ours(a):
             dist.destroy_process_group()
         return
     peak, peak_src = measured_peak()
-    # algorithmic bytes per launch ("bytes per unit"): norm 4 B, quantise+pack 4 + b/8 B per message
+    # algorithmic bytes per launch: norm 4 B, quantise+pack 4 + b/8 B per message
     # coordinate; master M*b/8 + 12 B, model quantise 4 + b_x/8 B per model coordinate.
     alg = [M * d * 4.0, M * d * (4.0 + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
     names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]

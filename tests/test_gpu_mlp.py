@@ -84,3 +84,30 @@ def test_network_full_size_rounds(dq):
     print("\n[nn] flips %d of %d, beyond band %d, worst alpha error %.2e" % (ls.flips, ls.coords, ls.far_flips, ls.worst_alpha))
     assert ls.far_flips == 0
     ls.close()
+
+
+def test_network_free_running_loss(dq):
+    """GPU and oracle run on their own for 60 rounds on the network; the objective agrees within 1e-4 relative."""
+    import torch
+    h, x = _net(500, 48, 12, 5, 4)
+    od = oracle.Dataset(h.format, h.n, h.d, h.values, h.labels)
+    kw = dict(B=20, bx=8, b=4, lambda2=1e-4, seed=42, model=1, hidden=12, classes=5)
+    cfg = dq.make_config(x.size, 4, **kw)
+    data = dq.Data(h)
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+    st = dq.State(x, n=h.n)
+    ocfg = oracle.make_config(x.size, 4, 20, 8, 4, l2=1e-4, seed=42, model=1, hidden=12, classes=5)
+    run = oracle.Run(ocfg, od, x)
+    P = torch.zeros(1, dtype=torch.float64, device="cuda")
+    first = last = None
+    for rnd in range(60):
+        if rnd % 20 == 0:
+            assert dq.dq_epoch_begin(ctx, st) == 0; run.epoch_begin()
+        assert dq.dq_round(ctx, st, rnd, 0.2) == 0; run.round(rnd, 0.2)
+        if rnd % 10 == 9:
+            assert dq.dq_objective(ctx, st.x, P) == 0
+            Po = oracle.mlp_objective(od, 12, 5, run.x, 0.0, 1e-4)
+            assert abs(P.item() - Po) <= 1e-4 * max(abs(Po), 1e-3), (rnd, P.item(), Po)
+            first = first if first is not None else Po; last = Po
+    assert last < first and dq.dq_poll_status(ctx) == (0, 0)
+    dq.dq_destroy(ctx)
