@@ -108,6 +108,20 @@ __device__ __forceinline__ unsigned long long l1_term(float a, int e)
     return (sh > -24) ? (unsigned long long)(mant >> (-sh)) : 0ull;
 }
 
+// The same term without integer shifts, for e >= -100 (so that 2^(23-e) is a normal fp32 number): with
+// t = |a| 2^(23-e) < 2^23, adding 2^23 toward zero leaves floor(t) in the significand, t - floor(t) is exact, and
+// the next 12 bits come out of a second add of the same kind; trunc(|a| 2^(35-e)) = 4096 floor(t) + floor(4096 frac t).
+// Every step is exact, so the two integers equal the ones l1_term produces.
+__device__ __forceinline__ void l1_term_split(float a, float scale23, uint32_t& hi, uint32_t& lo)
+{
+    const float t = __fmul_rn(fabsf(a), scale23);
+    const float m1 = __fadd_rz(t, 8388608.0f);
+    const float fr = __fsub_rn(t, __fsub_rn(m1, 8388608.0f));
+    const float m2 = __fmaf_rz(fr, 4096.0f, 8388608.0f);
+    hi += __float_as_uint(m1) & 0x007FFFFFu;
+    lo += __float_as_uint(m2) & 0x007FFFFFu;
+}
+
 __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restrict__ v, int64_t d, int vec_ok,
                                                            const uint32_t* __restrict__ norm_bits,
                                                            unsigned long long* __restrict__ l1_sum)
@@ -120,10 +134,23 @@ __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restri
     unsigned long long acc = 0;
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (int64_t)gridDim.x * blockDim.x;
     const int64_t ng = vec_ok ? (d >> 3) : 0;
-    for (int64_t g = tid; g < ng; g += nth) {
-        float a[8]; load8(row + (g << 3), a);
+    if (e >= -100) {
+        const float scale23 = __uint_as_float((uint32_t)(127 + 23 - e) << 23);     // 2^(23-e)
+        unsigned long long acc_hi = 0, acc_lo = 0;
+        for (int64_t g = tid; g < ng; g += nth) {
+            float a[8]; load8(row + (g << 3), a);
+            uint32_t hi = 0, lo = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc += l1_term(a[j], e);
+            for (int j = 0; j < 8; ++j) l1_term_split(a[j], scale23, hi, lo);
+            acc_hi += hi; acc_lo += lo;
+        }
+        acc = (acc_hi << 12) + acc_lo;
+    } else {
+        for (int64_t g = tid; g < ng; g += nth) {
+            float a[8]; load8(row + (g << 3), a);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc += l1_term(a[j], e);
+        }
     }
     for (int64_t i = (ng << 3) + tid; i < d; i += nth) acc += l1_term(__ldg(row + i), e);
 #pragma unroll
@@ -211,6 +238,218 @@ __device__ __forceinline__ uint32_t sparsify8(const float (&a)[8], float s, cons
         }
     }
     return mask;
+}
+
+// The survivor mask alone (same test as sparsify8).
+__device__ __forceinline__ uint32_t mask8(const float (&a)[8], float s, const uint32_t (&r)[4])
+{
+    uint32_t mask = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float y = __fmul_rn(__fmul_rn(fabsf(a[j]), s), 65536.0f);
+        const float uf = __fsub_rn(__uint_as_float(0x4B000000u | half16(r, j)), 8388608.0f);
+        mask |= (uint32_t)(uf < y) << j;
+    }
+    return mask;
+}
+
+// a[j] for a run-time j without moving the array to local memory.
+__device__ __forceinline__ float pick8(const float (&a)[8], int j)
+{
+    const float lo = (j & 2) ? ((j & 1) ? a[3] : a[2]) : ((j & 1) ? a[1] : a[0]);
+    const float hi = (j & 2) ? ((j & 1) ? a[7] : a[6]) : ((j & 1) ? a[5] : a[4]);
+    return (j & 4) ? hi : lo;
+}
+
+// beta_i = alpha_i / p_i of a survivor, p_i = m_i / 2^16 (see sparsify8).
+__device__ __forceinline__ float survivor_beta(float a, float s)
+{
+    const float y = __fmul_rn(__fmul_rn(fabsf(a), s), 65536.0f);
+    const float m = fminf(ceilf(y), 65536.0f);
+    return __fdiv_rn(__fmul_rn(a, 65536.0f), m);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Sparsifier mask pass over a whole vector, with staging: draw the mask, record ||beta_w||_inf, the number
+// of survivors of every chunk, and the survivors themselves.  A warp owns a chunk of kChunk coordinates;
+// it collects the chunk's (coordinate, beta) pairs in shared memory in ascending order, reserves a
+// segment of the worker's staging list with one atomic add and copies them there, so that the quantise/emit
+// step reads the few survivors instead of the whole vector again.  A chunk with more than kStash survivors,
+// or one that no longer fits the staging list, gets no segment: it sets the worker's fallback flag and is
+// redone from the vector by sparsify_emit_kernel.  Only lanes that hold a survivor do per-survivor work.
+// grid (blocks, M), blockDim = kThreads.  sb.count and sb.flags must be zero on entry.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+sparsify_stage_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
+                      const unsigned long long* __restrict__ l1_sum, float phi,
+                      const __grid_constant__ PhiloxKeys K, uint32_t round,
+                      uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
+                      int64_t nchunks, const RoundParams* __restrict__ rp, StageBufs sb, int M)
+{
+    __shared__ uint32_t s_idx[kThreads / 32][kStash];
+    __shared__ float s_val[kThreads / 32][kStash];
+    if (rp) round = rp->round;
+    const int w = blockIdx.y, lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
+    const float* row = v + (int64_t)w * d;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
+    uint32_t bmax = 0;
+    for (int64_t c = warp; c < nchunks; c += nwarps) {
+        uint32_t pos = 0;                                     // survivors of this chunk so far (same in every lane)
+        if (!sc.empty) {
+#pragma unroll 2
+            for (int it = 0; it < kChunk / 256; ++it) {
+                const int64_t g = c * (kChunk / 8) + it * 32 + lane, i0 = g << 3;
+                if (((c * (kChunk / 8) + it * 32) << 3) >= d) break;              // the whole warp is past the end
+                float a[8];
+                if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+                uint32_t r[4];
+                philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamMask, K, r);
+                const uint32_t mask = mask8(a, sc.s, r);
+                const uint32_t any = __ballot_sync(0xFFFFFFFFu, mask != 0u);
+                if (any) {
+                    const uint32_t cnt = __popc(mask);
+                    uint32_t before, total;
+                    if (__ballot_sync(0xFFFFFFFFu, cnt > 1u) == 0u) {             // at most one survivor per lane
+                        before = __popc(any & lt); total = __popc(any);
+                    } else {
+                        uint32_t incl = cnt;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+                        before = incl - cnt; total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                    }
+                    if (mask) {
+                        uint32_t p = pos + before, mm = mask;
+                        do {
+                            const int j = __ffs(mm) - 1; mm &= mm - 1u;
+                            const float beta = survivor_beta(pick8(a, j), sc.s);
+                            bmax = max(bmax, __float_as_uint(beta) & 0x7FFFFFFFu);
+                            if (p < (uint32_t)kStash) { s_idx[wib][p] = (uint32_t)(i0 + j); s_val[wib][p] = beta; }
+                            ++p;
+                        } while (mm);
+                    }
+                    pos += total;
+                }
+            }
+        }
+        __syncwarp();
+        uint32_t seg = kNoSegment;
+        if (pos > 0u) {
+            if (pos <= (uint32_t)kStash) {
+                uint32_t base = 0;
+                if (lane == 0) base = atomicAdd(sb.count + w, pos);
+                base = __shfl_sync(0xFFFFFFFFu, base, 0);
+                if ((int64_t)base + (int64_t)pos <= sb.cap) {
+                    uint32_t* di = sb.idx + (int64_t)w * sb.cap + base;
+                    float* dv = sb.val + (int64_t)w * sb.cap + base;
+                    for (uint32_t e = lane; e < pos; e += 32u) { di[e] = s_idx[wib][e]; dv[e] = s_val[wib][e]; }
+                    seg = base;
+                }
+            }
+            if (seg == kNoSegment && lane == 0) { sb.flags[w] = 1u; sb.flags[M] = 1u; }
+        }
+        if (lane == 0) {
+            if (chunk_cnt) chunk_cnt[(int64_t)w * (nchunks + 1) + c] = pos;
+            if (sb.seg) sb.seg[(int64_t)w * nchunks + c] = seg;
+        }
+        __syncwarp();                                         // the stash is reused by the next chunk
+    }
+    block_atomic_max(bmax, beta_norm_bits + w);
+}
+
+// 16-bit rounding draw of coordinate i (lane i & 7 of the Philox call of its group).
+__device__ __forceinline__ uint32_t grad_draw16(uint32_t i, uint32_t round, uint32_t worker, const PhiloxKeys& K)
+{
+    uint32_t r[4];
+    philox4x32_10(i >> 3, round, worker, kStreamGrad, K, r);
+    const uint32_t j = i & 7u;
+    const uint32_t wlo = (j & 2u) ? r[1] : r[0], whi = (j & 2u) ? r[3] : r[2];
+    const uint32_t word = (j & 4u) ? whi : wlo;
+    return (j & 1u) ? (word >> 16) : (word & 0xFFFFu);
+}
+
+// Scale of the survivors' quantiser and its reciprocal (rounded toward zero), written once per worker.
+template <int BITS>
+__device__ __forceinline__ float survivor_scale(const uint32_t* norm_bits, const uint32_t* beta_norm_bits, int w,
+                                                float* scale, int* status, bool writer)
+{
+    const uint32_t bb = beta_norm_bits[w];
+    const bool finite = bb < 0x7F800000u && norm_bits[w] < 0x7F800000u;
+    const float bnrm = __uint_as_float(bb);
+    if (writer) {
+        scale[w] = (finite && bb != 0u) ? __fdiv_rn(bnrm, (float)levels(BITS)) : 0.0f;
+        if (!finite) set_status(status, DQ_ERR_NONFINITE);
+    }
+    return (finite && bb != 0u) ? __fdiv_rd((float)levels(BITS), bnrm) : 0.0f;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Quantise the staged survivors (delta = ||beta||_inf / L, rounding draw keyed by the coordinate) and move
+// each chunk's segment to its place in the ascending (position, code) list.  Eight lanes per chunk.
+// grid (blocks, M).  The code buffer must be zero on entry.
+// ---------------------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(kThreads)
+sparsify_finish_sparse_kernel(const uint32_t* __restrict__ norm_bits, const uint32_t* __restrict__ beta_norm_bits,
+                              const __grid_constant__ PhiloxKeys K, uint32_t round, const uint32_t* __restrict__ chunk_off,
+                              int64_t nchunks, StageBufs sb, uint8_t* __restrict__ codes, int64_t stride,
+                              float* __restrict__ scale, uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status,
+                              const RoundParams* __restrict__ rp)
+{
+    if (rp) round = rp->round;
+    const int w = blockIdx.y;
+    const float inv = survivor_scale<BITS>(norm_bits, beta_norm_bits, w, scale, status, blockIdx.x == 0 && threadIdx.x == 0);
+    uint32_t* out = reinterpret_cast<uint32_t*>(codes + (int64_t)w * stride);
+    uint32_t* oidx = idx + (int64_t)w * cap;
+    const uint32_t* si = sb.idx + (int64_t)w * sb.cap;
+    const float* sv = sb.val + (int64_t)w * sb.cap;
+    const uint32_t* off = chunk_off + (int64_t)w * (nchunks + 1);
+    const int l8 = threadIdx.x & 7;
+    const int64_t sub = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3, nsub = ((int64_t)gridDim.x * blockDim.x) >> 3;
+    for (int64_t c = sub; c < nchunks; c += nsub) {
+        const uint32_t seg = sb.seg[(int64_t)w * nchunks + c];
+        if (seg == kNoSegment) continue;
+        const uint32_t first = off[c], cnt = off[c + 1] - first;
+        for (uint32_t e = l8; e < cnt; e += 8u) {
+            const int64_t p = (int64_t)first + e;
+            if (p >= cap) break;
+            const uint32_t i = si[seg + e];
+            const uint32_t s = round_fixed<BITS>(sv[seg + e], inv, grad_draw16(i, round, (uint32_t)w, K));
+            oidx[p] = i;
+            const uint32_t field = ((s >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
+            const int64_t bit = p * BITS;
+            atomicOr(out + (bit >> 5), field << (bit & 31));
+        }
+    }
+}
+
+// The same for the dense container: every staged survivor's code is OR-ed into its coordinate's field of the
+// zeroed packed message (order does not matter).  Workers whose staging is incomplete are skipped; the
+// re-reading pass writes their whole message.  grid (blocks, M).
+template <int BITS>
+__global__ void __launch_bounds__(kThreads)
+sparsify_scatter_dense_kernel(const uint32_t* __restrict__ norm_bits, const uint32_t* __restrict__ beta_norm_bits,
+                              const __grid_constant__ PhiloxKeys K, uint32_t round, StageBufs sb,
+                              uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale, int* __restrict__ status,
+                              const RoundParams* __restrict__ rp)
+{
+    if (rp) round = rp->round;
+    const int w = blockIdx.y;
+    const float inv = survivor_scale<BITS>(norm_bits, beta_norm_bits, w, scale, status, blockIdx.x == 0 && threadIdx.x == 0);
+    if (sb.flags[w]) return;
+    uint32_t* out = reinterpret_cast<uint32_t*>(codes + (int64_t)w * stride);
+    const uint32_t* si = sb.idx + (int64_t)w * sb.cap;
+    const float* sv = sb.val + (int64_t)w * sb.cap;
+    const int64_t n = sb.count[w];
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+        const uint32_t i = si[e];
+        const uint32_t s = round_fixed<BITS>(sv[e], inv, grad_draw16(i, round, (uint32_t)w, K));
+        const uint32_t field = ((s >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
+        const int64_t bit = (int64_t)i * BITS;
+        atomicOr(out + (bit >> 5), field << (bit & 31));
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -304,11 +543,15 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      int64_t nchunks, int64_t ngroups,
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
                      uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status, const RoundParams* __restrict__ rp,
-                     GroupList gl, int iters)
+                     GroupList gl, int iters,
+                     const uint32_t* __restrict__ redo_flags = nullptr /* [M + 1]: per worker, any; NULL: do everything */,
+                     const uint32_t* __restrict__ seg_tab = nullptr /* with redo_flags: only chunks without a segment */,
+                     int M = 0)
 {
+    const int w = blockIdx.y, lane = threadIdx.x & 31;
+    if (redo_flags && (redo_flags[M] == 0u || redo_flags[w] == 0u)) return;        // the staged path covered this worker
     if (rp) round = rp->round;
     const int64_t gpc = 32 * (int64_t)iters;
-    const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
     const uint32_t bb = beta_norm_bits[w];
     const bool finite = bb < 0x7F800000u && norm_bits[w] < 0x7F800000u;
@@ -326,6 +569,8 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
     const int64_t nch_eff = (SPARSE_OUT && gl.groups) ? ((int64_t)gl.count[w] + gpc - 1) / gpc : nchunks;
     for (int64_t c = warp; c < nch_eff; c += nwarps) {
         uint32_t pos = SPARSE_OUT ? chunk_off[(int64_t)w * (nchunks + 1) + c] : 0u;
+        if (SPARSE_OUT && seg_tab &&
+            (seg_tab[(int64_t)w * nchunks + c] != kNoSegment || chunk_off[(int64_t)w * (nchunks + 1) + c + 1] == pos)) continue;
         for (int it = 0; it < iters; ++it) {
             const int64_t pos_g = c * gpc + it * 32 + lane;
             const int64_t g = SPARSE_OUT ? group_at(gl, w, pos_g, d) : pos_g, i0 = g << 3;
@@ -1056,23 +1301,48 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
         norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
     }
     dim3 grid_c(list ? 64 : grid_for(nchunks * 32, ctx->sm_count), M);
-    sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
-                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks,
-                                                       ctx->rp_active, gl, iters);
-    ctx->launches += 2;
-    if (sparse_out) {
+    const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
+    if (list) {
+        sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
+                                                           ctx->beta_norm_bits, ctx->chunk_off, nchunks, ctx->rp_active, gl, iters);
         chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
         cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
             nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters)));
-        ctx->launches += 2;
+        ctx->launches += 4;
+        return;
+    }
+    // whole-vector mode: the mask pass stages the survivors; the steps after it touch the vector again only for
+    // the chunks (or workers) whose survivors did not fit the staging area
+    uint32_t* flags = ctx->stage_ctrl + M;
+    const StageBufs sb{ctx->stage_idx, ctx->stage_val, ctx->stage_ctrl, flags, sparse_out ? ctx->chunk_seg : nullptr, ctx->stage_cap};
+    cudaMemsetAsync(ctx->stage_ctrl, 0, sizeof(uint32_t) * (2 * (size_t)M + 1), st);
+    sparsify_stage_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
+                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks,
+                                                       ctx->rp_active, sb, M);
+    cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
+    ctx->launches += 2;
+    if (sparse_out) {
+        chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
+        dim3 grid_f(grid_for(nchunks * 8, ctx->sm_count), M);
+        DQ_DISPATCH_BITS(bits, (sparsify_finish_sparse_kernel<BITS_><<<grid_f, kThreads, 0, st>>>(
+            norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
+            out->idx, out->cap, ctx->status, ctx->rp_active)));
+        DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
+            v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
+            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters,
+            flags, ctx->chunk_seg, M)));
+        ctx->launches += 3;
     } else {
-        const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
+        dim3 grid_s(grid_for(ctx->stage_cap, ctx->sm_count), M);
+        DQ_DISPATCH_BITS(bits, (sparsify_scatter_dense_kernel<BITS_><<<grid_s, kThreads, 0, st>>>(
+            norm_bits, ctx->beta_norm_bits, ctx->keys, round, sb, out->codes, out->stride, out->scale, ctx->status, ctx->rp_active)));
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
-            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl, iters)));
-        ctx->launches += 1;
+            nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl, iters,
+            flags, nullptr, M)));
+        ctx->launches += 2;
     }
 }
 

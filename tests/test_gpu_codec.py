@@ -203,44 +203,76 @@ def _oracle_sparse(v, b, phi, seed, rnd):
     return out
 
 
+def _check_sparsify(dq, v, b, phi, seed, rnd):
+    """Both message formats of the sparsifier against the oracle, bit for bit, then the master step on the list."""
+    import torch
+    M, d = v.shape
+    want = _oracle_sparse(v, b, phi, seed, rnd)
+    # dense container
+    cfg = dq.make_config(d, M, b=b, seed=seed, sparsify=1, phi=phi)
+    rc, ctx = dq.dq_create(cfg); assert rc == 0
+    msgs = dq.Msgs(cfg); msgs.codes.fill_(0x77)
+    for _ in range(2):                                       # the second call meets the first call's scratch contents
+        assert dq.dq_quantize_sparsify_pack(ctx, _dev(v), None, rnd, msgs) == 0
+        assert dq.dq_poll_status(ctx) == (0, 0)
+        for w in range(M):
+            assert msgs.scale[w].item() == want[w]["delta"]
+            assert np.array_equal(msgs.codes[w].cpu().numpy(), oracle.pack(want[w]["codes"], b, msgs.stride))
+    dq.dq_destroy(ctx)
+    # (position, value) list
+    cfg = dq.make_config(d, M, b=b, seed=seed, sparsify=1, phi=phi, msg_format=dq.DQ_MSG_SPARSE)
+    rc, ctx = dq.dq_create(cfg); assert rc == 0
+    msgs = dq.Msgs(cfg); msgs.codes.fill_(0x77)
+    for _ in range(2):
+        assert dq.dq_quantize_sparsify_pack(ctx, _dev(v), None, rnd, msgs) == 0
+        assert dq.dq_poll_status(ctx) == (0, 0)
+        for w in range(M):
+            pos = np.nonzero(want[w]["Z"])[0]
+            assert msgs.nnz[w].item() == pos.size
+            assert np.array_equal(msgs.idx[w, :pos.size].cpu().numpy().astype(np.int64), pos)     # mask, ascending
+            assert msgs.scale[w].item() == want[w]["delta"]
+            assert np.array_equal(msgs.codes[w].cpu().numpy(), oracle.pack(want[w]["codes"][pos], b, msgs.stride))
+            out = torch.full((d,), 7.0, device="cuda")
+            assert dq.dq_unpack(ctx, msgs, w, out) == 0
+            assert np.array_equal(out.cpu().numpy(), want[w]["codes"].astype(F32) * want[w]["delta"])
+    # master step on the sparse messages
+    raw = np.stack([t["codes"] for t in want]); delta = np.array([t["delta"] for t in want], F32)
+    _run_master(dq, cfg, raw, delta, synth.normal_vector(d, 46), synth.normal_vector(d, 47), 0.2, msgs=msgs, ctx=ctx)
+    dq.dq_destroy(ctx)
+    return want
+
+
 @pytest.mark.parametrize("b", [2, 4, 8])
 @pytest.mark.parametrize("d,phi_frac", [(5, 0.0), (2048, 0.01), (4099, 0.0), (70001, 0.01), ((1 << 17) + 8, 0.001)])
 def test_sparsify_bit_exact_both_formats(dq, b, d, phi_frac):
     M, seed, rnd = 3, 777, 21
     v = _vectors(M, d, 5 * d + b)
     v[:, ::3] = 0                                            # exact zeros never survive
-    phi = phi_frac * d
-    want = _oracle_sparse(v, b, phi, seed, rnd)
-    # dense container
-    cfg = dq.make_config(d, M, b=b, seed=seed, sparsify=1, phi=phi)
-    rc, ctx = dq.dq_create(cfg); assert rc == 0
-    msgs = dq.Msgs(cfg); msgs.codes.fill_(0x77)
-    assert dq.dq_quantize_sparsify_pack(ctx, _dev(v), None, rnd, msgs) == 0
-    assert dq.dq_poll_status(ctx) == (0, 0)
-    for w in range(M):
-        assert msgs.scale[w].item() == want[w]["delta"]
-        assert np.array_equal(msgs.codes[w].cpu().numpy(), oracle.pack(want[w]["codes"], b, msgs.stride))
-    dq.dq_destroy(ctx)
-    # (position, value) list
-    cfg = dq.make_config(d, M, b=b, seed=seed, sparsify=1, phi=phi, msg_format=dq.DQ_MSG_SPARSE)
-    rc, ctx = dq.dq_create(cfg); assert rc == 0
-    msgs = dq.Msgs(cfg); msgs.codes.fill_(0x77)
-    assert dq.dq_quantize_sparsify_pack(ctx, _dev(v), None, rnd, msgs) == 0
-    assert dq.dq_poll_status(ctx) == (0, 0)
-    import torch
-    for w in range(M):
-        pos = np.nonzero(want[w]["Z"])[0]
-        assert msgs.nnz[w].item() == pos.size
-        assert np.array_equal(msgs.idx[w, :pos.size].cpu().numpy().astype(np.int64), pos)     # mask, ascending
-        assert msgs.scale[w].item() == want[w]["delta"]
-        assert np.array_equal(msgs.codes[w].cpu().numpy(), oracle.pack(want[w]["codes"][pos], b, msgs.stride))
-        out = torch.full((d,), 7.0, device="cuda")
-        assert dq.dq_unpack(ctx, msgs, w, out) == 0
-        assert np.array_equal(out.cpu().numpy(), want[w]["codes"].astype(F32) * want[w]["delta"])
-    # master step on the sparse messages
-    raw = np.stack([t["codes"] for t in want]); delta = np.array([t["delta"] for t in want], F32)
-    _run_master(dq, cfg, raw, delta, synth.normal_vector(d, 46), synth.normal_vector(d, 47), 0.2, msgs=msgs, ctx=ctx)
-    dq.dq_destroy(ctx)
+    _check_sparsify(dq, v, b, phi_frac * d, seed, rnd)
+
+
+@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("kind", ["dense", "near_limit", "half_empty"])
+def test_sparsify_beyond_the_staging_limits(dq, b, kind):
+    """Densities at which the survivors of a chunk (or of a whole vector) no longer fit the staging area, so that
+    the chunk or the worker is redone from the vector: every chunk ("dense", about 20 % survive), a mixture of
+    chunks on both sides of the limit ("near_limit", 6 % of +-1 entries), and the same behind an all-zero half."""
+    M, seed, rnd = 3, 4242, 5
+    d = (1 << 16) + 2048 + 8
+    g = np.random.default_rng(600 + b)
+    if kind == "dense":
+        v = _vectors(M, d, 31 + b, outliers=False); phi = 0.0
+    else:
+        v = np.where(g.random((M, d)) < 0.5, F32(-1), F32(1)).astype(F32)
+        phi = 0.06 * d
+        if kind == "half_empty":
+            v[:, : d // 2] = 0; phi = 0.03 * d
+    want = _check_sparsify(dq, v, b, phi, seed, rnd)
+    per_chunk = [np.add.reduceat(t["Z"].astype(np.int64), np.arange(0, d, 2048)) for t in want]
+    if kind == "dense":
+        assert min(c[:-1].min() for c in per_chunk) > 128
+    else:
+        assert any((c > 128).any() for c in per_chunk) and any(((c > 0) & (c <= 128)).any() for c in per_chunk)
 
 
 def test_sparse_capacity_overflow_is_reported(dq):
