@@ -117,13 +117,11 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     const int64_t chunk_slots = (d + 255) / 256 + 1;
     rc |= dev_alloc(&c->chunk_off, cfg->sparsify ? (size_t)M * chunk_slots : 1);
     rc |= dev_alloc(&c->tile_ptr, sparse ? (size_t)M * (c->nchunks + 1) : 1);
-    // staging area for the survivors of the mask pass: room for a density of 1/16, beyond which the
-    // sparsifier falls back to re-reading the vector
-    c->stage_cap = cfg->sparsify ? (d / 16 > 4096 ? d / 16 : (d < 4096 ? d : 4096)) : 0;
-    rc |= dev_alloc(&c->stage_idx, cfg->sparsify ? (size_t)M * c->stage_cap : 1);
-    rc |= dev_alloc(&c->stage_val, cfg->sparsify ? (size_t)M * c->stage_cap : 1);
-    rc |= dev_alloc(&c->stage_ctrl, (size_t)2 * M + 1);
-    rc |= dev_alloc(&c->chunk_seg, cfg->sparsify ? (size_t)M * c->nchunks : 1);
+    // staging area for the survivors of the mask pass: kStash entries per chunk, i.e. room for a density of 1/16,
+    // beyond which the sparsifier falls back to re-reading the vector
+    rc |= dev_alloc(&c->stage_idx, cfg->sparsify ? (size_t)M * c->nchunks * kStash : 1);
+    rc |= dev_alloc(&c->stage_val, cfg->sparsify ? (size_t)M * c->nchunks * kStash : 1);
+    rc |= dev_alloc(&c->stage_ctrl, (size_t)M + 1);
     rc |= dev_alloc(&c->xnorm_bits, 1);
     rc |= dev_alloc(&c->status, 1);
     rc |= dev_alloc(&c->bits, 2);
@@ -179,7 +177,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
 int dq_destroy(dq_ctx* c)
 {
     if (!c) return DQ_ERR_ARG;
-    void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->chunk_seg, c->xnorm_bits, c->status, c->bits,
+    void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
                     c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);

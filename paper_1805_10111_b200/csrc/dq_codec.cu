@@ -240,15 +240,19 @@ __device__ __forceinline__ uint32_t sparsify8(const float (&a)[8], float s, cons
     return mask;
 }
 
-// The survivor mask alone (same test as sparsify8).
+// The survivor mask without float compares or selects.  u < y for an integer draw u is u < ceil(y); adding 2^23 to
+// y with rounding toward +inf leaves ceil(y) in the significand (y <= 2^16 (1 + ulp) because phi is clamped to
+// |alpha|_1 / |alpha|_inf), the draw is placed under the same exponent with one logic operation, and the sign of
+// the difference of the two words is shifted into the mask.  Same mask as sparsify8.
 __device__ __forceinline__ uint32_t mask8(const float (&a)[8], float s, const uint32_t (&r)[4])
 {
     uint32_t mask = 0;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
+    for (int j = 7; j >= 0; --j) {
         const float y = __fmul_rn(__fmul_rn(fabsf(a[j]), s), 65536.0f);
-        const float uf = __fsub_rn(__uint_as_float(0x4B000000u | half16(r, j)), 8388608.0f);
-        mask |= (uint32_t)(uf < y) << j;
+        const uint32_t thr = __float_as_uint(__fadd_ru(y, 8388608.0f));
+        const uint32_t draw = (j & 1) ? __byte_perm(r[j >> 1], 0x4B000000u, 0x7632) : ((r[j >> 1] & 0xFFFFu) | 0x4B000000u);
+        mask = __funnelshift_l(draw - thr, mask, 1);          // (mask << 1) | (draw < thr)
     }
     return mask;
 }
@@ -271,90 +275,95 @@ __device__ __forceinline__ float survivor_beta(float a, float s)
 
 // ---------------------------------------------------------------------------------------------------
 // Sparsifier mask pass over a whole vector, with staging: draw the mask, record ||beta_w||_inf, the number
-// of survivors of every chunk, and the survivors themselves.  A warp owns a chunk of kChunk coordinates;
-// it collects the chunk's (coordinate, beta) pairs in shared memory in ascending order, reserves a
-// segment of the worker's staging list with one atomic add and copies them there, so that the quantise/emit
-// step reads the few survivors instead of the whole vector again.  A chunk with more than kStash survivors,
-// or one that no longer fits the staging list, gets no segment: it sets the worker's fallback flag and is
-// redone from the vector by sparsify_emit_kernel.  Only lanes that hold a survivor do per-survivor work.
-// grid (blocks, M), blockDim = kThreads.  sb.count and sb.flags must be zero on entry.
+// of survivors of every chunk, and the survivors themselves.  A warp owns a chunk of kChunk coordinates
+// and writes the chunk's (coordinate, beta) pairs, in ascending order, into the chunk's own slot of kStash
+// entries of the staging area, so that the quantise/emit step reads the few survivors instead of the whole
+// vector again.  A chunk with more than kStash survivors keeps only its count: it sets the worker's fallback
+// flag and is redone from the vector by sparsify_emit_kernel.  Only lanes that hold a survivor do
+// per-survivor work.  grid (blocks, M), blockDim = kThreads.  sb.flags must be zero on entry.
 // ---------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 3)
 sparsify_stage_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const uint32_t* __restrict__ norm_bits,
                       const unsigned long long* __restrict__ l1_sum, float phi,
                       const __grid_constant__ PhiloxKeys K, uint32_t round,
-                      uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
+                      uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt,
                       int64_t nchunks, const RoundParams* __restrict__ rp, StageBufs sb, int M)
 {
-    __shared__ uint32_t s_idx[kThreads / 32][kStash];
-    __shared__ float s_val[kThreads / 32][kStash];
     if (rp) round = rp->round;
-    const int w = blockIdx.y, lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
     const float* row = v + (int64_t)w * d;
     const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t lt = (1u << lane) - 1u;
     uint32_t bmax = 0;
-    for (int64_t c = warp; c < nchunks; c += nwarps) {
-        uint32_t pos = 0;                                     // survivors of this chunk so far (same in every lane)
-        if (!sc.empty) {
-#pragma unroll 2
-            for (int it = 0; it < kChunk / 256; ++it) {
-                const int64_t g = c * (kChunk / 8) + it * 32 + lane, i0 = g << 3;
-                if (((c * (kChunk / 8) + it * 32) << 3) >= d) break;              // the whole warp is past the end
-                float a[8];
-                if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
-                uint32_t r[4];
-                philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamMask, K, r);
-                const uint32_t mask = mask8(a, sc.s, r);
-                const uint32_t any = __ballot_sync(0xFFFFFFFFu, mask != 0u);
-                if (any) {
-                    const uint32_t cnt = __popc(mask);
-                    uint32_t before, total;
-                    if (__ballot_sync(0xFFFFFFFFu, cnt > 1u) == 0u) {             // at most one survivor per lane
-                        before = __popc(any & lt); total = __popc(any);
-                    } else {
-                        uint32_t incl = cnt;
+    uint32_t pos = 0;                                         // survivors of the current chunk so far (same in every lane)
+    uint32_t* di = nullptr; float* dv = nullptr;
+    // survivors of one step (32 groups of eight coordinates, one per lane): positions in index order, then beta
+    auto collect = [&](const float (&a)[8], uint32_t mask, uint32_t any, uint32_t g) {
+        const uint32_t cnt = __popc(mask);
+        uint32_t before, total;
+        if (__ballot_sync(0xFFFFFFFFu, cnt > 1u) == 0u) {                         // at most one survivor per lane
+            before = __popc(any & lt); total = __popc(any);
+        } else {
+            uint32_t incl = cnt;
 #pragma unroll
-                        for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
-                        before = incl - cnt; total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                    }
-                    if (mask) {
-                        uint32_t p = pos + before, mm = mask;
-                        do {
-                            const int j = __ffs(mm) - 1; mm &= mm - 1u;
-                            const float beta = survivor_beta(pick8(a, j), sc.s);
-                            bmax = max(bmax, __float_as_uint(beta) & 0x7FFFFFFFu);
-                            if (p < (uint32_t)kStash) { s_idx[wib][p] = (uint32_t)(i0 + j); s_val[wib][p] = beta; }
-                            ++p;
-                        } while (mm);
-                    }
-                    pos += total;
-                }
-            }
+            for (int o = 1; o < 32; o <<= 1) { uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+            before = incl - cnt; total = __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
-        __syncwarp();
-        uint32_t seg = kNoSegment;
-        if (pos > 0u) {
-            if (pos <= (uint32_t)kStash) {
-                uint32_t base = 0;
-                if (lane == 0) base = atomicAdd(sb.count + w, pos);
-                base = __shfl_sync(0xFFFFFFFFu, base, 0);
-                if ((int64_t)base + (int64_t)pos <= sb.cap) {
-                    uint32_t* di = sb.idx + (int64_t)w * sb.cap + base;
-                    float* dv = sb.val + (int64_t)w * sb.cap + base;
-                    for (uint32_t e = lane; e < pos; e += 32u) { di[e] = s_idx[wib][e]; dv[e] = s_val[wib][e]; }
-                    seg = base;
+        if (mask) {
+            uint32_t p = pos + before, mm = mask;
+            do {
+                const int j = __ffs(mm) - 1; mm &= mm - 1u;
+                const float beta = survivor_beta(pick8(a, j), sc.s);
+                bmax = max(bmax, __float_as_uint(beta) & 0x7FFFFFFFu);
+                if (p < (uint32_t)kStash) { di[p] = (g << 3) + (uint32_t)j; dv[p] = beta; }
+                ++p;
+            } while (mm);
+        }
+        pos += total;
+    };
+    // Two steps are drawn together so that their generator chains interleave.  The kernel is bound by the number
+    // of instructions it issues, so a chunk that lies wholly inside an aligned row takes a loop without bounds
+    // checks or 64-bit index arithmetic.
+    auto two_steps = [&](const float (&a)[8], const float (&b)[8], uint32_t g) {
+        uint32_t ra[4], rb[4];
+        philox4x32_10(g, round, (uint32_t)w, kStreamMask, K, ra);
+        philox4x32_10(g + 32u, round, (uint32_t)w, kStreamMask, K, rb);
+        const uint32_t ma = mask8(a, sc.s, ra), mb = mask8(b, sc.s, rb);
+        const uint32_t anya = __ballot_sync(0xFFFFFFFFu, ma != 0u), anyb = __ballot_sync(0xFFFFFFFFu, mb != 0u);
+        if (anya) collect(a, ma, anya, g);
+        if (anyb) collect(b, mb, anyb, g + 32u);
+    };
+    for (int64_t c = warp; c < nchunks; c += nwarps) {
+        pos = 0;
+        di = sb.idx + ((int64_t)w * nchunks + c) * kStash;
+        dv = sb.val + ((int64_t)w * nchunks + c) * kStash;
+        if (!sc.empty) {
+            const uint32_t g0 = (uint32_t)(c * (kChunk / 8)) + (uint32_t)lane;     // d <= 2^32: group numbers fit 32 bits
+            float bufa[8], bufb[8];
+            if (vec_ok && (c + 1) * kChunk <= d) {
+                const float* p = row + c * kChunk + lane * 8;
+#pragma unroll 1
+                for (int it = 0; it < kChunk / 256; it += 2) {
+                    load8(p, bufa); load8(p + 256, bufb);
+                    two_steps(bufa, bufb, g0 + (uint32_t)it * 32u);
+                    p += 512;
+                }
+            } else {
+#pragma unroll 1
+                for (int it = 0; it < kChunk / 256; it += 2) {
+                    const uint32_t g = g0 + (uint32_t)it * 32u;
+                    load8_guarded(row, (int64_t)g << 3, d, bufa);
+                    load8_guarded(row, ((int64_t)g + 32) << 3, d, bufb);
+                    two_steps(bufa, bufb, g);
                 }
             }
-            if (seg == kNoSegment && lane == 0) { sb.flags[w] = 1u; sb.flags[M] = 1u; }
         }
         if (lane == 0) {
-            if (chunk_cnt) chunk_cnt[(int64_t)w * (nchunks + 1) + c] = pos;
-            if (sb.seg) sb.seg[(int64_t)w * nchunks + c] = seg;
+            chunk_cnt[(int64_t)w * (nchunks + 1) + c] = pos;
+            if (pos > (uint32_t)kStash) { sb.flags[w] = 1u; sb.flags[M] = 1u; }
         }
-        __syncwarp();                                         // the stash is reused by the next chunk
     }
     block_atomic_max(bmax, beta_norm_bits + w);
 }
@@ -403,20 +412,19 @@ sparsify_finish_sparse_kernel(const uint32_t* __restrict__ norm_bits, const uint
     const float inv = survivor_scale<BITS>(norm_bits, beta_norm_bits, w, scale, status, blockIdx.x == 0 && threadIdx.x == 0);
     uint32_t* out = reinterpret_cast<uint32_t*>(codes + (int64_t)w * stride);
     uint32_t* oidx = idx + (int64_t)w * cap;
-    const uint32_t* si = sb.idx + (int64_t)w * sb.cap;
-    const float* sv = sb.val + (int64_t)w * sb.cap;
     const uint32_t* off = chunk_off + (int64_t)w * (nchunks + 1);
     const int l8 = threadIdx.x & 7;
     const int64_t sub = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3, nsub = ((int64_t)gridDim.x * blockDim.x) >> 3;
     for (int64_t c = sub; c < nchunks; c += nsub) {
-        const uint32_t seg = sb.seg[(int64_t)w * nchunks + c];
-        if (seg == kNoSegment) continue;
         const uint32_t first = off[c], cnt = off[c + 1] - first;
+        if (cnt > (uint32_t)kStash) continue;                                      // left to the re-reading pass
+        const uint32_t* si = sb.idx + ((int64_t)w * nchunks + c) * kStash;
+        const float* sv = sb.val + ((int64_t)w * nchunks + c) * kStash;
         for (uint32_t e = l8; e < cnt; e += 8u) {
             const int64_t p = (int64_t)first + e;
             if (p >= cap) break;
-            const uint32_t i = si[seg + e];
-            const uint32_t s = round_fixed<BITS>(sv[seg + e], inv, grad_draw16(i, round, (uint32_t)w, K));
+            const uint32_t i = si[e];
+            const uint32_t s = round_fixed<BITS>(sv[e], inv, grad_draw16(i, round, (uint32_t)w, K));
             oidx[p] = i;
             const uint32_t field = ((s >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
             const int64_t bit = p * BITS;
@@ -426,29 +434,34 @@ sparsify_finish_sparse_kernel(const uint32_t* __restrict__ norm_bits, const uint
 }
 
 // The same for the dense container: every staged survivor's code is OR-ed into its coordinate's field of the
-// zeroed packed message (order does not matter).  Workers whose staging is incomplete are skipped; the
-// re-reading pass writes their whole message.  grid (blocks, M).
+// zeroed packed message.  Workers with a chunk beyond the staging limit are skipped; the re-reading pass writes
+// their whole message.  chunk_cnt holds the chunks' counts (no prefix).  grid (blocks, M).
 template <int BITS>
 __global__ void __launch_bounds__(kThreads)
 sparsify_scatter_dense_kernel(const uint32_t* __restrict__ norm_bits, const uint32_t* __restrict__ beta_norm_bits,
-                              const __grid_constant__ PhiloxKeys K, uint32_t round, StageBufs sb,
-                              uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale, int* __restrict__ status,
-                              const RoundParams* __restrict__ rp)
+                              const __grid_constant__ PhiloxKeys K, uint32_t round, const uint32_t* __restrict__ chunk_cnt,
+                              int64_t nchunks, StageBufs sb, uint8_t* __restrict__ codes, int64_t stride,
+                              float* __restrict__ scale, int* __restrict__ status, const RoundParams* __restrict__ rp)
 {
     if (rp) round = rp->round;
     const int w = blockIdx.y;
     const float inv = survivor_scale<BITS>(norm_bits, beta_norm_bits, w, scale, status, blockIdx.x == 0 && threadIdx.x == 0);
     if (sb.flags[w]) return;
     uint32_t* out = reinterpret_cast<uint32_t*>(codes + (int64_t)w * stride);
-    const uint32_t* si = sb.idx + (int64_t)w * sb.cap;
-    const float* sv = sb.val + (int64_t)w * sb.cap;
-    const int64_t n = sb.count[w];
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
-        const uint32_t i = si[e];
-        const uint32_t s = round_fixed<BITS>(sv[e], inv, grad_draw16(i, round, (uint32_t)w, K));
-        const uint32_t field = ((s >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
-        const int64_t bit = (int64_t)i * BITS;
-        atomicOr(out + (bit >> 5), field << (bit & 31));
+    const uint32_t* cnts = chunk_cnt + (int64_t)w * (nchunks + 1);
+    const int l8 = threadIdx.x & 7;
+    const int64_t sub = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3, nsub = ((int64_t)gridDim.x * blockDim.x) >> 3;
+    for (int64_t c = sub; c < nchunks; c += nsub) {
+        const uint32_t cnt = cnts[c];
+        const uint32_t* si = sb.idx + ((int64_t)w * nchunks + c) * kStash;
+        const float* sv = sb.val + ((int64_t)w * nchunks + c) * kStash;
+        for (uint32_t e = l8; e < cnt; e += 8u) {
+            const uint32_t i = si[e];
+            const uint32_t s = round_fixed<BITS>(sv[e], inv, grad_draw16(i, round, (uint32_t)w, K));
+            const uint32_t field = ((s >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
+            const int64_t bit = (int64_t)i * BITS;
+            atomicOr(out + (bit >> 5), field << (bit & 31));
+        }
     }
 }
 
@@ -544,8 +557,8 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
                      uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status, const RoundParams* __restrict__ rp,
                      GroupList gl, int iters,
-                     const uint32_t* __restrict__ redo_flags = nullptr /* [M + 1]: per worker, any; NULL: do everything */,
-                     const uint32_t* __restrict__ seg_tab = nullptr /* with redo_flags: only chunks without a segment */,
+                     const uint32_t* __restrict__ redo_flags = nullptr /* [M + 1]: per worker, any; NULL: do everything.
+                        With sparse output only the chunks with more than kStash survivors are redone. */,
                      int M = 0)
 {
     const int w = blockIdx.y, lane = threadIdx.x & 31;
@@ -569,8 +582,7 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
     const int64_t nch_eff = (SPARSE_OUT && gl.groups) ? ((int64_t)gl.count[w] + gpc - 1) / gpc : nchunks;
     for (int64_t c = warp; c < nch_eff; c += nwarps) {
         uint32_t pos = SPARSE_OUT ? chunk_off[(int64_t)w * (nchunks + 1) + c] : 0u;
-        if (SPARSE_OUT && seg_tab &&
-            (seg_tab[(int64_t)w * nchunks + c] != kNoSegment || chunk_off[(int64_t)w * (nchunks + 1) + c + 1] == pos)) continue;
+        if (SPARSE_OUT && redo_flags && chunk_off[(int64_t)w * (nchunks + 1) + c + 1] - pos <= (uint32_t)kStash) continue;
         for (int it = 0; it < iters; ++it) {
             const int64_t pos_g = c * gpc + it * 32 + lane;
             const int64_t g = SPARSE_OUT ? group_at(gl, w, pos_g, d) : pos_g, i0 = g << 3;
@@ -1315,33 +1327,32 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     }
     // whole-vector mode: the mask pass stages the survivors; the steps after it touch the vector again only for
     // the chunks (or workers) whose survivors did not fit the staging area
-    uint32_t* flags = ctx->stage_ctrl + M;
-    const StageBufs sb{ctx->stage_idx, ctx->stage_val, ctx->stage_ctrl, flags, sparse_out ? ctx->chunk_seg : nullptr, ctx->stage_cap};
-    cudaMemsetAsync(ctx->stage_ctrl, 0, sizeof(uint32_t) * (2 * (size_t)M + 1), st);
+    uint32_t* flags = ctx->stage_ctrl;
+    const StageBufs sb{ctx->stage_idx, ctx->stage_val, flags};
+    cudaMemsetAsync(flags, 0, sizeof(uint32_t) * ((size_t)M + 1), st);
     sparsify_stage_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
-                                                       ctx->beta_norm_bits, sparse_out ? ctx->chunk_off : nullptr, nchunks,
-                                                       ctx->rp_active, sb, M);
+                                                       ctx->beta_norm_bits, ctx->chunk_off, nchunks, ctx->rp_active, sb, M);
     cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
     ctx->launches += 2;
+    dim3 grid_f(grid_for(nchunks * 8, ctx->sm_count), M);
     if (sparse_out) {
         chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
-        dim3 grid_f(grid_for(nchunks * 8, ctx->sm_count), M);
         DQ_DISPATCH_BITS(bits, (sparsify_finish_sparse_kernel<BITS_><<<grid_f, kThreads, 0, st>>>(
             norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
             out->idx, out->cap, ctx->status, ctx->rp_active)));
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
             nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters,
-            flags, ctx->chunk_seg, M)));
+            flags, M)));
         ctx->launches += 3;
     } else {
-        dim3 grid_s(grid_for(ctx->stage_cap, ctx->sm_count), M);
-        DQ_DISPATCH_BITS(bits, (sparsify_scatter_dense_kernel<BITS_><<<grid_s, kThreads, 0, st>>>(
-            norm_bits, ctx->beta_norm_bits, ctx->keys, round, sb, out->codes, out->stride, out->scale, ctx->status, ctx->rp_active)));
+        DQ_DISPATCH_BITS(bits, (sparsify_scatter_dense_kernel<BITS_><<<grid_f, kThreads, 0, st>>>(
+            norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
+            ctx->status, ctx->rp_active)));
         DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
             v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
             nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl, iters,
-            flags, nullptr, M)));
+            flags, M)));
         ctx->launches += 2;
     }
 }

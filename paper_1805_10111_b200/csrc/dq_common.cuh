@@ -11,11 +11,11 @@ constexpr uint32_t kMaster = 0xFFFFFFFFu;
 enum : uint32_t { kStreamModel = 0, kStreamGrad = 1, kStreamMask = 2, kStreamBatch = 3 };
 constexpr int kThreads = 256;
 constexpr int kChunk = 2048;   // coordinates one warp owns per step of the sparsifier (32 lanes x 8 x 8)
-constexpr int kStash = 128;    // survivors of one chunk that a warp can hold in shared memory before staging them
-constexpr uint32_t kNoSegment = 0xFFFFFFFFu;   // chunk without a staged segment (empty, or left to the re-reading pass)
+constexpr int kStash = 128;    // staged survivors per chunk (a density of 1/16); fuller chunks are redone from the vector
 
-// Staging area of the sparsifier (see sparsify_stage_kernel).
-struct StageBufs { uint32_t* idx; float* val; uint32_t* count; uint32_t* flags; uint32_t* seg; int64_t cap; };
+// Staging area of the sparsifier (see sparsify_stage_kernel): slot c of worker w starts at entry
+// (w * nchunks + c) * kStash; flags [M + 1] = some chunk of worker w (entry M: of any worker) exceeded its slot.
+struct StageBufs { uint32_t* idx; float* val; uint32_t* flags; };
 
 // The ten round keys of Philox4x32-10 depend on the seed only; the host expands them once so that the
 // kernels read them from the constant bank.
@@ -204,11 +204,9 @@ struct dq_ctx {
     uint32_t* chunk_off;        // [M][nchunks + 1] survivors per chunk, then their exclusive prefix
     uint32_t* tile_ptr;         // [M][nchunks + 1] first list entry of each coordinate tile (sparse master)
     // survivors staged by the sparsifier's mask pass, so that no later pass re-reads the vector
-    uint32_t* stage_idx;        // [M][stage_cap] coordinate of each staged survivor (ascending inside a chunk's segment)
-    float* stage_val;           // [M][stage_cap] its rescaled value beta_i
-    uint32_t* stage_ctrl;       // [M] entries reserved per worker, then [M + 1] fallback flags (per worker, any)
-    uint32_t* chunk_seg;        // [M][nchunks] first staged entry of each chunk, or kNoSegment
-    int64_t stage_cap;
+    uint32_t* stage_idx;        // [M][nchunks][kStash] coordinates of the staged survivors of each chunk, ascending
+    float* stage_val;           // [M][nchunks][kStash] their rescaled values beta_i
+    uint32_t* stage_ctrl;       // [M + 1] fallback flags (per worker, any)
     uint32_t* xnorm_bits;       // [1]   ||x||_inf when the caller supplies none
     int* status;                // sticky device status word
     int64_t nchunks;
