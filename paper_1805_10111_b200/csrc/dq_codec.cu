@@ -15,6 +15,7 @@ namespace dq {
 __global__ void __launch_bounds__(kThreads) norm_inf_kernel(const float* __restrict__ v, int64_t d, int vec_ok,
                                                             uint32_t* __restrict__ norm_bits)
 {
+    pdl_prologue();
     const float* row = v + (int64_t)blockIdx.y * d;
     uint32_t m = 0;
     const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (int64_t)gridDim.x * blockDim.x;
@@ -48,6 +49,7 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      float* __restrict__ zero_f = nullptr, int64_t zero_n = 0, uint32_t* __restrict__ zero_u = nullptr, int zero_un = 0,
                      const int32_t* __restrict__ bits_gate = nullptr /* run only if *bits_gate == BITS */)
 {
+    pdl_prologue();
     if (bits_gate && *bits_gate != BITS) return;
     if (rp) round = rp->round;
     if (DIFF) {   // also clears the buffers that the next stages of the round accumulate into
@@ -126,6 +128,7 @@ __global__ void __launch_bounds__(kThreads) norm_l1_kernel(const float* __restri
                                                            const uint32_t* __restrict__ norm_bits,
                                                            unsigned long long* __restrict__ l1_sum)
 {
+    pdl_prologue();
     const int w = blockIdx.y;
     const uint32_t nb = norm_bits[w];
     if (nb == 0u || nb >= 0x7F800000u) return;
@@ -170,6 +173,7 @@ __global__ void __launch_bounds__(kThreads) norm_l1_list_kernel(const float* __r
                                                                 const uint32_t* __restrict__ norm_bits,
                                                                 unsigned long long* __restrict__ l1_sum)
 {
+    pdl_prologue();
     const int w = blockIdx.y;
     const uint32_t nb = norm_bits[w];
     if (nb == 0u || nb >= 0x7F800000u) return;
@@ -289,6 +293,7 @@ sparsify_stage_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
                       uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt,
                       int64_t nchunks, const RoundParams* __restrict__ rp, StageBufs sb, int M)
 {
+    pdl_prologue();
     if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
@@ -407,6 +412,7 @@ sparsify_finish_sparse_kernel(const uint32_t* __restrict__ norm_bits, const uint
                               float* __restrict__ scale, uint32_t* __restrict__ idx, int64_t cap, int* __restrict__ status,
                               const RoundParams* __restrict__ rp)
 {
+    pdl_prologue();
     if (rp) round = rp->round;
     const int w = blockIdx.y;
     const float inv = survivor_scale<BITS>(norm_bits, beta_norm_bits, w, scale, status, blockIdx.x == 0 && threadIdx.x == 0);
@@ -443,6 +449,7 @@ sparsify_scatter_dense_kernel(const uint32_t* __restrict__ norm_bits, const uint
                               int64_t nchunks, StageBufs sb, uint8_t* __restrict__ codes, int64_t stride,
                               float* __restrict__ scale, int* __restrict__ status, const RoundParams* __restrict__ rp)
 {
+    pdl_prologue();
     if (rp) round = rp->round;
     const int w = blockIdx.y;
     const float inv = survivor_scale<BITS>(norm_bits, beta_norm_bits, w, scale, status, blockIdx.x == 0 && threadIdx.x == 0);
@@ -477,6 +484,7 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
                       uint32_t* __restrict__ beta_norm_bits, uint32_t* __restrict__ chunk_cnt /* may be NULL */,
                       int64_t nchunks, const RoundParams* __restrict__ rp, GroupList gl, int iters /* warp steps per chunk */)
 {
+    pdl_prologue();
     if (rp) round = rp->round;
     const int w = blockIdx.y, lane = threadIdx.x & 31;
     const SparsifyScale sc = sparsify_scale(norm_bits[w], l1_sum[w], phi);
@@ -519,6 +527,7 @@ __global__ void __launch_bounds__(kThreads)
 chunk_scan_kernel(uint32_t* __restrict__ chunk_off, int64_t nchunks, int64_t cap, uint32_t* __restrict__ nnz,
                   int* __restrict__ status)
 {
+    pdl_prologue();
     uint32_t* off = chunk_off + (int64_t)blockIdx.x * (nchunks + 1);
     __shared__ uint32_t s_warp[kThreads / 32];
     // each thread owns a contiguous run of entries: local sum, one block-wide scan of the sums, local prefix
@@ -637,6 +646,7 @@ __global__ void __launch_bounds__(kThreads)
 tile_ptr_kernel(const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* __restrict__ nnz, int64_t ntiles,
                 uint32_t* __restrict__ tile_ptr)
 {
+    pdl_prologue();
     const int w = blockIdx.y;
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t > ntiles) return;
@@ -710,6 +720,7 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
                     int vec8_ok, uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
 {
+    pdl_prologue();
     if (rp) { eta = rp->eta; theta = rp->theta; }
     if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     constexpr int W = (BITS == 8) ? 2 : 1;                  // code words per worker and thread
@@ -844,6 +855,7 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
                      const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
                      uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
 {
+    pdl_prologue();
     if (rp) { eta = rp->eta; theta = rp->theta; }
     if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     __shared__ float s_acc[kChunk];
@@ -924,6 +936,7 @@ master_dense_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, const
                         const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
                         uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
 {
+    pdl_prologue();
     if (rp) { eta = rp->eta; theta = rp->theta; }
     if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     constexpr int C = 32 / BITS;
@@ -1005,6 +1018,7 @@ master_sparse_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, cons
                          const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
                          uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
 {
+    pdl_prologue();
     if (rp) { eta = rp->eta; theta = rp->theta; }
     if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
     constexpr int R = kChunk / kThreads;                       // coordinates of the tile per thread
@@ -1069,6 +1083,7 @@ template <int BITS>
 __global__ void unpack_dense_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scale, int64_t d,
                                     float* __restrict__ out)
 {
+    pdl_prologue();
     const float dl = scale[0];
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t bit = i * BITS;
@@ -1081,6 +1096,7 @@ __global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const fl
                                      const uint32_t* __restrict__ idx, const uint32_t* __restrict__ nnz,
                                      float* __restrict__ out)
 {
+    pdl_prologue();
     const float dl = scale[0];
     const uint32_t n = nnz[0];
     for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
@@ -1097,6 +1113,7 @@ __global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const fl
 __global__ void __launch_bounds__(kThreads)
 count_touched_kernel(const uint32_t* __restrict__ touched, int64_t bm_words, uint32_t* __restrict__ seg_count, int nseg)
 {
+    pdl_prologue();
     // grid (nseg, M): set bits of one segment of kThreads bitmap words
     const int w = blockIdx.y;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -1117,6 +1134,7 @@ build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const 
                         const float* __restrict__ alpha, int64_t d, int vec_ok,
                         uint32_t* __restrict__ glist, int64_t cap, uint32_t* __restrict__ gcount, uint32_t* __restrict__ norm_bits)
 {
+    pdl_prologue();
     // grid (nseg, M): this segment's groups go to the list after those of the segments before it
     const int w = blockIdx.y;
     uint32_t* bm = touched + (int64_t)w * bm_words;
@@ -1159,6 +1177,7 @@ __global__ void __launch_bounds__(kThreads)
 clear_listed_groups_kernel(float* __restrict__ alpha, int64_t d, const uint32_t* __restrict__ glist, int64_t cap,
                            const uint32_t* __restrict__ gcount)
 {
+    pdl_prologue();
     const int w = blockIdx.y;
     float* row = alpha + (int64_t)w * d;
     const int64_t n = gcount[w];
@@ -1177,6 +1196,7 @@ __global__ void __launch_bounds__(kThreads)
 model_precision_kernel(const float* __restrict__ x, const float* __restrict__ xsnap, int64_t d, const uint32_t* __restrict__ norm_bits,
                        double* __restrict__ stats)
 {
+    pdl_prologue();
     const float nrm = __uint_as_float(norm_bits[0]);
     double inv[3];
     inv[0] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 1.0f) : 0.0;
@@ -1209,6 +1229,7 @@ model_precision_kernel(const float* __restrict__ x, const float* __restrict__ xs
 __global__ void select_bits_kernel(double* __restrict__ stats, const uint32_t* __restrict__ norm_bits, float mu, int accelerated,
                                    float theta, const RoundParams* __restrict__ rp, int32_t* __restrict__ bits)
 {
+    pdl_prologue();
     if (rp) theta = rp->theta;
     const float nrm = __uint_as_float(norm_bits[0]);
     const double mu_eff = accelerated ? (double)__fmul_rn(theta, mu) : (double)mu;
@@ -1241,7 +1262,7 @@ void launch_norm_inf(dq_ctx* ctx, const float* v, int64_t d, int M, uint32_t* no
 {
     if (!ctx->ninf_zeroed) cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * M, st);
     dim3 grid(grid_for((d + 7) / 8, ctx->sm_count), M);
-    norm_inf_kernel<<<grid, kThreads, 0, st>>>(v, d, vec_ok_for(v, d), norm_bits);
+    launch_k(norm_inf_kernel, grid, kThreads, 0, st, v, d, vec_ok_for(v, d), norm_bits);
     ctx->launches += 1;
 }
 
@@ -1254,14 +1275,12 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
     if (diff) {
         grid.x = max(grid.x, (unsigned)grid_for(zero_n / 4, ctx->sm_count));   // enough blocks for the clearing loop too
-        DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_, true><<<grid, kThreads, 0, st>>>(
-            v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
+        DQ_DISPATCH_BITS(bits, (launch_k(quantize_pack_kernel<BITS_, true>, grid, kThreads, 0, st, v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
             ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits_gate)));
         ctx->launches += 1;
         return;
     }
-    DQ_DISPATCH_BITS(bits, (quantize_pack_kernel<BITS_><<<grid, kThreads, 0, st>>>(
-        v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active)));
+    DQ_DISPATCH_BITS(bits, (launch_k(quantize_pack_kernel<BITS_>, grid, kThreads, 0, st, v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr)));
     ctx->launches += 1;
 }
 
@@ -1269,15 +1288,15 @@ void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const u
                         int32_t* bits, double* stats, cudaStream_t st)
 {
     cudaMemsetAsync(stats, 0, sizeof(double) * 4, st);
-    model_precision_kernel<<<grid_for(ctx->cfg.d / 4 + 1, ctx->sm_count), kThreads, 0, st>>>(x, xsnap, ctx->cfg.d, norm_bits, stats);
-    select_bits_kernel<<<1, 1, 0, st>>>(stats, norm_bits, mu, ctx->cfg.accelerated, theta, ctx->rp_active, bits);
+    launch_k(model_precision_kernel, grid_for(ctx->cfg.d / 4 + 1, ctx->sm_count), kThreads, 0, st, x, xsnap, ctx->cfg.d, norm_bits, stats);
+    launch_k(select_bits_kernel, 1, 1, 0, st, stats, norm_bits, mu, ctx->cfg.accelerated, theta, ctx->rp_active, bits);
     ctx->launches += 2;
 }
 
 void launch_clear_listed(dq_ctx* ctx, cudaStream_t st)
 {
     dim3 grid(16, ctx->cfg.M);
-    clear_listed_groups_kernel<<<grid, kThreads, 0, st>>>(ctx->alpha, ctx->cfg.d, ctx->glist, ctx->glist_cap, ctx->gcount);
+    launch_k(clear_listed_groups_kernel, grid, kThreads, 0, st, ctx->alpha, ctx->cfg.d, ctx->glist, ctx->glist_cap, ctx->gcount);
     ctx->launches += 1;
 }
 
@@ -1287,8 +1306,8 @@ void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st)
     if (!ctx->ninf_zeroed) cudaMemsetAsync(norm_bits, 0, sizeof(uint32_t) * c.M, st);
     const int nseg = (int)((ctx->bm_words + kThreads - 1) / kThreads);
     dim3 grid(nseg, c.M);
-    count_touched_kernel<<<grid, kThreads, 0, st>>>(ctx->touched, ctx->bm_words, ctx->seg_count, nseg);
-    build_group_list_kernel<<<grid, kThreads, 0, st>>>(ctx->touched, ctx->bm_words, ctx->seg_count, nseg, ctx->alpha, c.d,
+    launch_k(count_touched_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg);
+    launch_k(build_group_list_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg, ctx->alpha, c.d,
                                                         vec_ok_for(ctx->alpha, c.d), ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
     ctx->launches += 2;
     ctx->launches += 1;
@@ -1307,21 +1326,20 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     cudaMemsetAsync(ctx->l1_sum, 0, sizeof(unsigned long long) * M, st);
     cudaMemsetAsync(ctx->beta_norm_bits, 0, sizeof(uint32_t) * M, st);
     if (list) {
-        norm_l1_list_kernel<<<dim3(16, M), kThreads, 0, st>>>(v, d, vec_ok, gl, norm_bits, ctx->l1_sum);
+        launch_k(norm_l1_list_kernel, dim3(16, M), kThreads, 0, st, v, d, vec_ok, gl, norm_bits, ctx->l1_sum);
     } else {
         dim3 grid_l1(grid_for((d + 7) / 8, ctx->sm_count), M);
-        norm_l1_kernel<<<grid_l1, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum);
+        launch_k(norm_l1_kernel, grid_l1, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum);
     }
     dim3 grid_c(list ? 64 : grid_for(nchunks * 32, ctx->sm_count), M);
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     if (list) {
-        sparsify_count_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
+        launch_k(sparsify_count_kernel, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
                                                            ctx->beta_norm_bits, ctx->chunk_off, nchunks, ctx->rp_active, gl, iters);
-        chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
+        launch_k(chunk_scan_kernel, M, kThreads, 0, st, ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
         cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
-        DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
-            v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
-            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters)));
+        DQ_DISPATCH_BITS(bits, (launch_k(sparsify_emit_kernel<BITS_, true>, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
+            nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters, nullptr, 0)));
         ctx->launches += 4;
         return;
     }
@@ -1330,27 +1348,23 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     uint32_t* flags = ctx->stage_ctrl;
     const StageBufs sb{ctx->stage_idx, ctx->stage_val, flags};
     cudaMemsetAsync(flags, 0, sizeof(uint32_t) * ((size_t)M + 1), st);
-    sparsify_stage_kernel<<<grid_c, kThreads, 0, st>>>(v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
+    launch_k(sparsify_stage_kernel, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
                                                        ctx->beta_norm_bits, ctx->chunk_off, nchunks, ctx->rp_active, sb, M);
     cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
     ctx->launches += 2;
     dim3 grid_f(grid_for(nchunks * 8, ctx->sm_count), M);
     if (sparse_out) {
-        chunk_scan_kernel<<<M, kThreads, 0, st>>>(ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
-        DQ_DISPATCH_BITS(bits, (sparsify_finish_sparse_kernel<BITS_><<<grid_f, kThreads, 0, st>>>(
-            norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
+        launch_k(chunk_scan_kernel, M, kThreads, 0, st, ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
+        DQ_DISPATCH_BITS(bits, (launch_k(sparsify_finish_sparse_kernel<BITS_>, grid_f, kThreads, 0, st, norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
             out->idx, out->cap, ctx->status, ctx->rp_active)));
-        DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, true><<<grid_c, kThreads, 0, st>>>(
-            v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
+        DQ_DISPATCH_BITS(bits, (launch_k(sparsify_emit_kernel<BITS_, true>, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
             nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters,
             flags, M)));
         ctx->launches += 3;
     } else {
-        DQ_DISPATCH_BITS(bits, (sparsify_scatter_dense_kernel<BITS_><<<grid_f, kThreads, 0, st>>>(
-            norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
+        DQ_DISPATCH_BITS(bits, (launch_k(sparsify_scatter_dense_kernel<BITS_>, grid_f, kThreads, 0, st, norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
             ctx->status, ctx->rp_active)));
-        DQ_DISPATCH_BITS(bits, (sparsify_emit_kernel<BITS_, false><<<grid_c, kThreads, 0, st>>>(
-            v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
+        DQ_DISPATCH_BITS(bits, (launch_k(sparsify_emit_kernel<BITS_, false>, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, nullptr,
             nchunks, ngroups, out->codes, out->stride, out->scale, nullptr, 0, ctx->status, ctx->rp_active, gl, iters,
             flags, M)));
         ctx->launches += 2;
@@ -1372,11 +1386,9 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         const int grid = grid_for(nw, ctx->sm_count);
         const size_t smem = sizeof(float) * c.M;
         if (c.accelerated) {
-            DQ_DISPATCH_BITS(c.b, (master_dense_seq_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_seq_kernel<BITS_, true>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         } else {
-            DQ_DISPATCH_BITS(c.b, (master_dense_seq_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_seq_kernel<BITS_, false>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         }
         ctx->launches += 1;
         return;
@@ -1389,26 +1401,22 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         auto al32 = [](const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 31) == 0; };
         const int vec8_ok = al32(s->x) && al32(s->g_full) && al32(s->y) && al32(s->x_snap) && al32(s->x_sum);
         if (c.accelerated) {
-            DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, true><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_kernel<BITS_, true>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
         } else {
-            DQ_DISPATCH_BITS(c.b, (master_dense_kernel<BITS_, false><<<grid, kThreads, smem, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_kernel<BITS_, false>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
         }
         ctx->launches += 1;
     } else {
         const int64_t ntiles = (d + kChunk - 1) / kChunk;
         dim3 grid_t((unsigned)((ntiles + 1 + kThreads - 1) / kThreads), c.M);
-        tile_ptr_kernel<<<grid_t, kThreads, 0, st>>>(msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
+        launch_k(tile_ptr_kernel, grid_t, kThreads, 0, st, msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
         if (c.sequential) {
             const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
             if (c.accelerated) {
-                DQ_DISPATCH_BITS(c.b, (master_sparse_seq_kernel<BITS_, true><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
-                    msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+                DQ_DISPATCH_BITS(c.b, (launch_k(master_sparse_seq_kernel<BITS_, true>, grid, kThreads, sizeof(uint32_t) * 2 * c.M, st, msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                     s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
             } else {
-                DQ_DISPATCH_BITS(c.b, (master_sparse_seq_kernel<BITS_, false><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
-                    msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+                DQ_DISPATCH_BITS(c.b, (launch_k(master_sparse_seq_kernel<BITS_, false>, grid, kThreads, sizeof(uint32_t) * 2 * c.M, st, msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                     s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
             }
             ctx->launches += 2;
@@ -1416,12 +1424,10 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         }
         const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
         if (c.accelerated) {
-            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, true><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_sparse_kernel<BITS_, true>, grid, kThreads, sizeof(uint32_t) * 2 * c.M, st, msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                 s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         } else {
-            DQ_DISPATCH_BITS(c.b, (master_sparse_kernel<BITS_, false><<<grid, kThreads, sizeof(uint32_t) * 2 * c.M, st>>>(
-                msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_sparse_kernel<BITS_, false>, grid, kThreads, sizeof(uint32_t) * 2 * c.M, st, msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                 s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         }
         ctx->launches += 2;
@@ -1433,11 +1439,10 @@ void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, fl
     const dq_config& c = ctx->cfg;
     const uint8_t* codes = msgs->codes + (int64_t)w * msgs->stride;
     if (!sparse_msgs) {
-        DQ_DISPATCH_BITS(c.b, (unpack_dense_kernel<BITS_><<<grid_for(c.d, ctx->sm_count), kThreads, 0, st>>>(codes, msgs->scale + w, c.d, out)));
+        DQ_DISPATCH_BITS(c.b, (launch_k(unpack_dense_kernel<BITS_>, grid_for(c.d, ctx->sm_count), kThreads, 0, st, codes, msgs->scale + w, c.d, out)));
     } else {
         cudaMemsetAsync(out, 0, sizeof(float) * c.d, st);
-        DQ_DISPATCH_BITS(c.b, (unpack_sparse_kernel<BITS_><<<grid_for(msgs->cap, ctx->sm_count), kThreads, 0, st>>>(
-            codes, msgs->scale + w, msgs->idx + (int64_t)w * msgs->cap, msgs->nnz + w, out)));
+        DQ_DISPATCH_BITS(c.b, (launch_k(unpack_sparse_kernel<BITS_>, grid_for(msgs->cap, ctx->sm_count), kThreads, 0, st, codes, msgs->scale + w, msgs->idx + (int64_t)w * msgs->cap, msgs->nnz + w, out)));
     }
     ctx->launches += 1;
 }
@@ -1498,12 +1503,11 @@ extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, 
     if (cudaMemsetAsync(scratch, 0, sizeof(uint32_t) * (kStaticMaxMessages + 1), st) != cudaSuccess) return DQ_ERR_CUDA;
     const int vec_ok = vec_ok_for(v, d);
     dim3 grid_n(grid_for((d + 7) / 8, sms), M);
-    norm_inf_kernel<<<grid_n, kThreads, 0, st>>>(v, d, vec_ok, scratch);
+    launch_k(norm_inf_kernel, grid_n, kThreads, 0, st, v, d, vec_ok, scratch);
     const int64_t ngroups = dq_packed_bytes(d, b) / b;
     dim3 grid_q(grid_for(ngroups, sms), M);
     const PhiloxKeys keys = expand_keys(seed);
     int* flag = reinterpret_cast<int*>(scratch + kStaticMaxMessages);
-    DQ_DISPATCH_BITS(b, (quantize_pack_kernel<BITS_, false><<<grid_q, kThreads, 0, st>>>(
-        v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr)));
+    DQ_DISPATCH_BITS(b, (launch_k(quantize_pack_kernel<BITS_, false>, grid_q, kThreads, 0, st, v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr)));
     return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }

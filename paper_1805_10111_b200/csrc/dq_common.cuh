@@ -150,6 +150,31 @@ __device__ __forceinline__ void block_atomic_max(uint32_t v, uint32_t* dst)
     }
 }
 
+// Programmatic dependent launch.  Every kernel of the library begins with pdl_prologue(): it lets the next kernel
+// of the stream be scheduled as soon as all blocks of this one are resident (its blocks take the slots that free up
+// while this grid drains), then waits until the kernels before this one have completed and their writes are
+// visible.  Nothing before the wait may touch global memory.  In a kernel launched without the attribute both
+// instructions do nothing.
+__device__ __forceinline__ void pdl_prologue()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// Launch with the programmatic-serialization attribute: the gap between dependent kernels (drain, then launch)
+// is what bounds the small configurations, whose rounds are chains of microsecond kernels.
+template <class... P, class... A>
+inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args)
+{
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<A&&>(args)...);
+}
+
 struct ProxParams { float lambda1, lambda2, lo, hi; };
 
 // Where the sparsifier finds its groups of eight coordinates: every group of the vector (groups == NULL), or

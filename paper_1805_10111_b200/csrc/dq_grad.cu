@@ -93,6 +93,7 @@ template <int BITS>
 __global__ void dequant_diff_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ delta_x,
                                     const float* __restrict__ xsnap, int64_t d, float* __restrict__ diff)
 {
+    pdl_prologue();
     const float dl = *delta_x;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
         const int64_t bit = i * BITS;
@@ -111,6 +112,7 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
                        const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, float* __restrict__ alpha,
                        uint32_t* __restrict__ touched /* bitmap of groups of eight coordinates, may be NULL */, int64_t bm_words)
 {
+    pdl_prologue();
     clear_word(bs);
     const int lane = threadIdx.x & 31;
     const int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -144,6 +146,7 @@ worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labe
                          const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int64_t d,
                          float* __restrict__ alpha)
 {
+    pdl_prologue();
     __shared__ float s_r[kRowsPerBlock];
     __shared__ int64_t s_row[kRowsPerBlock];
     clear_word(bs);
@@ -216,6 +219,7 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
                              const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int64_t d,
                              float* __restrict__ alpha)
 {
+    pdl_prologue();
     constexpr int N = RowVec<T>::N;
     __shared__ float s_r[kRowsPerBlock];
     __shared__ const uint4* s_rowp[kRowsPerBlock];
@@ -266,6 +270,7 @@ worker_margins_kernel(const T* __restrict__ X, const float* __restrict__ labels,
                       const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d,
                       float* __restrict__ rbuf)
 {
+    pdl_prologue();
     clear_word(bs);
     const int lane = threadIdx.x & 31;
     const int64_t slot = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -281,6 +286,7 @@ __global__ void __launch_bounds__(kThreads)
 worker_colsum_kernel(const T* __restrict__ X, const int32_t* __restrict__ rows, const float* __restrict__ rbuf, int B, int64_t d,
                      float* __restrict__ alpha, uint32_t* __restrict__ norm_bits)
 {
+    pdl_prologue();
     constexpr int N = RowVec<T>::N;
     constexpr int kWarps = kThreads / 32;
     __shared__ float s_part[kWarps][32 * N];
@@ -329,6 +335,7 @@ full_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict__ 
                      const float* __restrict__ labels, const float* __restrict__ x, int64_t n, float* __restrict__ z_out,
                      double* __restrict__ g64)
 {
+    pdl_prologue();
     const int lane = threadIdx.x & 31;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     for (int64_t a = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; a < n; a += nwarps) {
@@ -346,6 +353,7 @@ __global__ void __launch_bounds__(kThreads)
 full_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ x, int64_t n,
                        int64_t d, float* __restrict__ z_out, double* __restrict__ g64)
 {
+    pdl_prologue();
     __shared__ float s_c[kRowsPerBlock];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int64_t a0 = (int64_t)blockIdx.x * kRowsPerBlock; a0 < n; a0 += (int64_t)gridDim.x * kRowsPerBlock) {
@@ -371,6 +379,7 @@ __global__ void __launch_bounds__(kThreads)
 full_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ x, int64_t n,
                            int64_t d, float* __restrict__ z_out, double* __restrict__ g64)
 {
+    pdl_prologue();
     constexpr int N = RowVec<T>::N;
     __shared__ float s_c[kRowsPerBlock];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -403,6 +412,7 @@ full_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ la
 
 __global__ void finish_full_grad_kernel(const double* __restrict__ g64, int64_t d, double inv_n, float* __restrict__ g)
 {
+    pdl_prologue();
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x)
         g[i] = (float)(g64[i] * inv_n);
 }
@@ -413,6 +423,7 @@ __global__ void __launch_bounds__(kThreads)
 epoch_state_kernel(float* __restrict__ x, float* __restrict__ xsnap, const float* __restrict__ y, float* __restrict__ xsum,
                    int64_t d, int accelerated, int64_t m_prev, float theta, uint32_t* __restrict__ normx_bits)
 {
+    pdl_prologue();
     uint32_t nmax = 0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
         float xi;
@@ -449,6 +460,7 @@ template <int FMT>
 __global__ void __launch_bounds__(kThreads)
 objective_loss_kernel(dq_data D, const float* __restrict__ x, double* __restrict__ P)
 {
+    pdl_prologue();
     const int lane = threadIdx.x & 31;
     const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     double acc = 0.0;
@@ -465,6 +477,7 @@ objective_loss_kernel(dq_data D, const float* __restrict__ x, double* __restrict
 __global__ void __launch_bounds__(kThreads)
 objective_reg_kernel(const float* __restrict__ x, int64_t d, float l1, float l2, double* __restrict__ P)
 {
+    pdl_prologue();
     double acc = 0.0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
         const double v = (double)x[i];
@@ -477,6 +490,7 @@ objective_reg_kernel(const float* __restrict__ x, int64_t d, float l1, float l2,
 __global__ void bits_kernel(int M, int64_t d, int bx, int b, int flag_round, int sparse_msgs, const uint32_t* __restrict__ nnz,
                             uint64_t* __restrict__ bits_down, uint64_t* __restrict__ bits_up)
 {
+    pdl_prologue();
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     *bits_down = flag_round ? (uint64_t)M : (uint64_t)M * (32ull + (uint64_t)bx * (uint64_t)d);
     uint64_t up = 0;
@@ -505,6 +519,7 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
                   const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
                   float* __restrict__ act_a, float* __restrict__ act_b)
 {
+    pdl_prologue();
     extern __shared__ float s_in[];                      // the row's features
     __shared__ int64_t s_row;
     clear_word(bs);
@@ -573,6 +588,7 @@ mlp_output_kernel(MlpShape sh, const float* __restrict__ labels, const int32_t* 
                   const float* __restrict__ act_b, float wgt, float* __restrict__ dz_a, float* __restrict__ dz_b,
                   float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b)
 {
+    pdl_prologue();
     extern __shared__ float s_z[];                       // [2 * classes]
     const int64_t slot = blockIdx.x;
     const int label = (int)labels[row_of_slot[slot]];
@@ -595,6 +611,7 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
                  const float* __restrict__ dz_b, const float* __restrict__ dh_a, const float* __restrict__ dh_b,
                  float* __restrict__ out, int64_t P, uint32_t* __restrict__ norm_bits, double* __restrict__ g64)
 {
+    pdl_prologue();
     typedef typename std::conditional<FULL, double, float>::type acc_t;
     extern __shared__ float s_w[];                       // per row of the group: dh_a[j] - handled below
     const int j = blockIdx.x, w = blockIdx.y;
@@ -659,15 +676,15 @@ static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStre
     const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
     const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
     const int64_t P = ctx->cfg.d;
-    mlp_hidden_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * sh.in, st>>>((const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
+    launch_k(mlp_hidden_kernel, (unsigned)D.n, kThreads, sizeof(float) * sh.in, st, (const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
                                                                              ctx->mlp_rows, ctx->mlp_act[0], nullptr);
-    mlp_output_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st>>>(sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
+    launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
         nullptr, (float)(1.0 / (double)D.n), ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr);
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * P, st);
     dim3 grid(sh.hidden + 1, (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
-    mlp_param_kernel<true><<<grid, kThreads, sizeof(float) * 2 * kMlpGroup, st>>>((const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
+    launch_k(mlp_param_kernel<true>, grid, kThreads, sizeof(float) * 2 * kMlpGroup, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
         ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
-    finish_full_grad_kernel<<<blocks_for(P, ctx->sm_count), kThreads, 0, st>>>(ctx->g64, P, 1.0, g);
+    launch_k(finish_full_grad_kernel, blocks_for(P, ctx->sm_count), kThreads, 0, st, ctx->g64, P, 1.0, g);
     ctx->launches += 4;
 }
 
@@ -678,13 +695,13 @@ static void launch_mlp_worker_grad(dq_ctx* ctx, const float* xhat, const dq_stat
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
     const unsigned R = (unsigned)(c.M * c.B);
     uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
-    mlp_hidden_kernel<<<R, kThreads, sizeof(float) * sh.in, st>>>((const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
+    launch_k(mlp_hidden_kernel, R, kThreads, sizeof(float) * sh.in, st, (const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
                                                                    ctx->mlp_act[0], ctx->mlp_act[1]);
-    mlp_output_kernel<<<R, kThreads, sizeof(float) * 2 * sh.classes, st>>>(sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
+    launch_k(mlp_output_kernel, R, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
         ctx->mlp_act[1], 1.0f / (float)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr);
     if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
     dim3 grid(sh.hidden + 1, c.M);
-    mlp_param_kernel<false><<<grid, kThreads, sizeof(float) * 2 * c.B, st>>>((const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
+    launch_k(mlp_param_kernel<false>, grid, kThreads, sizeof(float) * 2 * c.B, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
         ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
     ctx->launches += 3;
 }
@@ -694,28 +711,27 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
     uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
     cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
-    epoch_state_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(s->x, s->x_snap, s->y, s->x_sum, c.d, c.accelerated,
+    launch_k(epoch_state_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, s->x, s->x_snap, s->y, s->x_sum, c.d, c.accelerated,
                                                                             ctx->ticks_in_epoch, theta, nx);
     if (c.model == DQ_MODEL_MLP) { launch_mlp_full_grad(ctx, s->x_snap, s->g_full, st); ctx->launches += 1; return; }
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * c.d, st);
     if (D.format == DQ_CSR_F32) {
-        full_grad_csr_kernel<<<blocks_for(D.n * 32, ctx->sm_count), kThreads, 0, st>>>(
-            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, s->x_snap, D.n, s->z_snap, ctx->g64);
+        launch_k(full_grad_csr_kernel, blocks_for(D.n * 32, ctx->sm_count), kThreads, 0, st, (const float*)D.values, D.col_idx, D.row_ptr, D.labels, s->x_snap, D.n, s->z_snap, ctx->g64);
     } else {
         const int64_t nblk = (D.n + kRowsPerBlock - 1) / kRowsPerBlock;
         const int grid = (int)(nblk < (int64_t)ctx->sm_count * 8 ? nblk : (int64_t)ctx->sm_count * 8);
         const bool f32 = D.format == DQ_DENSE_F32;
         const bool vec = (D.d % (f32 ? 4 : 8)) == 0;
         if (f32 && vec)
-            full_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+            launch_k(full_grad_dense_vec_kernel<float>, grid, kThreads, 0, st, (const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
         else if (f32)
-            full_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+            launch_k(full_grad_dense_kernel<float>, grid, kThreads, 0, st, (const float*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
         else if (vec)
-            full_grad_dense_vec_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+            launch_k(full_grad_dense_vec_kernel<__nv_bfloat16>, grid, kThreads, 0, st, (const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
         else
-            full_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
+            launch_k(full_grad_dense_kernel<__nv_bfloat16>, grid, kThreads, 0, st, (const __nv_bfloat16*)D.values, D.labels, s->x_snap, D.n, D.d, s->z_snap, ctx->g64);
     }
-    finish_full_grad_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(ctx->g64, c.d, 1.0 / (double)D.n, s->g_full);
+    launch_k(finish_full_grad_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, ctx->g64, c.d, 1.0 / (double)D.n, s->g_full);
     ctx->launches += 3;
 }
 
@@ -745,8 +761,7 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
     const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n,
                             ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr};
     if (!ctx->diff_ready) {
-        DQ_DISPATCH_BITS(c.bx, (dequant_diff_kernel<BITS_><<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(
-            codes_x, delta_x, c.model == DQ_MODEL_MLP ? nullptr : s->x_snap, c.d, ctx->xhat_diff)));
+        DQ_DISPATCH_BITS(c.bx, (launch_k(dequant_diff_kernel<BITS_>, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, codes_x, delta_x, c.model == DQ_MODEL_MLP ? nullptr : s->x_snap, c.d, ctx->xhat_diff)));
         ctx->launches += 1;
     }
     if (c.model == DQ_MODEL_MLP) {        // xhat_diff holds xhat itself for the network (no reference subtracted)
@@ -755,8 +770,7 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
     }
     if (D.format == DQ_CSR_F32) {
         if (!ctx->alpha_zeroed && !list) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
-        worker_grad_csr_kernel<<<(int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st>>>(
-            (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha,
+        launch_k(worker_grad_csr_kernel, (int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st, (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha,
             list ? ctx->touched : nullptr, ctx->bm_words);
     } else {
         dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
@@ -770,27 +784,27 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
             const int gm = (int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads);
             const size_t smem = sizeof(float) * 2 * c.B;
             if (f32) {
-                worker_margins_kernel<float><<<gm, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap,
+                launch_k(worker_margins_kernel<float>, gm, kThreads, 0, st, (const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap,
                                                                        ctx->keys, bs, c.M, c.B, c.d, ctx->rbuf);
                 dim3 gc((unsigned)((c.d / 4 + 31) / 32), c.M);
-                worker_colsum_kernel<float><<<gc, kThreads, smem, st>>>((const float*)D.values, rows_eff, ctx->rbuf, c.B, c.d, alpha, nb);
+                launch_k(worker_colsum_kernel<float>, gc, kThreads, smem, st, (const float*)D.values, rows_eff, ctx->rbuf, c.B, c.d, alpha, nb);
             } else {
-                worker_margins_kernel<__nv_bfloat16><<<gm, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff,
+                launch_k(worker_margins_kernel<__nv_bfloat16>, gm, kThreads, 0, st, (const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff,
                                                                                s->z_snap, ctx->keys, bs, c.M, c.B, c.d, ctx->rbuf);
                 dim3 gc((unsigned)((c.d / 8 + 31) / 32), c.M);
-                worker_colsum_kernel<__nv_bfloat16><<<gc, kThreads, smem, st>>>((const __nv_bfloat16*)D.values, rows_eff, ctx->rbuf, c.B,
+                launch_k(worker_colsum_kernel<__nv_bfloat16>, gc, kThreads, smem, st, (const __nv_bfloat16*)D.values, rows_eff, ctx->rbuf, c.B,
                                                                                  c.d, alpha, nb);
             }
             ctx->launches += 2;
             return;
         } else if (f32 && vec)
-            worker_grad_dense_vec_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
+            launch_k(worker_grad_dense_vec_kernel<float>, grid, kThreads, 0, st, (const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else if (f32)
-            worker_grad_dense_kernel<float><<<grid, kThreads, 0, st>>>((const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
+            launch_k(worker_grad_dense_kernel<float>, grid, kThreads, 0, st, (const float*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else if (vec)
-            worker_grad_dense_vec_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
+            launch_k(worker_grad_dense_vec_kernel<__nv_bfloat16>, grid, kThreads, 0, st, (const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
         else
-            worker_grad_dense_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
+            launch_k(worker_grad_dense_kernel<__nv_bfloat16>, grid, kThreads, 0, st, (const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
     }
     ctx->launches += 1;
     if (list) { launch_build_group_list(ctx, reinterpret_cast<uint32_t*>(norm_inf), st); ctx->list_ready = true; }
@@ -804,30 +818,31 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
     if (c.model == DQ_MODEL_MLP) {
         const MlpShape sh = mlp_shape(ctx);
         const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
-        mlp_hidden_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * sh.in, st>>>((const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
+        launch_k(mlp_hidden_kernel, (unsigned)D.n, kThreads, sizeof(float) * sh.in, st, (const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
                                                                                  ctx->mlp_rows, nullptr, ctx->mlp_act[1]);
-        mlp_output_kernel<<<(unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st>>>(sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
+        launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
             ctx->mlp_act[1], (float)(1.0 / (double)D.n), nullptr, nullptr, nullptr, nullptr, P);
-        objective_reg_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(x, c.d, c.lambda1, c.lambda2, P);
+        launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
         ctx->launches += 3;
         return;
     }
     const int grid = blocks_for(D.n * 32, ctx->sm_count);
-    if (D.format == DQ_CSR_F32) objective_loss_kernel<DQ_CSR_F32><<<grid, kThreads, 0, st>>>(D, x, P);
-    else if (D.format == DQ_DENSE_F32) objective_loss_kernel<DQ_DENSE_F32><<<grid, kThreads, 0, st>>>(D, x, P);
-    else objective_loss_kernel<DQ_DENSE_BF16><<<grid, kThreads, 0, st>>>(D, x, P);
-    objective_reg_kernel<<<blocks_for(c.d, ctx->sm_count), kThreads, 0, st>>>(x, c.d, c.lambda1, c.lambda2, P);
+    if (D.format == DQ_CSR_F32) launch_k(objective_loss_kernel<DQ_CSR_F32>, grid, kThreads, 0, st, D, x, P);
+    else if (D.format == DQ_DENSE_F32) launch_k(objective_loss_kernel<DQ_DENSE_F32>, grid, kThreads, 0, st, D, x, P);
+    else launch_k(objective_loss_kernel<DQ_DENSE_BF16>, grid, kThreads, 0, st, D, x, P);
+    launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
     ctx->launches += 2;
 }
 
 __global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float eta, float theta)
 {
+    pdl_prologue();
     rp->round = round; rp->eta = eta; rp->theta = theta; rp->pad = 0u;
 }
 
 void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st)
 {
-    set_round_params_kernel<<<1, 1, 0, st>>>(ctx->rp_dev, round, eta, theta);
+    launch_k(set_round_params_kernel, 1, 1, 0, st, ctx->rp_dev, round, eta, theta);
     ctx->launches += 1;
 }
 
@@ -835,7 +850,7 @@ void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* 
                  cudaStream_t st)
 {
     const dq_config& c = ctx->cfg;
-    bits_kernel<<<1, 32, 0, st>>>(c.M, c.d, c.bx, c.b, flag_round, sparse_msgs ? 1 : 0, nnz, bits_down, bits_up);
+    launch_k(bits_kernel, 1, 32, 0, st, c.M, c.d, c.bx, c.b, flag_round, sparse_msgs ? 1 : 0, nnz, bits_down, bits_up);
     ctx->launches += 1;
 }
 
