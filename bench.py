@@ -209,7 +209,7 @@ TRAIN_CONFIGS = {
 
 
 def time_training_config(name, rounds=200, warmup=20):
-    """rounds/s of dq_round on one of the training configurations (full size, synthetic data), plus the bits
+    """rounds/s of dq_rounds on one of the training configurations (full size, synthetic data), plus the bits
     the paper's accounting charges per round."""
     import numpy as np
     import torch
@@ -232,8 +232,7 @@ def time_training_config(name, rounds=200, warmup=20):
     l0 = dq.dq_launch_count(ctx)
     e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
     e0.record()
-    for r in range(rounds):
-        dq.ok(dq.dq_round(ctx, st, warmup + r, eta, theta, bits[0:1], bits[1:2]))
+    dq.ok(dq.dq_rounds(ctx, st, warmup, rounds, eta, theta, bits[0:1], bits[1:2]))      # one call for all rounds of the epoch
     e1.record(); torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / rounds
     rc, status = dq.dq_poll_status(ctx)

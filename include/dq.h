@@ -89,7 +89,7 @@ typedef struct {
                                   the data must be DQ_DENSE_F32 with labels = class index, data.d = number of inputs, and
                                   d = hidden*(in+1) + classes*(hidden+1) with x = [W1 (hidden x in), b1, W2 (classes x hidden), b2] */
     int32_t hidden, classes;
-    int32_t reserved2;
+    int32_t no_fused;          /* 1: never run rounds in the one-cluster kernel (see dq_round); 0: use it where it applies */
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3
@@ -178,9 +178,21 @@ int dq_master_unpack_aggregate_prox(dq_ctx* ctx, const dq_msgs* msgs, dq_state* 
  * (Algorithm 3: of the first epoch only).
  * Unless no_graph is set, the first non-snapshot round on a given set of state/counter pointers records its
  * kernel sequence as a CUDA graph (this allocates); later rounds copy (round, eta, theta) to the device and
- * replay it.  Calling with other pointers records again. */
+ * replay it.  Calling with other pointers records again.
+ * Small problems (logistic model on DENSE_F32 or CSR_F32 data, dense messages, synchronous master, fixed b_x,
+ * d <= 8192, M <= 16, B <= 1024) skip the graph unless no_fused is set: their non-snapshot rounds run in ONE
+ * kernel on one thread-block cluster (block w is worker w; the blocks meet at the cluster barrier around the
+ * master step), because
+ * separate kernels would spend their time in launch gaps.  Results, buffers and layouts are the same. */
 int dq_round(dq_ctx* ctx, dq_state* st, uint32_t round, float eta, float theta,
              uint64_t* bits_down, uint64_t* bits_up, void* stream);
+
+/* nrounds consecutive rounds round0, round0 + 1, ... of the same epoch with the same (eta, theta), as by
+ * dq_round called once per round (Algorithm 1 steps 6-13 repeated; the caller places dq_epoch_begin between
+ * epochs).  Where the one-cluster kernel applies, all non-snapshot rounds of the call run in a single launch;
+ * otherwise the rounds are enqueued one after the other.  bits_down / bits_up hold the last round's counts. */
+int dq_rounds(dq_ctx* ctx, dq_state* st, uint32_t round0, int32_t nrounds, float eta, float theta,
+              uint64_t* bits_down, uint64_t* bits_up, void* stream);
 
 /* The round without its gradient stage, for callers that bring their own M gradient vectors v [M][d]:
  * quantise(+sparsify)+pack into the context's buffers, master step on `st`, then model quantisation of the

@@ -122,7 +122,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     rc |= dev_alloc(&c->stage_idx, cfg->sparsify ? (size_t)M * c->nchunks * kStash : 1);
     rc |= dev_alloc(&c->stage_val, cfg->sparsify ? (size_t)M * c->nchunks * kStash : 1);
     rc |= dev_alloc(&c->stage_ctrl, (size_t)M + 1);
-    rc |= dev_alloc(&c->xnorm_bits, 1);
+    rc |= dev_alloc(&c->xnorm_bits, 2);
     rc |= dev_alloc(&c->status, 1);
     rc |= dev_alloc(&c->bits, 2);
     rc |= dev_alloc(&c->rp_dev, 1);
@@ -170,6 +170,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (rc == DQ_OK && cudaMemset(c->bx_dev, 0, sizeof(int32_t)) != cudaSuccess) rc = DQ_ERR_CUDA;
     if (rc != DQ_OK) { dq_destroy(c); cudaGetLastError(); return DQ_ERR_CUDA; }
     c->epoch = -1;
+    small_round_setup(c);
     *out = c;
     return DQ_OK;
 }
@@ -381,6 +382,12 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
     if (ctx->epoch < 0) return DQ_ERR_ARG;                     // dq_epoch_begin has not run
     const dq_config& c = ctx->cfg;
     const int flag = c.snapshot_flag && ctx->rounds_in_epoch == 0 && (!c.accelerated || ctx->epoch == 0);
+    if (!flag && ctx->cluster_blocks > 0) {                  // small problem: the whole round in one cluster kernel
+        launch_round_cluster(ctx, s, round, 1, eta, theta, bits_down, bits_up, as_stream(stream));
+        ctx->rounds_in_epoch += 1;
+        ctx->ticks_in_epoch += 1;
+        return last_error();
+    }
     bool replayed = false;
     if (!flag && !ctx->graph_off && !c.no_graph) {
         const dq_state& g = ctx->graph_state;
@@ -402,6 +409,31 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
     }
     ctx->rounds_in_epoch += 1;
     ctx->ticks_in_epoch += ctx->cfg.sequential ? ctx->cfg.M : 1;
+    return last_error();
+}
+
+int dq_rounds(dq_ctx* ctx, dq_state* s, uint32_t round0, int32_t nrounds, float eta, float theta, uint64_t* bits_down,
+              uint64_t* bits_up, void* stream)
+{
+    if (!ctx || nrounds < 0) return DQ_ERR_ARG;
+    int32_t i = 0;
+    while (i < nrounds) {
+        const dq_config& c = ctx->cfg;
+        const bool flag = c.snapshot_flag && ctx->rounds_in_epoch == 0 && (!c.accelerated || ctx->epoch == 0);
+        if (flag || ctx->cluster_blocks == 0) {                // one round by the general path (it checks the arguments)
+            const int rc = dq_round(ctx, s, round0 + (uint32_t)i, eta, theta, bits_down, bits_up, stream);
+            if (rc != DQ_OK) return rc;
+            i += 1;
+            continue;
+        }
+        int rc = check_state(ctx, s);
+        if (rc != DQ_OK) return rc;
+        if (!ctx->has_data || !s->x_snap || !s->z_snap || !(eta > 0.0f) || !isfinite(eta) || ctx->epoch < 0) return DQ_ERR_ARG;
+        launch_round_cluster(ctx, s, round0 + (uint32_t)i, nrounds - i, eta, theta, bits_down, bits_up, as_stream(stream));
+        ctx->rounds_in_epoch += nrounds - i;
+        ctx->ticks_in_epoch += nrounds - i;
+        i = nrounds;
+    }
     return last_error();
 }
 

@@ -661,28 +661,6 @@ tile_ptr_kernel(const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* _
 // Master step: g = (1/M) sum_w code_w delta_w (fused multiply-adds in worker order), u = g + g_full,
 // prox step on x (Algorithms 1/2) or on y with the momentum combination (Algorithm 3), ||x||_inf.
 // ---------------------------------------------------------------------------------------------------
-__device__ __forceinline__ float prox_h(float v, float thr, float den, float lo, float hi)
-{
-    const float a = __fsub_rn(fabsf(v), thr);
-    float r = (a > 0.0f) ? copysignf(a, v) : 0.0f;
-    if (den != 1.0f) r = __fdiv_rn(r, den);
-    return fminf(fmaxf(r, lo), hi);
-}
-
-template <bool ACC>
-__device__ __forceinline__ float master_update(float acc, float inv_m, float eta, float theta, float thr, float den,
-                                               const ProxParams& pp, float g_full, float x_or_y, float xsnap,
-                                               float& y_out, float& xsum_io)
-{
-    const float u = __fadd_rn(__fmul_rn(acc, inv_m), g_full);
-    const float p = prox_h(__fmaf_rn(-eta, u, x_or_y), thr, den, pp.lo, pp.hi);
-    if (!ACC) return p;
-    y_out = p;
-    const float x = __fmaf_rn(theta, __fsub_rn(p, xsnap), xsnap);
-    xsum_io = __fadd_rn(xsum_io, x);
-    return x;
-}
-
 // acc[j] = fma(code_j, delta, acc[j]) for the 32/BITS codes of one packed word.  The integer-to-float
 // conversion avoids the conversion pipe: the code, biased by 2^(BITS-1), is placed in the mantissa of 2^23
 // (one byte permute) and the bias is subtracted exactly.

@@ -177,6 +177,31 @@ inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, c
 
 struct ProxParams { float lambda1, lambda2, lo, hi; };
 
+// prox of h = lambda1 |x|_1 + (lambda2/2) |x|^2 + indicator of [lo, hi] at v with step eta: thr = eta lambda1,
+// den = 1 + eta lambda2 (soft threshold, shrink, clip), and the master's update of one coordinate built on it
+// (Algorithm 1 step 9; Algorithm 3 step 9 with the momentum combination).
+__device__ __forceinline__ float prox_h(float v, float thr, float den, float lo, float hi)
+{
+    const float a = __fsub_rn(fabsf(v), thr);
+    float r = (a > 0.0f) ? copysignf(a, v) : 0.0f;
+    if (den != 1.0f) r = __fdiv_rn(r, den);
+    return fminf(fmaxf(r, lo), hi);
+}
+
+template <bool ACC>
+__device__ __forceinline__ float master_update(float acc, float inv_m, float eta, float theta, float thr, float den,
+                                               const ProxParams& pp, float g_full, float x_or_y, float xsnap,
+                                               float& y_out, float& xsum_io)
+{
+    const float u = __fadd_rn(__fmul_rn(acc, inv_m), g_full);
+    const float p = prox_h(__fmaf_rn(-eta, u, x_or_y), thr, den, pp.lo, pp.hi);
+    if (!ACC) return p;
+    y_out = p;
+    const float x = __fmaf_rn(theta, __fsub_rn(p, xsnap), xsnap);
+    xsum_io = __fadd_rn(xsum_io, x);
+    return x;
+}
+
 // Where the sparsifier finds its groups of eight coordinates: every group of the vector (groups == NULL), or
 // an ascending list of the groups that can hold a nonzero (groups [M][cap], count [M]).
 struct GroupList { const uint32_t* groups; const uint32_t* count; int64_t cap; };
@@ -263,6 +288,7 @@ struct dq_ctx {
     bool graph_off;
     // sparse gradients (CSR data, sparse messages): bitmap of touched groups, their ascending list, its length
     uint32_t* touched; uint32_t* glist; uint32_t* gcount; uint32_t* seg_count; int64_t bm_words; int64_t glist_cap;
+    int cluster_blocks;         // blocks of the one-cluster round kernel for small problems; 0: rounds run as separate kernels
     bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only
     bool list_ready;            // the list of this round has been built (consumed by the sparsifier launch)
     bool alpha_zeroed, ninf_zeroed, normx_zeroed;   // an earlier kernel of this round already cleared these

@@ -657,6 +657,286 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
 }
 
 // ---------------------------------------------------------------------------------------------------
+// Whole rounds in one kernel for small problems.  A round of Algorithm 1 / 3 is a chain of dependent stages; as
+// separate kernels each costs a launch gap of a few microseconds, which is all the time a problem of a few
+// thousand coordinates needs.  Here one thread-block cluster of M blocks runs `nrounds` consecutive rounds.
+// Block w IS worker w: it dequantises the broadcast model into its own shared memory (every block draws the same
+// codes, so nothing has to be exchanged), computes its minibatch gradient alpha_w there, takes the norm,
+// quantises and packs its message -- all behind block-level barriers only.  The blocks meet at the hardware
+// cluster barrier (release/acquire at cluster scope) twice per round: before the master step, which all blocks
+// share by coordinate range, and after it.  The arithmetic of every stage is that of the stand-alone kernels:
+// same quantiser, same draws, same master update; the global buffers and their layouts are the same too.
+// ---------------------------------------------------------------------------------------------------
+struct SmallRound {
+    // data
+    const float* values; const int32_t* col; const int64_t* row_ptr; const float* labels; int64_t n;
+    // problem
+    int64_t d; int M, B, bx, b; ProxParams pp;
+    // state
+    float* x; float* y; float* xsum; const float* xsnap; const float* gfull; const float* zsnap; uint32_t* normx;
+    // buffers of the round
+    float* alpha; uint32_t* ninf; int32_t* rows; uint8_t* codes_x; float* delta_x; uint32_t* xnorm2 /* [2] scratch */;
+    uint8_t* codes; int64_t stride; float* scale; uint64_t* bits_down; uint64_t* bits_up; int* status;
+    // what to run
+    uint32_t round0; int nrounds; float eta, theta;
+};
+
+constexpr int kSmallThreads = 1024;
+// A packed message is padded to 16 bytes, i.e. up to 64 coordinates at two bits: shared vectors carry that many zeros.
+__host__ __device__ inline int64_t small_round_pad(int64_t d) { return ((d + 63) / 64 + 1) * 64; }
+
+__device__ __forceinline__ void cluster_barrier()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Block-wide maximum through shared memory; every thread gets the result.
+__device__ __forceinline__ uint32_t small_block_max(uint32_t v, uint32_t* s_red)
+{
+    v = warp_max_u32(v);
+    __syncthreads();                                          // s_red may still be in use by the previous reduction
+    if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    uint32_t t = (threadIdx.x & 31) < (blockDim.x >> 5) ? s_red[threadIdx.x & 31] : 0u;
+    return warp_max_u32(t);
+}
+
+// Eight consecutive floats (16-byte aligned): from L2, through the read-only path, and the store.
+__device__ __forceinline__ void small_load8_cg(const float* p, float (&v)[8])
+{
+    const float4 lo = __ldcg(reinterpret_cast<const float4*>(p)), hi = __ldcg(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = lo.x; v[1] = lo.y; v[2] = lo.z; v[3] = lo.w; v[4] = hi.x; v[5] = hi.y; v[6] = hi.z; v[7] = hi.w;
+}
+__device__ __forceinline__ void small_load8_ro(const float* p, float (&v)[8])
+{
+    const float4 lo = __ldg(reinterpret_cast<const float4*>(p)), hi = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = lo.x; v[1] = lo.y; v[2] = lo.z; v[3] = lo.w; v[4] = hi.x; v[5] = hi.y; v[6] = hi.z; v[7] = hi.w;
+}
+__device__ __forceinline__ void small_store8(float* p, const float (&v)[8])
+{
+    reinterpret_cast<float4*>(p)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(p)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+// Q_(delta,b) of one vector held by this block (v in shared or global memory, read with plain loads when `shared`,
+// else from L2), packed codes to `out` if not NULL; with `diff`, code * delta - ref goes to shared memory.
+// Data that another block wrote earlier in the same launch is read with ld.global.cg: L2 is where the writes of
+// all blocks meet, and the read-only path may serve stale lines for such data.
+template <int BITS, bool SHARED_IN>
+__device__ __forceinline__ void small_quantize(const float* v, int64_t d, uint32_t nb, uint8_t* out, float* scale_out,
+                                               const PhiloxKeys& K, uint32_t round, uint32_t worker, uint32_t stream,
+                                               int* status, const float* __restrict__ ref, float* diff)
+{
+    const int64_t ngroups = ((((d * BITS + 7) / 8) + 15) / 16 * 16) / BITS;       // covers the zero padding
+    const float nrm = __uint_as_float(nb);
+    const bool ok = nb < 0x7F800000u && nb != 0u;
+    const float inv = ok ? __fdiv_rd((float)levels(BITS), nrm) : 0.0f;
+    const float delta = ok ? __fdiv_rn(nrm, (float)levels(BITS)) : 0.0f;
+    if (threadIdx.x == 0 && scale_out) { *scale_out = delta; if (nb >= 0x7F800000u) set_status(status, DQ_ERR_NONFINITE); }
+    const bool al16 = (reinterpret_cast<uintptr_t>(v) & 15) == 0 && (!ref || (reinterpret_cast<uintptr_t>(ref) & 15) == 0);
+    for (int64_t g = threadIdx.x; g < ngroups; g += blockDim.x) {
+        float a[8];
+        const int64_t i0 = g << 3;
+        const bool whole = SHARED_IN || (al16 && i0 + 8 <= d);     // shared vectors are padded with zeros past d
+        if (whole) {
+            const float4 lo = SHARED_IN ? reinterpret_cast<const float4*>(v + i0)[0] : __ldcg(reinterpret_cast<const float4*>(v + i0));
+            const float4 hi = SHARED_IN ? reinterpret_cast<const float4*>(v + i0)[1] : __ldcg(reinterpret_cast<const float4*>(v + i0) + 1);
+            a[0] = lo.x; a[1] = lo.y; a[2] = lo.z; a[3] = lo.w; a[4] = hi.x; a[5] = hi.y; a[6] = hi.z; a[7] = hi.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a[j] = (i0 + j < d) ? __ldcg(v + i0 + j) : 0.0f;
+        }
+        uint32_t r[4], s[8];
+        philox4x32_10((uint32_t)g, round, worker, stream, K, r);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+        if (out) store_group<BITS>(out + g * BITS, pack8<BITS>(s));
+        if (diff) {                                            // diff is a padded shared vector
+            float rf[8], o[8];
+            if (whole) {
+                const float4 lo = __ldg(reinterpret_cast<const float4*>(ref + i0)), hi = __ldg(reinterpret_cast<const float4*>(ref + i0) + 1);
+                rf[0] = lo.x; rf[1] = lo.y; rf[2] = lo.z; rf[3] = lo.w; rf[4] = hi.x; rf[5] = hi.y; rf[6] = hi.z; rf[7] = hi.w;
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) rf[j] = (i0 + j < d) ? ref[i0 + j] : 0.0f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) o[j] = (i0 + j < d) ? __fsub_rn(__fmul_rn((float)((int)((s[j] >> 16) & 0xFFu) - 128), delta), rf[j]) : 0.0f;
+            reinterpret_cast<float4*>(diff + i0)[0] = make_float4(o[0], o[1], o[2], o[3]);
+            reinterpret_cast<float4*>(diff + i0)[1] = make_float4(o[4], o[5], o[6], o[7]);
+        }
+    }
+}
+
+template <int FMT, bool ACC>
+__global__ void __launch_bounds__(kSmallThreads, 1)
+round_cluster_kernel(const __grid_constant__ SmallRound P, const __grid_constant__ PhiloxKeys K)
+{
+    pdl_prologue();
+    extern __shared__ float s_mem[];
+    __shared__ uint32_t s_red[32];
+    __shared__ float s_scale[16];
+    __shared__ float s_r[FMT == DQ_DENSE_F32 ? 1024 : 1];
+    __shared__ int64_t s_rowi[FMT == DQ_DENSE_F32 ? 1024 : 1];
+    const int64_t d = P.d; const int M = P.M, B = P.B;
+    const int64_t dpad = small_round_pad(d);                  // room for the zero padding of a packed message
+    float* s_diff = s_mem;                                    // [dpad] xhat - xsnap
+    float* s_alpha = s_mem + dpad;                            // [dpad] this worker's gradient difference, zeros past d
+    const int w = blockIdx.x, lane = threadIdx.x & 31;
+    const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, gnth = (int64_t)gridDim.x * blockDim.x;
+    for (int it = 0; it < P.nrounds; ++it) {
+        const uint32_t round = P.round0 + (uint32_t)it;
+        // ---- model: every block draws the same codes; block 0 also writes them out ---------------------------------
+        const uint32_t* nsrc = it == 0 ? P.normx : P.xnorm2 + ((it - 1) & 1);
+        const uint32_t nbx = __ldcg(nsrc);
+        if (gtid == 0) P.xnorm2[it & 1] = 0u;                 // read last in the previous round, two barriers ago
+        DQ_DISPATCH_BITS(P.bx, (small_quantize<BITS_, false>(P.x, d, nbx, w == 0 ? P.codes_x : nullptr, w == 0 ? P.delta_x : nullptr, K,
+                                                              round, kMaster, kStreamModel, P.status, P.xsnap, s_diff)));
+        for (int64_t i = (FMT == DQ_CSR_F32 ? 0 : d) + threadIdx.x; i < dpad; i += blockDim.x) s_alpha[i] = 0.0f;
+        __syncthreads();
+        // ---- worker w: slope differences of its sampled rows ------------------------------------------------------
+        if (FMT == DQ_CSR_F32) {
+            // sixteen lanes per row: a row of a text-like matrix has a few dozen nonzeros
+            const int sub = threadIdx.x >> 4, nsub = blockDim.x >> 4, l16 = threadIdx.x & 15;
+            const uint32_t submask = 0xFFFFu << (lane & 16);
+            for (int j = sub; j < B; j += nsub) {
+                const int64_t a = sample_row(K, round, w, j, M, P.n);
+                if (l16 == 0) P.rows[(int64_t)w * B + j] = (int32_t)a;
+                const int64_t k0 = P.row_ptr[a], k1 = P.row_ptr[a + 1];
+                const float ya = P.labels[a], za = P.zsnap[a];
+                double sdot = 0.0;
+#pragma unroll 4
+                for (int64_t k = k0 + l16; k < k1; k += 16) sdot += (double)__ldg(P.values + k) * (double)s_diff[__ldg(P.col + k)];
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) sdot += __shfl_xor_sync(submask, sdot, o);
+                const float r = slope_difference(ya, za, (float)sdot) / (float)B;
+                for (int64_t k = k0 + l16; k < k1; k += 16) atomicAdd(s_alpha + __ldg(P.col + k), r * __ldg(P.values + k));
+            }
+            __syncthreads();
+        } else {
+            const bool vec = (d & 3) == 0;
+            for (int j = threadIdx.x >> 5; j < B; j += (int)(blockDim.x >> 5)) {
+                const int64_t a = sample_row(K, round, w, j, M, P.n);
+                const float* row = P.values + a * d;
+                const float ya = P.labels[a], za = P.zsnap[a];     // in flight together with the row
+                float s0 = 0.0f, s1 = 0.0f, s2 = 0.0f, s3 = 0.0f;
+                if (vec) {
+#pragma unroll 8
+                    for (int64_t v = lane; v < (d >> 2); v += 32) {
+                        const float4 f = __ldg(reinterpret_cast<const float4*>(row) + v), x4 = reinterpret_cast<const float4*>(s_diff)[v];
+                        s0 = fmaf(f.x, x4.x, s0); s1 = fmaf(f.y, x4.y, s1); s2 = fmaf(f.z, x4.z, s2); s3 = fmaf(f.w, x4.w, s3);
+                    }
+                } else {
+#pragma unroll 8
+                    for (int64_t i = lane; i < d; i += 32) s0 = fmaf(__ldg(row + i), s_diff[i], s0);
+                }
+                const double dz = warp_sum(((double)s0 + (double)s1) + ((double)s2 + (double)s3));
+                if (lane == 0) {
+                    P.rows[(int64_t)w * B + j] = (int32_t)a;
+                    s_r[j] = slope_difference(ya, za, (float)dz) / (float)B; s_rowi[j] = a;
+                }
+            }
+            __syncthreads();
+            // alpha_w[i] = sum_j r_j a_j[i], rows in slot order (no atomics: reproducible bit for bit)
+            for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
+                float acc = 0.0f;
+#pragma unroll 16
+                for (int j = 0; j < B; ++j) acc = fmaf(s_r[j], __ldg(P.values + s_rowi[j] * d + i), acc);
+                s_alpha[i] = acc;
+            }
+            __syncthreads();
+        }
+        // ---- ||alpha_w||_inf, message w --------------------------------------------------------------------------------
+        uint32_t m = 0;
+        for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
+            const float av = s_alpha[i];
+            P.alpha[(int64_t)w * d + i] = av;
+            m = max(m, __float_as_uint(av) & 0x7FFFFFFFu);
+        }
+        m = small_block_max(m, s_red);
+        if (threadIdx.x == 0) P.ninf[w] = m;
+        DQ_DISPATCH_BITS(P.b, (small_quantize<BITS_, true>(s_alpha, d, m, P.codes + (int64_t)w * P.stride, P.scale + w, K, round, (uint32_t)w,
+                                                            kStreamGrad, P.status, nullptr, nullptr)));
+        cluster_barrier();
+        // ---- master step, groups of eight coordinates shared by all blocks -----------------------------------------------
+        {
+            if (threadIdx.x < M) s_scale[threadIdx.x] = __ldcg(P.scale + threadIdx.x);
+            __syncthreads();
+            const float inv_m = __fdiv_rn(1.0f, (float)M);
+            const float thr = __fmul_rn(P.eta, P.pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(P.eta, P.pp.lambda2));
+            const int b = P.b;
+            const bool al16 = ((reinterpret_cast<uintptr_t>(P.x) | reinterpret_cast<uintptr_t>(P.gfull) | reinterpret_cast<uintptr_t>(P.y) |
+                                reinterpret_cast<uintptr_t>(P.xsnap) | reinterpret_cast<uintptr_t>(P.xsum)) & 15) == 0;
+            uint32_t nmax = 0;
+            for (int64_t g = gtid; (g << 3) < d; g += gnth) {
+                const int64_t i0 = g << 3;
+                const bool whole = al16 && i0 + 8 <= d;
+                float cur[8], gf[8], xs[8], sm[8], acc[8];
+                float* tgt = ACC ? P.y : P.x;
+                if (whole) {
+                    small_load8_cg(tgt + i0, cur); small_load8_ro(P.gfull + i0, gf);
+                    if (ACC) { small_load8_ro(P.xsnap + i0, xs); small_load8_cg(P.xsum + i0, sm); }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const bool in = i0 + j < d;
+                        cur[j] = in ? __ldcg(tgt + i0 + j) : 0.0f; gf[j] = in ? P.gfull[i0 + j] : 0.0f;
+                        if (ACC) { xs[j] = in ? P.xsnap[i0 + j] : 0.0f; sm[j] = in ? __ldcg(P.xsum + i0 + j) : 0.0f; }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) { acc[j] = 0.0f; if (!ACC) { xs[j] = 0.0f; sm[j] = 0.0f; } }
+                // the group's codes are b bytes of every message
+                for (int w0 = 0; w0 < M; w0 += 4) {
+                    uint64_t cw[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint8_t* src = P.codes + (int64_t)min(w0 + k, M - 1) * P.stride + g * b;
+                        cw[k] = b == 8 ? (uint64_t)__ldcg(reinterpret_cast<const unsigned long long*>(src))
+                              : b == 4 ? (uint64_t)__ldcg(reinterpret_cast<const uint32_t*>(src))
+                                       : (uint64_t)__ldcg(reinterpret_cast<const unsigned short*>(src));
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        if (w0 + k < M) {
+                            const float sc = s_scale[w0 + k];
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const int code = (int)((int64_t)(cw[k] << (64 - b * (j + 1))) >> (64 - b));
+                                acc[j] = __fmaf_rn((float)code, sc, acc[j]);
+                            }
+                        }
+                    }
+                }
+                float xo[8], yo[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    xo[j] = master_update<ACC>(acc[j], inv_m, P.eta, P.theta, thr, den, P.pp, gf[j], cur[j], xs[j], yo[j], sm[j]);
+                    if (i0 + j < d) nmax = max(nmax, __float_as_uint(xo[j]) & 0x7FFFFFFFu);
+                }
+                if (whole) {
+                    small_store8(P.x + i0, xo);
+                    if (ACC) { small_store8(P.y + i0, yo); small_store8(P.xsum + i0, sm); }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (i0 + j < d) { P.x[i0 + j] = xo[j]; if (ACC) { P.y[i0 + j] = yo[j]; P.xsum[i0 + j] = sm[j]; } }
+                    }
+                }
+            }
+            nmax = small_block_max(nmax, s_red);
+            if (threadIdx.x == 0 && nmax != 0u) atomicMax(P.xnorm2 + (it & 1), nmax);
+            if (gtid == 0 && P.bits_down) {
+                const BitsArgs ba = {P.bits_down, P.bits_up, nullptr, 0, 0, P.bx, P.b, nullptr};
+                write_round_bits(ba, M, d);
+            }
+        }
+        cluster_barrier();
+    }
+    if (gtid == 0 && P.nrounds > 0) *P.normx = __ldcg(P.xnorm2 + ((P.nrounds - 1) & 1));
+}
+
+// ---------------------------------------------------------------------------------------------------
 // Host launchers
 // ---------------------------------------------------------------------------------------------------
 static inline int blocks_for(int64_t threads_needed, int sm_count, int per_sm = 8)
@@ -809,6 +1089,73 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
     ctx->launches += 1;
     if (list) { launch_build_group_list(ctx, reinterpret_cast<uint32_t*>(norm_inf), st); ctx->list_ready = true; }
     else launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
+}
+
+// ---- whole rounds in one cluster kernel ---------------------------------------------------------------------
+typedef void (*SmallRoundKernel)(const SmallRound, const PhiloxKeys);
+
+static SmallRoundKernel small_round_kernel_for(const dq_ctx* ctx)
+{
+    const bool csr = ctx->data.format == DQ_CSR_F32, acc = ctx->cfg.accelerated != 0;
+    if (csr) return acc ? round_cluster_kernel<DQ_CSR_F32, true> : round_cluster_kernel<DQ_CSR_F32, false>;
+    return acc ? round_cluster_kernel<DQ_DENSE_F32, true> : round_cluster_kernel<DQ_DENSE_F32, false>;
+}
+
+static void small_round_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int blocks, size_t smem, cudaStream_t st)
+{
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)blocks; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    *cfg = cudaLaunchConfig_t{};
+    cfg->gridDim = dim3((unsigned)blocks); cfg->blockDim = dim3(kSmallThreads); cfg->dynamicSmemBytes = smem; cfg->stream = st;
+    cfg->attrs = attr; cfg->numAttrs = 2;
+}
+
+static size_t small_round_smem(const dq_ctx* ctx) { return sizeof(float) * 2 * (size_t)small_round_pad(ctx->cfg.d); }
+
+// Decides once per context whether its rounds can run in the cluster kernel: logistic model on dense fp32 or CSR
+// data, dense messages, synchronous master, fixed model width, one block per worker (M <= 16, the largest
+// cluster), and a model of at most 8192 coordinates.
+void small_round_setup(dq_ctx* ctx)
+{
+    ctx->cluster_blocks = 0;
+    const dq_config& c = ctx->cfg;
+    if (!ctx->has_data || c.no_fused || c.model != DQ_MODEL_LOGISTIC || c.sparsify || c.sequential || c.mu > 0.0f) return;
+    if (ctx->data.format != DQ_DENSE_F32 && ctx->data.format != DQ_CSR_F32) return;
+    // beyond about one group of eight coordinates per thread the stages stop being latency-bound and one
+    // block per worker is slower than the whole GPU working through separate kernels
+    if (c.M > 16 || c.B > 1024 || c.d > 8 * kSmallThreads || small_round_smem(ctx) > 200 * 1024) return;
+    SmallRoundKernel kern = small_round_kernel_for(ctx);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)small_round_smem(ctx)) != cudaSuccess ||
+        (c.M > 8 && cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)) { cudaGetLastError(); return; }
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
+    small_round_config(&cfg, attr, c.M, small_round_smem(ctx), nullptr);
+    int nclusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&nclusters, kern, &cfg) == cudaSuccess && nclusters >= 1) ctx->cluster_blocks = c.M;
+    else cudaGetLastError();
+}
+
+void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds, float eta, float theta, uint64_t* bits_down,
+                          uint64_t* bits_up, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    SmallRound P;
+    P.values = (const float*)D.values; P.col = D.col_idx; P.row_ptr = D.row_ptr; P.labels = D.labels; P.n = D.n;
+    P.d = c.d; P.M = c.M; P.B = c.B; P.bx = c.bx; P.b = c.b; P.pp = ProxParams{c.lambda1, c.lambda2, c.box_lo, c.box_hi};
+    P.x = s->x; P.y = s->y; P.xsum = s->x_sum; P.xsnap = s->x_snap; P.gfull = s->g_full; P.zsnap = s->z_snap;
+    P.normx = reinterpret_cast<uint32_t*>(s->norm_x);
+    P.alpha = ctx->alpha; P.ninf = reinterpret_cast<uint32_t*>(ctx->ninf); P.rows = ctx->rows;
+    P.codes_x = ctx->codes_x; P.delta_x = ctx->delta_x; P.xnorm2 = ctx->xnorm_bits;
+    P.codes = ctx->msgs.codes; P.stride = ctx->msgs.stride; P.scale = ctx->msgs.scale;
+    P.bits_down = (bits_down || bits_up) ? (bits_down ? bits_down : ctx->bits) : nullptr;
+    P.bits_up = bits_up ? bits_up : ctx->bits + 1;
+    P.status = ctx->status;
+    P.round0 = round0; P.nrounds = nrounds; P.eta = eta; P.theta = theta;
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
+    small_round_config(&cfg, attr, ctx->cluster_blocks, small_round_smem(ctx), st);
+    cudaLaunchKernelEx(&cfg, small_round_kernel_for(ctx), P, ctx->keys);
+    ctx->launches += 1;
 }
 
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)

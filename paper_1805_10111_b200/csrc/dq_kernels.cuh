@@ -26,6 +26,9 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st);
 void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot, const dq_state* s,
                         uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st);
 bool worker_accumulates(const dq_ctx* ctx);
+void small_round_setup(dq_ctx* ctx);
+void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds, float eta, float theta, uint64_t* bits_down,
+                          uint64_t* bits_up, cudaStream_t st);
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st);
 void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st);
 void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* nnz, uint64_t* bits_down,

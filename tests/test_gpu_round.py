@@ -321,6 +321,10 @@ class Lockstep:
     ("bf16", dict(M=4, B=16, bx=8, b=8, box_lo=-1.0, box_hi=1.0, seed=7), 0.01),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, seed=8), 0.5),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=50.0, msg_format=1, seed=9), 0.5),
+    # the first two again as separate kernels (by default such small problems run in the one-cluster kernel)
+    ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=5, no_fused=1), 0.5),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=6, no_fused=1), 0.5),
+    ("dense8", dict(M=5, B=24, bx=4, b=2, lambda1=1e-4, lambda2=1e-3, box_lo=-0.5, box_hi=0.5, seed=10), 0.5),
 ])
 def test_lockstep_small(dq, name, kw, eta):
     h = _problem(name)
@@ -412,7 +416,7 @@ def test_lockstep_sequential_master(dq, name, kw):
 
 
 @pytest.mark.parametrize("name,kw", [
-    ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=21)),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=21, no_fused=1)),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=22)),
     ("bf16", dict(M=3, B=70, bx=8, b=8, box_lo=-1.0, box_hi=1.0, accelerated=1, seed=23)),
 ])
@@ -449,6 +453,51 @@ def test_graph_replay_equals_direct_launches(dq, name, kw):
     assert np.array_equal(outs[0][2], outs[1][2]) or name != "bf16"
 
 
+@pytest.mark.parametrize("name,kw", [
+    ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=31)),
+    ("dense8", dict(M=4, B=16, bx=8, b=4, lambda2=1e-4, accelerated=1, seed=32)),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=33)),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, seed=34)),
+])
+def test_rounds_in_one_call_equal_single_rounds(dq, name, kw):
+    """dq_rounds(n) must leave what n calls of dq_round leave.  The first three problems run in the one-cluster
+    kernel (one launch for all rounds after the snapshot round); the sparsified one takes the general path.  Dense
+    gradients are summed in a fixed order, so those runs agree bit for bit; CSR gradients use float atomics."""
+    import torch
+    h = _problem(name)
+    data = dq.Data(h)
+    x0 = synth.normal_vector(h.d, 84, 0.05)
+    acc = bool(kw.get("accelerated", 0))
+    theta, eta = (0.5, 0.05) if acc else (0.0, 0.3)
+    outs = []
+    for batched in (0, 1):
+        cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
+        rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+        st = dq.State(x0, n=h.n, accelerated=acc)
+        bits = torch.zeros(2, dtype=torch.int64, device="cuda")
+        rnd = 0
+        for epoch in range(2):
+            assert dq.dq_epoch_begin(ctx, st, theta) == 0
+            if batched:
+                l0 = dq.dq_launch_count(ctx)
+                assert dq.dq_rounds(ctx, st, rnd, 7, eta, theta, bits[0:1], bits[1:2]) == 0
+                if not kw.get("sparsify") and not (acc and epoch > 0):
+                    assert dq.dq_launch_count(ctx) - l0 < 7 + 6        # a snapshot round by kernels, then one launch
+                rnd += 7
+            else:
+                for t in range(7):
+                    assert dq.dq_round(ctx, st, rnd, eta, theta, bits[0:1], bits[1:2]) == 0
+                    rnd += 1
+        assert dq.dq_poll_status(ctx) == (0, 0)
+        outs.append((st.x.cpu().numpy().copy(), st.norm_x.item(), bits.cpu().numpy().copy()))
+        dq.dq_destroy(ctx)
+    if name != "csr":
+        assert np.array_equal(outs[0][0], outs[1][0]) and outs[0][1] == outs[1][1]
+    else:
+        assert np.allclose(outs[0][0], outs[1][0], rtol=1e-4, atol=1e-6)
+    assert np.array_equal(outs[0][2], outs[1][2])
+
+
 def test_select_model_bits_standalone(dq):
     import torch
     d = 100003
@@ -477,12 +526,14 @@ def _full_config(name):
         return dict(M=32, B=256, bx=8, b=8, box_lo=-10.0, box_hi=10.0, accelerated=1, seed=104), 1e-4, 10
 
 
-@pytest.mark.parametrize("name,rounds", [("c1", 100), ("c2", 100), ("c3", 4), ("c4", 20)])
-def test_lockstep_full_configs(dq, name, rounds):
+@pytest.mark.parametrize("name,rounds,no_fused", [("c1", 100, 0), ("c2", 100, 0), ("c1", 30, 1), ("c2", 30, 1), ("c3", 4, 0), ("c4", 20, 0)])
+def test_lockstep_full_configs(dq, name, rounds, no_fused):
     """The benchmark configurations at their full model width (c3, c4 with fewer rows so that the oracle
-    finishes in seconds); c4 reads "momentum 0.9" as theta = 0.1, eta = lr / theta."""
+    finishes in seconds); c4 reads "momentum 0.9" as theta = 0.1, eta = lr / theta.  c1 and c2 run in the
+    one-cluster kernel by default and once more as separate kernels."""
     h = _problem(name)
     kw, lr, m = _full_config(name)
+    kw = dict(kw, no_fused=no_fused)
     ls = Lockstep(dq, h, np.zeros(h.d, F32) if name != "c4" else synth.normal_vector(h.d, 75, 0.01), **kw)
     theta = F32(0.1) if name == "c4" else F32(0.0)
     eta = F32(lr) / theta if name == "c4" else F32(lr)
