@@ -358,8 +358,10 @@ def run_ours(a):
         return
     peak, peak_src = measured_peak()
     # algorithmic bytes per launch: norm 4 B, quantise+pack 4 + b/8 B per message
-    # coordinate; master M*b/8 + 12 B, model quantise 4 + b_x/8 B per model coordinate.
-    alg = [M * d * 4.0, M * d * (4.0 + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
+    # coordinate (8 + b/8 when sparsifying); master M*b/8 + 12 B, model quantise 4 + b_x/8 B per model coordinate.
+    # With sparsification the quantise stage is two passes over the vectors (||v||_1, which Lemma 2's probabilities
+    # need before the first mask bit can be drawn, then the mask pass that stages the survivors) plus the packed output.
+    alg = [M * d * 4.0, M * d * ((8.0 if a.sparsify else 4.0) + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
     names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
     stages = {n: {"ms": round(ms, 4), "alg_GBps": round(by / ms / 1e6, 1), "frac_of_peak": round(by / ms / 1e6 / peak, 4)}
               for n, ms, by in zip(names, stage_ms, alg)}
@@ -367,7 +369,7 @@ def run_ours(a):
                                               "frac_of_peak": round(d * 8.0 / select_ms / 1e6 / peak, 4)}
     qp = stages["quantize_pack"]
     tr = recorded_traffic(b) if not a.sparsify else None
-    roofline = {"kernel": "quantize_pack_kernel<%d>" % b if not a.sparsify else "sparsify (l1 + count + emit)",
+    roofline = {"kernel": "quantize_pack_kernel<%d>" % b if not a.sparsify else "norm_l1_kernel + sparsify_stage_kernel + sparsify_scatter_dense_kernel<%d>" % b,
                 "bound": "hbm", "achieved": qp["alg_GBps"], "peak": peak, "unit": "GB/s",
                 "frac": round(qp["alg_GBps"] / peak, 4), "peak_source": peak_src,
                 "traffic": None if tr is None else tr * M * d,
