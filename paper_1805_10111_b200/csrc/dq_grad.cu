@@ -504,7 +504,7 @@ __global__ void bits_kernel(int M, int64_t d, int bx, int b, int flag_round, int
 // cross-entropy.  Parameters x = [W1 (hidden x in, row-major), b1, W2 (classes x hidden), b2]; labels hold class
 // indices.  The worker needs grad f_B(xhat) - grad f_B(xsnap): three small kernels evaluate both parameter
 // vectors side by side (either may be absent: NULL), rows listed explicitly or drawn from the batch stream.
-//   mlp_hidden_kernel   block per sampled row: hidden activations (one warp per hidden unit, coalesced along in)
+//   mlp_hidden_kernel   block per tile of sampled rows and eight hidden units: hidden activations (one warp per unit, coalesced along in)
 //   mlp_output_kernel   block per sampled row: logits, softmax, d loss / d logits, d loss / d hidden (ReLU-gated)
 //   mlp_param_kernel    block per (hidden unit or the tail, worker): sums over the worker's rows, no atomics
 // ---------------------------------------------------------------------------------------------------
@@ -514,36 +514,60 @@ __device__ __forceinline__ int64_t mlp_off_b1(const MlpShape& s) { return (int64
 __device__ __forceinline__ int64_t mlp_off_w2(const MlpShape& s) { return mlp_off_b1(s) + s.hidden; }
 __device__ __forceinline__ int64_t mlp_off_b2(const MlpShape& s) { return mlp_off_w2(s) + (int64_t)s.classes * s.hidden; }
 
+constexpr int kMlpUnits = 8;         // hidden units whose first-layer gradients one block forms from the same rows
+constexpr int kMlpTile = 8;          // sampled rows that share one pass over a hidden unit's weights
+
+// grid (ceil(nslots / kMlpTile), ceil(hidden / 8)): a block holds kMlpTile rows in shared memory and each of its
+// eight warps owns one hidden unit, so a weight row is read once for the whole tile (a block per row would read the
+// first layer once per sample).  Per row the sum runs in the same order as before: lanes stride over the inputs,
+// then a butterfly across lanes.
 __global__ void __launch_bounds__(kThreads)
 mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restrict__ xa, const float* __restrict__ xb,
                   const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
-                  float* __restrict__ act_a, float* __restrict__ act_b)
+                  float* __restrict__ act_a, float* __restrict__ act_b, int64_t nslots)
 {
     pdl_prologue();
-    extern __shared__ float s_in[];                      // the row's features
-    __shared__ int64_t s_row;
+    extern __shared__ float s_in[];                      // [kMlpTile][in] features of the tile's rows
+    __shared__ int64_t s_row[kMlpTile];
     clear_word(bs);
-    const int64_t slot = blockIdx.x;
+    const int64_t slot0 = (int64_t)blockIdx.x * kMlpTile;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) {
-        const int64_t a = B > 0 ? batch_row(bs, K, (int)(slot / B), (int)(slot % B), B, true) : slot;   // B = 0: row = slot
-        s_row = a; if (row_of_slot) row_of_slot[slot] = (int32_t)a;
+    if (threadIdx.x < kMlpTile) {
+        const int64_t slot = slot0 + threadIdx.x;
+        int64_t a = -1;
+        if (slot < nslots) {
+            a = B > 0 ? batch_row(bs, K, (int)(slot / B), (int)(slot % B), B, blockIdx.y == 0) : slot;   // B = 0: row = slot
+            if (row_of_slot && blockIdx.y == 0) row_of_slot[slot] = (int32_t)a;
+        }
+        s_row[threadIdx.x] = a;
     }
     __syncthreads();
-    const float* row = X + s_row * sh.in;
-    for (int64_t i = threadIdx.x; i < sh.in; i += blockDim.x) s_in[i] = row[i];
+    for (int64_t q = threadIdx.x; q < (int64_t)kMlpTile * sh.in; q += blockDim.x) {
+        const int t = (int)(q / sh.in); const int64_t i = q - (int64_t)t * sh.in;
+        s_in[q] = s_row[t] >= 0 ? X[s_row[t] * sh.in + i] : 0.0f;
+    }
     __syncthreads();
-    for (int j = warp; j < sh.hidden; j += kThreads / 32) {
-        float sa = 0.0f, sb = 0.0f;
-        for (int64_t i = lane; i < sh.in; i += 32) {
-            const float f = s_in[i];
-            if (xa) sa = fmaf(xa[(int64_t)j * sh.in + i], f, sa);
-            if (xb) sb = fmaf(xb[(int64_t)j * sh.in + i], f, sb);
+    const int j = blockIdx.y * (kThreads / 32) + warp;
+    if (j >= sh.hidden) return;
+    float sa[kMlpTile], sb[kMlpTile];
+#pragma unroll
+    for (int t = 0; t < kMlpTile; ++t) { sa[t] = 0.0f; sb[t] = 0.0f; }
+#pragma unroll 2
+    for (int64_t i = lane; i < sh.in; i += 32) {
+        const float wa = xa ? xa[(int64_t)j * sh.in + i] : 0.0f, wb = xb ? xb[(int64_t)j * sh.in + i] : 0.0f;
+#pragma unroll
+        for (int t = 0; t < kMlpTile; ++t) {
+            const float f = s_in[(int64_t)t * sh.in + i];
+            sa[t] = fmaf(wa, f, sa[t]); sb[t] = fmaf(wb, f, sb[t]);
         }
-        sa = warp_sum(sa); sb = warp_sum(sb);
-        if (lane == 0) {
-            if (xa) act_a[slot * sh.hidden + j] = fmaxf(sa + xa[mlp_off_b1(sh) + j], 0.0f);
-            if (xb) act_b[slot * sh.hidden + j] = fmaxf(sb + xb[mlp_off_b1(sh) + j], 0.0f);
+    }
+    const float ba = xa ? xa[mlp_off_b1(sh) + j] : 0.0f, bb = xb ? xb[mlp_off_b1(sh) + j] : 0.0f;
+#pragma unroll
+    for (int t = 0; t < kMlpTile; ++t) {
+        const float va = warp_sum(sa[t]), vb = warp_sum(sb[t]);
+        if (lane == 0 && slot0 + t < nslots) {
+            if (xa) act_a[(slot0 + t) * sh.hidden + j] = fmaxf(va + ba, 0.0f);
+            if (xb) act_b[(slot0 + t) * sh.hidden + j] = fmaxf(vb + bb, 0.0f);
         }
     }
 }
@@ -613,28 +637,42 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
 {
     pdl_prologue();
     typedef typename std::conditional<FULL, double, float>::type acc_t;
-    extern __shared__ float s_w[];                       // per row of the group: dh_a[j] - handled below
-    const int j = blockIdx.x, w = blockIdx.y;
+    extern __shared__ float s_w[];                       // [kMlpUnits][B] slope differences, then [B] row indices
+    const int j0 = blockIdx.x * kMlpUnits, w = blockIdx.y;     // the block after the last tile of hidden units does W2, b2
     const int64_t r0 = (int64_t)w * B;
     const int nrows = (int)min((int64_t)B, total_rows - r0);
     uint32_t nmax = 0;
     float* o = FULL ? nullptr : out + (int64_t)w * P;
-    if (j < sh.hidden) {
-        // s_w[r] = dh_a[r][j], s_w[B + r] = dh_b[r][j]
-        for (int r = threadIdx.x; r < nrows; r += blockDim.x) {
-            s_w[r] = dh_a ? dh_a[(r0 + r) * sh.hidden + j] : 0.0f;
-            s_w[B + r] = dh_b ? dh_b[(r0 + r) * sh.hidden + j] : 0.0f;
+    if (j0 < sh.hidden) {
+        // s_w[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u]; the rows' indices sit behind them: no dependent load in the loop.
+        // The block's hidden units share every feature value that a thread loads.
+        int* s_rowid = reinterpret_cast<int*>(s_w + kMlpUnits * B);
+        for (int q = threadIdx.x; q < kMlpUnits * nrows; q += blockDim.x) {
+            const int u = q / nrows, r = q - u * nrows, j = j0 + u;
+            const float da = (dh_a && j < sh.hidden) ? dh_a[(r0 + r) * sh.hidden + j] : 0.0f;
+            const float db = (dh_b && j < sh.hidden) ? dh_b[(r0 + r) * sh.hidden + j] : 0.0f;
+            s_w[u * B + r] = da - db;
         }
+        for (int r = threadIdx.x; r < nrows; r += blockDim.x) s_rowid[r] = row_of_slot[r0 + r];
         __syncthreads();
         for (int64_t i = threadIdx.x; i <= sh.in; i += blockDim.x) {       // i == in: the bias b1[j]
-            acc_t s = 0;
+            acc_t s[kMlpUnits];
+#pragma unroll
+            for (int u = 0; u < kMlpUnits; ++u) s[u] = 0;
+#pragma unroll 4
             for (int r = 0; r < nrows; ++r) {
-                const float f = (i < sh.in) ? X[(int64_t)row_of_slot[r0 + r] * sh.in + i] : 1.0f;
-                s += (acc_t)((s_w[r] - s_w[B + r]) * f);
+                const float f = (i < sh.in) ? X[(int64_t)s_rowid[r] * sh.in + i] : 1.0f;
+#pragma unroll
+                for (int u = 0; u < kMlpUnits; ++u) s[u] += (acc_t)(s_w[u * B + r] * f);
             }
-            const int64_t pidx = (i < sh.in) ? (int64_t)j * sh.in + i : mlp_off_b1(sh) + j;
-            if (FULL) atomicAdd(g64 + pidx, (double)s);
-            else { o[pidx] = (float)s; nmax = max(nmax, __float_as_uint((float)s) & 0x7FFFFFFFu); }
+#pragma unroll
+            for (int u = 0; u < kMlpUnits; ++u) {
+                const int j = j0 + u;
+                if (j >= sh.hidden) break;
+                const int64_t pidx = (i < sh.in) ? (int64_t)j * sh.in + i : mlp_off_b1(sh) + j;
+                if (FULL) atomicAdd(g64 + pidx, (double)s[u]);
+                else { o[pidx] = (float)s[u]; nmax = max(nmax, __float_as_uint((float)s[u]) & 0x7FFFFFFFu); }
+            }
         }
     } else {
         const int nout = sh.classes * (sh.hidden + 1);                       // W2 entries then b2
@@ -948,6 +986,10 @@ static inline int blocks_for(int64_t threads_needed, int sm_count, int per_sm = 
 
 // ---- network launchers ------------------------------------------------------------------------------------
 static MlpShape mlp_shape(const dq_ctx* ctx) { return MlpShape{ctx->data.d, ctx->cfg.hidden, ctx->cfg.classes}; }
+static dim3 mlp_hidden_grid(int64_t nslots, const MlpShape& sh)
+{
+    return dim3((unsigned)((nslots + kMlpTile - 1) / kMlpTile), (unsigned)((sh.hidden + kThreads / 32 - 1) / (kThreads / 32)));
+}
 constexpr int kMlpGroup = 256;      // rows per block of the epoch-gradient sums
 
 // g <- (1/n) sum_i grad loss_i(x) over all rows (double sums), via the "a" slots of the activation buffers.
@@ -956,13 +998,13 @@ static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStre
     const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
     const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
     const int64_t P = ctx->cfg.d;
-    launch_k(mlp_hidden_kernel, (unsigned)D.n, kThreads, sizeof(float) * sh.in, st, (const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
-                                                                             ctx->mlp_rows, ctx->mlp_act[0], nullptr);
+    launch_k(mlp_hidden_kernel, mlp_hidden_grid(D.n, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
+                                                                             ctx->mlp_rows, ctx->mlp_act[0], nullptr, (int64_t)D.n);
     launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
         nullptr, (float)(1.0 / (double)D.n), ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr);
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * P, st);
-    dim3 grid(sh.hidden + 1, (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
-    launch_k(mlp_param_kernel<true>, grid, kThreads, sizeof(float) * 2 * kMlpGroup, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
+    dim3 grid((sh.hidden + kMlpUnits - 1) / kMlpUnits + 1, (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
+    launch_k(mlp_param_kernel<true>, grid, kThreads, sizeof(float) * (kMlpUnits + 1) * kMlpGroup, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
         ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
     launch_k(finish_full_grad_kernel, blocks_for(P, ctx->sm_count), kThreads, 0, st, ctx->g64, P, 1.0, g);
     ctx->launches += 4;
@@ -975,13 +1017,13 @@ static void launch_mlp_worker_grad(dq_ctx* ctx, const float* xhat, const dq_stat
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
     const unsigned R = (unsigned)(c.M * c.B);
     uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
-    launch_k(mlp_hidden_kernel, R, kThreads, sizeof(float) * sh.in, st, (const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
-                                                                   ctx->mlp_act[0], ctx->mlp_act[1]);
+    launch_k(mlp_hidden_kernel, mlp_hidden_grid(R, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
+                                                                   ctx->mlp_act[0], ctx->mlp_act[1], (int64_t)R);
     launch_k(mlp_output_kernel, R, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
         ctx->mlp_act[1], 1.0f / (float)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr);
     if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
-    dim3 grid(sh.hidden + 1, c.M);
-    launch_k(mlp_param_kernel<false>, grid, kThreads, sizeof(float) * 2 * c.B, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
+    dim3 grid((sh.hidden + kMlpUnits - 1) / kMlpUnits + 1, c.M);
+    launch_k(mlp_param_kernel<false>, grid, kThreads, sizeof(float) * (kMlpUnits + 1) * c.B, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
         ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
     ctx->launches += 3;
 }
@@ -1165,8 +1207,8 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
     if (c.model == DQ_MODEL_MLP) {
         const MlpShape sh = mlp_shape(ctx);
         const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
-        launch_k(mlp_hidden_kernel, (unsigned)D.n, kThreads, sizeof(float) * sh.in, st, (const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
-                                                                                 ctx->mlp_rows, nullptr, ctx->mlp_act[1]);
+        launch_k(mlp_hidden_kernel, mlp_hidden_grid(D.n, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
+                                                                                 ctx->mlp_rows, nullptr, ctx->mlp_act[1], (int64_t)D.n);
         launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
             ctx->mlp_act[1], (float)(1.0 / (double)D.n), nullptr, nullptr, nullptr, nullptr, P);
         launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
