@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--sequential", type=int, default=0, help="1: master applies one prox step per message")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="time the codec stages over d in {2^20,2^24,2^27} x b in {2,4,8} x sparsify off/on "
+                                                         "and print one JSON object with all points instead of the bench line")
     ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_round ('' for none)")
     return ap.parse_args()
 
@@ -392,10 +394,72 @@ def run_ours(a):
         dist.destroy_process_group()
 
 
+# ---------------------------------------------------------------------------------------------------------------
+# the quantiser/packer sweep of the c5 configuration (stage times only; inputs are drawn on the device)
+# ---------------------------------------------------------------------------------------------------------------
+def run_sweep(a):
+    import torch
+    import paper_1805_10111_b200 as dq
+    torch.cuda.set_device(0)
+    dq.lib()
+    peak, peak_src = measured_peak()
+    M, bx, eta = a.workers, 8, 0.1
+    points = []
+    for log2d in (20, 24, 27):
+        d = 1 << log2d
+        g = torch.Generator(device="cuda"); g.manual_seed(180510111 + log2d)
+        v = torch.randn((M, d), device="cuda", generator=g)
+        idx = torch.randint(0, d, (M, max(1, d // 1000)), device="cuda", generator=g)
+        v.scatter_(1, idx, v.gather(1, idx) * 100.0)                      # 0.1 % outliers x100
+        x0 = torch.randn(d, device="cuda", generator=g); gf = torch.randn(d, device="cuda", generator=g)
+        # at d = 2^20 one set of inputs (36 MiB) would sit in L2: rotate over enough copies to exceed it
+        copies = max(1, (256 << 20) // (M * d * 4))
+        vs = [v] + [v.clone() for _ in range(copies - 1)]
+        for sparsify in (0, 1):
+            for b in (2, 4, 8):
+                cfg = dq.make_config(d, M, b=b, bx=bx, seed=1805, lambda1=1e-6, sparsify=sparsify, phi=0.01 * d if sparsify else 0.0)
+                rc, ctx = dq.dq_create(cfg); dq.ok(rc, "dq_create")
+                st = dq.State(x0); st.g_full.copy_(gf)
+                msgs = dq.Msgs(cfg)
+                ninf = torch.zeros(M, device="cuda")
+                nbx = dq.dq_packed_bytes(d, bx)
+                codes_x = torch.zeros(nbx, dtype=torch.uint8, device="cuda"); delta_x = torch.zeros(1, device="cuda")
+                steps = 200 if log2d <= 20 else (60 if log2d <= 24 else 20)
+                ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+                for k in range(-3, steps):
+                    vk = vs[k % copies]
+                    e = ev[k] if k >= 0 else None
+                    if e: e[0].record()
+                    dq.ok(dq.dq_norm_inf(ctx, vk, M, ninf))
+                    if e: e[1].record()
+                    dq.ok(dq.dq_quantize_sparsify_pack(ctx, vk, ninf, 1000 + k, msgs))
+                    if e: e[2].record()
+                    dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta))
+                    if e: e[3].record()
+                    dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, 1000 + k, codes_x, delta_x))
+                    if e: e[4].record()
+                torch.cuda.synchronize()
+                rc, status = dq.dq_poll_status(ctx); assert rc == 0 and status == 0
+                ms = [sorted(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(steps))[steps // 2] for i in range(4)]   # medians
+                alg = [M * d * 4.0, M * d * ((8.0 if sparsify else 4.0) + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
+                names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
+                points.append({"log2d": log2d, "b": b, "sparsify": sparsify, "rounds_per_s": round(1000.0 / sum(ms), 1),
+                               "stages": {n: {"ms": round(t, 4), "alg_GBps": round(by / t / 1e6, 1), "frac_of_peak": round(by / t / 1e6 / peak, 3)}
+                                          for n, t, by in zip(names, ms, alg)}})
+                dq.dq_destroy(ctx)
+                del st, msgs
+        del v, vs, x0, gf
+        torch.cuda.empty_cache()
+    print(json.dumps({"sweep": "c5 quantiser/packer: M=%d, b_x=8, lambda1=1e-6, eta=0.1, phi=0.01d when sparsifying" % M,
+                      "peak_GBps": peak, "peak_source": peak_src, "l2_policy": "inputs rotated over >= 256 MiB", "points": points}))
+
+
 def main():
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.sweep:
+        run_sweep(a)
     else:
         run_ours(a)
 

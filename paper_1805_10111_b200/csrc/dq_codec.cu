@@ -692,7 +692,7 @@ __device__ __forceinline__ void accumulate_word(uint32_t word, float dl, float (
 
 // Dense messages.  Each thread owns the 32/BITS coordinates of one 32-bit code word per worker.
 template <int BITS, bool ACC>
-__global__ void __launch_bounds__(kThreads, BITS == 2 ? 3 : 4)
+__global__ void __launch_bounds__(kThreads, 4)
 master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
                     const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
@@ -721,7 +721,8 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
         const int64_t i0 = t * C;
         const bool fast = C >= 8 && vec8_ok && i0 + C <= d;
         float gfp[C >= 8 ? C : 8], curp[C >= 8 ? C : 8];     // issued before the code words so that all loads overlap
-        if (fast) {
+        constexpr bool kEarly = BITS != 2;                   // sixteen coordinates per thread: loading early costs a block per SM
+        if (fast && kEarly) {
 #pragma unroll
             for (int q = 0; q < C / 8; ++q) {
                 load8(g_full + i0 + q * 8, *reinterpret_cast<float(*)[8]>(gfp + q * 8));
@@ -773,6 +774,13 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
             }
         }
         float* target = ACC ? y : x;
+        if (fast && !kEarly) {
+#pragma unroll
+            for (int q = 0; q < C / 8; ++q) {
+                load8(g_full + i0 + q * 8, *reinterpret_cast<float(*)[8]>(gfp + q * 8));
+                load8_rw((ACC ? y : x) + i0 + q * 8, *reinterpret_cast<float(*)[8]>(curp + q * 8));
+            }
+        }
         if (fast) {                                          // 256-bit accesses: every 32-byte sector is used whole
 #pragma unroll
             for (int q = 0; q < C / 8; ++q) {

@@ -78,3 +78,61 @@ def test_codec_round_at_bench_size_on_samples(log2d, b):
     want = [oracle.q_code(x_gpu[i], invx, bx, oracle.u15(seed, rnd, oracle.MASTER, oracle.STREAM_MODEL, int(i))) for i in sample]
     assert np.array_equal(cx, np.array(want, np.int32))
     dq.dq_destroy(ctx)
+
+
+@pytest.mark.parametrize("log2d,workers", [(24, range(8)), (27, (5,))])
+def test_sparsified_messages_at_bench_size(log2d, workers):
+    """The sparsified stage as bench.py --sparsify 1 launches it (M = 8, b = 4, phi = 0.01 d): the norm pass, the mask
+    pass that stages the survivors, and their placement, for both containers.  The oracle redoes whole vectors: all
+    eight at d = 2^24, one at d = 2^27 (about ten seconds each); the other messages are checked through properties
+    that hold at any size."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    import paper_1805_10111_b200 as dq
+    d, M, b, seed, rnd = 1 << log2d, 8, 4, 1805, 1004
+    phi = 0.01 * d
+    g = synth.rng(700 + log2d)
+    hv = torch.empty((M, d), dtype=torch.float32).pin_memory()
+    v = hv.numpy()
+    for w in range(M):
+        g.standard_normal(d, dtype=np.float32, out=v[w])
+        v[w][g.integers(0, d, d // 1000)] *= F32(100.0)
+    dv = hv.cuda()
+    want = {}
+    for w in workers:
+        r = oracle.sparsify(v[w], phi, seed, rnd, w)
+        codes, delta, rc = oracle.quantize_survivors(r["beta"], r["Z"], b, seed, rnd, w)
+        assert rc == 0 and r["status"] == 0
+        want[w] = (np.nonzero(r["Z"])[0], codes, delta)
+    L = 2 ** (b - 1) - 1
+    for fmt in (dq.DQ_MSG_DENSE, dq.DQ_MSG_SPARSE):
+        cfg = dq.make_config(d, M, b=b, bx=8, seed=seed, sparsify=1, phi=phi, msg_format=fmt, sparse_cap=d // 64)
+        rc, ctx = dq.dq_create(cfg); assert rc == 0
+        msgs = dq.Msgs(cfg, cap=d // 64); ninf = torch.zeros(M, device="cuda")
+        assert dq.dq_norm_inf(ctx, dv, M, ninf) == 0
+        assert dq.dq_quantize_sparsify_pack(ctx, dv, ninf, rnd, msgs) == 0
+        assert dq.dq_poll_status(ctx) == (0, 0)
+        scale = msgs.scale.cpu().numpy()
+        for w in range(M):
+            row = msgs.codes[w].cpu().numpy()
+            if fmt == dq.DQ_MSG_DENSE:
+                lo, hi = row & 0x0F, row >> 4                                        # two codes per byte at b = 4
+                nz = int(np.count_nonzero(lo) + np.count_nonzero(hi))
+                assert 0 < nz <= 0.004 * d                                           # realised density about 0.2 %
+                assert max(int(np.abs(_codes_at(row, np.flatnonzero(lo) * 2, b)).max()), 1) <= L
+            else:
+                n = int(msgs.nnz[w].item())
+                idx = msgs.idx[w, :n].cpu().numpy().astype(np.int64)
+                assert np.all(np.diff(idx) > 0) and idx[-1] < d                      # ascending, in range
+                assert not row[(n * b + 7) // 8:].any()                              # nothing behind the list
+            if w in want:
+                pos, codes, delta = want[w]
+                assert scale[w] == delta
+                if fmt == dq.DQ_MSG_DENSE:
+                    assert np.array_equal(row, oracle.pack(codes, b, msgs.stride))
+                else:
+                    assert n == pos.size and np.array_equal(idx, pos)
+                    assert np.array_equal(row, oracle.pack(codes[pos], b, msgs.stride))
+        dq.dq_destroy(ctx)
+        del msgs
