@@ -326,9 +326,9 @@ def expected_sq_error(x, b):
 
 
 def select_bx(x, xsnap, mu):
-    """Returns (chosen width, expected errors at 2/4/8 bits, ||x - xsnap||^2)."""
+    """Returns (chosen width, expected errors at 2..11 bits, ||x - xsnap||^2)."""
     x, xsnap = _f32(x), _f32(xsnap)
-    err = np.zeros(3, np.float64); dist = np.zeros(1, np.float64)
+    err = np.zeros(10, np.float64); dist = np.zeros(1, np.float64)
     b = lib().dqo_select_bx(_p(x), _p(xsnap), x.size, float(mu), _p(err), _p(dist))
     return int(b), err, float(dist[0])
 

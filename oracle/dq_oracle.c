@@ -117,21 +117,26 @@ float dqo_scale_inv(float nrm, int b)
 
 /* One coordinate.  t = v*inv is the position on the code axis; z = floor(t)
  * and z+1 are the neighbouring grid points and rule (i) rounds up with
- * probability t - z.  The position is held in fixed point with 15 fractional
- * bits: r = fl(v*inv + 384) lies in [256,512) where fp32 spacing is 2^-15, so
- * the integer F = bits(r) - bits(256.0f) equals (t + 128) * 2^15 with t rounded
- * to nearest at 2^-15 (one fused rounding).  Adding a uniform 15-bit integer
- * and dropping the fraction rounds up with probability frac(F)/2^15.  Rule (ii)
+ * probability t - z.  The position is held in fixed point: with e = 8 for
+ * b <= 8 and e = b for the wider codes (b = 9, 10, 11, the widths of Table 1
+ * beyond a byte), r = fl(v*inv + 1.5 * 2^e) lies in [2^e, 2^(e+1)) where the
+ * fp32 spacing is 2^-(23-e), so the integer F = bits(r) - bits(2^e) equals
+ * (t + 2^(e-1)) * 2^(23-e) with t rounded to nearest at 2^-(23-e) (one fused
+ * rounding): 15 fractional bits up to 8-bit codes, then 14, 13, 12.  Adding a
+ * uniform integer of as many bits (the top bits of the coordinate's draw) and
+ * dropping the fraction rounds up with probability frac(F)/2^(23-e).  Rule (ii)
  * (outside the hull: nearest end point of dom(delta,b)) is the clamp. */
 int32_t dqo_q_code(float v, float inv, int b, uint32_t u15)
 {
-    float r = fmaf(v, inv, 384.0f);
-    float lo = 384.0f - (float)(1 << (b - 1));                   /* -2^(b-1): smallest member of dom */
-    float hi = 384.0f + (float)levels(b);                        /* 2^(b-1)-1: largest member        */
+    const int e = b <= 8 ? 8 : b, fbits = 23 - e;
+    const float off = 1.5f * (float)(1 << e);
+    float r = fmaf(v, inv, off);
+    float lo = off - (float)(1 << (b - 1));                      /* -2^(b-1): smallest member of dom */
+    float hi = off + (float)levels(b);                           /* 2^(b-1)-1: largest member        */
     r = fminf(fmaxf(r, lo), hi);
     uint32_t bits; memcpy(&bits, &r, 4);
-    uint32_t F = bits - 0x43800000u;                             /* bits(256.0f) */
-    return (int32_t)((F + u15) >> 15) - 128;
+    uint32_t F = bits - ((uint32_t)(127 + e) << 23);             /* bits(2^e) */
+    return (int32_t)((F + (u15 >> (15 - fbits))) >> fbits) - (1 << (e - 1));
 }
 
 float dqo_norm_inf(const float* v, int64_t d)
@@ -153,7 +158,7 @@ static int all_finite(const float* v, int64_t d)
 int dqo_quantize(const float* v, int64_t d, int b, uint64_t seed, uint32_t round, uint32_t worker,
                  uint32_t stream, int32_t* codes, float* delta)
 {
-    if (b < 2 || b > 8 || d < 0) return DQO_ERR_ARG;
+    if (b < 2 || b > 11 || d < 0) return DQO_ERR_ARG;
     if (!all_finite(v, d)) return DQO_ERR_NONFINITE;
     float nrm = dqo_norm_inf(v, d);
     if (nrm == 0.0f) { *delta = 0.0f; for (int64_t i = 0; i < d; ++i) codes[i] = 0; return DQO_OK; }
@@ -166,24 +171,32 @@ int dqo_quantize(const float* v, int64_t d, int b, uint64_t seed, uint32_t round
 
 /* ------------------------------------------------------------------------ */
 /* Message encoding: Section 3.1 counts b bits per coordinate; the container */
-/* is this build's choice: b-bit two's complement, coordinate j in byte      */
-/* j / (8/b) at bit offset (j mod (8/b)) * b, unused bits zero.              */
+/* is this build's choice: the codes as b-bit two's complement fields laid    */
+/* end to end, coordinate j in bits [j b, (j+1) b) of the message, bit k of   */
+/* the message being bit k mod 8 of byte k / 8; unused bits zero.  (For b     */
+/* dividing 8: coordinate j in byte j/(8/b) at bit offset (j mod (8/b)) b.)   */
 /* ------------------------------------------------------------------------ */
 void dqo_pack(const int32_t* codes, int64_t count, int b, uint8_t* out, int64_t out_bytes)
 {
     memset(out, 0, (size_t)out_bytes);
-    int per = 8 / b;
     uint32_t mask = (1u << b) - 1u;
-    for (int64_t j = 0; j < count; ++j)
-        out[j / per] |= (uint8_t)(((uint32_t)codes[j] & mask) << ((j % per) * b));
+    for (int64_t j = 0; j < count; ++j) {
+        uint32_t field = (uint32_t)codes[j] & mask;
+        for (int k = 0; k < b; ++k) {
+            int64_t bit = j * b + k;
+            if ((field >> k) & 1u) out[bit >> 3] |= (uint8_t)(1u << (bit & 7));
+        }
+    }
 }
 
 void dqo_unpack(const uint8_t* in, int64_t count, int b, int32_t* codes)
 {
-    int per = 8 / b;
-    uint32_t mask = (1u << b) - 1u;
     for (int64_t j = 0; j < count; ++j) {
-        uint32_t u = ((uint32_t)in[j / per] >> ((j % per) * b)) & mask;
+        uint32_t u = 0;
+        for (int k = 0; k < b; ++k) {
+            int64_t bit = j * b + k;
+            u |= (uint32_t)((in[bit >> 3] >> (bit & 7)) & 1u) << k;
+        }
         codes[j] = (u & (1u << (b - 1))) ? (int32_t)u - (1 << b) : (int32_t)u;   /* sign extend */
     }
 }
@@ -574,7 +587,7 @@ void dqo_master_step_sequential(const int32_t* codes, const float* delta, int M,
 /* b_x so that it holds.  Under rule (i) a coordinate between the grid points */
 /* z and z + delta has expected squared error (x - z)(z + delta - x)          */
 /* (proof of the appendix's first lemma), so the left side is a closed form.  */
-/* This build packs 2, 4 or 8 bits; the search is over those widths.          */
+/* The search is over the widths 2..11 of Table 1.                            */
 /* ------------------------------------------------------------------------ */
 double dqo_expected_sq_error(const float* x, int64_t d, int b)
 {
@@ -595,17 +608,16 @@ double dqo_sq_distance(const float* x, const float* y, int64_t d)
     return s;
 }
 
-/* Smallest width in {2, 4, 8} that satisfies the condition; 8 when none does.
- * err[0..2] receive the expected errors at 2, 4, 8 bits, *dist2 the squared distance. */
+/* Smallest width in 2..11 (the widths of Table 1) that satisfies the condition; 11 when none does.
+ * err[0..9] receive the expected errors at 2..11 bits, *dist2 the squared distance. */
 int dqo_select_bx(const float* x, const float* xsnap, int64_t d, float mu, double* err, double* dist2)
 {
-    static const int widths[3] = { 2, 4, 8 };
     double D = dqo_sq_distance(x, xsnap, d);
-    int chosen = 8;
-    for (int k = 2; k >= 0; --k) {
-        double e = dqo_expected_sq_error(x, d, widths[k]);
-        if (err) err[k] = e;
-        if (e <= (double)mu * D) chosen = widths[k];
+    int chosen = 11;
+    for (int b = 11; b >= 2; --b) {
+        double e = dqo_expected_sq_error(x, d, b);
+        if (err) err[b - 2] = e;
+        if (e <= (double)mu * D) chosen = b;
     }
     if (dist2) *dist2 = D;
     return chosen;

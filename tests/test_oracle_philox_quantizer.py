@@ -93,10 +93,17 @@ def test_scales(b):
 # ---------------------------------------------------------------------------------------------------
 # Q: one coordinate, exact
 # ---------------------------------------------------------------------------------------------------
-def _exact_fixed_point(v, inv):
-    """(t+128)*2^15 rounded to nearest-even, from exact rationals."""
+def _fixed_point_shape(b):
+    """(offset 2^(e-1) on the code axis, fractional bits) of the fixed-point position: e = 8 up to 8-bit codes, else b."""
+    e = 8 if b <= 8 else b
+    return 1 << (e - 1), 23 - e
+
+
+def _exact_fixed_point(v, inv, b=8):
+    """(t + offset) * 2^fbits rounded to nearest-even, from exact rationals."""
+    off, fb = _fixed_point_shape(b)
     t = Fraction(float(v)) * Fraction(float(inv))
-    s = (t + 128) * (1 << 15)
+    s = (t + off) * (1 << fb)
     fl = s.numerator // s.denominator
     rem = s - fl
     if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
@@ -104,46 +111,49 @@ def _exact_fixed_point(v, inv):
     return fl, t
 
 
-@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("b", [2, 3, 4, 5, 6, 7, 8, 9, 10, 11])
 def test_q_code_is_stochastic_rounding_with_exact_probability(b):
-    """Rule (i): the code is floor(t) or floor(t)+1 and, over ALL 2^15 values of the uniform draw, it is
-    rounded up exactly frac*2^15 times, with frac the fractional part of t at 15-bit resolution."""
+    """Rule (i): the code is floor(t) or floor(t)+1 and, over ALL values of the uniform draw, it is rounded up
+    exactly frac*2^fbits times, with frac the fractional part of t at the fixed-point resolution (15 fractional
+    bits up to 8-bit codes, 14/13/12 for 9/10/11 bits; the draw's top bits are used)."""
     L = 2 ** (b - 1) - 1
+    off, fb = _fixed_point_shape(b)
     g = np.random.default_rng(100 + b)
     nrm = F32(3.7)
     inv = oracle.scale_inv(nrm, b)
     us = [0, 1, 2, 12345, (1 << 14), (1 << 15) - 2, (1 << 15) - 1]
     for v in list((g.uniform(-1, 1, 60) * float(nrm)).astype(F32)) + [nrm, -nrm, F32(0.0), F32(1e-30)]:
-        F, t = _exact_fixed_point(v, inv)
-        z = F >> 15                                                   # floor at 15-bit resolution, +128
-        frac = F & 0x7FFF
-        assert abs(Fraction(F, 1 << 15) - 128 - t) <= Fraction(1, 1 << 16)      # resolution of the position
+        F, t = _exact_fixed_point(v, inv, b)
+        z = F >> fb                                                   # floor at the fixed-point resolution, + offset
+        frac = F & ((1 << fb) - 1)
+        assert abs(Fraction(F, 1 << fb) - off - t) <= Fraction(1, 1 << (fb + 1))      # resolution of the position
         for u in us:
             k = oracle.q_code(v, inv, b, u)
             assert -L <= k <= L
-            assert k == z - 128 + (1 if u + frac >= (1 << 15) else 0)
+            assert k == z - off + (1 if (u >> (15 - fb)) + frac >= (1 << fb) else 0)
         # exact count of round-ups over the whole uniform range, on a few values
-    for v in (g.uniform(-1, 1, 3) * float(nrm)).astype(F32):
-        F, _ = _exact_fixed_point(v, inv)
+    for v in (g.uniform(-1, 1, 3 if b in (2, 4, 8, 11) else 1) * float(nrm)).astype(F32):
+        F, _ = _exact_fixed_point(v, inv, b)
         ks = np.array([oracle.q_code(v, inv, b, u) for u in range(1 << 15)])
-        assert set(np.unique(ks)) <= {(F >> 15) - 128, (F >> 15) - 127}
-        assert int((ks == (F >> 15) - 127).sum()) == (F & 0x7FFF)
+        assert set(np.unique(ks)) <= {(F >> fb) - off, (F >> fb) - off + 1}
+        assert int((ks == (F >> fb) - off + 1).sum()) == (F & ((1 << fb) - 1)) << (15 - fb)
 
 
-@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("b", [2, 3, 4, 7, 8, 9, 10, 11])
 def test_q_rule_ii_clamps_to_dom(b):
     """Rule (ii): outside the hull of dom(delta,b) the nearest member: -2^(b-1) below, 2^(b-1)-1 above."""
     inv = oracle.scale_inv(F32(1.0), b)
     for u in (0, 77, (1 << 15) - 1):
         assert oracle.q_code(F32(50.0), inv, b, u) == 2 ** (b - 1) - 1
         assert oracle.q_code(F32(-50.0), inv, b, u) == -(2 ** (b - 1))
+        assert oracle.q_code(F32(1.0), inv, b, u) in (2 ** (b - 1) - 2, 2 ** (b - 1) - 1)     # the hull's own end stays inside
         assert oracle.q_code(F32(1e30), inv, b, u) == 2 ** (b - 1) - 1
 
 
 # ---------------------------------------------------------------------------------------------------
 # Q: vectors
 # ---------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("b", [2, 3, 4, 5, 6, 7, 8, 9, 10, 11])
 def test_code_range_and_neighbours(b):
     L = 2 ** (b - 1) - 1
     g = np.random.default_rng(b)
@@ -158,7 +168,8 @@ def test_code_range_and_neighbours(b):
         assert delta == nrm / F32(L)
         inv = oracle.scale_inv(nrm, b)
         t = np.array([float(Fraction(float(x)) * Fraction(float(inv))) for x in v])
-        fl = np.floor(np.round(t * 32768) / 32768)                      # t is a multiple of 2^-15 after rounding
+        res = float(1 << _fixed_point_shape(b)[1])
+        fl = np.floor(np.round(t * res) / res)                          # t is a multiple of the resolution after rounding
         assert np.all((codes == fl) | (codes == fl + 1))
         i = int(np.argmax(np.abs(v)))
         assert abs(codes[i]) >= L - 1                                   # the max coordinate sits at the end of the grid
@@ -185,7 +196,7 @@ def test_zero_and_nonfinite():
         assert oracle.quantize(v, 4, 1, 1, 1, 1)[2] == oracle.ERR_NONFINITE
 
 
-@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("b", [2, 4, 8, 5, 11])
 def test_unbiased_and_variance(b):
     """E[Q(v)] = v (Section 3.1 rule (i)) and E||Q(v)-v||^2 <= d delta^2/4 with per-coordinate variance
     (x-z)(z+delta-x) (appendix, first lemma and its proof)."""
@@ -205,7 +216,7 @@ def test_unbiased_and_variance(b):
     z = np.floor(v / delta) * delta
     var_exact = (v - z) * (z + delta - v)
     sd = np.sqrt(np.maximum(var_exact, 1e-30))
-    resol = delta * 2.0 ** -15                      # fixed-point position + fp32 scale rounding
+    resol = delta * 2.0 ** -_fixed_point_shape(b)[1]  # fixed-point position + fp32 scale rounding
     assert np.all(np.abs(mean - v) <= 5 * sd / np.sqrt(N) + resol)
     assert np.all(var_exact <= delta ** 2 / 4 + 1e-12)
     assert np.all(np.abs(mse - var_exact) <= 0.05 * delta ** 2 / 4 + resol * delta)
@@ -234,7 +245,7 @@ def _pack_bigint(codes, b, nbytes):
     return np.frombuffer(word.to_bytes(nbytes, "little"), dtype=np.uint8)
 
 
-@pytest.mark.parametrize("b", [2, 4, 8])
+@pytest.mark.parametrize("b", [2, 3, 4, 5, 6, 7, 8, 9, 10, 11])
 def test_pack_matches_bit_by_bit_and_roundtrips(b):
     g = np.random.default_rng(b)
     lo, hi = -(2 ** (b - 1)), 2 ** (b - 1) - 1
@@ -244,10 +255,9 @@ def test_pack_matches_bit_by_bit_and_roundtrips(b):
         assert buf.size % 16 == 0 and buf.size >= (d * b + 7) // 8
         assert np.array_equal(buf, _pack_bigint(codes, b, buf.size))    # includes zero tail/padding
         assert np.array_equal(oracle.unpack(buf, d, b), codes)
-    per = 8 // b
-    for lane in range(per):                                             # every code value in every lane
-        for k in range(lo, hi + 1):
-            codes = np.zeros(per, np.int32); codes[lane] = k
+    for lane in range(8):                                               # every code value at every bit phase of a byte
+        for k in (range(lo, hi + 1) if b <= 8 else list(range(lo, lo + 40)) + list(range(-20, 20)) + list(range(hi - 40, hi + 1))):
+            codes = np.zeros(8, np.int32); codes[lane] = k
             buf = oracle.pack(codes, b)
-            assert buf[0] == ((k % (1 << b)) << (lane * b)) and not buf[1:].any()
-            assert oracle.unpack(buf, per, b)[lane] == k
+            assert int.from_bytes(buf.tobytes(), "little") == (k % (1 << b)) << (lane * b)
+            assert oracle.unpack(buf, 8, b)[lane] == k
