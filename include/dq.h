@@ -19,14 +19,17 @@
  *   - Errors found on the host (bad argument, bad bit width, misaligned buffer) are returned immediately.
  *     Errors found by a kernel (non-finite norm, sparse message over capacity) set a sticky status word that
  *     dq_poll_status reads.
- *   - Bit widths b, b_x must be 2, 4 or 8 (b = 1 would give 2^(b-1)-1 = 0 levels).
+ *   - The gradient width b must be 2, 4 or 8; the model width b_x may be any of 2..11, the widths of Table 1
+ *     (b = 1 would give 2^(b-1)-1 = 0 levels).  Up to 8 bits the rounding position keeps 15 fractional bits, then
+ *     14, 13 and 12 for 9, 10 and 11 bits.
  *   - All random draws come from Philox4x32-10 with key = seed and counter
  *     (coordinate >> 3, round, worker, stream); the master's worker id is 0xFFFFFFFF; streams are
  *     0 model rounding, 1 gradient rounding, 2 sparsification mask, 3 minibatch sampling.  Equal
  *     (seed, round, inputs) give equal bytes.
  *
  * Packed code layout (message of Section 3.1: 32 bits for delta plus b bits per coordinate): codes are b-bit
- * two's complement; coordinate j of a message sits in byte j / (8/b) at bit offset (j mod (8/b)) * b.  The
+ * two's complement fields laid end to end: coordinate j occupies bits [j b, (j+1) b) of the message, bit k of the
+ * message being bit k mod 8 of byte k / 8 (for b dividing 8: byte j / (8/b) at bit offset (j mod (8/b)) * b).  The
  * bytes of one message are padded with zeros to dq_packed_bytes(d, b), a multiple of 16.  delta is kept in a
  * separate fp32 array.
  */
@@ -43,7 +46,7 @@ enum {
     DQ_OK = 0,
     DQ_ERR_ARG = 1,        /* NULL pointer, non-positive size, misaligned buffer                     */
     DQ_ERR_SHAPE = 2,      /* sizes inconsistent with the context (d, M, stride, capacity)            */
-    DQ_ERR_BITS = 3,       /* bit width not in {2, 4, 8}                                              */
+    DQ_ERR_BITS = 3,       /* b not in {2, 4, 8} or b_x outside 2..11                                 */
     DQ_ERR_NONFINITE = 4,  /* a vector to be quantised holds NaN or Inf                               */
     DQ_ERR_CAPACITY = 5,   /* a sparse message had more survivors than the buffers can hold           */
     DQ_ERR_CUDA = 6,       /* a CUDA runtime call failed                                              */
@@ -81,7 +84,7 @@ typedef struct {
     int32_t no_graph;          /* 1: dq_round launches its kernels one by one instead of replaying a CUDA graph */
     uint64_t seed;
     int64_t sparse_cap;        /* entries per worker in the context's own sparse message buffers; 0: d   */
-    float mu;                  /* > 0: dq_round picks b_x in {2,4,8} each round by condition (3)/(6); 0: fixed bx */
+    float mu;                  /* > 0: dq_round picks b_x in 2..11 each round by condition (3)/(6); 0: fixed bx */
     int32_t sequential;        /* 1: master applies the M messages one by one, one prox step each (Algorithm 1 step 9 as
                                   written; message w is w steps stale, delay <= M-1); 0: one step on their average */
     int32_t model;             /* DQ_MODEL_LOGISTIC (default) or DQ_MODEL_MLP: the 3-layer fully connected network of
@@ -134,9 +137,10 @@ int dq_quantize_model(dq_ctx* ctx, const float* x, const float* norm_x, uint32_t
                       uint8_t* codes_x, float* delta_x, void* stream);
 
 /* Model precision (condition (3); condition (6) for Algorithm 3 passes theta_s * mu): writes to *bits (device int)
- * the smallest width b in {2, 4, 8} with  E_Q ||Q_(delta,b)(x) - x||^2 <= mu ||x - x_snap||^2, 8 if none, where the
- * left side is the closed form sum_i (x_i - z_i)(z_i + delta - x_i) of rule (i).  stats (device double[4], may be
- * NULL) receives the expected errors at 2, 4, 8 bits and ||x - x_snap||^2.  norm_x: device ||x||_inf or NULL. */
+ * the smallest width b in 2..11 (the widths of Table 1) with  E_Q ||Q_(delta,b)(x) - x||^2 <= mu ||x - x_snap||^2,
+ * 11 if none, where the left side is the closed form sum_i (x_i - z_i)(z_i + delta - x_i) of rule (i).  stats
+ * (device double[11], may be NULL) receives the expected errors at 2..11 bits and ||x - x_snap||^2.  norm_x: device
+ * ||x||_inf or NULL. */
 int dq_select_model_bits(dq_ctx* ctx, const float* x, const float* x_snap, const float* norm_x, float mu,
                          int32_t* bits, double* stats, void* stream);
 

@@ -8,7 +8,8 @@ using namespace dq;
 
 namespace {
 
-bool bits_ok(int b) { return b == 2 || b == 4 || b == 8; }
+bool bits_ok(int b) { return b == 2 || b == 4 || b == 8; }                 // gradient messages
+bool model_bits_ok(int b) { return b >= 2 && b <= 11; }                    // the model: every width of Table 1
 bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
@@ -64,7 +65,7 @@ const char* dq_strerror(int status)
         case DQ_OK: return "ok";
         case DQ_ERR_ARG: return "bad argument (null, non-positive or misaligned)";
         case DQ_ERR_SHAPE: return "sizes inconsistent with the context";
-        case DQ_ERR_BITS: return "bit width must be 2, 4 or 8";
+        case DQ_ERR_BITS: return "bit width: the gradient takes 2, 4 or 8 bits, the model 2..11";
         case DQ_ERR_NONFINITE: return "vector to quantise holds NaN or Inf";
         case DQ_ERR_CAPACITY: return "sparse message exceeds its capacity";
         case DQ_ERR_CUDA: return "CUDA runtime error";
@@ -78,7 +79,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (!out || !cfg) return DQ_ERR_ARG;
     *out = nullptr;
     if (cfg->d < 1 || cfg->d > ((int64_t)1 << 32) || cfg->M < 1 || cfg->M > 4096 || cfg->B < 1) return DQ_ERR_ARG;
-    if (!bits_ok(cfg->b) || !bits_ok(cfg->bx)) return DQ_ERR_BITS;
+    if (!bits_ok(cfg->b) || !model_bits_ok(cfg->bx)) return DQ_ERR_BITS;
     if (cfg->msg_format == DQ_MSG_SPARSE && !cfg->sparsify) return DQ_ERR_ARG;
     if (cfg->msg_format != DQ_MSG_SPARSE && cfg->msg_format != DQ_MSG_DENSE) return DQ_ERR_ARG;
     if (!(cfg->box_lo <= cfg->box_hi) || cfg->lambda1 < 0 || cfg->lambda2 < 0) return DQ_ERR_ARG;
@@ -133,9 +134,9 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     rc |= dev_alloc(&c->msgs.scale, M);
     rc |= dev_alloc(&c->msgs.idx, sparse ? (size_t)c->msgs.cap * M : 1);
     rc |= dev_alloc(&c->msgs.nnz, M);
-    rc |= dev_alloc(&c->codes_x, (size_t)dq_packed_bytes(d, cfg->mu > 0.0f ? 8 : cfg->bx));
+    rc |= dev_alloc(&c->codes_x, (size_t)dq_packed_bytes(d, cfg->mu > 0.0f ? 11 : cfg->bx));
     rc |= dev_alloc(&c->bx_dev, 1);
-    rc |= dev_alloc(&c->prec_stats, 4);
+    rc |= dev_alloc(&c->prec_stats, 11);
     rc |= dev_alloc(&c->delta_x, 1);
     rc |= dev_alloc(&c->ninf, M);
     if (data) {
@@ -326,9 +327,9 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
             launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx),
                                  ctx->delta_x, round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
                                  reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
-        } else {     // condition (3): pick the width on the device, then launch all three widths; two return at once
+        } else {     // condition (3): pick the width on the device, then launch the three specialised widths and the general kernel; all but one return at once
             launch_select_bits(ctx, s->x, s->x_snap, nx, ctx->cfg.mu, theta, ctx->bx_dev, ctx->prec_stats, as_stream(st));
-            for (int bits = 2; bits <= 8; bits *= 2)
+            for (int bits : {2, 4, 8, 3})                      // 3 stands for "any other width": the general kernel reads it from the device
                 launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, bits, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, bits), ctx->delta_x,
                                      round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
                                      reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M, ctx->bx_dev);

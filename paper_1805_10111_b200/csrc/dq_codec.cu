@@ -1175,43 +1175,47 @@ clear_listed_groups_kernel(float* __restrict__ alpha, int64_t d, const uint32_t*
 }
 
 // ---------------------------------------------------------------------------------------------------
-// Model precision, condition (3): sums of frac (1 - frac) of x / delta_b for b = 2, 4, 8 (the expected squared
-// error of rule (i) in units of delta_b^2) and ||x - xsnap||^2, in double.  stats must be zero on entry.
+// Model precision, condition (3): sums of frac (1 - frac) of x / delta_b for b = 2..11 (the expected squared
+// error of rule (i) in units of delta_b^2; the widths of Table 1) and ||x - xsnap||^2, in double.
+// stats [kWidths + 1] must be zero on entry.
 // ---------------------------------------------------------------------------------------------------
+constexpr int kWidths = 10;          // candidate widths 2..11
+
 __global__ void __launch_bounds__(kThreads)
 model_precision_kernel(const float* __restrict__ x, const float* __restrict__ xsnap, int64_t d, const uint32_t* __restrict__ norm_bits,
                        double* __restrict__ stats)
 {
     pdl_prologue();
     const float nrm = __uint_as_float(norm_bits[0]);
-    double inv[3];
-    inv[0] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 1.0f) : 0.0;
-    inv[1] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 7.0f) : 0.0;
-    inv[2] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, 127.0f) : 0.0;
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    double inv[kWidths];
+#pragma unroll
+    for (int k = 0; k < kWidths; ++k) inv[k] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, (float)levels(k + 2)) : 0.0;
+    double acc[kWidths + 1];
+#pragma unroll
+    for (int k = 0; k <= kWidths; ++k) acc[k] = 0.0;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
         const double xi = (double)x[i], df = xi - (double)xsnap[i];
 #pragma unroll
-        for (int k = 0; k < 3; ++k) { const double t = xi * inv[k], fr = t - floor(t); acc[k] += fr * (1.0 - fr); }
-        acc[3] += df * df;
+        for (int k = 0; k < kWidths; ++k) { const double t = xi * inv[k], fr = t - floor(t); acc[k] += fr * (1.0 - fr); }
+        acc[kWidths] += df * df;
     }
-    __shared__ double s_part[kThreads / 32][4];
+    __shared__ double s_part[kThreads / 32][kWidths + 1];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k <= kWidths; ++k) {
         double v = acc[k];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
         if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5][k] = v;
     }
     __syncthreads();
-    if (threadIdx.x < 4) {
+    if (threadIdx.x <= kWidths) {
         double t = 0.0;
         for (int k = 0; k < (int)(blockDim.x >> 5); ++k) t += s_part[k][threadIdx.x];
         atomicAdd(stats + threadIdx.x, t);
     }
 }
 
-// Smallest width whose expected error is within mu ||x - xsnap||^2 (Algorithm 3: theta mu), 8 if none.
+// Smallest width whose expected error is within mu ||x - xsnap||^2 (Algorithm 3: theta mu), 11 if none.
 __global__ void select_bits_kernel(double* __restrict__ stats, const uint32_t* __restrict__ norm_bits, float mu, int accelerated,
                                    float theta, const RoundParams* __restrict__ rp, int32_t* __restrict__ bits)
 {
@@ -1219,16 +1223,95 @@ __global__ void select_bits_kernel(double* __restrict__ stats, const uint32_t* _
     if (rp) theta = rp->theta;
     const float nrm = __uint_as_float(norm_bits[0]);
     const double mu_eff = accelerated ? (double)__fmul_rn(theta, mu) : (double)mu;
-    const float L[3] = {1.0f, 7.0f, 127.0f};
-    const int widths[3] = {2, 4, 8};
-    int chosen = 8;
-    for (int k = 2; k >= 0; --k) {
-        const double delta = nrm > 0.0f ? (double)__fdiv_rn(nrm, L[k]) : 0.0;
-        const double e = stats[k] * delta * delta;
-        stats[k] = e;
-        if (e <= mu_eff * stats[3]) chosen = widths[k];
+    int chosen = kWidths + 1;
+    for (int b = kWidths + 1; b >= 2; --b) {
+        const double delta = nrm > 0.0f ? (double)__fdiv_rn(nrm, (float)levels(b)) : 0.0;
+        const double e = stats[b - 2] * delta * delta;
+        stats[b - 2] = e;
+        if (e <= mu_eff * stats[kWidths]) chosen = b;
     }
     *bits = chosen;
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Q_(delta,b) + pack for any width 2..11 (the model widths of Table 1 that do not divide eight: 3, 5, 6, 7, and
+// 9..11 bits).  The fixed-point position is r = fl(v inv + 1.5 2^e), e = 8 up to 8-bit codes and b beyond, whose
+// significand holds (t + 2^(e-1)) 2^(23-e); the top 23-e bits of the coordinate's draw are added and the fraction
+// dropped (15 fractional bits up to 8-bit codes, then 14, 13, 12).  A group of eight coordinates is b bytes of
+// the message, the codes laid end to end.  One vector (the model); width = *bits_dev if given (then the kernel
+// leaves 2, 4 and 8 bits to the kernels specialised for them), else bits_fixed.  With diff also writes
+// code * delta - ref and clears the next stages' accumulators, like quantize_pack_kernel<.., true>.
+// ---------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+quantize_pack_any_kernel(const float* __restrict__ v, int64_t d, const uint32_t* __restrict__ norm_bits, uint8_t* __restrict__ codes,
+                         float* __restrict__ scale, const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker,
+                         uint32_t stream, int* __restrict__ status, const RoundParams* __restrict__ rp,
+                         const float* __restrict__ ref, float* __restrict__ diff, float* __restrict__ zero_f, int64_t zero_n,
+                         uint32_t* __restrict__ zero_u, int zero_un, int bits_fixed, const int32_t* __restrict__ bits_dev)
+{
+    pdl_prologue();
+    const int bits = bits_dev ? *bits_dev : bits_fixed;
+    if (bits < 2 || bits > 11 || (bits_dev && (bits == 2 || bits == 4 || bits == 8))) return;
+    if (rp) round = rp->round;
+    const int64_t nth = (int64_t)gridDim.x * blockDim.x, tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (diff) {
+        for (int64_t i = tid; i < zero_n; i += nth) zero_f[i] = 0.0f;
+        if (tid < zero_un) zero_u[tid] = 0u;
+    }
+    const uint32_t nb = norm_bits[0];
+    const float nrm = __uint_as_float(nb);
+    const bool ok = nb < 0x7F800000u && nb != 0u;
+    const float Lf = (float)levels(bits);
+    const float inv = ok ? __fdiv_rd(Lf, nrm) : 0.0f;
+    const float delta = ok ? __fdiv_rn(nrm, Lf) : 0.0f;
+    if (tid == 0) { scale[0] = delta; if (nb >= 0x7F800000u) set_status(status, DQ_ERR_NONFINITE); }
+    const int e = bits <= 8 ? 8 : bits, fb = 23 - e;
+    const float off = 1.5f * (float)(1 << e);
+    const int half = 1 << (e - 1);
+    const uint32_t mask = (1u << bits) - 1u;
+    const int64_t nbytes = ((d * bits + 7) / 8 + 15) / 16 * 16;
+    const int64_t ngroups = (d + 7) >> 3;
+    for (int64_t g = tid; g < ngroups; g += nth) {
+        float a[8];
+        const int64_t i0 = g << 3;
+        load8_guarded(v, i0, d, a);
+        uint32_t r[4];
+        philox4x32_10((uint32_t)g, round, worker, stream, K, r);
+        unsigned long long lo = 0, hi = 0;                    // the group's 8 b <= 88 bits
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t F = __float_as_uint(__fmaf_rn(a[j], inv, off)) & 0x007FFFFFu;
+            const int code = (int)((F + (half16(r, j) >> (16 - fb))) >> fb) - half;
+            const unsigned long long field = (unsigned long long)((uint32_t)code & mask);
+            const int pos = j * bits;
+            if (pos < 64) { lo |= field << pos; if (pos + bits > 64) hi |= field >> (64 - pos); }
+            else hi |= field << (pos - 64);
+            if (diff && i0 + j < d) diff[i0 + j] = __fsub_rn(__fmul_rn((float)code, delta), ref ? ref[i0 + j] : 0.0f);
+        }
+        for (int k = 0; k < bits; ++k) {
+            const int64_t p = g * bits + k;
+            if (p < nbytes) codes[p] = (uint8_t)((k < 8 ? lo >> (8 * k) : hi >> (8 * (k - 8))) & 0xFFu);
+        }
+    }
+    for (int64_t p = ngroups * bits + tid; p < nbytes; p += nth) codes[p] = 0;     // padding behind the last group
+}
+
+// code * delta - ref for packed codes of any width (see quantize_pack_any_kernel for the layout).
+__global__ void __launch_bounds__(kThreads)
+dequant_diff_any_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ delta_x, const float* __restrict__ ref, int64_t d,
+                        float* __restrict__ diff, int bits)
+{
+    pdl_prologue();
+    const float dl = *delta_x;
+    const int64_t nbytes = ((d * bits + 7) / 8 + 15) / 16 * 16;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t bit = i * bits, p = bit >> 3;
+        uint32_t w = codes[p];
+        if (p + 1 < nbytes) w |= (uint32_t)codes[p + 1] << 8;
+        if (p + 2 < nbytes) w |= (uint32_t)codes[p + 2] << 16;
+        const int k = ((int)((w >> (bit & 7)) << (32 - bits))) >> (32 - bits);
+        diff[i] = __fsub_rn(__fmul_rn((float)k, dl), ref ? ref[i] : 0.0f);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -1257,6 +1340,12 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
                           uint32_t stream_id, cudaStream_t st, const float* ref, float* diff, float* zero_f, int64_t zero_n,
                           uint32_t* zero_u, int zero_un, const int32_t* bits_gate)
 {
+    if (bits != 2 && bits != 4 && bits != 8) {                 // a width that does not divide eight: one vector, general kernel
+        launch_k(quantize_pack_any_kernel, grid_for((d + 7) / 8, ctx->sm_count), kThreads, 0, st, v, d, norm_bits, codes, scale, ctx->keys,
+                 round, worker_base, stream_id, ctx->status, ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits, bits_gate);
+        ctx->launches += 1;
+        return;
+    }
     const int64_t ngroups = dq_packed_bytes(d, bits) / bits;
     dim3 grid(grid_for(ngroups, ctx->sm_count), M);
     if (diff) {
@@ -1273,10 +1362,16 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
 void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, float theta,
                         int32_t* bits, double* stats, cudaStream_t st)
 {
-    cudaMemsetAsync(stats, 0, sizeof(double) * 4, st);
-    launch_k(model_precision_kernel, grid_for(ctx->cfg.d / 4 + 1, ctx->sm_count), kThreads, 0, st, x, xsnap, ctx->cfg.d, norm_bits, stats);
+    cudaMemsetAsync(stats, 0, sizeof(double) * (kWidths + 1), st);
+    launch_k(model_precision_kernel, grid_for(ctx->cfg.d / 2 + 1, ctx->sm_count, 4), kThreads, 0, st, x, xsnap, ctx->cfg.d, norm_bits, stats);
     launch_k(select_bits_kernel, 1, 1, 0, st, stats, norm_bits, mu, ctx->cfg.accelerated, theta, ctx->rp_active, bits);
     ctx->launches += 2;
+}
+
+void launch_dequant_diff_any(dq_ctx* ctx, const uint8_t* codes, const float* delta_x, const float* ref, float* diff, int bits, cudaStream_t st)
+{
+    launch_k(dequant_diff_any_kernel, grid_for(ctx->cfg.d, ctx->sm_count), kThreads, 0, st, codes, delta_x, ref, ctx->cfg.d, diff, bits);
+    ctx->launches += 1;
 }
 
 void launch_clear_listed(dq_ctx* ctx, cudaStream_t st)

@@ -1082,7 +1082,9 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
     if (list) launch_clear_listed(ctx, st);                      // alpha is all-zero again before this round adds to it
     const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n,
                             ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr};
-    if (!ctx->diff_ready) {
+    if (!ctx->diff_ready && c.bx != 2 && c.bx != 4 && c.bx != 8) {
+        launch_dequant_diff_any(ctx, codes_x, delta_x, c.model == DQ_MODEL_MLP ? nullptr : s->x_snap, ctx->xhat_diff, c.bx, st);
+    } else if (!ctx->diff_ready) {
         DQ_DISPATCH_BITS(c.bx, (launch_k(dequant_diff_kernel<BITS_>, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, codes_x, delta_x, c.model == DQ_MODEL_MLP ? nullptr : s->x_snap, c.d, ctx->xhat_diff)));
         ctx->launches += 1;
     }
@@ -1164,6 +1166,7 @@ void small_round_setup(dq_ctx* ctx)
     ctx->cluster_blocks = 0;
     const dq_config& c = ctx->cfg;
     if (!ctx->has_data || c.no_fused || c.model != DQ_MODEL_LOGISTIC || c.sparsify || c.sequential || c.mu > 0.0f) return;
+    if (c.bx != 2 && c.bx != 4 && c.bx != 8) return;          // the kernel is specialised for the widths that divide eight
     if (ctx->data.format != DQ_DENSE_F32 && ctx->data.format != DQ_CSR_F32) return;
     // beyond about one group of eight coordinates per thread the stages stop being latency-bound and one
     // block per worker is slower than the whole GPU working through separate kernels

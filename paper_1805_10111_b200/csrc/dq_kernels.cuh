@@ -15,6 +15,7 @@ void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const u
                         int32_t* bits, double* stats, cudaStream_t st);
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
+void launch_dequant_diff_any(dq_ctx* ctx, const uint8_t* codes, const float* delta_x, const float* ref, float* diff, int bits, cudaStream_t st);
 void launch_clear_listed(dq_ctx* ctx, cudaStream_t st);
 void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st);
 void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,

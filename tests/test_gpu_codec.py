@@ -87,10 +87,12 @@ def test_quantize_misaligned_rows_and_large(dq):
         dq.dq_destroy(ctx)
 
 
-@pytest.mark.parametrize("bx", [2, 4, 8])
-def test_quantize_model_bit_exact(dq, bx):
+@pytest.mark.parametrize("bx", [2, 3, 4, 5, 6, 7, 8, 9, 10, 11])
+@pytest.mark.parametrize("d", [50021, 113, 8, 1])
+def test_quantize_model_bit_exact(dq, bx, d):
+    """Every model width of Table 1 (2..11 bits), including sizes whose last group of eight runs past the padded message."""
     import torch
-    d, seed, rnd = 50021, 99, 1234567
+    seed, rnd = 99, 1234567
     x = synth.normal_vector(d, 40, 0.3)
     cfg = dq.make_config(d, 2, bx=bx, seed=seed)
     rc, ctx = dq.dq_create(cfg); assert rc == 0

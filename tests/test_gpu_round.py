@@ -116,7 +116,7 @@ def test_epoch_begin_full_gradient(dq, name):
 
 
 @pytest.mark.parametrize("name", ["dense", "csr", "bf16", "bf16odd", "dense8"])
-@pytest.mark.parametrize("bx", [4, 8])
+@pytest.mark.parametrize("bx", [4, 8, 5, 11])
 def test_worker_gradient(dq, name, bx):
     import torch
     h = _problem(name)
@@ -325,6 +325,10 @@ class Lockstep:
     ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=5, no_fused=1), 0.5),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=6, no_fused=1), 0.5),
     ("dense8", dict(M=5, B=24, bx=4, b=2, lambda1=1e-4, lambda2=1e-3, box_lo=-0.5, box_hi=0.5, seed=10), 0.5),
+    # model widths that do not divide eight (Table 1 lists b_x from 2 to 11)
+    ("dense", dict(M=3, B=8, bx=5, b=8, lambda1=1e-4, seed=11), 0.5),
+    ("csr", dict(M=4, B=16, bx=11, b=4, lambda2=1e-5, seed=12), 0.5),
+    ("bf16", dict(M=4, B=16, bx=3, b=8, box_lo=-1.0, box_hi=1.0, seed=13), 0.01),
 ])
 def test_lockstep_small(dq, name, kw, eta):
     h = _problem(name)
@@ -371,7 +375,7 @@ def test_lockstep_accelerated_sparse(dq):
     ls.close()
 
 
-@pytest.mark.parametrize("mu,acc", [(1e-3, 0), (30.0, 0), (1e5, 0), (30.0, 1)])
+@pytest.mark.parametrize("mu,acc", [(1e-3, 0), (0.3, 0), (3.0, 0), (30.0, 0), (300.0, 0), (1e5, 0), (30.0, 1)])
 def test_lockstep_searched_model_bits(dq, mu, acc):
     """mu > 0: each round's model width comes from condition (3) (theta mu for Algorithm 3); codes, bits and iterates
     follow the oracle round by round."""
@@ -388,7 +392,8 @@ def test_lockstep_searched_model_bits(dq, mu, acc):
         for t in range(8):
             tr = ls.round(rnd, 0.5, theta)
             widths.add(tr["bx_used"]); rnd += 1
-    assert widths - {0} <= {2, 4, 8} and len(widths - {0}) >= 1
+    assert widths - {0} <= set(range(2, 12)) and len(widths - {0}) >= 1
+    print("\n[mu=%g acc=%d] widths chosen: %s" % (mu, acc, sorted(widths - {0})))
     ls.close()
 
 
@@ -504,14 +509,14 @@ def test_select_model_bits_standalone(dq):
     x = synth.normal_vector(d, 80); xs = (x + synth.normal_vector(d, 81, 0.02)).astype(F32)
     cfg = dq.make_config(d, 2)
     rc, ctx = dq.dq_create(cfg); assert rc == 0
-    bits = torch.zeros(1, dtype=torch.int32, device="cuda"); stats = torch.zeros(4, dtype=torch.float64, device="cuda")
+    bits = torch.zeros(1, dtype=torch.int32, device="cuda"); stats = torch.zeros(11, dtype=torch.float64, device="cuda")
     _, errs, dist = oracle.select_bx(x, xs, 1.0)
-    for mu in (errs[2] / dist * 0.5, errs[2] / dist * 1.5, errs[1] / dist * 1.5, errs[0] / dist * 1.5):
+    for mu in [errs[9] / dist * 0.5] + [errs[b - 2] / dist * 1.5 for b in (11, 9, 8, 6, 5, 4, 3, 2)]:
         assert dq.dq_select_model_bits(ctx, _dev(x), _dev(xs), None, mu, bits, stats) == 0
         want, _, _ = oracle.select_bx(x, xs, mu)
         assert bits.item() == want
         got = stats.cpu().numpy()
-        assert np.allclose(got[:3], errs, rtol=1e-9) and abs(got[3] - dist) <= 1e-11 * dist
+        assert np.allclose(got[:10], errs, rtol=1e-9) and abs(got[10] - dist) <= 1e-11 * dist
     dq.dq_destroy(ctx)
 
 
