@@ -109,6 +109,7 @@ def _declare(L):
         "dqo_sq_distance": (f64, [vp, vp, i64]),
         "dqo_select_bx": (i32, [vp, vp, i64, f32, vp, vp]),
         "dqo_round": (i32, [vp, vp, vp, u32, i32, f32, f32, vp]),
+        "dqo_round_delayed": (i32, [vp, vp, vp, u32, i32, f32, f32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(L, name)
@@ -368,10 +369,14 @@ class Run:
             return False
         return (not self.cfg.accelerated) or self.epoch == 0
 
-    def round(self, round_, eta, theta=0.0, trace=False):
+    def round(self, round_, eta, theta=0.0, trace=False, delays=None):
+        """delays: per worker, how many rounds of this epoch ago the model it works on was broadcast (Algorithm 1's
+        t - D(t); clamped to the rounds the epoch has had).  The run keeps the epoch's broadcasts for that."""
         cfg = self.cfg; d, M, B = cfg.d, cfg.M, cfg.B
         flag = self.is_flag_round()
         T = Trace(); keep = {}
+        if delays is not None and not trace:
+            keep = dict(xhat=np.zeros(d, np.float32)); T.xhat = _p(keep["xhat"])
         if trace:
             keep = dict(codes_x=np.zeros(d, np.int32), delta_x=np.zeros(1, np.float32), xhat=np.zeros(d, np.float32),
                         rows=np.zeros((M, B), np.int64), alpha=np.zeros((M, d), np.float32),
@@ -381,8 +386,19 @@ class Run:
                         phi_eff=np.zeros(M, np.float32), nnz=np.zeros(M, np.int64))
             for k, a in keep.items():
                 setattr(T, k, _p(a))
-        rc = lib().dqo_round(C.addressof(cfg), self.data.ref, C.addressof(self.state), round_, int(flag),
-                             float(eta), float(theta), C.addressof(T))
+        if delays is None:
+            rc = lib().dqo_round(C.addressof(cfg), self.data.ref, C.addressof(self.state), round_, int(flag),
+                                 float(eta), float(theta), C.addressof(T))
+        else:
+            if self.rounds_in_epoch == 0:
+                self.broadcasts = []                                       # low-precision models of this epoch, by round
+            t = self.rounds_in_epoch
+            used = [min(int(D), t) for D in delays]
+            ptrs = (C.c_void_p * M)(*[None if D == 0 else _p(self.broadcasts[t - D]) for D in used])
+            rc = lib().dqo_round_delayed(C.addressof(cfg), self.data.ref, C.addressof(self.state), round_, int(flag),
+                                         float(eta), float(theta), C.addressof(T), ptrs)
+            self.broadcasts.append(keep["xhat"].copy())
+            keep["delays_used"] = used
         self.rounds_in_epoch += 1
         self.ticks_in_epoch += cfg.M if cfg.sequential else 1
         keep.update(bits_down=int(T.bits_down), bits_up=int(T.bits_up), normx=np.float32(T.normx),

@@ -674,11 +674,25 @@ void dqo_epoch_begin(const dqo_config* C, const dqo_data* D, dqo_state* S, float
 }
 
 /* One inner iteration (Algorithm 1 steps 6-13, with Algorithm 2's step 12-13
- * or Algorithm 3's step 9) for M synchronous workers.  flag_round: the model
- * equals the snapshot, the master sends one flag bit and workers use xsnap
- * (end of the "Model Parameter Quantization" paragraph). */
+ * or Algorithm 3's step 9) for M workers.  flag_round: the model equals the
+ * snapshot, the master sends one flag bit and workers use xsnap (end of the
+ * "Model Parameter Quantization" paragraph).
+ * Delays (Algorithm 1 step 11 evaluates the gradient at x_{D(t)}, Assumption 3
+ * bounds t - D(t) by tau): when stale is given, worker w computes its gradient
+ * at the low-precision model stale[w] (one broadcast in an earlier round of
+ * the same epoch, kept by the caller) instead of this round's; stale[w] = NULL
+ * means this round's.  Everything else is unchanged. */
+int dqo_round_delayed(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t round, int flag_round,
+                      float eta, float theta, dqo_trace* T, const float* const* stale);
+
 int dqo_round(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t round, int flag_round,
               float eta, float theta, dqo_trace* T)
+{
+    return dqo_round_delayed(C, D, S, round, flag_round, eta, theta, T, NULL);
+}
+
+int dqo_round_delayed(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t round, int flag_round,
+                      float eta, float theta, dqo_trace* T, const float* const* stale)
 {
     const int64_t d = C->d; const int M = C->M, B = C->B;
     int rc = DQO_OK;
@@ -721,8 +735,9 @@ int dqo_round(const dqo_config* C, const dqo_data* D, dqo_state* S, uint32_t rou
         int64_t nnz = d;
         float ninf = 0.0f, n1 = 0.0f, phi_eff = 0.0f;
         dqo_sample_batch(C->seed, round, w, M, D->n, B, rows);
-        if (C->model == 1) dqo_mlp_worker_grad(D, C->hidden, C->classes, xhat, S->xsnap, rows, B, alpha, Sabs);
-        else dqo_worker_grad(D, xhat, S->xsnap, rows, B, alpha, Sabs);
+        const float* xw = (stale && stale[w]) ? stale[w] : xhat;     /* the model this worker pulled */
+        if (C->model == 1) dqo_mlp_worker_grad(D, C->hidden, C->classes, xw, S->xsnap, rows, B, alpha, Sabs);
+        else dqo_worker_grad(D, xw, S->xsnap, rows, B, alpha, Sabs);
         if (C->sparsify) {
             rc = dqo_sparsify(alpha, d, C->phi, C->seed, round, (uint32_t)w, beta, Z, NULL, &ninf, &n1, &phi_eff);
             if (rc == DQO_OK) rc = dqo_quantize_survivors(beta, Z, d, C->b, C->seed, round, (uint32_t)w, cw, &delta[w]);

@@ -206,6 +206,49 @@ def test_expected_error_closed_form_and_bit_width_search():
     assert oracle.select_bx(x, x, 1e9)[0] == 11                              # x = xsnap: nothing admissible (the flag bit handles it)
 
 
+def test_delayed_rounds_use_the_model_of_t_minus_delay():
+    """Algorithm 1 step 11 evaluates the gradient at x_{D(t)} with t - D(t) <= tau (Assumption 3).  With per-worker
+    delays the gradient difference of worker w must be the one at the low-precision model broadcast delays[w] rounds
+    earlier in the epoch (clamped to the epoch's start), re-derived here in float64 numpy from broadcasts that the
+    test rebuilds itself; zero delays must reproduce the ordinary round bit for bit."""
+    h, data = _problem()
+    M, B, tau = 3, 8, 2
+    cfg = oracle.make_config(h.d, M, B, 8, 8, l1=1e-4, seed=9)
+    x0 = synth.normal_vector(h.d, 35, 0.2)
+    run = oracle.Run(cfg, data, x0); ref = oracle.Run(cfg, data, x0)
+    g = np.random.default_rng(5)
+    X, y = h.values.astype(np.float64), h.labels
+    rnd = 0
+    for epoch in range(2):
+        run.epoch_begin(); ref.epoch_begin()
+        mine = []                                            # this epoch's broadcasts, rebuilt independently
+        for t in range(6):
+            delays = [int(v) for v in g.integers(0, tau + 1, M)] if epoch == 1 else [0] * M
+            x_before = run.x.copy()
+            tr = run.round(rnd, 0.4, trace=True, delays=delays)
+            if tr["flag_round"]:
+                mine.append(run.xsnap.copy())
+            else:
+                cx, dx, _ = oracle.quantize(x_before, 8, 9, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+                mine.append(cx.astype(F32) * dx)
+            assert tr["delays_used"] == [min(D, t) for D in delays]
+            for w in range(M):
+                xw = mine[t - min(delays[w], t)]
+                rows = tr["rows"][w]
+                want = ((_np_slope(X, y, rows, xw) - _np_slope(X, y, rows, run.xsnap))[:, None] * X[rows]).mean(axis=0)
+                assert np.allclose(tr["alpha"][w], want, rtol=1e-5, atol=1e-7), (epoch, t, w)
+            if epoch == 0:                                   # zero delays: the ordinary round
+                ref.round(rnd, 0.4)
+                assert np.array_equal(run.x, ref.x)
+            rnd += 1
+    # a delay matters: with every worker one round behind, the iterates leave the undelayed run's
+    a = oracle.Run(cfg, data, x0); b = oracle.Run(cfg, data, x0)
+    a.epoch_begin(); b.epoch_begin()
+    for t in range(4):
+        a.round(t, 0.4, delays=[1] * M); b.round(t, 0.4)
+    assert not np.array_equal(a.x, b.x)
+
+
 def test_round_with_searched_model_bits():
     """With mu > 0 every non-flag round quantises the model with the searched width and pays for that width."""
     h, data = _problem()
