@@ -93,6 +93,8 @@ typedef struct {
                                   d = hidden*(in+1) + classes*(hidden+1) with x = [W1 (hidden x in), b1, W2 (classes x hidden), b2] */
     int32_t hidden, classes;
     int32_t no_fused;          /* 1: never run rounds in the one-cluster kernel (see dq_round); 0: use it where it applies */
+    int32_t max_delay;         /* tau of Assumption 3: dq_round keeps the last tau + 1 broadcast models of the epoch so that
+                                  workers can be made to lag (dq_set_delays); 0: every worker uses the current broadcast */
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3
@@ -190,6 +192,14 @@ int dq_master_unpack_aggregate_prox(dq_ctx* ctx, const dq_msgs* msgs, dq_state* 
  * separate kernels would spend their time in launch gaps.  Results, buffers and layouts are the same. */
 int dq_round(dq_ctx* ctx, dq_state* st, uint32_t round, float eta, float theta,
              uint64_t* bits_down, uint64_t* bits_up, void* stream);
+
+/* Delays (Algorithm 1 step 11 evaluates the gradient at x_{D(t)}; Assumption 3: t - D(t) <= tau).  delays (HOST,
+ * [M], each in 0..max_delay; NULL: all zero) says for every worker how many rounds before the current one the model
+ * it works on was broadcast; it holds for the following dq_round calls until set again.  A delay is cut to the
+ * number of rounds the epoch has had (the first round's workers all see the current model).  Needs
+ * cfg.max_delay > 0 and the logistic model; such a context launches its rounds kernel by kernel (no graph, no
+ * one-cluster kernel).  Copies synchronously. */
+int dq_set_delays(dq_ctx* ctx, const int32_t* delays);
 
 /* nrounds consecutive rounds round0, round0 + 1, ... of the same epoch with the same (eta, theta), as by
  * dq_round called once per round (Algorithm 1 steps 6-13 repeated; the caller places dq_epoch_begin between

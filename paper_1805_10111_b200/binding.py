@@ -21,7 +21,7 @@ EXPORTS = ["dq_packed_bytes", "dq_create", "dq_destroy", "dq_epoch_begin", "dq_q
            "dq_norm_inf", "dq_quantize_sparsify_pack", "dq_master_unpack_aggregate_prox", "dq_round", "dq_codec_round",
            "dq_codec_host_setup", "dq_codec_round_host", "dq_unpack", "dq_objective", "dq_round_buffers",
            "dq_poll_status", "dq_launch_count", "dq_strerror", "dq_quantize_pack_static", "dq_select_model_bits",
-           "dq_last_model_bits", "dq_rounds"]
+           "dq_last_model_bits", "dq_rounds", "dq_set_delays"]
 
 
 class dq_data(C.Structure):
@@ -34,7 +34,7 @@ class dq_config(C.Structure):
                 ("lambda1", C.c_float), ("lambda2", C.c_float), ("box_lo", C.c_float), ("box_hi", C.c_float),
                 ("sparsify", C.c_int32), ("phi", C.c_float), ("msg_format", C.c_int32), ("accelerated", C.c_int32),
                 ("snapshot_flag", C.c_int32), ("no_graph", C.c_int32), ("seed", C.c_uint64), ("sparse_cap", C.c_int64), ("mu", C.c_float), ("sequential", C.c_int32),
-                ("model", C.c_int32), ("hidden", C.c_int32), ("classes", C.c_int32), ("no_fused", C.c_int32)]
+                ("model", C.c_int32), ("hidden", C.c_int32), ("classes", C.c_int32), ("no_fused", C.c_int32), ("max_delay", C.c_int32)]
 
 
 class dq_state(C.Structure):
@@ -76,6 +76,7 @@ def lib():
             "dq_master_unpack_aggregate_prox": (i32, [vp, C.POINTER(dq_msgs), C.POINTER(dq_state), f32, f32, vp]),
             "dq_round": (i32, [vp, C.POINTER(dq_state), u32, f32, f32, vp, vp, vp]),
             "dq_rounds": (i32, [vp, C.POINTER(dq_state), u32, i32, f32, f32, vp, vp, vp]),
+            "dq_set_delays": (i32, [vp, vp]),
             "dq_codec_round": (i32, [vp, vp, C.POINTER(dq_state), u32, f32, f32, vp, vp, vp]),
             "dq_codec_host_setup": (i32, [vp, vp, vp]),
             "dq_codec_round_host": (i32, [vp, vp, u32, f32, vp, vp, vp]),
@@ -163,9 +164,9 @@ class Msgs:
 
 
 def make_config(d, M, B=1, bx=8, b=8, lambda1=0.0, lambda2=0.0, box_lo=float("-inf"), box_hi=float("inf"), sparsify=0,
-                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0, sequential=0, model=0, hidden=0, classes=0, no_fused=0) -> dq_config:
+                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0, sequential=0, model=0, hidden=0, classes=0, no_fused=0, max_delay=0) -> dq_config:
     return dq_config(d, M, B, bx, b, lambda1, lambda2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, int(sequential), int(model), int(hidden), int(classes), int(no_fused))
+                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, int(sequential), int(model), int(hidden), int(classes), int(no_fused), int(max_delay))
 
 
 # ---- entry points (same names and order of arguments as include/dq.h) ---------------------------------------------
@@ -221,6 +222,14 @@ def dq_round(ctx, st: State, round_, eta, theta=0.0, bits_down=None, bits_up=Non
 def dq_rounds(ctx, st: State, round0, nrounds, eta, theta=0.0, bits_down=None, bits_up=None, stream=None):
     return lib().dq_rounds(ctx, C.byref(st.c), int(round0), int(nrounds), float(eta), float(theta), _ptr(bits_down),
                            _ptr(bits_up), _stream(stream))
+
+
+def dq_set_delays(ctx, delays):
+    """delays: sequence of M ints (rounds each worker lags), or None for no delay."""
+    if delays is None:
+        return lib().dq_set_delays(ctx, None)
+    arr = (C.c_int32 * len(delays))(*[int(v) for v in delays])
+    return lib().dq_set_delays(ctx, C.cast(arr, C.c_void_p))
 
 
 def dq_codec_round(ctx, v, st: State, round_, eta, theta, codes_x, delta_x, stream=None):

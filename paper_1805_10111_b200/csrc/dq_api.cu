@@ -85,6 +85,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (!(cfg->box_lo <= cfg->box_hi) || cfg->lambda1 < 0 || cfg->lambda2 < 0) return DQ_ERR_ARG;
     if (cfg->sparse_cap < 0 || cfg->sparse_cap > cfg->d) return DQ_ERR_ARG;
     if (!(cfg->mu >= 0.0f)) return DQ_ERR_ARG;
+    if (cfg->max_delay < 0 || cfg->max_delay > 64 || (cfg->max_delay > 0 && (!data || cfg->model != DQ_MODEL_LOGISTIC))) return DQ_ERR_ARG;
     if (data) {
         if (data->n < 1 || !data->values || !data->labels) return DQ_ERR_SHAPE;
         if (cfg->model == DQ_MODEL_MLP) {
@@ -142,7 +143,10 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (data) {
         rc |= dev_alloc(&c->alpha, (size_t)M * d);
         rc |= dev_alloc(&c->rows, (size_t)M * cfg->B);
-        rc |= dev_alloc(&c->xhat_diff, (size_t)d);
+        rc |= dev_alloc(&c->xhat_diff, (size_t)d * (cfg->max_delay + 1));     // a ring of broadcasts when workers may lag
+        rc |= dev_alloc(&c->delays_dev, M);
+        rc |= dev_alloc(&c->slots_dev, M);
+        if (rc == DQ_OK && cudaMemset(c->delays_dev, 0, sizeof(int32_t) * M) != cudaSuccess) rc = DQ_ERR_CUDA;
         rc |= dev_alloc(&c->g64, (size_t)d);
         rc |= dev_alloc(&c->rbuf, (size_t)M * cfg->B);
         if (cfg->model == DQ_MODEL_MLP) {
@@ -179,7 +183,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
 int dq_destroy(dq_ctx* c)
 {
     if (!c) return DQ_ERR_ARG;
-    void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->xnorm_bits, c->status, c->bits,
+    void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->delays_dev, c->slots_dev, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
                     c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
@@ -318,6 +322,16 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
 {
     int rc = DQ_OK;
     const bool adaptive = ctx->cfg.mu > 0.0f;
+    // delayed workers: this round's xhat - xsnap goes to its slot of the ring, and every worker is pointed at the
+    // slot of the broadcast it lags behind to
+    const int tau = ctx->cfg.max_delay;
+    float* const ring = ctx->xhat_diff;
+    if (tau > 0) {
+        const int t = (int)ctx->rounds_in_epoch;
+        ctx->xhat_diff = ring + (int64_t)(t % (tau + 1)) * ctx->cfg.d;
+        if (flag) cudaMemsetAsync(ctx->xhat_diff, 0, sizeof(float) * ctx->cfg.d, as_stream(st));   // xhat = xsnap
+        launch_set_slots(ctx, t, as_stream(st));
+    }
     if (!flag) {     // model quantisation that also emits xhat - xsnap for the workers
         const uint32_t* nx = reinterpret_cast<const uint32_t*>(s->norm_x);
         float* zf = worker_accumulates(ctx) ? ctx->alpha : nullptr;
@@ -338,7 +352,10 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     } else if (adaptive) {
         cudaMemsetAsync(ctx->bx_dev, 0, sizeof(int32_t), as_stream(st));
     }
+    ctx->xhat_diff = ring;                                   // the workers index the ring themselves
+    ctx->use_slots = tau > 0;
     rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
+    ctx->use_slots = false;
     ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = false;
     if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, st);
     ctx->list_ready = false;
@@ -390,7 +407,7 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
         return last_error();
     }
     bool replayed = false;
-    if (!flag && !ctx->graph_off && !c.no_graph) {
+    if (!flag && !ctx->graph_off && !c.no_graph && c.max_delay == 0) {
         const dq_state& g = ctx->graph_state;
         const bool same = ctx->graph_exec && g.x == s->x && g.x_snap == s->x_snap && g.g_full == s->g_full && g.y == s->y &&
                           g.x_sum == s->x_sum && g.norm_x == s->norm_x && g.z_snap == s->z_snap &&
@@ -411,6 +428,15 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
     ctx->rounds_in_epoch += 1;
     ctx->ticks_in_epoch += ctx->cfg.sequential ? ctx->cfg.M : 1;
     return last_error();
+}
+
+int dq_set_delays(dq_ctx* ctx, const int32_t* delays)
+{
+    if (!ctx || !ctx->has_data || ctx->cfg.max_delay <= 0) return DQ_ERR_ARG;
+    const int M = ctx->cfg.M;
+    if (!delays) return cudaMemset(ctx->delays_dev, 0, sizeof(int32_t) * M) == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+    for (int w = 0; w < M; ++w) if (delays[w] < 0 || delays[w] > ctx->cfg.max_delay) return DQ_ERR_ARG;
+    return cudaMemcpy(ctx->delays_dev, delays, sizeof(int32_t) * M, cudaMemcpyHostToDevice) == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }
 
 int dq_rounds(dq_ctx* ctx, dq_state* s, uint32_t round0, int32_t nrounds, float eta, float theta, uint64_t* bits_down,

@@ -288,6 +288,10 @@ struct dq_ctx {
     bool graph_off;
     // sparse gradients (CSR data, sparse messages): bitmap of touched groups, their ascending list, its length
     uint32_t* touched; uint32_t* glist; uint32_t* gcount; uint32_t* seg_count; int64_t bm_words; int64_t glist_cap;
+    // delayed workers: xhat_diff is a ring of max_delay + 1 vectors (slot = round in epoch mod ring size)
+    int32_t* delays_dev;        // [M] rounds each worker lags behind
+    int32_t* slots_dev;         // [M] ring slot each worker reads this round
+    bool use_slots;             // set while dq_round enqueues a round of a context with max_delay > 0
     int cluster_blocks;         // blocks of the one-cluster round kernel for small problems; 0: rounds run as separate kernels
     bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only
     bool list_ready;            // the list of this round has been built (consumed by the sparsifier launch)

@@ -72,7 +72,14 @@ __device__ __forceinline__ int64_t sample_row(const PhiloxKeys& K, uint32_t roun
 struct BatchSource {
     const int32_t* rows_in; int32_t* rows_out; uint32_t round; const RoundParams* rp; int M; int64_t n;
     uint32_t* zero_word;   // cleared by the first thread of the grid (the next stage's maximum), may be NULL
+    const int32_t* diff_slot; int64_t diff_stride;   // delayed workers: worker w reads xhat - xsnap at slot diff_slot[w]; NULL: slot 0
 };
+
+// xhat - xsnap as worker w sees it (the current broadcast, or an earlier one of the epoch when the worker lags).
+__device__ __forceinline__ const float* diff_of_worker(const BatchSource& bs, const float* diff, int w)
+{
+    return bs.diff_slot ? diff + (int64_t)bs.diff_slot[w] * bs.diff_stride : diff;
+}
 
 __device__ __forceinline__ void clear_word(const BatchSource& bs)
 {
@@ -120,7 +127,7 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
     const int w = (int)(slot / B);
     const int64_t a = batch_row(bs, K, w, (int)(slot % B), B, lane == 0);
     const int64_t k0 = row_ptr[a], k1 = row_ptr[a + 1];
-    const float dz = (float)warp_dot_csr(val, col, k0, k1, diff, lane);
+    const float dz = (float)warp_dot_csr(val, col, k0, k1, diff_of_worker(bs, diff, w), lane);
     const float r = slope_difference(labels[a], z_snap[a], dz) / (float)B;
     float* out = alpha + (int64_t)w * d;
     uint32_t* bm = touched ? touched + (int64_t)w * bm_words : nullptr;
@@ -155,7 +162,7 @@ worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labe
     const int nrows = min(kRowsPerBlock, B - j0);
     for (int j = warp; j < nrows; j += kThreads / 32) {
         const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
-        const float dz = (float)warp_dot_dense(X + a * d, diff, d, lane);
+        const float dz = (float)warp_dot_dense(X + a * d, diff_of_worker(bs, diff, w), d, lane);
         if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_row[j] = a; }
     }
     __syncthreads();
@@ -229,7 +236,7 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
     const int nrows = min(kRowsPerBlock, B - j0);
     for (int j = warp; j < nrows; j += kThreads / 32) {
         const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
-        const float dz = (float)warp_dot_dense_vec(X + a * d, diff, d, lane);
+        const float dz = (float)warp_dot_dense_vec(X + a * d, diff_of_worker(bs, diff, w), d, lane);
         if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_rowp[j] = reinterpret_cast<const uint4*>(X + a * d); }
     }
     __syncthreads();
@@ -277,7 +284,7 @@ worker_margins_kernel(const T* __restrict__ X, const float* __restrict__ labels,
     if (slot >= (int64_t)M * B) return;
     const int w = (int)(slot / B), j = (int)(slot % B);
     const int64_t a = batch_row(bs, K, w, j, B, lane == 0);
-    const float dz = (float)warp_dot_dense_vec(X + a * d, diff, d, lane);
+    const float dz = (float)warp_dot_dense_vec(X + a * d, diff_of_worker(bs, diff, w), d, lane);
     if (lane == 0) rbuf[slot] = slope_difference(labels[a], z_snap[a], dz) / (float)B;
 }
 
@@ -1081,7 +1088,8 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
     }
     if (list) launch_clear_listed(ctx, st);                      // alpha is all-zero again before this round adds to it
     const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n,
-                            ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr};
+                            ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr,
+                            ctx->use_slots ? ctx->slots_dev : nullptr, c.d};
     if (!ctx->diff_ready && c.bx != 2 && c.bx != 4 && c.bx != 8) {
         launch_dequant_diff_any(ctx, codes_x, delta_x, c.model == DQ_MODEL_MLP ? nullptr : s->x_snap, ctx->xhat_diff, c.bx, st);
     } else if (!ctx->diff_ready) {
@@ -1165,7 +1173,7 @@ void small_round_setup(dq_ctx* ctx)
 {
     ctx->cluster_blocks = 0;
     const dq_config& c = ctx->cfg;
-    if (!ctx->has_data || c.no_fused || c.model != DQ_MODEL_LOGISTIC || c.sparsify || c.sequential || c.mu > 0.0f) return;
+    if (!ctx->has_data || c.no_fused || c.model != DQ_MODEL_LOGISTIC || c.sparsify || c.sequential || c.mu > 0.0f || c.max_delay > 0) return;
     if (c.bx != 2 && c.bx != 4 && c.bx != 8) return;          // the kernel is specialised for the widths that divide eight
     if (ctx->data.format != DQ_DENSE_F32 && ctx->data.format != DQ_CSR_F32) return;
     // beyond about one group of eight coordinates per thread the stages stop being latency-bound and one
@@ -1224,6 +1232,20 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
     else launch_k(objective_loss_kernel<DQ_DENSE_BF16>, grid, kThreads, 0, st, D, x, P);
     launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
     ctx->launches += 2;
+}
+
+// Ring slot that each worker reads in round t of the epoch: the broadcast of round t - min(delay, t), ring of tau + 1.
+__global__ void set_slots_kernel(const int32_t* __restrict__ delays, int M, int t, int tau, int32_t* __restrict__ slots)
+{
+    pdl_prologue();
+    const int w = blockIdx.x * blockDim.x + threadIdx.x;
+    if (w < M) { const int D = min(min(max(delays[w], 0), tau), t); slots[w] = (t - D) % (tau + 1); }
+}
+
+void launch_set_slots(dq_ctx* ctx, int t, cudaStream_t st)
+{
+    launch_k(set_slots_kernel, (ctx->cfg.M + kThreads - 1) / kThreads, kThreads, 0, st, ctx->delays_dev, ctx->cfg.M, t, ctx->cfg.max_delay, ctx->slots_dev);
+    ctx->launches += 1;
 }
 
 __global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float eta, float theta)

@@ -28,6 +28,7 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
                         uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st);
 bool worker_accumulates(const dq_ctx* ctx);
 void small_round_setup(dq_ctx* ctx);
+void launch_set_slots(dq_ctx* ctx, int round_in_epoch, cudaStream_t st);
 void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds, float eta, float theta, uint64_t* bits_down,
                           uint64_t* bits_up, cudaStream_t st);
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st);

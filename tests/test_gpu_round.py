@@ -197,6 +197,7 @@ class Lockstep:
                    msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"],
                    mu=kw.get("mu", 0.0), sequential=kw.get("sequential", 0), model=kw.get("model", 0),
                    hidden=kw.get("hidden", 0), classes=kw.get("classes", 0))
+        assert not (set(kw) - {"M", "B", "bx", "b", "lambda1", "lambda2", "box_lo", "box_hi", "no_fused", "no_graph", "max_delay"} - set(okw)), kw
         d = x0.size                                        # parameters (equals the feature count for logistic regression)
         self.cfg = dq.make_config(d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
         self.ocfg = oracle.make_config(d, kw["M"], kw["B"], kw["bx"], kw["b"], **okw)
@@ -229,14 +230,16 @@ class Lockstep:
             self.st.z_snap.copy_(_dev(self.run.z_snap))
         assert nbad == 0, ("g_full", nbad, worst)
 
-    def round(self, rnd, eta, theta=0.0):
+    def round(self, rnd, eta, theta=0.0, delays=None):
         import torch
         dq, cfg, st, run = self.dq, self.cfg, self.st, self.run
         M, d, b = cfg.M, cfg.d, cfg.b
         self.sync_state()
         x_before = run.x.copy(); y_before = run.y.copy(); xsum_before = run.xsum.copy()
+        if delays is not None:
+            assert dq.dq_set_delays(self.ctx, delays) == 0
         assert dq.dq_round(self.ctx, st, rnd, eta, theta, self.bits[0:1], self.bits[1:2]) == 0
-        tr = run.round(rnd, eta, theta, trace=True)
+        tr = run.round(rnd, eta, theta, trace=True, delays=delays)
         assert tr["status"] == 0 and dq.dq_poll_status(self.ctx) == (0, 0)
         _, buf = dq.dq_round_buffers(self.ctx)
         m = buf["msgs"]
@@ -417,6 +420,35 @@ def test_lockstep_sequential_master(dq, name, kw):
         for t in range(6):
             ls.round(rnd, 0.05 if acc else 0.3, theta)
             rnd += 1
+    ls.close()
+
+
+@pytest.mark.parametrize("name,kw,eta", [
+    ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=41, max_delay=2), 0.5),
+    ("csr", dict(M=5, B=16, bx=8, b=4, lambda2=1e-5, seed=42, max_delay=3), 0.5),
+    ("bf16", dict(M=3, B=70, bx=8, b=8, box_lo=-1.0, box_hi=1.0, seed=43, max_delay=1), 0.01),
+    ("dense8", dict(M=4, B=8, bx=6, b=8, lambda1=1e-3, sequential=1, seed=44, max_delay=2), 0.3),
+    ("dense8", dict(M=4, B=16, bx=8, b=4, lambda2=1e-4, accelerated=1, seed=45, max_delay=2), 0.05),
+])
+def test_lockstep_delayed_workers(dq, name, kw, eta):
+    """Workers that lag by up to tau rounds (Algorithm 1 step 11 with x_{D(t)}, Assumption 3): every worker's gradient
+    difference must be the one at the model broadcast `delay` rounds earlier in the epoch, for all gradient kernels,
+    with the averaged and the one-by-one master, and with delays that change every round."""
+    h = _problem(name)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 85, 0.05), **kw)
+    g = np.random.default_rng(kw["seed"])
+    M, tau, acc = kw["M"], kw["max_delay"], bool(kw.get("accelerated", 0))
+    rnd = 0
+    for epoch in range(3):
+        theta = F32(2.0 / (epoch + 3)) if acc else F32(0.0)
+        ls.epoch(theta)
+        for t in range(2 * tau + 4):
+            delays = [int(v) for v in g.integers(0, tau + 1, M)] if epoch > 0 else [tau] * M
+            tr = ls.round(rnd, eta, theta, delays=delays)
+            assert tr["delays_used"] == [min(D, t) for D in delays]
+            rnd += 1
+    assert ls.far_flips == 0
+    assert dq.dq_set_delays(ls.ctx, [tau + 1] * M) == dq.DQ_ERR_ARG
     ls.close()
 
 
