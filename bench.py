@@ -6,7 +6,8 @@ d = 2^27 fp32 coordinates (N(0,1) with 0.1 % outliers x100), quantised to b = 4 
 and prox-updated by the master, and the new model requantised to b_x = 8 bits.  One "step" is one such
 round: ||v||_inf pass, quantise+pack, master unpack+aggregate+prox, model norm is fused, model quantise.
 Prints ONE JSON line: metric, value (whole-job rounds/s), per-stage times, roofline of the dominant kernel, clocks,
-end-to-end rate through host buffers, the CPU oracle's rate, and rounds/s of the training configurations.
+end-to-end rate through host buffers, the CPU oracle's rate, and rounds/s of the training configurations (each
+with the oracle's rate on the same data).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--log2d 27] [--bits 4]
 
@@ -210,7 +211,7 @@ TRAIN_CONFIGS = {
 }
 
 
-def time_training_config(name, rounds=200, warmup=20):
+def time_training_config(name, rounds=200, warmup=20, with_oracle=False):
     """rounds/s of dq_rounds on one of the training configurations (full size, synthetic data), plus the bits
     the paper's accounting charges per round."""
     import numpy as np
@@ -242,7 +243,33 @@ def time_training_config(name, rounds=200, warmup=20):
            "launches_per_round": (dq.dq_launch_count(ctx) - l0) / rounds, "bits_down": int(bits[0].item()),
            "bits_up": int(bits[1].item()), "bits_full_precision": 2 * cfg.M * 32 * int(cfg.d), "device_status": status}
     dq.dq_destroy(ctx)
+    if with_oracle:
+        out["cpu_oracle"] = oracle_training_rounds_per_sec(h, spec, x0)
     return out
+
+
+def oracle_training_rounds_per_sec(h, spec, x0, budget_s=6.0):
+    """The CPU oracle on the same data and settings: an epoch boundary, one untimed round, then whole rounds until
+    about budget_s seconds have gone (at least two).  Single thread."""
+    import numpy as np
+    import oracle
+    kw = spec["kw"]
+    ocfg = oracle.make_config(x0.size, kw["M"], kw["B"], kw["bx"], kw["b"], l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0),
+                              box_lo=kw.get("box_lo", -np.inf), box_hi=kw.get("box_hi", np.inf), sparsify=kw.get("sparsify", 0),
+                              phi=kw.get("phi", 0.0), msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0),
+                              seed=1805, model=kw.get("model", 0), hidden=kw.get("hidden", 0), classes=kw.get("classes", 0))
+    data = oracle.Dataset(h.format, h.n, h.d, h.values, h.labels, getattr(h, "col_idx", None), getattr(h, "row_ptr", None))
+    run = oracle.Run(ocfg, data, x0)
+    theta = spec["theta"]; eta = spec["lr"] / theta if theta else spec["lr"]
+    run.epoch_begin(theta)
+    run.round(0, eta, theta)
+    n, t0 = 0, time.perf_counter()
+    while n < 2 or time.perf_counter() - t0 < budget_s:
+        run.round(1 + n, eta, theta); n += 1
+        if n >= 200:
+            break
+    sec = (time.perf_counter() - t0) / n
+    return {"rounds_per_s": round(1.0 / sec, 3), "cores": 1, "kind": "oracle", "sample": "%d whole rounds at full size" % n}
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -388,7 +415,8 @@ def run_ours(a):
     del v, hv, st, msgs
     torch.cuda.empty_cache()
     if world == 1 and a.configs:
-        line["training_configs"] = {c: time_training_config(c) for c in a.configs.split(",") if c in TRAIN_CONFIGS}
+        line["training_configs"] = {c: time_training_config(c, with_oracle=not a.no_cpu_baseline)
+                                    for c in a.configs.split(",") if c in TRAIN_CONFIGS}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
