@@ -272,7 +272,7 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
 //                           served from L2.
 // ---------------------------------------------------------------------------------------------------
 template <class T>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 8)     // one wave: M B / 8 blocks must all be resident (a second, thin wave doubles the time)
 worker_margins_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
                       const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d,
                       float* __restrict__ rbuf)
@@ -308,13 +308,25 @@ worker_colsum_kernel(const T* __restrict__ X, const int32_t* __restrict__ rows, 
 #pragma unroll
     for (int q = 0; q < N; ++q) acc[q] = 0.0f;
     if (v < nv) {
-#pragma unroll 8
-        for (int j = warp; j < B; j += kWarps) {
-            float f[N];
-            RowVec<T>::unpack(__ldg(reinterpret_cast<const uint4*>(X + (int64_t)s_row[j] * d) + v), f);
-            const float r = s_r[j];
+        constexpr int U = 8;                       // row slabs in flight per lane; rows are taken in the same order as a plain loop
+        for (int j0 = warp; j0 < B; j0 += kWarps * U) {
+            uint4 q4[U]; float r[U];
 #pragma unroll
-            for (int q = 0; q < N; ++q) acc[q] = fmaf(r, f[q], acc[q]);
+            for (int u = 0; u < U; ++u) {
+                const int j = j0 + u * kWarps;
+                const bool in = j < B;
+                q4[u] = in ? __ldg(reinterpret_cast<const uint4*>(X + (int64_t)s_row[j] * d) + v) : make_uint4(0u, 0u, 0u, 0u);
+                r[u] = in ? s_r[j] : 0.0f;
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (j0 + u * kWarps < B) {
+                    float f[N];
+                    RowVec<T>::unpack(q4[u], f);
+#pragma unroll
+                    for (int q = 0; q < N; ++q) acc[q] = fmaf(r[u], f[q], acc[q]);
+                }
+            }
         }
     }
 #pragma unroll
