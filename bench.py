@@ -203,7 +203,10 @@ def recorded_traffic(bits):
 TRAIN_CONFIGS = {
     "c1": dict(gen="config1", kw=dict(M=4, B=16, bx=8, b=8, lambda1=1e-4), lr=1.0, theta=0.0, m=200),
     "c2": dict(gen="config2", kw=dict(M=8, B=64, bx=8, b=4, lambda2=1e-5), lr=1.0, theta=0.0, m=200),
-    "c3": dict(gen="config3", kw=dict(M=16, B=128, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1),
+    # sparse_cap: a message holds at most B * nnz/row = 12,800 entries here; the default capacity (d) would have the
+    # round clear 8 MiB of code buffers for a few hundred bytes of codes
+    "c3": dict(gen="config3", kw=dict(M=16, B=128, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1,
+                                      sparse_cap=1 << 14),
                lr=1.0, theta=0.0, m=200),
     "nn": dict(gen="config_nn", kw=dict(M=8, B=20, bx=8, b=4, lambda2=1e-4, model=1, hidden=100, classes=10), lr=0.1, theta=0.0, m=500),
     "c4": dict(gen="config4", kw=dict(M=32, B=256, bx=8, b=8, box_lo=-10.0, box_hi=10.0, accelerated=1), lr=1e-4,
