@@ -61,6 +61,12 @@ def _problem(name):
             _PROBLEMS[name] = synth.dense_bf16_logistic(300, 301, 63)         # rows off the 16-byte grid: scalar path
         elif name == "dense8":
             _PROBLEMS[name] = synth.dense_logistic(400, 256, 64)              # vector path for fp32 features
+        elif name == "dense_wide":
+            _PROBLEMS[name] = synth.dense_logistic(300, 8192, 65)             # the largest model the one-cluster kernel takes
+        elif name == "dense_tiny":
+            _PROBLEMS[name] = synth.dense_logistic(64, 7, 66)                 # less than one group of eight coordinates
+        elif name == "csr_small":
+            _PROBLEMS[name] = synth.sparse_logistic(2000, 3001, 20.0, 1.1, 67)
         elif name == "c1":
             _PROBLEMS[name] = synth.config1()
         elif name == "c2":
@@ -420,6 +426,34 @@ def test_lockstep_sequential_master(dq, name, kw):
         for t in range(6):
             ls.round(rnd, 0.05 if acc else 0.3, theta)
             rnd += 1
+    ls.close()
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("dense_wide", dict(M=16, B=4, bx=8, b=4, lambda1=1e-5, seed=51)),          # sixteen blocks: the largest (non-portable) cluster
+    ("dense_wide", dict(M=1, B=40, bx=4, b=8, lambda2=1e-3, seed=52)),          # a cluster of one block, more rows than warps
+    ("dense_tiny", dict(M=2, B=3, bx=2, b=2, box_lo=-0.3, box_hi=0.3, seed=53)),
+    ("csr_small", dict(M=16, B=70, bx=8, b=2, lambda1=1e-5, seed=54)),          # more rows than 16-lane groups in a block
+    ("csr_small", dict(M=7, B=5, bx=2, b=8, lambda2=1e-4, accelerated=1, seed=55)),
+])
+def test_lockstep_cluster_kernel_shapes(dq, name, kw):
+    """The one-cluster round kernel at the edges of what it takes: 1, 7 and 16 blocks, the largest model, a model
+    shorter than one group, minibatches larger than a block's warps, every pairing of narrow and wide codes."""
+    h = _problem(name)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 86, 0.05), **kw)
+    acc = bool(kw.get("accelerated", 0))
+    l0 = dq.dq_launch_count(ls.ctx)
+    rnd = 0
+    for epoch in range(2):
+        theta = F32(0.5) if acc else F32(0.0)
+        ls.epoch(theta)
+        l0 = dq.dq_launch_count(ls.ctx)
+        for t in range(5):
+            ls.round(rnd, 0.05 if acc else 0.4, theta)
+            rnd += 1
+        if epoch == 1:
+            assert dq.dq_launch_count(ls.ctx) - l0 <= 5 + 4                     # one launch per round (plus a snapshot round's few)
+    assert ls.far_flips == 0
     ls.close()
 
 
