@@ -357,11 +357,20 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
     ctx->use_slots = false;
     ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = false;
+    const BitsArgs ba = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag,
+                         sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b, (adaptive && !flag) ? ctx->bx_dev : nullptr};
+    // dense messages and an averaged master: quantiser and master step share one kernel (the codes would only travel
+    // to memory and back between them)
+    const bool merged = rc == DQ_OK && quantize_master_applies(ctx);
+    if (merged) {
+        launch_quantize_master(ctx, ctx->alpha, reinterpret_cast<const uint32_t*>(ctx->ninf), round, &ctx->msgs, s, eta, theta,
+                               as_stream(st), (bits_down || bits_up) ? &ba : nullptr);
+        ctx->list_ready = false; ctx->normx_zeroed = false;
+        return last_error();
+    }
     if (rc == DQ_OK) rc = dq_quantize_sparsify_pack(ctx, ctx->alpha, ctx->ninf, round, &ctx->msgs, st);
     ctx->list_ready = false;
     if (rc != DQ_OK) { ctx->normx_zeroed = false; return rc; }
-    const BitsArgs ba = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag,
-                         sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b, (adaptive && !flag) ? ctx->bx_dev : nullptr};
     launch_master(ctx, &ctx->msgs, sparse_messages(ctx), s, eta, theta, as_stream(st), (bits_down || bits_up) ? &ba : nullptr);
     ctx->normx_zeroed = false;
     return last_error();

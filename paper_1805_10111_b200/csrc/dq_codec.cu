@@ -661,6 +661,86 @@ tile_ptr_kernel(const uint32_t* __restrict__ idx, int64_t cap, const uint32_t* _
 // Master step: g = (1/M) sum_w code_w delta_w (fused multiply-adds in worker order), u = g + g_full,
 // prox step on x (Algorithms 1/2) or on y with the momentum combination (Algorithm 3), ||x||_inf.
 // ---------------------------------------------------------------------------------------------------
+// Quantise + pack + master step in one kernel (dense messages, averaged master).  Between the workers'
+// quantiser and the master's unpack the codes would only travel to memory and back.  A block owns a tile of
+// kQmTile model coordinates: its threads first quantise the tile for every worker (one group of eight coordinates of
+// one worker per task: same draws and codes as quantize_pack_kernel, written out as the packed messages of Section
+// 3.1) and leave the codes in shared memory; then each thread takes one coordinate, adds code * delta in worker
+// order and applies the prox step (Algorithm 1 steps 12 and 9; Algorithm 3 step 9).  norm_bits [M] are the
+// workers' ||alpha_w||_inf.  grid = tiles covering the zero padding of the packed messages; M <= kQmMaxWorkers.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kQmTile = 256;
+constexpr int kQmMaxWorkers = 128;
+
+template <int BITS, bool ACC>
+__global__ void __launch_bounds__(kThreads)
+quantize_master_kernel(const float* __restrict__ v, int64_t d, int M, int vec_ok, const uint32_t* __restrict__ norm_bits,
+                       uint8_t* __restrict__ codes, int64_t stride, float* __restrict__ scale,
+                       const __grid_constant__ PhiloxKeys K, uint32_t round, int64_t ngroups, int* __restrict__ status,
+                       const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
+                       const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
+                       uint32_t* __restrict__ normx_bits, const RoundParams* __restrict__ rp, BitsArgs ba)
+{
+    pdl_prologue();
+    if (rp) { round = rp->round; eta = rp->eta; theta = rp->theta; }
+    if (ba.down && blockIdx.x == 0 && threadIdx.x == 0) write_round_bits(ba, M, d);
+    extern __shared__ float s_q[];                           // [M] 1/delta_w rounded toward zero, [M] delta_w, [M][kQmTile] codes
+    float* s_inv = s_q; float* s_delta = s_q + M;
+    int8_t* s_code = reinterpret_cast<int8_t*>(s_q + 2 * M);
+    for (int w = threadIdx.x; w < M; w += blockDim.x) {
+        const uint32_t nb = norm_bits[w];
+        const bool ok = nb < 0x7F800000u && nb != 0u;
+        s_inv[w] = ok ? __fdiv_rd((float)levels(BITS), __uint_as_float(nb)) : 0.0f;
+        s_delta[w] = ok ? __fdiv_rn(__uint_as_float(nb), (float)levels(BITS)) : 0.0f;
+        if (blockIdx.x == 0) { scale[w] = s_delta[w]; if (nb >= 0x7F800000u) set_status(status, DQ_ERR_NONFINITE); }
+    }
+    __syncthreads();
+    constexpr int GT = kQmTile / 8;                          // groups per tile
+    const int64_t g_first = (int64_t)blockIdx.x * GT;
+    for (int task = threadIdx.x; task < M * GT; task += blockDim.x) {
+        const int w = task / GT, gl = task - w * GT;
+        const int64_t g = g_first + gl, i0 = g << 3;
+        uint32_t s[8];
+        if (g < ngroups) {
+            float a[8];
+            const float* row = v + (int64_t)w * d;
+            if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+            uint32_t r[4];
+            philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamGrad, K, r);
+            const float inv = s_inv[w];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+            store_group<BITS>(codes + (int64_t)w * stride + g * BITS, pack8<BITS>(s));
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = 128u << 16;
+        }
+        // the eight codes as bytes (code + 128 sits in byte 2 of each word)
+        const uint32_t lo = __byte_perm(__byte_perm(s[0], s[1], 0x0062), __byte_perm(s[2], s[3], 0x0062), 0x5410) ^ 0x80808080u;
+        const uint32_t hi = __byte_perm(__byte_perm(s[4], s[5], 0x0062), __byte_perm(s[6], s[7], 0x0062), 0x5410) ^ 0x80808080u;
+        *reinterpret_cast<uint2*>(s_code + (int64_t)w * kQmTile + gl * 8) = make_uint2(lo, hi);
+    }
+    __syncthreads();
+    const float inv_m = __fdiv_rn(1.0f, (float)M);
+    const float thr = __fmul_rn(eta, pp.lambda1), den = __fadd_rn(1.0f, __fmul_rn(eta, pp.lambda2));
+    uint32_t nmax = 0;
+    const int64_t i = (int64_t)blockIdx.x * kQmTile + threadIdx.x;
+    if (i < d) {
+        float* target = ACC ? y : x;
+        const float gf = g_full[i], cur = target[i];
+        const float xs = ACC ? xsnap[i] : 0.0f;
+        float sm = ACC ? xsum[i] : 0.0f, yo = 0.0f, acc = 0.0f;
+#pragma unroll 4
+        for (int w = 0; w < M; ++w) acc = __fmaf_rn((float)s_code[w * kQmTile + threadIdx.x], s_delta[w], acc);
+        const float xo = master_update<ACC>(acc, inv_m, eta, theta, thr, den, pp, gf, cur, xs, yo, sm);
+        x[i] = xo;
+        if (ACC) { y[i] = yo; xsum[i] = sm; }
+        nmax = __float_as_uint(xo) & 0x7FFFFFFFu;
+    }
+    block_atomic_max(nmax, normx_bits);
+}
+
+// ---------------------------------------------------------------------------------------------------
 // acc[j] = fma(code_j, delta, acc[j]) for the 32/BITS codes of one packed word.  The integer-to-float
 // conversion avoids the conversion pipe: the code, biased by 2^(BITS-1), is placed in the mantissa of 2^23
 // (one byte permute) and the bias is subtracted exactly.
@@ -1450,6 +1530,40 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
             flags, M)));
         ctx->launches += 2;
     }
+}
+
+// Quantiser and master step of a round in one kernel (dense messages, averaged master): the context's message buffers
+// receive the packed codes and scales as from launch_quantize_pack followed by launch_master.
+bool quantize_master_applies(const dq_ctx* ctx)
+{
+    const dq_config& c = ctx->cfg;
+    // the tile's codes of all workers sit in shared memory; very large models gain nothing from sharing a kernel
+    return !c.sparsify && !c.sequential && !c.no_fused && c.M <= kQmMaxWorkers && c.d <= ((int64_t)1 << 22);
+}
+
+void launch_quantize_master(dq_ctx* ctx, const float* v, const uint32_t* norm_bits, uint32_t round, const dq_msgs* msgs, dq_state* s,
+                            float eta, float theta, cudaStream_t st, const BitsArgs* bits)
+{
+    BitsArgs ba = {nullptr, nullptr, nullptr, 0, 0, 0, 0};
+    if (bits) ba = *bits;
+    const dq_config& c = ctx->cfg;
+    const int64_t d = c.d;
+    ProxParams pp{c.lambda1, c.lambda2, c.box_lo, c.box_hi};
+    uint32_t* nx = reinterpret_cast<uint32_t*>(s->norm_x);
+    if (!ctx->normx_zeroed) cudaMemsetAsync(nx, 0, sizeof(uint32_t), st);
+    const int64_t ngroups = dq_packed_bytes(d, c.b) / c.b;
+    const int grid = (int)((ngroups * 8 + kQmTile - 1) / kQmTile);
+    const size_t smem = sizeof(float) * 2 * c.M + (size_t)c.M * kQmTile;
+    if (c.accelerated) {
+        DQ_DISPATCH_BITS(c.b, (launch_k(quantize_master_kernel<BITS_, true>, grid, kThreads, smem, st, v, d, c.M, vec_ok_for(v, d), norm_bits,
+            msgs->codes, msgs->stride, msgs->scale, ctx->keys, round, ngroups, ctx->status, s->g_full, s->x, s->y, s->x_snap, s->x_sum,
+            eta, theta, pp, nx, ctx->rp_active, ba)));
+    } else {
+        DQ_DISPATCH_BITS(c.b, (launch_k(quantize_master_kernel<BITS_, false>, grid, kThreads, smem, st, v, d, c.M, vec_ok_for(v, d), norm_bits,
+            msgs->codes, msgs->stride, msgs->scale, ctx->keys, round, ngroups, ctx->status, s->g_full, s->x, s->y, s->x_snap, s->x_sum,
+            eta, theta, pp, nx, ctx->rp_active, ba)));
+    }
+    ctx->launches += 1;
 }
 
 void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,

@@ -20,6 +20,9 @@ void launch_clear_listed(dq_ctx* ctx, cudaStream_t st);
 void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st);
 void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state* s, float eta, float theta, cudaStream_t st,
                    const BitsArgs* bits = nullptr);
+bool quantize_master_applies(const dq_ctx* ctx);
+void launch_quantize_master(dq_ctx* ctx, const float* v, const uint32_t* norm_bits, uint32_t round, const dq_msgs* msgs, dq_state* s,
+                            float eta, float theta, cudaStream_t st, const BitsArgs* bits = nullptr);
 void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, float* out, cudaStream_t st);
 
 // gradients (dq_grad.cu)
