@@ -424,8 +424,12 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
         if (!same && capture_round(ctx, s, bits_down, bits_up) != DQ_OK) ctx->graph_off = true;   // fall back to direct launches
         if (!ctx->graph_off) {
             cudaStream_t st = as_stream(stream);
-            launch_set_round_params(ctx, round, eta, theta, st);    // scalars travel as kernel arguments: no host buffer to keep alive
+            // the round's last kernel advances the round number on the device: only a jump in the numbering or new
+            // step sizes need the launch that sets them (scalars travel as kernel arguments: no host buffer to keep alive)
+            if (!(ctx->rp_host_valid && ctx->rp_host.round == round && ctx->rp_host.eta == eta && ctx->rp_host.theta == theta))
+                launch_set_round_params(ctx, round, eta, theta, st);
             if (cudaGraphLaunch(ctx->graph_exec, st) != cudaSuccess) return DQ_ERR_CUDA;
+            ctx->rp_host = dq::RoundParams{round + 1u, eta, theta, 0u}; ctx->rp_host_valid = true;
             ctx->launches += ctx->graph_launches;
             replayed = true;
         }

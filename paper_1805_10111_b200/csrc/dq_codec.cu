@@ -738,6 +738,7 @@ quantize_master_kernel(const float* __restrict__ v, int64_t d, int M, int vec_ok
         nmax = __float_as_uint(xo) & 0x7FFFFFFFu;
     }
     block_atomic_max(nmax, normx_bits);
+    finish_round(rp);
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -909,6 +910,7 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
         }
     }
     block_atomic_max(nmax, normx_bits);
+    finish_round(rp);
 }
 
 // Sparse messages.  One block per tile of kChunk coordinates: the tile's sum is built in shared memory
@@ -964,6 +966,7 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
         __syncthreads();
     }
     block_atomic_max(nmax, normx_bits);
+    finish_round(rp);
 }
 
 // The 32/BITS codes of one packed word as floats (same conversion-free trick as accumulate_word).
@@ -1072,6 +1075,7 @@ master_dense_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, const
         }
     }
     block_atomic_max(nmax, normx_bits);
+    finish_round(rp);
 }
 
 // Sparse messages, sequential: per tile, every worker's (possibly empty) message is expanded into shared memory and
@@ -1142,6 +1146,7 @@ master_sparse_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, cons
         __syncthreads();
     }
     block_atomic_max(nmax, normx_bits);
+    finish_round(rp);
 }
 
 // Test utility: dequantise one message into a dense fp32 vector.

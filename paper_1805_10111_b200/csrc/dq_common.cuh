@@ -231,6 +231,18 @@ __device__ __forceinline__ void write_round_bits(const BitsArgs& ba, int M, int6
 // Per-round scalars kept in device memory so that a captured graph of a round can be replayed unchanged.
 struct RoundParams { uint32_t round; float eta; float theta; uint32_t pad; };
 
+// Last statement of the kernel that ends a replayed round: the block that finishes last advances the round number
+// held on the device (no block reads it afterwards), so that consecutive rounds need no launch that sets it.
+// pad counts the blocks that have finished.
+__device__ __forceinline__ void finish_round(const RoundParams* rp)
+{
+    if (rp && threadIdx.x == 0) {
+        RoundParams* p = const_cast<RoundParams*>(rp);
+        __threadfence();
+        if (atomicAdd(&p->pad, 1u) == gridDim.x * gridDim.y * gridDim.z - 1u) { p->pad = 0u; p->round += 1u; }
+    }
+}
+
 #define DQ_DISPATCH_BITS(bits, CALL)                 \
     switch (bits) {                                  \
         case 2: { constexpr int BITS_ = 2; CALL; } break; \
@@ -280,6 +292,7 @@ struct dq_ctx {
     // replay of whole rounds: per-round scalars on the device and the captured graph of a non-flag round
     dq::RoundParams* rp_dev;
     const dq::RoundParams* rp_active;   // non-null while a round is being captured
+    dq::RoundParams rp_host; bool rp_host_valid;   // what rp_dev holds once the work enqueued so far has run
     cudaStream_t cap_stream;
     cudaGraphExec_t graph_exec;
     dq_state graph_state;

@@ -529,11 +529,13 @@ def test_graph_replay_equals_direct_launches(dq, name, kw):
     ("dense8", dict(M=4, B=16, bx=8, b=4, lambda2=1e-4, accelerated=1, seed=32)),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=33)),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, seed=34)),
+    ("bf16", dict(M=3, B=70, bx=8, b=8, box_lo=-1.0, box_hi=1.0, accelerated=1, seed=35)),
+    ("bf16", dict(M=3, B=16, bx=5, b=4, lambda2=1e-4, sequential=1, seed=36)),
 ])
 def test_rounds_in_one_call_equal_single_rounds(dq, name, kw):
     """dq_rounds(n) must leave what n calls of dq_round leave.  The first three problems run in the one-cluster
-    kernel (one launch for all rounds after the snapshot round); the sparsified one takes the general path.  Dense
-    gradients are summed in a fixed order, so those runs agree bit for bit; CSR gradients use float atomics."""
+    kernel (one launch for all rounds after the snapshot round); the others take the kernel chain.  Dense gradients are summed in a fixed order, so those runs agree bit for
+    bit; CSR gradients use float atomics."""
     import torch
     h = _problem(name)
     data = dq.Data(h)
@@ -551,12 +553,12 @@ def test_rounds_in_one_call_equal_single_rounds(dq, name, kw):
             assert dq.dq_epoch_begin(ctx, st, theta) == 0
             if batched:
                 l0 = dq.dq_launch_count(ctx)
-                assert dq.dq_rounds(ctx, st, rnd, 7, eta, theta, bits[0:1], bits[1:2]) == 0
-                if not kw.get("sparsify") and not (acc and epoch > 0):
+                assert dq.dq_rounds(ctx, st, rnd, 19, eta, theta, bits[0:1], bits[1:2]) == 0
+                if name != "bf16" and not kw.get("sparsify") and not (acc and epoch > 0):
                     assert dq.dq_launch_count(ctx) - l0 < 7 + 6        # a snapshot round by kernels, then one launch
-                rnd += 7
+                rnd += 19
             else:
-                for t in range(7):
+                for t in range(19):
                     assert dq.dq_round(ctx, st, rnd, eta, theta, bits[0:1], bits[1:2]) == 0
                     rnd += 1
         assert dq.dq_poll_status(ctx) == (0, 0)
