@@ -113,8 +113,6 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     const bool sparse = cfg->sparsify && cfg->msg_format == DQ_MSG_SPARSE;
     int rc = DQ_OK;
     rc |= dev_alloc(&c->norm_bits, M);
-    rc |= dev_alloc(&c->beta_norm_bits, M);
-    rc |= dev_alloc(&c->l1_sum, M);
     // offset table of the sparsifier: one entry per chunk; list mode uses chunks of 32 groups (256 coordinates)
     const int64_t chunk_slots = (d + 255) / 256 + 1;
     rc |= dev_alloc(&c->chunk_off, cfg->sparsify ? (size_t)M * chunk_slots : 1);
@@ -139,7 +137,14 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     rc |= dev_alloc(&c->bx_dev, 1);
     rc |= dev_alloc(&c->prec_stats, 11);
     rc |= dev_alloc(&c->delta_x, 1);
-    rc |= dev_alloc(&c->ninf, M);
+    // ||alpha_w||_inf, ||beta_w||_inf and the fixed-point ||alpha_w||_1 sit in one block so that one kernel of a round
+    // can clear all three: [M] float | [M] u32 | [M] u64
+    rc |= dev_alloc(&c->norm_block, (size_t)4 * M);
+    if (c->norm_block) {
+        c->ninf = reinterpret_cast<float*>(c->norm_block);
+        c->beta_norm_bits = c->norm_block + M;
+        c->l1_sum = reinterpret_cast<unsigned long long*>(c->norm_block + 2 * (size_t)M);
+    }
     if (data) {
         rc |= dev_alloc(&c->alpha, (size_t)M * d);
         rc |= dev_alloc(&c->rows, (size_t)M * cfg->B);
@@ -183,8 +188,8 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
 int dq_destroy(dq_ctx* c)
 {
     if (!c) return DQ_ERR_ARG;
-    void* ptrs[] = {c->norm_bits, c->beta_norm_bits, c->l1_sum, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->delays_dev, c->slots_dev, c->xnorm_bits, c->status, c->bits,
-                    c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->ninf, c->alpha,
+    void* ptrs[] = {c->norm_bits, c->norm_block, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->delays_dev, c->slots_dev, c->xnorm_bits, c->status, c->bits,
+                    c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->alpha,
                     c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
@@ -340,15 +345,16 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
         if (!adaptive) {
             launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, ctx->cfg.bx, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, ctx->cfg.bx),
                                  ctx->delta_x, round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
-                                 reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M);
+                                 reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.sparsify ? 4 * ctx->cfg.M : ctx->cfg.M);
         } else {     // condition (3): pick the width on the device, then launch the three specialised widths and the general kernel; all but one return at once
             launch_select_bits(ctx, s->x, s->x_snap, nx, ctx->cfg.mu, theta, ctx->bx_dev, ctx->prec_stats, as_stream(st));
             for (int bits : {2, 4, 8, 3})                      // 3 stands for "any other width": the general kernel reads it from the device
                 launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, bits, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, bits), ctx->delta_x,
                                      round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
-                                     reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.M, ctx->bx_dev);
+                                     reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.sparsify ? 4 * ctx->cfg.M : ctx->cfg.M, ctx->bx_dev);
         }
         ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = ctx->normx_zeroed = true;
+        ctx->sp_norms_zeroed = ctx->cfg.sparsify != 0;          // the same kernel cleared ||beta||_inf and ||alpha||_1
     } else if (adaptive) {
         cudaMemsetAsync(ctx->bx_dev, 0, sizeof(int32_t), as_stream(st));
     }

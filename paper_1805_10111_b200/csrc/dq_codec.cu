@@ -56,7 +56,7 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
         const int64_t nth0 = (int64_t)gridDim.x * gridDim.y * blockDim.x;
         const int64_t tid0 = ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
         for (int64_t i = tid0; i < zero_n; i += nth0) zero_f[i] = 0.0f;
-        if (tid0 < zero_un) zero_u[tid0] = 0u;
+        for (int64_t i = tid0; i < zero_un; i += nth0) zero_u[i] = 0u;
     }
     const int w = blockIdx.y;
     const uint32_t nb = norm_bits[w];
@@ -525,9 +525,14 @@ sparsify_count_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
 // messages that exceed the capacity (their tail is dropped).
 __global__ void __launch_bounds__(kThreads)
 chunk_scan_kernel(uint32_t* __restrict__ chunk_off, int64_t nchunks, int64_t cap, uint32_t* __restrict__ nnz,
-                  int* __restrict__ status)
+                  int* __restrict__ status, uint8_t* __restrict__ clear_codes = nullptr /* [M][stride]: zeroed here if given */,
+                  int64_t stride = 0)
 {
     pdl_prologue();
+    if (clear_codes) {
+        uint4* row = reinterpret_cast<uint4*>(clear_codes + (int64_t)blockIdx.x * stride);      // stride is a multiple of 16
+        for (int64_t q = threadIdx.x; q < (stride >> 4); q += blockDim.x) row[q] = make_uint4(0u, 0u, 0u, 0u);
+    }
     uint32_t* off = chunk_off + (int64_t)blockIdx.x * (nchunks + 1);
     __shared__ uint32_t s_warp[kThreads / 32];
     // each thread owns a contiguous run of entries: local sum, one block-wide scan of the sums, local prefix
@@ -949,7 +954,7 @@ master_sparse_kernel(const uint8_t* __restrict__ codes, int64_t stride, const fl
                 const int64_t bit = (int64_t)e * BITS;
                 const int k = code_of<BITS>(__ldg(words + (bit >> 5)), (int)((bit & 31) / BITS));
                 const int li = (int)((int64_t)list[e] - lo);
-                s_acc[li] = __fmaf_rn((float)k, dl, s_acc[li]);
+                if ((unsigned)li < (unsigned)kChunk) s_acc[li] = __fmaf_rn((float)k, dl, s_acc[li]);     // a list entry outside its tile is dropped, never followed
             }
             __syncthreads();
         }
@@ -1341,7 +1346,7 @@ quantize_pack_any_kernel(const float* __restrict__ v, int64_t d, const uint32_t*
     const int64_t nth = (int64_t)gridDim.x * blockDim.x, tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (diff) {
         for (int64_t i = tid; i < zero_n; i += nth) zero_f[i] = 0.0f;
-        if (tid < zero_un) zero_u[tid] = 0u;
+        for (int64_t i = tid; i < zero_un; i += nth) zero_u[i] = 0u;
     }
     const uint32_t nb = norm_bits[0];
     const float nrm = __uint_as_float(nb);
@@ -1489,8 +1494,9 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     // step in list mode, where the work is small and parallelism matters more than the size of the offset table
     const int iters = list ? 1 : kChunk / 256;
     const int64_t nchunks = list ? (ctx->glist_cap + 31) / 32 : (d + kChunk - 1) / kChunk;
-    cudaMemsetAsync(ctx->l1_sum, 0, sizeof(unsigned long long) * M, st);
-    cudaMemsetAsync(ctx->beta_norm_bits, 0, sizeof(uint32_t) * M, st);
+    if (!(ctx->sp_norms_zeroed && v == ctx->alpha))           // both live in one block behind ninf: one clear covers them
+        cudaMemsetAsync(ctx->beta_norm_bits, 0, sizeof(uint32_t) * M + sizeof(unsigned long long) * M, st);
+    ctx->sp_norms_zeroed = false;
     if (list) {
         launch_k(norm_l1_list_kernel, dim3(16, M), kThreads, 0, st, v, d, vec_ok, gl, norm_bits, ctx->l1_sum);
     } else {
@@ -1502,8 +1508,7 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     if (list) {
         launch_k(sparsify_count_kernel, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round,
                                                            ctx->beta_norm_bits, ctx->chunk_off, nchunks, ctx->rp_active, gl, iters);
-        launch_k(chunk_scan_kernel, M, kThreads, 0, st, ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
-        cudaMemsetAsync(out->codes, 0, (size_t)out->stride * M, st);
+        launch_k(chunk_scan_kernel, M, kThreads, 0, st, ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status, out->codes, out->stride);
         DQ_DISPATCH_BITS(bits, (launch_k(sparsify_emit_kernel<BITS_, true>, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,
             nchunks, 0, out->codes, out->stride, out->scale, out->idx, out->cap, ctx->status, ctx->rp_active, gl, iters, nullptr, 0)));
         ctx->launches += 4;
@@ -1520,7 +1525,7 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     ctx->launches += 2;
     dim3 grid_f(grid_for(nchunks * 8, ctx->sm_count), M);
     if (sparse_out) {
-        launch_k(chunk_scan_kernel, M, kThreads, 0, st, ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status);
+        launch_k(chunk_scan_kernel, M, kThreads, 0, st, ctx->chunk_off, nchunks, out->cap, out->nnz, ctx->status, nullptr, 0);
         DQ_DISPATCH_BITS(bits, (launch_k(sparsify_finish_sparse_kernel<BITS_>, grid_f, kThreads, 0, st, norm_bits, ctx->beta_norm_bits, ctx->keys, round, ctx->chunk_off, nchunks, sb, out->codes, out->stride, out->scale,
             out->idx, out->cap, ctx->status, ctx->rp_active)));
         DQ_DISPATCH_BITS(bits, (launch_k(sparsify_emit_kernel<BITS_, true>, grid_c, kThreads, 0, st, v, d, vec_ok, norm_bits, ctx->l1_sum, ctx->cfg.phi, ctx->keys, round, ctx->beta_norm_bits, ctx->chunk_off,

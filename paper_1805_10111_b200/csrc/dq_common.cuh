@@ -150,14 +150,15 @@ __device__ __forceinline__ void block_atomic_max(uint32_t v, uint32_t* dst)
     }
 }
 
-// Programmatic dependent launch.  Every kernel of the library begins with pdl_prologue(): it lets the next kernel
-// of the stream be scheduled as soon as all blocks of this one are resident (its blocks take the slots that free up
-// while this grid drains), then waits until the kernels before this one have completed and their writes are
-// visible.  Nothing before the wait may touch global memory.  In a kernel launched without the attribute both
-// instructions do nothing.
+// Programmatic dependent launch.  Every launch of the library carries the programmatic-serialization attribute and
+// every kernel begins with pdl_prologue(), which waits until the kernel before it has completed and its writes are
+// visible; nothing before the wait may touch global memory.  No kernel signals its dependents early
+// (griddepcontrol.launch_dependents): a dependent's wait is released by that signal, not by the end of the grid, so
+// whatever a kernel wrote after signalling was read stale by its successor (seen with a small scan kernel between
+// two larger ones).  Without the signal the successor is released when the last block of this grid exits.
+// In a kernel launched without the attribute the instruction does nothing.
 __device__ __forceinline__ void pdl_prologue()
 {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
@@ -261,6 +262,8 @@ struct dq_ctx {
     int sm_count;
     // scratch owned by the context
     uint32_t* norm_bits;        // [M]   ||v_w||_inf bit patterns when the caller supplies none
+    uint32_t* norm_block;       // owner of ninf, beta_norm_bits and l1_sum (contiguous)
+    bool sp_norms_zeroed;       // an earlier kernel of this round already cleared beta_norm_bits and l1_sum
     uint32_t* beta_norm_bits;   // [M]   ||beta_w||_inf over survivors
     unsigned long long* l1_sum; // [M]   fixed-point ||alpha_w||_1
     uint32_t* chunk_off;        // [M][nchunks + 1] survivors per chunk, then their exclusive prefix
