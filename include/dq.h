@@ -183,8 +183,10 @@ int dq_master_unpack_aggregate_prox(dq_ctx* ctx, const dq_msgs* msgs, dq_state* 
  * The round is a snapshot round when snapshot_flag is set and it is the first round after dq_epoch_begin
  * (Algorithm 3: of the first epoch only).
  * Unless no_graph is set, the first non-snapshot round on a given set of state/counter pointers records its
- * kernel sequence as a CUDA graph (this allocates); later rounds copy (round, eta, theta) to the device and
- * replay it.  Calling with other pointers records again.
+ * kernel sequence as a CUDA graph (this allocates); later rounds replay it.  The graph's kernels read (round,
+ * eta, theta) from device memory, where the round's last kernel advances the round number, so consecutive rounds
+ * with the same step sizes cost one graph launch; anything else costs one small kernel that sets the three values.
+ * Calling with other pointers records again.
  * Small problems (logistic model on DENSE_F32 or CSR_F32 data, dense messages, synchronous master, fixed b_x,
  * d <= 8192, M <= 16, B <= 1024) skip the graph unless no_fused is set: their non-snapshot rounds run in ONE
  * kernel on one thread-block cluster (block w is worker w; the blocks meet at the cluster barrier around the
