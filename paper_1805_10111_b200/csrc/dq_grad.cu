@@ -13,11 +13,20 @@ constexpr int kRowsPerBlock = 16;   // rows of one worker handled by one block o
 
 __device__ __forceinline__ float sigmoidf_(float t) { return __fdiv_rn(1.0f, 1.0f + expf(-t)); }
 
-// slope(z) = d/dz log(1+exp(-y z)) = -y sigma(-y z).  The worker needs slope(zs + dz) - slope(zs); written
-// as y * sigma(-y (zs+dz)) * sigma(y zs) * expm1(y dz) it has no cancellation when dz is small.
+// slope(z) = d/dz log(1+exp(-y z)) = -y sigma(-y z).  The worker needs slope(zs + dz) - slope(zs)
+// = y (sigma(-u) - sigma(-(u+t))) with u = y zs, t = y dz.  Written as y sigma(-(u+t)) sigma(u) expm1(t) it has no
+// cancellation when dz is small.  Outside the range where every factor of that product is an ordinary fp32 number:
+//   t > 16: the two sigmoids differ by a factor of exp(16) or more, so their plain difference is accurate; it is taken
+//           on the side where both are small (sigma(-a) = 1 - sigma(a)), so nothing is lost against a value near 1;
+//   0 < t <= 16 and u + t > 80: sigma(-(u+t)) would underflow; sigma(-(u+t)) expm1(t) = -expm1(-t) / (exp(-t) + exp(u))
+//           keeps every factor finite (an infinite exp(u) gives the correct limit 0).
 __device__ __forceinline__ float slope_difference(float y, float zs, float dz)
 {
-    return y * sigmoidf_(-y * (zs + dz)) * sigmoidf_(y * zs) * expm1f(y * dz);
+    const float t = y * dz, u = y * zs;
+    if (t > 16.0f)
+        return y * (u + 0.5f * t >= 0.0f ? sigmoidf_(-u) - sigmoidf_(-(u + t)) : sigmoidf_(u + t) - sigmoidf_(u));
+    if (t > 0.0f && u + t > 80.0f) return y * sigmoidf_(u) * __fdiv_rn(-expm1f(-t), expf(-t) + expf(u));
+    return y * sigmoidf_(-y * (zs + dz)) * sigmoidf_(u) * expm1f(t);
 }
 
 __device__ __forceinline__ double warp_sum(double v)

@@ -93,6 +93,31 @@ def _abs_grad_scale(h, x):
     return (S / h.n).astype(F32)
 
 
+def _row(h, a):
+    """(columns, values as float64) of data row a."""
+    if h.format == synth.CSR_F32:
+        k0, k1 = int(h.row_ptr[a]), int(h.row_ptr[a + 1])
+        return h.col_idx[k0:k1].astype(np.int64), h.values[k0:k1].astype(np.float64)
+    v = h.values[a] if h.format == synth.DENSE_F32 else synth.bf16_bits_to_f32(h.values[a])
+    return np.arange(h.d), v.astype(np.float64)
+
+
+def _margin_slack(h, rows, xhat, xsnap, rel=1e-5):
+    """What the conditioning of the margin difference adds to the tolerance scale S.  A worker's slope difference is a
+    function of dz = <a, xhat - xsnap> with |d slope / d dz| <= 1/4.  The differences xhat_i - xsnap_i are held in fp32 and
+    summed in fp32 (dense rows), so dz carries an absolute error of about 2^-24 rho_a, rho_a = sum_i |a_i| |xhat_i - xsnap_i|,
+    however small dz itself comes out when the terms cancel: a relative bound on dz, and so on the slope difference of
+    that row, does not exist.  Allowed here: 2^-23 rho_a / 4 per row on the slope, i.e. (1/B) sum_a |a_ai| 2^-23 rho_a / 4 on
+    coordinate i, returned in units of `rel` so that it can be added to S."""
+    diff = xhat.astype(np.float64) - xsnap.astype(np.float64)
+    slack = np.zeros(h.d)
+    for a in rows:
+        cols, vals = _row(h, int(a))
+        rho = np.abs(vals * diff[cols]).sum()
+        np.add.at(slack, cols, np.abs(vals) * (2.0 ** -25 * rho / len(rows)))
+    return (slack / rel).astype(np.float64)
+
+
 @pytest.mark.parametrize("name", ["dense", "csr", "bf16", "bf16odd", "dense8"])
 def test_epoch_begin_full_gradient(dq, name):
     import torch
@@ -193,6 +218,43 @@ def test_worker_gradient_large_minibatch(dq, name):
     dq.dq_destroy(ctx)
 
 
+@pytest.mark.parametrize("name", ["dense", "csr", "bf16", "dense8"])
+@pytest.mark.parametrize("B", [1, 37, 70])
+def test_worker_gradient_far_model(dq, name, B):
+    """A low-precision model far from the snapshot: margins move by hundreds, so exp(y dz) and exp(y (zs + dz)) leave the
+    fp32 range for many rows.  Every slope difference must still be finite and within tolerance (B = 1: a worker's whole
+    gradient is one row's slope difference, nothing averages an error away)."""
+    import torch
+    h = _problem(name)
+    M, seed, rnd, bx = 3, 23, 4, 8
+    xs = synth.normal_vector(h.d, 86, 0.3)
+    x = (xs + synth.normal_vector(h.d, 87, 100.0)).astype(F32)
+    cfg = dq.make_config(h.d, M, B=B, bx=bx, seed=seed)
+    data = dq.Data(h)
+    rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+    st = dq.State(xs, n=h.n)
+    assert dq.dq_epoch_begin(ctx, st) == 0
+    cx, dx, _ = oracle.quantize(x, bx, seed, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+    xhat = cx.astype(F32) * dx
+    alpha = torch.full((M, h.d), 3.0, device="cuda"); ninf = torch.zeros(M, device="cuda")
+    assert dq.dq_worker_grad(ctx, _dev(oracle.pack(cx, bx)), _dev(np.array([dx], F32)), 0, st, rnd, None, alpha, ninf) == 0
+    assert dq.dq_poll_status(ctx) == (0, 0)
+    a_gpu = alpha.cpu().numpy()
+    assert np.isfinite(a_gpu).all()
+    big = 0
+    for w in range(M):
+        rows = oracle.sample_batch(seed, rnd, w, M, h.n, B)
+        a, S = oracle.worker_grad(_odata(h), xhat, xs, rows)
+        nbad, worst = _close(a_gpu[w], a, S + _margin_slack(h, rows, xhat, xs))
+        assert nbad == 0, (w, nbad, worst)
+        assert ninf[w].item() == np.abs(a_gpu[w]).max()
+        for r_ in rows:
+            cols, vals = _row(h, int(r_))
+            big += abs(vals @ (xhat.astype(np.float64) - xs.astype(np.float64))[cols]) > 90.0
+    assert big > 0 or B == 1            # the case must reach the range where exp overflows in fp32
+    dq.dq_destroy(ctx)
+
+
 class Lockstep:
     """Runs the GPU library and the oracle side by side, restarting the GPU from the oracle's state every round."""
 
@@ -264,13 +326,18 @@ class Lockstep:
         raw_gpu = np.zeros((M, d), np.int32)
         round_flips = 0
         for w in range(M):
-            nbad, worst = _close(a_gpu[w], tr["alpha"][w], tr["S"][w])
+            S_w = tr["S"][w]
+            if cfg.model != dq.DQ_MODEL_MLP and not tr["flag_round"]:
+                used = tr["delays_used"][w] if delays is not None else 0
+                xhat_w = tr["xhat"] if used == 0 else run.broadcasts[len(run.broadcasts) - 1 - used]
+                S_w = S_w + _margin_slack(self.h, tr["rows"][w], xhat_w, run.xsnap)
+            nbad, worst = _close(a_gpu[w], tr["alpha"][w], S_w)
             self.worst_alpha = max(self.worst_alpha, worst)
             if nbad:
                 ora = tr["alpha"][w].astype(np.float64); err = np.abs(a_gpu[w].astype(np.float64) - ora)
-                sc = np.maximum(np.maximum(np.abs(ora), 1e-3 * np.abs(ora).max()), tr["S"][w])
+                sc = np.maximum(np.maximum(np.abs(ora), 1e-3 * np.abs(ora).max()), S_w)
                 for i in np.argsort(-(err / sc))[:4]:
-                    print("coordinate", int(i), "gpu", a_gpu[w][i], "oracle", tr["alpha"][w][i], "S", tr["S"][w][i], "scale", sc[i])
+                    print("coordinate", int(i), "gpu", a_gpu[w][i], "oracle", tr["alpha"][w][i], "S", S_w[i], "scale", sc[i])
             assert nbad == 0, ("alpha", rnd, w, nbad, worst)
             # the GPU's codes are exactly the oracle's quantiser applied to the GPU's gradient
             if cfg.sparsify:
@@ -338,6 +405,10 @@ class Lockstep:
     ("dense", dict(M=3, B=8, bx=5, b=8, lambda1=1e-4, seed=11), 0.5),
     ("csr", dict(M=4, B=16, bx=11, b=4, lambda2=1e-5, seed=12), 0.5),
     ("bf16", dict(M=4, B=16, bx=3, b=8, box_lo=-1.0, box_hi=1.0, seed=13), 0.01),
+    # one row per minibatch and a coarse model: a worker's whole gradient hangs on one margin difference
+    ("dense_wide", dict(M=16, B=1, bx=3, b=8, box_lo=-0.5, box_hi=2.0, seed=46, no_fused=1), 0.3),
+    ("csr", dict(M=16, B=1, bx=3, b=4, box_lo=-0.5, box_hi=0.5, seed=47), 0.3),
+    ("dense_tiny", dict(M=17, B=1, bx=6, b=4, box_lo=-2.0, box_hi=0.5, sparsify=1, phi=50.0, seed=48), 0.3),
 ])
 def test_lockstep_small(dq, name, kw, eta):
     h = _problem(name)
