@@ -201,11 +201,11 @@ __global__ void __launch_bounds__(kThreads) norm_l1_list_kernel(const float* __r
 }
 
 // Per-worker constants of eq. (4) with Lemma 2's probabilities, from the two norms.
-struct SparsifyScale { float s; bool empty; };
+struct SparsifyScale { float s; bool empty; bool s_inf; };   // s_inf: |alpha|_1 so small that s overflowed
 
 __device__ __forceinline__ SparsifyScale sparsify_scale(uint32_t nb, unsigned long long l1, float phi)
 {
-    SparsifyScale r; r.s = 0.0f; r.empty = true;
+    SparsifyScale r; r.s = 0.0f; r.empty = true; r.s_inf = false;
     if (nb == 0u || nb >= 0x7F800000u) return r;
     const float ninf = __uint_as_float(nb);
     int e; (void)frexpf(ninf, &e);
@@ -213,7 +213,7 @@ __device__ __forceinline__ SparsifyScale sparsify_scale(uint32_t nb, unsigned lo
     if (n1 == 0.0f) return r;
     const float cap = __fdiv_rn(n1, ninf);                       // Lemma 2: phi <= |alpha|_1 / |alpha|_inf
     const float phi_eff = (phi > 0.0f) ? fminf(phi, cap) : cap;
-    r.s = __fdiv_rn(phi_eff, n1); r.empty = false;
+    r.s = __fdiv_rn(phi_eff, n1); r.empty = false; r.s_inf = r.s > 3.4028234e38f;
     return r;
 }
 
@@ -247,7 +247,8 @@ __device__ __forceinline__ uint32_t sparsify8(const float (&a)[8], float s, cons
 // The survivor mask without float compares or selects.  u < y for an integer draw u is u < ceil(y); adding 2^23 to
 // y with rounding toward +inf leaves ceil(y) in the significand (y <= 2^16 (1 + ulp) because phi is clamped to
 // |alpha|_1 / |alpha|_inf), the draw is placed under the same exponent with one logic operation, and the sign of
-// the difference of the two words is shifted into the mask.  Same mask as sparsify8.
+// the difference of the two words is shifted into the mask.  Same mask as sparsify8 for every y that is a number
+// (a zero coordinate under an infinite s gives a NaN: the caller clears those bits).
 __device__ __forceinline__ uint32_t mask8(const float (&a)[8], float s, const uint32_t (&r)[4])
 {
     uint32_t mask = 0;
@@ -335,7 +336,11 @@ sparsify_stage_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
         uint32_t ra[4], rb[4];
         philox4x32_10(g, round, (uint32_t)w, kStreamMask, K, ra);
         philox4x32_10(g + 32u, round, (uint32_t)w, kStreamMask, K, rb);
-        const uint32_t ma = mask8(a, sc.s, ra), mb = mask8(b, sc.s, rb);
+        uint32_t ma = mask8(a, sc.s, ra), mb = mask8(b, sc.s, rb);
+        if (sc.s_inf) {                       // 0 * inf is a NaN, which mask8's integer test would take for a survivor
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { if (a[j] == 0.0f) ma &= ~(1u << j); if (b[j] == 0.0f) mb &= ~(1u << j); }
+        }
         const uint32_t anya = __ballot_sync(0xFFFFFFFFu, ma != 0u), anyb = __ballot_sync(0xFFFFFFFFu, mb != 0u);
         if (anya) collect(a, ma, anya, g);
         if (anyb) collect(b, mb, anyb, g + 32u);

@@ -277,6 +277,36 @@ def test_sparsify_beyond_the_staging_limits(dq, b, kind):
         assert any((c > 128).any() for c in per_chunk) and any(((c > 0) & (c <= 128)).any() for c in per_chunk)
 
 
+@pytest.mark.parametrize("b", [2, 8])
+@pytest.mark.parametrize("d", [1, 9, 4099])
+def test_sparsify_subnormal_vectors(dq, b, d):
+    """||alpha||_1 so small that phi / ||alpha||_1 overflows: every nonzero coordinate survives with p = 1, and a zero
+    coordinate (0 * inf) must not turn into a survivor, in either message format."""
+    g = np.random.default_rng(300 + d)
+    v = (g.integers(-3, 4, (3, d)) * np.float64(1.4e-45)).astype(F32)          # a few units of the smallest subnormal, and zeros
+    v[:, 0] = F32(4e-45)
+    want = _check_sparsify(dq, v, b, 0.0, 4242, 6)
+    for w in range(3):
+        assert np.array_equal(want[w]["Z"], v[w] != 0)
+
+
+def test_sparsify_survivor_overflow_is_reported(dq):
+    """A survivor alpha_i / p_i beyond the fp32 range: the oracle reports a non-finite vector, and so must the library."""
+    g = np.random.default_rng(301)
+    d, M, b, seed, rnd = 2049, 2, 4, 77, 9
+    v = (g.standard_normal((M, d)) * 1e-6).astype(F32)
+    v[0, 5] = F32(3e38); v[1, 2000] = F32(-3e38)
+    r = oracle.sparsify(v[0], 0.0, seed, rnd, 0)
+    assert oracle.quantize_survivors(r["beta"], r["Z"], b, seed, rnd, 0)[2] == dq.DQ_ERR_NONFINITE
+    for fmt in (dq.DQ_MSG_DENSE, dq.DQ_MSG_SPARSE):
+        cfg = dq.make_config(d, M, b=b, seed=seed, sparsify=1, phi=0.0, msg_format=fmt)
+        rc, ctx = dq.dq_create(cfg); assert rc == 0
+        msgs = dq.Msgs(cfg)
+        assert dq.dq_quantize_sparsify_pack(ctx, _dev(v), None, rnd, msgs) == 0
+        assert dq.dq_poll_status(ctx) == (0, dq.DQ_ERR_NONFINITE)
+        dq.dq_destroy(ctx)
+
+
 def test_sparse_capacity_overflow_is_reported(dq):
     d, M = 30000, 2
     v = _vectors(M, d, 3, outliers=False)
