@@ -248,7 +248,7 @@ __device__ __forceinline__ uint32_t sparsify8(const float (&a)[8], float s, cons
 // y with rounding toward +inf leaves ceil(y) in the significand (y <= 2^16 (1 + ulp) because phi is clamped to
 // |alpha|_1 / |alpha|_inf), the draw is placed under the same exponent with one logic operation, and the sign of
 // the difference of the two words is shifted into the mask.  Same mask as sparsify8 for every y that is a number
-// (a zero coordinate under an infinite s gives a NaN: the caller clears those bits).
+// (a zero coordinate under an infinite s gives a NaN: the stage kernel clears those bits before it counts).
 __device__ __forceinline__ uint32_t mask8(const float (&a)[8], float s, const uint32_t (&r)[4])
 {
     uint32_t mask = 0;
@@ -307,6 +307,11 @@ sparsify_stage_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
     uint32_t* di = nullptr; float* dv = nullptr;
     // survivors of one step (32 groups of eight coordinates, one per lane): positions in index order, then beta
     auto collect = [&](const float (&a)[8], uint32_t mask, uint32_t any, uint32_t g) {
+        if (sc.s_inf) {                       // 0 * inf is a NaN, which mask8's integer test takes for a survivor
+#pragma unroll
+            for (int j = 0; j < 8; ++j) if (a[j] == 0.0f) mask &= ~(1u << j);
+            any = __ballot_sync(0xFFFFFFFFu, mask != 0u);
+        }
         const uint32_t cnt = __popc(mask);
         uint32_t before, total;
         if (__ballot_sync(0xFFFFFFFFu, cnt > 1u) == 0u) {                         // at most one survivor per lane
@@ -336,11 +341,7 @@ sparsify_stage_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const 
         uint32_t ra[4], rb[4];
         philox4x32_10(g, round, (uint32_t)w, kStreamMask, K, ra);
         philox4x32_10(g + 32u, round, (uint32_t)w, kStreamMask, K, rb);
-        uint32_t ma = mask8(a, sc.s, ra), mb = mask8(b, sc.s, rb);
-        if (sc.s_inf) {                       // 0 * inf is a NaN, which mask8's integer test would take for a survivor
-#pragma unroll
-            for (int j = 0; j < 8; ++j) { if (a[j] == 0.0f) ma &= ~(1u << j); if (b[j] == 0.0f) mb &= ~(1u << j); }
-        }
+        const uint32_t ma = mask8(a, sc.s, ra), mb = mask8(b, sc.s, rb);
         const uint32_t anya = __ballot_sync(0xFFFFFFFFu, ma != 0u), anyb = __ballot_sync(0xFFFFFFFFu, mb != 0u);
         if (anya) collect(a, ma, anya, g);
         if (anyb) collect(b, mb, anyb, g + 32u);
