@@ -81,3 +81,63 @@ def test_random_configurations(dq, block):
             ls.close()
         except AssertionError as e:
             raise AssertionError("trial %d %s n=%d d=%d %r: %r" % (trial, kind, h.n, h.d, kw, e)) from e
+
+
+def test_random_configurations_every_chain_leaves_the_same_iterates(dq):
+    """The same rounds by single calls (graph replay), by dq_rounds in random chunks, without graphs, and as separate
+    kernels must leave the same bits in x (and y), the same ||x||_inf and the same bit counts.  Drawn among dense
+    problems whose gradient sums have a fixed order (one block of rows per worker, or the two-kernel column sums);
+    where the one-cluster kernel applies, the separate-kernel chain sums in another order and is left out."""
+    import torch
+    done = 0
+    for trial in range(200):
+        g = np.random.default_rng([1806, trial])
+        kind, h, kw, tau = draw_case(g)
+        for k in ("no_fused", "no_graph", "max_delay"):
+            kw.pop(k, None)
+        if kind == "csr":
+            continue                                               # float atomics
+        vec = (h.d % 4 == 0) if kind == "dense" else (h.d % 8 == 0)
+        if not (kw["B"] <= 16 or (vec and kw["B"] >= 64)):
+            kw["B"] = int(g.choice([1, 8, 16]))
+        cluster = (not kw.get("sparsify") and not kw.get("sequential") and kw.get("mu", 0.0) == 0.0 and kw["bx"] in (2, 4, 8)
+                   and h.d <= 8192 and kw["M"] <= 16)
+        acc = bool(kw.get("accelerated", 0))
+        theta, eta = (0.5, 0.02 if kind == "bf16" else 0.05) if acc else (0.0, 0.01 if kind == "bf16" else 0.3)
+        x0 = synth.normal_vector(h.d, int(g.integers(1, 1000)), 0.05)
+        data = dq.Data(h)
+        nr = int(g.integers(3, 25))
+        chunks, left = [], nr
+        while left > 0:
+            chunks.append(int(g.integers(1, left + 1))); left -= chunks[-1]
+        outs = {}
+        for variant in ("single", "batched", "no_graph") + (() if cluster else ("no_fused",)):
+            extra = {"no_graph": 1} if variant == "no_graph" else ({"no_fused": 1} if variant == "no_fused" else {})
+            cfg = dq.make_config(h.d, kw["M"], **{k: v for k, v in kw.items() if k != "M"}, **extra)
+            rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+            st = dq.State(x0, n=h.n, accelerated=acc)
+            bits = torch.zeros(2, dtype=torch.int64, device="cuda")
+            rnd = 0
+            for epoch in range(2):
+                assert dq.dq_epoch_begin(ctx, st, theta) == 0
+                if variant == "batched":
+                    for c in chunks:
+                        assert dq.dq_rounds(ctx, st, rnd, c, eta, theta, bits[0:1], bits[1:2]) == 0
+                        rnd += c
+                else:
+                    for t in range(nr):
+                        assert dq.dq_round(ctx, st, rnd, eta, theta, bits[0:1], bits[1:2]) == 0
+                        rnd += 1
+            assert dq.dq_poll_status(ctx) == (0, 0), (trial, variant)
+            outs[variant] = (st.x.cpu().numpy().copy(), st.norm_x.item(), bits.cpu().numpy().copy(),
+                             st.y.cpu().numpy().copy() if acc else None)
+            dq.dq_destroy(ctx)
+        ref = outs["single"]
+        for variant, o in outs.items():
+            where = (trial, variant, kind, h.d, kw, chunks)
+            assert np.array_equal(ref[0], o[0]) and ref[1] == o[1], where
+            assert np.array_equal(ref[2], o[2]), where
+            if acc:
+                assert np.array_equal(ref[3], o[3]), where
+        done += 1
+    assert done >= 100
