@@ -125,7 +125,13 @@ float dqo_scale_inv(float nrm, int b)
  * rounding): 15 fractional bits up to 8-bit codes, then 14, 13, 12.  Adding a
  * uniform integer of as many bits (the top bits of the coordinate's draw) and
  * dropping the fraction rounds up with probability frac(F)/2^(23-e).  Rule (ii)
- * (outside the hull: nearest end point of dom(delta,b)) is the clamp. */
+ * (outside the hull: nearest end point of dom(delta,b)) is the clamp.
+ * This fixed-point form IS the reading taken of rule (i)'s "with probability
+ * (x - z)/delta" (the paper gives no resolution for the draw); it cannot be
+ * checked against the rule by eye, so tests/test_oracle_philox_quantizer.py
+ * (test_q_code_is_stochastic_rounding_with_exact_probability) counts, over all
+ * 2^15 draws, how often a coordinate is rounded up and compares the count with
+ * frac(t) 2^15 computed from exact rationals. */
 int32_t dqo_q_code(float v, float inv, int b, uint32_t u15)
 {
     const int e = b <= 8 ? 8 : b, fbits = 23 - e;
@@ -245,9 +251,16 @@ int dqo_sparsify(const float* alpha, int64_t d, float phi, uint64_t seed, uint32
     float s = phi_eff / n1;
     if (phi_eff_out) *phi_eff_out = phi_eff;
     for (int64_t i = 0; i < d; ++i) {
-        float p = fabsf(alpha[i]) * s;
-        float scaled = ceilf(p * 65536.0f);                       /* exact power-of-two scaling */
-        uint32_t m = (scaled >= 65536.0f) ? 65536u : (uint32_t)scaled;
+        /* p_i * 2^16 rounded up, as an integer in 0..2^16.  A zero coordinate has p_i = 0 whatever s is and
+         * never survives; this is said first because with ||alpha||_1 subnormal s = phi/||alpha||_1 overflows
+         * to +inf and 0 * inf would be a NaN (no NaN may reach the integer conversion).  A nonzero coordinate
+         * under an overflowed s has p_i = inf, clamped to 1 like every p_i >= 1. */
+        float a = fabsf(alpha[i]);
+        uint32_t m = 0;
+        if (a != 0.0f) {
+            float scaled = ceilf((a * s) * 65536.0f);             /* exact power-of-two scaling */
+            m = (scaled >= 65536.0f) ? 65536u : (uint32_t)scaled;
+        }
         uint32_t u = dqo_u16(seed, round, worker, DQO_STREAM_MASK, (uint64_t)i);
         int z = (u < m);
         Z[i] = (uint8_t)z;

@@ -162,6 +162,37 @@ def test_sparsifier_probabilities_and_budget():
             assert m[i] == 65536 and Z[i] and beta[i] == alpha[i]        # equality budget keeps the max coordinate
 
 
+def test_sparsifier_subnormal_vectors_exact():
+    """eq. (4) on vectors whose l1 norm is a subnormal number, against exact rationals.  (a) phi/|alpha|_1 still a finite
+    fp32 number: every p_i 2^16 equals Lemma 2's value computed with fractions.  (b) phi/|alpha|_1 beyond the fp32
+    range: a zero coordinate has p_i = 0 and never survives, a nonzero one has p_i = 1 (eq. (4) allows any
+    0 < p_i <= 1), so beta = alpha; no NaN reaches a code, a mask bit or a norm."""
+    sub = lambda k, e: F32(math.ldexp(float(k), e))
+    # (a) |alpha|_1 = 2^-127 (subnormal), budget 1: s = 2^127 is finite
+    alpha = np.array([sub(1, -128), 0.0, sub(-1, -129), sub(1, -129), 0.0], F32)
+    r = oracle.sparsify(alpha, 1.0, 4, 2, 1)
+    n1 = sum(Fraction(abs(float(t))) for t in alpha)
+    assert r["status"] == 0 and Fraction(float(r["n1"])) == n1 == Fraction(1, 2 ** 127) and r["phi_eff"] == 1.0
+    want_m = [math.ceil(Fraction(abs(float(t))) * 1 / n1 * 65536) for t in alpha]          # p_i = |alpha_i| phi / |alpha|_1
+    assert list(r["m"]) == want_m == [32768, 0, 16384, 16384, 0]
+    u = [oracle.u16(4, 2, 1, oracle.STREAM_MASK, i) for i in range(alpha.size)]
+    assert list(r["Z"]) == [int(ui < mi) for ui, mi in zip(u, want_m)]
+    for i in range(alpha.size):
+        want = Fraction(float(alpha[i])) * 65536 / want_m[i] if r["Z"][i] else 0           # alpha_i / p_i
+        assert Fraction(float(r["beta"][i])) == want
+    # (b) |alpha|_1 = 6 * 2^-149: phi_eff / |alpha|_1 = 2^149 / 3 overflows
+    alpha = np.array([sub(3, -149), 0.0, sub(-1, -149), 0.0, sub(2, -149), 0.0, 0.0], F32)
+    for phi in (0.0, 1.5, 100.0):
+        r = oracle.sparsify(alpha, phi, 4, 3, 0)
+        assert r["status"] == 0 and Fraction(float(r["n1"])) == Fraction(6, 2 ** 149)
+        assert r["phi_eff"] == (2.0 if phi != 1.5 else 1.5)                                 # clamp of Lemma 2: 6/3
+        assert list(r["m"]) == [65536, 0, 65536, 0, 65536, 0, 0]
+        assert list(r["Z"]) == [1, 0, 1, 0, 1, 0, 0]
+        assert np.array_equal(r["beta"], alpha) and not np.isnan(r["beta"]).any()
+        codes, delta, rc = oracle.quantize_survivors(r["beta"], r["Z"], 4, 4, 3, 0)
+        assert rc == 0 and np.isfinite(delta) and not codes[[1, 3, 5, 6]].any() and np.abs(codes).max() <= 7
+
+
 def test_sparsifier_moments():
     """E[beta] = alpha, E||beta||^2 = sum alpha_i^2/p_i (= |alpha|_1^2/phi at Lemma 2's p), E[nnz] = sum p_i."""
     g = np.random.default_rng(7)
