@@ -18,7 +18,7 @@
  *     default stream).  No call synchronises the device unless it says so.
  *   - Errors found on the host (bad argument, bad bit width, misaligned buffer) are returned immediately.
  *     Errors found by a kernel (non-finite norm, sparse message over capacity) set a sticky status word that
- *     dq_poll_status reads.
+ *     dq_poll_status reads.  A vector that holds a NaN or an Inf is quantised to scale 0 and all-zero codes.
  *   - The gradient width b must be 2, 4 or 8; the model width b_x may be any of 2..11, the widths of Table 1
  *     (b = 1 would give 2^(b-1)-1 = 0 levels).  Up to 8 bits the rounding position keeps 15 fractional bits, then
  *     14, 13 and 12 for 9, 10 and 11 bits.
@@ -238,7 +238,10 @@ int dq_codec_round_host(dq_ctx* ctx, const float* v_host, uint32_t round, float 
  *   - All calls on a device share the one array, which still holds the previous call's norms; each call
  *     clears what it needs on `stream` first.  Two calls whose GPU work overlaps (different streams, or
  *     different threads) race on it: serialise them.
- *   - A non-finite vector gets scale 0 and all-zero codes; there is no status word to poll. */
+ *   - A message that holds a NaN or an Inf gets scale 0 and all-zero codes (every coordinate, the non-finite ones
+ *     included); there is no status word to poll.  scale must be 4-byte aligned.
+ *   - The first call on a device may be made from several host threads at once.  The return value reports this call's
+ *     own launches only. */
 #define DQ_STATIC_MAX_MESSAGES 1024
 int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, uint64_t seed, uint32_t round,
                             uint8_t* codes, int64_t stride, float* scale, void* stream);

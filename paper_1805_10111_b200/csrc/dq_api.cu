@@ -347,7 +347,7 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
                                  ctx->delta_x, round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
                                  reinterpret_cast<uint32_t*>(ctx->ninf), ctx->cfg.sparsify ? 4 * ctx->cfg.M : ctx->cfg.M);
         } else {     // condition (3): pick the width on the device, then launch the three specialised widths and the general kernel; all but one return at once
-            launch_select_bits(ctx, s->x, s->x_snap, nx, ctx->cfg.mu, theta, ctx->bx_dev, ctx->prec_stats, as_stream(st));
+            launch_select_bits(ctx, s->x, s->x_snap, nx, ctx->cfg.mu, ctx->cfg.accelerated, theta, ctx->bx_dev, ctx->prec_stats, as_stream(st));
             for (int bits : {2, 4, 8, 3})                      // 3 stands for "any other width": the general kernel reads it from the device
                 launch_quantize_pack(ctx, s->x, ctx->cfg.d, 1, bits, nx, ctx->codes_x, dq_packed_bytes(ctx->cfg.d, bits), ctx->delta_x,
                                      round, kMaster, kStreamModel, as_stream(st), ref, ctx->xhat_diff, zf, zn,
@@ -491,9 +491,7 @@ int dq_select_model_bits(dq_ctx* ctx, const float* x, const float* x_snap, const
     const uint32_t* nb = reinterpret_cast<const uint32_t*>(norm_x);
     if (!nb) { launch_norm_inf(ctx, x, ctx->cfg.d, 1, ctx->xnorm_bits, st); nb = ctx->xnorm_bits; }
     // theta is folded into mu by the caller here, so the kernel is told "not accelerated"
-    const int acc = ctx->cfg.accelerated; ctx->cfg.accelerated = 0;
-    launch_select_bits(ctx, x, x_snap, nb, mu, 0.0f, bits, stats ? stats : ctx->prec_stats, st);
-    ctx->cfg.accelerated = acc;
+    launch_select_bits(ctx, x, x_snap, nb, mu, 0, 0.0f, bits, stats ? stats : ctx->prec_stats, st);
     return last_error();
 }
 

@@ -2,6 +2,8 @@
 // and 12), sparsification (eq. (4), Lemma 2; Algorithm 2 steps 12-13), and the master's unpack +
 // aggregate + prox step (Algorithm 1 step 9, Algorithm 3 step 9).  All are bandwidth kernels: 256-bit
 // coalesced loads, one Philox call per eight coordinates, codes packed in registers.
+#include <atomic>
+
 #include "dq_common.cuh"
 #include "dq_kernels.cuh"
 
@@ -74,13 +76,19 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
     const uint32_t worker = worker_base + (uint32_t)w;
     const int64_t nth = (int64_t)gridDim.x * blockDim.x;
     for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < ngroups; g += nth) {
-        float a[8];
         const int64_t i0 = g << 3;
-        if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
-        uint32_t r[4], s[8];
-        philox4x32_10((uint32_t)g, round, worker, stream, K, r);
+        uint32_t s[8];
+        if (finite) {
+            float a[8];
+            if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
+            uint32_t r[4];
+            philox4x32_10((uint32_t)g, round, worker, stream, K, r);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+            for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+        } else {                                   // NaN or Inf in the message: every code is 0 (a NaN would pick its own bits)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = 128u << 16;
+        }
         store_group<BITS>(out + g * BITS, pack8<BITS>(s));
         if (DIFF) {
 #pragma unroll
@@ -581,6 +589,7 @@ sparsify_emit_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                         With sparse output only the chunks with more than kStash survivors are redone. */,
                      int M = 0)
 {
+    pdl_prologue();
     const int w = blockIdx.y, lane = threadIdx.x & 31;
     if (redo_flags && (redo_flags[M] == 0u || redo_flags[w] == 0u)) return;        // the staged path covered this worker
     if (rp) round = rp->round;
@@ -721,6 +730,10 @@ quantize_master_kernel(const float* __restrict__ v, int64_t d, int M, int vec_ok
             const float inv = s_inv[w];
 #pragma unroll
             for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+            if (norm_bits[w] >= 0x7F800000u) {               // NaN or Inf in the message: every code is 0
+#pragma unroll
+                for (int j = 0; j < 8; ++j) s[j] = 128u << 16;
+            }
             store_group<BITS>(codes + (int64_t)w * stride + g * BITS, pack8<BITS>(s));
         } else {
 #pragma unroll
@@ -1133,7 +1146,9 @@ master_sparse_seq_kernel(const uint8_t* __restrict__ codes, int64_t stride, cons
             const uint32_t* words = reinterpret_cast<const uint32_t*>(codes + (int64_t)w * stride);
             for (uint32_t e = e0 + threadIdx.x; e < e1; e += blockDim.x) {
                 const int64_t bit = (int64_t)e * BITS;
-                s_q[(int)((int64_t)list[e] - lo)] = (float)code_of<BITS>(__ldg(words + (bit >> 5)), (int)((bit & 31) / BITS));
+                const int li = (int)((int64_t)list[e] - lo);
+                if ((unsigned)li < (unsigned)kChunk)                               // a list entry outside its tile is dropped, never followed
+                    s_q[li] = (float)code_of<BITS>(__ldg(words + (bit >> 5)), (int)((bit & 31) / BITS));
             }
             __syncthreads();
             const float dl = scale[w];
@@ -1176,13 +1191,14 @@ __global__ void unpack_dense_kernel(const uint8_t* __restrict__ codes, const flo
 template <int BITS>
 __global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const float* __restrict__ scale,
                                      const uint32_t* __restrict__ idx, const uint32_t* __restrict__ nnz,
-                                     float* __restrict__ out)
+                                     int64_t d, float* __restrict__ out)
 {
     pdl_prologue();
     const float dl = scale[0];
     const uint32_t n = nnz[0];
     for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         const int64_t bit = (int64_t)e * BITS;
+        if ((int64_t)idx[e] >= d) continue;                                        // a position beyond the vector is dropped
         out[idx[e]] = __fmul_rn((float)code_of<BITS>(reinterpret_cast<const uint32_t*>(codes)[bit >> 5], (int)((bit & 31) / BITS)), dl);
     }
 }
@@ -1377,7 +1393,7 @@ quantize_pack_any_kernel(const float* __restrict__ v, int64_t d, const uint32_t*
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t F = __float_as_uint(__fmaf_rn(a[j], inv, off)) & 0x007FFFFFu;
-            const int code = (int)((F + (half16(r, j) >> (16 - fb))) >> fb) - half;
+            const int code = ok ? (int)((F + (half16(r, j) >> (16 - fb))) >> fb) - half : 0;    // zero or non-finite norm: code 0
             const unsigned long long field = (unsigned long long)((uint32_t)code & mask);
             const int pos = j * bits;
             if (pos < 64) { lo |= field << pos; if (pos + bits > 64) hi |= field >> (64 - pos); }
@@ -1455,12 +1471,12 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     ctx->launches += 1;
 }
 
-void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, float theta,
-                        int32_t* bits, double* stats, cudaStream_t st)
+void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, int accelerated,
+                        float theta, int32_t* bits, double* stats, cudaStream_t st)
 {
     cudaMemsetAsync(stats, 0, sizeof(double) * (kWidths + 1), st);
     launch_k(model_precision_kernel, grid_for(ctx->cfg.d / 2 + 1, ctx->sm_count, 4), kThreads, 0, st, x, xsnap, ctx->cfg.d, norm_bits, stats);
-    launch_k(select_bits_kernel, 1, 1, 0, st, stats, norm_bits, mu, ctx->cfg.accelerated, theta, ctx->rp_active, bits);
+    launch_k(select_bits_kernel, 1, 1, 0, st, stats, norm_bits, mu, accelerated, theta, ctx->rp_active, bits);
     ctx->launches += 2;
 }
 
@@ -1653,7 +1669,7 @@ void launch_unpack(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, int w, fl
         DQ_DISPATCH_BITS(c.b, (launch_k(unpack_dense_kernel<BITS_>, grid_for(c.d, ctx->sm_count), kThreads, 0, st, codes, msgs->scale + w, c.d, out)));
     } else {
         cudaMemsetAsync(out, 0, sizeof(float) * c.d, st);
-        DQ_DISPATCH_BITS(c.b, (launch_k(unpack_sparse_kernel<BITS_>, grid_for(msgs->cap, ctx->sm_count), kThreads, 0, st, codes, msgs->scale + w, msgs->idx + (int64_t)w * msgs->cap, msgs->nnz + w, out)));
+        DQ_DISPATCH_BITS(c.b, (launch_k(unpack_sparse_kernel<BITS_>, grid_for(msgs->cap, ctx->sm_count), kThreads, 0, st, codes, msgs->scale + w, msgs->idx + (int64_t)w * msgs->cap, msgs->nnz + w, c.d, out)));
     }
     ctx->launches += 1;
 }
@@ -1674,21 +1690,25 @@ constexpr int kStaticMaxDevices = 64;
 // [0, kStaticMaxMessages): ||v_w||_inf bit patterns; [kStaticMaxMessages]: non-finite flag of the last call.
 static __device__ __align__(256) uint32_t g_static_scratch[kStaticMaxMessages + 64];
 
-struct StaticSlot { uint32_t* ptr; int sm_count; bool ready; };
+struct StaticSlot { uint32_t* ptr; int sm_count; std::atomic<int> ready; };
 StaticSlot g_static_slot[kStaticMaxDevices];
 
-// Looks up the device address of the scratch array for the current device (first call on that device).
+// Looks up the device address of the scratch array for the current device (first call on that device).  Two host
+// threads may make that first call together: both look the address up and store the same values; `ready` is
+// published with release order after the values and read with acquire order before them, so no thread sees the flag
+// without the values.
 int static_scratch_for_current_device(uint32_t** ptr, int* sm_count)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kStaticMaxDevices) return DQ_ERR_CUDA;
     StaticSlot& s = g_static_slot[dev];
-    if (!s.ready) {
+    if (s.ready.load(std::memory_order_acquire) == 0) {
         void* p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) { cudaGetLastError(); return DQ_ERR_CUDA; }
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return DQ_ERR_CUDA;
-        s.ptr = static_cast<uint32_t*>(p); s.sm_count = sms; s.ready = true;
+        s.ptr = static_cast<uint32_t*>(p); s.sm_count = sms;
+        s.ready.store(1, std::memory_order_release);
     }
     *ptr = s.ptr; *sm_count = s.sm_count;
     return DQ_OK;
@@ -1704,7 +1724,8 @@ extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, 
     if (b != 2 && b != 4 && b != 8) return DQ_ERR_BITS;
     if (M > kStaticMaxMessages) return DQ_ERR_SHAPE;                       // beyond the fixed scratch
     if (d > ((int64_t)1 << 32)) return DQ_ERR_SHAPE;
-    if ((reinterpret_cast<uintptr_t>(codes) & 15) || (stride & 15) || (reinterpret_cast<uintptr_t>(v) & 3)) return DQ_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(codes) & 15) || (stride & 15) || (reinterpret_cast<uintptr_t>(v) & 3) ||
+        (reinterpret_cast<uintptr_t>(scale) & 3)) return DQ_ERR_ARG;
     if (stride < dq_packed_bytes(d, b)) return DQ_ERR_SHAPE;
     uint32_t* scratch = nullptr; int sms = 0;
     int rc = static_scratch_for_current_device(&scratch, &sms);
@@ -1714,11 +1735,12 @@ extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, 
     if (cudaMemsetAsync(scratch, 0, sizeof(uint32_t) * (kStaticMaxMessages + 1), st) != cudaSuccess) return DQ_ERR_CUDA;
     const int vec_ok = vec_ok_for(v, d);
     dim3 grid_n(grid_for((d + 7) / 8, sms), M);
-    launch_k(norm_inf_kernel, grid_n, kThreads, 0, st, v, d, vec_ok, scratch);
+    if (launch_k(norm_inf_kernel, grid_n, kThreads, 0, st, v, d, vec_ok, scratch) != cudaSuccess) return DQ_ERR_CUDA;
     const int64_t ngroups = dq_packed_bytes(d, b) / b;
     dim3 grid_q(grid_for(ngroups, sms), M);
     const PhiloxKeys keys = expand_keys(seed);
     int* flag = reinterpret_cast<int*>(scratch + kStaticMaxMessages);
-    DQ_DISPATCH_BITS(b, (launch_k(quantize_pack_kernel<BITS_, false>, grid_q, kThreads, 0, st, v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr)));
-    return cudaGetLastError() == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
+    cudaError_t err = cudaSuccess;             // this launch's own result, not whatever error an earlier call left behind
+    DQ_DISPATCH_BITS(b, (err = launch_k(quantize_pack_kernel<BITS_, false>, grid_q, kThreads, 0, st, v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr)));
+    return err == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }

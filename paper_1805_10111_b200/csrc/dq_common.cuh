@@ -165,7 +165,7 @@ __device__ __forceinline__ void pdl_prologue()
 // Launch with the programmatic-serialization attribute: the gap between dependent kernels (drain, then launch)
 // is what bounds the small configurations, whose rounds are chains of microsecond kernels.
 template <class... P, class... A>
-inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args)
+inline cudaError_t launch_k(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A&&... args)
 {
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -173,7 +173,7 @@ inline void launch_k(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, c
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaLaunchKernelEx(&cfg, kernel, static_cast<A&&>(args)...);
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<A&&>(args)...);
 }
 
 struct ProxParams { float lambda1, lambda2, lo, hi; };

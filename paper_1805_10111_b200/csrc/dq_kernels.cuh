@@ -11,8 +11,8 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
                           uint32_t stream_id, cudaStream_t st, const float* ref = nullptr, float* diff = nullptr,
                           float* zero_f = nullptr, int64_t zero_n = 0, uint32_t* zero_u = nullptr, int zero_un = 0,
                           const int32_t* bits_gate = nullptr);
-void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, float theta,
-                        int32_t* bits, double* stats, cudaStream_t st);
+void launch_select_bits(dq_ctx* ctx, const float* x, const float* xsnap, const uint32_t* norm_bits, float mu, int accelerated,
+                        float theta, int32_t* bits, double* stats, cudaStream_t st);
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
                           uint32_t round, const dq_msgs* out, bool sparse_out, cudaStream_t st);
 void launch_dequant_diff_any(dq_ctx* ctx, const uint8_t* codes, const float* delta_x, const float* ref, float* diff, int bits, cudaStream_t st);
@@ -36,7 +36,5 @@ void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds
                           uint64_t* bits_up, cudaStream_t st);
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st);
 void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st);
-void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* nnz, uint64_t* bits_down,
-                 uint64_t* bits_up, cudaStream_t st);
 
 }  // namespace dq

@@ -117,9 +117,23 @@ def test_zero_and_nonfinite_vectors(dq):
     assert dq.dq_poll_status(ctx) == (0, dq.DQ_ERR_NONFINITE)
     assert dq.dq_poll_status(ctx) == (0, 0)                  # cleared after being read
     assert msgs.scale[1].item() == 0 and not msgs.codes[1].any().item()
+    assert msgs.scale[2].item() == 0 and not msgs.codes[2].any().item()      # the NaN coordinate's own code is 0 too
     c, dl, _ = oracle.quantize(v[0], 4, 1, 0, 0, oracle.STREAM_GRAD)
     assert np.array_equal(msgs.codes[0].cpu().numpy(), oracle.pack(c, 4, msgs.stride))
+    assert oracle.quantize(v[2], 4, 1, 0, 2, oracle.STREAM_GRAD)[2] == oracle.ERR_NONFINITE   # the oracle refuses the vector
     dq.dq_destroy(ctx)
+    # the model quantiser for every width, NaN and Inf, and the merged quantiser + master kernel of a whole round
+    import torch
+    for bx, bad in ((8, np.inf), (2, np.nan), (5, -np.inf), (11, np.nan)):
+        x = synth.normal_vector(d, 41, 0.3); x[d - 1] = bad
+        cfg = dq.make_config(d, 2, bx=bx, seed=2)
+        rc, ctx = dq.dq_create(cfg); assert rc == 0
+        nb = dq.dq_packed_bytes(d, bx)
+        codes = torch.full((nb,), 0x55, dtype=torch.uint8, device="cuda"); delta = torch.full((1,), 3.0, device="cuda")
+        assert dq.dq_quantize_model(ctx, _dev(x), None, 5, codes, delta) == 0
+        assert dq.dq_poll_status(ctx) == (0, dq.DQ_ERR_NONFINITE)
+        assert delta.item() == 0 and not codes.any().item()
+        dq.dq_destroy(ctx)
 
 
 def test_argument_errors(dq):

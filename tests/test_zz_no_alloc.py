@@ -30,6 +30,8 @@ def test_static_entry_matches_context_entry_twice_in_a_row():
         v[0, 17] *= 100.0
         if c["rnd"] == 9:
             v[1] = 0.0                                           # a zero vector must come out as scale 0, codes 0
+        if c["rnd"] == 4:
+            v[3, 5] = np.nan; v[4, d - 1] = np.inf               # so must a vector that holds a NaN or an Inf
         dv = torch.from_numpy(v).cuda()
         cfg = dq.make_config(d, M, b=b, seed=seed)
         rc, ctx = dq.dq_create(cfg); assert rc == 0
@@ -42,6 +44,8 @@ def test_static_entry_matches_context_entry_twice_in_a_row():
         assert torch.equal(got_scale, want.scale)
         assert torch.equal(got_codes, want.codes)
         assert got_scale.max().item() > 0
+        if c["rnd"] == 4:
+            assert not got_scale[3:].any().item() and not got_codes[3:].any().item()
         dq.dq_destroy(ctx)
     # sizes beyond the fixed scratch, and bad arguments, are refused before anything is launched
     small = torch.zeros((2, 64), device="cuda"); codes = torch.zeros((2, 64), dtype=torch.uint8, device="cuda")
