@@ -4,10 +4,19 @@
 Default workload ("c5"): the quantiser/packer bandwidth configuration -- M = 8 worker gradient vectors of
 d = 2^27 fp32 coordinates (N(0,1) with 0.1 % outliers x100), quantised to b = 4 bits and packed, aggregated
 and prox-updated by the master, and the new model requantised to b_x = 8 bits.  One "step" is one such
-round: ||v||_inf pass, quantise+pack, master unpack+aggregate+prox, model norm is fused, model quantise.
-Prints ONE JSON line: metric, value (whole-job rounds/s), per-stage times, roofline of the dominant kernel, clocks,
-end-to-end rate through host buffers, the CPU oracle's rate, and rounds/s of the training configurations (each
-with the oracle's rate on the same data).
+round: ||v||_inf pass, quantise+pack, master unpack+aggregate+prox (model norm fused), model quantise.
+Prints ONE JSON line:
+  value / ms_per_step    whole-job rounds/s over exactly --steps steps (CUDA events, max over ranks)
+  stages                 per-stage time, algorithmic GB/s and fraction of the HBM peak, twice: over the timed steps
+                         (short run: the GPU usually still boosts) and from a loop of >= --sustain-s seconds per stage
+                         with the SM clock sampled every 20 ms (where the 1 kW power cap settles the clock)
+  roofline               the dominant kernel (quantise+pack) against the measured copy bandwidth
+  sweep                  the c5 grid d in {2^24, 2^27} x b in {2,4,8} x sparsify off/on, each point with its own
+                         clock record, fractions of the measured peak and of the nominal 8 TB/s
+  e2e                    the same round through host buffers (copies inside the timed region)
+  cpu_baseline           the CPU oracle on a bounded slice of the workload, threads stated
+  training_configs       rounds/s of dq_rounds on c1..c4 and the network, per-stage times of the stage entry
+                         points called one by one, bits per round, and the oracle's rate on the same data
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--log2d 27] [--bits 4]
 
@@ -30,6 +39,8 @@ sys.path.insert(0, ROOT)
 
 METRIC = "simulated-worker rounds/sec"
 UNIT = "rounds/s"
+NOMINAL_HBM_GBPS = 8000.0          # the figure the target is worded against
+SEED = 1805
 
 
 def parse_args():
@@ -44,10 +55,11 @@ def parse_args():
     ap.add_argument("--sparsify", type=int, default=0)
     ap.add_argument("--sequential", type=int, default=0, help="1: master applies one prox step per message")
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--sustain-s", type=float, default=1.5, help="seconds each stage is looped for the sustained-clock figure (0: skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--sweep", action="store_true", help="time the codec stages over d in {2^20,2^24,2^27} x b in {2,4,8} x sparsify off/on "
-                                                         "and print one JSON object with all points instead of the bench line")
-    ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_round ('' for none)")
+    ap.add_argument("--no-sweep", action="store_true", help="leave the c5 grid out of the line")
+    ap.add_argument("--sweep", action="store_true", help="print only the c5 grid (adds d = 2^20) as one JSON object")
+    ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_rounds ('' for none)")
     return ap.parse_args()
 
 
@@ -62,45 +74,73 @@ def workload_config(a):
 # ---------------------------------------------------------------------------------------------------------------
 # CPU oracle leg (cpu_baseline of the main line, and the whole of --impl reference)
 # ---------------------------------------------------------------------------------------------------------------
-def oracle_rounds_per_sec(a, steps, warmup, log2_sample=22):
-    """Times the oracle's codec round on a d = 2^log2_sample slice of the workload; work is linear in d, so
-    the rate is scaled by 2^log2_sample / d.  Returns (scaled rounds/s, seconds per sampled round, description)."""
+def oracle_codec_round(v, x, g, b, rnd, sparsify, pool=None):
+    """One codec round of the oracle as it stands: every worker's message, the master step, the model's codes.
+    pool: a thread pool over the M independent workers (the C functions release the interpreter lock)."""
     import numpy as np
     import oracle
+    M, ds = v.shape
+
+    def one(w):
+        if sparsify:
+            r = oracle.sparsify(v[w], 0.01 * ds, SEED, rnd, w)
+            return oracle.quantize_survivors(r["beta"], r["Z"], b, SEED, rnd, w)[:2]
+        return oracle.quantize(v[w], b, SEED, rnd, w, oracle.STREAM_GRAD)[:2]
+
+    res = list(pool.map(one, range(M))) if pool is not None else [one(w) for w in range(M)]
+    raw = np.stack([r[0] for r in res]); delta = np.array([r[1] for r in res], np.float32)
+    oracle.master_step(raw, delta, g, x, 0.1, l1=1e-6)
+    oracle.quantize(x, 8, SEED, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+
+
+def oracle_rounds_per_sec(a, steps, warmup, log2_sample, threads):
+    """Times the oracle's codec round on a d = 2^log2_sample slice of the workload (same recipe, same M, b, sparsify);
+    the work is linear in d, so the full-size rate is the slice's rate times 2^log2_sample / d.  Returns
+    (rounds/s at full size, seconds per sampled round, description)."""
+    from concurrent.futures import ThreadPoolExecutor
     from paper_1805_10111_b200 import synth
-    ds = 1 << min(log2_sample, a.log2d)
-    M, b = a.workers, a.bits
-    v, x, g = synth.config5(ds, M)
+    ls = min(log2_sample, a.log2d)
+    ds = 1 << ls
+    v, x, g = synth.config5(ds, a.workers)
     x = x.copy()
+    pool = ThreadPoolExecutor(threads) if threads > 1 else None
     times = []
     for rnd in range(warmup + steps):
         t0 = time.perf_counter()
-        raw = np.zeros((M, ds), np.int32); delta = np.zeros(M, np.float32)
-        for w in range(M):
-            if a.sparsify:
-                r = oracle.sparsify(v[w], 0.01 * ds, 1805, rnd, w)
-                raw[w], delta[w], _ = oracle.quantize_survivors(r["beta"], r["Z"], b, 1805, rnd, w)
-            else:
-                raw[w], delta[w], _ = oracle.quantize(v[w], b, 1805, rnd, w, oracle.STREAM_GRAD)
-        oracle.master_step(raw, delta, g, x, 0.1, l1=1e-6)
-        oracle.quantize(x, 8, 1805, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+        oracle_codec_round(v, x, g, a.bits, rnd, a.sparsify, pool)
         if rnd >= warmup:
             times.append(time.perf_counter() - t0)
+    if pool is not None:
+        pool.shutdown()
     sec = sum(times) / len(times)
-    scaled = (1.0 / sec) * ds / (1 << a.log2d)
-    return scaled, sec, "oracle codec round on a d=2^%d slice (%d rounds, single thread), rate scaled by d" % (min(log2_sample, a.log2d), steps)
+    what = ("oracle codec round on a d=2^%d slice of the workload (%d timed rounds, %d thread%s over the %d workers; master step and "
+            "model quantiser single-threaded)%s" % (ls, steps, threads, "" if threads == 1 else "s", a.workers,
+                                                     "" if ls == a.log2d else "; rate scaled by 2^%d/d (work is linear in d)" % ls))
+    return (1.0 / sec) * ds / (1 << a.log2d), sec, what
+
+
+def host_threads(M):
+    return max(1, min(M, os.cpu_count() or 1))
 
 
 def run_reference(a):
+    """--impl reference: the oracle, as it stands, on the host cores.  Runs exactly --warmup + --steps rounds, each on a
+    slice of the workload sized (from one calibration round at d = 2^18) so that the whole run takes about a minute."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    steps = max(1, min(a.steps, 8)); warm = max(0, min(a.warmup, 1))
-    val, sec, what = oracle_rounds_per_sec(a, steps, warm)
+    threads = host_threads(a.workers)
+    _, sec18, _ = oracle_rounds_per_sec(a, steps=1, warmup=0, log2_sample=min(18, a.log2d), threads=threads)
+    budget = 60.0 / max(1, a.steps + a.warmup)                               # seconds per round
+    ls = min(18, a.log2d)
+    while ls < a.log2d and sec18 * (1 << (ls + 1 - min(18, a.log2d))) <= budget:
+        ls += 1
+    val, sec, what = oracle_rounds_per_sec(a, a.steps, a.warmup, ls, threads)
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": a.gpus, "steps": a.steps,
             "warmup": a.warmup, "ms_per_step": 1000.0 / val, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(a),
-            "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what,
+                             "seconds_per_sampled_round": sec, "extrapolated": ls != a.log2d},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -110,14 +150,15 @@ def run_reference(a):
 # helpers
 # ---------------------------------------------------------------------------------------------------------------
 class ClockSampler:
+    """nvidia-smi polled every `period_ms` while a timed region runs (read-only queries; no setting is touched)."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index):
+    def __init__(self, index, period_ms=20):
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS,
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", str(period_ms)],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
@@ -125,7 +166,7 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
@@ -147,8 +188,8 @@ class ClockSampler:
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
         sm.sort()
-        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(smax), "power_w_max": max(power), "samples": len(sm),
-                "reasons": sorted(reasons)}
+        return {"sm_mhz": sm[len(sm) // 2], "sm_mhz_min": sm[0], "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def max_over_ranks(value, dist=None, device="cpu"):
@@ -197,8 +238,24 @@ def recorded_traffic(bits):
     return float(k.group(1))
 
 
+STAGE_NAMES = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
+
+
+def codec_alg_bytes(M, d, b, bx, sparsify):
+    """Algorithmic bytes per launch of the four codec stages: norm 4 B and quantise+pack 4 + b/8 B per message
+    coordinate (8 + b/8 when sparsifying: ||v||_1 must be known before the first mask bit can be drawn, so the vectors
+    are read twice), master M b/8 + 12 B and model quantise 4 + b_x/8 B per model coordinate."""
+    return [M * d * 4.0, M * d * ((8.0 if sparsify else 4.0) + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
+
+
+def stage_report(ms_list, alg, peak):
+    return {n: {"ms": round(ms, 4), "alg_GBps": round(by / ms / 1e6, 1), "frac_of_peak": round(by / ms / 1e6 / peak, 4),
+                "frac_of_8TBps": round(by / ms / 1e6 / NOMINAL_HBM_GBPS, 4)}
+            for n, ms, by in zip(STAGE_NAMES, ms_list, alg)}
+
+
 # ---------------------------------------------------------------------------------------------------------------
-# whole training rounds (dq_round) on the four training configurations
+# whole training rounds (dq_rounds) on the training configurations, and their stages one by one
 # ---------------------------------------------------------------------------------------------------------------
 TRAIN_CONFIGS = {
     "c1": dict(gen="config1", kw=dict(M=4, B=16, bx=8, b=8, lambda1=1e-4), lr=1.0, theta=0.0, m=200),
@@ -214,9 +271,68 @@ TRAIN_CONFIGS = {
 }
 
 
-def time_training_config(name, rounds=200, warmup=20, with_oracle=False):
-    """rounds/s of dq_rounds on one of the training configurations (full size, synthetic data), plus the bits
-    the paper's accounting charges per round."""
+class _Raw:
+    """A device address owned by the library, passed back to it."""
+    def __init__(self, ptr):
+        self._p = ptr
+
+    def data_ptr(self):
+        return self._p
+
+
+def time_training_stages(dq, ctx, cfg, h, st, eta, theta, peak, reps=60):
+    """The four stage entry points called one after the other on the context's own buffers (so the touched-group list
+    of sparse gradients is used as in dq_round), CUDA events between them.  dq_round itself merges stages (the model
+    quantiser also writes xhat - xsnap and clears accumulators, quantiser and master share a kernel for dense
+    messages, small problems run in one cluster kernel), so these are the stages' stand-alone costs."""
+    import torch
+    _, buf = dq.dq_round_buffers(ctx)
+    alpha, ninf = _Raw(buf["alpha"]), _Raw(buf["norm_inf"])
+    codes_x, delta_x = _Raw(buf["codes_x"]), _Raw(buf["delta_x"])
+    msgs = type("OwnMsgs", (), {"c": buf["msgs"]})()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(reps)]
+    for k in range(-3, reps):
+        rnd = 100000 + k
+        e = ev[k] if k >= 0 else None
+        if e: e[0].record()
+        dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, rnd, codes_x, delta_x))
+        if e: e[1].record()
+        dq.ok(dq.dq_worker_grad(ctx, codes_x, delta_x, 0, st, rnd, None, alpha, ninf))
+        if e: e[2].record()
+        dq.ok(dq.dq_quantize_sparsify_pack(ctx, alpha, ninf, rnd, msgs))
+        if e: e[3].record()
+        dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta, theta))
+        if e: e[4].record()
+    torch.cuda.synchronize()
+    ms = [sorted(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(reps))[reps // 2] for i in range(4)]
+    M, B, d, b, bx = cfg.M, cfg.B, int(cfg.d), cfg.b, cfg.bx
+    if cfg.model == 1:
+        grad_bytes, grad_what = M * B * h.d * 4.0 + 2 * d * 4.0, "sampled rows (fp32) + both parameter vectors"
+    elif h.format == 1:
+        nnz_row = float(h.row_ptr[-1]) / h.n
+        grad_bytes, grad_what = M * B * nnz_row * 8.0, "8 B per gathered nonzero (%.0f per row)" % nnz_row
+    else:
+        grad_bytes, grad_what = M * B * h.d * (4.0 if h.format == 0 else 2.0), "sampled rows read once"
+    sparse = bool(cfg.sparsify) and cfg.msg_format == 1
+    alg = {"quantize_model": d * (4.0 + bx / 8.0), "worker_grad": grad_bytes,
+           "quantize_sparsify_pack": None if sparse else M * d * ((8.0 if cfg.sparsify else 4.0) + b / 8.0),
+           "master_unpack_aggregate_prox": d * ((0.0 if sparse else M * b / 8.0) + (32.0 if cfg.accelerated else 12.0))}
+    out = {}
+    for (name, by), t in zip(alg.items(), ms):
+        out[name] = {"us": round(t * 1000.0, 2)}
+        if by is not None:
+            out[name].update(alg_bytes=int(by), alg_GBps=round(by / t / 1e6, 1), frac_of_peak=round(by / t / 1e6 / peak, 4),
+                             frac_of_8TBps=round(by / t / 1e6 / NOMINAL_HBM_GBPS, 4))
+    out["worker_grad"]["bytes_counted"] = grad_what
+    if sparse:
+        out["quantize_sparsify_pack"]["note"] = "works on the list of touched groups (KBs): bound by kernel latency, no bandwidth figure"
+    out["sum_us"] = round(sum(ms) * 1000.0, 2)
+    return out
+
+
+def time_training_config(name, rounds=200, warmup=20, with_oracle=False, peak=None):
+    """rounds/s of dq_rounds on one of the training configurations (full size, synthetic data), the stages one by one,
+    and the bits the paper's accounting charges per round."""
     import numpy as np
     import torch
     import paper_1805_10111_b200 as dq
@@ -225,7 +341,7 @@ def time_training_config(name, rounds=200, warmup=20, with_oracle=False):
     h = getattr(synth, spec["gen"])()
     is_nn = spec["kw"].get("model", 0) == 1
     x0 = synth.mlp_init(h.d, spec["kw"]["hidden"], spec["kw"]["classes"], 9) if is_nn else np.zeros(h.d, np.float32)
-    cfg = dq.make_config(x0.size, spec["kw"]["M"], seed=1805, **{k: v for k, v in spec["kw"].items() if k != "M"})
+    cfg = dq.make_config(x0.size, spec["kw"]["M"], seed=SEED, **{k: v for k, v in spec["kw"].items() if k != "M"})
     data = dq.Data(h)
     rc, ctx = dq.dq_create(cfg, data); dq.ok(rc, "dq_create " + name)
     st = dq.State(x0, n=h.n, accelerated=bool(cfg.accelerated))
@@ -235,23 +351,28 @@ def time_training_config(name, rounds=200, warmup=20, with_oracle=False):
     for r in range(warmup):
         dq.ok(dq.dq_round(ctx, st, r, eta, theta))
     torch.cuda.synchronize()
+    sampler = ClockSampler(torch.cuda.current_device())
     l0 = dq.dq_launch_count(ctx)
     e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
     e0.record()
     dq.ok(dq.dq_rounds(ctx, st, warmup, rounds, eta, theta, bits[0:1], bits[1:2]))      # one call for all rounds of the epoch
     e1.record(); torch.cuda.synchronize()
+    clocks = sampler.stop()
     ms = e0.elapsed_time(e1) / rounds
-    rc, status = dq.dq_poll_status(ctx)
+    launches = (dq.dq_launch_count(ctx) - l0) / rounds
     out = {"rounds_per_s": round(1000.0 / ms, 1), "ms_per_round": round(ms, 4), "n": h.n, "d": int(cfg.d), "M": cfg.M, "B": cfg.B,
-           "launches_per_round": (dq.dq_launch_count(ctx) - l0) / rounds, "bits_down": int(bits[0].item()),
-           "bits_up": int(bits[1].item()), "bits_full_precision": 2 * cfg.M * 32 * int(cfg.d), "device_status": status}
+           "launches_per_round": launches, "bits_down": int(bits[0].item()),
+           "bits_up": int(bits[1].item()), "bits_full_precision": 2 * cfg.M * 32 * int(cfg.d), "clocks": clocks}
+    out["stages_one_by_one"] = time_training_stages(dq, ctx, cfg, h, st, eta, theta, peak or measured_peak()[0])
+    rc, status = dq.dq_poll_status(ctx)
+    out["device_status"] = status
     dq.dq_destroy(ctx)
     if with_oracle:
         out["cpu_oracle"] = oracle_training_rounds_per_sec(h, spec, x0)
     return out
 
 
-def oracle_training_rounds_per_sec(h, spec, x0, budget_s=6.0):
+def oracle_training_rounds_per_sec(h, spec, x0, budget_s=5.0):
     """The CPU oracle on the same data and settings: an epoch boundary, one untimed round, then whole rounds until
     about budget_s seconds have gone (at least two).  Single thread."""
     import numpy as np
@@ -260,7 +381,7 @@ def oracle_training_rounds_per_sec(h, spec, x0, budget_s=6.0):
     ocfg = oracle.make_config(x0.size, kw["M"], kw["B"], kw["bx"], kw["b"], l1=kw.get("lambda1", 0.0), l2=kw.get("lambda2", 0.0),
                               box_lo=kw.get("box_lo", -np.inf), box_hi=kw.get("box_hi", np.inf), sparsify=kw.get("sparsify", 0),
                               phi=kw.get("phi", 0.0), msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0),
-                              seed=1805, model=kw.get("model", 0), hidden=kw.get("hidden", 0), classes=kw.get("classes", 0))
+                              seed=SEED, model=kw.get("model", 0), hidden=kw.get("hidden", 0), classes=kw.get("classes", 0))
     data = oracle.Dataset(h.format, h.n, h.d, h.values, h.labels, getattr(h, "col_idx", None), getattr(h, "row_ptr", None))
     run = oracle.Run(ocfg, data, x0)
     theta = spec["theta"]; eta = spec["lr"] / theta if theta else spec["lr"]
@@ -273,6 +394,102 @@ def oracle_training_rounds_per_sec(h, spec, x0, budget_s=6.0):
             break
     sec = (time.perf_counter() - t0) / n
     return {"rounds_per_s": round(1.0 / sec, 3), "cores": 1, "kind": "oracle", "sample": "%d whole rounds at full size" % n}
+
+
+# ---------------------------------------------------------------------------------------------------------------
+# the quantiser/packer grid of the c5 configuration: stage times per point, each with its own clock record
+# ---------------------------------------------------------------------------------------------------------------
+def time_codec_point(dq, vs, x0, gf, M, d, b, bx, sparsify, peak, reps, device_index, eta=0.1):
+    """Median stage times of the codec round over `reps` rounds on the vectors vs (a list of [M][d] device arrays that
+    the rounds rotate over), with the SM clock sampled meanwhile."""
+    import torch
+    cfg = dq.make_config(d, M, b=b, bx=bx, seed=SEED, lambda1=1e-6, sparsify=sparsify, phi=0.01 * d if sparsify else 0.0)
+    rc, ctx = dq.dq_create(cfg); dq.ok(rc, "dq_create")
+    st = dq.State(x0); st.g_full.copy_(gf)
+    msgs = dq.Msgs(cfg)
+    ninf = torch.zeros(M, device="cuda")
+    nbx = dq.dq_packed_bytes(d, bx)
+    codes_x = torch.zeros(nbx, dtype=torch.uint8, device="cuda"); delta_x = torch.zeros(1, device="cuda")
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(reps)]
+    sampler = None
+    for k in range(-3, reps):
+        if k == 0:
+            torch.cuda.synchronize(); sampler = ClockSampler(device_index)
+        vk = vs[k % len(vs)]
+        e = ev[k] if k >= 0 else None
+        if e: e[0].record()
+        dq.ok(dq.dq_norm_inf(ctx, vk, M, ninf))
+        if e: e[1].record()
+        dq.ok(dq.dq_quantize_sparsify_pack(ctx, vk, ninf, 1000 + k, msgs))
+        if e: e[2].record()
+        dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta))
+        if e: e[3].record()
+        dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, 1000 + k, codes_x, delta_x))
+        if e: e[4].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    rc, status = dq.dq_poll_status(ctx); assert rc == 0 and status == 0
+    ms = [sorted(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(reps))[reps // 2] for i in range(4)]   # medians
+    point = {"log2d": d.bit_length() - 1, "b": b, "sparsify": sparsify, "rounds_per_s": round(1000.0 / sum(ms), 1),
+             "stages": stage_report(ms, codec_alg_bytes(M, d, b, bx, sparsify), peak), "clocks": clocks, "reps": reps}
+    if sparsify:      # realised density of worker 0's message: nonzero entries of the dequantised vector
+        out = torch.empty(d, device="cuda")
+        dq.ok(dq.dq_unpack(ctx, msgs, 0, out))
+        point["realised_density"] = round(float(torch.count_nonzero(out).item()) / d, 6)
+        del out
+    dq.dq_destroy(ctx)
+    return point
+
+
+def codec_grid(dq, v, x0, gf, M, bx, peak, device_index, log2ds=(24, 27), with_clean_input=True):
+    """d x b x sparsify off/on.  v [M][2^27] holds the workload's vectors; smaller d take a leading part of it (the same
+    distribution).  At d = 2^20 one set of inputs would sit in L2, so the rounds rotate over enough copies to exceed it."""
+    import torch
+    points = []
+    flat = v.view(-1)
+    for log2d in log2ds:
+        d = 1 << log2d
+        copies = max(1, min((256 << 20) // (M * d * 4), flat.numel() // (M * d)))
+        vs = [flat[c * M * d:(c + 1) * M * d].view(M, d) for c in range(copies)]
+        xs, gs = x0[:d].contiguous(), gf[:d].contiguous()
+        reps = 200 if log2d <= 20 else (40 if log2d <= 24 else 12)
+        for sparsify in (0, 1):
+            for b in (2, 4, 8):
+                points.append(time_codec_point(dq, vs, xs, gs, M, d, b, bx, sparsify, peak, reps, device_index))
+    if with_clean_input:
+        # the budget phi = 0.01 d exceeds ||v||_1/||v||_inf on vectors with x100 outliers (Lemma 2's condition clamps it to
+        # about 0.2 % density); on plain N(0,1) vectors the same budget is feasible and 1 % density is realised
+        d = 1 << 24
+        g = torch.Generator(device="cuda"); g.manual_seed(180510111)
+        clean = torch.randn((M, d), device="cuda", generator=g)
+        p = time_codec_point(dq, [clean], x0[:d].contiguous(), gf[:d].contiguous(), M, d, 4, bx, 1, peak, 40, device_index)
+        p["input"] = "N(0,1) without outliers"
+        points.append(p)
+        del clean
+    return points
+
+
+def time_stage_sustained(fns, min_s, device_index):
+    """Each stage alone in a loop of at least min_s seconds (so that the power cap, not the boost clock, sets the pace),
+    CUDA events around every call, SM clock sampled every 20 ms.  Returns per stage (median ms, clock record)."""
+    import torch
+    out = []
+    for fn in fns:
+        fn(); torch.cuda.synchronize()
+        sampler = ClockSampler(device_index)
+        times = []
+        t0 = time.perf_counter()
+        while time.perf_counter() - t0 < min_s:
+            ev = [torch.cuda.Event(enable_timing=True) for _ in range(33)]
+            ev[0].record()
+            for k in range(32):
+                fn(); ev[k + 1].record()
+            torch.cuda.synchronize()
+            times += [ev[k].elapsed_time(ev[k + 1]) for k in range(32)]
+        clocks = sampler.stop()
+        half = sorted(times[len(times) // 2:])                  # the second half of the loop: the clock has settled
+        out.append((half[len(half) // 2], clocks, len(times)))
+    return out
 
 
 # ---------------------------------------------------------------------------------------------------------------
@@ -295,8 +512,8 @@ def run_ours(a):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dq.lib()
 
-    d, M, b, bx, eta, seed = 1 << a.log2d, a.workers, a.bits, 8, 0.1, 1805
-    cfg = dq.make_config(d, M, b=b, bx=bx, seed=seed, lambda1=1e-6, sparsify=a.sparsify, phi=0.01 * d if a.sparsify else 0.0,
+    d, M, b, bx, eta = 1 << a.log2d, a.workers, a.bits, 8, 0.1
+    cfg = dq.make_config(d, M, b=b, bx=bx, seed=SEED, lambda1=1e-6, sparsify=a.sparsify, phi=0.01 * d if a.sparsify else 0.0,
                          sequential=a.sequential)
     rc, ctx = dq.dq_create(cfg); dq.ok(rc, "dq_create")
 
@@ -316,15 +533,15 @@ def run_ours(a):
     nbx = dq.dq_packed_bytes(d, bx)
     codes_x = torch.zeros(nbx, dtype=torch.uint8, device="cuda"); delta_x = torch.zeros(1, device="cuda")
 
+    stage_fns = [lambda rnd=0: dq.ok(dq.dq_norm_inf(ctx, v, M, ninf)),
+                 lambda rnd=0: dq.ok(dq.dq_quantize_sparsify_pack(ctx, v, ninf, rnd, msgs)),
+                 lambda rnd=0: dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta)),
+                 lambda rnd=0: dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, rnd, codes_x, delta_x))]
+
     def step(rnd, ev=None):
-        if ev: ev[0].record()
-        dq.ok(dq.dq_norm_inf(ctx, v, M, ninf))
-        if ev: ev[1].record()
-        dq.ok(dq.dq_quantize_sparsify_pack(ctx, v, ninf, rnd, msgs))
-        if ev: ev[2].record()
-        dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta))
-        if ev: ev[3].record()
-        dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, rnd, codes_x, delta_x))
+        for i, fn in enumerate(stage_fns):
+            if ev: ev[i].record()
+            fn(rnd)
         if ev: ev[4].record()
 
     def barrier():
@@ -332,7 +549,8 @@ def run_ours(a):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for rnd in range(max(3, a.warmup)):
+    warm = max(3, a.warmup)
+    for rnd in range(warm):
         step(rnd)
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(a.steps)]
     barrier()
@@ -353,9 +571,22 @@ def run_ours(a):
     total_ms = max_over_ranks(total_ms, dist, "cuda")
     ms_per_step = total_ms / a.steps
     value = whole_job_rate(world, a.steps, total_ms)
+    peak, peak_src = measured_peak()
+    alg = codec_alg_bytes(M, d, b, bx, a.sparsify)
+
+    # every stage alone, long enough for the clock to settle under the power cap
+    sustained = None
+    if rank == 0 and world == 1 and a.sustain_s > 0:
+        res = time_stage_sustained(stage_fns, a.sustain_s, local)
+        sustained = {}
+        for n, (ms, ck, calls), by in zip(STAGE_NAMES, res, alg):
+            sustained[n] = {"ms": round(ms, 4), "alg_GBps": round(by / ms / 1e6, 1), "frac_of_peak": round(by / ms / 1e6 / peak, 4),
+                            "frac_of_8TBps": round(by / ms / 1e6 / NOMINAL_HBM_GBPS, 4), "sm_mhz": ck.get("sm_mhz"),
+                            "ms_x_mhz": None if ck.get("sm_mhz") is None else round(ms * ck["sm_mhz"], 1),
+                            "power_w_max": ck.get("power_w_max"), "reasons": ck.get("reasons"), "calls": calls}
 
     # the optional width search of condition (3) on the same model (not part of the default round, mu = 0)
-    sel_bits = torch.zeros(1, dtype=torch.int32, device="cuda"); sel_stats = torch.zeros(4, dtype=torch.float64, device="cuda")
+    sel_bits = torch.zeros(1, dtype=torch.int32, device="cuda"); sel_stats = torch.zeros(11, dtype=torch.float64, device="cuda")
     xs_dev = torch.from_numpy(x0).cuda()
     for _ in range(3):
         dq.ok(dq.dq_select_model_bits(ctx, st.x, xs_dev, st.norm_x, 1.0, sel_bits, sel_stats))
@@ -388,15 +619,7 @@ def run_ours(a):
         if dist is not None:
             dist.destroy_process_group()
         return
-    peak, peak_src = measured_peak()
-    # algorithmic bytes per launch: norm 4 B, quantise+pack 4 + b/8 B per message
-    # coordinate (8 + b/8 when sparsifying); master M*b/8 + 12 B, model quantise 4 + b_x/8 B per model coordinate.
-    # With sparsification the quantise stage is two passes over the vectors (||v||_1, which Lemma 2's probabilities
-    # need before the first mask bit can be drawn, then the mask pass that stages the survivors) plus the packed output.
-    alg = [M * d * 4.0, M * d * ((8.0 if a.sparsify else 4.0) + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
-    names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
-    stages = {n: {"ms": round(ms, 4), "alg_GBps": round(by / ms / 1e6, 1), "frac_of_peak": round(by / ms / 1e6 / peak, 4)}
-              for n, ms, by in zip(names, stage_ms, alg)}
+    stages = stage_report(stage_ms, alg, peak)
     stages["select_model_bits(optional)"] = {"ms": round(select_ms, 4), "alg_GBps": round(d * 8.0 / select_ms / 1e6, 1),
                                               "frac_of_peak": round(d * 8.0 / select_ms / 1e6 / peak, 4)}
     qp = stages["quantize_pack"]
@@ -404,83 +627,61 @@ def run_ours(a):
     roofline = {"kernel": "quantize_pack_kernel<%d>" % b if not a.sparsify else "norm_l1_kernel + sparsify_stage_kernel + sparsify_scatter_dense_kernel<%d>" % b,
                 "bound": "hbm", "achieved": qp["alg_GBps"], "peak": peak, "unit": "GB/s",
                 "frac": round(qp["alg_GBps"] / peak, 4), "peak_source": peak_src,
+                "frac_of_8TBps": qp["frac_of_8TBps"],
+                "regime": "timed steps: %d steps, median SM clock %s MHz, reasons %s" % (a.steps, clocks.get("sm_mhz"), clocks.get("reasons")),
                 "traffic": None if tr is None else tr * M * d,
                 "alg_bytes_per_launch": alg[1]}
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": max(3, a.warmup),
+    if sustained:
+        roofline["sustained"] = {k: sustained["quantize_pack"][k] for k in ("ms", "alg_GBps", "frac_of_peak", "sm_mhz", "reasons")}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": a.steps, "warmup": warm,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": workload_config(a), "roofline": roofline,
-            "stages": stages, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+            "stages": stages, "stages_sustained": sustained, "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "bits_per_round": {"down": M * (32 + bx * d), "up_dense": M * (32 + b * d), "full_precision": 2 * M * 32 * d}}
-    if world == 1 and not a.no_cpu_baseline:
-        val, sec, what = oracle_rounds_per_sec(a, steps=6, warmup=1)
-        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what}
     dq.dq_destroy(ctx)
-    del v, hv, st, msgs
+    del st, msgs
+    if world == 1 and not a.no_sweep and a.log2d >= 27:
+        xd = torch.from_numpy(x0).cuda(); gd = torch.from_numpy(gf).cuda()
+        line["sweep"] = {"what": "c5 grid: M=%d, b_x=8, lambda1=1e-6, eta=0.1, phi=0.01d when sparsifying; medians over `reps` rounds; "
+                                 "fractions of the measured copy peak and of the nominal 8 TB/s" % M,
+                         "peak_GBps": peak, "points": codec_grid(dq, v, xd, gd, M, bx, peak, local)}
+        below = [(p["log2d"], p["b"], p["sparsify"], n, s["frac_of_peak"]) for p in line["sweep"]["points"]
+                 for n, s in p["stages"].items() if n in ("quantize_pack", "master_unpack_aggregate_prox") and s["frac_of_peak"] < 0.70]
+        line["sweep"]["below_0.70_of_measured_peak"] = below
+        del xd, gd
+    del v
     torch.cuda.empty_cache()
+    if world == 1 and not a.no_cpu_baseline:
+        threads = host_threads(M)
+        val, sec, what = oracle_rounds_per_sec(a, steps=2, warmup=0, log2_sample=24, threads=threads)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": what,
+                                "seconds_per_sampled_round": round(sec, 3), "extrapolated": a.log2d > 24}
+        if threads > 1:
+            val1, sec1, _ = oracle_rounds_per_sec(a, steps=1, warmup=0, log2_sample=22, threads=1)
+            line["cpu_baseline"]["single_thread_value"] = val1
+    del hv
     if world == 1 and a.configs:
-        line["training_configs"] = {c: time_training_config(c, with_oracle=not a.no_cpu_baseline)
+        line["training_configs"] = {c: time_training_config(c, with_oracle=not a.no_cpu_baseline, peak=peak)
                                     for c in a.configs.split(",") if c in TRAIN_CONFIGS}
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
 
 
-# ---------------------------------------------------------------------------------------------------------------
-# the quantiser/packer sweep of the c5 configuration (stage times only; inputs are drawn on the device)
-# ---------------------------------------------------------------------------------------------------------------
 def run_sweep(a):
+    """Only the grid (with d = 2^20 added), on vectors drawn on the device."""
     import torch
     import paper_1805_10111_b200 as dq
     torch.cuda.set_device(0)
     dq.lib()
     peak, peak_src = measured_peak()
-    M, bx, eta = a.workers, 8, 0.1
-    points = []
-    for log2d in (20, 24, 27):
-        d = 1 << log2d
-        g = torch.Generator(device="cuda"); g.manual_seed(180510111 + log2d)
-        v = torch.randn((M, d), device="cuda", generator=g)
-        idx = torch.randint(0, d, (M, max(1, d // 1000)), device="cuda", generator=g)
-        v.scatter_(1, idx, v.gather(1, idx) * 100.0)                      # 0.1 % outliers x100
-        x0 = torch.randn(d, device="cuda", generator=g); gf = torch.randn(d, device="cuda", generator=g)
-        # at d = 2^20 one set of inputs (36 MiB) would sit in L2: rotate over enough copies to exceed it
-        copies = max(1, (256 << 20) // (M * d * 4))
-        vs = [v] + [v.clone() for _ in range(copies - 1)]
-        for sparsify in (0, 1):
-            for b in (2, 4, 8):
-                cfg = dq.make_config(d, M, b=b, bx=bx, seed=1805, lambda1=1e-6, sparsify=sparsify, phi=0.01 * d if sparsify else 0.0)
-                rc, ctx = dq.dq_create(cfg); dq.ok(rc, "dq_create")
-                st = dq.State(x0); st.g_full.copy_(gf)
-                msgs = dq.Msgs(cfg)
-                ninf = torch.zeros(M, device="cuda")
-                nbx = dq.dq_packed_bytes(d, bx)
-                codes_x = torch.zeros(nbx, dtype=torch.uint8, device="cuda"); delta_x = torch.zeros(1, device="cuda")
-                steps = 200 if log2d <= 20 else (60 if log2d <= 24 else 20)
-                ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
-                for k in range(-3, steps):
-                    vk = vs[k % copies]
-                    e = ev[k] if k >= 0 else None
-                    if e: e[0].record()
-                    dq.ok(dq.dq_norm_inf(ctx, vk, M, ninf))
-                    if e: e[1].record()
-                    dq.ok(dq.dq_quantize_sparsify_pack(ctx, vk, ninf, 1000 + k, msgs))
-                    if e: e[2].record()
-                    dq.ok(dq.dq_master_unpack_aggregate_prox(ctx, msgs, st, eta))
-                    if e: e[3].record()
-                    dq.ok(dq.dq_quantize_model(ctx, st.x, st.norm_x, 1000 + k, codes_x, delta_x))
-                    if e: e[4].record()
-                torch.cuda.synchronize()
-                rc, status = dq.dq_poll_status(ctx); assert rc == 0 and status == 0
-                ms = [sorted(ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(steps))[steps // 2] for i in range(4)]   # medians
-                alg = [M * d * 4.0, M * d * ((8.0 if sparsify else 4.0) + b / 8.0), d * (M * b / 8.0 + 12.0), d * (4.0 + bx / 8.0)]
-                names = ["norm_inf", "quantize_pack", "master_unpack_aggregate_prox", "quantize_model"]
-                points.append({"log2d": log2d, "b": b, "sparsify": sparsify, "rounds_per_s": round(1000.0 / sum(ms), 1),
-                               "stages": {n: {"ms": round(t, 4), "alg_GBps": round(by / t / 1e6, 1), "frac_of_peak": round(by / t / 1e6 / peak, 3)}
-                                          for n, t, by in zip(names, ms, alg)}})
-                dq.dq_destroy(ctx)
-                del st, msgs
-        del v, vs, x0, gf
-        torch.cuda.empty_cache()
+    M, d = a.workers, 1 << 27
+    g = torch.Generator(device="cuda"); g.manual_seed(180510111 + 27)
+    v = torch.randn((M, d), device="cuda", generator=g)
+    idx = torch.randint(0, d, (M, max(1, d // 1000)), device="cuda", generator=g)
+    v.scatter_(1, idx, v.gather(1, idx) * 100.0)                      # 0.1 % outliers x100
+    x0 = torch.randn(d, device="cuda", generator=g); gf = torch.randn(d, device="cuda", generator=g)
+    points = codec_grid(dq, v, x0, gf, M, 8, peak, 0, log2ds=(20, 24, 27))
     print(json.dumps({"sweep": "c5 quantiser/packer: M=%d, b_x=8, lambda1=1e-6, eta=0.1, phi=0.01d when sparsifying" % M,
                       "peak_GBps": peak, "peak_source": peak_src, "l2_policy": "inputs rotated over >= 256 MiB", "points": points}))
 

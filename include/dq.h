@@ -25,7 +25,11 @@
  *   - All random draws come from Philox4x32-10 with key = seed and counter
  *     (coordinate >> 3, round, worker, stream); the master's worker id is 0xFFFFFFFF; streams are
  *     0 model rounding, 1 gradient rounding, 2 sparsification mask, 3 minibatch sampling.  Equal
- *     (seed, round, inputs) give equal bytes.
+ *     (seed, round, inputs) give equal bytes from every stage of a round on the same kernel path: dense rows are
+ *     summed in slot order, CSR rows on an exact integer grid, norms as integer maxima / integer sums.  (The
+ *     one-cluster kernel and the separate kernels form a row's margin in different orders; each agrees with itself.)
+ *     The exception is dq_epoch_begin: the epoch's full gradient is summed with double-precision atomics, so a
+ *     coordinate of g_full may differ in its last place between two runs.
  *
  * Packed code layout (message of Section 3.1: 32 bits for delta plus b bits per coordinate): codes are b-bit
  * two's complement fields laid end to end: coordinate j occupies bits [j b, (j+1) b) of the message, bit k of the

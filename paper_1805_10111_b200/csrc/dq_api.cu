@@ -1,5 +1,6 @@
 // C ABI of libdq (see include/dq.h): argument checks, scratch ownership and the order of kernel launches.
 #include <math.h>
+#include <string.h>
 #include <new>
 
 #include "dq_kernels.cuh"
@@ -163,6 +164,22 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
                 rc |= dev_alloc(&c->mlp_dz[k], rmax * cfg->classes);
             }
         }
+        if (data->format == DQ_CSR_F32) {
+            // integer grid of the CSR gradient accumulator: a minibatch sum is at most max |a_ij| in magnitude (B terms
+            // of at most max |a_ij| / B), so with max |a_ij| < 2^e one unit of 2^(e-61) keeps every sum below 2^61
+            rc |= dev_alloc(&c->acc64, (size_t)M * d);
+            int64_t nnz = 0; uint32_t vbits = 0;
+            if (rc == DQ_OK && (cudaMemset(c->acc64, 0, sizeof(long long) * M * d) != cudaSuccess ||
+                                cudaMemcpy(&nnz, data->row_ptr + data->n, sizeof(int64_t), cudaMemcpyDeviceToHost) != cudaSuccess)) rc = DQ_ERR_CUDA;
+            if (rc == DQ_OK && nnz > 0) {
+                launch_norm_inf(c, static_cast<const float*>(data->values), nnz, 1, c->xnorm_bits, nullptr);
+                if (cudaMemcpy(&vbits, c->xnorm_bits, sizeof(uint32_t), cudaMemcpyDeviceToHost) != cudaSuccess) rc = DQ_ERR_CUDA;
+            }
+            float vmax; memcpy(&vmax, &vbits, sizeof(float));
+            int e = 0;
+            if (vbits != 0u && vbits < 0x7F800000u) (void)frexpf(vmax, &e);
+            c->acc_scale = ldexp(1.0, 61 - e); c->acc_inv = ldexp(1.0, e - 61);
+        }
         c->list_mode = sparse && data->format == DQ_CSR_F32;
         if (c->list_mode) {
             c->glist_cap = (d + 7) / 8;
@@ -180,6 +197,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (rc == DQ_OK && cudaMemset(c->bx_dev, 0, sizeof(int32_t)) != cudaSuccess) rc = DQ_ERR_CUDA;
     if (rc != DQ_OK) { dq_destroy(c); cudaGetLastError(); return DQ_ERR_CUDA; }
     c->epoch = -1;
+    if (fused_grad_setup(c) != DQ_OK) { dq_destroy(c); cudaGetLastError(); return DQ_ERR_CUDA; }
     small_round_setup(c);
     *out = c;
     return DQ_OK;
@@ -190,7 +208,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->norm_block, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->delays_dev, c->slots_dev, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->rbuf, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->acc64, c->rbuf, c->fused_part, c->fused_cnt, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);

@@ -1205,8 +1205,9 @@ __global__ void unpack_sparse_kernel(const uint8_t* __restrict__ codes, const fl
 
 // ---------------------------------------------------------------------------------------------------
 // Sparse gradients.  The worker kernel marks every group of eight coordinates it adds to in a bitmap.
-// build_group_list turns each worker's bitmap into the ascending list of those groups, clears the bitmap
-// and folds ||alpha_w||_inf over the listed groups (all other coordinates are zero).  One block per worker.
+// build_group_list turns each worker's bitmap into the ascending list of those groups, clears the bitmap,
+// turns the integer accumulator of the listed groups into alpha_w (one rounding to fp32; the accumulator is
+// zeroed again) and folds ||alpha_w||_inf over them (all other coordinates are zero).
 // ---------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads)
 count_touched_kernel(const uint32_t* __restrict__ touched, int64_t bm_words, uint32_t* __restrict__ seg_count, int nseg)
@@ -1229,7 +1230,7 @@ count_touched_kernel(const uint32_t* __restrict__ touched, int64_t bm_words, uin
 
 __global__ void __launch_bounds__(kThreads)
 build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const uint32_t* __restrict__ seg_count, int nseg,
-                        const float* __restrict__ alpha, int64_t d, int vec_ok,
+                        FixedAcc fa, float* __restrict__ alpha, int64_t d,
                         uint32_t* __restrict__ glist, int64_t cap, uint32_t* __restrict__ gcount, uint32_t* __restrict__ norm_bits)
 {
     pdl_prologue();
@@ -1237,7 +1238,8 @@ build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const 
     const int w = blockIdx.y;
     uint32_t* bm = touched + (int64_t)w * bm_words;
     uint32_t* list = glist + (int64_t)w * cap;
-    const float* row = alpha + (int64_t)w * d;
+    float* row = alpha + (int64_t)w * d;
+    long long* acc = fa.acc + (int64_t)w * d;
     __shared__ uint32_t s_warp[kThreads / 32];
     __shared__ uint32_t s_base[kThreads / 32];
     // base = sum of the earlier segments' counts (all threads help)
@@ -1262,10 +1264,16 @@ build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const 
         const int bit = __ffs(word) - 1; word &= word - 1;
         const int64_t g = (i << 5) + bit, i0 = g << 3;
         list[pos++] = (uint32_t)g;
-        float a[8];
-        if (vec_ok && i0 + 8 <= d) load8(row + i0, a); else load8_guarded(row, i0, d, a);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) nmax = max(nmax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
+        for (int j = 0; j < 8; ++j) {
+            if (i0 + j < d) {
+                const long long q = acc[i0 + j];
+                if (q != 0) acc[i0 + j] = 0;
+                const float a = (float)((double)q * fa.inv_scale);
+                row[i0 + j] = a;
+                nmax = max(nmax, __float_as_uint(a) & 0x7FFFFFFFu);
+            }
+        }
     }
     block_atomic_max(nmax, norm_bits + w);
 }
@@ -1500,8 +1508,9 @@ void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st)
     const int nseg = (int)((ctx->bm_words + kThreads - 1) / kThreads);
     dim3 grid(nseg, c.M);
     launch_k(count_touched_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg);
-    launch_k(build_group_list_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg, ctx->alpha, c.d,
-                                                        vec_ok_for(ctx->alpha, c.d), ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
+    const FixedAcc fa = {ctx->acc64, ctx->acc_scale, ctx->acc_inv};
+    launch_k(build_group_list_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg, fa, ctx->alpha, c.d,
+                                                        ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
     ctx->launches += 2;
     ctx->launches += 1;
 }

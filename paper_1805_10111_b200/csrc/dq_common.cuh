@@ -214,6 +214,9 @@ __device__ __forceinline__ int64_t group_at(const GroupList& gl, int w, int64_t 
     return (p < (int64_t)gl.count[w]) ? (int64_t)gl.groups[(int64_t)w * gl.cap + p] : -1;
 }
 
+// Integer accumulator of the CSR worker gradients: acc [M][d], one unit = 1 / scale (scale a power of two).
+struct FixedAcc { long long* acc; double scale; double inv_scale; };
+
 // Transmitted-bit counters of a round, written by the master kernel when `down` is set (Section 3.1 message sizes).
 struct BitsArgs { uint64_t* down; uint64_t* up; const uint32_t* nnz; int flag_round, sparse_msgs, bx, b;
                   const int32_t* bx_dev; /* width chosen on the device this round, overrides bx when set */ };
@@ -283,10 +286,14 @@ struct dq_ctx {
     float* delta_x;
     float* xhat_diff;           // [d] dequantised model minus snapshot
     double* g64;                // [d] full-gradient accumulator
+    long long* acc64;           // [M][d] CSR data: integer accumulator of the worker gradients, all-zero between rounds
+    double acc_scale, acc_inv;  // its grid: one unit is 2^-shift, shift from max |a_ij| so that a minibatch sum cannot overflow
     float* rbuf;                // [M][B] slope differences of the sampled rows
+    float* fused_part;          // [SMs + M][d] column sums per (block, worker) of the one-pass dense gradient kernel; NULL: not in use
+    uint32_t* fused_cnt;        // [M] blocks that have handed in their sums for a worker (zero between launches)
     int32_t* bx_dev;            // model width chosen by condition (3) this round
     // network workload: sampled-row indices and per-row activations / derivatives of the two parameter vectors
-    int32_t* mlp_rows; float* mlp_act[2]; float* mlp_dz[2]; float* mlp_dh[2];
+    int32_t* mlp_rows; double* mlp_act[2]; float* mlp_dz[2]; float* mlp_dh[2];
     double* prec_stats;         // [4] expected errors at 2/4/8 bits and ||x - xsnap||^2
     dq_msgs msgs;
     uint64_t* bits;             // [2] device counters

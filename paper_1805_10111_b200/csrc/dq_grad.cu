@@ -1,6 +1,6 @@
 // Gradient kernels: the worker's variance-reduced minibatch gradient (Algorithm 1 step 11), the epoch's
 // full gradient (step 5), the epoch-boundary state update (steps 3/14, Algorithm 3 steps 3/15), the
-// objective of eq. (1) and the transmitted-bit counters.  f_a(x) = log(1 + exp(-y_a <a_a, x>)).
+// objective of eq. (1).  f_a(x) = log(1 + exp(-y_a <a_a, x>)).
 #include <cuda_bf16.h>
 #include <type_traits>
 
@@ -120,12 +120,22 @@ __global__ void dequant_diff_kernel(const uint8_t* __restrict__ codes, const flo
 
 // ---------------------------------------------------------------------------------------------------
 // CSR worker gradient: one warp per sampled row.  dz = <a, xhat - xsnap>, slope difference, then the
-// row is scattered into alpha_w with fp32 atomics (alpha must be zero on entry).
+// row is scattered into the worker's accumulator.  The scatter meets other rows of the minibatch in any order,
+// so the accumulator is an integer grid on which addition is exact: every term r_a a_ai (the product is exact in
+// double) is rounded once to a multiple of 2^-shift and added as a 64-bit integer.  shift is chosen by the host
+// from max |a_ai| so that the sum of a minibatch cannot overflow (|r_a| <= 1/B).  Equal inputs therefore give
+// equal bits whatever the order of the atomics; acc_to_alpha_kernel / build_group_list_kernel turn the integers
+// into alpha_w (one rounding to fp32) and put the zeros back.  acc must be zero on entry.
 // ---------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void fixed_add(long long* dst, float r, float a, double scale)
+{
+    atomicAdd(reinterpret_cast<unsigned long long*>(dst), (unsigned long long)__double2ll_rn((double)r * (double)a * scale));
+}
+
 __global__ void __launch_bounds__(kThreads)
 worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict__ col, const int64_t* __restrict__ row_ptr,
                        const float* __restrict__ labels, const float* __restrict__ diff, const float* __restrict__ z_snap,
-                       const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, float* __restrict__ alpha,
+                       const __grid_constant__ PhiloxKeys K, BatchSource bs, int M, int B, int64_t d, FixedAcc fa,
                        uint32_t* __restrict__ touched /* bitmap of groups of eight coordinates, may be NULL */, int64_t bm_words)
 {
     pdl_prologue();
@@ -138,11 +148,11 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
     const int64_t k0 = row_ptr[a], k1 = row_ptr[a + 1];
     const float dz = (float)warp_dot_csr(val, col, k0, k1, diff_of_worker(bs, diff, w), lane);
     const float r = slope_difference(labels[a], z_snap[a], dz) / (float)B;
-    float* out = alpha + (int64_t)w * d;
+    long long* out = fa.acc + (int64_t)w * d;
     uint32_t* bm = touched ? touched + (int64_t)w * bm_words : nullptr;
     for (int64_t k = k0 + lane; k < k1; k += 32) {
         const int32_t c = __ldg(col + k);
-        atomicAdd(out + c, r * __ldg(val + k));
+        fixed_add(out + c, r, __ldg(val + k), fa.scale);
         if (bm) {
             const uint32_t bit = 1u << ((c >> 3) & 31);
             uint32_t* word = bm + (c >> 8);
@@ -151,10 +161,31 @@ worker_grad_csr_kernel(const float* __restrict__ val, const int32_t* __restrict_
     }
 }
 
+// alpha_w = the accumulated integers scaled back (one rounding to fp32), ||alpha_w||_inf, and the accumulator is
+// left all-zero for the next round.  grid (blocks, M); norm_bits must be zero on entry.
+__global__ void __launch_bounds__(kThreads)
+acc_to_alpha_kernel(FixedAcc fa, int64_t d, float* __restrict__ alpha, uint32_t* __restrict__ norm_bits)
+{
+    pdl_prologue();
+    const int w = blockIdx.y;
+    long long* acc = fa.acc + (int64_t)w * d;
+    float* out = alpha + (int64_t)w * d;
+    uint32_t nmax = 0;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
+        const long long q = acc[i];
+        if (q != 0) acc[i] = 0;
+        const float a = (float)((double)q * fa.inv_scale);
+        out[i] = a;
+        nmax = max(nmax, __float_as_uint(a) & 0x7FFFFFFFu);
+    }
+    block_atomic_max(nmax, norm_bits + w);
+}
+
 // ---------------------------------------------------------------------------------------------------
-// Dense worker gradient (fp32 or bf16 features).  grid (ceil(B / kRowsPerBlock), M).  Phase A: one warp
-// per row computes the slope difference; phase B: threads own columns and add the block's rows.
-// alpha must be zero on entry when more than one block serves a worker.
+// Dense worker gradient (fp32 or bf16 features) for small minibatches and for rows off the 16-byte grid.
+// grid (1, M): one block per worker takes the minibatch in chunks of kRowsPerBlock rows.  Phase A: one warp
+// per row computes the slope difference; phase B: threads own columns and add the chunk's rows in slot order,
+// so alpha_w is the same bit pattern on every run (no atomics).
 // ---------------------------------------------------------------------------------------------------
 template <class T>
 __global__ void __launch_bounds__(kThreads)
@@ -167,19 +198,21 @@ worker_grad_dense_kernel(const T* __restrict__ X, const float* __restrict__ labe
     __shared__ int64_t s_row[kRowsPerBlock];
     clear_word(bs);
     const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int j0 = blockIdx.x * kRowsPerBlock;
-    const int nrows = min(kRowsPerBlock, B - j0);
-    for (int j = warp; j < nrows; j += kThreads / 32) {
-        const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
-        const float dz = (float)warp_dot_dense(X + a * d, diff_of_worker(bs, diff, w), d, lane);
-        if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_row[j] = a; }
-    }
-    __syncthreads();
     float* out = alpha + (int64_t)w * d;
-    for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
-        float s = 0.0f;
-        for (int j = 0; j < nrows; ++j) s = fmaf(s_r[j], to_float(X[s_row[j] * d + i]), s);
-        if (gridDim.x == 1) out[i] = s; else atomicAdd(out + i, s);
+    for (int j0 = 0; j0 < B; j0 += kRowsPerBlock) {
+        const int nrows = min(kRowsPerBlock, B - j0);
+        for (int j = warp; j < nrows; j += kThreads / 32) {
+            const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
+            const float dz = (float)warp_dot_dense(X + a * d, diff_of_worker(bs, diff, w), d, lane);
+            if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_row[j] = a; }
+        }
+        __syncthreads();
+        for (int64_t i = threadIdx.x; i < d; i += blockDim.x) {
+            float s = j0 == 0 ? 0.0f : out[i];                   // the same thread wrote it one chunk ago
+            for (int j = 0; j < nrows; ++j) s = fmaf(s_r[j], to_float(X[s_row[j] * d + i]), s);
+            out[i] = s;
+        }
+        __syncthreads();
     }
 }
 
@@ -226,9 +259,9 @@ __device__ __forceinline__ double warp_dot_dense_vec(const T* __restrict__ row, 
     return warp_sum(((double)s[0] + (double)s[1]) + ((double)s[2] + (double)s[3]));
 }
 
-// Vectorised dense worker gradient: same plan as worker_grad_dense_kernel with 16-byte loads and
-// 16-byte atomics (d a multiple of the vector width).  The rows read in phase A are read again in phase
-// B while they are still in L2.
+// Vectorised dense worker gradient: same plan as worker_grad_dense_kernel with 16-byte loads and stores
+// (d a multiple of the vector width).  The rows read in phase A are read again in phase B while they are
+// still in L2.
 template <class T>
 __global__ void __launch_bounds__(kThreads)
 worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
@@ -241,34 +274,36 @@ worker_grad_dense_vec_kernel(const T* __restrict__ X, const float* __restrict__ 
     __shared__ const uint4* s_rowp[kRowsPerBlock];
     clear_word(bs);
     const int w = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int j0 = blockIdx.x * kRowsPerBlock;
-    const int nrows = min(kRowsPerBlock, B - j0);
-    for (int j = warp; j < nrows; j += kThreads / 32) {
-        const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
-        const float dz = (float)warp_dot_dense_vec(X + a * d, diff_of_worker(bs, diff, w), d, lane);
-        if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_rowp[j] = reinterpret_cast<const uint4*>(X + a * d); }
-    }
-    __syncthreads();
     const int nv = (int)(d / N);
     float* out = alpha + (int64_t)w * d;
-    for (int v = threadIdx.x; v < nv; v += blockDim.x) {
-        float acc[N];
+    for (int j0 = 0; j0 < B; j0 += kRowsPerBlock) {
+        const int nrows = min(kRowsPerBlock, B - j0);
+        for (int j = warp; j < nrows; j += kThreads / 32) {
+            const int64_t a = batch_row(bs, K, w, j0 + j, B, lane == 0);
+            const float dz = (float)warp_dot_dense_vec(X + a * d, diff_of_worker(bs, diff, w), d, lane);
+            if (lane == 0) { s_r[j] = slope_difference(labels[a], z_snap[a], dz) / (float)B; s_rowp[j] = reinterpret_cast<const uint4*>(X + a * d); }
+        }
+        __syncthreads();
+        for (int v = threadIdx.x; v < nv; v += blockDim.x) {
+            float acc[N];
+            float4* o4 = reinterpret_cast<float4*>(out + (int64_t)v * N);
 #pragma unroll
-        for (int q = 0; q < N; ++q) acc[q] = 0.0f;
+            for (int q = 0; q < N / 4; ++q) {                     // the same thread wrote it one chunk ago
+                const float4 prev = j0 == 0 ? make_float4(0.0f, 0.0f, 0.0f, 0.0f) : o4[q];
+                acc[q * 4] = prev.x; acc[q * 4 + 1] = prev.y; acc[q * 4 + 2] = prev.z; acc[q * 4 + 3] = prev.w;
+            }
 #pragma unroll 4
-        for (int j = 0; j < nrows; ++j) {
-            float f[N];
-            RowVec<T>::unpack(__ldg(s_rowp[j] + v), f);
-            const float r = s_r[j];
+            for (int j = 0; j < nrows; ++j) {
+                float f[N];
+                RowVec<T>::unpack(__ldg(s_rowp[j] + v), f);
+                const float r = s_r[j];
 #pragma unroll
-            for (int q = 0; q < N; ++q) acc[q] = fmaf(r, f[q], acc[q]);
-        }
-        float4* o4 = reinterpret_cast<float4*>(out + (int64_t)v * N);
+                for (int q = 0; q < N; ++q) acc[q] = fmaf(r, f[q], acc[q]);
+            }
 #pragma unroll
-        for (int q = 0; q < N / 4; ++q) {
-            const float4 val = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
-            if (gridDim.x == 1) o4[q] = val; else atomicAdd(o4 + q, val);
+            for (int q = 0; q < N / 4; ++q) o4[q] = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
         }
+        __syncthreads();
     }
 }
 
@@ -353,6 +388,295 @@ worker_colsum_kernel(const T* __restrict__ X, const int32_t* __restrict__ rows, 
         }
     }
     block_atomic_max(nmax, norm_bits + w);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Dense worker gradient in ONE pass over the sampled rows (Algorithm 1 step 11 for large minibatches).
+// alpha_w = sum_j r_j a_j needs r_j = slope difference of row j, which needs the whole row's margin: a two-kernel
+// plan reads every row twice.  Here a row is staged on chip once and used for both.
+//
+//   tiles      a tile is kFusedRows consecutive minibatch slots of one worker; the M * ceil(B / 8) tiles are split
+//              into contiguous runs, one run per block (one block per SM)
+//   staging    warp 1 draws the tile's row indices and issues one bulk asynchronous copy per row into a ring of
+//              kFusedStages shared-memory stages; an mbarrier per stage counts the bytes
+//   margins    thread v owns the 16-byte column group v of every row: it keeps the tile's eight groups in registers,
+//              forms eight partial dot products with its slice of xhat - xsnap, the warp folds them in a fixed
+//              butterfly, and warp 0 adds the warps' partial sums in warp order (double) and turns the eight margins
+//              into slope differences
+//   columns    one tile later every thread adds r_j * row_j to its columns from the registers it kept
+//   combine    a block's column sums for a worker go to a scratch slot; the block that completes a worker (a
+//              counter tells it; nobody waits) adds that worker's slots in block order, writes alpha_w and
+//              ||alpha_w||_inf.  The order of every sum is fixed, so alpha is reproducible bit for bit.
+// The only waits are on the stage barriers; each is bounded, after which the block records DQ_ERR_TIMEOUT, waits
+// (bounded again) for the copies it still has in flight and returns.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kFusedRows = 8;                      // rows per tile
+constexpr int kFusedStages = 3;                    // tiles in flight per block
+constexpr int kFusedWarps = 16;                    // sixteen warps: four per scheduler, 128 registers each
+constexpr int kFusedThreads = kFusedWarps * 32;
+constexpr int kFusedMaxRowBytes = 8192;            // one 16-byte group per thread
+constexpr int kFusedRowPad = 16;                   // bytes between staged rows beyond the row itself (bank spread)
+constexpr long long kFusedWaitCycles = 1ll << 31;  // about a second: no copy takes that long
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" :: "r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Waits for the phase with the given parity, for at most kFusedWaitCycles clock cycles.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (clock64() - t0 > kFusedWaitCycles) return false;
+    }
+    return true;
+}
+// One row: global -> shared, completion counted in bytes on the stage's barrier (both addresses and the size are
+// multiples of 16).  The copy is this block's own: no multicast.
+__device__ __forceinline__ void bulk_row_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+// Eight per-lane values -> per-row sums over the warp in 9 shuffles: each step hands half of the remaining rows
+// to the partner lane.  Afterwards lane L holds the sum of row ((L >> 4) & 1) * 4 + ((L >> 3) & 1) * 2 + ((L >> 2) & 1).
+__device__ __forceinline__ float fold8(float (&p)[8], int lane)
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float send = (lane & 16) ? p[i] : p[i + 4], keep = (lane & 16) ? p[i + 4] : p[i];
+        p[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float send = (lane & 8) ? p[i] : p[i + 2], keep = (lane & 8) ? p[i + 2] : p[i];
+        p[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 8);
+    }
+    {
+        const float send = (lane & 4) ? p[0] : p[1], keep = (lane & 4) ? p[1] : p[0];
+        p[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 4);
+    }
+    p[0] += __shfl_xor_sync(0xFFFFFFFFu, p[0], 2);
+    p[0] += __shfl_xor_sync(0xFFFFFFFFu, p[0], 1);
+    return p[0];
+}
+
+// Work split of the fused kernel: worker and first slot of tile t, the run of tiles of block b.
+struct FusedPlan {
+    int M, B, tiles_per_worker, ntiles, nblocks;
+    __host__ __device__ int tile_begin(int b) const { return (int)(((long long)b * ntiles) / nblocks); }
+    __host__ __device__ int worker_of(int t) const { return t / tiles_per_worker; }
+    // blocks whose runs touch worker w: the owners of its first and last tile
+    __host__ __device__ int block_of_tile(int t) const
+    {
+        int b = (int)(((long long)t * nblocks) / ntiles);          // tile_begin(b) <= t holds for this b or the next ones
+        while (b + 1 < nblocks && tile_begin(b + 1) <= t) ++b;
+        while (tile_begin(b) > t) --b;
+        return b;
+    }
+};
+
+template <class T>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
+                         const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, FusedPlan pl,
+                         int64_t d, float* __restrict__ alpha, uint32_t* __restrict__ norm_bits,
+                         float* __restrict__ part /* [nblocks + M][d] column sums of (block, worker) */,
+                         uint32_t* __restrict__ counters /* [M], zero between launches */, int* __restrict__ status)
+{
+    pdl_prologue();
+    clear_word(bs);
+    constexpr int N = RowVec<T>::N;                          // features per 16-byte group
+    constexpr int S = kFusedStages, R = kFusedRows;
+    extern __shared__ __align__(128) unsigned char s_stage[];    // [S][R][row_bytes + pad]
+    __shared__ __align__(8) uint64_t s_full[S];
+    __shared__ float s_part[2][kFusedWarps][R];
+    __shared__ float s_r[2][R];
+    __shared__ float s_lab[S + 1][R], s_zs[S + 1][R];           // ring of S + 1: tile it + S is issued while tile it's entries are read
+    __shared__ uint32_t s_max[kFusedWarps];
+    __shared__ int s_abort, s_last, s_issued;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool slope_warp = warp == 0, load_warp = warp == 1;       // the two extra duties sit on different warps so that they overlap
+    const int row_bytes = (int)(d * (int64_t)sizeof(T)), stride = row_bytes + kFusedRowPad;
+    const int nvec = row_bytes >> 4;
+    const int v = tid;                                       // this thread's column group
+    const bool active = v < nvec;
+    const int blk = blockIdx.x;
+    const int t0 = pl.tile_begin(blk), ntl = pl.tile_begin(blk + 1) - t0;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(&s_full[s], 1);
+        s_abort = 0; s_last = 0; s_issued = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // warp 1: draw the rows of tile `it` of this block's run and start their copies into stage it % S
+    auto issue = [&](int it) {
+        const int t = t0 + it, stage = it % S, slot = it % (S + 1);
+        const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
+        const int nvalid = min(R, pl.B - j0);
+        if (lane == 0) { mbar_arrive_expect_tx(&s_full[stage], (uint32_t)(nvalid * row_bytes)); s_issued = it + 1; }
+        __syncwarp();
+        if (lane < R) {
+            if (lane < nvalid) {
+                const int64_t a = batch_row(bs, K, w, j0 + lane, pl.B, true);
+                // label and snapshot margin travel beside the row (4-byte asynchronous copies: nobody waits for them here)
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(smem_u32(&s_lab[slot][lane])), "l"(labels + a) : "memory");
+                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(smem_u32(&s_zs[slot][lane])), "l"(z_snap + a) : "memory");
+                bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
+            }
+        }
+    };
+    if (load_warp) {
+        for (int it = 0; it < min(S, ntl); ++it) issue(it);
+        asm volatile("cp.async.wait_all;" ::: "memory");     // labels and margins of the first tiles (the rows stay in flight)
+    }
+
+    float acc[N], dreg[N];
+#pragma unroll
+    for (int n = 0; n < N; ++n) { acc[n] = 0.0f; dreg[n] = 0.0f; }
+    uint4 q_old[R], q_new[R];
+#pragma unroll
+    for (int r = 0; r < R; ++r) q_old[r] = make_uint4(0u, 0u, 0u, 0u);
+    int w_prev = -1, nvalid_prev = 0;
+
+    int it = 0;
+    for (; it <= ntl; ++it) {
+        const int t = t0 + it, par = it & 1, stage = it % S;
+        const int w_cur = it < ntl ? pl.worker_of(t) : -1;
+        const int j0 = it < ntl ? (t - w_cur * pl.tiles_per_worker) * R : 0;
+        const int nvalid = it < ntl ? min(R, pl.B - j0) : 0;
+        // ---- front: margins of tile it ----------------------------------------------------------------------------
+        if (it < ntl) {
+            if (w_cur != w_prev && active) {                 // this worker's xhat - xsnap (a lagging worker reads an older one)
+                const float4* dv = reinterpret_cast<const float4*>(diff_of_worker(bs, diff, w_cur)) + (size_t)v * (N / 4);
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) { const float4 x4 = __ldg(dv + q); dreg[q * 4] = x4.x; dreg[q * 4 + 1] = x4.y; dreg[q * 4 + 2] = x4.z; dreg[q * 4 + 3] = x4.w; }
+            }
+            if (!mbar_wait_bounded(&s_full[stage], (uint32_t)((it / S) & 1))) { s_abort = 1; set_status(status, DQ_ERR_TIMEOUT); }
+            float p[R];
+            const unsigned char* base = s_stage + (size_t)stage * R * stride + (size_t)v * 16;
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                q_new[r] = (active && r < nvalid) ? *reinterpret_cast<const uint4*>(base + (size_t)r * stride) : make_uint4(0u, 0u, 0u, 0u);
+                float f[N];
+                RowVec<T>::unpack(q_new[r], f);
+                float s = 0.0f;
+#pragma unroll
+                for (int n = 0; n < N; ++n) s = fmaf(f[n], dreg[n], s);
+                p[r] = s;
+            }
+            const float folded = fold8(p, lane);
+            if ((lane & 3) == 0) s_part[par][warp][((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = folded;
+        }
+        __syncthreads();                                     // A(it): the stage has been read, the partial margins are visible
+        if (s_abort) break;
+        // ---- warp 1: the copies of tile it + S into the stage that was just read; warp 0: slopes of tile it ---------
+        if (load_warp && it < ntl) {
+            asm volatile("cp.async.wait_all;" ::: "memory");     // labels and margins of the tiles issued so far: tile it + 1's are
+            if (it + S < ntl) issue(it + S);                     // visible to warp 0 after the next barrier
+        }
+        if (slope_warp && it < ntl) {
+            if (lane < R) {
+                float rj = 0.0f;
+                if (lane < nvalid) {
+                    double dz = 0.0;
+#pragma unroll
+                    for (int k = 0; k < kFusedWarps; ++k) dz += (double)s_part[par][k][lane];
+                    rj = slope_difference(s_lab[it % (S + 1)][lane], s_zs[it % (S + 1)][lane], (float)dz) / (float)pl.B;
+                }
+                s_r[par][lane] = rj;
+            }
+            __syncwarp();
+        }
+        // ---- back: add the rows of tile it - 1 to the columns ------------------------------------------------------
+        if (it > 0) {
+#pragma unroll
+            for (int r = 0; r < R; ++r) {
+                if (r < nvalid_prev) {
+                    const float rr = s_r[par ^ 1][r];
+                    float f[N];
+                    RowVec<T>::unpack(q_old[r], f);
+#pragma unroll
+                    for (int n = 0; n < N; ++n) acc[n] = fmaf(rr, f[n], acc[n]);
+                }
+            }
+        }
+        // ---- a worker's last tile in this block has been added: hand its column sums over ---------------------------
+        if (it > 0 && w_cur != w_prev) {
+            const int w = w_prev;
+            if (active) {
+                float4* dst = reinterpret_cast<float4*>(part + (size_t)(blk + w) * d) + (size_t)v * (N / 4);
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) dst[q] = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
+            }
+#pragma unroll
+            for (int n = 0; n < N; ++n) acc[n] = 0.0f;
+            __threadfence();
+            __syncthreads();
+            const int b_first = pl.block_of_tile(w * pl.tiles_per_worker), b_last = pl.block_of_tile((w + 1) * pl.tiles_per_worker - 1);
+            if (tid == 0) {
+                const uint32_t old = atomicAdd(counters + w, 1u);
+                s_last = old == (uint32_t)(b_last - b_first);
+                if (s_last) counters[w] = 0u;                // every block of this worker has added: ready for the next launch
+            }
+            __syncthreads();
+            if (s_last) {                                    // this block completes worker w: slots in block order
+                __threadfence();
+                uint32_t nmax = 0;
+                if (active) {
+                    float sum[N];
+#pragma unroll
+                    for (int n = 0; n < N; ++n) sum[n] = 0.0f;
+                    for (int bb = b_first; bb <= b_last; ++bb) {
+                        const float4* src = reinterpret_cast<const float4*>(part + (size_t)(bb + w) * d) + (size_t)v * (N / 4);
+#pragma unroll
+                        for (int q = 0; q < N / 4; ++q) {
+                            const float4 x4 = __ldcg(src + q);
+                            sum[q * 4] += x4.x; sum[q * 4 + 1] += x4.y; sum[q * 4 + 2] += x4.z; sum[q * 4 + 3] += x4.w;
+                        }
+                    }
+                    float4* out = reinterpret_cast<float4*>(alpha + (size_t)w * d) + (size_t)v * (N / 4);
+#pragma unroll
+                    for (int q = 0; q < N / 4; ++q) out[q] = make_float4(sum[q * 4], sum[q * 4 + 1], sum[q * 4 + 2], sum[q * 4 + 3]);
+#pragma unroll
+                    for (int n = 0; n < N; ++n) nmax = max(nmax, __float_as_uint(sum[n]) & 0x7FFFFFFFu);
+                }
+                nmax = warp_max_u32(nmax);
+                if (lane == 0) s_max[warp] = nmax;
+                __syncthreads();
+                if (tid == 0) {
+                    uint32_t m = 0;
+                    for (int k = 0; k < kFusedWarps; ++k) m = max(m, s_max[k]);
+                    norm_bits[w] = m;
+                }
+                __syncthreads();
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < R; ++r) q_old[r] = q_new[r];
+        w_prev = w_cur; nvalid_prev = nvalid;
+    }
+    if (s_abort && tid == 0) {
+        // a copy did not arrive in time: give the copies still in flight a bounded time to land before the block's
+        // shared memory is released
+        for (int k = it; k < s_issued; ++k) (void)mbar_wait_bounded(&s_full[k % S], (uint32_t)((k / S) & 1));
+    }
 }
 
 // ---------------------------------------------------------------------------------------------------
@@ -514,19 +838,6 @@ objective_reg_kernel(const float* __restrict__ x, int64_t d, float l1, float l2,
     block_add_double(acc, P);
 }
 
-// Transmitted bits of one round by the paper's message sizes (Section 3.1; remark after Theorem 3).
-__global__ void bits_kernel(int M, int64_t d, int bx, int b, int flag_round, int sparse_msgs, const uint32_t* __restrict__ nnz,
-                            uint64_t* __restrict__ bits_down, uint64_t* __restrict__ bits_up)
-{
-    pdl_prologue();
-    if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    *bits_down = flag_round ? (uint64_t)M : (uint64_t)M * (32ull + (uint64_t)bx * (uint64_t)d);
-    uint64_t up = 0;
-    int logd = 0; while (((int64_t)1 << logd) < d) ++logd;
-    for (int w = 0; w < M; ++w) up += sparse_msgs ? 32ull + (uint64_t)nnz[w] * (uint64_t)(logd + b) : 32ull + (uint64_t)b * (uint64_t)d;
-    *bits_up = up;
-}
-
 // ---------------------------------------------------------------------------------------------------
 // Second smooth part (Section 5.2): 3-layer fully connected network, in -> hidden (ReLU) -> classes, softmax
 // cross-entropy.  Parameters x = [W1 (hidden x in, row-major), b1, W2 (classes x hidden), b2]; labels hold class
@@ -534,7 +845,11 @@ __global__ void bits_kernel(int M, int64_t d, int bx, int b, int flag_round, int
 // vectors side by side (either may be absent: NULL), rows listed explicitly or drawn from the batch stream.
 //   mlp_hidden_kernel   block per tile of sampled rows and eight hidden units: hidden activations (one warp per unit, coalesced along in)
 //   mlp_output_kernel   block per sampled row: logits, softmax, d loss / d logits, d loss / d hidden (ReLU-gated)
-//   mlp_param_kernel    block per (hidden unit or the tail, worker): sums over the worker's rows, no atomics
+//   mlp_param_kernel    block per (tile of hidden units or the tail, worker): sums over the worker's rows, no atomics
+// The forward pass (hidden pre-activations, activations, logits, softmax) runs in double precision: a class
+// probability depends on sums of hundreds of products that cancel, and an fp32 sum's error of 2^-24 of the
+// absolute terms passes through the softmax into every coordinate of the gradient, where the attainable accuracy
+// is set by much smaller per-sample terms.  The derivatives leave the forward pass rounded to fp32 once.
 // ---------------------------------------------------------------------------------------------------
 struct MlpShape { int64_t in; int hidden, classes; };
 
@@ -544,15 +859,15 @@ __device__ __forceinline__ int64_t mlp_off_b2(const MlpShape& s) { return mlp_of
 
 constexpr int kMlpUnits = 8;         // hidden units whose first-layer gradients one block forms from the same rows
 constexpr int kMlpTile = 8;          // sampled rows that share one pass over a hidden unit's weights
+constexpr int kMlpRowChunk = 128;    // rows whose slope differences a block of mlp_param_kernel stages at a time
 
 // grid (ceil(nslots / kMlpTile), ceil(hidden / 8)): a block holds kMlpTile rows in shared memory and each of its
 // eight warps owns one hidden unit, so a weight row is read once for the whole tile (a block per row would read the
-// first layer once per sample).  Per row the sum runs in the same order as before: lanes stride over the inputs,
-// then a butterfly across lanes.
+// first layer once per sample).  Lanes stride over the inputs, then a butterfly across lanes.
 __global__ void __launch_bounds__(kThreads)
 mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restrict__ xa, const float* __restrict__ xb,
                   const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
-                  float* __restrict__ act_a, float* __restrict__ act_b, int64_t nslots)
+                  double* __restrict__ act_a, double* __restrict__ act_b, int64_t nslots)
 {
     pdl_prologue();
     extern __shared__ float s_in[];                      // [kMlpTile][in] features of the tile's rows
@@ -577,58 +892,58 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
     __syncthreads();
     const int j = blockIdx.y * (kThreads / 32) + warp;
     if (j >= sh.hidden) return;
-    float sa[kMlpTile], sb[kMlpTile];
+    double sa[kMlpTile], sb[kMlpTile];
 #pragma unroll
-    for (int t = 0; t < kMlpTile; ++t) { sa[t] = 0.0f; sb[t] = 0.0f; }
+    for (int t = 0; t < kMlpTile; ++t) { sa[t] = 0.0; sb[t] = 0.0; }
 #pragma unroll 2
     for (int64_t i = lane; i < sh.in; i += 32) {
-        const float wa = xa ? xa[(int64_t)j * sh.in + i] : 0.0f, wb = xb ? xb[(int64_t)j * sh.in + i] : 0.0f;
+        const double wa = xa ? (double)xa[(int64_t)j * sh.in + i] : 0.0, wb = xb ? (double)xb[(int64_t)j * sh.in + i] : 0.0;
 #pragma unroll
         for (int t = 0; t < kMlpTile; ++t) {
-            const float f = s_in[(int64_t)t * sh.in + i];
-            sa[t] = fmaf(wa, f, sa[t]); sb[t] = fmaf(wb, f, sb[t]);
+            const double f = (double)s_in[(int64_t)t * sh.in + i];
+            sa[t] = fma(wa, f, sa[t]); sb[t] = fma(wb, f, sb[t]);
         }
     }
-    const float ba = xa ? xa[mlp_off_b1(sh) + j] : 0.0f, bb = xb ? xb[mlp_off_b1(sh) + j] : 0.0f;
+    const double ba = xa ? (double)xa[mlp_off_b1(sh) + j] : 0.0, bb = xb ? (double)xb[mlp_off_b1(sh) + j] : 0.0;
 #pragma unroll
     for (int t = 0; t < kMlpTile; ++t) {
-        const float va = warp_sum(sa[t]), vb = warp_sum(sb[t]);
+        const double va = warp_sum(sa[t]), vb = warp_sum(sb[t]);
         if (lane == 0 && slot0 + t < nslots) {
-            if (xa) act_a[(slot0 + t) * sh.hidden + j] = fmaxf(va + ba, 0.0f);
-            if (xb) act_b[(slot0 + t) * sh.hidden + j] = fmaxf(vb + bb, 0.0f);
+            if (xa) act_a[(slot0 + t) * sh.hidden + j] = fmax(va + ba, 0.0);
+            if (xb) act_b[(slot0 + t) * sh.hidden + j] = fmax(vb + bb, 0.0);
         }
     }
 }
 
 // One model of one row: logits -> softmax -> dz = (p - onehot) * wgt, dh_j = relu'(h_j) sum_c dz_c W2[c][j]; returns loss.
-__device__ __forceinline__ void mlp_output_one(const MlpShape& sh, const float* __restrict__ x, const float* __restrict__ act,
-                                               int label, float wgt, float* __restrict__ dz, float* __restrict__ dh,
-                                               float* s_z, double* loss_out)
+__device__ __forceinline__ void mlp_output_one(const MlpShape& sh, const float* __restrict__ x, const double* __restrict__ act,
+                                               int label, double wgt, float* __restrict__ dz, float* __restrict__ dh,
+                                               double* s_z, double* loss_out)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int c = warp; c < sh.classes; c += kThreads / 32) {
-        float s = 0.0f;
-        for (int j = lane; j < sh.hidden; j += 32) s = fmaf(x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], act[j], s);
+        double s = 0.0;
+        for (int j = lane; j < sh.hidden; j += 32) s = fma((double)x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], act[j], s);
         s = warp_sum(s);
-        if (lane == 0) s_z[c] = s + x[mlp_off_b2(sh) + c];
+        if (lane == 0) s_z[c] = s + (double)x[mlp_off_b2(sh) + c];
     }
     __syncthreads();
-    float zmax = -INFINITY, sum = 0.0f, others = 0.0f;      // others: the sum without the label's term, so that
-    for (int c = 0; c < sh.classes; ++c) zmax = fmaxf(zmax, s_z[c]);     // p_label - 1 = -others/sum has no cancellation
-    for (int c = 0; c < sh.classes; ++c) { const float e = expf(s_z[c] - zmax); sum += e; if (c != label) others += e; }
-    if (threadIdx.x == 0 && loss_out) *loss_out = (double)(zmax + logf(sum)) - (double)s_z[label];
+    double zmax = -INFINITY, sum = 0.0, others = 0.0;       // others: the sum without the label's term, so that
+    for (int c = 0; c < sh.classes; ++c) zmax = fmax(zmax, s_z[c]);      // p_label - 1 = -others/sum has no cancellation
+    for (int c = 0; c < sh.classes; ++c) { const double e = exp(s_z[c] - zmax); sum += e; if (c != label) others += e; }
+    if (threadIdx.x == 0 && loss_out) *loss_out = (zmax + log(sum)) - s_z[label];
     __syncthreads();
     for (int c = threadIdx.x; c < sh.classes; c += blockDim.x) {
-        const float v = (c == label ? -others / sum : expf(s_z[c] - zmax) / sum) * wgt;
+        const double v = (c == label ? -others / sum : exp(s_z[c] - zmax) / sum) * wgt;
         s_z[sh.classes + c] = v;
-        if (dz) dz[c] = v;
+        if (dz) dz[c] = (float)v;
     }
     __syncthreads();
     if (dh) {
         for (int j = threadIdx.x; j < sh.hidden; j += blockDim.x) {
-            float s = 0.0f;
-            for (int c = 0; c < sh.classes; ++c) s = fmaf(s_z[sh.classes + c], x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], s);
-            dh[j] = act[j] > 0.0f ? s : 0.0f;
+            double s = 0.0;
+            for (int c = 0; c < sh.classes; ++c) s = fma(s_z[sh.classes + c], (double)x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], s);
+            dh[j] = act[j] > 0.0 ? (float)s : 0.0f;
         }
     }
     __syncthreads();
@@ -636,70 +951,88 @@ __device__ __forceinline__ void mlp_output_one(const MlpShape& sh, const float* 
 
 __global__ void __launch_bounds__(kThreads)
 mlp_output_kernel(MlpShape sh, const float* __restrict__ labels, const int32_t* __restrict__ row_of_slot,
-                  const float* __restrict__ xa, const float* __restrict__ xb, const float* __restrict__ act_a,
-                  const float* __restrict__ act_b, float wgt, float* __restrict__ dz_a, float* __restrict__ dz_b,
+                  const float* __restrict__ xa, const float* __restrict__ xb, const double* __restrict__ act_a,
+                  const double* __restrict__ act_b, double wgt, float* __restrict__ dz_a, float* __restrict__ dz_b,
                   float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b)
 {
     pdl_prologue();
-    extern __shared__ float s_z[];                       // [2 * classes]
+    extern __shared__ double s_zd[];                     // [2 * classes]
     const int64_t slot = blockIdx.x;
     const int label = (int)labels[row_of_slot[slot]];
-    if (xa) mlp_output_one(sh, xa, act_a + slot * sh.hidden, label, wgt, dz_a + slot * sh.classes, dh_a + slot * sh.hidden, s_z, nullptr);
+    if (xa) mlp_output_one(sh, xa, act_a + slot * sh.hidden, label, wgt, dz_a + slot * sh.classes, dh_a + slot * sh.hidden, s_zd, nullptr);
     if (xb) {
         double loss = 0.0;
         mlp_output_one(sh, xb, act_b + slot * sh.hidden, label, wgt, dz_b ? dz_b + slot * sh.classes : nullptr,
-                       dh_b ? dh_b + slot * sh.hidden : nullptr, s_z, loss_b ? &loss : nullptr);
-        if (loss_b && threadIdx.x == 0) atomicAdd(loss_b, loss * (double)wgt);
+                       dh_b ? dh_b + slot * sh.hidden : nullptr, s_zd, loss_b ? &loss : nullptr);
+        if (loss_b && threadIdx.x == 0) atomicAdd(loss_b, loss * wgt);
     }
 }
 
-// grid (hidden + 1, groups): block (j, w) sums over the rows [w*B, (w+1)*B) of its group.  j < hidden: row j of W1 and
-// b1[j]; j == hidden: W2 and b2.  Output = model a minus model b (either may be absent).  FULL: double sums added to
-// g64 with atomics (epoch gradient over many groups); otherwise stored to out [groups][P] with the norm folded in.
+// grid (ceil(hidden / kMlpUnits) + 1, groups): block (j, w) sums over the rows [w*B, (w+1)*B) of its group, in slot
+// order and in double.  Blocks before the last: rows j0 .. j0 + kMlpUnits - 1 of W1 and their b1; last block: W2 and b2.
+// Output = model a minus model b (either may be absent).  FULL: sums added to g64 with atomics (epoch gradient over
+// many groups); otherwise rounded once and stored to out [groups][P] with the norm folded in.
 template <bool FULL>
 __global__ void __launch_bounds__(kThreads)
 mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __restrict__ row_of_slot, int B, int64_t total_rows,
-                 const float* __restrict__ act_a, const float* __restrict__ act_b, const float* __restrict__ dz_a,
+                 const double* __restrict__ act_a, const double* __restrict__ act_b, const float* __restrict__ dz_a,
                  const float* __restrict__ dz_b, const float* __restrict__ dh_a, const float* __restrict__ dh_b,
                  float* __restrict__ out, int64_t P, uint32_t* __restrict__ norm_bits, double* __restrict__ g64)
 {
     pdl_prologue();
-    typedef typename std::conditional<FULL, double, float>::type acc_t;
-    extern __shared__ float s_w[];                       // [kMlpUnits][B] slope differences, then [B] row indices
+    __shared__ double s_w[kMlpUnits][kMlpRowChunk];      // slope differences of a chunk of rows
+    __shared__ int s_rowid[kMlpRowChunk];
     const int j0 = blockIdx.x * kMlpUnits, w = blockIdx.y;     // the block after the last tile of hidden units does W2, b2
     const int64_t r0 = (int64_t)w * B;
     const int nrows = (int)min((int64_t)B, total_rows - r0);
     uint32_t nmax = 0;
     float* o = FULL ? nullptr : out + (int64_t)w * P;
     if (j0 < sh.hidden) {
-        // s_w[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u]; the rows' indices sit behind them: no dependent load in the loop.
-        // The block's hidden units share every feature value that a thread loads.
-        int* s_rowid = reinterpret_cast<int*>(s_w + kMlpUnits * B);
-        for (int q = threadIdx.x; q < kMlpUnits * nrows; q += blockDim.x) {
-            const int u = q / nrows, r = q - u * nrows, j = j0 + u;
-            const float da = (dh_a && j < sh.hidden) ? dh_a[(r0 + r) * sh.hidden + j] : 0.0f;
-            const float db = (dh_b && j < sh.hidden) ? dh_b[(r0 + r) * sh.hidden + j] : 0.0f;
-            s_w[u * B + r] = da - db;
-        }
-        for (int r = threadIdx.x; r < nrows; r += blockDim.x) s_rowid[r] = row_of_slot[r0 + r];
-        __syncthreads();
-        for (int64_t i = threadIdx.x; i <= sh.in; i += blockDim.x) {       // i == in: the bias b1[j]
-            acc_t s[kMlpUnits];
+        // s_w[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u]; the rows' indices sit beside them: no dependent load in the loop.
+        // The block's hidden units share every feature value that a thread loads.  A thread owns the inputs
+        // i = threadIdx.x + k * blockDim.x (i == in: the bias b1[j]) and keeps their sums across the chunks of rows.
+        constexpr int kOwn = 4;                                             // inputs per thread and pass
+        for (int64_t ibase = 0; ibase <= sh.in; ibase += (int64_t)kOwn * blockDim.x) {
+            double s[kOwn][kMlpUnits];
 #pragma unroll
-            for (int u = 0; u < kMlpUnits; ++u) s[u] = 0;
-#pragma unroll 4
-            for (int r = 0; r < nrows; ++r) {
-                const float f = (i < sh.in) ? X[(int64_t)s_rowid[r] * sh.in + i] : 1.0f;
+            for (int k = 0; k < kOwn; ++k)
 #pragma unroll
-                for (int u = 0; u < kMlpUnits; ++u) s[u] += (acc_t)(s_w[u * B + r] * f);
+                for (int u = 0; u < kMlpUnits; ++u) s[k][u] = 0.0;
+            for (int c0 = 0; c0 < nrows; c0 += kMlpRowChunk) {
+                const int cn = min(kMlpRowChunk, nrows - c0);
+                __syncthreads();
+                for (int q = threadIdx.x; q < kMlpUnits * cn; q += blockDim.x) {
+                    const int u = q / cn, r = q - u * cn, j = j0 + u;
+                    const float da = (dh_a && j < sh.hidden) ? dh_a[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
+                    const float db = (dh_b && j < sh.hidden) ? dh_b[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
+                    s_w[u][r] = (double)da - (double)db;
+                }
+                for (int r = threadIdx.x; r < cn; r += blockDim.x) s_rowid[r] = row_of_slot[r0 + c0 + r];
+                __syncthreads();
+#pragma unroll
+                for (int k = 0; k < kOwn; ++k) {
+                    const int64_t i = ibase + threadIdx.x + (int64_t)k * blockDim.x;
+                    if (i > sh.in) continue;
+#pragma unroll 2
+                    for (int r = 0; r < cn; ++r) {
+                        const double f = (i < sh.in) ? (double)X[(int64_t)s_rowid[r] * sh.in + i] : 1.0;
+#pragma unroll
+                        for (int u = 0; u < kMlpUnits; ++u) s[k][u] = fma(s_w[u][r], f, s[k][u]);
+                    }
+                }
             }
 #pragma unroll
-            for (int u = 0; u < kMlpUnits; ++u) {
-                const int j = j0 + u;
-                if (j >= sh.hidden) break;
-                const int64_t pidx = (i < sh.in) ? (int64_t)j * sh.in + i : mlp_off_b1(sh) + j;
-                if (FULL) atomicAdd(g64 + pidx, (double)s[u]);
-                else { o[pidx] = (float)s[u]; nmax = max(nmax, __float_as_uint((float)s[u]) & 0x7FFFFFFFu); }
+            for (int k = 0; k < kOwn; ++k) {
+                const int64_t i = ibase + threadIdx.x + (int64_t)k * blockDim.x;
+                if (i > sh.in) continue;
+#pragma unroll
+                for (int u = 0; u < kMlpUnits; ++u) {
+                    const int j = j0 + u;
+                    if (j >= sh.hidden) break;
+                    const int64_t pidx = (i < sh.in) ? (int64_t)j * sh.in + i : mlp_off_b1(sh) + j;
+                    if (FULL) atomicAdd(g64 + pidx, s[k][u]);
+                    else { o[pidx] = (float)s[k][u]; nmax = max(nmax, __float_as_uint((float)s[k][u]) & 0x7FFFFFFFu); }
+                }
             }
         }
     } else {
@@ -707,15 +1040,15 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
         for (int t = threadIdx.x; t < nout; t += blockDim.x) {
             const bool bias = t >= sh.classes * sh.hidden;
             const int c = bias ? t - sh.classes * sh.hidden : t / sh.hidden, jj = bias ? 0 : t % sh.hidden;
-            acc_t s = 0;
+            double s = 0.0;
             for (int r = 0; r < nrows; ++r) {
                 const int64_t q = r0 + r;
-                const float ta = dz_a ? dz_a[q * sh.classes + c] * (bias ? 1.0f : act_a[q * sh.hidden + jj]) : 0.0f;
-                const float tb = dz_b ? dz_b[q * sh.classes + c] * (bias ? 1.0f : act_b[q * sh.hidden + jj]) : 0.0f;
-                s += (acc_t)(ta - tb);
+                const double ta = dz_a ? (double)dz_a[q * sh.classes + c] * (bias ? 1.0 : act_a[q * sh.hidden + jj]) : 0.0;
+                const double tb = dz_b ? (double)dz_b[q * sh.classes + c] * (bias ? 1.0 : act_b[q * sh.hidden + jj]) : 0.0;
+                s += ta - tb;
             }
             const int64_t pidx = bias ? mlp_off_b2(sh) + c : mlp_off_w2(sh) + (int64_t)c * sh.hidden + jj;
-            if (FULL) atomicAdd(g64 + pidx, (double)s);
+            if (FULL) atomicAdd(g64 + pidx, s);
             else { o[pidx] = (float)s; nmax = max(nmax, __float_as_uint((float)s) & 0x7FFFFFFFu); }
         }
     }
@@ -745,6 +1078,7 @@ struct SmallRound {
     uint8_t* codes; int64_t stride; float* scale; uint64_t* bits_down; uint64_t* bits_up; int* status;
     // what to run
     uint32_t round0; int nrounds; float eta, theta;
+    double acc_scale, acc_inv;      // CSR data: the integer grid of the gradient accumulator (see worker_grad_csr_kernel)
 };
 
 constexpr int kSmallThreads = 1024;
@@ -816,6 +1150,10 @@ __device__ __forceinline__ void small_quantize(const float* v, int64_t d, uint32
         philox4x32_10((uint32_t)g, round, worker, stream, K, r);
 #pragma unroll
         for (int j = 0; j < 8; ++j) s[j] = round_fixed<BITS>(a[j], inv, half16(r, j));
+        if (nb >= 0x7F800000u) {                               // NaN or Inf in the vector: every code is 0
+#pragma unroll
+            for (int j = 0; j < 8; ++j) s[j] = 128u << 16;
+        }
         if (out) store_group<BITS>(out + g * BITS, pack8<BITS>(s));
         if (diff) {                                            // diff is a padded shared vector
             float rf[8], o[8];
@@ -848,6 +1186,7 @@ round_cluster_kernel(const __grid_constant__ SmallRound P, const __grid_constant
     const int64_t dpad = small_round_pad(d);                  // room for the zero padding of a packed message
     float* s_diff = s_mem;                                    // [dpad] xhat - xsnap
     float* s_alpha = s_mem + dpad;                            // [dpad] this worker's gradient difference, zeros past d
+    long long* s_acc = reinterpret_cast<long long*>(s_mem + 2 * dpad);   // [d] CSR data: exact integer accumulator (dpad is even: 8-byte aligned)
     const int w = blockIdx.x, lane = threadIdx.x & 31;
     const int64_t gtid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, gnth = (int64_t)gridDim.x * blockDim.x;
     for (int it = 0; it < P.nrounds; ++it) {
@@ -858,7 +1197,8 @@ round_cluster_kernel(const __grid_constant__ SmallRound P, const __grid_constant
         if (gtid == 0) P.xnorm2[it & 1] = 0u;                 // read last in the previous round, two barriers ago
         DQ_DISPATCH_BITS(P.bx, (small_quantize<BITS_, false>(P.x, d, nbx, w == 0 ? P.codes_x : nullptr, w == 0 ? P.delta_x : nullptr, K,
                                                               round, kMaster, kStreamModel, P.status, P.xsnap, s_diff)));
-        for (int64_t i = (FMT == DQ_CSR_F32 ? 0 : d) + threadIdx.x; i < dpad; i += blockDim.x) s_alpha[i] = 0.0f;
+        for (int64_t i = d + threadIdx.x; i < dpad; i += blockDim.x) s_alpha[i] = 0.0f;
+        if (FMT == DQ_CSR_F32) for (int64_t i = threadIdx.x; i < d; i += blockDim.x) s_acc[i] = 0;
         __syncthreads();
         // ---- worker w: slope differences of its sampled rows ------------------------------------------------------
         if (FMT == DQ_CSR_F32) {
@@ -876,8 +1216,10 @@ round_cluster_kernel(const __grid_constant__ SmallRound P, const __grid_constant
 #pragma unroll
                 for (int o = 8; o > 0; o >>= 1) sdot += __shfl_xor_sync(submask, sdot, o);
                 const float r = slope_difference(ya, za, (float)sdot) / (float)B;
-                for (int64_t k = k0 + l16; k < k1; k += 16) atomicAdd(s_alpha + __ldg(P.col + k), r * __ldg(P.values + k));
+                for (int64_t k = k0 + l16; k < k1; k += 16) fixed_add(s_acc + __ldg(P.col + k), r, __ldg(P.values + k), P.acc_scale);
             }
+            __syncthreads();
+            for (int64_t i = threadIdx.x; i < d; i += blockDim.x) s_alpha[i] = (float)((double)s_acc[i] * P.acc_inv);
             __syncthreads();
         } else {
             const bool vec = (d & 3) == 0;
@@ -1028,11 +1370,11 @@ static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStre
     const int64_t P = ctx->cfg.d;
     launch_k(mlp_hidden_kernel, mlp_hidden_grid(D.n, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
                                                                              ctx->mlp_rows, ctx->mlp_act[0], nullptr, (int64_t)D.n);
-    launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
-        nullptr, (float)(1.0 / (double)D.n), ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr);
+    launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(double) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
+        nullptr, 1.0 / (double)D.n, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr);
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * P, st);
     dim3 grid((sh.hidden + kMlpUnits - 1) / kMlpUnits + 1, (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
-    launch_k(mlp_param_kernel<true>, grid, kThreads, sizeof(float) * (kMlpUnits + 1) * kMlpGroup, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
+    launch_k(mlp_param_kernel<true>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
         ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
     launch_k(finish_full_grad_kernel, blocks_for(P, ctx->sm_count), kThreads, 0, st, ctx->g64, P, 1.0, g);
     ctx->launches += 4;
@@ -1047,11 +1389,11 @@ static void launch_mlp_worker_grad(dq_ctx* ctx, const float* xhat, const dq_stat
     uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
     launch_k(mlp_hidden_kernel, mlp_hidden_grid(R, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
                                                                    ctx->mlp_act[0], ctx->mlp_act[1], (int64_t)R);
-    launch_k(mlp_output_kernel, R, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
-        ctx->mlp_act[1], 1.0f / (float)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr);
+    launch_k(mlp_output_kernel, R, kThreads, sizeof(double) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
+        ctx->mlp_act[1], 1.0 / (double)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr);
     if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
     dim3 grid((sh.hidden + kMlpUnits - 1) / kMlpUnits + 1, c.M);
-    launch_k(mlp_param_kernel<false>, grid, kThreads, sizeof(float) * (kMlpUnits + 1) * c.B, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
+    launch_k(mlp_param_kernel<false>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
         ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
     ctx->launches += 3;
 }
@@ -1085,15 +1427,44 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
     ctx->launches += 3;
 }
 
+// The one-pass kernel takes dense rows of at most kFusedMaxRowBytes on the 16-byte grid; the context then owns its
+// scratch (column sums per (block, worker), per-worker counters).
+static size_t fused_grad_smem(const dq_ctx* ctx)
+{
+    const size_t row_bytes = (size_t)ctx->cfg.d * (ctx->data.format == DQ_DENSE_F32 ? 4 : 2);
+    return (size_t)kFusedStages * kFusedRows * (row_bytes + kFusedRowPad);
+}
+bool fused_grad_applies(const dq_ctx* ctx) { return ctx->fused_part != nullptr && !ctx->cfg.no_fused; }
+
+// Called once per context: scratch and the shared-memory opt-in of the one-pass dense gradient kernel.
+int fused_grad_setup(dq_ctx* ctx)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    if (!ctx->has_data || c.model != DQ_MODEL_LOGISTIC || (D.format != DQ_DENSE_F32 && D.format != DQ_DENSE_BF16)) return DQ_OK;
+    const size_t row_bytes = (size_t)c.d * (D.format == DQ_DENSE_F32 ? 4 : 2);
+    if (row_bytes > kFusedMaxRowBytes || (row_bytes & 15) || c.B < 64) return DQ_OK;
+    const int smem = (int)fused_grad_smem(ctx);
+    const cudaError_t e = D.format == DQ_DENSE_F32
+        ? cudaFuncSetAttribute(worker_grad_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+        : cudaFuncSetAttribute(worker_grad_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) { cudaGetLastError(); return DQ_OK; }          // the two-kernel path remains
+    int resident = 0;                                                    // a block must fit an SM (registers, shared memory)
+    const cudaError_t o = D.format == DQ_DENSE_F32
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, worker_grad_fused_kernel<float>, kFusedThreads, (size_t)smem)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, worker_grad_fused_kernel<__nv_bfloat16>, kFusedThreads, (size_t)smem);
+    if (o != cudaSuccess || resident < 1) { cudaGetLastError(); return DQ_OK; }
+    if (cudaMalloc(reinterpret_cast<void**>(&ctx->fused_part), sizeof(float) * (size_t)(ctx->sm_count + c.M) * c.d) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&ctx->fused_cnt), sizeof(uint32_t) * c.M) != cudaSuccess ||
+        cudaMemset(ctx->fused_cnt, 0, sizeof(uint32_t) * c.M) != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
 // Whether the worker stage accumulates into alpha with atomics (and so needs it cleared first).
 bool worker_accumulates(const dq_ctx* ctx)
 {
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
-    if (c.model == DQ_MODEL_MLP) return false;
-    if (D.format == DQ_CSR_F32) return !ctx->list_mode;
-    const bool vec = (c.d % (D.format == DQ_DENSE_F32 ? 4 : 8)) == 0;
-    if (vec && c.B >= 64) return false;                        // column sums are stored, not added
-    return (c.B + kRowsPerBlock - 1) / kRowsPerBlock > 1;
+    (void)c; (void)D;
+    return false;      // every gradient kernel stores alpha: CSR rows meet in an integer accumulator that is kept all-zero between rounds
 }
 
 void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, int is_snapshot, const dq_state* s,
@@ -1122,15 +1493,37 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         return;
     }
     if (D.format == DQ_CSR_F32) {
-        if (!ctx->alpha_zeroed && !list) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
-        launch_k(worker_grad_csr_kernel, (int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st, (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, alpha,
+        const FixedAcc fa = {ctx->acc64, ctx->acc_scale, ctx->acc_inv};
+        launch_k(worker_grad_csr_kernel, (int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st, (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, fa,
             list ? ctx->touched : nullptr, ctx->bm_words);
+        ctx->launches += 1;
+        if (list) { launch_build_group_list(ctx, reinterpret_cast<uint32_t*>(norm_inf), st); ctx->list_ready = true; return; }
+        uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
+        if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
+        dim3 gc((unsigned)blocks_for(c.d, ctx->sm_count, 2), c.M);
+        launch_k(acc_to_alpha_kernel, gc, kThreads, 0, st, fa, c.d, alpha, nb);
+        ctx->launches += 1;
+        return;
     } else {
-        dim3 grid((c.B + kRowsPerBlock - 1) / kRowsPerBlock, c.M);
+        dim3 grid(1, c.M);
         const bool f32 = D.format == DQ_DENSE_F32;
         const bool vec = (c.d % (f32 ? 4 : 8)) == 0 && (reinterpret_cast<uintptr_t>(alpha) & 15) == 0;   // data is 16-byte aligned by contract
-        if (grid.x > 1 && !ctx->alpha_zeroed && !(vec && c.B >= 64)) cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
-        if (vec && c.B >= 64) {        // large minibatch: margins, then atomics-free column sums with the norm folded in
+        if (vec && c.B >= 64 && fused_grad_applies(ctx)) {      // large minibatch, rows that fit a stage: one pass over the rows
+            FusedPlan pl;
+            pl.M = c.M; pl.B = c.B; pl.tiles_per_worker = (c.B + kFusedRows - 1) / kFusedRows;
+            pl.ntiles = c.M * pl.tiles_per_worker; pl.nblocks = pl.ntiles < ctx->sm_count ? pl.ntiles : ctx->sm_count;
+            const size_t smem = fused_grad_smem(ctx);
+            uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
+            if (f32)
+                launch_k(worker_grad_fused_kernel<float>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
+                         s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status);
+            else
+                launch_k(worker_grad_fused_kernel<__nv_bfloat16>, pl.nblocks, kFusedThreads, smem, st, (const __nv_bfloat16*)D.values, D.labels,
+                         ctx->xhat_diff, s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status);
+            ctx->launches += 1;
+            return;
+        }
+        if (vec && c.B >= 64) {        // large minibatch, long rows: margins, then atomics-free column sums with the norm folded in
             const int32_t* rows_eff = batch_idx ? batch_idx : ctx->rows;
             uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
             if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
@@ -1160,8 +1553,7 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
             launch_k(worker_grad_dense_kernel<__nv_bfloat16>, grid, kThreads, 0, st, (const __nv_bfloat16*)D.values, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.B, c.d, alpha);
     }
     ctx->launches += 1;
-    if (list) { launch_build_group_list(ctx, reinterpret_cast<uint32_t*>(norm_inf), st); ctx->list_ready = true; }
-    else launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
+    launch_norm_inf(ctx, alpha, c.d, c.M, reinterpret_cast<uint32_t*>(norm_inf), st);
 }
 
 // ---- whole rounds in one cluster kernel ---------------------------------------------------------------------
@@ -1185,7 +1577,11 @@ static void small_round_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* att
     cfg->attrs = attr; cfg->numAttrs = 2;
 }
 
-static size_t small_round_smem(const dq_ctx* ctx) { return sizeof(float) * 2 * (size_t)small_round_pad(ctx->cfg.d); }
+static size_t small_round_smem(const dq_ctx* ctx)
+{
+    const size_t acc = ctx->data.format == DQ_CSR_F32 ? sizeof(long long) * (size_t)ctx->cfg.d : 0;
+    return sizeof(float) * 2 * (size_t)small_round_pad(ctx->cfg.d) + acc;
+}
 
 // Decides once per context whether its rounds can run in the cluster kernel: logistic model on dense fp32 or CSR
 // data, dense messages, synchronous master, fixed model width, one block per worker (M <= 16, the largest
@@ -1226,6 +1622,7 @@ void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds
     P.bits_up = bits_up ? bits_up : ctx->bits + 1;
     P.status = ctx->status;
     P.round0 = round0; P.nrounds = nrounds; P.eta = eta; P.theta = theta;
+    P.acc_scale = ctx->acc_scale; P.acc_inv = ctx->acc_inv;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute attr[2];
     small_round_config(&cfg, attr, ctx->cluster_blocks, small_round_smem(ctx), st);
     cudaLaunchKernelEx(&cfg, small_round_kernel_for(ctx), P, ctx->keys);
@@ -1241,8 +1638,8 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
         const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
         launch_k(mlp_hidden_kernel, mlp_hidden_grid(D.n, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
                                                                                  ctx->mlp_rows, nullptr, ctx->mlp_act[1], (int64_t)D.n);
-        launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(float) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
-            ctx->mlp_act[1], (float)(1.0 / (double)D.n), nullptr, nullptr, nullptr, nullptr, P);
+        launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(double) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
+            ctx->mlp_act[1], 1.0 / (double)D.n, nullptr, nullptr, nullptr, nullptr, P);
         launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
         ctx->launches += 3;
         return;
@@ -1278,14 +1675,6 @@ __global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float e
 void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st)
 {
     launch_k(set_round_params_kernel, 1, 1, 0, st, ctx->rp_dev, round, eta, theta);
-    ctx->launches += 1;
-}
-
-void launch_bits(dq_ctx* ctx, int flag_round, bool sparse_msgs, const uint32_t* nnz, uint64_t* bits_down, uint64_t* bits_up,
-                 cudaStream_t st)
-{
-    const dq_config& c = ctx->cfg;
-    launch_k(bits_kernel, 1, 32, 0, st, c.M, c.d, c.bx, c.b, flag_round, sparse_msgs ? 1 : 0, nnz, bits_down, bits_up);
     ctx->launches += 1;
 }
 

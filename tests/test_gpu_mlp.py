@@ -111,3 +111,63 @@ def test_network_free_running_loss(dq):
             first = first if first is not None else Po; last = Po
     assert last < first and dq.dq_poll_status(ctx) == (0, 0)
     dq.dq_destroy(ctx)
+
+
+def _draw_network_case(g):
+    """One random network configuration: any layer sizes up to the paper's 784-100-10 and beyond, any minibatch from one
+    row, every model width, every regulariser, with and without sparsification, momentum and the one-by-one master."""
+    n_in = int(g.integers(3, 785)); hidden = int(g.integers(1, 301)); classes = int(g.integers(2, 18))
+    if g.random() < 0.15:
+        n_in, hidden, classes = 784, 100, 10                                   # the shape of Section 5.2
+    n = int(g.integers(60, 400))
+    h, x = _net(n, n_in, hidden, classes, int(g.integers(1, 1000)))
+    M = int(g.choice([1, 2, 4, 8, 17])); B = min(int(g.choice([1, 2, 3, 20, 64, 100, 150])), n)
+    kw = dict(M=M, B=B, bx=int(g.integers(2, 12)), b=int(g.choice([2, 4, 8])), seed=int(g.integers(1, 1 << 30)), model=1,
+              hidden=hidden, classes=classes)
+    r = g.random()
+    if r < 0.4:
+        kw["lambda2"] = 1e-4
+    elif r < 0.6:
+        kw["lambda1"] = 1e-5
+    else:
+        kw.update(box_lo=-2.0, box_hi=2.0)
+    if g.random() < 0.3:
+        kw.update(sparsify=1, phi=float(g.choice([0.0, 20.0])), msg_format=int(g.integers(0, 2)))
+    if g.random() < 0.3:
+        kw["accelerated"] = 1
+    if g.random() < 0.2:
+        kw["sequential"] = 1
+    if g.random() < 0.2:
+        kw["no_fused"] = 1
+    if g.random() < 0.15:
+        kw["no_graph"] = 1
+    if g.random() < 0.15:
+        kw["mu"] = float(g.choice([0.3, 30.0]))
+    return h, x, kw
+
+
+def test_network_random_shapes(dq):
+    """200 seeded random network shapes (3..784 inputs, 1..300 hidden units, 2..17 classes, minibatches from one row)
+    through two epochs of lockstep rounds: every coordinate of every worker's gradient difference within
+    1e-5 max(|oracle|, S_i, 1e-3 ||oracle||_inf), the epoch gradient within 2e-5, codes bit-exact on the GPU's own
+    gradient, no flip outside the threshold band.  A failure names its trial, which reproduces alone."""
+    worst = 0.0
+    for trial in range(200):
+        g = np.random.default_rng([1807, trial])
+        h, x, kw = _draw_network_case(g)
+        acc = bool(kw.get("accelerated", 0))
+        try:
+            ls = Lockstep(dq, h, x, **kw)
+            rnd = 0
+            for ep in range(2):
+                theta = F32(2.0 / (ep + 3)) if acc else F32(0.0)
+                ls.epoch(theta)
+                for t in range(4):
+                    ls.round(rnd, (0.02 / float(theta)) if acc else 0.1, theta)
+                    rnd += 1
+            assert ls.far_flips == 0, ("far flips", ls.far_flips)
+            worst = max(worst, ls.worst_alpha)
+            ls.close()
+        except AssertionError as e:
+            raise AssertionError("trial %d n=%d n_in=%d %r: %r" % (trial, h.n, h.d, kw, e)) from e
+    print("\n[nn random shapes] worst gradient error %.2e of the tolerance scale (bound 1e-5)" % worst)

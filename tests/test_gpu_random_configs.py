@@ -85,9 +85,9 @@ def test_random_configurations(dq, block):
 
 def test_random_configurations_every_chain_leaves_the_same_iterates(dq):
     """The same rounds by single calls (graph replay), by dq_rounds in random chunks, without graphs, and as separate
-    kernels must leave the same bits in x (and y), the same ||x||_inf and the same bit counts.  Drawn among dense
-    problems whose gradient sums have a fixed order (one block of rows per worker, or the two-kernel column sums);
-    where the one-cluster kernel applies, the separate-kernel chain sums in another order and is left out."""
+    kernels must leave the same bits in x (and y), the same ||x||_inf and the same bit counts.  Every gradient kernel
+    sums in a fixed order (dense rows) or on an exact integer grid (CSR rows); where the one-cluster kernel applies,
+    the separate-kernel chain forms its margins in another order and is left out."""
     import torch
     done = 0
     for trial in range(200):
@@ -95,11 +95,6 @@ def test_random_configurations_every_chain_leaves_the_same_iterates(dq):
         kind, h, kw, tau = draw_case(g)
         for k in ("no_fused", "no_graph", "max_delay"):
             kw.pop(k, None)
-        if kind == "csr":
-            continue                                               # float atomics
-        vec = (h.d % 4 == 0) if kind == "dense" else (h.d % 8 == 0)
-        if not (kw["B"] <= 16 or (vec and kw["B"] >= 64)):
-            kw["B"] = int(g.choice([1, 8, 16]))
         cluster = (not kw.get("sparsify") and not kw.get("sequential") and kw.get("mu", 0.0) == 0.0 and kw["bx"] in (2, 4, 8)
                    and h.d <= 8192 and kw["M"] <= 16)
         acc = bool(kw.get("accelerated", 0))
