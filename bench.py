@@ -59,6 +59,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="leave the c5 grid out of the line")
     ap.add_argument("--sweep", action="store_true", help="print only the c5 grid (adds d = 2^20) as one JSON object")
+    ap.add_argument("--only-training", action="store_true", help="time only the training configurations of --configs (one JSON object)")
+    ap.add_argument("--train-rounds", type=int, default=200, help="rounds timed per training configuration")
     ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_rounds ('' for none)")
     return ap.parse_args()
 
@@ -686,10 +688,22 @@ def run_sweep(a):
                       "peak_GBps": peak, "peak_source": peak_src, "l2_policy": "inputs rotated over >= 256 MiB", "points": points}))
 
 
+def run_training_only(a):
+    import torch
+    import paper_1805_10111_b200 as dq
+    torch.cuda.set_device(0)
+    dq.lib()
+    peak, _ = measured_peak()
+    print(json.dumps({"training_configs": {c: time_training_config(c, rounds=a.train_rounds, with_oracle=not a.no_cpu_baseline, peak=peak)
+                                           for c in a.configs.split(",") if c in TRAIN_CONFIGS}}))
+
+
 def main():
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.only_training:
+        run_training_only(a)
     elif a.sweep:
         run_sweep(a)
     else:

@@ -96,7 +96,10 @@ typedef struct {
                                   the data must be DQ_DENSE_F32 with labels = class index, data.d = number of inputs, and
                                   d = hidden*(in+1) + classes*(hidden+1) with x = [W1 (hidden x in), b1, W2 (classes x hidden), b2] */
     int32_t hidden, classes;
-    int32_t no_fused;          /* 1: never run rounds in the one-cluster kernel (see dq_round); 0: use it where it applies */
+    int32_t no_fused;          /* 0: merged kernels where they apply (the one-cluster round, quantiser + master in one kernel, the
+                                  one-pass dense gradient); 1: every stage as its own kernel(s), the plan the merged ones are tested
+                                  against; 2: like 1, but the one-pass dense gradient stays on, in its CUDA-core form (bfloat16 rows
+                                  otherwise take its tensor-core form) */
     int32_t max_delay;         /* tau of Assumption 3: dq_round keeps the last tau + 1 broadcast models of the epoch so that
                                   workers can be made to lag (dq_set_delays); 0: every worker uses the current broadcast */
 } dq_config;

@@ -397,13 +397,16 @@ worker_colsum_kernel(const T* __restrict__ X, const int32_t* __restrict__ rows, 
 //
 //   tiles      a tile is kFusedRows consecutive minibatch slots of one worker; the M * ceil(B / 8) tiles are split
 //              into contiguous runs, one run per block (one block per SM)
-//   staging    warp 1 draws the tile's row indices and issues one bulk asynchronous copy per row into a ring of
-//              kFusedStages shared-memory stages; an mbarrier per stage counts the bytes
-//   margins    thread v owns the 16-byte column group v of every row: it keeps the tile's eight groups in registers,
-//              forms eight partial dot products with its slice of xhat - xsnap, the warp folds them in a fixed
-//              butterfly, and warp 0 adds the warps' partial sums in warp order (double) and turns the eight margins
-//              into slope differences
-//   columns    one tile later every thread adds r_j * row_j to its columns from the registers it kept
+//   staging    the load warp draws the tile's row indices and issues one bulk asynchronous copy per row into a ring
+//              of kFusedStages shared-memory stages; an mbarrier per stage counts the bytes, a second one counts the
+//              compute warps that have taken their groups out of the stage (then it is refilled)
+//   margins    compute thread v owns the 16-byte column group v of every row: it keeps the tile's eight groups in
+//              registers, forms eight partial dot products with its slice of xhat - xsnap, the warp folds them in a
+//              fixed butterfly, and the slope warp adds the warps' partial sums in warp order (double) and turns the
+//              eight margins into slope differences
+//   columns    one tile later the compute threads add r_j * row_j to their columns from the registers they kept;
+//              warps hand over through mbarriers (partials ready / slopes ready), so nobody waits for the slope warp
+//              unless it falls a whole tile behind
 //   combine    a block's column sums for a worker go to a scratch slot; the block that completes a worker (a
 //              counter tells it; nobody waits) adds that worker's slots in block order, writes alpha_w and
 //              ||alpha_w||_inf.  The order of every sum is fixed, so alpha is reproducible bit for bit.
@@ -412,8 +415,8 @@ worker_colsum_kernel(const T* __restrict__ X, const int32_t* __restrict__ rows, 
 // ---------------------------------------------------------------------------------------------------
 constexpr int kFusedRows = 8;                      // rows per tile
 constexpr int kFusedStages = 3;                    // tiles in flight per block
-constexpr int kFusedWarps = 16;                    // sixteen warps: four per scheduler, 128 registers each
-constexpr int kFusedThreads = kFusedWarps * 32;
+constexpr int kFusedComputeWarps = 16;             // one 16-byte column group per compute thread
+constexpr int kFusedThreads = (kFusedComputeWarps + 2) * 32;   // + the slope warp and the load warp
 constexpr int kFusedMaxRowBytes = 8192;            // one 16-byte group per thread
 constexpr int kFusedRowPad = 16;                   // bytes between staged rows beyond the row itself (bank spread)
 constexpr long long kFusedWaitCycles = 1ll << 31;  // about a second: no copy takes that long
@@ -427,6 +430,10 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count)
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity)
 {
@@ -491,7 +498,7 @@ struct FusedPlan {
     }
 };
 
-template <class T>
+template <class T, bool MMA>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
                          const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, FusedPlan pl,
@@ -502,180 +509,330 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
     pdl_prologue();
     clear_word(bs);
     constexpr int N = RowVec<T>::N;                          // features per 16-byte group
-    constexpr int S = kFusedStages, R = kFusedRows;
+    constexpr int S = kFusedStages, R = kFusedRows, CW = kFusedComputeWarps;
     extern __shared__ __align__(128) unsigned char s_stage[];    // [S][R][row_bytes + pad]
-    __shared__ __align__(8) uint64_t s_full[S];
-    __shared__ float s_part[2][kFusedWarps][R];
+    __shared__ __align__(8) uint64_t s_full[S], s_empty[S], s_pready[2], s_rready[2];
+    __shared__ float s_part[2][CW][R];
     __shared__ float s_r[2][R];
-    __shared__ float s_lab[S + 1][R], s_zs[S + 1][R];           // ring of S + 1: tile it + S is issued while tile it's entries are read
-    __shared__ uint32_t s_max[kFusedWarps];
+    __shared__ __align__(4) uint16_t s_rsplit[2][3][R];          // MMA: the slopes as three bfloat16 terms (hi + mid + lo = r to 24 bits)
+    __shared__ float s_lab[S + 2][R], s_zs[S + 2][R];           // ring of S + 2: tiles it + S and it + S + 1 can be issued while tile it's entries are still read
+    __shared__ uint32_t s_max[CW];
     __shared__ int s_abort, s_last, s_issued;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool slope_warp = warp == 0, load_warp = warp == 1;       // the two extra duties sit on different warps so that they overlap
+    const bool slope_warp = warp == CW, load_warp = warp == CW + 1, compute = warp < CW;
     const int row_bytes = (int)(d * (int64_t)sizeof(T)), stride = row_bytes + kFusedRowPad;
     const int nvec = row_bytes >> 4;
-    const int v = tid;                                       // this thread's column group
-    const bool active = v < nvec;
+    const int v = tid;                                       // a compute thread's column group
+    const bool active = compute && v < nvec;
     const int blk = blockIdx.x;
     const int t0 = pl.tile_begin(blk), ntl = pl.tile_begin(blk + 1) - t0;
+    // MMA: xhat - xsnap of the current worker as three bfloat16 terms, [3][d], behind the stages
+    uint16_t* s_dsplit = reinterpret_cast<uint16_t*>(s_stage + (size_t)S * R * stride);
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) mbar_init(&s_full[s], 1);
+        for (int s = 0; s < S; ++s) { mbar_init(&s_full[s], 1); mbar_init(&s_empty[s], CW); }
+        for (int s = 0; s < 2; ++s) { mbar_init(&s_pready[s], CW); mbar_init(&s_rready[s], 1); }
         s_abort = 0; s_last = 0; s_issued = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
 
-    // warp 1: draw the rows of tile `it` of this block's run and start their copies into stage it % S
-    auto issue = [&](int it) {
-        const int t = t0 + it, stage = it % S, slot = it % (S + 1);
-        const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
-        const int nvalid = min(R, pl.B - j0);
-        if (lane == 0) { mbar_arrive_expect_tx(&s_full[stage], (uint32_t)(nvalid * row_bytes)); s_issued = it + 1; }
-        __syncwarp();
-        if (lane < R) {
-            if (lane < nvalid) {
-                const int64_t a = batch_row(bs, K, w, j0 + lane, pl.B, true);
-                // label and snapshot margin travel beside the row (4-byte asynchronous copies: nobody waits for them here)
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(smem_u32(&s_lab[slot][lane])), "l"(labels + a) : "memory");
-                asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" :: "r"(smem_u32(&s_zs[slot][lane])), "l"(z_snap + a) : "memory");
-                bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
-            }
+    // A wait that gives up: after kFusedWaitCycles the block is marked aborted, DQ_ERR_TIMEOUT is recorded, and from
+    // then on no wait of this block blocks any more.  Every thread still walks through the same barriers to the end
+    // (the results are void, the status says so), so nothing is left hanging.
+    auto wait = [&](uint64_t* bar, uint32_t parity) {
+        if (*reinterpret_cast<volatile int*>(&s_abort)) return;
+        if (mbar_try_wait(bar, parity)) return;
+        const long long c0 = clock64();
+        while (!mbar_try_wait(bar, parity)) {
+            if (*reinterpret_cast<volatile int*>(&s_abort)) return;
+            if (clock64() - c0 > kFusedWaitCycles) { s_abort = 1; set_status(status, DQ_ERR_TIMEOUT); return; }
         }
     };
-    if (load_warp) {
-        for (int it = 0; it < min(S, ntl); ++it) issue(it);
-        asm volatile("cp.async.wait_all;" ::: "memory");     // labels and margins of the first tiles (the rows stay in flight)
-    }
+    const auto worker_at = [&](int it) { return it < ntl ? pl.worker_of(t0 + it) : -1; };
+    // a worker's last tile in this block has been added when the next tile belongs to another worker (or the run ends)
+    const auto flush_at = [&](int it) { return it > 0 && worker_at(it) != worker_at(it - 1); };
 
-    float acc[N], dreg[N];
-#pragma unroll
-    for (int n = 0; n < N; ++n) { acc[n] = 0.0f; dreg[n] = 0.0f; }
-    uint4 q_old[R], q_new[R];
-#pragma unroll
-    for (int r = 0; r < R; ++r) q_old[r] = make_uint4(0u, 0u, 0u, 0u);
-    int w_prev = -1, nvalid_prev = 0;
+    // load warp: draw the rows of tile `it` of this block's run and start their copies into stage it % S
+    auto issue = [&](int it) {
+        const int t = t0 + it, stage = it % S, slot = it % (S + 2);
+        const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
+        const int nvalid = min(R, pl.B - j0);
+        if (lane < nvalid) {
+            const int64_t a = batch_row(bs, K, w, j0 + lane, pl.B, true);
+            bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
+            // the row's label and snapshot margin go beside it.  They are stored before this warp's arrival on the stage's
+            // barrier below, so whoever has seen the stage full (and whoever hears from them) sees them too.
+            const float lab = __ldg(labels + a), zs = __ldg(z_snap + a);
+            s_lab[slot][lane] = lab; s_zs[slot][lane] = zs;
+        }
+        if (MMA && nvalid < R) {         // the tensor-core path multiplies whole tiles: rows past the minibatch's end must read as zeros
+            uint4* z = reinterpret_cast<uint4*>(s_stage + ((size_t)stage * R + nvalid) * stride);
+            for (int q = lane; q < (R - nvalid) * (stride >> 4); q += 32) z[q] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncwarp();
+        // the byte count is announced after the copies were started: the phase cannot complete before this arrival
+        if (lane == 0) { mbar_arrive_expect_tx(&s_full[stage], (uint32_t)(nvalid * row_bytes)); s_issued = it + 1; }
+    };
 
-    int it = 0;
-    for (; it <= ntl; ++it) {
-        const int t = t0 + it, par = it & 1, stage = it % S;
-        const int w_cur = it < ntl ? pl.worker_of(t) : -1;
-        const int j0 = it < ntl ? (t - w_cur * pl.tiles_per_worker) * R : 0;
-        const int nvalid = it < ntl ? min(R, pl.B - j0) : 0;
-        // ---- front: margins of tile it ----------------------------------------------------------------------------
-        if (it < ntl) {
-            if (w_cur != w_prev && active) {                 // this worker's xhat - xsnap (a lagging worker reads an older one)
-                const float4* dv = reinterpret_cast<const float4*>(diff_of_worker(bs, diff, w_cur)) + (size_t)v * (N / 4);
+    // the flush of worker w: every thread of the block takes part in its barriers
+    float acc[N];
 #pragma unroll
-                for (int q = 0; q < N / 4; ++q) { const float4 x4 = __ldg(dv + q); dreg[q * 4] = x4.x; dreg[q * 4 + 1] = x4.y; dreg[q * 4 + 2] = x4.z; dreg[q * 4 + 3] = x4.w; }
-            }
-            if (!mbar_wait_bounded(&s_full[stage], (uint32_t)((it / S) & 1))) { s_abort = 1; set_status(status, DQ_ERR_TIMEOUT); }
-            float p[R];
-            const unsigned char* base = s_stage + (size_t)stage * R * stride + (size_t)v * 16;
+    for (int n = 0; n < N; ++n) acc[n] = 0.0f;
+    auto flush = [&](int w) {
+        if (!MMA && active) {
+            float4* dst = reinterpret_cast<float4*>(part + (size_t)(blk + w) * d) + (size_t)v * (N / 4);
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                q_new[r] = (active && r < nvalid) ? *reinterpret_cast<const uint4*>(base + (size_t)r * stride) : make_uint4(0u, 0u, 0u, 0u);
-                float f[N];
-                RowVec<T>::unpack(q_new[r], f);
-                float s = 0.0f;
-#pragma unroll
-                for (int n = 0; n < N; ++n) s = fmaf(f[n], dreg[n], s);
-                p[r] = s;
-            }
-            const float folded = fold8(p, lane);
-            if ((lane & 3) == 0) s_part[par][warp][((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = folded;
+            for (int q = 0; q < N / 4; ++q) dst[q] = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
         }
-        __syncthreads();                                     // A(it): the stage has been read, the partial margins are visible
-        if (s_abort) break;
-        // ---- warp 1: the copies of tile it + S into the stage that was just read; warp 0: slopes of tile it ---------
-        if (load_warp && it < ntl) {
-            asm volatile("cp.async.wait_all;" ::: "memory");     // labels and margins of the tiles issued so far: tile it + 1's are
-            if (it + S < ntl) issue(it + S);                     // visible to warp 0 after the next barrier
-        }
-        if (slope_warp && it < ntl) {
-            if (lane < R) {
-                float rj = 0.0f;
-                if (lane < nvalid) {
-                    double dz = 0.0;
 #pragma unroll
-                    for (int k = 0; k < kFusedWarps; ++k) dz += (double)s_part[par][k][lane];
-                    rj = slope_difference(s_lab[it % (S + 1)][lane], s_zs[it % (S + 1)][lane], (float)dz) / (float)pl.B;
+        for (int n = 0; n < N; ++n) acc[n] = 0.0f;
+        __threadfence();
+        __syncthreads();
+        const int b_first = pl.block_of_tile(w * pl.tiles_per_worker), b_last = pl.block_of_tile((w + 1) * pl.tiles_per_worker - 1);
+        if (tid == 0) {
+            const uint32_t old = atomicAdd(counters + w, 1u);
+            s_last = old == (uint32_t)(b_last - b_first);
+            if (s_last) counters[w] = 0u;                    // every block of this worker has added: ready for the next launch
+        }
+        __syncthreads();
+        if (s_last) {                                        // this block completes worker w: slots in block order
+            __threadfence();
+            uint32_t nmax = 0;
+            if (active) {
+                float sum[N];
+#pragma unroll
+                for (int n = 0; n < N; ++n) sum[n] = 0.0f;
+                for (int bb = b_first; bb <= b_last; ++bb) {
+                    const float4* src = reinterpret_cast<const float4*>(part + (size_t)(bb + w) * d) + (size_t)v * (N / 4);
+#pragma unroll
+                    for (int q = 0; q < N / 4; ++q) {
+                        const float4 x4 = __ldcg(src + q);
+                        sum[q * 4] += x4.x; sum[q * 4 + 1] += x4.y; sum[q * 4 + 2] += x4.z; sum[q * 4 + 3] += x4.w;
+                    }
                 }
-                s_r[par][lane] = rj;
+                float4* out = reinterpret_cast<float4*>(alpha + (size_t)w * d) + (size_t)v * (N / 4);
+#pragma unroll
+                for (int q = 0; q < N / 4; ++q) out[q] = make_float4(sum[q * 4], sum[q * 4 + 1], sum[q * 4 + 2], sum[q * 4 + 3]);
+#pragma unroll
+                for (int n = 0; n < N; ++n) nmax = max(nmax, __float_as_uint(sum[n]) & 0x7FFFFFFFu);
+            }
+            nmax = warp_max_u32(nmax);
+            if (compute && lane == 0) s_max[warp] = nmax;
+            __syncthreads();
+            if (tid == 0) {
+                uint32_t m = 0;
+                for (int k = 0; k < CW; ++k) m = max(m, s_max[k]);
+                norm_bits[w] = m;
+            }
+            __syncthreads();
+        }
+    };
+
+    if (load_warp) {
+        // ---- copies: S tiles ahead; a stage is refilled once every compute warp has taken its groups out of it -------
+        for (int it = 0; it < min(S, ntl); ++it) issue(it);
+        for (int it = 0; it <= ntl; ++it) {
+            if (flush_at(it)) flush(worker_at(it - 1));
+            if (it + S < ntl) {
+                wait(&s_empty[it % S], (uint32_t)((it / S) & 1));
+                issue(it + S);
+            }
+        }
+    } else if (slope_warp) {
+        // ---- slopes: margins of tile it from the warps' partial sums (warp order, double), slope differences --------
+        for (int it = 0; it <= ntl; ++it) {
+            if (flush_at(it)) flush(worker_at(it - 1));
+            if (it == ntl) break;
+            const int par = it & 1;
+            const int w_cur = worker_at(it), j0 = (t0 + it - w_cur * pl.tiles_per_worker) * R;
+            const int nvalid = min(R, pl.B - j0);
+            wait(&s_pready[par], (uint32_t)((it >> 1) & 1));
+            // lane = 4 * row + quarter: a quarter of the warps' partial sums each, then the quarters in order
+            const int row = lane >> 2, qtr = lane & 3;
+            double dz = 0.0;
+#pragma unroll
+            for (int k = 0; k < CW / 4; ++k) dz += (double)s_part[par][qtr * (CW / 4) + k][row];
+            const double d1 = __shfl_xor_sync(0xFFFFFFFFu, dz, 1);
+            dz = (qtr & 1) ? d1 + dz : dz + d1;                  // (q0 + q1), (q2 + q3): the same order in both lanes
+            const double d2 = __shfl_xor_sync(0xFFFFFFFFu, dz, 2);
+            dz = (qtr & 2) ? d2 + dz : dz + d2;
+            if (qtr == 0) {
+                float rj = 0.0f;
+                if (row < nvalid) {
+                    const int slot = it % (S + 2);
+                    rj = slope_difference(*reinterpret_cast<volatile float*>(&s_lab[slot][row]), *reinterpret_cast<volatile float*>(&s_zs[slot][row]), (float)dz) / (float)pl.B;
+                }
+                s_r[par][row] = rj;
+                if (MMA) {
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(rj);
+                    const float r1 = rj - __bfloat162float(hi);
+                    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                    s_rsplit[par][0][row] = __bfloat16_as_ushort(hi); s_rsplit[par][1][row] = __bfloat16_as_ushort(mid);
+                    s_rsplit[par][2][row] = __bfloat16_as_ushort(lo);
+                }
             }
             __syncwarp();
+            if (lane == 0) mbar_arrive(&s_rready[par]);
         }
-        // ---- back: add the rows of tile it - 1 to the columns ------------------------------------------------------
-        if (it > 0) {
+    } else if (MMA) {
+        // ---- compute warps, tensor cores -----------------------------------------------------------------------------
+        // Both products of a tile run as warp-level bf16 MMAs with fp32 accumulation; an fp32 factor enters as three
+        // bfloat16 terms in three columns of the narrow operand.  Warp wp owns the columns [wp cpw, (wp + 1) cpw).
+        //   margins  D[variant][row] += sum_k diff_variant[k] X[row][k]: m16n8k16, A = the three terms of xhat - xsnap
+        //            (rows 0..2 of 16), B = the tile's eight rows straight from the stage (ldmatrix)
+        //   columns  D[col][variant] += sum_row X[row][col] r_variant[row]: m16n8k8, A = the tile transposed
+        //            (ldmatrix.trans), B = the three terms of the slopes; 16 columns x 8 per MMA, 4 accumulators each
+        const int g = lane >> 2, c2 = (lane & 3) * 2;
+        const int ksteps = (int)(d >> 4), kpw = (ksteps + CW - 1) / CW;               // 16-column steps in all, per warp
+        const int k_first = warp * kpw, k_count = max(0, min(kpw, ksteps - k_first));
+        float cacc[kFusedMaxRowBytes / 2 / 16 / CW][4];                               // [m-tile][4]: columns of this warp
 #pragma unroll
-            for (int r = 0; r < R; ++r) {
-                if (r < nvalid_prev) {
-                    const float rr = s_r[par ^ 1][r];
-                    float f[N];
-                    RowVec<T>::unpack(q_old[r], f);
-#pragma unroll
-                    for (int n = 0; n < N; ++n) acc[n] = fmaf(rr, f[n], acc[n]);
-                }
-            }
-        }
-        // ---- a worker's last tile in this block has been added: hand its column sums over ---------------------------
-        if (it > 0 && w_cur != w_prev) {
-            const int w = w_prev;
-            if (active) {
-                float4* dst = reinterpret_cast<float4*>(part + (size_t)(blk + w) * d) + (size_t)v * (N / 4);
-#pragma unroll
-                for (int q = 0; q < N / 4; ++q) dst[q] = make_float4(acc[q * 4], acc[q * 4 + 1], acc[q * 4 + 2], acc[q * 4 + 3]);
-            }
-#pragma unroll
-            for (int n = 0; n < N; ++n) acc[n] = 0.0f;
-            __threadfence();
-            __syncthreads();
-            const int b_first = pl.block_of_tile(w * pl.tiles_per_worker), b_last = pl.block_of_tile((w + 1) * pl.tiles_per_worker - 1);
-            if (tid == 0) {
-                const uint32_t old = atomicAdd(counters + w, 1u);
-                s_last = old == (uint32_t)(b_last - b_first);
-                if (s_last) counters[w] = 0u;                // every block of this worker has added: ready for the next launch
-            }
-            __syncthreads();
-            if (s_last) {                                    // this block completes worker w: slots in block order
-                __threadfence();
-                uint32_t nmax = 0;
-                if (active) {
-                    float sum[N];
-#pragma unroll
-                    for (int n = 0; n < N; ++n) sum[n] = 0.0f;
-                    for (int bb = b_first; bb <= b_last; ++bb) {
-                        const float4* src = reinterpret_cast<const float4*>(part + (size_t)(bb + w) * d) + (size_t)v * (N / 4);
-#pragma unroll
-                        for (int q = 0; q < N / 4; ++q) {
-                            const float4 x4 = __ldcg(src + q);
-                            sum[q * 4] += x4.x; sum[q * 4 + 1] += x4.y; sum[q * 4 + 2] += x4.z; sum[q * 4 + 3] += x4.w;
-                        }
+        for (int i = 0; i < kFusedMaxRowBytes / 2 / 16 / CW; ++i) { cacc[i][0] = cacc[i][1] = cacc[i][2] = cacc[i][3] = 0.0f; }
+        int w_prev = -1;
+        const uint32_t lane_row_off = (uint32_t)((lane & 7) * stride + ((lane >> 3) & 1) * 16);   // ldmatrix: lanes 0-7 first matrix, 8-15 second
+        for (int it = 0; it <= ntl; ++it) {
+            const int par = it & 1, stage = it % S;
+            const int w_cur = worker_at(it);
+            if (it < ntl) {
+                if (w_cur != w_prev) {                       // new worker: its xhat - xsnap as hi + mid + lo
+                    asm volatile("bar.sync 1, %0;" :: "n"(CW * 32) : "memory");      // every compute warp is done with the old terms
+                    const float* dv = diff_of_worker(bs, diff, w_cur);
+                    for (int64_t i = tid; i < d; i += CW * 32) {
+                        const float x = __ldg(dv + i);
+                        const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                        const float r1 = x - __bfloat162float(hi);
+                        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                        const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                        s_dsplit[i] = __bfloat16_as_ushort(hi); s_dsplit[d + i] = __bfloat16_as_ushort(mid); s_dsplit[2 * d + i] = __bfloat16_as_ushort(lo);
                     }
-                    float4* out = reinterpret_cast<float4*>(alpha + (size_t)w * d) + (size_t)v * (N / 4);
-#pragma unroll
-                    for (int q = 0; q < N / 4; ++q) out[q] = make_float4(sum[q * 4], sum[q * 4 + 1], sum[q * 4 + 2], sum[q * 4 + 3]);
-#pragma unroll
-                    for (int n = 0; n < N; ++n) nmax = max(nmax, __float_as_uint(sum[n]) & 0x7FFFFFFFu);
+                    asm volatile("bar.sync 1, %0;" :: "n"(CW * 32) : "memory");
                 }
-                nmax = warp_max_u32(nmax);
-                if (lane == 0) s_max[warp] = nmax;
-                __syncthreads();
-                if (tid == 0) {
-                    uint32_t m = 0;
-                    for (int k = 0; k < kFusedWarps; ++k) m = max(m, s_max[k]);
-                    norm_bits[w] = m;
+                wait(&s_full[stage], (uint32_t)((it / S) & 1));
+                const uint32_t sbase = smem_u32(s_stage + (size_t)stage * R * stride) + lane_row_off;
+                float c0 = 0.0f, c1 = 0.0f, c2r = 0.0f, c3 = 0.0f;
+#pragma unroll 4
+                for (int ks = 0; ks < k_count; ++ks) {
+                    const int col = (k_first + ks) << 4;
+                    uint32_t a0 = 0u, a2 = 0u, b0, b1;
+                    if (g < 3) {
+                        const uint16_t* dp = s_dsplit + (size_t)g * d + col + c2;
+                        a0 = *reinterpret_cast<const uint32_t*>(dp); a2 = *reinterpret_cast<const uint32_t*>(dp + 8);
+                    }
+                    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(sbase + (uint32_t)col * 2u));
+                    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                 : "+f"(c0), "+f"(c1), "+f"(c2r), "+f"(c3) : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
                 }
-                __syncthreads();
+                // rows 0..2 of D hold the three terms' sums for tile rows c2, c2 + 1: add them up (the other rows are zero)
+#pragma unroll
+                for (int o = 4; o < 32; o <<= 1) { c0 += __shfl_xor_sync(0xFFFFFFFFu, c0, o); c1 += __shfl_xor_sync(0xFFFFFFFFu, c1, o); }
+                if (it >= 2) wait(&s_rready[par], (uint32_t)(((it - 2) >> 1) & 1));      // the slopes of tile it - 2 have been formed: its partial sums are free
+                if (lane < 4) { s_part[par][warp][c2] = c0; s_part[par][warp][c2 + 1] = c1; }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_pready[par]);
             }
-        }
+            if (it > 0) {
+                // back: the rows of tile it - 1 (still in their stage) times their slopes
+                wait(&s_rready[par ^ 1], (uint32_t)(((it - 1) >> 1) & 1));
+                const int pstage = (it - 1) % S;
+                const uint32_t sbase = smem_u32(s_stage + (size_t)pstage * R * stride) + lane_row_off;
+                const uint32_t b0 = g < 3 ? *reinterpret_cast<const uint32_t*>(&s_rsplit[par ^ 1][g][c2]) : 0u;
 #pragma unroll
-        for (int r = 0; r < R; ++r) q_old[r] = q_new[r];
-        w_prev = w_cur; nvalid_prev = nvalid;
+                for (int i = 0; i < kFusedMaxRowBytes / 2 / 16 / CW; ++i) {
+                    if (i < k_count) {
+                        const int col = (k_first + i) << 4;
+                        uint32_t a0, a1;
+                        asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(a0), "=r"(a1) : "r"(sbase + (uint32_t)col * 2u));
+                        asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                                     : "+f"(cacc[i][0]), "+f"(cacc[i][1]), "+f"(cacc[i][2]), "+f"(cacc[i][3]) : "r"(a0), "r"(a1), "r"(b0));
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_empty[pstage]);    // the tile has been used for both products: the stage may be refilled
+            }
+            if (flush_at(it)) {
+                // column sum = hi + mid + lo columns of D: lanes with c2 == 0 hold the first two, their neighbour the third
+                float* dst = part + (size_t)(blk + w_prev) * d;
+#pragma unroll
+                for (int i = 0; i < kFusedMaxRowBytes / 2 / 16 / CW; ++i) {
+                    float u0 = cacc[i][0] + cacc[i][1], u1 = cacc[i][2] + cacc[i][3];
+                    u0 += __shfl_xor_sync(0xFFFFFFFFu, u0, 1); u1 += __shfl_xor_sync(0xFFFFFFFFu, u1, 1);
+                    if (i < k_count && c2 == 0) { const int col = ((k_first + i) << 4) + g; dst[col] = u0; dst[col + 8] = u1; }
+                    cacc[i][0] = cacc[i][1] = cacc[i][2] = cacc[i][3] = 0.0f;
+                }
+                flush(w_prev);
+            }
+            w_prev = w_cur;
+        }
+    } else {
+        // ---- compute warps, CUDA cores ---------------------------------------------------------------------------------
+        float dreg[N];
+#pragma unroll
+        for (int n = 0; n < N; ++n) dreg[n] = 0.0f;
+        uint4 q_old[R], q_new[R];
+#pragma unroll
+        for (int r = 0; r < R; ++r) q_old[r] = q_new[r] = make_uint4(0u, 0u, 0u, 0u);
+        int w_prev = -1, nvalid_prev = 0;
+        for (int it = 0; it <= ntl; ++it) {
+            const int par = it & 1, stage = it % S;
+            const int w_cur = worker_at(it);
+            const int j0 = it < ntl ? (t0 + it - w_cur * pl.tiles_per_worker) * R : 0;
+            const int nvalid = it < ntl ? min(R, pl.B - j0) : 0;
+            if (it < ntl) {
+                // front: margins of tile it
+                if (w_cur != w_prev && active) {             // this worker's xhat - xsnap (a lagging worker reads an older one)
+                    const float4* dv = reinterpret_cast<const float4*>(diff_of_worker(bs, diff, w_cur)) + (size_t)v * (N / 4);
+#pragma unroll
+                    for (int q = 0; q < N / 4; ++q) { const float4 x4 = __ldg(dv + q); dreg[q * 4] = x4.x; dreg[q * 4 + 1] = x4.y; dreg[q * 4 + 2] = x4.z; dreg[q * 4 + 3] = x4.w; }
+                }
+                wait(&s_full[stage], (uint32_t)((it / S) & 1));
+                const unsigned char* base = s_stage + (size_t)stage * R * stride + (size_t)v * 16;
+#pragma unroll
+                for (int r = 0; r < R; ++r)
+                    q_new[r] = (active && r < nvalid) ? *reinterpret_cast<const uint4*>(base + (size_t)r * stride) : make_uint4(0u, 0u, 0u, 0u);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_empty[stage]);     // this warp's groups are in registers: the stage may be refilled
+                float p[R];
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    float f[N];
+                    RowVec<T>::unpack(q_new[r], f);
+                    float s = 0.0f;
+#pragma unroll
+                    for (int n = 0; n < N; ++n) s = fmaf(f[n], dreg[n], s);
+                    p[r] = s;
+                }
+                if (it >= 2) wait(&s_rready[par], (uint32_t)(((it - 2) >> 1) & 1));      // the slopes of tile it - 2 have been formed: its partial sums are free
+                const float folded = fold8(p, lane);
+                if ((lane & 3) == 0) s_part[par][warp][((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = folded;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_pready[par]);
+            }
+            if (it > 0) {
+                // back: add the rows of tile it - 1 to the columns
+                wait(&s_rready[par ^ 1], (uint32_t)(((it - 1) >> 1) & 1));
+#pragma unroll
+                for (int r = 0; r < R; ++r) {
+                    if (r < nvalid_prev) {
+                        const float rr = s_r[par ^ 1][r];
+                        float f[N];
+                        RowVec<T>::unpack(q_old[r], f);
+#pragma unroll
+                        for (int n = 0; n < N; ++n) acc[n] = fmaf(rr, f[n], acc[n]);
+                    }
+                }
+            }
+            if (flush_at(it)) flush(w_prev);
+#pragma unroll
+            for (int r = 0; r < R; ++r) q_old[r] = q_new[r];
+            w_prev = w_cur; nvalid_prev = nvalid;
+        }
     }
+    __syncthreads();
     if (s_abort && tid == 0) {
         // a copy did not arrive in time: give the copies still in flight a bounded time to land before the block's
         // shared memory is released
-        for (int k = it; k < s_issued; ++k) (void)mbar_wait_bounded(&s_full[k % S], (uint32_t)((k / S) & 1));
+        for (int k = 0; k < s_issued; ++k) (void)mbar_wait_bounded(&s_full[k % S], (uint32_t)((k / S) & 1));
     }
 }
 
@@ -1429,12 +1586,22 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
 
 // The one-pass kernel takes dense rows of at most kFusedMaxRowBytes on the 16-byte grid; the context then owns its
 // scratch (column sums per (block, worker), per-worker counters).
+// bfloat16 rows whose length is a multiple of 16 take the tensor-core variant (no_fused = 2 keeps the CUDA-core one)
+static bool fused_grad_mma(const dq_ctx* ctx) { return ctx->data.format == DQ_DENSE_BF16 && (ctx->cfg.d & 15) == 0 && ctx->cfg.no_fused != 2; }
 static size_t fused_grad_smem(const dq_ctx* ctx)
 {
     const size_t row_bytes = (size_t)ctx->cfg.d * (ctx->data.format == DQ_DENSE_F32 ? 4 : 2);
-    return (size_t)kFusedStages * kFusedRows * (row_bytes + kFusedRowPad);
+    return (size_t)kFusedStages * kFusedRows * (row_bytes + kFusedRowPad) + (fused_grad_mma(ctx) ? 3 * row_bytes : 0);
 }
-bool fused_grad_applies(const dq_ctx* ctx) { return ctx->fused_part != nullptr && !ctx->cfg.no_fused; }
+bool fused_grad_applies(const dq_ctx* ctx) { return ctx->fused_part != nullptr && ctx->cfg.no_fused != 1; }
+typedef void (*FusedKernelF32)(const float*, const float*, const float*, const float*, const PhiloxKeys, BatchSource, FusedPlan, int64_t,
+                               float*, uint32_t*, float*, uint32_t*, int*);
+typedef void (*FusedKernelBf16)(const __nv_bfloat16*, const float*, const float*, const float*, const PhiloxKeys, BatchSource, FusedPlan,
+                                int64_t, float*, uint32_t*, float*, uint32_t*, int*);
+static FusedKernelBf16 fused_kernel_bf16(const dq_ctx* ctx)
+{
+    return fused_grad_mma(ctx) ? worker_grad_fused_kernel<__nv_bfloat16, true> : worker_grad_fused_kernel<__nv_bfloat16, false>;
+}
 
 // Called once per context: scratch and the shared-memory opt-in of the one-pass dense gradient kernel.
 int fused_grad_setup(dq_ctx* ctx)
@@ -1444,14 +1611,14 @@ int fused_grad_setup(dq_ctx* ctx)
     const size_t row_bytes = (size_t)c.d * (D.format == DQ_DENSE_F32 ? 4 : 2);
     if (row_bytes > kFusedMaxRowBytes || (row_bytes & 15) || c.B < 64) return DQ_OK;
     const int smem = (int)fused_grad_smem(ctx);
-    const cudaError_t e = D.format == DQ_DENSE_F32
-        ? cudaFuncSetAttribute(worker_grad_fused_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
-        : cudaFuncSetAttribute(worker_grad_fused_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    const FusedKernelF32 kf = worker_grad_fused_kernel<float, false>;
+    const FusedKernelBf16 kb = fused_kernel_bf16(ctx);
+    const cudaError_t e = D.format == DQ_DENSE_F32 ? cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
+                                                   : cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) { cudaGetLastError(); return DQ_OK; }          // the two-kernel path remains
     int resident = 0;                                                    // a block must fit an SM (registers, shared memory)
-    const cudaError_t o = D.format == DQ_DENSE_F32
-        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, worker_grad_fused_kernel<float>, kFusedThreads, (size_t)smem)
-        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, worker_grad_fused_kernel<__nv_bfloat16>, kFusedThreads, (size_t)smem);
+    const cudaError_t o = D.format == DQ_DENSE_F32 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kf, kFusedThreads, (size_t)smem)
+                                                   : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kb, kFusedThreads, (size_t)smem);
     if (o != cudaSuccess || resident < 1) { cudaGetLastError(); return DQ_OK; }
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->fused_part), sizeof(float) * (size_t)(ctx->sm_count + c.M) * c.d) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&ctx->fused_cnt), sizeof(uint32_t) * c.M) != cudaSuccess ||
@@ -1515,10 +1682,10 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
             const size_t smem = fused_grad_smem(ctx);
             uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
             if (f32)
-                launch_k(worker_grad_fused_kernel<float>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
+                launch_k(worker_grad_fused_kernel<float, false>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
                          s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status);
             else
-                launch_k(worker_grad_fused_kernel<__nv_bfloat16>, pl.nblocks, kFusedThreads, smem, st, (const __nv_bfloat16*)D.values, D.labels,
+                launch_k(fused_kernel_bf16(ctx), pl.nblocks, kFusedThreads, smem, st, (const __nv_bfloat16*)D.values, D.labels,
                          ctx->xhat_diff, s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status);
             ctx->launches += 1;
             return;
