@@ -97,11 +97,13 @@ typedef struct {
                                   d = hidden*(in+1) + classes*(hidden+1) with x = [W1 (hidden x in), b1, W2 (classes x hidden), b2] */
     int32_t hidden, classes;
     int32_t no_fused;          /* 0: merged kernels where they apply (the one-cluster round, quantiser + master in one kernel, the
-                                  one-pass dense gradient); 1: every stage as its own kernel(s), the plan the merged ones are tested
-                                  against; 2: like 1, but the one-pass dense gradient stays on, in its CUDA-core form (bfloat16 rows
-                                  otherwise take its tensor-core form) */
+                                  one-pass dense gradient carrying the whole round); 1: every stage as its own kernel(s), the plan
+                                  the merged ones are tested against; 2: like 1, but the dense gradient stage stays one pass */
     int32_t max_delay;         /* tau of Assumption 3: dq_round keeps the last tau + 1 broadcast models of the epoch so that
                                   workers can be made to lag (dq_set_delays); 0: every worker uses the current broadcast */
+    int32_t tensor_cores;      /* 1: the one-pass dense gradient forms X (xhat - xsnap) and X^T r of bfloat16 rows (d a multiple of
+                                  16) as bf16 tensor-core MMAs with fp32 accumulation, the fp32 factors split into three bfloat16
+                                  terms; 0: fp32 FMAs on CUDA cores (the default: measured faster, see the profiles) */
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3

@@ -344,6 +344,14 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
                          uint64_t* bits_up, void* st)
 {
     int rc = DQ_OK;
+    if (!flag && fused_round_applies(ctx)) {                 // large dense minibatches: model and message quantisers ride in the gradient kernel
+        const BitsArgs ba0 = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, 0, 0, ctx->cfg.bx, ctx->cfg.b, nullptr};
+        launch_fused_round(ctx, s, round, as_stream(st));
+        ctx->normx_zeroed = true;                            // the gradient kernel's last block cleared ||x||_inf for the master's maximum
+        launch_master(ctx, &ctx->msgs, false, s, eta, theta, as_stream(st), (bits_down || bits_up) ? &ba0 : nullptr);
+        ctx->normx_zeroed = false;
+        return last_error();
+    }
     const bool adaptive = ctx->cfg.mu > 0.0f;
     // delayed workers: this round's xhat - xsnap goes to its slot of the ring, and every worker is pointed at the
     // slot of the broadcast it lags behind to

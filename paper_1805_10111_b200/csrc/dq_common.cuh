@@ -291,6 +291,7 @@ struct dq_ctx {
     float* rbuf;                // [M][B] slope differences of the sampled rows
     float* fused_part;          // [SMs + M][d] column sums per (block, worker) of the one-pass dense gradient kernel; NULL: not in use
     uint32_t* fused_cnt;        // [M] blocks that have handed in their sums for a worker (zero between launches)
+    uint32_t* fused_done;       // [1] workers whose message is complete, when the kernel carries the whole round
     int32_t* bx_dev;            // model width chosen by condition (3) this round
     // network workload: sampled-row indices and per-row activations / derivatives of the two parameter vectors
     int32_t* mlp_rows; double* mlp_act[2]; float* mlp_dz[2]; float* mlp_dh[2];

@@ -485,17 +485,30 @@ __device__ __forceinline__ float fold8(float (&p)[8], int lane)
 
 // Work split of the fused kernel: worker and first slot of tile t, the run of tiles of block b.
 struct FusedPlan {
-    int M, B, tiles_per_worker, ntiles, nblocks;
-    __host__ __device__ int tile_begin(int b) const { return (int)(((long long)b * ntiles) / nblocks); }
+    int M, B, tiles_per_worker, ntiles, nblocks;              // ntiles * nblocks < 2^32 (checked by the host)
+    __host__ __device__ int tile_begin(int b) const { return (int)(((unsigned)b * (unsigned)ntiles) / (unsigned)nblocks); }
     __host__ __device__ int worker_of(int t) const { return t / tiles_per_worker; }
     // blocks whose runs touch worker w: the owners of its first and last tile
     __host__ __device__ int block_of_tile(int t) const
     {
-        int b = (int)(((long long)t * nblocks) / ntiles);          // tile_begin(b) <= t holds for this b or the next ones
+        int b = (int)(((unsigned)t * (unsigned)nblocks) / (unsigned)ntiles);       // tile_begin(b) <= t holds for this b or the next ones
         while (b + 1 < nblocks && tile_begin(b + 1) <= t) ++b;
         while (tile_begin(b) > t) --b;
         return b;
     }
+};
+
+// The stages next to the gradient, when its kernel carries them (dense messages, fixed model width 2/4/8, no
+// delays).  Prologue: every block quantises the model itself (all blocks draw the same Philox stream, so the
+// broadcast of Algorithm 1 step 8 needs no exchange; block 0 writes the packed model).  Epilogue: the block that
+// completes a worker quantises and packs that worker's message (step 12) while alpha_w is still in its registers.
+// The master step (step 9) needs every message and stays a kernel of its own.  Nobody waits for anybody: counters
+// decide who goes on.
+struct FusedRound {
+    int fold;                                                 // 0: gradient only
+    const float* x; const float* xsnap; const uint32_t* normx_in; uint8_t* codes_x; float* delta_x; int bx;   // model quantiser
+    int b; uint8_t* codes; int64_t stride; float* scale;                                                      // messages
+    uint32_t* normx_out; uint32_t* done;
 };
 
 template <class T, bool MMA>
@@ -504,10 +517,12 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
                          const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, FusedPlan pl,
                          int64_t d, float* __restrict__ alpha, uint32_t* __restrict__ norm_bits,
                          float* __restrict__ part /* [nblocks + M][d] column sums of (block, worker) */,
-                         uint32_t* __restrict__ counters /* [M], zero between launches */, int* __restrict__ status)
+                         uint32_t* __restrict__ counters /* [M], zero between launches */, int* __restrict__ status,
+                         const __grid_constant__ FusedRound fr)
 {
     pdl_prologue();
     clear_word(bs);
+    const uint32_t round = bs.rp ? bs.rp->round : bs.round;
     constexpr int N = RowVec<T>::N;                          // features per 16-byte group
     constexpr int S = kFusedStages, R = kFusedRows, CW = kFusedComputeWarps;
     extern __shared__ __align__(128) unsigned char s_stage[];    // [S][R][row_bytes + pad]
@@ -517,7 +532,8 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
     __shared__ __align__(4) uint16_t s_rsplit[2][3][R];          // MMA: the slopes as three bfloat16 terms (hi + mid + lo = r to 24 bits)
     __shared__ float s_lab[S + 2][R], s_zs[S + 2][R];           // ring of S + 2: tiles it + S and it + S + 1 can be issued while tile it's entries are still read
     __shared__ uint32_t s_max[CW];
-    __shared__ int s_abort, s_last, s_issued;
+    __shared__ int s_abort, s_last, s_issued, s_bfirst, s_blast;
+    __shared__ uint32_t s_norm;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool slope_warp = warp == CW, load_warp = warp == CW + 1, compute = warp < CW;
     const int row_bytes = (int)(d * (int64_t)sizeof(T)), stride = row_bytes + kFusedRowPad;
@@ -552,22 +568,47 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
     // a worker's last tile in this block has been added when the next tile belongs to another worker (or the run ends)
     const auto flush_at = [&](int it) { return it > 0 && worker_at(it) != worker_at(it - 1); };
 
-    // load warp: draw the rows of tile `it` of this block's run and start their copies into stage it % S
-    auto issue = [&](int it) {
-        const int t = t0 + it, stage = it % S, slot = it % (S + 2);
+    // load warp: draw the rows of tile `it` of this block's run and start their copies into stage it % S (returns this
+    // lane's row, or -1), then fetch the rows' labels and snapshot margins and announce the tile
+    int part_w = -1; int64_t part_lo = 0; uint64_t part_cnt = 0;
+    auto issue_rows = [&](int it) -> int64_t {
+        const int t = t0 + it, stage = it % S;
         const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
         const int nvalid = min(R, pl.B - j0);
+        if (w != part_w) {               // the worker's partition of the rows (two 64-bit divisions: once per worker, not per row)
+            part_w = w;
+            part_lo = ((int64_t)w * bs.n) / bs.M; part_cnt = (uint64_t)(((int64_t)(w + 1) * bs.n) / bs.M - part_lo);
+        }
+        int64_t a = -1;
         if (lane < nvalid) {
-            const int64_t a = batch_row(bs, K, w, j0 + lane, pl.B, true);
+            const int j = j0 + lane;
+            const int64_t slot_j = (int64_t)w * pl.B + j;
+            if (bs.rows_in) {
+                a = bs.rows_in[slot_j];
+            } else {                     // the same draw as sample_row
+                uint32_t r4[4];
+                philox4x32_10((uint32_t)(j >> 2), round, (uint32_t)w, kStreamBatch, K, r4);
+                const uint32_t word = (j & 3) == 0 ? r4[0] : (j & 3) == 1 ? r4[1] : (j & 3) == 2 ? r4[2] : r4[3];
+                a = part_lo + (int64_t)(((uint64_t)word * part_cnt) >> 32);
+                if (bs.rows_out) bs.rows_out[slot_j] = (int32_t)a;
+            }
             bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
-            // the row's label and snapshot margin go beside it.  They are stored before this warp's arrival on the stage's
-            // barrier below, so whoever has seen the stage full (and whoever hears from them) sees them too.
-            const float lab = __ldg(labels + a), zs = __ldg(z_snap + a);
-            s_lab[slot][lane] = lab; s_zs[slot][lane] = zs;
         }
         if (MMA && nvalid < R) {         // the tensor-core path multiplies whole tiles: rows past the minibatch's end must read as zeros
             uint4* z = reinterpret_cast<uint4*>(s_stage + ((size_t)stage * R + nvalid) * stride);
             for (int q = lane; q < (R - nvalid) * (stride >> 4); q += 32) z[q] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        return a;
+    };
+    auto issue_labels = [&](int it, int64_t a) {
+        const int t = t0 + it, stage = it % S, slot = it % (S + 2);
+        const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
+        const int nvalid = min(R, pl.B - j0);
+        if (a >= 0) {
+            // the row's label and snapshot margin go beside it.  They are stored before this warp's arrival on the stage's
+            // barrier below, so whoever has seen the stage full (and whoever hears from them) sees them too.
+            const float lab = __ldg(labels + a), zs = __ldg(z_snap + a);
+            s_lab[slot][lane] = lab; s_zs[slot][lane] = zs;
         }
         __syncwarp();
         // the byte count is announced after the copies were started: the phase cannot complete before this arrival
@@ -588,26 +629,39 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
         for (int n = 0; n < N; ++n) acc[n] = 0.0f;
         __threadfence();
         __syncthreads();
-        const int b_first = pl.block_of_tile(w * pl.tiles_per_worker), b_last = pl.block_of_tile((w + 1) * pl.tiles_per_worker - 1);
         if (tid == 0) {
+            const int bf = pl.block_of_tile(w * pl.tiles_per_worker), bl = pl.block_of_tile((w + 1) * pl.tiles_per_worker - 1);
+            s_bfirst = bf; s_blast = bl;
             const uint32_t old = atomicAdd(counters + w, 1u);
-            s_last = old == (uint32_t)(b_last - b_first);
+            s_last = old == (uint32_t)(bl - bf);
             if (s_last) counters[w] = 0u;                    // every block of this worker has added: ready for the next launch
         }
         __syncthreads();
         if (s_last) {                                        // this block completes worker w: slots in block order
+            const int b_first = s_bfirst, b_last = s_blast;
             __threadfence();
             uint32_t nmax = 0;
+            float sum[N];
+#pragma unroll
+            for (int n = 0; n < N; ++n) sum[n] = 0.0f;
             if (active) {
-                float sum[N];
+                constexpr int U = 4;                             // slots fetched together: their loads overlap, the adds keep block order
+                for (int bb0 = b_first; bb0 <= b_last; bb0 += U) {
+                    float4 x4[U][N / 4];
 #pragma unroll
-                for (int n = 0; n < N; ++n) sum[n] = 0.0f;
-                for (int bb = b_first; bb <= b_last; ++bb) {
-                    const float4* src = reinterpret_cast<const float4*>(part + (size_t)(bb + w) * d) + (size_t)v * (N / 4);
+                    for (int u = 0; u < U; ++u) {
+                        const float4* src = reinterpret_cast<const float4*>(part + (size_t)(min(bb0 + u, b_last) + w) * d) + (size_t)v * (N / 4);
 #pragma unroll
-                    for (int q = 0; q < N / 4; ++q) {
-                        const float4 x4 = __ldcg(src + q);
-                        sum[q * 4] += x4.x; sum[q * 4 + 1] += x4.y; sum[q * 4 + 2] += x4.z; sum[q * 4 + 3] += x4.w;
+                        for (int q = 0; q < N / 4; ++q) x4[u][q] = __ldcg(src + q);
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u) {
+                        if (bb0 + u <= b_last) {
+#pragma unroll
+                            for (int q = 0; q < N / 4; ++q) {
+                                sum[q * 4] += x4[u][q].x; sum[q * 4 + 1] += x4[u][q].y; sum[q * 4 + 2] += x4[u][q].z; sum[q * 4 + 3] += x4[u][q].w;
+                            }
+                        }
                     }
                 }
                 float4* out = reinterpret_cast<float4*>(alpha + (size_t)w * d) + (size_t)v * (N / 4);
@@ -622,20 +676,109 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
             if (tid == 0) {
                 uint32_t m = 0;
                 for (int k = 0; k < CW; ++k) m = max(m, s_max[k]);
-                norm_bits[w] = m;
+                norm_bits[w] = m; s_norm = m;
             }
             __syncthreads();
+            if (fr.fold) {
+                // ---- message w: Q_(delta,b) of alpha_w with delta from ||alpha_w||_inf, packed (Algorithm 1 step 12) -------
+                const uint32_t nb = s_norm;
+                const bool ok = nb < 0x7F800000u && nb != 0u;
+                const int L = levels(fr.b);
+                const float inv = ok ? __fdiv_rd((float)L, __uint_as_float(nb)) : 0.0f;
+                if (tid == 0) {
+                    fr.scale[w] = ok ? __fdiv_rn(__uint_as_float(nb), (float)L) : 0.0f;
+                    if (nb >= 0x7F800000u) set_status(status, DQ_ERR_NONFINITE);
+                }
+                const int ngroups = (int)(fr.stride / fr.b);                    // covers the zero padding of the packed message
+                if (compute) {
+                    // a thread holds N consecutive coordinates; a Philox call serves a group of eight
+                    for (int base = 0; base < ngroups; base += (CW * 32 * N) >> 3) {     // the same trip count in every thread (shuffles inside)
+                        const int g = base + ((v * N) >> 3);
+                        uint32_t r4[4], q[8];
+                        philox4x32_10((uint32_t)g, round, (uint32_t)w, kStreamGrad, K, r4);
+                        float a8[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) a8[j] = 0.0f;
+                        if (N == 8) {
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) a8[j] = (active && base == 0) ? sum[j % N] : 0.0f;
+                        } else {                                                    // N == 4: the group's other half sits in the neighbour lane
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const float mine = (active && base == 0) ? sum[j % N] : 0.0f;
+                                const float other = __shfl_xor_sync(0xFFFFFFFFu, mine, 1);
+                                a8[j] = (v & 1) ? other : mine; a8[4 + j] = (v & 1) ? mine : other;
+                            }
+                        }
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) q[j] = nb < 0x7F800000u ? round_fixed<8>(a8[j], inv, half16(r4, j)) : (128u << 16);
+                        if (g < ngroups && (N == 8 || !(v & 1))) {
+                            uint8_t* dst = fr.codes + (size_t)w * fr.stride + (size_t)g * fr.b;
+                            if (fr.b == 8) store_group<8>(dst, pack8<8>(q)); else if (fr.b == 4) store_group<4>(dst, pack8<4>(q)); else store_group<2>(dst, pack8<2>(q));
+                        }
+                    }
+                }
+                // ---- the block that completes the last message clears ||x||_inf for the master kernel's maximum (every block has
+                // long read it: the model was quantised in the prologue) -------------------------------------------------------
+                __threadfence();
+                __syncthreads();
+                if (tid == 0) {
+                    const uint32_t old = atomicAdd(fr.done, 1u);
+                    if (old == (uint32_t)(pl.M - 1)) { *fr.done = 0u; *fr.normx_out = 0u; }
+                }
+            }
+        }
+    };
+
+    // Prologue of a whole round: Q_(delta_x, b_x) of the model for this thread's N coordinates (every block draws the same
+    // codes; block 0 writes the packed model and delta_x), returned as xhat - xsnap.
+    auto model_diff = [&](float (&out)[N]) {
+        const uint32_t nb = *fr.normx_in;
+        const bool ok = nb < 0x7F800000u && nb != 0u;
+        const int L = levels(fr.bx);
+        const float inv = ok ? __fdiv_rd((float)L, __uint_as_float(nb)) : 0.0f;
+        const float delta = ok ? __fdiv_rn(__uint_as_float(nb), (float)L) : 0.0f;
+        if (blk == 0 && tid == 0) { *fr.delta_x = delta; if (nb >= 0x7F800000u) set_status(status, DQ_ERR_NONFINITE); }
+        const int ngroups_x = (int)((((d * fr.bx + 7) / 8 + 15) / 16 * 16) / fr.bx);      // block 0 also writes the padding of the packed model
+        for (int base = 0; base < (blk == 0 ? ngroups_x : 1); base += (CW * 32 * N) >> 3) {
+            const int g = base + ((v * N) >> 3);
+            const int64_t i0 = (int64_t)g << 3;
+            float a8[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a8[j] = (i0 + j < d) ? __ldcg(fr.x + i0 + j) : 0.0f;   // x is rewritten at the end of this launch: no read-only path
+            uint32_t r4[4], q[8];
+            philox4x32_10((uint32_t)g, round, kMaster, kStreamModel, K, r4);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) q[j] = nb < 0x7F800000u ? round_fixed<8>(a8[j], inv, half16(r4, j)) : (128u << 16);
+            if (blk == 0 && g < ngroups_x && (N == 8 || !(v & 1))) {
+                uint8_t* dst = fr.codes_x + (size_t)g * fr.bx;
+                if (fr.bx == 8) store_group<8>(dst, pack8<8>(q)); else if (fr.bx == 4) store_group<4>(dst, pack8<4>(q)); else store_group<2>(dst, pack8<2>(q));
+            }
+            if (base == 0) {
+#pragma unroll
+                for (int n = 0; n < N; ++n) {
+                    const int j = N == 8 ? n : (v & 1) * 4 + n;
+                    const int64_t i = i0 + j;
+                    const float k = (float)((int)((q[j] >> 16) & 0xFFu) - 128);
+                    out[n] = (active && i < d) ? __fsub_rn(__fmul_rn(k, delta), __ldg(fr.xsnap + i)) : 0.0f;
+                }
+            }
         }
     };
 
     if (load_warp) {
         // ---- copies: S tiles ahead; a stage is refilled once every compute warp has taken its groups out of it -------
-        for (int it = 0; it < min(S, ntl); ++it) issue(it);
+        int64_t a0[S];
+#pragma unroll
+        for (int k = 0; k < S; ++k) a0[k] = k < ntl ? issue_rows(k) : -1;      // all row copies of the first tiles first,
+#pragma unroll
+        for (int k = 0; k < S; ++k) if (k < ntl) issue_labels(k, a0[k]);        // then the small loads that would hold them up
         for (int it = 0; it <= ntl; ++it) {
             if (flush_at(it)) flush(worker_at(it - 1));
             if (it + S < ntl) {
                 wait(&s_empty[it % S], (uint32_t)((it / S) & 1));
-                issue(it + S);
+                const int64_t a = issue_rows(it + S);
+                issue_labels(it + S, a);
             }
         }
     } else if (slope_warp) {
@@ -691,11 +834,27 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
         for (int i = 0; i < kFusedMaxRowBytes / 2 / 16 / CW; ++i) { cacc[i][0] = cacc[i][1] = cacc[i][2] = cacc[i][3] = 0.0f; }
         int w_prev = -1;
         const uint32_t lane_row_off = (uint32_t)((lane & 7) * stride + ((lane >> 3) & 1) * 16);   // ldmatrix: lanes 0-7 first matrix, 8-15 second
+        if (fr.fold) {                                       // the model's xhat - xsnap, formed here, as hi + mid + lo
+            float df[N];
+            model_diff(df);
+            if (active) {
+#pragma unroll
+                for (int n = 0; n < N; ++n) {
+                    const int64_t i = (int64_t)v * N + n;
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(df[n]);
+                    const float r1 = df[n] - __bfloat162float(hi);
+                    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                    s_dsplit[i] = __bfloat16_as_ushort(hi); s_dsplit[d + i] = __bfloat16_as_ushort(mid); s_dsplit[2 * d + i] = __bfloat16_as_ushort(lo);
+                }
+            }
+            asm volatile("bar.sync 1, %0;" :: "n"(CW * 32) : "memory");
+        }
         for (int it = 0; it <= ntl; ++it) {
             const int par = it & 1, stage = it % S;
             const int w_cur = worker_at(it);
             if (it < ntl) {
-                if (w_cur != w_prev) {                       // new worker: its xhat - xsnap as hi + mid + lo
+                if (!fr.fold && w_cur != w_prev) {           // new worker: its xhat - xsnap as hi + mid + lo
                     asm volatile("bar.sync 1, %0;" :: "n"(CW * 32) : "memory");      // every compute warp is done with the old terms
                     const float* dv = diff_of_worker(bs, diff, w_cur);
                     for (int64_t i = tid; i < d; i += CW * 32) {
@@ -769,6 +928,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
         float dreg[N];
 #pragma unroll
         for (int n = 0; n < N; ++n) dreg[n] = 0.0f;
+        if (fr.fold) model_diff(dreg);                       // the model's xhat - xsnap, formed here
         uint4 q_old[R], q_new[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) q_old[r] = q_new[r] = make_uint4(0u, 0u, 0u, 0u);
@@ -780,7 +940,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
             const int nvalid = it < ntl ? min(R, pl.B - j0) : 0;
             if (it < ntl) {
                 // front: margins of tile it
-                if (w_cur != w_prev && active) {             // this worker's xhat - xsnap (a lagging worker reads an older one)
+                if (!fr.fold && w_cur != w_prev && active) {   // this worker's xhat - xsnap (a lagging worker reads an older one)
                     const float4* dv = reinterpret_cast<const float4*>(diff_of_worker(bs, diff, w_cur)) + (size_t)v * (N / 4);
 #pragma unroll
                     for (int q = 0; q < N / 4; ++q) { const float4 x4 = __ldg(dv + q); dreg[q * 4] = x4.x; dreg[q * 4 + 1] = x4.y; dreg[q * 4 + 2] = x4.z; dreg[q * 4 + 3] = x4.w; }
@@ -1586,8 +1746,8 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
 
 // The one-pass kernel takes dense rows of at most kFusedMaxRowBytes on the 16-byte grid; the context then owns its
 // scratch (column sums per (block, worker), per-worker counters).
-// bfloat16 rows whose length is a multiple of 16 take the tensor-core variant (no_fused = 2 keeps the CUDA-core one)
-static bool fused_grad_mma(const dq_ctx* ctx) { return ctx->data.format == DQ_DENSE_BF16 && (ctx->cfg.d & 15) == 0 && ctx->cfg.no_fused != 2; }
+// bfloat16 rows whose length is a multiple of 16 can take the tensor-core variant (cfg.tensor_cores)
+static bool fused_grad_mma(const dq_ctx* ctx) { return ctx->data.format == DQ_DENSE_BF16 && (ctx->cfg.d & 15) == 0 && ctx->cfg.tensor_cores != 0; }
 static size_t fused_grad_smem(const dq_ctx* ctx)
 {
     const size_t row_bytes = (size_t)ctx->cfg.d * (ctx->data.format == DQ_DENSE_F32 ? 4 : 2);
@@ -1595,12 +1755,59 @@ static size_t fused_grad_smem(const dq_ctx* ctx)
 }
 bool fused_grad_applies(const dq_ctx* ctx) { return ctx->fused_part != nullptr && ctx->cfg.no_fused != 1; }
 typedef void (*FusedKernelF32)(const float*, const float*, const float*, const float*, const PhiloxKeys, BatchSource, FusedPlan, int64_t,
-                               float*, uint32_t*, float*, uint32_t*, int*);
+                               float*, uint32_t*, float*, uint32_t*, int*, const FusedRound);
 typedef void (*FusedKernelBf16)(const __nv_bfloat16*, const float*, const float*, const float*, const PhiloxKeys, BatchSource, FusedPlan,
-                                int64_t, float*, uint32_t*, float*, uint32_t*, int*);
+                                int64_t, float*, uint32_t*, float*, uint32_t*, int*, const FusedRound);
 static FusedKernelBf16 fused_kernel_bf16(const dq_ctx* ctx)
 {
     return fused_grad_mma(ctx) ? worker_grad_fused_kernel<__nv_bfloat16, true> : worker_grad_fused_kernel<__nv_bfloat16, false>;
+}
+
+static FusedPlan fused_plan(const dq_ctx* ctx)
+{
+    const dq_config& c = ctx->cfg;
+    FusedPlan pl;
+    pl.M = c.M; pl.B = c.B; pl.tiles_per_worker = (c.B + kFusedRows - 1) / kFusedRows;
+    pl.ntiles = c.M * pl.tiles_per_worker; pl.nblocks = pl.ntiles < ctx->sm_count ? pl.ntiles : ctx->sm_count;
+    return pl;
+}
+
+static void launch_fused(dq_ctx* ctx, const BatchSource& bs, const dq_state* s, float* alpha, uint32_t* nb, const FusedRound& fr, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    const FusedPlan pl = fused_plan(ctx);
+    const size_t smem = fused_grad_smem(ctx);
+    if (D.format == DQ_DENSE_F32)
+        launch_k(worker_grad_fused_kernel<float, false>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
+                 s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status, fr);
+    else
+        launch_k(fused_kernel_bf16(ctx), pl.nblocks, kFusedThreads, smem, st, (const __nv_bfloat16*)D.values, D.labels,
+                 ctx->xhat_diff, s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status, fr);
+    ctx->launches += 1;
+}
+
+// Model quantiser and message quantiser inside the gradient kernel: dense rows that take the one-pass kernel, dense
+// messages, a fixed model width of 2, 4 or 8 bits, no lagging workers.  (The master step follows as its own kernel.)
+bool fused_round_applies(const dq_ctx* ctx)
+{
+    const dq_config& c = ctx->cfg;
+    if (!ctx->fused_part || c.no_fused || c.sparsify || c.mu > 0.0f || c.max_delay > 0 || c.B < 64) return false;
+    if (c.bx != 2 && c.bx != 4 && c.bx != 8) return false;
+    const int64_t elt = ctx->data.format == DQ_DENSE_F32 ? 4 : 8;
+    return (c.d % elt) == 0;
+}
+
+void launch_fused_round(dq_ctx* ctx, dq_state* s, uint32_t round, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg; const dq_data& D = ctx->data;
+    const BatchSource bs = {nullptr, ctx->rows, round, ctx->rp_active, c.M, D.n, nullptr, nullptr, c.d};
+    FusedRound fr = {};
+    fr.fold = 1;
+    fr.normx_in = reinterpret_cast<const uint32_t*>(s->norm_x); fr.codes_x = ctx->codes_x; fr.delta_x = ctx->delta_x; fr.bx = c.bx;
+    fr.b = c.b; fr.codes = ctx->msgs.codes; fr.stride = ctx->msgs.stride; fr.scale = ctx->msgs.scale;
+    fr.x = s->x; fr.xsnap = s->x_snap;
+    fr.normx_out = reinterpret_cast<uint32_t*>(s->norm_x); fr.done = ctx->fused_done;
+    launch_fused(ctx, bs, s, ctx->alpha, reinterpret_cast<uint32_t*>(ctx->ninf), fr, st);
 }
 
 // Called once per context: scratch and the shared-memory opt-in of the one-pass dense gradient kernel.
@@ -1610,6 +1817,7 @@ int fused_grad_setup(dq_ctx* ctx)
     if (!ctx->has_data || c.model != DQ_MODEL_LOGISTIC || (D.format != DQ_DENSE_F32 && D.format != DQ_DENSE_BF16)) return DQ_OK;
     const size_t row_bytes = (size_t)c.d * (D.format == DQ_DENSE_F32 ? 4 : 2);
     if (row_bytes > kFusedMaxRowBytes || (row_bytes & 15) || c.B < 64) return DQ_OK;
+    if ((int64_t)c.M * ((c.B + kFusedRows - 1) / kFusedRows) > ((int64_t)1 << 24)) return DQ_OK;    // the tile arithmetic is 32-bit
     const int smem = (int)fused_grad_smem(ctx);
     const FusedKernelF32 kf = worker_grad_fused_kernel<float, false>;
     const FusedKernelBf16 kb = fused_kernel_bf16(ctx);
@@ -1621,8 +1829,9 @@ int fused_grad_setup(dq_ctx* ctx)
                                                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, kb, kFusedThreads, (size_t)smem);
     if (o != cudaSuccess || resident < 1) { cudaGetLastError(); return DQ_OK; }
     if (cudaMalloc(reinterpret_cast<void**>(&ctx->fused_part), sizeof(float) * (size_t)(ctx->sm_count + c.M) * c.d) != cudaSuccess ||
-        cudaMalloc(reinterpret_cast<void**>(&ctx->fused_cnt), sizeof(uint32_t) * c.M) != cudaSuccess ||
-        cudaMemset(ctx->fused_cnt, 0, sizeof(uint32_t) * c.M) != cudaSuccess) return DQ_ERR_CUDA;
+        cudaMalloc(reinterpret_cast<void**>(&ctx->fused_cnt), sizeof(uint32_t) * (c.M + 1)) != cudaSuccess ||
+        cudaMemset(ctx->fused_cnt, 0, sizeof(uint32_t) * (c.M + 1)) != cudaSuccess) return DQ_ERR_CUDA;
+    ctx->fused_done = ctx->fused_cnt + c.M;
     return DQ_OK;
 }
 
@@ -1676,18 +1885,8 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         const bool f32 = D.format == DQ_DENSE_F32;
         const bool vec = (c.d % (f32 ? 4 : 8)) == 0 && (reinterpret_cast<uintptr_t>(alpha) & 15) == 0;   // data is 16-byte aligned by contract
         if (vec && c.B >= 64 && fused_grad_applies(ctx)) {      // large minibatch, rows that fit a stage: one pass over the rows
-            FusedPlan pl;
-            pl.M = c.M; pl.B = c.B; pl.tiles_per_worker = (c.B + kFusedRows - 1) / kFusedRows;
-            pl.ntiles = c.M * pl.tiles_per_worker; pl.nblocks = pl.ntiles < ctx->sm_count ? pl.ntiles : ctx->sm_count;
-            const size_t smem = fused_grad_smem(ctx);
-            uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
-            if (f32)
-                launch_k(worker_grad_fused_kernel<float, false>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
-                         s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status);
-            else
-                launch_k(fused_kernel_bf16(ctx), pl.nblocks, kFusedThreads, smem, st, (const __nv_bfloat16*)D.values, D.labels,
-                         ctx->xhat_diff, s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status);
-            ctx->launches += 1;
+            FusedRound fr = {};                                   // the gradient stage alone
+            launch_fused(ctx, bs, s, alpha, reinterpret_cast<uint32_t*>(norm_inf), fr, st);
             return;
         }
         if (vec && c.B >= 64) {        // large minibatch, long rows: margins, then atomics-free column sums with the norm folded in

@@ -32,6 +32,8 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
 bool worker_accumulates(const dq_ctx* ctx);
 int fused_grad_setup(dq_ctx* ctx);
 bool fused_grad_applies(const dq_ctx* ctx);
+bool fused_round_applies(const dq_ctx* ctx);
+void launch_fused_round(dq_ctx* ctx, dq_state* s, uint32_t round, cudaStream_t st);
 void small_round_setup(dq_ctx* ctx);
 void launch_set_slots(dq_ctx* ctx, int round_in_epoch, cudaStream_t st);
 void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds, float eta, float theta, uint64_t* bits_down,

@@ -207,18 +207,18 @@ def test_worker_gradient(dq, name, bx):
     dq.dq_destroy(ctx)
 
 
-@pytest.mark.parametrize("name,M,B,no_fused", [("bf16", 2, 70, 0), ("dense8", 2, 70, 0), ("bf16x16", 3, 70, 0), ("bf16x16", 5, 264, 0),
-                                               ("bf16x16", 3, 70, 2), ("bf16x16", 2, 70, 1), ("dense_wide", 2, 70, 0)])
-def test_worker_gradient_large_minibatch(dq, name, M, B, no_fused):
-    """B >= 64 takes the one-pass dense kernel (rows staged once; bf16 rows on the 16-column grid by tensor-core MMAs,
-    no_fused = 2: by CUDA cores) or, for rows too long to stage or with no_fused = 1, margins then column sums in two
+@pytest.mark.parametrize("name,M,B,no_fused,tc", [("bf16", 2, 70, 0, 0), ("dense8", 2, 70, 0, 0), ("bf16x16", 3, 70, 0, 1), ("bf16x16", 5, 264, 0, 1),
+                                                  ("bf16x16", 3, 70, 0, 0), ("bf16x16", 2, 70, 1, 0), ("dense_wide", 2, 70, 0, 0)])
+def test_worker_gradient_large_minibatch(dq, name, M, B, no_fused, tc):
+    """B >= 64 takes the one-pass dense kernel (rows staged once; with tensor_cores = 1, bf16 rows on the 16-column grid by
+    MMAs, else by CUDA cores) or, for rows too long to stage or with no_fused = 1, margins then column sums in two
     kernels.  No atomics anywhere: reproducible bit for bit.  B = 70 ends on a tile of 6 rows."""
     import torch
     h = _problem(name)
     seed, rnd, bx = 31, 8, 8
     xs = synth.normal_vector(h.d, 76, 0.3)
     x = (xs + synth.normal_vector(h.d, 77, 0.02)).astype(F32)
-    cfg = dq.make_config(h.d, M, B=B, bx=bx, seed=seed, no_fused=no_fused)
+    cfg = dq.make_config(h.d, M, B=B, bx=bx, seed=seed, no_fused=no_fused, tensor_cores=tc)
     data = dq.Data(h)
     rc, ctx = dq.dq_create(cfg, data); assert rc == 0
     st = dq.State(xs, n=h.n)
@@ -252,6 +252,9 @@ def test_worker_gradient_large_minibatch(dq, name, M, B, no_fused):
     ("csr", dict(M=5, B=33, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=62)),       # touched-group list
     ("dense", dict(M=3, B=37, bx=8, b=8, lambda1=1e-4, seed=63, no_fused=1)),                            # three chunks of rows per worker
     ("bf16", dict(M=3, B=50, bx=8, b=8, box_lo=-1.0, box_hi=1.0, seed=64)),
+    ("bf16", dict(M=5, B=70, bx=8, b=4, box_lo=-1.0, box_hi=1.0, seed=65)),                              # whole round in the one-pass kernel, CUDA cores
+    ("bf16x16", dict(M=7, B=100, bx=4, b=2, lambda1=1e-5, seed=66, tensor_cores=1)),                     # the same on tensor cores
+    ("dense8", dict(M=4, B=64, bx=2, b=8, lambda2=1e-4, seed=67)),                                       # fp32 rows
 ])
 def test_same_round_twice_gives_the_same_bytes(dq, name, kw):
     """Equal (seed, round, state) must give equal bytes: the same rounds run twice from the same state leave identical
@@ -344,7 +347,7 @@ class Lockstep:
                    msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"],
                    mu=kw.get("mu", 0.0), sequential=kw.get("sequential", 0), model=kw.get("model", 0),
                    hidden=kw.get("hidden", 0), classes=kw.get("classes", 0))
-        assert not (set(kw) - {"M", "B", "bx", "b", "lambda1", "lambda2", "box_lo", "box_hi", "no_fused", "no_graph", "max_delay"} - set(okw)), kw
+        assert not (set(kw) - {"M", "B", "bx", "b", "lambda1", "lambda2", "box_lo", "box_hi", "no_fused", "no_graph", "max_delay", "tensor_cores"} - set(okw)), kw
         d = x0.size                                        # parameters (equals the feature count for logistic regression)
         self.cfg = dq.make_config(d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
         self.ocfg = oracle.make_config(d, kw["M"], kw["B"], kw["bx"], kw["b"], **okw)
@@ -522,6 +525,11 @@ class Lockstep:
     ("dense", dict(M=3, B=8, bx=5, b=8, lambda1=1e-4, seed=11), 0.5),
     ("csr", dict(M=4, B=16, bx=11, b=4, lambda2=1e-5, seed=12), 0.5),
     ("bf16", dict(M=4, B=16, bx=3, b=8, box_lo=-1.0, box_hi=1.0, seed=13), 0.01),
+    # large minibatches: the whole round runs in the one-pass gradient kernel (fp32 rows; bf16 rows by CUDA cores and by tensor cores)
+    ("dense8", dict(M=5, B=64, bx=8, b=4, lambda1=1e-4, seed=56), 0.5),
+    ("bf16", dict(M=4, B=70, bx=4, b=8, box_lo=-1.0, box_hi=1.0, seed=57), 0.01),
+    ("bf16x16", dict(M=6, B=100, bx=8, b=2, lambda2=1e-4, seed=58, tensor_cores=1), 0.01),
+    ("bf16x16", dict(M=3, B=64, bx=2, b=4, box_lo=-0.5, box_hi=0.5, seed=59), 0.01),
     # one row per minibatch and a coarse model: a worker's whole gradient hangs on one margin difference
     ("dense_wide", dict(M=16, B=1, bx=3, b=8, box_lo=-0.5, box_hi=2.0, seed=46, no_fused=1), 0.3),
     ("csr", dict(M=16, B=1, bx=3, b=4, box_lo=-0.5, box_hi=0.5, seed=47), 0.3),
@@ -782,7 +790,7 @@ def _full_config(name):
 
 
 @pytest.mark.parametrize("name,rounds,no_fused", [("c1", 100, 0), ("c2", 100, 0), ("c1", 30, 1), ("c2", 30, 1), ("c3", 100, 0), ("c4", 100, 0),
-                                                  ("c4", 20, 1), ("c4", 20, 2)])
+                                                  ("c4", 20, 1), ("c4", 20, 2), ("c4", 20, 3)])
 def test_lockstep_full_configs(dq, name, rounds, no_fused):
     """The benchmark configurations at their full model width for 100 rounds (c3, c4 with fewer rows so that the oracle
     finishes in seconds per round; the width, the workers and the minibatches are the full ones); c4 reads "momentum 0.9"
@@ -790,7 +798,7 @@ def test_lockstep_full_configs(dq, name, rounds, no_fused):
     kernels."""
     h = _problem(name)
     kw, lr, m = _full_config(name)
-    kw = dict(kw, no_fused=no_fused)
+    kw = dict(kw, no_fused=no_fused) if no_fused < 3 else dict(kw, tensor_cores=1)      # 3: the default plan with the tensor-core gradient
     ls = Lockstep(dq, h, np.zeros(h.d, F32) if name != "c4" else synth.normal_vector(h.d, 75, 0.01), **kw)
     theta = F32(0.1) if name == "c4" else F32(0.0)
     eta = F32(lr) / theta if name == "c4" else F32(lr)
