@@ -61,6 +61,9 @@ def parse_args():
     ap.add_argument("--sweep", action="store_true", help="print only the c5 grid (adds d = 2^20) as one JSON object")
     ap.add_argument("--only-training", action="store_true", help="time only the training configurations of --configs (one JSON object)")
     ap.add_argument("--train-rounds", type=int, default=200, help="rounds timed per training configuration")
+    ap.add_argument("--tensor-cores", type=int, default=0, help="training configurations: dq_config.tensor_cores (1: both products of the "
+                                                                "dense bf16 gradient as MMAs, 2: the margins only)")
+    ap.add_argument("--no-fused", type=int, default=0, help="training configurations: dq_config.no_fused")
     ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_rounds ('' for none)")
     return ap.parse_args()
 
@@ -332,7 +335,7 @@ def time_training_stages(dq, ctx, cfg, h, st, eta, theta, peak, reps=60):
     return out
 
 
-def time_training_config(name, rounds=200, warmup=20, with_oracle=False, peak=None):
+def time_training_config(name, rounds=200, warmup=20, with_oracle=False, peak=None, extra=None):
     """rounds/s of dq_rounds on one of the training configurations (full size, synthetic data), the stages one by one,
     and the bits the paper's accounting charges per round."""
     import numpy as np
@@ -343,7 +346,7 @@ def time_training_config(name, rounds=200, warmup=20, with_oracle=False, peak=No
     h = getattr(synth, spec["gen"])()
     is_nn = spec["kw"].get("model", 0) == 1
     x0 = synth.mlp_init(h.d, spec["kw"]["hidden"], spec["kw"]["classes"], 9) if is_nn else np.zeros(h.d, np.float32)
-    cfg = dq.make_config(x0.size, spec["kw"]["M"], seed=SEED, **{k: v for k, v in spec["kw"].items() if k != "M"})
+    cfg = dq.make_config(x0.size, spec["kw"]["M"], seed=SEED, **{k: v for k, v in spec["kw"].items() if k != "M"}, **(extra or {}))
     data = dq.Data(h)
     rc, ctx = dq.dq_create(cfg, data); dq.ok(rc, "dq_create " + name)
     st = dq.State(x0, n=h.n, accelerated=bool(cfg.accelerated))
@@ -694,7 +697,9 @@ def run_training_only(a):
     torch.cuda.set_device(0)
     dq.lib()
     peak, _ = measured_peak()
-    print(json.dumps({"training_configs": {c: time_training_config(c, rounds=a.train_rounds, with_oracle=not a.no_cpu_baseline, peak=peak)
+    extra = {"tensor_cores": a.tensor_cores, "no_fused": a.no_fused}
+    print(json.dumps({"dq_config": extra,
+                      "training_configs": {c: time_training_config(c, rounds=a.train_rounds, with_oracle=not a.no_cpu_baseline, peak=peak, extra=extra)
                                            for c in a.configs.split(",") if c in TRAIN_CONFIGS}}))
 
 

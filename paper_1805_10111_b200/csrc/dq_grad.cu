@@ -511,7 +511,10 @@ struct FusedRound {
     uint32_t* normx_out; uint32_t* done;
 };
 
-template <class T, bool MMA>
+// MODE 0: both products by fp32 FMAs on CUDA cores (any row type).  MODE 1: both products of bfloat16 rows as
+// tensor-core MMAs.  MODE 2: the margins X (xhat - xsnap) as MMAs straight from the stage, the column sums X^T r
+// by FMAs from the registers that keep the tile (so a stage is free again as soon as the margins are formed).
+template <class T, int MODE>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labels, const float* __restrict__ diff,
                          const float* __restrict__ z_snap, const __grid_constant__ PhiloxKeys K, BatchSource bs, FusedPlan pl,
@@ -525,6 +528,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
     const uint32_t round = bs.rp ? bs.rp->round : bs.round;
     constexpr int N = RowVec<T>::N;                          // features per 16-byte group
     constexpr int S = kFusedStages, R = kFusedRows, CW = kFusedComputeWarps;
+    constexpr bool MMA = MODE == 1, MMA_FRONT = MODE != 0;
     extern __shared__ __align__(128) unsigned char s_stage[];    // [S][R][row_bytes + pad]
     __shared__ __align__(8) uint64_t s_full[S], s_empty[S], s_pready[2], s_rready[2];
     __shared__ float s_part[2][CW][R];
@@ -594,7 +598,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
             }
             bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
         }
-        if (MMA && nvalid < R) {         // the tensor-core path multiplies whole tiles: rows past the minibatch's end must read as zeros
+        if (MMA_FRONT && nvalid < R) {   // the tensor-core paths multiply whole tiles: rows past the minibatch's end must read as zeros
             uint4* z = reinterpret_cast<uint4*>(s_stage + ((size_t)stage * R + nvalid) * stride);
             for (int q = lane; q < (R - nvalid) * (stride >> 4); q += 32) z[q] = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -743,9 +747,14 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
         for (int base = 0; base < (blk == 0 ? ngroups_x : 1); base += (CW * 32 * N) >> 3) {
             const int g = base + ((v * N) >> 3);
             const int64_t i0 = (int64_t)g << 3;
-            float a8[8];
+            float a8[8], xs8[N];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) a8[j] = (i0 + j < d) ? __ldcg(fr.x + i0 + j) : 0.0f;   // x is rewritten at the end of this launch: no read-only path
+            for (int j = 0; j < 8; ++j) a8[j] = (i0 + j < d) ? __ldcg(fr.x + i0 + j) : 0.0f;
+#pragma unroll
+            for (int n = 0; n < N; ++n) {                    // the snapshot's coordinates travel together with the model's
+                const int64_t i = i0 + (N == 8 ? n : (v & 1) * 4 + n);
+                xs8[n] = (base == 0 && active && i < d) ? __ldg(fr.xsnap + i) : 0.0f;
+            }
             uint32_t r4[4], q[8];
             philox4x32_10((uint32_t)g, round, kMaster, kStreamModel, K, r4);
 #pragma unroll
@@ -760,7 +769,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
                     const int j = N == 8 ? n : (v & 1) * 4 + n;
                     const int64_t i = i0 + j;
                     const float k = (float)((int)((q[j] >> 16) & 0xFFu) - 128);
-                    out[n] = (active && i < d) ? __fsub_rn(__fmul_rn(k, delta), __ldg(fr.xsnap + i)) : 0.0f;
+                    out[n] = (active && i < d) ? __fsub_rn(__fmul_rn(k, delta), xs8[n]) : 0.0f;
                 }
             }
         }
@@ -929,6 +938,25 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
 #pragma unroll
         for (int n = 0; n < N; ++n) dreg[n] = 0.0f;
         if (fr.fold) model_diff(dreg);                       // the model's xhat - xsnap, formed here
+        const int g = lane >> 2, c2 = (lane & 3) * 2;        // MMA_FRONT: this lane's row of A / pair of columns of D
+        const int ksteps = (int)(d >> 4), kpw = (ksteps + CW - 1) / CW;
+        const int k_first = warp * kpw, k_count = max(0, min(kpw, ksteps - k_first));
+        const uint32_t lane_row_off = (uint32_t)((lane & 7) * stride + ((lane >> 3) & 1) * 16);
+        auto split_to_smem = [&](const float (&df)[N]) {     // this thread's N coordinates of xhat - xsnap as hi + mid + lo
+            if (active) {
+#pragma unroll
+                for (int n = 0; n < N; ++n) {
+                    const int64_t i = (int64_t)v * N + n;
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(df[n]);
+                    const float r1 = df[n] - __bfloat162float(hi);
+                    const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+                    const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+                    s_dsplit[i] = __bfloat16_as_ushort(hi); s_dsplit[d + i] = __bfloat16_as_ushort(mid); s_dsplit[2 * d + i] = __bfloat16_as_ushort(lo);
+                }
+            }
+            asm volatile("bar.sync 1, %0;" :: "n"(CW * 32) : "memory");
+        };
+        if (MMA_FRONT && fr.fold) split_to_smem(dreg);
         uint4 q_old[R], q_new[R];
 #pragma unroll
         for (int r = 0; r < R; ++r) q_old[r] = q_new[r] = make_uint4(0u, 0u, 0u, 0u);
@@ -940,31 +968,64 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
             const int nvalid = it < ntl ? min(R, pl.B - j0) : 0;
             if (it < ntl) {
                 // front: margins of tile it
-                if (!fr.fold && w_cur != w_prev && active) {   // this worker's xhat - xsnap (a lagging worker reads an older one)
-                    const float4* dv = reinterpret_cast<const float4*>(diff_of_worker(bs, diff, w_cur)) + (size_t)v * (N / 4);
+                if (!fr.fold && w_cur != w_prev) {             // this worker's xhat - xsnap (a lagging worker reads an older one)
+                    if (MMA_FRONT) asm volatile("bar.sync 1, %0;" :: "n"(CW * 32) : "memory");    // every compute warp is done with the old terms
+                    if (active) {
+                        const float4* dv = reinterpret_cast<const float4*>(diff_of_worker(bs, diff, w_cur)) + (size_t)v * (N / 4);
 #pragma unroll
-                    for (int q = 0; q < N / 4; ++q) { const float4 x4 = __ldg(dv + q); dreg[q * 4] = x4.x; dreg[q * 4 + 1] = x4.y; dreg[q * 4 + 2] = x4.z; dreg[q * 4 + 3] = x4.w; }
+                        for (int q = 0; q < N / 4; ++q) { const float4 x4 = __ldg(dv + q); dreg[q * 4] = x4.x; dreg[q * 4 + 1] = x4.y; dreg[q * 4 + 2] = x4.z; dreg[q * 4 + 3] = x4.w; }
+                    }
+                    if (MMA_FRONT) split_to_smem(dreg);
                 }
                 wait(&s_full[stage], (uint32_t)((it / S) & 1));
                 const unsigned char* base = s_stage + (size_t)stage * R * stride + (size_t)v * 16;
+                if (nvalid == R && active) {
 #pragma unroll
-                for (int r = 0; r < R; ++r)
-                    q_new[r] = (active && r < nvalid) ? *reinterpret_cast<const uint4*>(base + (size_t)r * stride) : make_uint4(0u, 0u, 0u, 0u);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&s_empty[stage]);     // this warp's groups are in registers: the stage may be refilled
-                float p[R];
+                    for (int r = 0; r < R; ++r) q_new[r] = *reinterpret_cast<const uint4*>(base + (size_t)r * stride);
+                } else {
 #pragma unroll
-                for (int r = 0; r < R; ++r) {
-                    float f[N];
-                    RowVec<T>::unpack(q_new[r], f);
-                    float s = 0.0f;
-#pragma unroll
-                    for (int n = 0; n < N; ++n) s = fmaf(f[n], dreg[n], s);
-                    p[r] = s;
+                    for (int r = 0; r < R; ++r)
+                        q_new[r] = (active && r < nvalid) ? *reinterpret_cast<const uint4*>(base + (size_t)r * stride) : make_uint4(0u, 0u, 0u, 0u);
                 }
-                if (it >= 2) wait(&s_rready[par], (uint32_t)(((it - 2) >> 1) & 1));      // the slopes of tile it - 2 have been formed: its partial sums are free
-                const float folded = fold8(p, lane);
-                if ((lane & 3) == 0) s_part[par][warp][((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = folded;
+                if (!MMA_FRONT) {
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s_empty[stage]);     // this warp's groups are in registers: the stage may be refilled
+                    float p[R];
+#pragma unroll
+                    for (int r = 0; r < R; ++r) {
+                        float f[N];
+                        RowVec<T>::unpack(q_new[r], f);
+                        float s = 0.0f;
+#pragma unroll
+                        for (int n = 0; n < N; ++n) s = fmaf(f[n], dreg[n], s);
+                        p[r] = s;
+                    }
+                    if (it >= 2) wait(&s_rready[par], (uint32_t)(((it - 2) >> 1) & 1));      // the slopes of tile it - 2 have been formed: its partial sums are free
+                    const float folded = fold8(p, lane);
+                    if ((lane & 3) == 0) s_part[par][warp][((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1)] = folded;
+                } else {
+                    // margins by MMA from the stage: D[term][row] += sum_k diff_term[k] X[row][k] over this warp's columns
+                    const uint32_t sbase = smem_u32(s_stage + (size_t)stage * R * stride) + lane_row_off;
+                    float c0 = 0.0f, c1 = 0.0f, c2r = 0.0f, c3 = 0.0f;
+#pragma unroll 4
+                    for (int ks = 0; ks < k_count; ++ks) {
+                        const int col = (k_first + ks) << 4;
+                        uint32_t a0 = 0u, a2 = 0u, b0, b1;
+                        if (g < 3) {
+                            const uint16_t* dp = s_dsplit + (size_t)g * d + col + c2;
+                            a0 = *reinterpret_cast<const uint32_t*>(dp); a2 = *reinterpret_cast<const uint32_t*>(dp + 8);
+                        }
+                        asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(b0), "=r"(b1) : "r"(sbase + (uint32_t)col * 2u));
+                        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                                     : "+f"(c0), "+f"(c1), "+f"(c2r), "+f"(c3) : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&s_empty[stage]);     // the margins are formed and the groups are in registers
+#pragma unroll
+                    for (int o = 4; o < 32; o <<= 1) { c0 += __shfl_xor_sync(0xFFFFFFFFu, c0, o); c1 += __shfl_xor_sync(0xFFFFFFFFu, c1, o); }
+                    if (it >= 2) wait(&s_rready[par], (uint32_t)(((it - 2) >> 1) & 1));
+                    if (lane < 4) { s_part[par][warp][c2] = c0; s_part[par][warp][c2 + 1] = c1; }
+                }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&s_pready[par]);
             }
@@ -973,7 +1034,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
                 wait(&s_rready[par ^ 1], (uint32_t)(((it - 1) >> 1) & 1));
 #pragma unroll
                 for (int r = 0; r < R; ++r) {
-                    if (r < nvalid_prev) {
+                    if (r < nvalid_prev) {                   // (rows past the end were loaded as zeros, but their slot of s_r is stale)
                         const float rr = s_r[par ^ 1][r];
                         float f[N];
                         RowVec<T>::unpack(q_old[r], f);
@@ -1746,8 +1807,13 @@ void launch_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, cudaStream_t st)
 
 // The one-pass kernel takes dense rows of at most kFusedMaxRowBytes on the 16-byte grid; the context then owns its
 // scratch (column sums per (block, worker), per-worker counters).
-// bfloat16 rows whose length is a multiple of 16 can take the tensor-core variant (cfg.tensor_cores)
-static bool fused_grad_mma(const dq_ctx* ctx) { return ctx->data.format == DQ_DENSE_BF16 && (ctx->cfg.d & 15) == 0 && ctx->cfg.tensor_cores != 0; }
+// bfloat16 rows whose length is a multiple of 16 can take a tensor-core variant (cfg.tensor_cores: 1 both products, 2 the margins)
+static int fused_grad_mode(const dq_ctx* ctx)
+{
+    if (ctx->data.format != DQ_DENSE_BF16 || (ctx->cfg.d & 15) != 0) return 0;
+    return ctx->cfg.tensor_cores == 1 ? 1 : ctx->cfg.tensor_cores == 2 ? 2 : 0;
+}
+static bool fused_grad_mma(const dq_ctx* ctx) { return fused_grad_mode(ctx) != 0; }
 static size_t fused_grad_smem(const dq_ctx* ctx)
 {
     const size_t row_bytes = (size_t)ctx->cfg.d * (ctx->data.format == DQ_DENSE_F32 ? 4 : 2);
@@ -1760,7 +1826,8 @@ typedef void (*FusedKernelBf16)(const __nv_bfloat16*, const float*, const float*
                                 int64_t, float*, uint32_t*, float*, uint32_t*, int*, const FusedRound);
 static FusedKernelBf16 fused_kernel_bf16(const dq_ctx* ctx)
 {
-    return fused_grad_mma(ctx) ? worker_grad_fused_kernel<__nv_bfloat16, true> : worker_grad_fused_kernel<__nv_bfloat16, false>;
+    const int mode = fused_grad_mode(ctx);
+    return mode == 1 ? worker_grad_fused_kernel<__nv_bfloat16, 1> : mode == 2 ? worker_grad_fused_kernel<__nv_bfloat16, 2> : worker_grad_fused_kernel<__nv_bfloat16, 0>;
 }
 
 static FusedPlan fused_plan(const dq_ctx* ctx)
@@ -1778,7 +1845,7 @@ static void launch_fused(dq_ctx* ctx, const BatchSource& bs, const dq_state* s, 
     const FusedPlan pl = fused_plan(ctx);
     const size_t smem = fused_grad_smem(ctx);
     if (D.format == DQ_DENSE_F32)
-        launch_k(worker_grad_fused_kernel<float, false>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
+        launch_k(worker_grad_fused_kernel<float, 0>, pl.nblocks, kFusedThreads, smem, st, (const float*)D.values, D.labels, ctx->xhat_diff,
                  s->z_snap, ctx->keys, bs, pl, c.d, alpha, nb, ctx->fused_part, ctx->fused_cnt, ctx->status, fr);
     else
         launch_k(fused_kernel_bf16(ctx), pl.nblocks, kFusedThreads, smem, st, (const __nv_bfloat16*)D.values, D.labels,
@@ -1819,7 +1886,7 @@ int fused_grad_setup(dq_ctx* ctx)
     if (row_bytes > kFusedMaxRowBytes || (row_bytes & 15) || c.B < 64) return DQ_OK;
     if ((int64_t)c.M * ((c.B + kFusedRows - 1) / kFusedRows) > ((int64_t)1 << 24)) return DQ_OK;    // the tile arithmetic is 32-bit
     const int smem = (int)fused_grad_smem(ctx);
-    const FusedKernelF32 kf = worker_grad_fused_kernel<float, false>;
+    const FusedKernelF32 kf = worker_grad_fused_kernel<float, 0>;
     const FusedKernelBf16 kb = fused_kernel_bf16(ctx);
     const cudaError_t e = D.format == DQ_DENSE_F32 ? cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, smem)
                                                    : cudaFuncSetAttribute(kb, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);

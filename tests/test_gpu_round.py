@@ -208,7 +208,7 @@ def test_worker_gradient(dq, name, bx):
 
 
 @pytest.mark.parametrize("name,M,B,no_fused,tc", [("bf16", 2, 70, 0, 0), ("dense8", 2, 70, 0, 0), ("bf16x16", 3, 70, 0, 1), ("bf16x16", 5, 264, 0, 1),
-                                                  ("bf16x16", 3, 70, 0, 0), ("bf16x16", 2, 70, 1, 0), ("dense_wide", 2, 70, 0, 0)])
+                                                  ("bf16x16", 3, 70, 0, 0), ("bf16x16", 3, 70, 0, 2), ("bf16x16", 2, 70, 1, 0), ("dense_wide", 2, 70, 0, 0)])
 def test_worker_gradient_large_minibatch(dq, name, M, B, no_fused, tc):
     """B >= 64 takes the one-pass dense kernel (rows staged once; with tensor_cores = 1, bf16 rows on the 16-column grid by
     MMAs, else by CUDA cores) or, for rows too long to stage or with no_fused = 1, margins then column sums in two
@@ -529,7 +529,7 @@ class Lockstep:
     ("dense8", dict(M=5, B=64, bx=8, b=4, lambda1=1e-4, seed=56), 0.5),
     ("bf16", dict(M=4, B=70, bx=4, b=8, box_lo=-1.0, box_hi=1.0, seed=57), 0.01),
     ("bf16x16", dict(M=6, B=100, bx=8, b=2, lambda2=1e-4, seed=58, tensor_cores=1), 0.01),
-    ("bf16x16", dict(M=3, B=64, bx=2, b=4, box_lo=-0.5, box_hi=0.5, seed=59), 0.01),
+    ("bf16x16", dict(M=3, B=64, bx=2, b=4, box_lo=-0.5, box_hi=0.5, seed=59, tensor_cores=2), 0.01),
     # one row per minibatch and a coarse model: a worker's whole gradient hangs on one margin difference
     ("dense_wide", dict(M=16, B=1, bx=3, b=8, box_lo=-0.5, box_hi=2.0, seed=46, no_fused=1), 0.3),
     ("csr", dict(M=16, B=1, bx=3, b=4, box_lo=-0.5, box_hi=0.5, seed=47), 0.3),
@@ -790,7 +790,7 @@ def _full_config(name):
 
 
 @pytest.mark.parametrize("name,rounds,no_fused", [("c1", 100, 0), ("c2", 100, 0), ("c1", 30, 1), ("c2", 30, 1), ("c3", 100, 0), ("c4", 100, 0),
-                                                  ("c4", 20, 1), ("c4", 20, 2), ("c4", 20, 3)])
+                                                  ("c4", 20, 1), ("c4", 20, 2), ("c4", 20, 3), ("c4", 20, 4)])
 def test_lockstep_full_configs(dq, name, rounds, no_fused):
     """The benchmark configurations at their full model width for 100 rounds (c3, c4 with fewer rows so that the oracle
     finishes in seconds per round; the width, the workers and the minibatches are the full ones); c4 reads "momentum 0.9"
@@ -798,7 +798,7 @@ def test_lockstep_full_configs(dq, name, rounds, no_fused):
     kernels."""
     h = _problem(name)
     kw, lr, m = _full_config(name)
-    kw = dict(kw, no_fused=no_fused) if no_fused < 3 else dict(kw, tensor_cores=1)      # 3: the default plan with the tensor-core gradient
+    kw = dict(kw, no_fused=no_fused) if no_fused < 3 else dict(kw, tensor_cores=no_fused - 2)   # 3, 4: the default plan with a tensor-core gradient
     ls = Lockstep(dq, h, np.zeros(h.d, F32) if name != "c4" else synth.normal_vector(h.d, 75, 0.01), **kw)
     theta = F32(0.1) if name == "c4" else F32(0.0)
     eta = F32(lr) / theta if name == "c4" else F32(lr)
