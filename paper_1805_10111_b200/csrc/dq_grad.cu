@@ -1221,9 +1221,11 @@ objective_reg_kernel(const float* __restrict__ x, int64_t d, float l1, float l2,
 // cross-entropy.  Parameters x = [W1 (hidden x in, row-major), b1, W2 (classes x hidden), b2]; labels hold class
 // indices.  The worker needs grad f_B(xhat) - grad f_B(xsnap): three small kernels evaluate both parameter
 // vectors side by side (either may be absent: NULL), rows listed explicitly or drawn from the batch stream.
-//   mlp_hidden_kernel   block per tile of sampled rows and eight hidden units: hidden activations (one warp per unit, coalesced along in)
+//   mlp_hidden_kernel   block per tile of eight sampled rows and eight hidden units: hidden activations of both parameter
+//                       vectors as 8x8x4 fp64 tensor-core MMAs (rows x units x inputs)
 //   mlp_output_kernel   block per sampled row: logits, softmax, d loss / d logits, d loss / d hidden (ReLU-gated)
-//   mlp_param_kernel    block per (tile of hidden units or the tail, worker): sums over the worker's rows, no atomics
+//   mlp_param_kernel    block per (tile of eight hidden units or the tail, worker): the first-layer gradient as 8x8x4 fp64
+//                       MMAs (units x inputs x rows) over the worker's rows in slot order, no atomics
 // The forward pass (hidden pre-activations, activations, logits, softmax) runs in double precision: a class
 // probability depends on sums of hundreds of products that cancel, and an fp32 sum's error of 2^-24 of the
 // absolute terms passes through the softmax into every coordinate of the gradient, where the attainable accuracy
@@ -1239,9 +1241,18 @@ constexpr int kMlpUnits = 8;         // hidden units whose first-layer gradients
 constexpr int kMlpTile = 8;          // sampled rows that share one pass over a hidden unit's weights
 constexpr int kMlpRowChunk = 128;    // rows whose slope differences a block of mlp_param_kernel stages at a time
 
-// grid (ceil(nslots / kMlpTile), ceil(hidden / 8)): a block holds kMlpTile rows in shared memory and each of its
-// eight warps owns one hidden unit, so a weight row is read once for the whole tile (a block per row would read the
-// first layer once per sample).  Lanes stride over the inputs, then a butterfly across lanes.
+// D (8x8, fp64) += A (8x4, row-major) * B (4x8, column-major) on the tensor cores' double-precision path: every
+// product and sum is an IEEE fp64 fused multiply-add.  Lane l holds A[l / 4][l % 4], B[l % 4][l / 4] and the pair
+// D[l / 4][2 (l % 4)], D[l / 4][2 (l % 4) + 1].
+__device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, double b)
+{
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+}
+
+// grid (ceil(nslots / kMlpTile), ceil(hidden / 8)): a block forms the pre-activations of kMlpTile sampled rows and
+// eight hidden units, for both parameter vectors, as 8x8 fp64 tensor-core tiles: A = the rows' features (staged in
+// shared memory), B = the units' weight rows.  The inputs are split over the block's eight warps in steps of four;
+// the warps' partial tiles are added in warp order, then bias and ReLU.
 __global__ void __launch_bounds__(kThreads)
 mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restrict__ xa, const float* __restrict__ xb,
                   const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
@@ -1250,6 +1261,7 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
     pdl_prologue();
     extern __shared__ float s_in[];                      // [kMlpTile][in] features of the tile's rows
     __shared__ int64_t s_row[kMlpTile];
+    __shared__ double s_red[kThreads / 32][2][kMlpTile * 8];      // [warp][model][row * 8 + unit]
     clear_word(bs);
     const int64_t slot0 = (int64_t)blockIdx.x * kMlpTile;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -1268,27 +1280,36 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
         s_in[q] = s_row[t] >= 0 ? X[s_row[t] * sh.in + i] : 0.0f;
     }
     __syncthreads();
-    const int j = blockIdx.y * (kThreads / 32) + warp;
-    if (j >= sh.hidden) return;
-    double sa[kMlpTile], sb[kMlpTile];
-#pragma unroll
-    for (int t = 0; t < kMlpTile; ++t) { sa[t] = 0.0; sb[t] = 0.0; }
-#pragma unroll 2
-    for (int64_t i = lane; i < sh.in; i += 32) {
-        const double wa = xa ? (double)xa[(int64_t)j * sh.in + i] : 0.0, wb = xb ? (double)xb[(int64_t)j * sh.in + i] : 0.0;
-#pragma unroll
-        for (int t = 0; t < kMlpTile; ++t) {
-            const double f = (double)s_in[(int64_t)t * sh.in + i];
-            sa[t] = fma(wa, f, sa[t]); sb[t] = fma(wb, f, sb[t]);
-        }
+    const int j0 = blockIdx.y * 8;
+    const int kk = lane & 3, rn = lane >> 2;             // this lane's k of A and B; its row of A / unit of B
+    const int ju = j0 + rn;
+    const bool unit_ok = ju < sh.hidden;
+    const float* wa = (xa && unit_ok) ? xa + (int64_t)ju * sh.in : nullptr;
+    const float* wb = (xb && unit_ok) ? xb + (int64_t)ju * sh.in : nullptr;
+    const float* arow = s_in + (int64_t)rn * sh.in;
+    double da0 = 0.0, da1 = 0.0, db0 = 0.0, db1 = 0.0;
+    const int64_t ksteps = (sh.in + 3) >> 2;
+#pragma unroll 4
+    for (int64_t ks = warp; ks < ksteps; ks += kThreads / 32) {
+        const int64_t i = (ks << 2) + kk;
+        const bool in = i < sh.in;
+        const double a = in ? (double)arow[i] : 0.0;
+        const double ba = (in && wa) ? (double)__ldg(wa + i) : 0.0, bb = (in && wb) ? (double)__ldg(wb + i) : 0.0;
+        dmma_8x8x4(da0, da1, a, ba);
+        dmma_8x8x4(db0, db1, a, bb);
     }
-    const double ba = xa ? (double)xa[mlp_off_b1(sh) + j] : 0.0, bb = xb ? (double)xb[mlp_off_b1(sh) + j] : 0.0;
+    s_red[warp][0][rn * 8 + kk * 2] = da0; s_red[warp][0][rn * 8 + kk * 2 + 1] = da1;
+    s_red[warp][1][rn * 8 + kk * 2] = db0; s_red[warp][1][rn * 8 + kk * 2 + 1] = db1;
+    __syncthreads();
+    if (threadIdx.x < 2 * kMlpTile * 8) {
+        const int model = threadIdx.x / (kMlpTile * 8), e = threadIdx.x % (kMlpTile * 8), t = e >> 3, u = e & 7;
+        const float* xm = model == 0 ? xa : xb;
+        double* act = model == 0 ? act_a : act_b;
+        if (xm && j0 + u < sh.hidden && slot0 + t < nslots) {
+            double v = 0.0;
 #pragma unroll
-    for (int t = 0; t < kMlpTile; ++t) {
-        const double va = warp_sum(sa[t]), vb = warp_sum(sb[t]);
-        if (lane == 0 && slot0 + t < nslots) {
-            if (xa) act_a[(slot0 + t) * sh.hidden + j] = fmax(va + ba, 0.0);
-            if (xb) act_b[(slot0 + t) * sh.hidden + j] = fmax(vb + bb, 0.0);
+            for (int k = 0; k < kThreads / 32; ++k) v += s_red[k][model][e];
+            act[(slot0 + t) * sh.hidden + j0 + u] = fmax(v + (double)xm[mlp_off_b1(sh) + j0 + u], 0.0);
         }
     }
 }
@@ -1366,52 +1387,64 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
     uint32_t nmax = 0;
     float* o = FULL ? nullptr : out + (int64_t)w * P;
     if (j0 < sh.hidden) {
-        // s_w[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u]; the rows' indices sit beside them: no dependent load in the loop.
-        // The block's hidden units share every feature value that a thread loads.  A thread owns the inputs
-        // i = threadIdx.x + k * blockDim.x (i == in: the bias b1[j]) and keeps their sums across the chunks of rows.
-        constexpr int kOwn = 4;                                             // inputs per thread and pass
-        for (int64_t ibase = 0; ibase <= sh.in; ibase += (int64_t)kOwn * blockDim.x) {
-            double s[kOwn][kMlpUnits];
+        // First-layer gradient of eight hidden units as 8x8 fp64 tensor-core tiles: D[unit][input] += sum_r A[unit][r] B[r][input]
+        // with A[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u] (staged in shared memory, a chunk of rows at a time) and
+        // B[r][i] = feature i of row r.  A warp owns tiles of eight inputs (kTiles of them per pass, 8 * kTiles * 8 inputs per
+        // block and pass) and keeps their sums across the chunks of rows; rows enter in slot order.
+        constexpr int kTiles = 8;
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const int kk = lane & 3, un = lane >> 2;             // this lane's k (row of the chunk) of A and B; its unit of A / input of B
+        double bias = 0.0;                                   // thread u < 8: d loss / d b1[j0 + u]
+        for (int64_t ibase = 0; ibase < sh.in; ibase += (int64_t)(kThreads / 32) * kTiles * 8) {
+            double acc[kTiles][2];
 #pragma unroll
-            for (int k = 0; k < kOwn; ++k)
-#pragma unroll
-                for (int u = 0; u < kMlpUnits; ++u) s[k][u] = 0.0;
+            for (int t = 0; t < kTiles; ++t) { acc[t][0] = 0.0; acc[t][1] = 0.0; }
             for (int c0 = 0; c0 < nrows; c0 += kMlpRowChunk) {
                 const int cn = min(kMlpRowChunk, nrows - c0);
                 __syncthreads();
-                for (int q = threadIdx.x; q < kMlpUnits * cn; q += blockDim.x) {
-                    const int u = q / cn, r = q - u * cn, j = j0 + u;
-                    const float da = (dh_a && j < sh.hidden) ? dh_a[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
-                    const float db = (dh_b && j < sh.hidden) ? dh_b[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
-                    s_w[u][r] = (double)da - (double)db;
+                for (int q = threadIdx.x; q < kMlpUnits * kMlpRowChunk; q += blockDim.x) {
+                    const int u = q / kMlpRowChunk, r = q - u * kMlpRowChunk, j = j0 + u;
+                    const bool in = r < cn && j < sh.hidden;
+                    const float da = (dh_a && in) ? dh_a[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
+                    const float db = (dh_b && in) ? dh_b[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
+                    s_w[u][r] = (double)da - (double)db;     // zero beyond the chunk's rows
                 }
-                for (int r = threadIdx.x; r < cn; r += blockDim.x) s_rowid[r] = row_of_slot[r0 + c0 + r];
+                for (int r = threadIdx.x; r < kMlpRowChunk; r += blockDim.x) s_rowid[r] = r < cn ? row_of_slot[r0 + c0 + r] : -1;
                 __syncthreads();
+                if (ibase == 0 && threadIdx.x < kMlpUnits) for (int r = 0; r < cn; ++r) bias += s_w[threadIdx.x][r];
+                const int ksteps = (cn + 3) >> 2;
 #pragma unroll
-                for (int k = 0; k < kOwn; ++k) {
-                    const int64_t i = ibase + threadIdx.x + (int64_t)k * blockDim.x;
-                    if (i > sh.in) continue;
-#pragma unroll 2
-                    for (int r = 0; r < cn; ++r) {
-                        const double f = (i < sh.in) ? (double)X[(int64_t)s_rowid[r] * sh.in + i] : 1.0;
-#pragma unroll
-                        for (int u = 0; u < kMlpUnits; ++u) s[k][u] = fma(s_w[u][r], f, s[k][u]);
+                for (int t = 0; t < kTiles; ++t) {
+                    const int64_t i = ibase + ((int64_t)(warp * kTiles + t) << 3) + un;       // this lane's input column of tile t
+                    if (ibase + ((int64_t)(warp * kTiles + t) << 3) >= sh.in) break;          // (the same for the whole warp)
+#pragma unroll 4
+                    for (int ks = 0; ks < ksteps; ++ks) {
+                        const int r = (ks << 2) + kk;
+                        const int row = s_rowid[r];
+                        const double a = s_w[un][r];
+                        const double b = (row >= 0 && i < sh.in) ? (double)__ldg(X + (int64_t)row * sh.in + i) : 0.0;
+                        dmma_8x8x4(acc[t][0], acc[t][1], a, b);
                     }
                 }
             }
 #pragma unroll
-            for (int k = 0; k < kOwn; ++k) {
-                const int64_t i = ibase + threadIdx.x + (int64_t)k * blockDim.x;
-                if (i > sh.in) continue;
+            for (int t = 0; t < kTiles; ++t) {
+                const int64_t i0 = ibase + ((int64_t)(warp * kTiles + t) << 3) + kk * 2;      // D[un][2 kk], D[un][2 kk + 1]
+                const int j = j0 + un;
 #pragma unroll
-                for (int u = 0; u < kMlpUnits; ++u) {
-                    const int j = j0 + u;
-                    if (j >= sh.hidden) break;
-                    const int64_t pidx = (i < sh.in) ? (int64_t)j * sh.in + i : mlp_off_b1(sh) + j;
-                    if (FULL) atomicAdd(g64 + pidx, s[k][u]);
-                    else { o[pidx] = (float)s[k][u]; nmax = max(nmax, __float_as_uint((float)s[k][u]) & 0x7FFFFFFFu); }
+                for (int e = 0; e < 2; ++e) {
+                    if (j < sh.hidden && i0 + e < sh.in) {
+                        const int64_t pidx = (int64_t)j * sh.in + i0 + e;
+                        if (FULL) atomicAdd(g64 + pidx, acc[t][e]);
+                        else { o[pidx] = (float)acc[t][e]; nmax = max(nmax, __float_as_uint((float)acc[t][e]) & 0x7FFFFFFFu); }
+                    }
                 }
             }
+        }
+        if (threadIdx.x < kMlpUnits && j0 + (int)threadIdx.x < sh.hidden) {
+            const int64_t pidx = mlp_off_b1(sh) + j0 + threadIdx.x;
+            if (FULL) atomicAdd(g64 + pidx, bias);
+            else { o[pidx] = (float)bias; nmax = max(nmax, __float_as_uint((float)bias) & 0x7FFFFFFFu); }
         }
     } else {
         const int nout = sh.classes * (sh.hidden + 1);                       // W2 entries then b2
