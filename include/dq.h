@@ -95,7 +95,7 @@ typedef struct {
                                   Section 5.2, in -> hidden (ReLU) -> classes with softmax cross-entropy.  For the network
                                   the data must be DQ_DENSE_F32 with labels = class index, data.d = number of inputs, and
                                   d = hidden*(in+1) + classes*(hidden+1) with x = [W1 (hidden x in), b1, W2 (classes x hidden), b2] */
-    int32_t hidden, classes;
+    int32_t hidden, classes;      /* hidden + 3*classes <= 3072 */
     int32_t no_fused;          /* 0: merged kernels where they apply (the one-cluster round, quantiser + master in one kernel, the
                                   one-pass dense gradient carrying the whole round); 1: every stage as its own kernel(s), the plan
                                   the merged ones are tested against; 2: like 1, but the dense gradient stage stays one pass */

@@ -91,6 +91,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
         if (data->n < 1 || !data->values || !data->labels) return DQ_ERR_SHAPE;
         if (cfg->model == DQ_MODEL_MLP) {
             if (data->format != DQ_DENSE_F32 || cfg->hidden < 1 || cfg->classes < 2 || data->d < 1) return DQ_ERR_ARG;
+            if (cfg->hidden + 3 * (int64_t)cfg->classes > 3072) return DQ_ERR_ARG;   // the output layer's row fits 48 KB of shared memory
             if (cfg->d != (int64_t)cfg->hidden * (data->d + 1) + (int64_t)cfg->classes * (cfg->hidden + 1)) return DQ_ERR_SHAPE;
         } else if (cfg->model != DQ_MODEL_LOGISTIC || data->d != cfg->d) {
             return DQ_ERR_SHAPE;

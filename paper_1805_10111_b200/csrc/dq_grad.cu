@@ -1238,7 +1238,7 @@ __device__ __forceinline__ int64_t mlp_off_w2(const MlpShape& s) { return mlp_of
 __device__ __forceinline__ int64_t mlp_off_b2(const MlpShape& s) { return mlp_off_w2(s) + (int64_t)s.classes * s.hidden; }
 
 constexpr int kMlpUnits = 8;         // hidden units whose first-layer gradients one block forms from the same rows
-constexpr int kMlpTile = 8;          // sampled rows that share one pass over a hidden unit's weights
+constexpr int kMlpTile = 16;         // sampled rows that share one pass over a hidden unit's weights
 constexpr int kMlpRowChunk = 128;    // rows whose slope differences a block of mlp_param_kernel stages at a time
 
 // D (8x8, fp64) += A (8x4, row-major) * B (4x8, column-major) on the tensor cores' double-precision path: every
@@ -1246,20 +1246,40 @@ constexpr int kMlpRowChunk = 128;    // rows whose slope differences a block of 
 // D[l / 4][2 (l % 4)], D[l / 4][2 (l % 4) + 1].
 __device__ __forceinline__ void dmma_8x8x4(double& d0, double& d1, double a, double b)
 {
-    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
+    asm("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0,%1}, {%2}, {%3}, {%0,%1};" : "+d"(d0), "+d"(d1) : "d"(a), "d"(b));
 }
 
-// grid (ceil(nslots / kMlpTile), ceil(hidden / 8)): a block forms the pre-activations of kMlpTile sampled rows and
-// eight hidden units, for both parameter vectors, as 8x8 fp64 tensor-core tiles: A = the rows' features (staged in
-// shared memory), B = the units' weight rows.  The inputs are split over the block's eight warps in steps of four;
-// the warps' partial tiles are added in warp order, then bias and ReLU.
+// Four consecutive floats of a row starting at feature i (zero beyond the row's end, or when the row is absent).
+// VEC: the row length is a multiple of four and the rows are 16-byte aligned, so one 16-byte load serves.
+template <bool VEC>
+__device__ __forceinline__ float4 mlp_load4(const float* __restrict__ p, int i, int in)
+{
+    float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+    if (!p || i >= in) return v;
+    if (VEC) return __ldg(reinterpret_cast<const float4*>(p + i));
+    v.x = __ldg(p + i);
+    if (i + 1 < in) v.y = __ldg(p + i + 1);
+    if (i + 2 < in) v.z = __ldg(p + i + 2);
+    if (i + 3 < in) v.w = __ldg(p + i + 3);
+    return v;
+}
+
+// grid (ceil(nslots / kMlpTile), ceil(hidden / 8)): a block forms the pre-activations of kMlpTile = 16 sampled rows
+// (two tiles of eight) and eight hidden units, for both parameter vectors, as 8x8 fp64 tensor-core tiles: A = the
+// rows' features, B = the units' weight rows, both read straight from global memory (L2-resident).  A lane loads
+// 16 bytes of its row and of its unit's two weight rows per chunk of 16 inputs: input 16 c + 4 (lane % 4) + e is
+// the lane's k of the chunk's e-th MMA step (the order of a sum's terms is free, and fixed here), so every 32-byte
+// sector that is fetched is used, and four row tiles x models share each weight load.  The chunks are split over
+// the block's eight warps, kMlpBatch chunks in flight per warp; the warps' partial tiles are added in warp order,
+// then bias and ReLU.
+constexpr int kMlpBatch = 3;
+template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
 mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restrict__ xa, const float* __restrict__ xb,
                   const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
                   double* __restrict__ act_a, double* __restrict__ act_b, int64_t nslots)
 {
     pdl_prologue();
-    extern __shared__ float s_in[];                      // [kMlpTile][in] features of the tile's rows
     __shared__ int64_t s_row[kMlpTile];
     __shared__ double s_red[kThreads / 32][2][kMlpTile * 8];      // [warp][model][row * 8 + unit]
     clear_word(bs);
@@ -1275,34 +1295,54 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
         s_row[threadIdx.x] = a;
     }
     __syncthreads();
-    for (int64_t q = threadIdx.x; q < (int64_t)kMlpTile * sh.in; q += blockDim.x) {
-        const int t = (int)(q / sh.in); const int64_t i = q - (int64_t)t * sh.in;
-        s_in[q] = s_row[t] >= 0 ? X[s_row[t] * sh.in + i] : 0.0f;
-    }
-    __syncthreads();
     const int j0 = blockIdx.y * 8;
     const int kk = lane & 3, rn = lane >> 2;             // this lane's k of A and B; its row of A / unit of B
     const int ju = j0 + rn;
     const bool unit_ok = ju < sh.hidden;
-    const float* wa = (xa && unit_ok) ? xa + (int64_t)ju * sh.in : nullptr;
-    const float* wb = (xb && unit_ok) ? xb + (int64_t)ju * sh.in : nullptr;
-    const float* arow = s_in + (int64_t)rn * sh.in;
-    double da0 = 0.0, da1 = 0.0, db0 = 0.0, db1 = 0.0;
-    const int64_t ksteps = (sh.in + 3) >> 2;
-#pragma unroll 4
-    for (int64_t ks = warp; ks < ksteps; ks += kThreads / 32) {
-        const int64_t i = (ks << 2) + kk;
-        const bool in = i < sh.in;
-        const double a = in ? (double)arow[i] : 0.0;
-        const double ba = (in && wa) ? (double)__ldg(wa + i) : 0.0, bb = (in && wb) ? (double)__ldg(wb + i) : 0.0;
-        dmma_8x8x4(da0, da1, a, ba);
-        dmma_8x8x4(db0, db1, a, bb);
+    const int in = (int)sh.in;
+    const float* wa = (xa && unit_ok) ? xa + (int64_t)ju * in : nullptr;
+    const float* wb = (xb && unit_ok) ? xb + (int64_t)ju * in : nullptr;
+    const float* arow0 = s_row[rn] >= 0 ? X + s_row[rn] * in : nullptr;
+    const float* arow1 = s_row[8 + rn] >= 0 ? X + s_row[8 + rn] * in : nullptr;
+    double d[2][2][2];                                   // [row tile][model][pair]
+#pragma unroll
+    for (int q = 0; q < 8; ++q) (&d[0][0][0])[q] = 0.0;
+    const int nchunk = (in + 15) >> 4;
+    constexpr int W = kThreads / 32;
+    for (int c0 = warp; c0 < nchunk; c0 += W * kMlpBatch) {
+        float4 fa0[kMlpBatch], fa1[kMlpBatch], fwa[kMlpBatch], fwb[kMlpBatch];
+#pragma unroll
+        for (int u = 0; u < kMlpBatch; ++u) {
+            const int i = ((c0 + u * W) << 4) + (kk << 2);   // beyond the last chunk i >= in: zeros
+            fa0[u] = mlp_load4<VEC>(arow0, i, in);
+            fa1[u] = mlp_load4<VEC>(arow1, i, in);
+            fwa[u] = mlp_load4<VEC>(wa, i, in);
+            fwb[u] = mlp_load4<VEC>(wb, i, in);
+        }
+#pragma unroll
+        for (int u = 0; u < kMlpBatch; ++u) {
+            if (c0 + u * W >= nchunk) break;             // (the same for the whole warp)
+            const float a0[4] = {fa0[u].x, fa0[u].y, fa0[u].z, fa0[u].w}, a1[4] = {fa1[u].x, fa1[u].y, fa1[u].z, fa1[u].w};
+            const float ba[4] = {fwa[u].x, fwa[u].y, fwa[u].z, fwa[u].w}, bb[4] = {fwb[u].x, fwb[u].y, fwb[u].z, fwb[u].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                dmma_8x8x4(d[0][0][0], d[0][0][1], (double)a0[e], (double)ba[e]);
+                dmma_8x8x4(d[0][1][0], d[0][1][1], (double)a0[e], (double)bb[e]);
+                dmma_8x8x4(d[1][0][0], d[1][0][1], (double)a1[e], (double)ba[e]);
+                dmma_8x8x4(d[1][1][0], d[1][1][1], (double)a1[e], (double)bb[e]);
+            }
+        }
     }
-    s_red[warp][0][rn * 8 + kk * 2] = da0; s_red[warp][0][rn * 8 + kk * 2 + 1] = da1;
-    s_red[warp][1][rn * 8 + kk * 2] = db0; s_red[warp][1][rn * 8 + kk * 2 + 1] = db1;
+#pragma unroll
+    for (int rt = 0; rt < 2; ++rt)
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            s_red[warp][m][(rt * 8 + rn) * 8 + kk * 2] = d[rt][m][0];
+            s_red[warp][m][(rt * 8 + rn) * 8 + kk * 2 + 1] = d[rt][m][1];
+        }
     __syncthreads();
-    if (threadIdx.x < 2 * kMlpTile * 8) {
-        const int model = threadIdx.x / (kMlpTile * 8), e = threadIdx.x % (kMlpTile * 8), t = e >> 3, u = e & 7;
+    for (int q = threadIdx.x; q < 2 * kMlpTile * 8; q += blockDim.x) {
+        const int model = q / (kMlpTile * 8), e = q % (kMlpTile * 8), t = e >> 3, u = e & 7;
         const float* xm = model == 0 ? xa : xb;
         double* act = model == 0 ? act_a : act_b;
         if (xm && j0 + u < sh.hidden && slot0 + t < nslots) {
@@ -1314,64 +1354,105 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
     }
 }
 
-// One model of one row: logits -> softmax -> dz = (p - onehot) * wgt, dh_j = relu'(h_j) sum_c dz_c W2[c][j]; returns loss.
-__device__ __forceinline__ void mlp_output_one(const MlpShape& sh, const float* __restrict__ x, const double* __restrict__ act,
-                                               int label, double wgt, float* __restrict__ dz, float* __restrict__ dh,
-                                               double* s_z, double* loss_out)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int c = warp; c < sh.classes; c += kThreads / 32) {
-        double s = 0.0;
-        for (int j = lane; j < sh.hidden; j += 32) s = fma((double)x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], act[j], s);
-        s = warp_sum(s);
-        if (lane == 0) s_z[c] = s + (double)x[mlp_off_b2(sh) + c];
-    }
-    __syncthreads();
-    double zmax = -INFINITY, sum = 0.0, others = 0.0;       // others: the sum without the label's term, so that
-    for (int c = 0; c < sh.classes; ++c) zmax = fmax(zmax, s_z[c]);      // p_label - 1 = -others/sum has no cancellation
-    for (int c = 0; c < sh.classes; ++c) { const double e = exp(s_z[c] - zmax); sum += e; if (c != label) others += e; }
-    if (threadIdx.x == 0 && loss_out) *loss_out = (zmax + log(sum)) - s_z[label];
-    __syncthreads();
-    for (int c = threadIdx.x; c < sh.classes; c += blockDim.x) {
-        const double v = (c == label ? -others / sum : exp(s_z[c] - zmax) / sum) * wgt;
-        s_z[sh.classes + c] = v;
-        if (dz) dz[c] = (float)v;
-    }
-    __syncthreads();
-    if (dh) {
-        for (int j = threadIdx.x; j < sh.hidden; j += blockDim.x) {
-            double s = 0.0;
-            for (int c = 0; c < sh.classes; ++c) s = fma(s_z[sh.classes + c], (double)x[mlp_off_w2(sh) + (int64_t)c * sh.hidden + j], s);
-            dh[j] = act[j] > 0.0 ? (float)s : 0.0f;
-        }
-    }
-    __syncthreads();
-}
-
+// Block per sampled row, both parameter vectors side by side: logits (a warp per (model, class)), softmax,
+// dz = (p - onehot) * wgt, dh_j = relu'(h_j) sum_c dz_c W2[c][j], and the loss of model b.  One thread per
+// (model, class) takes the exponential; every sum runs in class order.  p_label - 1 is formed as -others / sum
+// (the sum without the label's term), which has no cancellation.
 __global__ void __launch_bounds__(kThreads)
 mlp_output_kernel(MlpShape sh, const float* __restrict__ labels, const int32_t* __restrict__ row_of_slot,
                   const float* __restrict__ xa, const float* __restrict__ xb, const double* __restrict__ act_a,
                   const double* __restrict__ act_b, double wgt, float* __restrict__ dz_a, float* __restrict__ dz_b,
-                  float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b)
+                  float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b, int staged)
 {
     pdl_prologue();
-    extern __shared__ double s_zd[];                     // [2 * classes]
+    extern __shared__ double s_zd[];     // [2 models][logits, exponentials, dz][classes], [2][hidden] activations, staged: [2][W2, b2]
+    const int C = sh.classes, H = sh.hidden;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t slot = blockIdx.x;
     const int label = (int)labels[row_of_slot[slot]];
-    if (xa) mlp_output_one(sh, xa, act_a + slot * sh.hidden, label, wgt, dz_a + slot * sh.classes, dh_a + slot * sh.hidden, s_zd, nullptr);
-    if (xb) {
-        double loss = 0.0;
-        mlp_output_one(sh, xb, act_b + slot * sh.hidden, label, wgt, dz_b ? dz_b + slot * sh.classes : nullptr,
-                       dh_b ? dh_b + slot * sh.hidden : nullptr, s_zd, loss_b ? &loss : nullptr);
-        if (loss_b && threadIdx.x == 0) atomicAdd(loss_b, loss * wgt);
+    double* s_act = s_zd + 6 * C;
+    float* s_w2 = reinterpret_cast<float*>(s_act + 2 * H);
+    const int nw2 = C * H + C;                           // W2 and b2 are adjacent in the parameter vector
+    if (staged) {
+        for (int q0 = threadIdx.x; q0 < 2 * nw2; q0 += 8 * kThreads) {      // eight loads in flight per thread
+            float v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int q = q0 + u * kThreads, m = q >= nw2;
+                const float* x = m ? xb : xa;
+                v[u] = (x && q < 2 * nw2) ? __ldg(x + mlp_off_w2(sh) + (q - m * nw2)) : 0.0f;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) if (q0 + u * kThreads < 2 * nw2) s_w2[q0 + u * kThreads] = v[u];
+        }
+    }
+    for (int q = threadIdx.x; q < 2 * H; q += blockDim.x) {
+        const int m = q >= H, j = q - m * H;
+        const double* act = m ? act_b : act_a;
+        s_act[q] = ((m ? xb : xa) && act) ? act[slot * H + j] : 0.0;
+    }
+    __syncthreads();
+    for (int q = warp; q < 2 * C; q += kThreads / 32) {
+        const int m = q >= C, c = q - m * C;
+        const float* x = m ? xb : xa;
+        if (!x) continue;
+        const float* w2 = staged ? s_w2 + m * nw2 : x + mlp_off_w2(sh);
+        const float* wrow = w2 + (int64_t)c * H;
+        const double* act = s_act + m * H;
+        double s = 0.0;
+#pragma unroll 4
+        for (int j = lane; j < H; j += 32) s = fma((double)wrow[j], act[j], s);
+        s = warp_sum(s);
+        if (lane == 0) s_zd[m * 3 * C + c] = s + (double)w2[(int64_t)C * H + c];
+    }
+    __syncthreads();
+    for (int q = threadIdx.x; q < 2 * C; q += blockDim.x) {
+        const int m = q >= C, c = q - m * C;
+        if (!(m ? xb : xa)) continue;
+        const double* z = s_zd + m * 3 * C;
+        double zmax = -INFINITY;
+        for (int cc = 0; cc < C; ++cc) zmax = fmax(zmax, z[cc]);
+        s_zd[m * 3 * C + C + c] = exp(z[c] - zmax);
+    }
+    __syncthreads();
+    for (int q = threadIdx.x; q < 2 * C; q += blockDim.x) {
+        const int m = q >= C, c = q - m * C;
+        if (!(m ? xb : xa)) continue;
+        const double* z = s_zd + m * 3 * C;
+        const double* e = z + C;
+        double sum = 0.0, others = 0.0;
+        for (int cc = 0; cc < C; ++cc) { sum += e[cc]; if (cc != label) others += e[cc]; }
+        const double v = (c == label ? -others / sum : e[c] / sum) * wgt;
+        s_zd[m * 3 * C + 2 * C + c] = v;
+        float* dz = m ? dz_b : dz_a;
+        if (dz) dz[slot * C + c] = (float)v;
+        if (m && c == 0 && loss_b) {
+            double zmax = -INFINITY;
+            for (int cc = 0; cc < C; ++cc) zmax = fmax(zmax, z[cc]);
+            atomicAdd(loss_b, ((zmax + log(sum)) - z[label]) * wgt);
+        }
+    }
+    __syncthreads();
+    for (int q = threadIdx.x; q < 2 * H; q += blockDim.x) {
+        const int m = q >= H, j = q - m * H;
+        const float* x = m ? xb : xa;
+        float* dh = m ? dh_b : dh_a;
+        if (!x || !dh) continue;
+        const double* dzs = s_zd + m * 3 * C + 2 * C;
+        const float* wcol = (staged ? s_w2 + m * nw2 : x + mlp_off_w2(sh)) + j;
+        double s = 0.0;
+#pragma unroll 10
+        for (int c = 0; c < C; ++c) s = fma(dzs[c], (double)wcol[(int64_t)c * H], s);
+        dh[slot * H + j] = s_act[q] > 0.0 ? (float)s : 0.0f;
     }
 }
 
-// grid (ceil(hidden / kMlpUnits) + 1, groups): block (j, w) sums over the rows [w*B, (w+1)*B) of its group, in slot
-// order and in double.  Blocks before the last: rows j0 .. j0 + kMlpUnits - 1 of W1 and their b1; last block: W2 and b2.
+// grid (ceil(hidden / kMlpUnits) + ceil(classes (hidden + 1) / threads), groups): block (j, w) sums over the rows
+// [w*B, (w+1)*B) of its group, in slot order and in double.  The first ceil(hidden / kMlpUnits) blocks: rows
+// j0 .. j0 + kMlpUnits - 1 of W1 and their b1; the blocks after them: W2 and b2, an entry per thread.
 // Output = model a minus model b (either may be absent).  FULL: sums added to g64 with atomics (epoch gradient over
 // many groups); otherwise rounded once and stored to out [groups][P] with the norm folded in.
-template <bool FULL>
+template <bool FULL, bool VEC>
 __global__ void __launch_bounds__(kThreads)
 mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __restrict__ row_of_slot, int B, int64_t total_rows,
                  const double* __restrict__ act_a, const double* __restrict__ act_b, const float* __restrict__ dz_a,
@@ -1379,62 +1460,88 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
                  float* __restrict__ out, int64_t P, uint32_t* __restrict__ norm_bits, double* __restrict__ g64)
 {
     pdl_prologue();
-    __shared__ double s_w[kMlpUnits][kMlpRowChunk];      // slope differences of a chunk of rows
+    constexpr int kTiles = 13, W = kThreads / 32, kPassIn = W * kTiles * 8, kR = 8;
+    constexpr int kStage = (kR * (kPassIn / 4) + kThreads - 1) / kThreads;     // 16-byte groups a thread stages per eight rows
+    __shared__ __align__(16) float s_x[kR][kPassIn + 8]; // features of eight rows, the inputs of the current pass (+8: bank spread)
+    __shared__ double s_w[kMlpUnits][kR];                // slope differences of those rows
     __shared__ int s_rowid[kMlpRowChunk];
-    const int j0 = blockIdx.x * kMlpUnits, w = blockIdx.y;     // the block after the last tile of hidden units does W2, b2
+    const int j0 = blockIdx.x * kMlpUnits, w = blockIdx.y;     // the blocks after the last tile of hidden units do W2, b2
     const int64_t r0 = (int64_t)w * B;
     const int nrows = (int)min((int64_t)B, total_rows - r0);
     uint32_t nmax = 0;
     float* o = FULL ? nullptr : out + (int64_t)w * P;
     if (j0 < sh.hidden) {
         // First-layer gradient of eight hidden units as 8x8 fp64 tensor-core tiles: D[unit][input] += sum_r A[unit][r] B[r][input]
-        // with A[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u] (staged in shared memory, a chunk of rows at a time) and
-        // B[r][i] = feature i of row r.  A warp owns tiles of eight inputs (kTiles of them per pass, 8 * kTiles * 8 inputs per
-        // block and pass) and keeps their sums across the chunks of rows; rows enter in slot order.
-        constexpr int kTiles = 8;
+        // with A[u][r] = dh_a[r][j0 + u] - dh_b[r][j0 + u] and B[r][i] = feature i of row r, both staged in shared memory
+        // eight rows at a time (the rows with 16-byte loads by the whole block).  Tiles of eight inputs are dealt to the
+        // warps round robin, kTiles per warp and pass (8 * 13 tiles cover the 784 inputs of the image workloads in one
+        // pass); a warp keeps its tiles' sums across the rows.  Rows enter in slot order.
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         const int kk = lane & 3, un = lane >> 2;             // this lane's k (row of the chunk) of A and B; its unit of A / input of B
+        const int in = (int)sh.in, ntile = (in + 7) >> 3;
         double bias = 0.0;                                   // thread u < 8: d loss / d b1[j0 + u]
-        for (int64_t ibase = 0; ibase < sh.in; ibase += (int64_t)(kThreads / 32) * kTiles * 8) {
+        for (int in0 = 0; in0 < in; in0 += kPassIn) {
+            const int tile0 = in0 >> 3;
+            const int nv = ((min(kPassIn, in - in0) + 7) >> 3) << 1;     // 16-byte groups per staged row
             double acc[kTiles][2];
 #pragma unroll
             for (int t = 0; t < kTiles; ++t) { acc[t][0] = 0.0; acc[t][1] = 0.0; }
             for (int c0 = 0; c0 < nrows; c0 += kMlpRowChunk) {
                 const int cn = min(kMlpRowChunk, nrows - c0);
                 __syncthreads();
-                for (int q = threadIdx.x; q < kMlpUnits * kMlpRowChunk; q += blockDim.x) {
-                    const int u = q / kMlpRowChunk, r = q - u * kMlpRowChunk, j = j0 + u;
-                    const bool in = r < cn && j < sh.hidden;
-                    const float da = (dh_a && in) ? dh_a[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
-                    const float db = (dh_b && in) ? dh_b[(r0 + c0 + r) * sh.hidden + j] : 0.0f;
-                    s_w[u][r] = (double)da - (double)db;     // zero beyond the chunk's rows
-                }
-                for (int r = threadIdx.x; r < kMlpRowChunk; r += blockDim.x) s_rowid[r] = r < cn ? row_of_slot[r0 + c0 + r] : -1;
+                for (int r = threadIdx.x; r < cn; r += blockDim.x) s_rowid[r] = row_of_slot[r0 + c0 + r];
                 __syncthreads();
-                if (ibase == 0 && threadIdx.x < kMlpUnits) for (int r = 0; r < cn; ++r) bias += s_w[threadIdx.x][r];
-                const int ksteps = (cn + 3) >> 2;
+                // eight rows at a time; the loads of the next eight are in flight while these are multiplied
+                float4 buf[kStage]; float wa = 0.0f, wb = 0.0f;
+                auto fetch = [&](int c1) {
+                    const int rn = min(kR, cn - c1);
 #pragma unroll
-                for (int t = 0; t < kTiles; ++t) {
-                    const int64_t i = ibase + ((int64_t)(warp * kTiles + t) << 3) + un;       // this lane's input column of tile t
-                    if (ibase + ((int64_t)(warp * kTiles + t) << 3) >= sh.in) break;          // (the same for the whole warp)
-#pragma unroll 4
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        const int r = (ks << 2) + kk;
-                        const int row = s_rowid[r];
-                        const double a = s_w[un][r];
-                        const double b = (row >= 0 && i < sh.in) ? (double)__ldg(X + (int64_t)row * sh.in + i) : 0.0;
-                        dmma_8x8x4(acc[t][0], acc[t][1], a, b);
+                    for (int it = 0; it < kStage; ++it) {
+                        const int q = threadIdx.x + it * kThreads, r = q / nv, v = q - r * nv;
+                        const float* xr = r < rn ? X + (int64_t)s_rowid[c1 + min(r, rn - 1)] * in : nullptr;
+                        buf[it] = mlp_load4<VEC>(xr, in0 + 4 * v, in);     // (rows beyond the chunk: zeros)
+                    }
+                    if (threadIdx.x < kMlpUnits * kR) {
+                        const int u = threadIdx.x / kR, r = threadIdx.x % kR, j = j0 + u;
+                        const bool ok = r < rn && j < sh.hidden;
+                        wa = (dh_a && ok) ? dh_a[(r0 + c0 + c1 + r) * sh.hidden + j] : 0.0f;
+                        wb = (dh_b && ok) ? dh_b[(r0 + c0 + c1 + r) * sh.hidden + j] : 0.0f;
+                    }
+                };
+                fetch(0);
+                for (int c1 = 0; c1 < cn; c1 += kR) {
+                    const int rn = min(kR, cn - c1);
+                    if (c1) __syncthreads();                 // the previous eight rows have been used
+#pragma unroll
+                    for (int it = 0; it < kStage; ++it) {
+                        const int q = threadIdx.x + it * kThreads, r = q / nv, v = q - r * nv;
+                        if (r < kR) *reinterpret_cast<float4*>(&s_x[r][4 * v]) = buf[it];
+                    }
+                    if (threadIdx.x < kMlpUnits * kR) s_w[threadIdx.x / kR][threadIdx.x % kR] = (double)wa - (double)wb;   // zero beyond the last row
+                    __syncthreads();
+                    if (c1 + kR < cn) fetch(c1 + kR);
+                    if (in0 == 0 && threadIdx.x < kMlpUnits) for (int r = 0; r < rn; ++r) bias += s_w[threadIdx.x][r];
+#pragma unroll
+                    for (int ks = 0; ks < kR / 4; ++ks) {
+                        if (ks * 4 < rn) {
+                            const int r = (ks << 2) + kk;
+                            const double a = s_w[un][r];
+#pragma unroll
+                            for (int t = 0; t < kTiles; ++t)
+                                if (tile0 + t * W + warp < ntile)                                  // (the same for the whole warp)
+                                    dmma_8x8x4(acc[t][0], acc[t][1], a, (double)s_x[r][((t * W + warp) << 3) + un]);
+                        }
                     }
                 }
             }
 #pragma unroll
             for (int t = 0; t < kTiles; ++t) {
-                const int64_t i0 = ibase + ((int64_t)(warp * kTiles + t) << 3) + kk * 2;      // D[un][2 kk], D[un][2 kk + 1]
+                const int i0 = ((tile0 + t * W + warp) << 3) + kk * 2;                        // D[un][2 kk], D[un][2 kk + 1]
                 const int j = j0 + un;
 #pragma unroll
                 for (int e = 0; e < 2; ++e) {
-                    if (j < sh.hidden && i0 + e < sh.in) {
-                        const int64_t pidx = (int64_t)j * sh.in + i0 + e;
+                    if (j < sh.hidden && i0 + e < in) {
+                        const int64_t pidx = (int64_t)j * in + i0 + e;
                         if (FULL) atomicAdd(g64 + pidx, acc[t][e]);
                         else { o[pidx] = (float)acc[t][e]; nmax = max(nmax, __float_as_uint((float)acc[t][e]) & 0x7FFFFFFFu); }
                     }
@@ -1447,11 +1554,13 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
             else { o[pidx] = (float)bias; nmax = max(nmax, __float_as_uint((float)bias) & 0x7FFFFFFFu); }
         }
     } else {
-        const int nout = sh.classes * (sh.hidden + 1);                       // W2 entries then b2
-        for (int t = threadIdx.x; t < nout; t += blockDim.x) {
+        const int nout = sh.classes * (sh.hidden + 1);                       // W2 entries then b2, one per thread
+        const int t = (int)(blockIdx.x - (sh.hidden + kMlpUnits - 1) / kMlpUnits) * (int)blockDim.x + (int)threadIdx.x;
+        if (t < nout) {
             const bool bias = t >= sh.classes * sh.hidden;
             const int c = bias ? t - sh.classes * sh.hidden : t / sh.hidden, jj = bias ? 0 : t % sh.hidden;
             double s = 0.0;
+#pragma unroll 4
             for (int r = 0; r < nrows; ++r) {
                 const int64_t q = r0 + r;
                 const double ta = dz_a ? (double)dz_a[q * sh.classes + c] * (bias ? 1.0 : act_a[q * sh.hidden + jj]) : 0.0;
@@ -1772,6 +1881,27 @@ static dim3 mlp_hidden_grid(int64_t nslots, const MlpShape& sh)
     return dim3((unsigned)((nslots + kMlpTile - 1) / kMlpTile), (unsigned)((sh.hidden + kThreads / 32 - 1) / (kThreads / 32)));
 }
 constexpr int kMlpGroup = 256;      // rows per block of the epoch-gradient sums
+static unsigned mlp_param_grid_x(const MlpShape& sh)
+{
+    return (unsigned)((sh.hidden + kMlpUnits - 1) / kMlpUnits + (sh.classes * (sh.hidden + 1) + kThreads - 1) / kThreads);
+}
+// Shared memory of mlp_output_kernel; *staged: both models' output layers fit beside the per-row scratch.
+static size_t mlp_output_smem(const MlpShape& sh, int* staged)
+{
+    const size_t base = sizeof(double) * (6 * (size_t)sh.classes + 2 * (size_t)sh.hidden);
+    const size_t w2 = sizeof(float) * 2 * ((size_t)sh.classes * sh.hidden + sh.classes);
+    *staged = base + w2 <= 48u * 1024u;
+    return base + (*staged ? w2 : 0);
+}
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static void launch_mlp_hidden(dq_ctx* ctx, int64_t nslots, const MlpShape& sh, const float* xa, const float* xb, const BatchSource& bs,
+                              int B, double* act_a, double* act_b, cudaStream_t st)
+{
+    const float* X = (const float*)ctx->data.values;
+    const bool vec = sh.in % 4 == 0 && aligned16(X) && aligned16(xa) && aligned16(xb);       // rows and weight rows on 16-byte boundaries
+    if (vec) launch_k(mlp_hidden_kernel<true>, mlp_hidden_grid(nslots, sh), kThreads, 0, st, X, sh, xa, xb, ctx->keys, bs, B, ctx->mlp_rows, act_a, act_b, nslots);
+    else launch_k(mlp_hidden_kernel<false>, mlp_hidden_grid(nslots, sh), kThreads, 0, st, X, sh, xa, xb, ctx->keys, bs, B, ctx->mlp_rows, act_a, act_b, nslots);
+}
 
 // g <- (1/n) sum_i grad loss_i(x) over all rows (double sums), via the "a" slots of the activation buffers.
 static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStream_t st)
@@ -1779,14 +1909,18 @@ static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStre
     const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
     const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
     const int64_t P = ctx->cfg.d;
-    launch_k(mlp_hidden_kernel, mlp_hidden_grid(D.n, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, x, nullptr, ctx->keys, none, 0,
-                                                                             ctx->mlp_rows, ctx->mlp_act[0], nullptr, (int64_t)D.n);
-    launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(double) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
-        nullptr, 1.0 / (double)D.n, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr);
+    launch_mlp_hidden(ctx, D.n, sh, x, nullptr, none, 0, ctx->mlp_act[0], nullptr, st);
+    int staged; const size_t osm = mlp_output_smem(sh, &staged);
+    launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, osm, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
+        nullptr, 1.0 / (double)D.n, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, staged);
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * P, st);
-    dim3 grid((sh.hidden + kMlpUnits - 1) / kMlpUnits + 1, (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
-    launch_k(mlp_param_kernel<true>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
-        ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
+    dim3 grid(mlp_param_grid_x(sh), (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
+    if (sh.in % 4 == 0 && aligned16(D.values))
+        launch_k(mlp_param_kernel<true, true>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
+            ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
+    else
+        launch_k(mlp_param_kernel<true, false>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, kMlpGroup, D.n,
+            ctx->mlp_act[0], nullptr, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, P, nullptr, ctx->g64);
     launch_k(finish_full_grad_kernel, blocks_for(P, ctx->sm_count), kThreads, 0, st, ctx->g64, P, 1.0, g);
     ctx->launches += 4;
 }
@@ -1798,14 +1932,18 @@ static void launch_mlp_worker_grad(dq_ctx* ctx, const float* xhat, const dq_stat
     const dq_config& c = ctx->cfg; const dq_data& D = ctx->data; const MlpShape sh = mlp_shape(ctx);
     const unsigned R = (unsigned)(c.M * c.B);
     uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
-    launch_k(mlp_hidden_kernel, mlp_hidden_grid(R, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, xhat, s->x_snap, ctx->keys, bs, c.B, ctx->mlp_rows,
-                                                                   ctx->mlp_act[0], ctx->mlp_act[1], (int64_t)R);
-    launch_k(mlp_output_kernel, R, kThreads, sizeof(double) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
-        ctx->mlp_act[1], 1.0 / (double)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr);
+    launch_mlp_hidden(ctx, R, sh, xhat, s->x_snap, bs, c.B, ctx->mlp_act[0], ctx->mlp_act[1], st);
+    int staged; const size_t osm = mlp_output_smem(sh, &staged);
+    launch_k(mlp_output_kernel, R, kThreads, osm, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
+        ctx->mlp_act[1], 1.0 / (double)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr, staged);
     if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
-    dim3 grid((sh.hidden + kMlpUnits - 1) / kMlpUnits + 1, c.M);
-    launch_k(mlp_param_kernel<false>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
-        ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
+    dim3 grid(mlp_param_grid_x(sh), c.M);
+    if (sh.in % 4 == 0 && aligned16(D.values))
+        launch_k(mlp_param_kernel<false, true>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
+            ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
+    else
+        launch_k(mlp_param_kernel<false, false>, grid, kThreads, 0, st, (const float*)D.values, sh, ctx->mlp_rows, c.B, (int64_t)R,
+            ctx->mlp_act[0], ctx->mlp_act[1], ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], alpha, c.d, nb, nullptr);
     ctx->launches += 3;
 }
 
@@ -2102,10 +2240,10 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
     if (c.model == DQ_MODEL_MLP) {
         const MlpShape sh = mlp_shape(ctx);
         const BatchSource none = {nullptr, nullptr, 0u, nullptr, 1, D.n, nullptr};
-        launch_k(mlp_hidden_kernel, mlp_hidden_grid(D.n, sh), kThreads, sizeof(float) * kMlpTile * sh.in, st, (const float*)D.values, sh, nullptr, x, ctx->keys, none, 0,
-                                                                                 ctx->mlp_rows, nullptr, ctx->mlp_act[1], (int64_t)D.n);
-        launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, sizeof(double) * 2 * sh.classes, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
-            ctx->mlp_act[1], 1.0 / (double)D.n, nullptr, nullptr, nullptr, nullptr, P);
+        launch_mlp_hidden(ctx, D.n, sh, nullptr, x, none, 0, nullptr, ctx->mlp_act[1], st);
+        int staged; const size_t osm = mlp_output_smem(sh, &staged);
+        launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, osm, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
+            ctx->mlp_act[1], 1.0 / (double)D.n, nullptr, nullptr, nullptr, nullptr, P, staged);
         launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
         ctx->launches += 3;
         return;
