@@ -200,6 +200,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     c->epoch = -1;
     if (fused_grad_setup(c) != DQ_OK) { dq_destroy(c); cudaGetLastError(); return DQ_ERR_CUDA; }
     small_round_setup(c);
+    sparse_message_setup(c);
     *out = c;
     return DQ_OK;
 }
@@ -209,7 +210,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->norm_block, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->delays_dev, c->slots_dev, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->acc64, c->rbuf, c->fused_part, c->fused_cnt, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->acc64, c->rbuf, c->fused_part, c->fused_cnt, c->ptouched, c->gtmp, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -387,9 +388,24 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     }
     ctx->xhat_diff = ring;                                   // the workers index the ring themselves
     ctx->use_slots = tau > 0;
+    // sparse gradients into sparse messages: one cluster kernel takes over from the worker kernel's accumulator
+    const bool msg_kernel = !flag && sparse_message_applies(ctx);
+    ctx->defer_list = msg_kernel;
     rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
+    ctx->defer_list = false;
     ctx->use_slots = false;
     ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = false;
+    if (msg_kernel && rc == DQ_OK) {
+        const BitsArgs bam = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag, 1, ctx->cfg.bx, ctx->cfg.b,
+                              (adaptive && !flag) ? ctx->bx_dev : nullptr};
+        launch_sparse_message(ctx, round, &ctx->msgs, as_stream(st));
+        ctx->sp_norms_zeroed = false;
+        ctx->tile_ptr_ready = true;
+        launch_master(ctx, &ctx->msgs, true, s, eta, theta, as_stream(st), (bits_down || bits_up) ? &bam : nullptr);
+        ctx->tile_ptr_ready = false;
+        ctx->list_ready = false; ctx->normx_zeroed = false;
+        return last_error();
+    }
     const BitsArgs ba = {bits_down ? bits_down : ctx->bits, bits_up ? bits_up : ctx->bits + 1, ctx->msgs.nnz, flag,
                          sparse_messages(ctx) ? 1 : 0, ctx->cfg.bx, ctx->cfg.b, (adaptive && !flag) ? ctx->bx_dev : nullptr};
     // dense messages and an averaged master: quantiser and master step share one kernel (the codes would only travel

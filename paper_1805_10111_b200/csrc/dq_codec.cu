@@ -1229,7 +1229,7 @@ count_touched_kernel(const uint32_t* __restrict__ touched, int64_t bm_words, uin
 }
 
 __global__ void __launch_bounds__(kThreads)
-build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const uint32_t* __restrict__ seg_count, int nseg,
+build_group_list_kernel(uint32_t* __restrict__ touched, uint32_t* __restrict__ ptouched /* may be NULL */, int64_t bm_words, const uint32_t* __restrict__ seg_count, int nseg,
                         FixedAcc fa, float* __restrict__ alpha, int64_t d,
                         uint32_t* __restrict__ glist, int64_t cap, uint32_t* __restrict__ gcount, uint32_t* __restrict__ norm_bits)
 {
@@ -1249,7 +1249,10 @@ build_group_list_kernel(uint32_t* __restrict__ touched, int64_t bm_words, const 
     if ((threadIdx.x & 31) == 0) s_base[threadIdx.x >> 5] = part;
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t word = 0;
-    if (i < bm_words) { word = bm[i]; if (word) bm[i] = 0u; }
+    if (i < bm_words) {
+        word = bm[i]; if (word) bm[i] = 0u;
+        if (ptouched) ptouched[(int64_t)w * bm_words + i] = word;      // kept for the kernel that works from bitmaps (sparse_message_kernel)
+    }
     const uint32_t c = __popc(word);
     uint32_t incl = c;
 #pragma unroll
@@ -1291,6 +1294,329 @@ clear_listed_groups_kernel(float* __restrict__ alpha, int64_t d, const uint32_t*
         const int64_t i0 = (int64_t)glist[(int64_t)w * cap + p] << 3;
 #pragma unroll
         for (int j = 0; j < 8; ++j) if (i0 + j < d) row[i0 + j] = 0.0f;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Sparse gradient -> sparse message in one kernel (CSR data, sparsifier of eq. (4), (position, code) messages).
+// From the integer accumulator and the bitmap of touched groups that the worker kernel leaves behind to the
+// finished message of Section 3.1 and the master's tile pointers; the steps are those of the stand-alone kernels
+// (list of touched groups, alpha and ||alpha||_inf, integer-grid ||alpha||_1, survivor mask, ||beta||_inf, quantise
+// and emit in ascending order) with the same draws and arithmetic.  A worker is served by a thread-block cluster
+// of kMsgCluster blocks, each owning a range of the bitmap and the groups listed in it.  A round touches a few
+// thousand groups per worker, so the kernel's time is a chain of memory round trips: a block keeps its groups'
+// numbers in shared memory and (up to kMsgKeep groups per thread) their values in registers, so that only the
+// accumulator is read from memory; the three points where a step needs a value over the whole worker (list length
+// with ||alpha||_inf, ||alpha||_1, survivor counts with ||beta||_inf) are cluster barriers, with the blocks'
+// partial values written into each other's shared memory.  A block with more groups than it can keep re-reads
+// them (group numbers from a scratch list, values from alpha).
+// grid (kMsgCluster, M), cluster (kMsgCluster, 1, 1), kMsgThreads threads.
+// ---------------------------------------------------------------------------------------------------
+constexpr int kMsgCluster = 8;
+constexpr int kMsgThreads = 512;
+constexpr int kMsgKeep = 2;                       // groups per thread whose values stay in registers
+
+struct SparseMsg {
+    uint32_t* touched; uint32_t* ptouched; int64_t bm_words;    // [M][bm_words] bitmaps of touched groups: this round's (cleared here) and
+                                                  // the previous round's (whose groups get their zeros back; replaced by this round's)
+    FixedAcc fa;                                  // integer accumulator (zeroed again here)
+    float* alpha; int64_t d;                      // [M][d] receives alpha_w; zero outside the listed groups
+    uint32_t* glist; uint32_t* gtmp; int64_t gcap; uint32_t* gcount;   // ascending list of touched groups (out), scratch of the same size
+    uint32_t* norm_bits; unsigned long long* l1_sum; uint32_t* beta_norm_bits;     // [M] each, written here
+    float phi; uint32_t round; const RoundParams* rp;
+    uint8_t* codes; int64_t stride; float* scale; uint32_t* idx; int64_t cap; uint32_t* nnz;    // the messages
+    uint32_t* tile_ptr; int64_t ntiles;           // [M][ntiles + 1] first list entry of every tile of kChunk coordinates
+    int* status;
+};
+
+template <int BITS>
+__global__ void __launch_bounds__(kMsgThreads, 1)
+sparse_message_kernel(const __grid_constant__ SparseMsg A, const __grid_constant__ PhiloxKeys K)
+{
+    pdl_prologue();
+    constexpr int NW = kMsgThreads / 32, kKeepCap = kMsgKeep * kMsgThreads;
+    const int w = blockIdx.y, r = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ uint32_t s_scan[NW];
+    __shared__ unsigned long long s_red[NW];
+    __shared__ uint32_t s_list[kKeepCap];
+    __shared__ __align__(16) unsigned long long s_ex[3][kMsgCluster][2];      // written by the cluster's blocks, one pair each
+    const uint32_t round = A.rp ? A.rp->round : A.round;
+    const int64_t d = A.d;
+    uint32_t* bm = A.touched + (int64_t)w * A.bm_words;
+    uint32_t* pbm = A.ptouched + (int64_t)w * A.bm_words;
+    float* row = A.alpha + (int64_t)w * d;
+    long long* acc = A.fa.acc + (int64_t)w * d;
+    const bool vec = (d & 7) == 0;                            // every group of a row starts on a 32-byte boundary
+
+    // sum or maximum of one value per thread over the block (every thread gets the result)
+    auto block_reduce = [&](unsigned long long v, bool is_max) -> unsigned long long {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { const unsigned long long t = __shfl_xor_sync(0xFFFFFFFFu, v, o); v = is_max ? (t > v ? t : v) : v + t; }
+        if (lane == 0) s_red[warp] = v;
+        __syncthreads();
+        unsigned long long tot = 0;
+        for (int k = 0; k < NW; ++k) tot = is_max ? (s_red[k] > tot ? s_red[k] : tot) : tot + s_red[k];
+        __syncthreads();
+        return tot;
+    };
+    // exclusive prefix of one count per thread in thread order, and the block's total
+    auto block_scan = [&](uint32_t c, uint32_t& total) -> uint32_t {
+        uint32_t incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+        if (lane == 31) s_scan[warp] = incl;
+        __syncthreads();
+        uint32_t base = 0, tot = 0;
+        for (int k = 0; k < NW; ++k) { const uint32_t t = s_scan[k]; if (k < warp) base += t; tot += t; }
+        __syncthreads();
+        total = tot;
+        return base + incl - c;
+    };
+    // every block hands its pair (v0, v1) to all blocks of the cluster (slot = which of the three meetings)
+    unsigned long long all0[kMsgCluster], all1[kMsgCluster];
+    auto exchange = [&](int slot, unsigned long long v0, unsigned long long v1) {
+        if (tid < kMsgCluster) {
+            const uint32_t local = (uint32_t)__cvta_generic_to_shared(&s_ex[slot][r][0]);
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(tid));
+            asm volatile("st.shared::cluster.v2.u64 [%0], {%1, %2};" :: "r"(remote), "l"(v0), "l"(v1) : "memory");
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+#pragma unroll
+        for (int k = 0; k < kMsgCluster; ++k) { all0[k] = s_ex[slot][k][0]; all1[k] = s_ex[slot][k][1]; }
+    };
+    // alpha is written in this kernel: no read-only path for its loads
+    auto load_group = [&](int64_t i0, float (&a)[8]) {
+        if (vec) { load8_rw(row + i0, a); return; }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a[j] = (i0 + j < d) ? *reinterpret_cast<volatile float*>(row + i0 + j) : 0.0f;
+    };
+
+    // ---- 0: zero this worker's code words; in this block's range of the bitmaps: zeros back into the groups of the
+    //         previous round, this round's groups to the block's list, bitmaps rolled over
+    {
+        uint4* c16 = reinterpret_cast<uint4*>(A.codes + (int64_t)w * A.stride);            // stride is a multiple of 16
+        for (int64_t q = (int64_t)r * kMsgThreads + tid; q < (A.stride >> 4); q += kMsgCluster * kMsgThreads) c16[q] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    const int64_t wpb = (A.bm_words + kMsgCluster - 1) / kMsgCluster;
+    const int64_t w0 = (int64_t)r * wpb, w1 = min(A.bm_words, w0 + wpb);
+    uint32_t* tmp = A.gtmp + (int64_t)w * A.gcap + (w0 << 5);           // this block's scratch list: it has at most 32 groups per word
+    uint32_t cl = 0;                                          // groups listed by this block
+    for (int64_t i = w0; i < w1; i += kMsgThreads) {
+        const int64_t wi = i + tid;
+        uint32_t word = 0, old = 0;
+        if (wi < w1) { word = bm[wi]; old = pbm[wi]; }
+        if (word != old) pbm[wi] = word;
+        if (word) bm[wi] = 0u;
+        while (old) {
+            const int bit = __ffs(old) - 1; old &= old - 1;
+            const int64_t i0 = ((wi << 5) + bit) << 3;
+            if (vec) { float4* q = reinterpret_cast<float4*>(row + i0); q[0] = make_float4(0.f, 0.f, 0.f, 0.f); q[1] = make_float4(0.f, 0.f, 0.f, 0.f); }
+            else for (int j = 0; j < 8; ++j) if (i0 + j < d) row[i0 + j] = 0.0f;
+        }
+        uint32_t total;
+        uint32_t pos = cl + block_scan(__popc(word), total);
+        while (word) {
+            const int bit = __ffs(word) - 1; word &= word - 1;
+            const uint32_t g = (uint32_t)((wi << 5) + bit);
+            if (pos < (uint32_t)kKeepCap) s_list[pos] = g;
+            tmp[pos++] = g;
+        }
+        cl += total;
+    }
+    __syncthreads();                                          // the zeros are in place before alpha is stored; the list is complete
+    const bool keep = cl <= (uint32_t)kKeepCap;               // this block's groups fit shared memory and registers
+    const uint32_t g_last = cl ? (keep ? s_list[cl - 1] : __ldcg(tmp + cl - 1)) : 0u;
+    auto group_at_entry = [&](uint32_t e) -> uint32_t { return keep ? s_list[e] : __ldcg(tmp + e); };
+
+    // ---- 1: accumulator -> alpha (one rounding to fp32), accumulator zeroed, ||alpha||_inf
+    float ka[kMsgKeep][8];
+    uint32_t kg[kMsgKeep], kmask[kMsgKeep];
+    uint32_t amax = 0;
+    auto make_alpha = [&](uint32_t g, float (&a)[8]) {
+        const int64_t i0 = (int64_t)g << 3;
+        long long q[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) q[j] = (i0 + j < d) ? acc[i0 + j] : 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (q[j] != 0) acc[i0 + j] = 0;
+            a[j] = (float)((double)q[j] * A.fa.inv_scale);
+            amax = max(amax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
+        }
+        if (vec) {
+            float4* o = reinterpret_cast<float4*>(row + i0);
+            o[0] = make_float4(a[0], a[1], a[2], a[3]); o[1] = make_float4(a[4], a[5], a[6], a[7]);
+        } else {
+            for (int j = 0; j < 8; ++j) if (i0 + j < d) row[i0 + j] = a[j];
+        }
+    };
+    if (keep) {
+#pragma unroll
+        for (int k = 0; k < kMsgKeep; ++k) {
+            const uint32_t e = tid + k * kMsgThreads;
+            kg[k] = 0; kmask[k] = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) ka[k][j] = 0.0f;
+            if (e < cl) { kg[k] = s_list[e]; make_alpha(kg[k], ka[k]); }
+        }
+    } else {
+        for (uint32_t e = tid; e < cl; e += kMsgThreads) { float a[8]; make_alpha(__ldcg(tmp + e), a); }
+    }
+    exchange(0, ((unsigned long long)cl << 32) | block_reduce(amax, true), g_last);
+    uint32_t base = 0, count = 0, nb = 0;
+    int64_t t_before = -1;                                    // tile of the last group listed by a block before this one
+    bool last_block = true;                                   // no block after this one lists a group
+#pragma unroll
+    for (int k = 0; k < kMsgCluster; ++k) {
+        const uint32_t c = (uint32_t)(all0[k] >> 32);
+        if (k < r) { base += c; if (c) t_before = (int64_t)((uint32_t)all1[k] >> 8); }
+        if (k > r && c) last_block = false;
+        count += c; nb = max(nb, (uint32_t)all0[k]);
+    }
+    {   // the worker's list: this block's groups after those of the blocks before it
+        uint32_t* list = A.glist + (int64_t)w * A.gcap + base;
+        for (uint32_t e = tid; e < cl; e += kMsgThreads) list[e] = group_at_entry(e);
+        if (r == 0 && tid == 0) { A.gcount[w] = count; A.norm_bits[w] = nb; }
+    }
+
+    // ---- 2: ||alpha||_1 on the integer grid of ||alpha||_inf's exponent
+    unsigned long long l1 = 0;
+    if (nb != 0u && nb < 0x7F800000u) {
+        int ee; (void)frexpf(__uint_as_float(nb), &ee);
+        if (keep) {
+#pragma unroll
+            for (int k = 0; k < kMsgKeep; ++k)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) l1 += l1_term(ka[k][j], ee);              // (entries beyond the list hold zeros)
+        } else {
+            for (uint32_t e = tid; e < cl; e += kMsgThreads) {
+                float a[8]; load_group((int64_t)__ldcg(tmp + e) << 3, a);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) l1 += l1_term(a[j], ee);
+            }
+        }
+    }
+    exchange(1, block_reduce(l1, false), 0ull);
+    l1 = 0;
+#pragma unroll
+    for (int k = 0; k < kMsgCluster; ++k) l1 += all0[k];
+    if (r == 0 && tid == 0) A.l1_sum[w] = l1;
+    const SparsifyScale sc = sparsify_scale(nb, l1, A.phi);
+
+    // ---- 3: survivor mask of every listed group: survivors and ||beta||_inf
+    uint32_t nsurv = 0, bmax = 0;
+    auto draw_mask = [&](uint32_t g, const float (&a)[8], float (&beta)[8]) -> uint32_t {
+        uint32_t rr[4];
+        philox4x32_10(g, round, (uint32_t)w, kStreamMask, K, rr);
+        return sparsify8(a, sc.s, rr, beta);
+    };
+    auto count_mask = [&](uint32_t mask, const float (&beta)[8]) {
+        if (mask) {
+            nsurv += __popc(mask);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) bmax = max(bmax, __float_as_uint(beta[j]) & 0x7FFFFFFFu);
+        }
+    };
+    if (!sc.empty) {
+        if (keep) {
+#pragma unroll
+            for (int k = 0; k < kMsgKeep; ++k) {
+                if (tid + k * kMsgThreads < cl) {
+                    float beta[8];
+                    kmask[k] = draw_mask(kg[k], ka[k], beta);
+                    count_mask(kmask[k], beta);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) ka[k][j] = beta[j];               // from here on the registers hold beta
+                }
+            }
+        } else {
+            for (uint32_t e = tid; e < cl; e += kMsgThreads) {
+                const uint32_t g = __ldcg(tmp + e);
+                float a[8], beta[8]; load_group((int64_t)g << 3, a);
+                count_mask(draw_mask(g, a, beta), beta);
+            }
+        }
+    }
+    exchange(2, (block_reduce(nsurv, false) << 32) | block_reduce(bmax, true), 0ull);
+    uint32_t offset = 0, total = 0, bb = 0;
+#pragma unroll
+    for (int k = 0; k < kMsgCluster; ++k) {
+        const uint32_t c = (uint32_t)(all0[k] >> 32);
+        if (k < r) offset += c;
+        total += c; bb = max(bb, (uint32_t)all0[k]);
+    }
+    const bool finite = bb < 0x7F800000u && nb < 0x7F800000u;
+    const float bnrm = __uint_as_float(bb);
+    const float inv = (finite && bb != 0u) ? __fdiv_rd((float)levels(BITS), bnrm) : 0.0f;
+    const uint32_t nnzc = (int64_t)total > A.cap ? (uint32_t)A.cap : total;
+    if (r == 0 && tid == 0) {
+        A.beta_norm_bits[w] = bb;
+        A.scale[w] = (finite && bb != 0u) ? __fdiv_rn(bnrm, (float)levels(BITS)) : 0.0f;
+        A.nnz[w] = nnzc;
+        if (!finite) set_status(A.status, DQ_ERR_NONFINITE);
+        if ((int64_t)total > A.cap) set_status(A.status, DQ_ERR_CAPACITY);
+    }
+
+    // ---- 4: quantise the survivors (delta = ||beta||_inf / L, rounding draw keyed by the coordinate) and emit
+    //         (position, code) in ascending order; the master's tile pointers from neighbouring groups
+    uint8_t* out = A.codes + (int64_t)w * A.stride;
+    uint32_t* oidx = A.idx + (int64_t)w * A.cap;
+    uint32_t* tp = A.tile_ptr + (int64_t)w * (A.ntiles + 1);
+    constexpr int kTileShift = 8;                             // kChunk coordinates = 256 groups
+    static_assert(kChunk == 8 << kTileShift, "tile of kChunk coordinates");
+    if (count == 0) {
+        for (int64_t t = (int64_t)r * kMsgThreads + tid; t <= A.ntiles; t += kMsgCluster * kMsgThreads) tp[t] = 0u;
+        return;
+    }
+    auto emit = [&](uint32_t e, uint32_t g, uint32_t mask, const float (&beta)[8], uint32_t p) {
+        // tiles that begin between the previous group and this one start at this group's first survivor
+        const int64_t t_cur = g >> kTileShift, t_prev = e > 0 ? (int64_t)(group_at_entry(e - 1) >> kTileShift) : t_before;
+        const uint32_t pc = p < nnzc ? p : nnzc;
+        for (int64_t t = t_prev + 1; t <= t_cur; ++t) tp[t] = pc;
+        if (last_block && e == cl - 1) for (int64_t t = t_cur + 1; t <= A.ntiles; ++t) tp[t] = nnzc;
+        if (!mask) return;
+        uint32_t rr[4];
+        philox4x32_10(g, round, (uint32_t)w, kStreamGrad, K, rr);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if ((mask >> j) & 1u) {
+                if ((int64_t)p < A.cap) {
+                    const uint32_t s8 = round_fixed<BITS>(beta[j], inv, half16(rr, j));
+                    oidx[p] = (g << 3) + (uint32_t)j;
+                    const uint32_t field = ((s8 >> 16) ^ (BITS == 8 ? 0x80u : 0u)) & ((1u << BITS) - 1u);
+                    const int64_t bit = (int64_t)p * BITS;
+                    atomicOr(reinterpret_cast<uint32_t*>(out) + (bit >> 5), field << (bit & 31));
+                }
+                ++p;
+            }
+        }
+    };
+    uint32_t run = offset;
+    if (keep) {
+#pragma unroll
+        for (int k = 0; k < kMsgKeep; ++k) {
+            if ((uint32_t)(k * kMsgThreads) >= cl) break;             // (the same for the whole block)
+            const uint32_t e = tid + k * kMsgThreads;
+            uint32_t tile_total;
+            const uint32_t p = run + block_scan(__popc(kmask[k]), tile_total);
+            run += tile_total;
+            if (e < cl) emit(e, kg[k], kmask[k], ka[k], p);
+        }
+    } else {
+        for (uint32_t eb = 0; eb < cl; eb += kMsgThreads) {
+            const uint32_t e = eb + tid;
+            uint32_t g = 0, mask = 0;
+            float beta[8];
+            if (e < cl) {
+                g = __ldcg(tmp + e);
+                if (!sc.empty) { float a[8]; load_group((int64_t)g << 3, a); mask = draw_mask(g, a, beta); }
+            }
+            uint32_t tile_total;
+            const uint32_t p = run + block_scan(__popc(mask), tile_total);
+            run += tile_total;
+            if (e < cl) emit(e, g, mask, beta, p);
+        }
     }
 }
 
@@ -1509,10 +1835,9 @@ void launch_build_group_list(dq_ctx* ctx, uint32_t* norm_bits, cudaStream_t st)
     dim3 grid(nseg, c.M);
     launch_k(count_touched_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg);
     const FixedAcc fa = {ctx->acc64, ctx->acc_scale, ctx->acc_inv};
-    launch_k(build_group_list_kernel, grid, kThreads, 0, st, ctx->touched, ctx->bm_words, ctx->seg_count, nseg, fa, ctx->alpha, c.d,
+    launch_k(build_group_list_kernel, grid, kThreads, 0, st, ctx->touched, ctx->ptouched, ctx->bm_words, ctx->seg_count, nseg, fa, ctx->alpha, c.d,
                                                         ctx->glist, ctx->glist_cap, ctx->gcount, norm_bits);
     ctx->launches += 2;
-    ctx->launches += 1;
 }
 
 void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bits, const uint32_t* norm_bits,
@@ -1571,6 +1896,49 @@ void launch_sparsify_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
             flags, M)));
         ctx->launches += 2;
     }
+}
+
+// One cluster kernel from the CSR worker kernel's accumulator to the sparse messages and the master's tile pointers.
+void sparse_message_setup(dq_ctx* ctx)
+{
+    ctx->msg_cluster = false;
+    const dq_config& c = ctx->cfg;
+    if (!ctx->list_mode || c.no_fused || (c.b != 2 && c.b != 4 && c.b != 8)) return;
+    const size_t bm_bytes = sizeof(uint32_t) * (size_t)c.M * ctx->bm_words, list_bytes = sizeof(uint32_t) * (size_t)c.M * ctx->glist_cap;
+    if (cudaMalloc(&ctx->ptouched, bm_bytes) != cudaSuccess || cudaMalloc(&ctx->gtmp, list_bytes) != cudaSuccess ||
+        cudaMemset(ctx->ptouched, 0, bm_bytes) != cudaSuccess) {
+        cudaFree(ctx->ptouched); cudaFree(ctx->gtmp); ctx->ptouched = nullptr; ctx->gtmp = nullptr; cudaGetLastError(); return;
+    }
+    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{}; cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kMsgCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(kMsgCluster, (unsigned)c.M); cfg.blockDim = dim3(kMsgThreads); cfg.attrs = attr; cfg.numAttrs = 1;
+    int nclusters = 0;
+    cudaError_t e = cudaErrorInvalidValue;
+    DQ_DISPATCH_BITS(c.b, (e = cudaOccupancyMaxActiveClusters(&nclusters, sparse_message_kernel<BITS_>, &cfg)));
+    if (e == cudaSuccess && nclusters >= 1) ctx->msg_cluster = true; else cudaGetLastError();
+}
+
+bool sparse_message_applies(const dq_ctx* ctx) { return ctx->msg_cluster && ctx->list_mode && ctx->cfg.sparsify && ctx->msgs.idx != nullptr; }
+
+void launch_sparse_message(dq_ctx* ctx, uint32_t round, const dq_msgs* out, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg;
+    SparseMsg A;
+    A.touched = ctx->touched; A.ptouched = ctx->ptouched; A.bm_words = ctx->bm_words; A.fa = FixedAcc{ctx->acc64, ctx->acc_scale, ctx->acc_inv};
+    A.alpha = ctx->alpha; A.d = c.d; A.glist = ctx->glist; A.gtmp = ctx->gtmp; A.gcap = ctx->glist_cap; A.gcount = ctx->gcount;
+    A.norm_bits = reinterpret_cast<uint32_t*>(ctx->ninf); A.l1_sum = ctx->l1_sum; A.beta_norm_bits = ctx->beta_norm_bits;
+    A.phi = c.phi; A.round = round; A.rp = ctx->rp_active;
+    A.codes = out->codes; A.stride = out->stride; A.scale = out->scale; A.idx = out->idx; A.cap = out->cap; A.nnz = out->nnz;
+    A.tile_ptr = ctx->tile_ptr; A.ntiles = ctx->nchunks; A.status = ctx->status;
+    cudaLaunchConfig_t cfg = cudaLaunchConfig_t{}; cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = kMsgCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(kMsgCluster, (unsigned)c.M); cfg.blockDim = dim3(kMsgThreads); cfg.stream = st; cfg.attrs = attr; cfg.numAttrs = 2;
+    DQ_DISPATCH_BITS(c.b, (cudaLaunchKernelEx(&cfg, sparse_message_kernel<BITS_>, A, ctx->keys)));
+    ctx->launches += 1;
 }
 
 // Quantiser and master step of a round in one kernel (dense messages, averaged master): the context's message buffers
@@ -1645,7 +2013,8 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
     } else {
         const int64_t ntiles = (d + kChunk - 1) / kChunk;
         dim3 grid_t((unsigned)((ntiles + 1 + kThreads - 1) / kThreads), c.M);
-        launch_k(tile_ptr_kernel, grid_t, kThreads, 0, st, msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
+        const int tp_launch = ctx->tile_ptr_ready ? 0 : 1;      // the message kernel may have written the tile pointers already
+        if (tp_launch) launch_k(tile_ptr_kernel, grid_t, kThreads, 0, st, msgs->idx, msgs->cap, msgs->nnz, ntiles, ctx->tile_ptr);
         if (c.sequential) {
             const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
             if (c.accelerated) {
@@ -1655,7 +2024,7 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
                 DQ_DISPATCH_BITS(c.b, (launch_k(master_sparse_seq_kernel<BITS_, false>, grid, kThreads, sizeof(uint32_t) * 2 * c.M, st, msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                     s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
             }
-            ctx->launches += 2;
+            ctx->launches += 1 + tp_launch;
             return;
         }
         const int grid = (int)(ntiles < (int64_t)ctx->sm_count * 8 ? ntiles : (int64_t)ctx->sm_count * 8);
@@ -1666,7 +2035,7 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
             DQ_DISPATCH_BITS(c.b, (launch_k(master_sparse_kernel<BITS_, false>, grid, kThreads, sizeof(uint32_t) * 2 * c.M, st, msgs->codes, msgs->stride, msgs->scale, msgs->idx, msgs->cap, ctx->tile_ptr, ntiles, c.M, d, s->g_full, s->x,
                 s->y, s->x_snap, s->x_sum, eta, theta, pp, nx, ctx->rp_active, ba)));
         }
-        ctx->launches += 2;
+        ctx->launches += 1 + tp_launch;
     }
 }
 

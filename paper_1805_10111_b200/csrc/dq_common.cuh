@@ -319,6 +319,11 @@ struct dq_ctx {
     int cluster_blocks;         // blocks of the one-cluster round kernel for small problems; 0: rounds run as separate kernels
     bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only
     bool list_ready;            // the list of this round has been built (consumed by the sparsifier launch)
+    bool msg_cluster;           // sparse gradients become sparse messages in one cluster kernel (sparse_message_kernel)
+    bool defer_list;            // set while dq_round enqueues such a round: the worker kernel leaves list, alpha and norm to it
+    bool tile_ptr_ready;        // set while dq_round enqueues such a round: the master's tile pointers are already written
+    uint32_t* ptouched;         // [M][bm_words] the previous round's bitmap (the groups of alpha that are not zero)
+    uint32_t* gtmp;             // [M][glist_cap] per-block scratch lists of that kernel
     bool alpha_zeroed, ninf_zeroed, normx_zeroed;   // an earlier kernel of this round already cleared these
     bool diff_ready;            // the model-quantise kernel of this round already wrote xhat - xsnap
     // bookkeeping

@@ -2090,9 +2090,10 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         cudaMemsetAsync(alpha, 0, sizeof(float) * c.M * c.d, st);
         cudaMemsetAsync(norm_inf, 0, sizeof(float) * c.M, st);
         if (list) cudaMemsetAsync(ctx->gcount, 0, sizeof(uint32_t) * c.M, st);
+        if (list && ctx->ptouched) cudaMemsetAsync(ctx->ptouched, 0, sizeof(uint32_t) * c.M * ctx->bm_words, st);
         return;
     }
-    if (list) launch_clear_listed(ctx, st);                      // alpha is all-zero again before this round adds to it
+    if (list && !ctx->defer_list) launch_clear_listed(ctx, st);  // alpha is all-zero again before this round adds to it
     const BatchSource bs = {batch_idx, batch_idx ? nullptr : ctx->rows, round, ctx->rp_active, c.M, D.n,
                             ctx->normx_zeroed ? reinterpret_cast<uint32_t*>(s->norm_x) : nullptr,
                             ctx->use_slots ? ctx->slots_dev : nullptr, c.d};
@@ -2111,6 +2112,7 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
         launch_k(worker_grad_csr_kernel, (int)(((int64_t)c.M * c.B * 32 + kThreads - 1) / kThreads), kThreads, 0, st, (const float*)D.values, D.col_idx, D.row_ptr, D.labels, ctx->xhat_diff, s->z_snap, ctx->keys, bs, c.M, c.B, c.d, fa,
             list ? ctx->touched : nullptr, ctx->bm_words);
         ctx->launches += 1;
+        if (list && ctx->defer_list) return;                 // the message kernel turns bitmap and accumulator into list, alpha and norm
         if (list) { launch_build_group_list(ctx, reinterpret_cast<uint32_t*>(norm_inf), st); ctx->list_ready = true; return; }
         uint32_t* nb = reinterpret_cast<uint32_t*>(norm_inf);
         if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);

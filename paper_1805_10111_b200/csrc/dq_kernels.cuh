@@ -31,6 +31,9 @@ void launch_worker_grad(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_
                         uint32_t round, const int32_t* batch_idx, float* alpha, float* norm_inf, cudaStream_t st);
 bool worker_accumulates(const dq_ctx* ctx);
 int fused_grad_setup(dq_ctx* ctx);
+void sparse_message_setup(dq_ctx* ctx);
+bool sparse_message_applies(const dq_ctx* ctx);
+void launch_sparse_message(dq_ctx* ctx, uint32_t round, const dq_msgs* out, cudaStream_t st);
 bool fused_grad_applies(const dq_ctx* ctx);
 bool fused_round_applies(const dq_ctx* ctx);
 void launch_fused_round(dq_ctx* ctx, dq_state* s, uint32_t round, cudaStream_t st);
