@@ -1312,7 +1312,7 @@ clear_listed_groups_kernel(float* __restrict__ alpha, int64_t d, const uint32_t*
 // them (group numbers from a scratch list, values from alpha).
 // grid (kMsgCluster, M), cluster (kMsgCluster, 1, 1), kMsgThreads threads.
 // ---------------------------------------------------------------------------------------------------
-constexpr int kMsgCluster = 8;
+constexpr int kMsgCluster = 4;
 constexpr int kMsgThreads = 512;
 constexpr int kMsgKeep = 2;                       // groups per thread whose values stay in registers
 
@@ -1440,9 +1440,12 @@ sparse_message_kernel(const __grid_constant__ SparseMsg A, const __grid_constant
         for (int j = 0; j < 8; ++j) q[j] = (i0 + j < d) ? acc[i0 + j] : 0;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            if (q[j] != 0) acc[i0 + j] = 0;
-            a[j] = (float)((double)q[j] * A.fa.inv_scale);
-            amax = max(amax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
+            a[j] = 0.0f;
+            if (q[j] != 0) {                                  // (most coordinates of a touched group are untouched)
+                acc[i0 + j] = 0;
+                a[j] = (float)((double)q[j] * A.fa.inv_scale);
+                amax = max(amax, __float_as_uint(a[j]) & 0x7FFFFFFFu);
+            }
         }
         if (vec) {
             float4* o = reinterpret_cast<float4*>(row + i0);
