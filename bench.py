@@ -64,7 +64,7 @@ def parse_args():
     ap.add_argument("--tensor-cores", type=int, default=0, help="training configurations: dq_config.tensor_cores (1: both products of the "
                                                                 "dense bf16 gradient as MMAs, 2: the margins only)")
     ap.add_argument("--no-fused", type=int, default=0, help="training configurations: dq_config.no_fused")
-    ap.add_argument("--configs", default="c1,c2,c3,c4,nn", help="training configurations to time with dq_rounds ('' for none)")
+    ap.add_argument("--configs", default="c1,c2,c2_tau3,c3,c4,nn", help="training configurations to time with dq_rounds ('' for none)")
     return ap.parse_args()
 
 
@@ -265,6 +265,9 @@ def stage_report(ms_list, alg, peak):
 TRAIN_CONFIGS = {
     "c1": dict(gen="config1", kw=dict(M=4, B=16, bx=8, b=8, lambda1=1e-4), lr=1.0, theta=0.0, m=200),
     "c2": dict(gen="config2", kw=dict(M=8, B=64, bx=8, b=4, lambda2=1e-5), lr=1.0, theta=0.0, m=200),
+    # the same rounds with workers that lag 0..3 rounds behind the master (Algorithm 1 step 11, x_{D(t)}): what delays cost
+    "c2_tau3": dict(gen="config2", kw=dict(M=8, B=64, bx=8, b=4, lambda2=1e-5, max_delay=3), lr=1.0, theta=0.0, m=200,
+                    delays=[0, 1, 2, 3, 0, 1, 2, 3]),
     # sparse_cap: a message holds at most B * nnz/row = 12,800 entries here; the default capacity (d) would have the
     # round clear 8 MiB of code buffers for a few hundred bytes of codes
     "c3": dict(gen="config3", kw=dict(M=16, B=128, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1,
@@ -349,6 +352,8 @@ def time_training_config(name, rounds=200, warmup=20, with_oracle=False, peak=No
     cfg = dq.make_config(x0.size, spec["kw"]["M"], seed=SEED, **{k: v for k, v in spec["kw"].items() if k != "M"}, **(extra or {}))
     data = dq.Data(h)
     rc, ctx = dq.dq_create(cfg, data); dq.ok(rc, "dq_create " + name)
+    if spec.get("delays"):
+        dq.ok(dq.dq_set_delays(ctx, spec["delays"]))
     st = dq.State(x0, n=h.n, accelerated=bool(cfg.accelerated))
     theta = spec["theta"]; eta = spec["lr"] / theta if theta else spec["lr"]
     bits = torch.zeros(2, dtype=torch.int64, device="cuda")
@@ -372,7 +377,7 @@ def time_training_config(name, rounds=200, warmup=20, with_oracle=False, peak=No
     rc, status = dq.dq_poll_status(ctx)
     out["device_status"] = status
     dq.dq_destroy(ctx)
-    if with_oracle:
+    if with_oracle and not spec.get("delays"):       # the CPU figure is taken without delays (they change no arithmetic cost there)
         out["cpu_oracle"] = oracle_training_rounds_per_sec(h, spec, x0)
     return out
 

@@ -361,7 +361,9 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     float* const ring = ctx->xhat_diff;
     if (tau > 0) {
         const int t = (int)ctx->rounds_in_epoch;
-        ctx->xhat_diff = ring + (int64_t)(t % (tau + 1)) * ctx->cfg.d;
+        // while a round is captured for replay the kernels take the epoch's round counter from the device instead
+        if (ctx->rp_active) ctx->diff_ring = tau + 1;
+        else ctx->xhat_diff = ring + (int64_t)(t % (tau + 1)) * ctx->cfg.d;
         if (flag) cudaMemsetAsync(ctx->xhat_diff, 0, sizeof(float) * ctx->cfg.d, as_stream(st));   // xhat = xsnap
         launch_set_slots(ctx, t, as_stream(st));
     }
@@ -387,6 +389,7 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
         cudaMemsetAsync(ctx->bx_dev, 0, sizeof(int32_t), as_stream(st));
     }
     ctx->xhat_diff = ring;                                   // the workers index the ring themselves
+    ctx->diff_ring = 0;
     ctx->use_slots = tau > 0;
     // sparse gradients into sparse messages: one cluster kernel takes over from the worker kernel's accumulator
     const bool msg_kernel = !flag && sparse_message_applies(ctx);
@@ -465,7 +468,7 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
         return last_error();
     }
     bool replayed = false;
-    if (!flag && !ctx->graph_off && !c.no_graph && c.max_delay == 0) {
+    if (!flag && !ctx->graph_off && !c.no_graph) {
         const dq_state& g = ctx->graph_state;
         const bool same = ctx->graph_exec && g.x == s->x && g.x_snap == s->x_snap && g.g_full == s->g_full && g.y == s->y &&
                           g.x_sum == s->x_sum && g.norm_x == s->norm_x && g.z_snap == s->z_snap &&
@@ -475,10 +478,12 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
             cudaStream_t st = as_stream(stream);
             // the round's last kernel advances the round number on the device: only a jump in the numbering or new
             // step sizes need the launch that sets them (scalars travel as kernel arguments: no host buffer to keep alive)
-            if (!(ctx->rp_host_valid && ctx->rp_host.round == round && ctx->rp_host.eta == eta && ctx->rp_host.theta == theta))
-                launch_set_round_params(ctx, round, eta, theta, st);
+            const uint32_t t_epoch = (uint32_t)ctx->rounds_in_epoch;
+            if (!(ctx->rp_host_valid && ctx->rp_host.round == round && ctx->rp_host.eta == eta && ctx->rp_host.theta == theta &&
+                  ctx->rp_host.t_epoch == t_epoch))
+                launch_set_round_params(ctx, round, eta, theta, t_epoch, st);
             if (cudaGraphLaunch(ctx->graph_exec, st) != cudaSuccess) return DQ_ERR_CUDA;
-            ctx->rp_host = dq::RoundParams{round + 1u, eta, theta, 0u}; ctx->rp_host_valid = true;
+            ctx->rp_host = dq::RoundParams{round + 1u, eta, theta, 0u, t_epoch + 1u, {0u, 0u, 0u}}; ctx->rp_host_valid = true;
             ctx->launches += ctx->graph_launches;
             replayed = true;
         }

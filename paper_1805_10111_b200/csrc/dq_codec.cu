@@ -49,11 +49,13 @@ quantize_pack_kernel(const float* __restrict__ v, int64_t d, int vec_ok, const u
                      int64_t ngroups, int* __restrict__ status, const RoundParams* __restrict__ rp,
                      const float* __restrict__ ref = nullptr, float* __restrict__ diff = nullptr,
                      float* __restrict__ zero_f = nullptr, int64_t zero_n = 0, uint32_t* __restrict__ zero_u = nullptr, int zero_un = 0,
-                     const int32_t* __restrict__ bits_gate = nullptr /* run only if *bits_gate == BITS */)
+                     const int32_t* __restrict__ bits_gate = nullptr /* run only if *bits_gate == BITS */,
+                     int ring = 0 /* diff is a ring of this many vectors: write the slot of the device's round counter */)
 {
     pdl_prologue();
     if (bits_gate && *bits_gate != BITS) return;
     if (rp) round = rp->round;
+    if (DIFF && rp && ring > 1) diff += (int64_t)(rp->t_epoch % (uint32_t)ring) * d;
     if (DIFF) {   // also clears the buffers that the next stages of the round accumulate into
         const int64_t nth0 = (int64_t)gridDim.x * gridDim.y * blockDim.x;
         const int64_t tid0 = ((int64_t)blockIdx.y * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
@@ -1639,15 +1641,36 @@ model_precision_kernel(const float* __restrict__ x, const float* __restrict__ xs
     double inv[kWidths];
 #pragma unroll
     for (int k = 0; k < kWidths; ++k) inv[k] = nrm > 0.0f ? 1.0 / (double)__fdiv_rn(nrm, (float)levels(k + 2)) : 0.0;
+    // The kernel is bound by the double-precision pipe, so the fraction costs as few of its operations as exactness
+    // allows: with M = 1.5 * 2^52, x inv + M rounded toward -inf is M + floor(x inv) (one fused operation), M minus that
+    // is -floor exactly, a second fused operation gives frac = x inv - floor rounded once, and frac (1 - frac) is
+    // accumulated as sum frac - sum frac^2: five operations per width.
+    const double kMagic = 6755399441055744.0;
+    double s1[kWidths], s2[kWidths], dist = 0.0;
+#pragma unroll
+    for (int k = 0; k < kWidths; ++k) { s1[k] = 0.0; s2[k] = 0.0; }
+    auto one = [&](float xf, float sf) {
+        const double xi = (double)xf, df = xi - (double)sf;
+#pragma unroll
+        for (int k = 0; k < kWidths; ++k) {
+            const double nfl = kMagic - __fma_rd(xi, inv[k], kMagic);
+            const double fr = fma(xi, inv[k], nfl);
+            s1[k] += fr; s2[k] = fma(fr, fr, s2[k]);
+        }
+        dist = fma(df, df, dist);
+    };
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (int64_t)gridDim.x * blockDim.x;
+    const bool vec = ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(xsnap)) & 15) == 0;
+    const int64_t nq = vec ? (d >> 2) : 0;
+    for (int64_t q = tid; q < nq; q += nth) {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(x) + q), b = __ldg(reinterpret_cast<const float4*>(xsnap) + q);
+        one(a.x, b.x); one(a.y, b.y); one(a.z, b.z); one(a.w, b.w);
+    }
+    for (int64_t i = (nq << 2) + tid; i < d; i += nth) one(x[i], xsnap[i]);
     double acc[kWidths + 1];
 #pragma unroll
-    for (int k = 0; k <= kWidths; ++k) acc[k] = 0.0;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < d; i += (int64_t)gridDim.x * blockDim.x) {
-        const double xi = (double)x[i], df = xi - (double)xsnap[i];
-#pragma unroll
-        for (int k = 0; k < kWidths; ++k) { const double t = xi * inv[k], fr = t - floor(t); acc[k] += fr * (1.0 - fr); }
-        acc[kWidths] += df * df;
-    }
+    for (int k = 0; k < kWidths; ++k) acc[k] = s1[k] - s2[k];
+    acc[kWidths] = dist;
     __shared__ double s_part[kThreads / 32][kWidths + 1];
 #pragma unroll
     for (int k = 0; k <= kWidths; ++k) {
@@ -1696,12 +1719,13 @@ quantize_pack_any_kernel(const float* __restrict__ v, int64_t d, const uint32_t*
                          float* __restrict__ scale, const __grid_constant__ PhiloxKeys K, uint32_t round, uint32_t worker,
                          uint32_t stream, int* __restrict__ status, const RoundParams* __restrict__ rp,
                          const float* __restrict__ ref, float* __restrict__ diff, float* __restrict__ zero_f, int64_t zero_n,
-                         uint32_t* __restrict__ zero_u, int zero_un, int bits_fixed, const int32_t* __restrict__ bits_dev)
+                         uint32_t* __restrict__ zero_u, int zero_un, int bits_fixed, const int32_t* __restrict__ bits_dev, int ring)
 {
     pdl_prologue();
     const int bits = bits_dev ? *bits_dev : bits_fixed;
     if (bits < 2 || bits > 11 || (bits_dev && (bits == 2 || bits == 4 || bits == 8))) return;
     if (rp) round = rp->round;
+    if (diff && rp && ring > 1) diff += (int64_t)(rp->t_epoch % (uint32_t)ring) * d;
     const int64_t nth = (int64_t)gridDim.x * blockDim.x, tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (diff) {
         for (int64_t i = tid; i < zero_n; i += nth) zero_f[i] = 0.0f;
@@ -1791,7 +1815,7 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
 {
     if (bits != 2 && bits != 4 && bits != 8) {                 // a width that does not divide eight: one vector, general kernel
         launch_k(quantize_pack_any_kernel, grid_for((d + 7) / 8, ctx->sm_count), kThreads, 0, st, v, d, norm_bits, codes, scale, ctx->keys,
-                 round, worker_base, stream_id, ctx->status, ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits, bits_gate);
+                 round, worker_base, stream_id, ctx->status, ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits, bits_gate, ctx->diff_ring);
         ctx->launches += 1;
         return;
     }
@@ -1800,11 +1824,11 @@ void launch_quantize_pack(dq_ctx* ctx, const float* v, int64_t d, int M, int bit
     if (diff) {
         grid.x = max(grid.x, (unsigned)grid_for(zero_n / 4, ctx->sm_count));   // enough blocks for the clearing loop too
         DQ_DISPATCH_BITS(bits, (launch_k(quantize_pack_kernel<BITS_, true>, grid, kThreads, 0, st, v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status,
-            ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits_gate)));
+            ctx->rp_active, ref, diff, zero_f, zero_n, zero_u, zero_un, bits_gate, ctx->diff_ring)));
         ctx->launches += 1;
         return;
     }
-    DQ_DISPATCH_BITS(bits, (launch_k(quantize_pack_kernel<BITS_>, grid, kThreads, 0, st, v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr)));
+    DQ_DISPATCH_BITS(bits, (launch_k(quantize_pack_kernel<BITS_>, grid, kThreads, 0, st, v, d, vec_ok_for(v, d), norm_bits, codes, stride, scale, ctx->keys, round, worker_base, stream_id, ngroups, ctx->status, ctx->rp_active, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr, 0)));
     ctx->launches += 1;
 }
 
@@ -2122,6 +2146,6 @@ extern "C" int dq_quantize_pack_static(const float* v, int64_t d, int M, int b, 
     const PhiloxKeys keys = expand_keys(seed);
     int* flag = reinterpret_cast<int*>(scratch + kStaticMaxMessages);
     cudaError_t err = cudaSuccess;             // this launch's own result, not whatever error an earlier call left behind
-    DQ_DISPATCH_BITS(b, (err = launch_k(quantize_pack_kernel<BITS_, false>, grid_q, kThreads, 0, st, v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr)));
+    DQ_DISPATCH_BITS(b, (err = launch_k(quantize_pack_kernel<BITS_, false>, grid_q, kThreads, 0, st, v, d, vec_ok, scratch, codes, stride, scale, keys, round, 0u, kStreamGrad, ngroups, flag, nullptr, nullptr, nullptr, nullptr, 0, nullptr, 0, nullptr, 0)));
     return err == cudaSuccess ? DQ_OK : DQ_ERR_CUDA;
 }

@@ -233,7 +233,7 @@ __device__ __forceinline__ void write_round_bits(const BitsArgs& ba, int M, int6
 }
 
 // Per-round scalars kept in device memory so that a captured graph of a round can be replayed unchanged.
-struct RoundParams { uint32_t round; float eta; float theta; uint32_t pad; };
+struct RoundParams { uint32_t round; float eta; float theta; uint32_t pad; uint32_t t_epoch; uint32_t unused[3]; };   // t_epoch: rounds since the epoch began
 
 // Last statement of the kernel that ends a replayed round: the block that finishes last advances the round number
 // held on the device (no block reads it afterwards), so that consecutive rounds need no launch that sets it.
@@ -243,7 +243,7 @@ __device__ __forceinline__ void finish_round(const RoundParams* rp)
     if (rp && threadIdx.x == 0) {
         RoundParams* p = const_cast<RoundParams*>(rp);
         __threadfence();
-        if (atomicAdd(&p->pad, 1u) == gridDim.x * gridDim.y * gridDim.z - 1u) { p->pad = 0u; p->round += 1u; }
+        if (atomicAdd(&p->pad, 1u) == gridDim.x * gridDim.y * gridDim.z - 1u) { p->pad = 0u; p->round += 1u; p->t_epoch += 1u; }
     }
 }
 
@@ -316,6 +316,7 @@ struct dq_ctx {
     int32_t* delays_dev;        // [M] rounds each worker lags behind
     int32_t* slots_dev;         // [M] ring slot each worker reads this round
     bool use_slots;             // set while dq_round enqueues a round of a context with max_delay > 0
+    int diff_ring;              // set while such a round is captured: slots of the ring, the kernels pick this round's from the device's round counter
     int cluster_blocks;         // blocks of the one-cluster round kernel for small problems; 0: rounds run as separate kernels
     bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only
     bool list_ready;            // the list of this round has been built (consumed by the sparsifier launch)

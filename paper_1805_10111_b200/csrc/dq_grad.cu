@@ -2259,28 +2259,30 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
 }
 
 // Ring slot that each worker reads in round t of the epoch: the broadcast of round t - min(delay, t), ring of tau + 1.
-__global__ void set_slots_kernel(const int32_t* __restrict__ delays, int M, int t, int tau, int32_t* __restrict__ slots)
+__global__ void set_slots_kernel(const int32_t* __restrict__ delays, int M, int t, int tau, int32_t* __restrict__ slots,
+                                 const RoundParams* __restrict__ rp)
 {
     pdl_prologue();
+    if (rp) t = (int)rp->t_epoch;
     const int w = blockIdx.x * blockDim.x + threadIdx.x;
     if (w < M) { const int D = min(min(max(delays[w], 0), tau), t); slots[w] = (t - D) % (tau + 1); }
 }
 
 void launch_set_slots(dq_ctx* ctx, int t, cudaStream_t st)
 {
-    launch_k(set_slots_kernel, (ctx->cfg.M + kThreads - 1) / kThreads, kThreads, 0, st, ctx->delays_dev, ctx->cfg.M, t, ctx->cfg.max_delay, ctx->slots_dev);
+    launch_k(set_slots_kernel, (ctx->cfg.M + kThreads - 1) / kThreads, kThreads, 0, st, ctx->delays_dev, ctx->cfg.M, t, ctx->cfg.max_delay, ctx->slots_dev, ctx->rp_active);
     ctx->launches += 1;
 }
 
-__global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float eta, float theta)
+__global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float eta, float theta, uint32_t t_epoch)
 {
     pdl_prologue();
-    rp->round = round; rp->eta = eta; rp->theta = theta; rp->pad = 0u;
+    rp->round = round; rp->eta = eta; rp->theta = theta; rp->pad = 0u; rp->t_epoch = t_epoch;
 }
 
-void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st)
+void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, uint32_t t_epoch, cudaStream_t st)
 {
-    launch_k(set_round_params_kernel, 1, 1, 0, st, ctx->rp_dev, round, eta, theta);
+    launch_k(set_round_params_kernel, 1, 1, 0, st, ctx->rp_dev, round, eta, theta, t_epoch);
     ctx->launches += 1;
 }
 

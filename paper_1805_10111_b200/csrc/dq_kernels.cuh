@@ -42,6 +42,6 @@ void launch_set_slots(dq_ctx* ctx, int round_in_epoch, cudaStream_t st);
 void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds, float eta, float theta, uint64_t* bits_down,
                           uint64_t* bits_up, cudaStream_t st);
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st);
-void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, cudaStream_t st);
+void launch_set_round_params(dq_ctx* ctx, uint32_t round, float eta, float theta, uint32_t t_epoch, cudaStream_t st);
 
 }  // namespace dq

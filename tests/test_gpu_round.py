@@ -686,11 +686,14 @@ def test_lockstep_delayed_workers(dq, name, kw, eta):
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda2=1e-5, seed=21, no_fused=1)),
     ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=22)),
     ("bf16", dict(M=3, B=70, bx=8, b=8, box_lo=-1.0, box_hi=1.0, accelerated=1, seed=23)),
+    ("csr", dict(M=5, B=16, bx=8, b=4, lambda2=1e-5, seed=24, max_delay=3)),
+    ("dense8", dict(M=4, B=16, bx=6, b=4, lambda2=1e-4, seed=25, max_delay=2)),
 ])
 def test_graph_replay_equals_direct_launches(dq, name, kw):
     """dq_round replays a captured CUDA graph by default; with no_graph = 1 it launches the same kernels one by one.
     Both must leave identical bytes everywhere (dense rows are summed in a fixed order, CSR rows on an exact integer
-    grid), also after switching to a second state (re-capture)."""
+    grid), also after switching to a second state (re-capture), and with lagging workers (the replayed kernels take
+    the ring slot from the round counter kept on the device)."""
     import torch
     h = _problem(name)
     data = dq.Data(h)
@@ -700,13 +703,16 @@ def test_graph_replay_equals_direct_launches(dq, name, kw):
     for no_graph in (0, 1):
         cfg = dq.make_config(h.d, kw["M"], no_graph=no_graph, **{k: v for k, v in kw.items() if k != "M"})
         rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+        tau = kw.get("max_delay", 0)
+        if tau:
+            assert dq.dq_set_delays(ctx, [w % (tau + 1) for w in range(kw["M"])]) == 0
         states = [dq.State(x0, n=h.n, accelerated=acc), dq.State(x0 * F32(0.5), n=h.n, accelerated=acc)]
         bits = torch.zeros(2, dtype=torch.int64, device="cuda")
         rnd = 0
         for st in states:                                   # the second state forces a new capture
             for epoch in range(2):
                 assert dq.dq_epoch_begin(ctx, st, 0.5 if acc else 0.0) == 0
-                for t in range(5):
+                for t in range(5 + 2 * tau):
                     assert dq.dq_round(ctx, st, rnd, 0.05 if acc else 0.3, 0.5 if acc else 0.0, bits[0:1], bits[1:2]) == 0
                     rnd += 1
         assert dq.dq_poll_status(ctx) == (0, 0)
