@@ -208,8 +208,10 @@ int dq_round(dq_ctx* ctx, dq_state* st, uint32_t round, float eta, float theta,
  * [M], each in 0..max_delay; NULL: all zero) says for every worker how many rounds before the current one the model
  * it works on was broadcast; it holds for the following dq_round calls until set again.  A delay is cut to the
  * number of rounds the epoch has had (the first round's workers all see the current model).  Needs
- * cfg.max_delay > 0 and the logistic model; such a context launches its rounds kernel by kernel (no graph, no
- * one-cluster kernel).  Copies synchronously. */
+ * cfg.max_delay > 0; both models take delays (for the network the kept broadcasts are the low-precision parameters
+ * themselves).  Such a context replays its rounds as a captured graph like any other (the kernels pick the
+ * broadcast of a lagging worker from a round counter kept on the device), but not in the one-cluster kernel.
+ * Copies synchronously. */
 int dq_set_delays(dq_ctx* ctx, const int32_t* delays);
 
 /* nrounds consecutive rounds round0, round0 + 1, ... of the same epoch with the same (eta, theta), as by

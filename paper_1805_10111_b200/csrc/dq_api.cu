@@ -86,7 +86,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (!(cfg->box_lo <= cfg->box_hi) || cfg->lambda1 < 0 || cfg->lambda2 < 0) return DQ_ERR_ARG;
     if (cfg->sparse_cap < 0 || cfg->sparse_cap > cfg->d) return DQ_ERR_ARG;
     if (!(cfg->mu >= 0.0f)) return DQ_ERR_ARG;
-    if (cfg->max_delay < 0 || cfg->max_delay > 64 || (cfg->max_delay > 0 && (!data || cfg->model != DQ_MODEL_LOGISTIC))) return DQ_ERR_ARG;
+    if (cfg->max_delay < 0 || cfg->max_delay > 64 || (cfg->max_delay > 0 && !data)) return DQ_ERR_ARG;
     if (data) {
         if (data->n < 1 || !data->values || !data->labels) return DQ_ERR_SHAPE;
         if (cfg->model == DQ_MODEL_MLP) {
@@ -364,7 +364,10 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
         // while a round is captured for replay the kernels take the epoch's round counter from the device instead
         if (ctx->rp_active) ctx->diff_ring = tau + 1;
         else ctx->xhat_diff = ring + (int64_t)(t % (tau + 1)) * ctx->cfg.d;
-        if (flag) cudaMemsetAsync(ctx->xhat_diff, 0, sizeof(float) * ctx->cfg.d, as_stream(st));   // xhat = xsnap
+        if (flag) {                                          // xhat = xsnap: a zero difference; the network's ring holds xhat itself
+            if (ctx->cfg.model == DQ_MODEL_MLP) cudaMemcpyAsync(ctx->xhat_diff, s->x_snap, sizeof(float) * ctx->cfg.d, cudaMemcpyDeviceToDevice, as_stream(st));
+            else cudaMemsetAsync(ctx->xhat_diff, 0, sizeof(float) * ctx->cfg.d, as_stream(st));
+        }
         launch_set_slots(ctx, t, as_stream(st));
     }
     if (!flag) {     // model quantisation that also emits xhat - xsnap for the workers

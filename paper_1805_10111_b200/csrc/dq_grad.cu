@@ -1275,26 +1275,38 @@ __device__ __forceinline__ float4 mlp_load4(const float* __restrict__ p, int i, 
 constexpr int kMlpBatch = 3;
 template <bool VEC>
 __global__ void __launch_bounds__(kThreads)
-mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restrict__ xa, const float* __restrict__ xb,
+mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* xa, const float* __restrict__ xb,
                   const __grid_constant__ PhiloxKeys K, BatchSource bs, int B, int32_t* __restrict__ row_of_slot,
                   double* __restrict__ act_a, double* __restrict__ act_b, int64_t nslots)
 {
     pdl_prologue();
-    __shared__ int64_t s_row[kMlpTile];
+    __shared__ int64_t s_row[kMlpTile], s_slot[kMlpTile];
     __shared__ double s_red[kThreads / 32][2][kMlpTile * 8];      // [warp][model][row * 8 + unit]
     clear_word(bs);
-    const int64_t slot0 = (int64_t)blockIdx.x * kMlpTile;
+    // Workers that lag read their own copy of the model (a slot of the ring): then a tile holds rows of one worker only.
+    const bool per_worker = B > 0 && bs.diff_slot != nullptr;
+    const int tpw = per_worker ? (B + kMlpTile - 1) / kMlpTile : 1;             // tiles per worker
+    const int tile_w = per_worker ? (int)blockIdx.x / tpw : 0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x < kMlpTile) {
-        const int64_t slot = slot0 + threadIdx.x;
+        int64_t slot;
+        if (per_worker) {
+            const int j = ((int)blockIdx.x % tpw) * kMlpTile + (int)threadIdx.x;
+            slot = j < B ? (int64_t)tile_w * B + j : -1;
+        } else {
+            slot = (int64_t)blockIdx.x * kMlpTile + threadIdx.x;
+        }
         int64_t a = -1;
-        if (slot < nslots) {
+        if (slot >= 0 && slot < nslots) {
             a = B > 0 ? batch_row(bs, K, (int)(slot / B), (int)(slot % B), B, blockIdx.y == 0) : slot;   // B = 0: row = slot
             if (row_of_slot && blockIdx.y == 0) row_of_slot[slot] = (int32_t)a;
+        } else {
+            slot = -1;
         }
-        s_row[threadIdx.x] = a;
+        s_row[threadIdx.x] = a; s_slot[threadIdx.x] = slot;
     }
     __syncthreads();
+    if (per_worker && xa) xa = diff_of_worker(bs, xa, tile_w);
     const int j0 = blockIdx.y * 8;
     const int kk = lane & 3, rn = lane >> 2;             // this lane's k of A and B; its row of A / unit of B
     const int ju = j0 + rn;
@@ -1345,11 +1357,11 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
         const int model = q / (kMlpTile * 8), e = q % (kMlpTile * 8), t = e >> 3, u = e & 7;
         const float* xm = model == 0 ? xa : xb;
         double* act = model == 0 ? act_a : act_b;
-        if (xm && j0 + u < sh.hidden && slot0 + t < nslots) {
+        if (xm && j0 + u < sh.hidden && s_slot[t] >= 0) {
             double v = 0.0;
 #pragma unroll
             for (int k = 0; k < kThreads / 32; ++k) v += s_red[k][model][e];
-            act[(slot0 + t) * sh.hidden + j0 + u] = fmax(v + (double)xm[mlp_off_b1(sh) + j0 + u], 0.0);
+            act[s_slot[t] * sh.hidden + j0 + u] = fmax(v + (double)xm[mlp_off_b1(sh) + j0 + u], 0.0);
         }
     }
 }
@@ -1360,11 +1372,13 @@ mlp_hidden_kernel(const float* __restrict__ X, MlpShape sh, const float* __restr
 // (the sum without the label's term), which has no cancellation.
 __global__ void __launch_bounds__(kThreads)
 mlp_output_kernel(MlpShape sh, const float* __restrict__ labels, const int32_t* __restrict__ row_of_slot,
-                  const float* __restrict__ xa, const float* __restrict__ xb, const double* __restrict__ act_a,
+                  const float* xa, const float* __restrict__ xb, const double* __restrict__ act_a,
                   const double* __restrict__ act_b, double wgt, float* __restrict__ dz_a, float* __restrict__ dz_b,
-                  float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b, int staged)
+                  float* __restrict__ dh_a, float* __restrict__ dh_b, double* __restrict__ loss_b, int staged,
+                  int B, const int32_t* __restrict__ a_slot, int64_t a_stride /* lagging workers: model a of worker slot / B sits in ring slot a_slot[.] */)
 {
     pdl_prologue();
+    if (a_slot && xa) xa += (int64_t)a_slot[blockIdx.x / B] * a_stride;
     extern __shared__ double s_zd[];     // [2 models][logits, exponentials, dz][classes], [2][hidden] activations, staged: [2][W2, b2]
     const int C = sh.classes, H = sh.hidden;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -1563,8 +1577,9 @@ mlp_param_kernel(const float* __restrict__ X, MlpShape sh, const int32_t* __rest
 #pragma unroll 4
             for (int r = 0; r < nrows; ++r) {
                 const int64_t q = r0 + r;
-                const double ta = dz_a ? (double)dz_a[q * sh.classes + c] * (bias ? 1.0 : act_a[q * sh.hidden + jj]) : 0.0;
-                const double tb = dz_b ? (double)dz_b[q * sh.classes + c] * (bias ? 1.0 : act_b[q * sh.hidden + jj]) : 0.0;
+                // both products rounded on their own (no fused multiply-subtract): equal models cancel exactly
+                const double ta = dz_a ? __dmul_rn((double)dz_a[q * sh.classes + c], bias ? 1.0 : act_a[q * sh.hidden + jj]) : 0.0;
+                const double tb = dz_b ? __dmul_rn((double)dz_b[q * sh.classes + c], bias ? 1.0 : act_b[q * sh.hidden + jj]) : 0.0;
                 s += ta - tb;
             }
             const int64_t pidx = bias ? mlp_off_b2(sh) + c : mlp_off_w2(sh) + (int64_t)c * sh.hidden + jj;
@@ -1876,8 +1891,9 @@ static inline int blocks_for(int64_t threads_needed, int sm_count, int per_sm = 
 
 // ---- network launchers ------------------------------------------------------------------------------------
 static MlpShape mlp_shape(const dq_ctx* ctx) { return MlpShape{ctx->data.d, ctx->cfg.hidden, ctx->cfg.classes}; }
-static dim3 mlp_hidden_grid(int64_t nslots, const MlpShape& sh)
+static dim3 mlp_hidden_grid(int64_t nslots, const MlpShape& sh, int M = 0, int B = 0 /* both set: tiles of one worker each */)
 {
+    if (M > 0) return dim3((unsigned)(M * ((B + kMlpTile - 1) / kMlpTile)), (unsigned)((sh.hidden + 7) / 8));
     return dim3((unsigned)((nslots + kMlpTile - 1) / kMlpTile), (unsigned)((sh.hidden + kThreads / 32 - 1) / (kThreads / 32)));
 }
 constexpr int kMlpGroup = 256;      // rows per block of the epoch-gradient sums
@@ -1898,9 +1914,11 @@ static void launch_mlp_hidden(dq_ctx* ctx, int64_t nslots, const MlpShape& sh, c
                               int B, double* act_a, double* act_b, cudaStream_t st)
 {
     const float* X = (const float*)ctx->data.values;
-    const bool vec = sh.in % 4 == 0 && aligned16(X) && aligned16(xa) && aligned16(xb);       // rows and weight rows on 16-byte boundaries
-    if (vec) launch_k(mlp_hidden_kernel<true>, mlp_hidden_grid(nslots, sh), kThreads, 0, st, X, sh, xa, xb, ctx->keys, bs, B, ctx->mlp_rows, act_a, act_b, nslots);
-    else launch_k(mlp_hidden_kernel<false>, mlp_hidden_grid(nslots, sh), kThreads, 0, st, X, sh, xa, xb, ctx->keys, bs, B, ctx->mlp_rows, act_a, act_b, nslots);
+    // rows and weight rows on 16-byte boundaries; a lagging worker's parameters start slot * d floats into the ring
+    const bool vec = sh.in % 4 == 0 && aligned16(X) && aligned16(xa) && aligned16(xb) && (!(B > 0 && bs.diff_slot) || bs.diff_stride % 4 == 0);
+    const dim3 grid = (B > 0 && bs.diff_slot) ? mlp_hidden_grid(nslots, sh, (int)(nslots / B), B) : mlp_hidden_grid(nslots, sh);
+    if (vec) launch_k(mlp_hidden_kernel<true>, grid, kThreads, 0, st, X, sh, xa, xb, ctx->keys, bs, B, ctx->mlp_rows, act_a, act_b, nslots);
+    else launch_k(mlp_hidden_kernel<false>, grid, kThreads, 0, st, X, sh, xa, xb, ctx->keys, bs, B, ctx->mlp_rows, act_a, act_b, nslots);
 }
 
 // g <- (1/n) sum_i grad loss_i(x) over all rows (double sums), via the "a" slots of the activation buffers.
@@ -1912,7 +1930,7 @@ static void launch_mlp_full_grad(dq_ctx* ctx, const float* x, float* g, cudaStre
     launch_mlp_hidden(ctx, D.n, sh, x, nullptr, none, 0, ctx->mlp_act[0], nullptr, st);
     int staged; const size_t osm = mlp_output_smem(sh, &staged);
     launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, osm, st, sh, D.labels, ctx->mlp_rows, x, nullptr, ctx->mlp_act[0],
-        nullptr, 1.0 / (double)D.n, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, staged);
+        nullptr, 1.0 / (double)D.n, ctx->mlp_dz[0], nullptr, ctx->mlp_dh[0], nullptr, nullptr, staged, 1, nullptr, 0);
     cudaMemsetAsync(ctx->g64, 0, sizeof(double) * P, st);
     dim3 grid(mlp_param_grid_x(sh), (unsigned)((D.n + kMlpGroup - 1) / kMlpGroup));
     if (sh.in % 4 == 0 && aligned16(D.values))
@@ -1935,7 +1953,7 @@ static void launch_mlp_worker_grad(dq_ctx* ctx, const float* xhat, const dq_stat
     launch_mlp_hidden(ctx, R, sh, xhat, s->x_snap, bs, c.B, ctx->mlp_act[0], ctx->mlp_act[1], st);
     int staged; const size_t osm = mlp_output_smem(sh, &staged);
     launch_k(mlp_output_kernel, R, kThreads, osm, st, sh, D.labels, ctx->mlp_rows, xhat, s->x_snap, ctx->mlp_act[0],
-        ctx->mlp_act[1], 1.0 / (double)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr, staged);
+        ctx->mlp_act[1], 1.0 / (double)c.B, ctx->mlp_dz[0], ctx->mlp_dz[1], ctx->mlp_dh[0], ctx->mlp_dh[1], nullptr, staged, c.B, bs.diff_slot, bs.diff_stride);
     if (!ctx->ninf_zeroed) cudaMemsetAsync(nb, 0, sizeof(uint32_t) * c.M, st);
     dim3 grid(mlp_param_grid_x(sh), c.M);
     if (sh.in % 4 == 0 && aligned16(D.values))
@@ -2245,7 +2263,7 @@ void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st)
         launch_mlp_hidden(ctx, D.n, sh, nullptr, x, none, 0, nullptr, ctx->mlp_act[1], st);
         int staged; const size_t osm = mlp_output_smem(sh, &staged);
         launch_k(mlp_output_kernel, (unsigned)D.n, kThreads, osm, st, sh, D.labels, ctx->mlp_rows, nullptr, x, nullptr,
-            ctx->mlp_act[1], 1.0 / (double)D.n, nullptr, nullptr, nullptr, nullptr, P, staged);
+            ctx->mlp_act[1], 1.0 / (double)D.n, nullptr, nullptr, nullptr, nullptr, P, staged, 1, nullptr, 0);
         launch_k(objective_reg_kernel, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, x, c.d, c.lambda1, c.lambda2, P);
         ctx->launches += 3;
         return;

@@ -73,6 +73,30 @@ def test_network_lockstep_rounds(dq, extra):
     ls.close()
 
 
+@pytest.mark.parametrize("extra", [dict(max_delay=2), dict(max_delay=3, accelerated=1, box_lo=-2.0, box_hi=2.0)])
+def test_network_lockstep_delayed_workers(dq, extra):
+    """Lagging workers on the network (Algorithm 1 step 11 with x_{D(t)}): each worker's gradient difference is taken at
+    the low-precision parameters broadcast `delay` rounds earlier in the epoch (the ring keeps xhat itself here), with
+    delays that change every round; B = 20 rows per worker do not fill the kernel's row tiles."""
+    h, x = _net(400, 48, 12, 5, 5)
+    kw = dict(M=4, B=20, bx=8, b=4, lambda2=1e-4, seed=46, model=1, hidden=12, classes=5)
+    kw.update(extra)
+    ls = Lockstep(dq, h, x, **kw)
+    g = np.random.default_rng(46)
+    acc, tau, M = bool(extra.get("accelerated", 0)), extra["max_delay"], kw["M"]
+    rnd = 0
+    for s_ in range(1, 4):
+        theta = F32(2.0 / (s_ + 2)) if acc else F32(0.0)
+        ls.epoch(theta)
+        for t in range(2 * tau + 3):
+            delays = [int(v) for v in g.integers(0, tau + 1, M)] if s_ > 1 else [tau] * M
+            tr = ls.round(rnd, 0.05 if acc else 0.2, theta, delays=delays)
+            assert tr["delays_used"] == [min(D, t) for D in delays]
+            rnd += 1
+    assert ls.far_flips == 0
+    ls.close()
+
+
 def test_network_full_size_rounds(dq):
     """784-100-10 on 2,000 image-shaped rows, M = 8 workers, B = 20, b_x = 8, b = 4 (the paper's setting for this model)."""
     h, x = _net(2000, 784, 100, 10, 3)
