@@ -534,6 +534,10 @@ class Lockstep:
     ("dense_wide", dict(M=16, B=1, bx=3, b=8, box_lo=-0.5, box_hi=2.0, seed=46, no_fused=1), 0.3),
     ("csr", dict(M=16, B=1, bx=3, b=4, box_lo=-0.5, box_hi=0.5, seed=47), 0.3),
     ("dense_tiny", dict(M=17, B=1, bx=6, b=4, box_lo=-2.0, box_hi=0.5, sparsify=1, phi=50.0, seed=48), 0.3),
+    # sparse gradients into sparse messages with more touched groups per block of the message kernel than it keeps in
+    # registers (its re-reading path), and with so few that most blocks of a worker's cluster list nothing
+    ("c2", dict(M=3, B=400, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=300.0, msg_format=1, seed=60), 0.5),
+    ("c2", dict(M=3, B=1, bx=8, b=2, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=61), 0.5),
 ])
 def test_lockstep_small(dq, name, kw, eta):
     h = _problem(name)
