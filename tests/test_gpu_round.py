@@ -536,7 +536,7 @@ class Lockstep:
     ("dense_tiny", dict(M=17, B=1, bx=6, b=4, box_lo=-2.0, box_hi=0.5, sparsify=1, phi=50.0, seed=48), 0.3),
     # sparse gradients into sparse messages with more touched groups per block of the message kernel than it keeps in
     # registers (its re-reading path), and with so few that most blocks of a worker's cluster list nothing
-    ("c2", dict(M=3, B=400, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=300.0, msg_format=1, seed=60), 0.5),
+    ("c3", dict(M=3, B=400, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.01 * (1 << 20), msg_format=1, seed=60), 0.5),
     ("c2", dict(M=3, B=1, bx=8, b=2, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=61), 0.5),
 ])
 def test_lockstep_small(dq, name, kw, eta):
