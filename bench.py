@@ -630,8 +630,14 @@ def run_ours(a):
             dist.destroy_process_group()
         return
     stages = stage_report(stage_ms, alg, peak)
+    # the width search is bound by the double-precision pipe: about 63 of its lane-slots per coordinate (ten widths x
+    # five operations, two fp32->fp64 conversions at a quarter of the rate, the squared distance) on 64 lanes per SM
+    sm_ghz = (clocks.get("sm_mhz") or 1965.0) / 1000.0
+    alu_peak = 148 * 64 * sm_ghz * 1e9 / 63.0                      # coordinates per second
     stages["select_model_bits(optional)"] = {"ms": round(select_ms, 4), "alg_GBps": round(d * 8.0 / select_ms / 1e6, 1),
-                                              "frac_of_peak": round(d * 8.0 / select_ms / 1e6 / peak, 4)}
+                                              "frac_of_peak": round(d * 8.0 / select_ms / 1e6 / peak, 4), "bound": "alu",
+                                              "alu_peak_coordinates_per_s": round(alu_peak, 0),
+                                              "frac_of_alu_peak": round(d / (select_ms * 1e-3) / alu_peak, 4)}
     qp = stages["quantize_pack"]
     tr = recorded_traffic(b) if not a.sparsify else None
     roofline = {"kernel": "quantize_pack_kernel<%d>" % b if not a.sparsify else "norm_l1_kernel + sparsify_stage_kernel + sparsify_scatter_dense_kernel<%d>" % b,
