@@ -572,11 +572,13 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
     // a worker's last tile in this block has been added when the next tile belongs to another worker (or the run ends)
     const auto flush_at = [&](int it) { return it > 0 && worker_at(it) != worker_at(it - 1); };
 
-    // load warp: draw the rows of tile `it` of this block's run and start their copies into stage it % S (returns this
-    // lane's row, or -1), then fetch the rows' labels and snapshot margins and announce the tile
+    // load warp, in three steps per tile so that no load of one tile holds up the copies of another: draw_row (this
+    // lane's row of tile `it`, or -1), copy_rows (start the row copies into stage it % S), publish (labels and snapshot
+    // margins beside the rows, then the announcement of the tile).  The labels are fetched into registers one tile
+    // ahead, between draw_row and publish.
     int part_w = -1; int64_t part_lo = 0; uint64_t part_cnt = 0;
-    auto issue_rows = [&](int it) -> int64_t {
-        const int t = t0 + it, stage = it % S;
+    auto draw_row = [&](int it) -> int64_t {
+        const int t = t0 + it;
         const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
         const int nvalid = min(R, pl.B - j0);
         if (w != part_w) {               // the worker's partition of the rows (two 64-bit divisions: once per worker, not per row)
@@ -596,24 +598,26 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
                 a = part_lo + (int64_t)(((uint64_t)word * part_cnt) >> 32);
                 if (bs.rows_out) bs.rows_out[slot_j] = (int32_t)a;
             }
-            bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
         }
+        return a;
+    };
+    auto copy_rows = [&](int it, int64_t a) {
+        const int t = t0 + it, stage = it % S;
+        const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
+        const int nvalid = min(R, pl.B - j0);
+        if (a >= 0) bulk_row_load(s_stage + ((size_t)stage * R + lane) * stride, X + a * d, (uint32_t)row_bytes, &s_full[stage]);
         if (MMA_FRONT && nvalid < R) {   // the tensor-core paths multiply whole tiles: rows past the minibatch's end must read as zeros
             uint4* z = reinterpret_cast<uint4*>(s_stage + ((size_t)stage * R + nvalid) * stride);
             for (int q = lane; q < (R - nvalid) * (stride >> 4); q += 32) z[q] = make_uint4(0u, 0u, 0u, 0u);
         }
-        return a;
     };
-    auto issue_labels = [&](int it, int64_t a) {
+    auto publish = [&](int it, int64_t a, float lab, float zs) {
         const int t = t0 + it, stage = it % S, slot = it % (S + 2);
         const int w = pl.worker_of(t), j0 = (t - w * pl.tiles_per_worker) * R;
         const int nvalid = min(R, pl.B - j0);
-        if (a >= 0) {
-            // the row's label and snapshot margin go beside it.  They are stored before this warp's arrival on the stage's
-            // barrier below, so whoever has seen the stage full (and whoever hears from them) sees them too.
-            const float lab = __ldg(labels + a), zs = __ldg(z_snap + a);
-            s_lab[slot][lane] = lab; s_zs[slot][lane] = zs;
-        }
+        // the row's label and snapshot margin go beside it.  They are stored before this warp's arrival on the stage's
+        // barrier below, so whoever has seen the stage full (and whoever hears from them) sees them too.
+        if (a >= 0) { s_lab[slot][lane] = lab; s_zs[slot][lane] = zs; }
         __syncwarp();
         // the byte count is announced after the copies were started: the phase cannot complete before this arrival
         if (lane == 0) { mbar_arrive_expect_tx(&s_full[stage], (uint32_t)(nvalid * row_bytes)); s_issued = it + 1; }
@@ -777,17 +781,27 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
 
     if (load_warp) {
         // ---- copies: S tiles ahead; a stage is refilled once every compute warp has taken its groups out of it -------
-        int64_t a0[S];
+        int64_t a0[S]; float lab0[S], zs0[S];
 #pragma unroll
-        for (int k = 0; k < S; ++k) a0[k] = k < ntl ? issue_rows(k) : -1;      // all row copies of the first tiles first,
+        for (int k = 0; k < S; ++k) {                        // rows of the first tiles, their small loads in flight,
+            a0[k] = k < ntl ? draw_row(k) : -1; lab0[k] = zs0[k] = 0.0f;
+            if (a0[k] >= 0) { lab0[k] = __ldg(labels + a0[k]); zs0[k] = __ldg(z_snap + a0[k]); }
+        }
 #pragma unroll
-        for (int k = 0; k < S; ++k) if (k < ntl) issue_labels(k, a0[k]);        // then the small loads that would hold them up
+        for (int k = 0; k < S; ++k) if (k < ntl) copy_rows(k, a0[k]);              // all row copies,
+#pragma unroll
+        for (int k = 0; k < S; ++k) if (k < ntl) publish(k, a0[k], lab0[k], zs0[k]);   // then the announcements
+        int64_t a_n = S < ntl ? draw_row(S) : -1;            // one tile ahead: its labels arrive while the stage is still in use
+        float lab_n = 0.0f, zs_n = 0.0f;
+        if (a_n >= 0) { lab_n = __ldg(labels + a_n); zs_n = __ldg(z_snap + a_n); }
         for (int it = 0; it <= ntl; ++it) {
             if (flush_at(it)) flush(worker_at(it - 1));
             if (it + S < ntl) {
                 wait(&s_empty[it % S], (uint32_t)((it / S) & 1));
-                const int64_t a = issue_rows(it + S);
-                issue_labels(it + S, a);
+                copy_rows(it + S, a_n);
+                publish(it + S, a_n, lab_n, zs_n);
+                a_n = it + S + 1 < ntl ? draw_row(it + S + 1) : -1;
+                if (a_n >= 0) { lab_n = __ldg(labels + a_n); zs_n = __ldg(z_snap + a_n); }
             }
         }
     } else if (slope_warp) {
