@@ -566,6 +566,7 @@ worker_grad_fused_kernel(const T* __restrict__ X, const float* __restrict__ labe
         while (!mbar_try_wait(bar, parity)) {
             if (*reinterpret_cast<volatile int*>(&s_abort)) return;
             if (clock64() - c0 > kFusedWaitCycles) { s_abort = 1; set_status(status, DQ_ERR_TIMEOUT); return; }
+            if (!compute) __nanosleep(200);                  // the load and slope warps have a tile's time of slack: their polling must not take issue slots from the compute warps
         }
     };
     const auto worker_at = [&](int it) { return it < ntl ? pl.worker_of(t0 + it) : -1; };
