@@ -727,6 +727,43 @@ def test_graph_replay_equals_direct_launches(dq, name, kw):
     assert np.array_equal(outs[0][2], outs[1][2])
 
 
+def test_sparse_round_with_too_small_messages(dq):
+    """CSR data, sparse messages whose capacity is below the number of survivors: the round reports DQ_ERR_CAPACITY,
+    every message holds exactly `cap` entries, they are the first `cap` entries (positions and codes) of the message a
+    large enough buffer receives, and the master step runs on them (tile pointers stay inside the list)."""
+    import torch
+    h = _problem("csr")
+    data = dq.Data(h)
+    x0 = synth.normal_vector(h.d, 86, 0.05)
+    kw = dict(B=64, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=71)
+    got = []
+    small = 6
+    for cap in (small, 0):
+        cfg = dq.make_config(h.d, 4, **kw, **({"sparse_cap": cap} if cap else {}))
+        rc, ctx = dq.dq_create(cfg, data); assert rc == 0
+        st = dq.State(x0, n=h.n)
+        assert dq.dq_epoch_begin(ctx, st, 0.0) == 0
+        for rnd in range(2):                                # a snapshot round, then a round with gradients
+            assert dq.dq_round(ctx, st, rnd, 0.3, 0.0) == 0
+        rc, status = dq.dq_poll_status(ctx)
+        assert rc == 0 and status == (dq.DQ_ERR_CAPACITY if cap else 0)
+        _, buf = dq.dq_round_buffers(ctx)
+        m = buf["msgs"]
+        nnz = dq.device_view(m.nnz, 4, torch.int32).cpu().numpy()
+        idx = dq.device_view(m.idx, 4 * m.cap, torch.int32).cpu().numpy().reshape(4, m.cap)
+        codes = dq.device_view(m.codes, 4 * m.stride, torch.uint8).cpu().numpy().reshape(4, m.stride)
+        scale = dq.device_view(m.scale, 4, torch.float32).cpu().numpy()
+        got.append((nnz.copy(), idx.copy(), codes.copy(), scale.copy(), st.x.cpu().numpy().copy()))
+        assert np.all(np.isfinite(got[-1][4]))
+        dq.dq_destroy(ctx)
+    (nnz_s, idx_s, codes_s, scale_s, _), (nnz_l, idx_l, codes_l, scale_l, _) = got
+    assert np.all(nnz_l > small) and np.all(nnz_s == small), (nnz_l, nnz_s)
+    assert np.array_equal(scale_s, scale_l)
+    for w in range(4):
+        assert np.array_equal(idx_s[w, :small], idx_l[w, :small])
+        assert np.array_equal(codes_s[w, :small * 4 // 8], codes_l[w, :small * 4 // 8])
+
+
 @pytest.mark.parametrize("name,kw", [
     ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=31)),
     ("dense8", dict(M=4, B=16, bx=8, b=4, lambda2=1e-4, accelerated=1, seed=32)),
