@@ -369,9 +369,12 @@ class Run:
             return False
         return (not self.cfg.accelerated) or self.epoch == 0
 
-    def round(self, round_, eta, theta=0.0, trace=False, delays=None):
-        """delays: per worker, how many rounds of this epoch ago the model it works on was broadcast (Algorithm 1's
-        t - D(t); clamped to the rounds the epoch has had).  The run keeps the epoch's broadcasts for that."""
+    def round(self, round_, eta, theta=0.0, trace=False, delays=None, across_epochs=False):
+        """delays: per worker, how many rounds ago the model it works on was broadcast (Algorithm 1's t - D(t)).  By
+        default a delay is cut to the rounds the epoch has had; with across_epochs it may reach back into the
+        previous epoch (cut to the rounds the run has had): the worker then evaluates the previous epoch's
+        low-precision model against THIS epoch's snapshot and full gradient, as step 11 is written.  The run keeps
+        the broadcasts for that."""
         cfg = self.cfg; d, M, B = cfg.d, cfg.M, cfg.B
         flag = self.is_flag_round()
         T = Trace(); keep = {}
@@ -390,9 +393,9 @@ class Run:
             rc = lib().dqo_round(C.addressof(cfg), self.data.ref, C.addressof(self.state), round_, int(flag),
                                  float(eta), float(theta), C.addressof(T))
         else:
-            if self.rounds_in_epoch == 0:
-                self.broadcasts = []                                       # low-precision models of this epoch, by round
-            t = self.rounds_in_epoch
+            if not hasattr(self, "broadcasts") or (self.rounds_in_epoch == 0 and not across_epochs):
+                self.broadcasts = []                                       # low-precision models by round (of this epoch, or of the run)
+            t = len(self.broadcasts)
             used = [min(int(D), t) for D in delays]
             ptrs = (C.c_void_p * M)(*[None if D == 0 else _p(self.broadcasts[t - D]) for D in used])
             rc = lib().dqo_round_delayed(C.addressof(cfg), self.data.ref, C.addressof(self.state), round_, int(flag),

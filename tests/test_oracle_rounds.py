@@ -249,6 +249,47 @@ def test_delayed_rounds_use_the_model_of_t_minus_delay():
     assert not np.array_equal(a.x, b.x)
 
 
+def test_delays_reach_across_the_epoch_boundary():
+    """With across_epochs a delay is cut to the rounds of the whole run: in the first rounds of an epoch a lagging
+    worker evaluates the PREVIOUS epoch's low-precision model against the NEW snapshot (Algorithm 1 step 11 with
+    t - D(t) <= tau across the outer loop).  Re-derived in float64 numpy from broadcasts that the test rebuilds itself;
+    a worker with delay 0 in the epoch's first round still sends exactly zero (x = xsnap there)."""
+    h, data = _problem()
+    M, B, tau = 3, 8, 2
+    cfg = oracle.make_config(h.d, M, B, 8, 8, l1=1e-4, seed=11)
+    x0 = synth.normal_vector(h.d, 36, 0.2)
+    run = oracle.Run(cfg, data, x0)
+    X, y = h.values.astype(np.float64), h.labels
+    mine = []                                                # every broadcast of the run, rebuilt independently
+    rnd = 0
+    crossed = 0
+    for epoch in range(3):
+        run.epoch_begin()
+        for t in range(4):
+            delays = [tau, 0, 1] if t == 0 else [int(v) for v in np.random.default_rng(100 + rnd).integers(0, tau + 1, M)]
+            x_before = run.x.copy()
+            tr = run.round(rnd, 0.4, trace=True, delays=delays, across_epochs=True)
+            if tr["flag_round"]:
+                mine.append(run.xsnap.copy())
+            else:
+                cx, dx, _ = oracle.quantize(x_before, 8, 11, rnd, oracle.MASTER, oracle.STREAM_MODEL)
+                mine.append(cx.astype(F32) * dx)
+            assert tr["delays_used"] == [min(D, rnd) for D in delays]
+            for w in range(M):
+                used = min(delays[w], rnd)
+                xw = mine[rnd - used]
+                crossed += int(used > t)
+                rows = tr["rows"][w]
+                want = ((_np_slope(X, y, rows, xw) - _np_slope(X, y, rows, run.xsnap))[:, None] * X[rows]).mean(axis=0)
+                assert np.allclose(tr["alpha"][w], want, rtol=1e-5, atol=1e-7), (epoch, t, w)
+                if t == 0 and used == 0:
+                    assert not np.any(tr["alpha"][w])
+                if t == 0 and used > 0 and epoch > 0:
+                    assert np.any(tr["alpha"][w])              # the old model is not the new snapshot
+            rnd += 1
+    assert crossed >= 4
+
+
 def test_round_with_searched_model_bits():
     """With mu > 0 every non-flag round quantises the model with the searched width and pays for that width."""
     h, data = _problem()
