@@ -104,6 +104,10 @@ typedef struct {
     int32_t tensor_cores;      /* 1: the one-pass dense gradient forms X (xhat - xsnap) and X^T r of bfloat16 rows (d a multiple of
                                   16) as bf16 tensor-core MMAs with fp32 accumulation, the fp32 factors split into three bfloat16
                                   terms; 0: fp32 FMAs on CUDA cores (the default: measured faster, see the profiles) */
+    int32_t delay_across_epochs; /* with max_delay > 0: 1 lets a delay reach back into the previous epoch (the worker then evaluates
+                                  the previous epoch's low-precision model against the new snapshot and full gradient); 0 (default)
+                                  cuts a delay to the rounds the epoch has had.  Such a context launches its rounds kernel by
+                                  kernel (no captured graph) */
 } dq_config;
 
 /* Optimiser state, all [d] fp32 device vectors owned by the caller.  y and x_sum are used by Algorithm 3
@@ -207,7 +211,8 @@ int dq_round(dq_ctx* ctx, dq_state* st, uint32_t round, float eta, float theta,
 /* Delays (Algorithm 1 step 11 evaluates the gradient at x_{D(t)}; Assumption 3: t - D(t) <= tau).  delays (HOST,
  * [M], each in 0..max_delay; NULL: all zero) says for every worker how many rounds before the current one the model
  * it works on was broadcast; it holds for the following dq_round calls until set again.  A delay is cut to the
- * number of rounds the epoch has had (the first round's workers all see the current model).  Needs
+ * number of rounds the epoch has had (the first round's workers all see the current model), or, with
+ * cfg.delay_across_epochs, to the rounds the context has had since its first epoch began.  Needs
  * cfg.max_delay > 0; both models take delays (for the network the kept broadcasts are the low-precision parameters
  * themselves).  Such a context replays its rounds as a captured graph like any other (the kernels pick the
  * broadcast of a lagging worker from a round counter kept on the device), but not in the one-cluster kernel.

@@ -35,7 +35,7 @@ class dq_config(C.Structure):
                 ("sparsify", C.c_int32), ("phi", C.c_float), ("msg_format", C.c_int32), ("accelerated", C.c_int32),
                 ("snapshot_flag", C.c_int32), ("no_graph", C.c_int32), ("seed", C.c_uint64), ("sparse_cap", C.c_int64), ("mu", C.c_float), ("sequential", C.c_int32),
                 ("model", C.c_int32), ("hidden", C.c_int32), ("classes", C.c_int32), ("no_fused", C.c_int32), ("max_delay", C.c_int32),
-                ("tensor_cores", C.c_int32)]
+                ("tensor_cores", C.c_int32), ("delay_across_epochs", C.c_int32)]
 
 
 class dq_state(C.Structure):
@@ -165,9 +165,9 @@ class Msgs:
 
 
 def make_config(d, M, B=1, bx=8, b=8, lambda1=0.0, lambda2=0.0, box_lo=float("-inf"), box_hi=float("inf"), sparsify=0,
-                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0, sequential=0, model=0, hidden=0, classes=0, no_fused=0, max_delay=0, tensor_cores=0) -> dq_config:
+                phi=0.0, msg_format=DQ_MSG_DENSE, accelerated=0, snapshot_flag=1, seed=0, sparse_cap=0, no_graph=0, mu=0.0, sequential=0, model=0, hidden=0, classes=0, no_fused=0, max_delay=0, tensor_cores=0, delay_across_epochs=0) -> dq_config:
     return dq_config(d, M, B, bx, b, lambda1, lambda2, box_lo, box_hi, int(sparsify), phi, msg_format, int(accelerated),
-                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, int(sequential), int(model), int(hidden), int(classes), int(no_fused), int(max_delay), int(tensor_cores))
+                     int(snapshot_flag), int(no_graph), seed, sparse_cap, mu, int(sequential), int(model), int(hidden), int(classes), int(no_fused), int(max_delay), int(tensor_cores), int(delay_across_epochs))
 
 
 # ---- entry points (same names and order of arguments as include/dq.h) ---------------------------------------------

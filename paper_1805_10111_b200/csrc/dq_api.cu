@@ -87,6 +87,7 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
     if (cfg->sparse_cap < 0 || cfg->sparse_cap > cfg->d) return DQ_ERR_ARG;
     if (!(cfg->mu >= 0.0f)) return DQ_ERR_ARG;
     if (cfg->max_delay < 0 || cfg->max_delay > 64 || (cfg->max_delay > 0 && !data)) return DQ_ERR_ARG;
+    if (cfg->delay_across_epochs && (cfg->max_delay <= 0 || cfg->mu > 0.0f)) return DQ_ERR_ARG;   // needs a ring, and a fixed model width to re-read it
     if (data) {
         if (data->n < 1 || !data->values || !data->labels) return DQ_ERR_SHAPE;
         if (cfg->model == DQ_MODEL_MLP) {
@@ -151,6 +152,10 @@ int dq_create(dq_ctx** out, const dq_config* cfg, const dq_data* data)
         rc |= dev_alloc(&c->alpha, (size_t)M * d);
         rc |= dev_alloc(&c->rows, (size_t)M * cfg->B);
         rc |= dev_alloc(&c->xhat_diff, (size_t)d * (cfg->max_delay + 1));     // a ring of broadcasts when workers may lag
+        if (cfg->max_delay > 0 && cfg->delay_across_epochs && cfg->model == DQ_MODEL_LOGISTIC) {
+            rc |= dev_alloc(&c->xhat_ring, (size_t)d * (cfg->max_delay + 1));
+            if (rc == DQ_OK && cudaMemset(c->xhat_ring, 0, sizeof(float) * (size_t)d * (cfg->max_delay + 1)) != cudaSuccess) rc = DQ_ERR_CUDA;
+        }
         rc |= dev_alloc(&c->delays_dev, M);
         rc |= dev_alloc(&c->slots_dev, M);
         if (rc == DQ_OK && cudaMemset(c->delays_dev, 0, sizeof(int32_t) * M) != cudaSuccess) rc = DQ_ERR_CUDA;
@@ -210,7 +215,7 @@ int dq_destroy(dq_ctx* c)
     if (!c) return DQ_ERR_ARG;
     void* ptrs[] = {c->norm_bits, c->norm_block, c->chunk_off, c->tile_ptr, c->stage_idx, c->stage_val, c->stage_ctrl, c->delays_dev, c->slots_dev, c->xnorm_bits, c->status, c->bits,
                     c->msgs.codes, c->msgs.scale, c->msgs.idx, c->msgs.nnz, c->codes_x, c->delta_x, c->alpha,
-                    c->rows, c->xhat_diff, c->g64, c->acc64, c->rbuf, c->fused_part, c->fused_cnt, c->ptouched, c->gtmp, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
+                    c->rows, c->xhat_diff, c->g64, c->acc64, c->rbuf, c->fused_part, c->fused_cnt, c->ptouched, c->gtmp, c->xhat_ring, c->rp_dev, c->touched, c->glist, c->gcount, c->seg_count, c->bx_dev, c->prec_stats, c->mlp_rows, c->mlp_act[0], c->mlp_act[1], c->mlp_dz[0], c->mlp_dz[1], c->mlp_dh[0], c->mlp_dh[1], c->hx, c->hg, c->hv, c->hnorm};
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (void* p : ptrs) if (p) cudaFree(p);
@@ -325,6 +330,10 @@ int dq_epoch_begin(dq_ctx* ctx, dq_state* s, float theta, void* stream)
     if (rc != DQ_OK) return rc;
     if (!s->x_snap || !s->z_snap || !aligned(s->x_snap, 16)) return DQ_ERR_ARG;
     launch_epoch_begin(ctx, s, theta, as_stream(stream));
+    const bool across = ctx->cfg.max_delay > 0 && ctx->cfg.delay_across_epochs;
+    if (across && ctx->xhat_ring && ctx->ring_rounds > 0)    // the kept broadcasts against the new snapshot
+        launch_rediff_ring(ctx, s->x_snap, as_stream(stream));
+    if (!across) ctx->ring_rounds = 0;
     ctx->rounds_in_epoch = 0;
     ctx->ticks_in_epoch = 0;
     ctx->epoch += 1;
@@ -360,13 +369,15 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     const int tau = ctx->cfg.max_delay;
     float* const ring = ctx->xhat_diff;
     if (tau > 0) {
-        const int t = (int)ctx->rounds_in_epoch;
+        const int t = (int)ctx->ring_rounds;
         // while a round is captured for replay the kernels take the epoch's round counter from the device instead
         if (ctx->rp_active) ctx->diff_ring = tau + 1;
         else ctx->xhat_diff = ring + (int64_t)(t % (tau + 1)) * ctx->cfg.d;
         if (flag) {                                          // xhat = xsnap: a zero difference; the network's ring holds xhat itself
             if (ctx->cfg.model == DQ_MODEL_MLP) cudaMemcpyAsync(ctx->xhat_diff, s->x_snap, sizeof(float) * ctx->cfg.d, cudaMemcpyDeviceToDevice, as_stream(st));
             else cudaMemsetAsync(ctx->xhat_diff, 0, sizeof(float) * ctx->cfg.d, as_stream(st));
+            if (ctx->xhat_ring)
+                cudaMemcpyAsync(ctx->xhat_ring + (int64_t)(t % (tau + 1)) * ctx->cfg.d, s->x_snap, sizeof(float) * ctx->cfg.d, cudaMemcpyDeviceToDevice, as_stream(st));
         }
         launch_set_slots(ctx, t, as_stream(st));
     }
@@ -388,6 +399,8 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
         }
         ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = ctx->normx_zeroed = true;
         ctx->sp_norms_zeroed = ctx->cfg.sparsify != 0;          // the same kernel cleared ||beta||_inf and ||alpha||_1
+        if (ctx->xhat_ring)                                  // delays across epochs: keep the broadcast itself as well
+            launch_dequant_xhat(ctx, ctx->codes_x, ctx->delta_x, ctx->xhat_ring + (int64_t)((int)ctx->ring_rounds % (tau + 1)) * ctx->cfg.d, as_stream(st));
     } else if (adaptive) {
         cudaMemsetAsync(ctx->bx_dev, 0, sizeof(int32_t), as_stream(st));
     }
@@ -397,7 +410,10 @@ static int enqueue_round(dq_ctx* ctx, dq_state* s, uint32_t round, int flag, flo
     // sparse gradients into sparse messages: one cluster kernel takes over from the worker kernel's accumulator
     const bool msg_kernel = !flag && sparse_message_applies(ctx);
     ctx->defer_list = msg_kernel;
-    rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, flag, s, round, nullptr, ctx->alpha, ctx->ninf, st);
+    // a snapshot round's gradient differences are zero, unless a worker still works on a model of the previous epoch
+    const bool across = tau > 0 && ctx->cfg.delay_across_epochs;
+    if (flag && across) ctx->diff_ready = true;              // (this round's slot of the ring holds the zero difference)
+    rc = dq_worker_grad(ctx, ctx->codes_x, ctx->delta_x, (flag && !across) ? 1 : 0, s, round, nullptr, ctx->alpha, ctx->ninf, st);
     ctx->defer_list = false;
     ctx->use_slots = false;
     ctx->diff_ready = ctx->alpha_zeroed = ctx->ninf_zeroed = false;
@@ -466,12 +482,12 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
     const int flag = c.snapshot_flag && ctx->rounds_in_epoch == 0 && (!c.accelerated || ctx->epoch == 0);
     if (!flag && ctx->cluster_blocks > 0) {                  // small problem: the whole round in one cluster kernel
         launch_round_cluster(ctx, s, round, 1, eta, theta, bits_down, bits_up, as_stream(stream));
-        ctx->rounds_in_epoch += 1;
+        ctx->rounds_in_epoch += 1; ctx->ring_rounds += 1;
         ctx->ticks_in_epoch += 1;
         return last_error();
     }
     bool replayed = false;
-    if (!flag && !ctx->graph_off && !c.no_graph) {
+    if (!flag && !ctx->graph_off && !c.no_graph && !(c.max_delay > 0 && c.delay_across_epochs)) {
         const dq_state& g = ctx->graph_state;
         const bool same = ctx->graph_exec && g.x == s->x && g.x_snap == s->x_snap && g.g_full == s->g_full && g.y == s->y &&
                           g.x_sum == s->x_sum && g.norm_x == s->norm_x && g.z_snap == s->z_snap &&
@@ -481,7 +497,7 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
             cudaStream_t st = as_stream(stream);
             // the round's last kernel advances the round number on the device: only a jump in the numbering or new
             // step sizes need the launch that sets them (scalars travel as kernel arguments: no host buffer to keep alive)
-            const uint32_t t_epoch = (uint32_t)ctx->rounds_in_epoch;
+            const uint32_t t_epoch = (uint32_t)ctx->ring_rounds;
             if (!(ctx->rp_host_valid && ctx->rp_host.round == round && ctx->rp_host.eta == eta && ctx->rp_host.theta == theta &&
                   ctx->rp_host.t_epoch == t_epoch))
                 launch_set_round_params(ctx, round, eta, theta, t_epoch, st);
@@ -495,7 +511,7 @@ int dq_round(dq_ctx* ctx, dq_state* s, uint32_t round, float eta, float theta, u
         rc = enqueue_round(ctx, s, round, flag, eta, theta, bits_down, bits_up, stream);
         if (rc != DQ_OK) return rc;
     }
-    ctx->rounds_in_epoch += 1;
+    ctx->rounds_in_epoch += 1; ctx->ring_rounds += 1;
     ctx->ticks_in_epoch += ctx->cfg.sequential ? ctx->cfg.M : 1;
     return last_error();
 }
@@ -527,7 +543,7 @@ int dq_rounds(dq_ctx* ctx, dq_state* s, uint32_t round0, int32_t nrounds, float 
         if (rc != DQ_OK) return rc;
         if (!ctx->has_data || !s->x_snap || !s->z_snap || !(eta > 0.0f) || !isfinite(eta) || ctx->epoch < 0) return DQ_ERR_ARG;
         launch_round_cluster(ctx, s, round0 + (uint32_t)i, nrounds - i, eta, theta, bits_down, bits_up, as_stream(stream));
-        ctx->rounds_in_epoch += nrounds - i;
+        ctx->rounds_in_epoch += nrounds - i; ctx->ring_rounds += nrounds - i;
         ctx->ticks_in_epoch += nrounds - i;
         i = nrounds;
     }

@@ -316,6 +316,9 @@ struct dq_ctx {
     int32_t* delays_dev;        // [M] rounds each worker lags behind
     int32_t* slots_dev;         // [M] ring slot each worker reads this round
     bool use_slots;             // set while dq_round enqueues a round of a context with max_delay > 0
+    float* xhat_ring;           // delays across epochs (logistic model): the broadcasts themselves, [max_delay + 1][d], from which the ring of
+                                // differences is formed again when the snapshot changes
+    int64_t ring_rounds;        // rounds the ring has seen (since the epoch began, or since the first epoch with delays across epochs)
     int diff_ring;              // set while such a round is captured: slots of the ring, the kernels pick this round's from the device's round counter
     int cluster_blocks;         // blocks of the one-cluster round kernel for small problems; 0: rounds run as separate kernels
     bool list_mode;             // dq_round keeps alpha zero outside the listed groups and works on the list only

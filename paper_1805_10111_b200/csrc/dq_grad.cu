@@ -2307,6 +2307,33 @@ void launch_set_slots(dq_ctx* ctx, int t, cudaStream_t st)
     ctx->launches += 1;
 }
 
+// Delays across epochs: the ring of xhat - xsnap formed again from the kept broadcasts when the snapshot has changed
+// (the same single subtraction as in the model quantiser, so a slot equals what that round would have written against
+// the new snapshot).
+__global__ void __launch_bounds__(kThreads)
+rediff_ring_kernel(const float* __restrict__ xhat_ring, const float* __restrict__ xsnap, int64_t d, int nslots, float* __restrict__ diff_ring)
+{
+    pdl_prologue();
+    const int64_t n = d * nslots, nth = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nth) diff_ring[i] = __fsub_rn(xhat_ring[i], xsnap[i % d]);
+}
+
+void launch_rediff_ring(dq_ctx* ctx, const float* x_snap, cudaStream_t st)
+{
+    const int nslots = ctx->cfg.max_delay + 1;
+    launch_k(rediff_ring_kernel, blocks_for(ctx->cfg.d * nslots, ctx->sm_count), kThreads, 0, st, (const float*)ctx->xhat_ring, x_snap, ctx->cfg.d, nslots, ctx->xhat_diff);
+    ctx->launches += 1;
+}
+
+// xhat = codes * delta_x of the packed model (no reference subtracted).
+void launch_dequant_xhat(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, float* xhat, cudaStream_t st)
+{
+    const dq_config& c = ctx->cfg;
+    if (c.bx != 2 && c.bx != 4 && c.bx != 8) { launch_dequant_diff_any(ctx, codes_x, delta_x, nullptr, xhat, c.bx, st); return; }
+    DQ_DISPATCH_BITS(c.bx, (launch_k(dequant_diff_kernel<BITS_>, blocks_for(c.d, ctx->sm_count), kThreads, 0, st, codes_x, delta_x, (const float*)nullptr, c.d, xhat)));
+    ctx->launches += 1;
+}
+
 __global__ void set_round_params_kernel(RoundParams* rp, uint32_t round, float eta, float theta, uint32_t t_epoch)
 {
     pdl_prologue();

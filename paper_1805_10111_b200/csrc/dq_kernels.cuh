@@ -39,6 +39,8 @@ bool fused_round_applies(const dq_ctx* ctx);
 void launch_fused_round(dq_ctx* ctx, dq_state* s, uint32_t round, cudaStream_t st);
 void small_round_setup(dq_ctx* ctx);
 void launch_set_slots(dq_ctx* ctx, int round_in_epoch, cudaStream_t st);
+void launch_rediff_ring(dq_ctx* ctx, const float* x_snap, cudaStream_t st);
+void launch_dequant_xhat(dq_ctx* ctx, const uint8_t* codes_x, const float* delta_x, float* xhat, cudaStream_t st);
 void launch_round_cluster(dq_ctx* ctx, dq_state* s, uint32_t round0, int nrounds, float eta, float theta, uint64_t* bits_down,
                           uint64_t* bits_up, cudaStream_t st);
 void launch_objective(dq_ctx* ctx, const float* x, double* P, cudaStream_t st);

@@ -97,6 +97,25 @@ def test_network_lockstep_delayed_workers(dq, extra):
     ls.close()
 
 
+def test_network_delays_across_epochs(dq):
+    """The same for the network: the ring keeps the low-precision parameters themselves, so a worker that lags over
+    the epoch boundary evaluates last epoch's parameters against the new snapshot."""
+    h, x = _net(400, 48, 12, 5, 6)
+    kw = dict(M=4, B=20, bx=8, b=4, lambda2=1e-4, seed=47, model=1, hidden=12, classes=5, max_delay=2, delay_across_epochs=1)
+    ls = Lockstep(dq, h, x, **kw)
+    g = np.random.default_rng(47)
+    rnd = 0
+    for s_ in range(3):
+        ls.epoch(F32(0.0))
+        for t in range(5):
+            delays = [2] * 4 if t == 0 else [int(v) for v in g.integers(0, 3, 4)]
+            tr = ls.round(rnd, 0.2, F32(0.0), delays=delays)
+            assert tr["delays_used"] == [min(D, rnd) for D in delays]
+            rnd += 1
+    assert ls.far_flips == 0
+    ls.close()
+
+
 def test_network_full_size_rounds(dq):
     """784-100-10 on 2,000 image-shaped rows, M = 8 workers, B = 20, b_x = 8, b = 4 (the paper's setting for this model)."""
     h, x = _net(2000, 784, 100, 10, 3)

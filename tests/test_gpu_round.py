@@ -347,7 +347,7 @@ class Lockstep:
                    msg_format=kw.get("msg_format", 0), accelerated=kw.get("accelerated", 0), seed=kw["seed"],
                    mu=kw.get("mu", 0.0), sequential=kw.get("sequential", 0), model=kw.get("model", 0),
                    hidden=kw.get("hidden", 0), classes=kw.get("classes", 0))
-        assert not (set(kw) - {"M", "B", "bx", "b", "lambda1", "lambda2", "box_lo", "box_hi", "no_fused", "no_graph", "max_delay", "tensor_cores"} - set(okw)), kw
+        assert not (set(kw) - {"M", "B", "bx", "b", "lambda1", "lambda2", "box_lo", "box_hi", "no_fused", "no_graph", "max_delay", "tensor_cores", "delay_across_epochs"} - set(okw)), kw
         d = x0.size                                        # parameters (equals the feature count for logistic regression)
         self.cfg = dq.make_config(d, kw["M"], **{k: v for k, v in kw.items() if k != "M"})
         self.ocfg = oracle.make_config(d, kw["M"], kw["B"], kw["bx"], kw["b"], **okw)
@@ -389,7 +389,7 @@ class Lockstep:
         if delays is not None:
             assert dq.dq_set_delays(self.ctx, delays) == 0
         assert dq.dq_round(self.ctx, st, rnd, eta, theta, self.bits[0:1], self.bits[1:2]) == 0
-        tr = run.round(rnd, eta, theta, trace=True, delays=delays)
+        tr = run.round(rnd, eta, theta, trace=True, delays=delays, across_epochs=bool(cfg.delay_across_epochs))
         assert tr["status"] == 0 and dq.dq_poll_status(self.ctx) == (0, 0)
         _, buf = dq.dq_round_buffers(self.ctx)
         m = buf["msgs"]
@@ -409,12 +409,13 @@ class Lockstep:
         round_flips = 0; same_survivors = True
         for w in range(M):
             S_w = tr["S"][w]; slack_w = np.zeros(d)
-            if cfg.model != dq.DQ_MODEL_MLP and not tr["flag_round"]:
+            stale = delays is not None and tr["delays_used"][w] > 0      # (in a snapshot round only a lagging worker has a gradient)
+            if cfg.model != dq.DQ_MODEL_MLP and (not tr["flag_round"] or stale):
                 used = tr["delays_used"][w] if delays is not None else 0
                 xhat_w = tr["xhat"] if used == 0 else run.broadcasts[len(run.broadcasts) - 1 - used]
                 slack_w = _margin_slack(self.h, tr["rows"][w], xhat_w, run.xsnap)
                 S_w = S_w + slack_w
-            elif cfg.model == dq.DQ_MODEL_MLP and not tr["flag_round"]:
+            elif cfg.model == dq.DQ_MODEL_MLP and (not tr["flag_round"] or stale):
                 slack_w = (_softmax_rounding_floor(self.h, tr["rows"][w], tr["xhat"], cfg.hidden, cfg.classes)
                            + _softmax_rounding_floor(self.h, tr["rows"][w], run.xsnap, cfg.hidden, cfg.classes))
                 S_w = S_w + slack_w
@@ -683,6 +684,36 @@ def test_lockstep_delayed_workers(dq, name, kw, eta):
             rnd += 1
     assert ls.far_flips == 0
     assert dq.dq_set_delays(ls.ctx, [tau + 1] * M) == dq.DQ_ERR_ARG
+    ls.close()
+
+
+@pytest.mark.parametrize("name,kw,eta", [
+    ("dense", dict(M=3, B=8, bx=8, b=8, lambda1=1e-4, seed=81, max_delay=2, delay_across_epochs=1), 0.5),
+    ("csr", dict(M=5, B=16, bx=5, b=4, lambda2=1e-5, seed=82, max_delay=3, delay_across_epochs=1), 0.5),
+    ("csr", dict(M=4, B=16, bx=8, b=4, lambda1=1e-6, sparsify=1, phi=0.0, msg_format=1, seed=83, max_delay=2, delay_across_epochs=1), 0.5),
+    ("bf16", dict(M=3, B=70, bx=8, b=8, box_lo=-1.0, box_hi=1.0, seed=84, max_delay=2, delay_across_epochs=1), 0.01),
+    ("dense8", dict(M=4, B=16, bx=8, b=4, lambda2=1e-4, accelerated=1, seed=85, max_delay=2, delay_across_epochs=1), 0.05),
+])
+def test_lockstep_delays_across_epochs(dq, name, kw, eta):
+    """Delays that reach back over the epoch boundary: in the first rounds of an epoch a lagging worker's gradient
+    difference is taken at the previous epoch's low-precision model against the new snapshot (the library forms its
+    ring of differences again from the kept broadcasts when the snapshot changes); a snapshot round still sends
+    exact zeros for the workers that do not lag."""
+    h = _problem(name)
+    ls = Lockstep(dq, h, synth.normal_vector(h.d, 87, 0.05), **kw)
+    g = np.random.default_rng(kw["seed"])
+    M, tau, acc = kw["M"], kw["max_delay"], bool(kw.get("accelerated", 0))
+    rnd = 0; crossed = 0
+    for epoch in range(3):
+        theta = F32(2.0 / (epoch + 3)) if acc else F32(0.0)
+        ls.epoch(theta)
+        for t in range(tau + 3):
+            delays = [tau] * M if t == 0 else [int(v) for v in g.integers(0, tau + 1, M)]
+            tr = ls.round(rnd, eta, theta, delays=delays)
+            assert tr["delays_used"] == [min(D, rnd) for D in delays]
+            crossed += sum(1 for D in tr["delays_used"] if D > t)
+            rnd += 1
+    assert crossed >= 2 * M and ls.far_flips == 0
     ls.close()
 
 
