@@ -798,8 +798,10 @@ __device__ __forceinline__ void accumulate_word(uint32_t word, float dl, float (
 }
 
 // Dense messages.  Each thread owns the 32/BITS coordinates of one 32-bit code word per worker.
-template <int BITS, bool ACC>
-__global__ void __launch_bounds__(kThreads, 4)
+// BATCH: code words (workers) in flight per thread.  8 keeps four blocks per SM for models that stream from HBM; 32 is
+// for models of a few thousand coordinates, where the kernel's time is the number of dependent batches of loads.
+template <int BITS, bool ACC, int BATCH = 8>
+__global__ void __launch_bounds__(kThreads, BATCH == 8 ? 4 : 2)
 master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const float* __restrict__ scale, int M, int64_t d,
                     const float* __restrict__ g_full, float* __restrict__ x, float* __restrict__ y,
                     const float* __restrict__ xsnap, float* __restrict__ xsum, float eta, float theta, ProxParams pp,
@@ -836,7 +838,7 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
                 load8_rw((ACC ? y : x) + i0 + q * 8, *reinterpret_cast<float(*)[8]>(curp + q * 8));
             }
         }
-        if (BITS == 4) {      // the two loop shapes compute the same thing; each bit width uses the one that the
+        if (BITS == 4 && BATCH == 8) {      // the two loop shapes compute the same thing; each bit width uses the one that the
                               // compiler schedules better (measured: registers and load placement differ)
             const uint32_t* wp = words + t * W;
             int w0 = 0;
@@ -863,16 +865,16 @@ master_dense_kernel(const uint8_t* __restrict__ codes, int64_t stride, const flo
                 for (int q = 0; q < W; ++q) accumulate_word<BITS>(wd[q], s_scale[w0], acc[q]);
             }
         } else {
-            for (int w0 = 0; w0 < M; w0 += 8) {             // batches of eight code words in flight; rows clamped, tail predicated
-                uint32_t wd[8][W];
+            for (int w0 = 0; w0 < M; w0 += BATCH) {         // batches of BATCH code words in flight; rows clamped, tail predicated
+                uint32_t wd[BATCH][W];
     #pragma unroll
-                for (int k = 0; k < 8; ++k) {
+                for (int k = 0; k < BATCH; ++k) {
                     const uint32_t* wq = words + (int64_t)min(w0 + k, M - 1) * wstride;
                     if (W == 2) { const uint2 u = __ldg(reinterpret_cast<const uint2*>(wq) + t); wd[k][0] = u.x; wd[k][W - 1] = u.y; }
                     else wd[k][0] = __ldg(wq + t);
                 }
     #pragma unroll
-                for (int k = 0; k < 8; ++k) {
+                for (int k = 0; k < BATCH; ++k) {
                     if (w0 + k < M) {
     #pragma unroll
                         for (int q = 0; q < W; ++q) accumulate_word<BITS>(wd[k][q], s_scale[w0 + k], acc[q]);
@@ -2031,7 +2033,12 @@ void launch_master(dq_ctx* ctx, const dq_msgs* msgs, bool sparse_msgs, dq_state*
         const size_t smem = sizeof(float) * c.M;
         auto al32 = [](const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 31) == 0; };
         const int vec8_ok = al32(s->x) && al32(s->g_full) && al32(s->y) && al32(s->x_snap) && al32(s->x_sum);
-        if (c.accelerated) {
+        const bool small = nwords <= (int64_t)ctx->sm_count * kThreads && c.M > 8;     // less than a block per SM: latency, not bandwidth
+        if (small && c.accelerated) {
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_kernel<BITS_, true, 32>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
+        } else if (small) {
+            DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_kernel<BITS_, false, 32>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
+        } else if (c.accelerated) {
             DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_kernel<BITS_, true>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
         } else {
             DQ_DISPATCH_BITS(c.b, (launch_k(master_dense_kernel<BITS_, false>, grid, kThreads, smem, st, msgs->codes, msgs->stride, msgs->scale, c.M, d, s->g_full, s->x, s->y, s->x_snap, s->x_sum, eta, theta, pp, vec8_ok, nx, ctx->rp_active, ba)));
